@@ -1,0 +1,331 @@
+"""TEST INFRASTRUCTURE: CPU plan builder (integer only) - the oracle for ``sched_build``.
+
+The paper gives the scheduler as principles, not as a listing (Section 7.1.2 and the
+lessons of Section 7.4.1):
+
+  * one persistent thread block pinned to each SM, processing tasks in a loop;
+  * the fixed block-to-SM mapping lets the schedule be planned in advance;
+  * each block gets the tasks whose data lives in its SM's local partition (die);
+  * data and work are split between the partitions in proportion to their SM counts;
+  * the assignment is static;
+  * what matters is *which* physical SMs are used, not only how many (Section 1).
+
+Everything more concrete below is this build's reading of those principles, taken
+step by step in a fixed order so that the CUDA builder can be compared bytewise.
+
+Work units.  tiles_m = ceil(M / tile_m), tiles_n = ceil(N / tile_n); the K range is cut
+into ``k_splits`` runs of whole k-slabs (``k_unit`` elements each).  Unit id
+u = (tm * tiles_n + tn) * k_splits + ks.
+
+Steps.
+  1. raster order R: tile rows in groups of ``raster_group`` g; inside a group tn is the
+     outer loop, tm the middle one, ks the innermost.  g = 1 is the plain row-major raster.
+  2. SM set S (ascending), drawn from the SMs not in ``avoid``:
+       oblivious, seed 0   the b lowest ids;
+       oblivious, seed !=0 Fisher-Yates over the ascending candidate list
+                           (i from last down to 1, j = mix64(mix64(seed)+i) mod (i+1)),
+                           first b entries, sorted;
+       die_compact/affinity  primary die first (preferred_die, else the die with more
+                           candidates, tie -> lower id), then the other; inside a die whole
+                           TPCs dealt round-robin over that die's GPCs (ascending GPC id,
+                           unplaced SMs with gpc < 0 form a last pseudo-GPC), ascending SM id
+                           inside a GPC, until b SMs are taken.
+  3. per-die SM counts n_d and rank of each chosen SM inside its die (ascending id).
+  4. quotas q_d = floor(n_u * n_d / b); leftover units go one each to the dies in
+     descending order of (n_u * n_d mod b), tie -> lower die id.
+  5. unit -> die:
+       oblivious    R[i] goes to S[i mod b]; the unit's die is that SM's die;
+       die_compact  die 0 takes R[0..q_0), die 1 takes the rest (contiguous bands);
+       affinity     margin m(u) = local_0(u) - local_1(u) where local_d counts the bytes of
+                    the unit's A panel, B panel and C tile that sit in chunks of die d
+                    (negated when invert_affinity); preferred die = 0 if m > 0, 1 if m < 0,
+                    the die_compact band's die if m == 0; units sorted by (|m| descending,
+                    raster index ascending) are given to their preferred die while its
+                    quota lasts, else to the other die; each die's queue is then put back
+                    in raster order.
+  6. static lists: entry i of die d's queue goes to the SM of rank (i mod n_d) in d.
+  7. export: flat int32 words (see ``export``).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+OBLIVIOUS, DIE_COMPACT, AFFINITY = 0, 1, 2
+LAYOUT_ROWMAJOR, LAYOUT_PAGED = 0, 1
+PLAN_MAGIC = 0x41475031      # "AGP1"
+_MASK = (1 << 64) - 1
+
+
+def mix64(x: int) -> int:
+    """The repo's 64-bit mixer, restated here independently of the CUDA side."""
+    x = (x + 0x9E3779B97F4A7C15) & _MASK
+    x ^= x >> 30
+    x = (x * 0xBF58476D1CE4E5B9) & _MASK
+    x ^= x >> 27
+    x = (x * 0x94D049BB133111EB) & _MASK
+    x ^= x >> 31
+    return x
+
+
+def default_policy(**kw) -> dict:
+    p = dict(kind=OBLIVIOUS, seed=0, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1,
+             k_unit=64, raster_group=1, preferred_die=-1, invert_affinity=0,
+             static_assign=1, avoid=(), a=None, b=None, c=None)
+    p.update(kw)
+    return p
+
+
+def operand(offset: int, row_stride: int, elem_bytes: int, layout: int = LAYOUT_ROWMAJOR,
+            page_table=None) -> dict:
+    return dict(offset=int(offset), row_stride=int(row_stride), elem_bytes=int(elem_bytes),
+                layout=layout, page_table=page_table)
+
+
+# ----------------------------------------------------------------------------- step 1
+def raster_order(tiles_m: int, tiles_n: int, k_splits: int, g: int) -> list[int]:
+    g = max(1, g)
+    R = []
+    for tm0 in range(0, tiles_m, g):
+        for tn in range(tiles_n):
+            for tm in range(tm0, min(tiles_m, tm0 + g)):
+                for ks in range(k_splits):
+                    R.append((tm * tiles_n + tn) * k_splits + ks)
+    return R
+
+
+# ----------------------------------------------------------------------------- step 2
+def select_sms(topo: dict, b: int, pol: dict) -> list[int]:
+    n_sm = topo["n_sm"]
+    avoid = set(int(s) for s in pol["avoid"])
+    cand = [s for s in range(n_sm) if s not in avoid]
+    if b < 1 or b > len(cand):
+        raise ValueError("sm_budget out of range")
+    if pol["kind"] == OBLIVIOUS:
+        if pol["seed"] == 0:
+            return cand[:b]
+        arr = list(cand)
+        base = mix64(int(pol["seed"]))
+        for i in range(len(arr) - 1, 0, -1):
+            j = mix64((base + i) & _MASK) % (i + 1)
+            arr[i], arr[j] = arr[j], arr[i]
+        return sorted(arr[:b])
+    die, gpc, tpc = topo["die"], topo["gpc"], topo["tpc"]
+    n_gpc = topo["n_gpc"]
+    cnt = [sum(1 for s in cand if die[s] == d) for d in (0, 1)]
+    if pol["preferred_die"] in (0, 1):
+        primary = pol["preferred_die"]
+    else:
+        primary = 0 if cnt[0] >= cnt[1] else 1
+    S = []
+    for d in (primary, 1 - primary):
+        # candidate TPCs of this die, grouped by GPC key (gpc < 0 -> pseudo-GPC n_gpc)
+        groups: dict[int, dict[int, list[int]]] = {}
+        for s in cand:
+            if die[s] != d:
+                continue
+            key = int(gpc[s]) if gpc[s] >= 0 else n_gpc
+            groups.setdefault(key, {}).setdefault(int(tpc[s]), []).append(s)
+        keys = sorted(groups)
+        lists = {k: [groups[k][t] for t in sorted(groups[k])] for k in keys}
+        p = 0
+        while len(S) < b and any(p < len(lists[k]) for k in keys):
+            for k in keys:
+                if p < len(lists[k]):
+                    for s in lists[k][p]:
+                        if len(S) < b:
+                            S.append(s)
+            p += 1
+        if len(S) >= b:
+            break
+    return sorted(S)
+
+
+# ----------------------------------------------------------------------------- step 4
+def quotas(n_u: int, n_d: list[int], b: int) -> list[int]:
+    q = [n_u * n // b for n in n_d]
+    rem = [n_u * n % b for n in n_d]
+    left = n_u - sum(q)
+    order = sorted(range(len(n_d)), key=lambda d: (-rem[d], d))
+    for d in order:
+        if left == 0:
+            break
+        if n_d[d] > 0:
+            q[d] += 1
+            left -= 1
+    assert left == 0
+    return q
+
+
+# ----------------------------------------------------------------------------- step 5 helpers
+def k_range(pol: dict, ks: int) -> tuple[int, int]:
+    """Element range [k0, k1) of split ks: whole k-slabs, the first splits take the longer runs."""
+    K, ku = pol["K"], pol["k_unit"]
+    n_slab = -(-K // ku)
+    per = -(-n_slab // pol["k_splits"])
+    s0 = min(n_slab, ks * per)
+    s1 = min(n_slab, (ks + 1) * per)
+    return min(K, s0 * ku), min(K, s1 * ku)
+
+
+def _bytes_per_die_interval(amap: dict, start: int, end: int) -> list[int]:
+    """Bytes of [start, end) (offsets from the probed base) that lie in chunks of die 0 / 1."""
+    cb = amap["chunk_bytes"]
+    doc = amap["die_of_chunk"]
+    out = [0, 0]
+    pos = start
+    while pos < end:
+        c = pos // cb
+        nxt = min(end, (c + 1) * cb)
+        out[int(doc[c])] += nxt - pos
+        pos = nxt
+    return out
+
+
+def unit_local_bytes(pol: dict, amap: dict, u: int) -> list[int]:
+    """local_d(u): bytes of unit u's A panel, B panel and C tile in chunks of die d."""
+    tiles_n = -(-pol["N"] // pol["tile_n"])
+    ks = u % pol["k_splits"]
+    t = u // pol["k_splits"]
+    tm, tn = t // tiles_n, t % tiles_n
+    r0, r1 = tm * pol["tile_m"], min(pol["M"], (tm + 1) * pol["tile_m"])
+    c0, c1 = tn * pol["tile_n"], min(pol["N"], (tn + 1) * pol["tile_n"])
+    k0, k1 = k_range(pol, ks)
+    tot = [0, 0]
+
+    def add(op, row_lo, row_hi, col_lo, col_hi):
+        if op is None:
+            return
+        eb = op["elem_bytes"]
+        for r in range(row_lo, row_hi):
+            s = op["offset"] + r * op["row_stride"] + col_lo * eb
+            e = op["offset"] + r * op["row_stride"] + col_hi * eb
+            v = _bytes_per_die_interval(amap, s, e)
+            tot[0] += v[0]
+            tot[1] += v[1]
+
+    add(pol["a"], r0, r1, k0, k1)                      # A panel: rows of the tile, k-range columns
+    bop = pol["b"]
+    if bop is not None and bop["layout"] == LAYOUT_PAGED:
+        # weights stored as pages of [16 k x tile_n] elements; logical page of (tn, k16)
+        ppt = -(-pol["K"] // 16)
+        cb = amap["chunk_bytes"]
+        for k16 in range(k0 // 16, -(-k1 // 16)):
+            phys = int(bop["page_table"][tn * ppt + k16])
+            tot[int(amap["die_of_chunk"][phys])] += cb
+    else:
+        add(bop, k0, k1, c0, c1)                       # B panel: k-range rows, tile columns
+    add(pol["c"], r0, r1, c0, c1)                      # C tile
+    return tot
+
+
+# ----------------------------------------------------------------------------- whole plan
+def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
+    M, N, K = pol["M"], pol["N"], pol["K"]
+    tiles_m = -(-M // pol["tile_m"])
+    tiles_n = -(-N // pol["tile_n"])
+    ksp = pol["k_splits"]
+    n_u = tiles_m * tiles_n * ksp
+    R = raster_order(tiles_m, tiles_n, ksp, pol["raster_group"])
+    S = select_sms(topo, b, pol)
+    die = topo["die"]
+    sm_die = [int(die[s]) for s in S]
+    n_d = [sm_die.count(0), sm_die.count(1)]
+    rank = []
+    seen = [0, 0]
+    for d in sm_die:
+        rank.append(seen[d])
+        seen[d] += 1
+    slots_of_die = [[i for i, d in enumerate(sm_die) if d == dd] for dd in (0, 1)]
+    q = quotas(n_u, n_d, b)
+
+    sm_q = [[] for _ in S]
+    if pol["kind"] == OBLIVIOUS:
+        die_q = [[], []]
+        for i, u in enumerate(R):
+            slot = i % b
+            sm_q[slot].append(u)
+            die_q[sm_die[slot]].append(u)
+    else:
+        if pol["kind"] == DIE_COMPACT:
+            die_q = [R[:q[0]], R[q[0]:]]
+        else:
+            if amap is None:
+                raise ValueError("affinity policy needs an affinity map")
+            items = []
+            for i, u in enumerate(R):
+                l0, l1 = unit_local_bytes(pol, amap, u)
+                m = l0 - l1
+                if pol["invert_affinity"]:
+                    m = -m
+                if m > 0:
+                    pref = 0
+                elif m < 0:
+                    pref = 1
+                else:
+                    pref = 0 if i < q[0] else 1
+                items.append((-abs(m), i, u, pref))
+            items.sort()
+            got = [[], []]
+            for _, i, u, pref in items:
+                d = pref if len(got[pref]) < q[pref] else 1 - pref
+                got[d].append((i, u))
+            die_q = [[u for _, u in sorted(g)] for g in got]
+        for d in (0, 1):
+            for i, u in enumerate(die_q[d]):
+                sm_q[slots_of_die[d][i % n_d[d]]].append(u)
+
+    smid_to_slot = [-1] * topo["n_sm"]
+    for i, s in enumerate(S):
+        smid_to_slot[s] = i
+    return dict(kind=pol["kind"], n_sm=topo["n_sm"], b=b, n_units=n_u, tiles_m=tiles_m,
+                tiles_n=tiles_n, k_splits=ksp, tile_m=pol["tile_m"], tile_n=pol["tile_n"],
+                M=M, N=N, K=K, static_assign=pol["static_assign"],
+                sm_list=S, sm_die=sm_die, rank_in_die=rank, die_sm_count=n_d,
+                die_q=die_q, sm_q=sm_q, smid_to_slot=smid_to_slot, quotas=q)
+
+
+def export(plan: dict) -> np.ndarray:
+    """Flat int32 image compared bytewise with the library's ``ag_plan_export``:
+
+    header[16] = magic, kind, n_sm, b, n_die(2), n_units, tiles_m, tiles_n, k_splits,
+                 tile_m, tile_n, M, N, K, static_assign, 0
+    then sm_list[b], sm_die[b], rank_in_die[b], die_sm_count[2], die_q_off[3],
+    die_q[n_units], sm_q_off[b+1], sm_q[n_units], smid_to_slot[n_sm].
+    """
+    p = plan
+    w = [PLAN_MAGIC, p["kind"], p["n_sm"], p["b"], 2, p["n_units"], p["tiles_m"], p["tiles_n"],
+         p["k_splits"], p["tile_m"], p["tile_n"], p["M"], p["N"], p["K"], p["static_assign"], 0]
+    w += p["sm_list"] + p["sm_die"] + p["rank_in_die"] + p["die_sm_count"]
+    w += [0, len(p["die_q"][0]), len(p["die_q"][0]) + len(p["die_q"][1])]
+    w += p["die_q"][0] + p["die_q"][1]
+    off = [0]
+    for lst in p["sm_q"]:
+        off.append(off[-1] + len(lst))
+    w += off
+    for lst in p["sm_q"]:
+        w += lst
+    w += p["smid_to_slot"]
+    return np.array(w, dtype=np.int32)
+
+
+# ----------------------------------------------------------------------------- die-view packing
+def build_page_table(unit_die: list[int], pages_per_unit: int, amap: dict) -> list[int]:
+    """Indirect allocation by remapping (Section 7.1.1, Eq. 1): logical page j of the
+    packed operand lives in one of the two physical chunks (2j, 2j+1); the one whose
+    measured die equals the die that owns the page's unit is taken.  The measured
+    chunk->die bit replaces the parity-of-masked-physical-address selector of Eq. 1,
+    which needs a physical base address that an unmodified driver does not expose.
+    If both chunks of a pair sit on the same die (the pair rule fails), chunk 2j is used.
+    """
+    doc = amap["die_of_chunk"]
+    table = []
+    for u, d in enumerate(unit_die):
+        for p in range(pages_per_unit):
+            j = u * pages_per_unit + p
+            if int(doc[2 * j]) == d:
+                table.append(2 * j)
+            elif int(doc[2 * j + 1]) == d:
+                table.append(2 * j + 1)
+            else:
+                table.append(2 * j)
+    return table

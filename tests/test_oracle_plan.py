@@ -1,0 +1,252 @@
+"""Pins for the CPU plan builder: hand-derived tiny plans, invariants the paper's scheduling
+principles imply, the printed remap formula, and published mixer vectors."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import plan as op
+from paper_2609_24270_b200 import inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+TOY = dict(n_sm=4, n_tpc=2, n_gpc=2, n_die=2, tpc=[0, 0, 1, 1], gpc=[0, 0, 1, 1],
+           die=[0, 0, 1, 1], is_random=[0, 0, 0, 0], gpc_die=[0, 1])
+
+
+def golden():
+    out = {}
+    for line in open(os.path.join(GOLD, "plan_tiny.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, q0, q1, smq = [f.strip() for f in line.split("|")]
+        out[name] = ([int(x) for x in q0.split()], [int(x) for x in q1.split()],
+                     [[int(x) for x in s.split()] for s in smq.split(";")])
+    return out
+
+
+def toy_amap_case_d():
+    doc = np.zeros(512, dtype=np.uint8)
+    for r in range(256):
+        tm = r // 128
+        for tn in (0, 1):
+            u = tm * 2 + tn
+            if u == 0:
+                d = 1
+            elif u == 1:
+                d = 0 if (r % 128) < 96 else 1
+            elif u == 2:
+                d = 0
+            else:
+                d = 0 if (r % 128) < 64 else 1
+            doc[2 * r + tn] = d
+    return dict(chunk_bytes=1024, die_of_chunk=doc)
+
+
+def test_hand_derived_tiny_plans():
+    g = golden()
+    base = dict(M=256, N=512, K=64)
+    cases = {
+        "obl_b3": (op.default_policy(kind=op.OBLIVIOUS, **base), None, 3),
+        "dc_b3": (op.default_policy(kind=op.DIE_COMPACT, **base), None, 3),
+        "dc_g2_k2_b4": (op.default_policy(kind=op.DIE_COMPACT, M=256, N=512, K=128, k_splits=2,
+                                          raster_group=2), None, 4),
+        "aff_b4": (op.default_policy(kind=op.AFFINITY, c=op.operand(0, 2048, 4), **base),
+                   toy_amap_case_d(), 4),
+        "aff_inv_b4": (op.default_policy(kind=op.AFFINITY, invert_affinity=1,
+                                         c=op.operand(0, 2048, 4), **base), toy_amap_case_d(), 4),
+    }
+    for name, (pol, amap, b) in cases.items():
+        p = op.build_plan(TOY, amap, b, pol)
+        assert (p["die_q"][0], p["die_q"][1], p["sm_q"]) == g[name], name
+
+
+def test_case_d_margins_by_brute_force_byte_count():
+    """local_d(u) against a per-byte count over the whole C tile."""
+    amap = toy_amap_case_d()
+    pol = op.default_policy(kind=op.AFFINITY, M=256, N=512, K=64, c=op.operand(0, 2048, 4))
+    want_margin = {0: -131072, 1: 65536, 2: 131072, 3: 0}
+    for u in range(4):
+        tm, tn = u // 2, u % 2
+        cnt = [0, 0]
+        for r in range(tm * 128, tm * 128 + 128):
+            for byte in range(r * 2048 + tn * 1024, r * 2048 + tn * 1024 + 1024):
+                cnt[int(amap["die_of_chunk"][byte // 1024])] += 1
+        assert op.unit_local_bytes(pol, amap, u) == cnt
+        assert cnt[0] - cnt[1] == want_margin[u]
+
+
+def test_interval_counting_unaligned():
+    doc = np.array([0, 1, 1, 0, 1], dtype=np.uint8)
+    amap = dict(chunk_bytes=100, die_of_chunk=doc)
+    # [50, 430): 50 of chunk0(d0), 100 c1(d1), 100 c2(d1), 100 c3(d0), 30 c4(d1)
+    assert op._bytes_per_die_interval(amap, 50, 430) == [150, 230]
+    assert op._bytes_per_die_interval(amap, 120, 120) == [0, 0]
+
+
+def test_raster_orders():
+    assert op.raster_order(2, 3, 1, 1) == [0, 1, 2, 3, 4, 5]
+    assert op.raster_order(3, 2, 1, 2) == [0, 2, 1, 3, 4, 5]
+    assert sorted(op.raster_order(5, 7, 3, 4)) == list(range(105))
+
+
+def test_quota_proportional_to_die_sm_count():
+    # the 70/78 split the paper reports for some B200 chips (Section 7.1)
+    assert op.quotas(2048, [70, 78], 148) == [969, 1079]
+    assert op.quotas(2048, [74, 74], 148) == [1024, 1024]
+    assert op.quotas(10, [0, 5], 5) == [0, 10]
+    for n_u in (1, 7, 512, 2047):
+        for n0 in (1, 16, 37, 70):
+            q = op.quotas(n_u, [n0, 148 - n0], 148)
+            assert sum(q) == n_u
+            assert abs(q[0] / n_u - n0 / 148) <= 1.0 / n_u + 1e-12
+
+
+def test_mixer_published_vectors():
+    # splitmix64 seeded with 0: published first three outputs
+    assert op.mix64(0) == 0xE220A8397B1DCDAF
+    assert op.mix64(0x9E3779B97F4A7C15) == 0x6E789E6AA1B965F4
+    assert op.mix64((2 * 0x9E3779B97F4A7C15) & ((1 << 64) - 1)) == 0x06C45D188009454F
+    # the vectorised generator-side copy agrees with the scalar one
+    xs = np.array([0, 1, 12345, 2 ** 63 + 5], dtype=np.uint64)
+    assert [int(v) for v in inputs.mix64_np(xs)] == [op.mix64(int(x)) for x in xs]
+
+
+def check_invariants(topo, plan, pol, b, avoid=()):
+    S = plan["sm_list"]
+    assert len(S) == b and S == sorted(set(S)) and not (set(S) & set(avoid))
+    assert all(0 <= s < topo["n_sm"] for s in S)
+    assert [int(topo["die"][s]) for s in S] == plan["sm_die"]
+    assert sum(plan["die_sm_count"]) == b
+    n_u = plan["n_units"]
+    assert sorted(plan["die_q"][0] + plan["die_q"][1]) == list(range(n_u))
+    assert sorted(u for l in plan["sm_q"] for u in l) == list(range(n_u))
+    for slot, lst in enumerate(plan["sm_q"]):
+        if pol["kind"] != op.OBLIVIOUS:
+            d = plan["sm_die"][slot]
+            assert set(lst) <= set(plan["die_q"][d])
+    if pol["kind"] != op.OBLIVIOUS:
+        assert [len(q) for q in plan["die_q"]] == plan["quotas"]
+    for s, slot in enumerate(plan["smid_to_slot"]):
+        assert (slot >= 0) == (s in S)
+        if slot >= 0:
+            assert S[slot] == s
+    lens = [len(l) for l in plan["sm_q"]]
+    if pol["kind"] == op.OBLIVIOUS:
+        assert max(lens) - min(lens) <= 1
+
+
+@pytest.mark.parametrize("die0", [70, 72, 74])
+@pytest.mark.parametrize("kind", [op.OBLIVIOUS, op.DIE_COMPACT])
+@pytest.mark.parametrize("b", [16, 37, 74, 148])
+def test_invariants_on_synthetic_b200(die0, kind, b):
+    topo = inputs.synthetic_topo(die0_sms=die0, seed=die0)
+    assert int((topo["die"] == 0).sum()) == die0 and topo["n_sm"] == 148
+    pol = op.default_policy(kind=kind, M=4096, N=4096, K=4096, raster_group=4)
+    plan = op.build_plan(topo, None, b, pol)
+    check_invariants(topo, plan, pol, b)
+    exp = op.export(plan)
+    assert exp.dtype == np.int32 and exp[0] == op.PLAN_MAGIC
+    assert len(exp) == 16 + 3 * b + 2 + 3 + plan["n_units"] + b + 1 + plan["n_units"] + 148
+
+
+def test_seeded_subsets_and_avoid_mask():
+    topo = inputs.synthetic_topo()
+    pol1 = op.default_policy(kind=op.OBLIVIOUS, seed=1, M=4096, N=4096, K=4096)
+    pol2 = op.default_policy(kind=op.OBLIVIOUS, seed=2, M=4096, N=4096, K=4096)
+    s1, s1b, s2 = op.select_sms(topo, 32, pol1), op.select_sms(topo, 32, pol1), op.select_sms(topo, 32, pol2)
+    assert s1 == s1b and s1 != s2 and len(set(s1)) == 32
+    # every SM is drawn about equally often over many seeds (Fisher-Yates is unbiased)
+    hits = np.zeros(148)
+    for seed in range(1, 401):
+        for s in op.select_sms(topo, 37, op.default_policy(kind=op.OBLIVIOUS, seed=seed, M=1, N=1, K=1)):
+            hits[s] += 1
+    assert hits.min() > 60 and hits.max() < 140           # mean 100
+    avoid = list(range(0, 148, 2))
+    pol = op.default_policy(kind=op.DIE_COMPACT, M=4096, N=4096, K=4096, avoid=avoid)
+    plan = op.build_plan(topo, None, 40, pol)
+    check_invariants(topo, plan, pol, 40, avoid)
+    with pytest.raises(ValueError):
+        op.select_sms(topo, 75, pol)
+
+
+def test_die_compact_is_compact_and_gpc_balanced():
+    topo = inputs.synthetic_topo(die0_sms=70, seed=3)     # die 1 is the larger (78)
+    pol = op.default_policy(kind=op.DIE_COMPACT, M=4096, N=4096, K=4096)
+    S = op.select_sms(topo, 32, pol)
+    assert all(topo["die"][s] == 1 for s in S)            # fits in the primary (larger) die
+    per_gpc = np.bincount([topo["gpc"][s] for s in S], minlength=8)
+    used = per_gpc[per_gpc > 0]
+    assert len(used) == 4 and used.max() - used.min() <= 2        # whole TPCs dealt round-robin
+    assert all((s ^ 1) in S for s in S)                   # whole TPCs
+    S = op.select_sms(topo, 100, pol)
+    assert sum(1 for s in S if topo["die"][s] == 1) == 78  # primary die exhausted first
+    pol0 = op.default_policy(kind=op.DIE_COMPACT, M=4096, N=4096, K=4096, preferred_die=0)
+    assert all(topo["die"][s] == 0 for s in op.select_sms(topo, 32, pol0))
+
+
+def test_equal_dies_split_c_in_halves():
+    topo = inputs.synthetic_topo(die0_sms=74)
+    pol = op.default_policy(kind=op.DIE_COMPACT, M=8192, N=8192, K=8192)
+    plan = op.build_plan(topo, None, 148, pol)
+    assert plan["die_q"][0] == list(range(1024)) and plan["die_q"][1] == list(range(1024, 2048))
+
+
+def test_all_ties_affinity_equals_die_compact():
+    topo = inputs.synthetic_topo(die0_sms=72)
+    # A rows are 8 KB = one aligned chunk pair (dies 0,1): every margin is exactly 0
+    kw = dict(M=1024, N=1024, K=4096, tile_m=128, tile_n=256)
+    pa = op.default_policy(kind=op.AFFINITY, a=op.operand(0, 8192, 2), **kw)
+    pd = op.default_policy(kind=op.DIE_COMPACT, **kw)
+    amap = dict(chunk_bytes=4096, die_of_chunk=(np.arange(4096) & 1).astype(np.uint8))
+    assert op.unit_local_bytes(pa, amap, 5) == [128 * 4096, 128 * 4096]
+    e_a = op.export(op.build_plan(topo, amap, 148, pa))
+    e_d = op.export(op.build_plan(topo, None, 148, pd))
+    assert e_a[1] == op.AFFINITY and e_d[1] == op.DIE_COMPACT
+    assert np.array_equal(e_a[2:], e_d[2:])               # identical apart from the kind word
+
+
+def test_packing_by_plan_is_recovered_by_affinity():
+    """Pack the weight pages of each unit onto the die a die_compact plan gave the unit;
+    the affinity policy must then rebuild that plan, and invert_affinity its mirror."""
+    topo = inputs.synthetic_topo(die0_sms=70, seed=9)
+    kw = dict(M=16, N=2048, K=1024, tile_m=16, tile_n=128, k_splits=2)
+    pd = op.default_policy(kind=op.DIE_COMPACT, **kw)
+    plan_d = op.build_plan(topo, None, 148, pd)
+    n_tiles = 16
+    ppt = 1024 // 16                                       # pages per n-tile
+    pages_per_unit = ppt // 2
+    unit_die = [0] * plan_d["n_units"]
+    for d in (0, 1):
+        for u in plan_d["die_q"][d]:
+            unit_die[u] = d
+    n_log = n_tiles * ppt
+    amap = dict(chunk_bytes=4096, die_of_chunk=inputs.synthetic_chunk_die(2 * n_log, seed=5))
+    doc = amap["die_of_chunk"]
+    assert all(doc[2 * j] != doc[2 * j + 1] for j in range(n_log))      # pair rule of Section 7.1.1
+    table = op.build_page_table(unit_die, pages_per_unit, amap)
+    assert all(int(doc[table[u * pages_per_unit + p]]) == unit_die[u]
+               for u in range(plan_d["n_units"]) for p in range(pages_per_unit))
+    bop = op.operand(0, 0, 2, layout=op.LAYOUT_PAGED, page_table=table)
+    pa = op.default_policy(kind=op.AFFINITY, b=bop, **kw)
+    plan_a = op.build_plan(topo, amap, 148, pa)
+    assert plan_a["die_q"] == plan_d["die_q"] and plan_a["sm_q"] == plan_d["sm_q"]
+    pi = op.default_policy(kind=op.AFFINITY, invert_affinity=1, b=bop, **kw)
+    plan_i = op.build_plan(topo, amap, 148, pi)
+    # the mirror: as many units as quotas allow sit on the *other* die
+    on_wrong = sum(1 for d in (0, 1) for u in plan_i["die_q"][d] if unit_die[u] != d)
+    assert on_wrong == 2 * min(plan_d["quotas"])
+    check_invariants(topo, plan_i, pi, 148)
+
+
+def test_page_table_matches_printed_remap_formula():
+    """Eq. 1 (appendix on address remapping): page_phys = 2j + [parity((page_start + 2j) & MASK) xor P]
+    when a chunk's die is parity((page_start + chunk) & MASK) and bit 0 is in MASK."""
+    MASK, start = 0b1011_0110_1, 0x5A2C0                   # even start page, bit 0 in the mask
+    par = lambda x: bin(x).count("1") & 1
+    n_log = 4096
+    doc = np.array([par((start + c) & MASK) for c in range(2 * n_log)], dtype=np.uint8)
+    amap = dict(chunk_bytes=4096, die_of_chunk=doc)
+    for P in (0, 1):
+        table = op.build_page_table([P] * n_log, 1, amap)
+        want = [2 * j + (par((start + 2 * j) & MASK) ^ P) for j in range(n_log)]
+        assert table == want
