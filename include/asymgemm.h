@@ -1,0 +1,228 @@
+/*
+ * asymgemm.h - C ABI of the asymmetry-aware persistent BF16 GEMM library for NVIDIA B200
+ * (sm_100a).
+ *
+ * The library follows "Dissecting How Die Scaling Breaks GPU Fine-grained Scheduling":
+ * first discover the chip-specific compute topology (Section 5) and the memory-affinity
+ * layout (Section 6), then let a persistent kernel use both to decide which physical SMs
+ * run and which output tiles each one takes (Section 7.1.2, lessons of Section 7.4.1).
+ *
+ * Conventions
+ *   - Every call returns an ag_status; nothing throws, nothing calls exit().
+ *   - "host" / "device" is stated for every pointer.  Device pointers are plain CUDA
+ *     device addresses on the current device (cudaSetDevice is the caller's business).
+ *   - ag_topo_map and ag_policy are caller-owned plain structs.  ag_affinity_map and
+ *     ag_plan are library-owned opaque handles released by the matching *_destroy.
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x the
+ *     calls that launch kernels return AG_ERR_UNSUPPORTED_ARCH.
+ *   - Every device-side wait is bounded; if one runs out the kernel records
+ *     AG_ERR_TIMEOUT in the plan's status word (see ag_last_status) and returns.
+ */
+#ifndef ASYMGEMM_H_
+#define ASYMGEMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AG_MAX_SM 256
+#define AG_MAX_GPC 32
+#define AG_MAX_DIE 2
+#define AG_CHUNK_BYTES 4096 /* partition interleave granularity reported in Section 6.1.2 */
+
+typedef enum {
+    AG_OK = 0,
+    AG_ERR_ARG = 1,              /* null pointer, bad size, misaligned buffer, plan/shape mismatch */
+    AG_ERR_CUDA = 2,             /* a CUDA runtime/driver call failed (see ag_last_cuda_error) */
+    AG_ERR_UNSUPPORTED_ARCH = 3, /* device is not sm_100 */
+    AG_ERR_TIMEOUT = 4,          /* a bounded device-side wait ran out */
+    AG_ERR_UNMANNED_SM = 5,      /* an SM of the plan never got a thread block */
+    AG_ERR_NOISY_PROBE = 6,      /* latency tiers could not be separated */
+    AG_ERR_STALE_AMAP = 7,       /* affinity map does not belong to this buffer */
+    AG_ERR_NOMEM = 8
+} ag_status;
+
+/* ---- compute topology (Section 5, Section 6.1.1) -------------------------------------- */
+typedef struct {
+    int32_t n_sm, n_tpc, n_gpc, n_die;
+    int32_t tpc[AG_MAX_SM];        /* TPC of SM s: two consecutive SM ids share a TPC (Section 5.1.2) */
+    int32_t gpc[AG_MAX_SM];        /* GPC class of SM s, -1 if it could not be placed */
+    int32_t die[AG_MAX_SM];        /* memory-affinity partition (die) of SM s; die 0 = die of SM 0 */
+    uint8_t is_random[AG_MAX_SM];  /* 1: never seen in a thread-block cluster larger than 2 (Section 5.1.1) */
+    int32_t die_sm_count[AG_MAX_DIE];
+    int32_t gpc_sm_count[AG_MAX_GPC];
+    int32_t gpc_die[AG_MAX_GPC];
+    uint32_t lat_near_cycles, lat_far_cycles, lat_threshold; /* HBM latency tiers seen by the probe */
+    uint32_t l2_near_cycles, l2_far_cycles;                  /* L2-hit latency, same-die / other-die reader */
+    int32_t n_unplaced;            /* SMs left with gpc == -1 */
+    int32_t device;                /* CUDA device ordinal the map was measured on */
+    uint32_t sm_clock_khz;         /* SM clock rate reported by the device at probe time */
+    uint32_t flags;                /* AG_TOPO_* bits of the phases that ran */
+} ag_topo_map;
+
+#define AG_TOPO_CENSUS 1u
+#define AG_TOPO_CLUSTER 2u
+#define AG_TOPO_LATENCY 4u
+#define AG_TOPO_BANDWIDTH 8u
+
+/*
+ * topo_discover - build the SM -> TPC/GPC/die map of the current device.
+ * Section 5.1.1 (cluster probing: SMs that co-occur in a thread-block cluster share a GPC),
+ * Section 5.1.2 (L2-bandwidth probing places the remaining "random" SMs),
+ * Section 6.1.1 (HBM latency seen from every SM splits the SMs into two partitions).
+ *   map  host pointer, caller-owned, fully overwritten.
+ * Allocates and frees its own device scratch; synchronises the device.
+ * Errors: AG_ERR_ARG (null), AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_NOISY_PROBE
+ * (two latency tiers not found), AG_ERR_UNMANNED_SM (census did not see every SM).
+ */
+ag_status topo_discover(ag_topo_map* map);
+
+/* Same with a choice of phases (AG_TOPO_* bits); skipped phases leave gpc = -1 / die = 0. */
+ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases);
+
+/*
+ * ag_topo_from_observations - the host half of topo_discover on recorded observations
+ * (no device needed): union-find over cluster co-occurrence (Section 5.1.1) and two-tier
+ * split of per-SM latency vectors (Section 6.1.1).
+ *   cluster_sm[cluster_off[c] .. cluster_off[c+1])  SM ids seen together in cluster c (host)
+ *   lat[s * n_ref + r]  min latency in cycles from SM s to reference chunk r (host)
+ *   map  host, out.  Errors: AG_ERR_ARG, AG_ERR_NOISY_PROBE.
+ */
+ag_status ag_topo_from_observations(int32_t n_sm, const int32_t* cluster_sm, const int32_t* cluster_off,
+                                    int32_t n_clusters, const uint32_t* lat, int32_t n_ref,
+                                    ag_topo_map* map);
+
+/*
+ * ag_topo_place_by_gain - decision rule of Section 5.1.2 for one unplaced TPC: given the
+ * bandwidth gain (bytes/s) of adding the TPC to the known SMs of each candidate GPC and the
+ * TPC's solo bandwidth, return the index of the GPC it contends with (smallest gain, below
+ * solo_bw * margin while the runner-up is above it), or -1 if the sweep is ambiguous.
+ */
+int32_t ag_topo_place_by_gain(const double* gain, int32_t n_candidates, double solo_bw);
+
+/* ---- memory affinity (Section 6.1) ------------------------------------------------------ */
+typedef struct ag_affinity_map ag_affinity_map;
+
+/*
+ * affinity_probe - chunk -> die map of a device buffer from HBM access latency
+ * (Section 6.1.1 and the HBM-latency kernel of the appendix: invalidate the L2 line, load it
+ * with an L1-bypassing load, time the round trip with the SM cycle counter; the minimum over
+ * several lines of the chunk is kept).  A chunk is AG_CHUNK_BYTES; die 0 is the die of SM 0.
+ *   buf    device pointer, 4096-byte aligned; contents are preserved (each probed 128-byte
+ *          line is saved before the L2 invalidation and written back afterwards).  Nothing
+ *          else may touch the buffer while the probe runs.
+ *   bytes  multiple of 4096.
+ *   amap   host, out: new handle.
+ * Runs topo_discover's census + latency phases internally when no map has been supplied via
+ * ag_affinity_probe_with_map.  Synchronises the device.
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_NOISY_PROBE, AG_ERR_NOMEM.
+ */
+ag_status affinity_probe(void* buf, size_t bytes, ag_affinity_map** amap);
+ag_status ag_affinity_probe_with_map(void* buf, size_t bytes, const ag_topo_map* map,
+                                     ag_affinity_map** amap);
+/* Build a handle from a given chunk->die table (host, one byte per chunk, values 0/1):
+ * lets plans be built for a recorded or synthetic layout. */
+ag_status ag_affinity_from_table(const void* buf, size_t bytes, const uint8_t* die_of_chunk,
+                                 size_t n_chunks, ag_affinity_map** amap);
+/* Copy out the chunk->die table (host, cap bytes) and/or the raw min-latency cycles. */
+ag_status ag_affinity_export(const ag_affinity_map* amap, uint8_t* die_of_chunk, size_t cap,
+                             size_t* n_chunks);
+ag_status ag_affinity_cycles(const ag_affinity_map* amap, uint32_t* cycles, size_t cap);
+/* Probe again from an SM of the other die; returns in *mismatches how many chunks are not
+ * the complement of the stored table (Section 6.1.1: the two groups of SMs see opposite tiers). */
+ag_status ag_affinity_check_complement(const ag_affinity_map* amap, const ag_topo_map* map,
+                                       size_t* mismatches);
+void ag_affinity_destroy(ag_affinity_map* amap);
+
+/* ---- plan (Section 7.1.2) ------------------------------------------------------------ */
+enum { AG_OBLIVIOUS = 0, AG_DIE_COMPACT = 1, AG_AFFINITY = 2 };
+enum { AG_LAYOUT_ROWMAJOR = 0, AG_LAYOUT_PAGED = 1 };
+
+typedef struct {
+    int32_t present;        /* 0: operand not counted by the affinity policy */
+    int32_t layout;         /* AG_LAYOUT_ROWMAJOR: rows of row_stride bytes; AG_LAYOUT_PAGED: B only,
+                               pages of [16 k x tile_n] elements, page of (tn, k16) = tn*ceil(K/16)+k16 */
+    int64_t offset;         /* byte offset of element (0,0) from the probed buffer's base */
+    int64_t row_stride;     /* bytes between rows (row-major) */
+    int32_t elem_bytes;
+    int32_t reserved;
+    const int32_t* page_table; /* host; AG_LAYOUT_PAGED: chunk index (in the probed buffer) of each logical page */
+    int64_t n_pages;
+} ag_operand_desc;
+
+typedef struct {
+    int32_t kind;            /* AG_OBLIVIOUS | AG_DIE_COMPACT | AG_AFFINITY */
+    int32_t M, N, K;
+    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}; skinny kernel: M<=... x 128 */
+    int32_t k_splits;        /* >= 1, runs of whole k-slabs */
+    int32_t k_unit;          /* elements per k-slab (64) */
+    int32_t raster_group;    /* tile rows per raster group (>= 1) */
+    int32_t preferred_die;   /* -1: the die with more usable SMs */
+    int32_t invert_affinity; /* 1: send every unit to the die that holds fewer of its bytes */
+    int32_t static_assign;   /* 1: static per-SM lists (the paper's mode); 0: CTAs pull from per-die queues */
+    uint64_t seed;           /* oblivious only: 0 = lowest SM ids, else seeded random subset */
+    uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
+    ag_operand_desc a, b, c;
+} ag_policy;
+
+typedef struct ag_plan ag_plan;
+
+/*
+ * sched_build - choose sm_budget physical SMs and give every work unit (output tile x
+ * k-split) to exactly one of them.  Section 7.1.2: persistent block per SM, schedule planned
+ * in advance, each block takes the tasks whose data lives in its SM's partition, work split
+ * between partitions in proportion to their SM counts; static assignment (Section 7.4.1).
+ * The plan is computed by CUDA kernels and stays on the device for gemm_persistent.
+ *   map     host, from topo_discover (or any consistent map with n_sm = device SM count)
+ *   amap    handle or NULL; required for AG_AFFINITY
+ *   policy  host
+ *   plan    host, out: new handle
+ * Errors: AG_ERR_ARG (budget out of range, bad tile shape, empty k-split, operand outside the
+ * probed buffer, AG_AFFINITY without amap), AG_ERR_CUDA, AG_ERR_NOMEM.
+ */
+ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* amap, int sm_budget,
+                      const ag_policy* policy, ag_plan** plan);
+/* Flat int32 image of the plan (host, cap words): header[16] = magic 0x41475031, kind, n_sm,
+ * b, n_die, n_units, tiles_m, tiles_n, k_splits, tile_m, tile_n, M, N, K, static_assign, 0;
+ * then sm_list[b], sm_die[b], rank_in_die[b], die_sm_count[2], die_q_off[3], die_q[n_units],
+ * sm_q_off[b+1], sm_q[n_units], smid_to_slot[n_sm]. */
+ag_status ag_plan_export(const ag_plan* plan, int32_t* out, size_t cap, size_t* n_words);
+/* Affinity margins local_0 - local_1 per raster index (host, cap entries), for spot checks. */
+ag_status ag_plan_margins(const ag_plan* plan, int64_t* out, size_t cap);
+/* Executed-by record of the last launches: SM id that ran unit u and how often it ran
+ * (host arrays of n_units entries, either may be NULL); ag_plan_reset_record zeroes the counts. */
+ag_status ag_plan_tile_record(const ag_plan* plan, int32_t* owner_sm, int32_t* run_count, size_t cap);
+ag_status ag_plan_reset_record(ag_plan* plan);
+/* Device status word of the most recent launch (call after synchronising its stream). */
+ag_status ag_last_status(const ag_plan* plan);
+void ag_plan_destroy(ag_plan* plan);
+
+/*
+ * gemm_persistent - C = A * B on the SMs of the plan.  One persistent thread block per
+ * planned SM reads %smid, takes its slot of the plan and loops over its work units
+ * (Section 7.1.2); TMA feeds shared memory, tcgen05 MMAs accumulate in tensor memory in fp32.
+ *   A  device, M x K bf16 row-major, 16-byte aligned, K % 8 == 0
+ *   B  device, K x N bf16 row-major, 16-byte aligned, N % 8 == 0
+ *   C  device, M x N fp32 row-major, 16-byte aligned; overwritten (zeroed first when the plan
+ *      has k_splits > 1, partial sums are then added with reductions in memory)
+ *   plan  built for the same M, N, K, else AG_ERR_ARG
+ *   cuda_stream  a cudaStream_t (NULL = default stream).  Asynchronous.
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA.  Device-side trouble
+ * (AG_ERR_TIMEOUT, AG_ERR_UNMANNED_SM) is reported by ag_last_status.
+ */
+ag_status gemm_persistent(const void* A, const void* B, void* C, int M, int N, int K,
+                          const ag_plan* plan, void* cuda_stream);
+
+const char* ag_strerror(ag_status s);
+/* Last CUDA error code seen by the calling thread inside the library (0 = none). */
+int ag_last_cuda_error(void);
+/* Number of kernels this library has launched in this process (for launch accounting). */
+uint64_t ag_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASYMGEMM_H_ */

@@ -1,0 +1,318 @@
+"""ctypes binding over the C ABI declared in include/asymgemm.h (argument marshalling only).
+
+Every step of the path runs inside libasymgemm.so; this module never computes anything
+itself and has no fallback: if the library is missing, importing it raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libasymgemm.so")
+
+AG_MAX_SM, AG_MAX_GPC, AG_MAX_DIE, AG_CHUNK_BYTES = 256, 32, 2, 4096
+AG_OBLIVIOUS, AG_DIE_COMPACT, AG_AFFINITY = 0, 1, 2
+AG_LAYOUT_ROWMAJOR, AG_LAYOUT_PAGED = 0, 1
+AG_TOPO_CENSUS, AG_TOPO_CLUSTER, AG_TOPO_LATENCY, AG_TOPO_BANDWIDTH = 1, 2, 4, 8
+(AG_OK, AG_ERR_ARG, AG_ERR_CUDA, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_TIMEOUT, AG_ERR_UNMANNED_SM,
+ AG_ERR_NOISY_PROBE, AG_ERR_STALE_AMAP, AG_ERR_NOMEM) = range(9)
+
+EXPORTED = [
+    "topo_discover", "ag_topo_discover_phases", "ag_topo_from_observations", "ag_topo_place_by_gain",
+    "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
+    "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_destroy",
+    "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
+    "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_strerror", "ag_last_cuda_error",
+    "ag_kernel_launch_count",
+]
+
+
+class TopoMap(C.Structure):
+    _fields_ = [
+        ("n_sm", C.c_int32), ("n_tpc", C.c_int32), ("n_gpc", C.c_int32), ("n_die", C.c_int32),
+        ("tpc", C.c_int32 * AG_MAX_SM), ("gpc", C.c_int32 * AG_MAX_SM), ("die", C.c_int32 * AG_MAX_SM),
+        ("is_random", C.c_uint8 * AG_MAX_SM),
+        ("die_sm_count", C.c_int32 * AG_MAX_DIE), ("gpc_sm_count", C.c_int32 * AG_MAX_GPC),
+        ("gpc_die", C.c_int32 * AG_MAX_GPC),
+        ("lat_near_cycles", C.c_uint32), ("lat_far_cycles", C.c_uint32), ("lat_threshold", C.c_uint32),
+        ("l2_near_cycles", C.c_uint32), ("l2_far_cycles", C.c_uint32),
+        ("n_unplaced", C.c_int32), ("device", C.c_int32), ("sm_clock_khz", C.c_uint32), ("flags", C.c_uint32),
+    ]
+
+    def as_dict(self) -> dict:
+        n = self.n_sm
+        return dict(n_sm=n, n_tpc=self.n_tpc, n_gpc=self.n_gpc, n_die=self.n_die,
+                    tpc=list(self.tpc[:n]), gpc=list(self.gpc[:n]), die=list(self.die[:n]),
+                    is_random=list(self.is_random[:n]), die_sm_count=list(self.die_sm_count),
+                    gpc_sm_count=list(self.gpc_sm_count[:max(self.n_gpc, 0)]),
+                    gpc_die=list(self.gpc_die[:max(self.n_gpc, 0)]),
+                    lat_near_cycles=self.lat_near_cycles, lat_far_cycles=self.lat_far_cycles,
+                    lat_threshold=self.lat_threshold, l2_near_cycles=self.l2_near_cycles,
+                    l2_far_cycles=self.l2_far_cycles, n_unplaced=self.n_unplaced, device=self.device,
+                    sm_clock_khz=self.sm_clock_khz, flags=self.flags)
+
+    @classmethod
+    def from_dict(cls, d: dict) -> "TopoMap":
+        m = cls()
+        m.n_sm, m.n_tpc, m.n_gpc, m.n_die = d["n_sm"], d["n_tpc"], d["n_gpc"], d.get("n_die", 2)
+        for s in range(d["n_sm"]):
+            m.tpc[s], m.gpc[s], m.die[s] = int(d["tpc"][s]), int(d["gpc"][s]), int(d["die"][s])
+            m.is_random[s] = int(d["is_random"][s])
+        for g in range(d["n_gpc"]):
+            m.gpc_die[g] = int(d["gpc_die"][g])
+        m.die_sm_count[0] = sum(1 for s in range(d["n_sm"]) if d["die"][s] == 0)
+        m.die_sm_count[1] = d["n_sm"] - m.die_sm_count[0]
+        m.flags = AG_TOPO_CENSUS | AG_TOPO_CLUSTER | AG_TOPO_LATENCY
+        return m
+
+
+class OperandDesc(C.Structure):
+    _fields_ = [("present", C.c_int32), ("layout", C.c_int32), ("offset", C.c_int64),
+                ("row_stride", C.c_int64), ("elem_bytes", C.c_int32), ("reserved", C.c_int32),
+                ("page_table", C.POINTER(C.c_int32)), ("n_pages", C.c_int64)]
+
+
+class Policy(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32),
+                ("tile_m", C.c_int32), ("tile_n", C.c_int32), ("k_splits", C.c_int32), ("k_unit", C.c_int32),
+                ("raster_group", C.c_int32), ("preferred_die", C.c_int32), ("invert_affinity", C.c_int32),
+                ("static_assign", C.c_int32), ("seed", C.c_uint64), ("avoid_sm_mask", C.c_uint64 * 4),
+                ("a", OperandDesc), ("b", OperandDesc), ("c", OperandDesc)]
+
+
+class AgError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {strerror(status)} (status {status}, cuda error {lib().ag_last_cuda_error()})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_24270_b200.build` "
+                          "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, sz, i32 = C.c_void_p, C.c_size_t, C.c_int32
+    L.topo_discover.argtypes = [C.POINTER(TopoMap)]
+    L.ag_topo_discover_phases.argtypes = [C.POINTER(TopoMap), C.c_uint32]
+    L.ag_topo_from_observations.argtypes = [i32, vp, vp, i32, vp, i32, C.POINTER(TopoMap)]
+    L.ag_topo_place_by_gain.argtypes = [C.POINTER(C.c_double), i32, C.c_double]
+    L.ag_topo_place_by_gain.restype = i32
+    L.affinity_probe.argtypes = [vp, sz, C.POINTER(vp)]
+    L.ag_affinity_probe_with_map.argtypes = [vp, sz, C.POINTER(TopoMap), C.POINTER(vp)]
+    L.ag_affinity_from_table.argtypes = [vp, sz, vp, sz, C.POINTER(vp)]
+    L.ag_affinity_export.argtypes = [vp, vp, sz, C.POINTER(sz)]
+    L.ag_affinity_cycles.argtypes = [vp, vp, sz]
+    L.ag_affinity_check_complement.argtypes = [vp, C.POINTER(TopoMap), C.POINTER(sz)]
+    L.ag_affinity_destroy.argtypes = [vp]
+    L.ag_affinity_destroy.restype = None
+    L.sched_build.argtypes = [C.POINTER(TopoMap), vp, C.c_int, C.POINTER(Policy), C.POINTER(vp)]
+    L.ag_plan_export.argtypes = [vp, vp, sz, C.POINTER(sz)]
+    L.ag_plan_margins.argtypes = [vp, vp, sz]
+    L.ag_plan_tile_record.argtypes = [vp, vp, vp, sz]
+    L.ag_plan_reset_record.argtypes = [vp]
+    L.ag_last_status.argtypes = [vp]
+    L.ag_plan_destroy.argtypes = [vp]
+    L.ag_plan_destroy.restype = None
+    L.gemm_persistent.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.ag_strerror.argtypes = [C.c_int]
+    L.ag_strerror.restype = C.c_char_p
+    L.ag_last_cuda_error.restype = C.c_int
+    L.ag_kernel_launch_count.restype = C.c_uint64
+    _lib = L
+    return L
+
+
+def strerror(status: int) -> str:
+    return lib().ag_strerror(status).decode()
+
+
+def _check(status: int, what: str):
+    if status != AG_OK:
+        raise AgError(status, what)
+
+
+def kernel_launch_count() -> int:
+    return int(lib().ag_kernel_launch_count())
+
+
+# ---- topology -----------------------------------------------------------------------------
+def topo_discover(phases: int | None = None) -> TopoMap:
+    m = TopoMap()
+    if phases is None:
+        _check(lib().topo_discover(C.byref(m)), "topo_discover")
+    else:
+        _check(lib().ag_topo_discover_phases(C.byref(m), phases), "ag_topo_discover_phases")
+    return m
+
+
+def topo_from_observations(n_sm: int, clusters: list[list[int]], lat: np.ndarray | None) -> TopoMap:
+    flat = np.array([s for c in clusters for s in c], dtype=np.int32)
+    off = np.zeros(len(clusters) + 1, dtype=np.int32)
+    off[1:] = np.cumsum([len(c) for c in clusters])
+    m = TopoMap()
+    if lat is not None:
+        lat = np.ascontiguousarray(lat, dtype=np.uint32)
+        n_ref, lp = lat.shape[1], lat.ctypes.data
+    else:
+        n_ref, lp = 0, None
+    _check(lib().ag_topo_from_observations(n_sm, flat.ctypes.data if len(flat) else None, off.ctypes.data,
+                                           len(clusters), lp, n_ref, C.byref(m)), "ag_topo_from_observations")
+    return m
+
+
+def topo_place_by_gain(gains, solo_bw: float) -> int:
+    arr = (C.c_double * len(gains))(*gains)
+    return int(lib().ag_topo_place_by_gain(arr, len(gains), solo_bw))
+
+
+# ---- affinity ---------------------------------------------------------------------------------
+class AffinityMap:
+    def __init__(self, handle):
+        self.handle = handle
+
+    def export(self) -> np.ndarray:
+        n = C.c_size_t()
+        _check(lib().ag_affinity_export(self.handle, None, 0, C.byref(n)), "ag_affinity_export")
+        out = np.empty(n.value, dtype=np.uint8)
+        _check(lib().ag_affinity_export(self.handle, out.ctypes.data, out.size, C.byref(n)), "ag_affinity_export")
+        return out
+
+    def cycles(self) -> np.ndarray:
+        out = np.empty(len(self.export()), dtype=np.uint32)
+        _check(lib().ag_affinity_cycles(self.handle, out.ctypes.data, out.size), "ag_affinity_cycles")
+        return out
+
+    def check_complement(self, topo: TopoMap) -> int:
+        n = C.c_size_t()
+        _check(lib().ag_affinity_check_complement(self.handle, C.byref(topo), C.byref(n)), "ag_affinity_check_complement")
+        return int(n.value)
+
+    def destroy(self):
+        if self.handle:
+            lib().ag_affinity_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def affinity_probe(dev_ptr: int, nbytes: int, topo: TopoMap | None = None) -> AffinityMap:
+    h = C.c_void_p()
+    if topo is None:
+        _check(lib().affinity_probe(dev_ptr, nbytes, C.byref(h)), "affinity_probe")
+    else:
+        _check(lib().ag_affinity_probe_with_map(dev_ptr, nbytes, C.byref(topo), C.byref(h)), "ag_affinity_probe_with_map")
+    return AffinityMap(h)
+
+
+def affinity_from_table(dev_ptr: int, die_of_chunk: np.ndarray) -> AffinityMap:
+    t = np.ascontiguousarray(die_of_chunk, dtype=np.uint8)
+    h = C.c_void_p()
+    _check(lib().ag_affinity_from_table(dev_ptr, t.size * AG_CHUNK_BYTES, t.ctypes.data, t.size, C.byref(h)),
+           "ag_affinity_from_table")
+    return AffinityMap(h)
+
+
+# ---- plan -------------------------------------------------------------------------------------
+def make_policy(kind=AG_OBLIVIOUS, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1, k_unit=64, raster_group=1,
+                preferred_die=-1, invert_affinity=0, static_assign=1, seed=0, avoid=(), a=None, b=None, c=None):
+    """a/b/c: None or dict(offset, row_stride, elem_bytes[, layout, page_table])."""
+    p = Policy()
+    p.kind, p.M, p.N, p.K, p.tile_m, p.tile_n = kind, M, N, K, tile_m, tile_n
+    p.k_splits, p.k_unit, p.raster_group = k_splits, k_unit, raster_group
+    p.preferred_die, p.invert_affinity, p.static_assign, p.seed = preferred_die, invert_affinity, static_assign, seed
+    for s in avoid:
+        p.avoid_sm_mask[s >> 6] |= 1 << (s & 63)
+    keep = []
+    for name, op in (("a", a), ("b", b), ("c", c)):
+        d = getattr(p, name)
+        if op is None:
+            d.present = 0
+            continue
+        d.present = 1
+        d.layout = op.get("layout", AG_LAYOUT_ROWMAJOR)
+        d.offset, d.row_stride, d.elem_bytes = op["offset"], op["row_stride"], op["elem_bytes"]
+        if op.get("page_table") is not None:
+            t = np.ascontiguousarray(op["page_table"], dtype=np.int32)
+            keep.append(t)
+            d.page_table = t.ctypes.data_as(C.POINTER(C.c_int32))
+            d.n_pages = t.size
+    p._keepalive = keep
+    return p
+
+
+class Plan:
+    def __init__(self, handle):
+        self.handle = handle
+
+    def export(self) -> np.ndarray:
+        n = C.c_size_t()
+        _check(lib().ag_plan_export(self.handle, None, 0, C.byref(n)), "ag_plan_export")
+        out = np.empty(n.value, dtype=np.int32)
+        _check(lib().ag_plan_export(self.handle, out.ctypes.data, out.size, C.byref(n)), "ag_plan_export")
+        return out
+
+    def parsed(self) -> dict:
+        w = self.export()
+        b, n_u, n_sm = int(w[3]), int(w[5]), int(w[2])
+        o = 16
+        d = dict(kind=int(w[1]), n_sm=n_sm, b=b, n_units=n_u, tiles_m=int(w[6]), tiles_n=int(w[7]))
+        for name, ln in (("sm_list", b), ("sm_die", b), ("rank_in_die", b), ("die_sm_count", 2), ("die_q_off", 3),
+                         ("die_q", n_u), ("sm_q_off", b + 1), ("sm_q", n_u), ("smid_to_slot", n_sm)):
+            d[name] = w[o:o + ln].copy()
+            o += ln
+        return d
+
+    def margins(self) -> np.ndarray:
+        n_u = int(self.export()[5])
+        out = np.empty(n_u, dtype=np.int64)
+        _check(lib().ag_plan_margins(self.handle, out.ctypes.data, out.size), "ag_plan_margins")
+        return out
+
+    def tile_record(self):
+        n_u = int(self.export()[5])
+        owner = np.empty(n_u, dtype=np.int32)
+        count = np.empty(n_u, dtype=np.int32)
+        _check(lib().ag_plan_tile_record(self.handle, owner.ctypes.data, count.ctypes.data, n_u), "ag_plan_tile_record")
+        return owner, count
+
+    def reset_record(self):
+        _check(lib().ag_plan_reset_record(self.handle), "ag_plan_reset_record")
+
+    def last_status(self) -> int:
+        return int(lib().ag_last_status(self.handle))
+
+    def destroy(self):
+        if self.handle:
+            lib().ag_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def sched_build(topo: TopoMap, amap: AffinityMap | None, sm_budget: int, policy: Policy) -> Plan:
+    h = C.c_void_p()
+    _check(lib().sched_build(C.byref(topo), amap.handle if amap is not None else None, sm_budget,
+                             C.byref(policy), C.byref(h)), "sched_build")
+    return Plan(h)
+
+
+def gemm_persistent(a_ptr: int, b_ptr: int, c_ptr: int, M: int, N: int, K: int, plan: Plan, stream: int = 0):
+    """Raw device pointers in, asynchronous on `stream` (a cudaStream_t value, 0 = default)."""
+    _check(lib().gemm_persistent(a_ptr, b_ptr, c_ptr, M, N, K, plan.handle, stream), "gemm_persistent")

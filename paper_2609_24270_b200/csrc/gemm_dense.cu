@@ -1,0 +1,459 @@
+// gemm_persistent: persistent, warp-specialised BF16 GEMM for sm_100a whose thread blocks are
+// pinned to the physical SMs of a plan (Section 7.1.2 of the paper: one persistent block per
+// SM, each block reads which SM it runs on and processes the task list planned for that SM).
+//
+// One block per SM (the shared-memory footprint forbids a second one).  A block that lands
+// on an SM outside the plan leaves; a member takes its slot and loops over its work units:
+//   warp 0  (one lane)  scheduler + TMA producer: next unit -> ring, A/B k-slabs -> smem ring
+//   warp 1  (one lane)  tcgen05.mma issuer, accumulators in tensor memory (two buffers)
+//   warps 2-5           epilogue: tcgen05.ld -> registers -> swizzled smem -> TMA store
+// Operands: A row-major (K-major) and B row-major (N-major) are both consumed in place; the
+// MMA descriptors describe B as an MN-major operand, so no transpose pass exists.
+#include <string.h>
+
+#include <mutex>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace ag {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kThreads = 192;
+constexpr int kRing = 8;            // depth of the unit-id ring between the scheduler and its consumers
+constexpr int kEpiWarps = 4;
+constexpr int kEpiBufBytes = 32 * 32 * 4;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s
+
+template <int BN>
+struct Cfg {
+    static constexpr int a_bytes = BM * BK * 2;
+    static constexpr int b_bytes = BK * BN * 2;
+    static constexpr int stage_bytes = a_bytes + b_bytes;
+    static constexpr int epi_bytes = kEpiWarps * 2 * kEpiBufBytes;
+    static constexpr int bar_bytes = 1024;
+    static constexpr int budget = 227 * 1024 - 1024 /*alignment slack*/ - epi_bytes - bar_bytes;
+    static constexpr int stages = budget / stage_bytes > 8 ? 8 : budget / stage_bytes;
+    static constexpr int smem_bytes = stages * stage_bytes + epi_bytes + bar_bytes + 1024;
+    static constexpr int tmem_cols = 2 * BN < 32 ? 32 : 2 * BN;  // power of two for BN in {64,128,256}
+};
+
+struct GemmParams {
+    const int32_t* image;   // plan image (device)
+    PlanCtrl* ctrl;
+    int32_t* tile_owner;
+    int32_t* tile_count;
+    int M, N, K;
+    int b, n_units, n_sm;
+    int tiles_n, k_splits, kslabs_total, kslabs_per_split;
+    int static_assign;
+    unsigned int epoch;
+    unsigned long long wait_limit_ns;
+};
+
+struct SharedCtl {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t sched_full[kRing];
+    uint64_t sched_empty[kRing];
+    uint64_t mma_drain;
+    int ring[kRing];
+    uint32_t tmem_base;
+    int abort_flag;
+    int member;
+};
+
+__device__ __forceinline__ void report_timeout(const GemmParams& p, int role) {
+    if (atomicCAS(&p.ctrl->status, 0, (int)AG_ERR_TIMEOUT) == 0) p.ctrl->status_info = (role << 16) | (int)smid();
+}
+
+// Dynamic mode: take the next index of die d's queue; the 64-bit head carries the epoch of the
+// launch that last touched it, so it resets itself.  Returns -1 when the queue is drained.
+__device__ inline int pop_queue(unsigned long long* head, unsigned int epoch, int len) {
+    for (int tries = 0; tries < 100000; ++tries) {
+        unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(head);
+        if ((unsigned int)(cur >> 32) != epoch) {
+            if (len <= 0) return -1;
+            const unsigned long long nv = ((unsigned long long)epoch << 32) | 1ull;
+            if (atomicCAS(head, cur, nv) == cur) return 0;
+            continue;
+        }
+        const int idx = (int)(cur & 0xffffffffull);
+        if (idx >= len) return -1;
+        if (atomicCAS(head, cur, cur + 1) == cur) return idx;
+    }
+    return -1;
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                  const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t s_stage = base;
+    const uint32_t s_epi = base + C::stages * C::stage_bytes;
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + C::stages * C::stage_bytes + C::epi_bytes);
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const PlanLayout lay{p.b, p.n_units, p.n_sm};
+    const int my_sm = (int)smid();
+    const int slot = p.image[lay.smid_to_slot() + my_sm];
+
+    if (slot < 0) {
+        // Not in the plan.  Stay resident until every planned SM has a block (or ~40 us pass), so
+        // that blocks still being placed can only land on SMs that have none yet.
+        const uint64_t t0 = globaltimer_ns();
+        while (true) {
+            int ok = 1;
+            for (int i = tid; i < p.b; i += kThreads)
+                ok &= (*reinterpret_cast<volatile unsigned int*>(&p.ctrl->claimed[i]) == p.epoch);
+            if (__syncthreads_and(ok)) break;
+            if (globaltimer_ns() - t0 > 40000ull) break;
+            __nanosleep(200);
+        }
+        return;
+    }
+    if (tid == 0) {
+        ctl->member = atomicMax(&p.ctrl->claimed[slot], p.epoch) < p.epoch;
+        ctl->abort_flag = 0;
+    }
+    __syncthreads();
+    if (!ctl->member) return;  // a second block on an SM whose slot is already taken
+
+    if (tid == 0) {
+        for (int i = 0; i < C::stages; ++i) {
+            mbar_init(smem_u32(&ctl->full[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), kEpiWarps);
+        }
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(smem_u32(&ctl->sched_full[i]), 1);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps);
+        }
+        mbar_init(smem_u32(&ctl->mma_drain), 1);
+        mbar_fence_init();
+        prefetch_tmap(&tm_a);
+        prefetch_tmap(&tm_b);
+        prefetch_tmap(&tm_c);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), C::tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const uint64_t limit = p.wait_limit_ns;
+
+    if (warp == 0) {
+        // ------------------------------------------------ scheduler + TMA producer (one lane)
+        if (lane == 0) {
+            const int my_die = p.image[lay.sm_die() + slot];
+            int cur_slot = slot, idx = 0;
+            int list_off = p.image[lay.sm_q_off() + slot], list_len = p.image[lay.sm_q_off() + slot + 1] - list_off;
+            int scan = 0;          // static mode: next slot to look at for adoption
+            int dyn_die = my_die;  // dynamic mode: queue being drained
+            uint32_t it = 0, kit = 0;
+            bool ok = true;
+            while (ok) {
+                int u = -1;
+                if (p.static_assign) {
+                    while (true) {
+                        if (idx < list_len) { u = p.image[lay.sm_q() + list_off + idx++]; break; }
+                        // own list done: run the list of any planned SM that never got a block
+                        bool adopted = false;
+                        for (; scan < p.b; ++scan) {
+                            if (*reinterpret_cast<volatile unsigned int*>(&p.ctrl->claimed[scan]) == p.epoch) continue;
+                            if (atomicMax(&p.ctrl->claimed[scan], p.epoch) < p.epoch) {
+                                cur_slot = scan;
+                                list_off = p.image[lay.sm_q_off() + cur_slot];
+                                list_len = p.image[lay.sm_q_off() + cur_slot + 1] - list_off;
+                                idx = 0;
+                                atomicAdd(&p.ctrl->adopted, 1u);
+                                adopted = true;
+                                ++scan;
+                                break;
+                            }
+                        }
+                        if (!adopted) break;
+                    }
+                } else {
+                    for (int t = 0; t < 2 && u < 0; ++t) {
+                        const int q_off = p.image[lay.die_q_off() + dyn_die];
+                        const int q_len = p.image[lay.die_q_off() + dyn_die + 1] - q_off;
+                        const int e = pop_queue(&p.ctrl->die_head[dyn_die], p.epoch, q_len);
+                        if (e >= 0) u = p.image[lay.die_q() + q_off + e];
+                        else dyn_die ^= 1;  // own die drained: help the other one
+                    }
+                }
+                const int r = it % kRing;
+                if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                    report_timeout(p, 1);
+                    ok = false;
+                    break;
+                }
+                ctl->ring[r] = u;
+                mbar_arrive(smem_u32(&ctl->sched_full[r]));
+                ++it;
+                if (u < 0) break;
+                const int ks = u % p.k_splits, t = u / p.k_splits;
+                const int tm = t / p.tiles_n, tn = t % p.tiles_n;
+                const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
+                const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+                for (int s = s0; s < s1; ++s, ++kit) {
+                    const int st = kit % C::stages;
+                    if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / C::stages) & 1) ^ 1, abort_flag, limit)) {
+                        report_timeout(p, 2);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&ctl->full[st]);
+                    const uint32_t sa = s_stage + st * C::stage_bytes, sb = sa + C::a_bytes;
+                    mbar_expect_tx(bar, C::stage_bytes);
+                    tma_load_2d(sa, &tm_a, bar, s * BK, tm * BM);
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tm_b, bar, tn * BN + j * 64, s * BK);
+                }
+            }
+            if (!ok) {
+                // gave up: let the copies already in flight land before the block leaves
+                const uint32_t n_out = kit < (uint32_t)C::stages ? kit : (uint32_t)C::stages;
+                for (uint32_t j = 0; j < n_out; ++j) {
+                    const uint32_t k2 = kit - 1 - j;
+                    int dummy = 0;
+                    mbar_wait(smem_u32(&ctl->full[k2 % C::stages]), (k2 / C::stages) & 1, &dummy, 2000000ull);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BM, BN, 0, 1);
+            uint32_t kit = 0, tile_it = 0;
+            bool ok = true;
+            for (uint32_t it = 0; ok; ++it) {
+                const int r = it % kRing;
+                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    report_timeout(p, 3);
+                    break;
+                }
+                const int u = ctl->ring[r];
+                mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                if (u < 0) break;
+                const int ks = u % p.k_splits;
+                const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
+                const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+                const uint32_t acc = tile_it & 1;
+                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
+                    report_timeout(p, 4);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int s = s0; s < s1; ++s, ++kit) {
+                    const int st = kit % C::stages;
+                    if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / C::stages) & 1, abort_flag, limit)) {
+                        report_timeout(p, 5);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = s_stage + st * C::stage_bytes, sb = sa + C::a_bytes;
+                    // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart.
+                    // B: N-major, 128-byte swizzle: 64-column blocks 8 KB apart (LBO), 8-k groups 1 KB apart (SBO).
+#pragma unroll
+                    for (int k4 = 0; k4 < BK / 16; ++k4) {
+                        const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
+                        const uint64_t db = make_smem_desc(sb + k4 * 2048, BK * 128, 1024, 2);
+                        tc_mma_f16(d_tmem, da, db, idesc, (s > s0 || k4 > 0) ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->empty[st]));  // slot reusable once these MMAs have read it
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                ++tile_it;
+            }
+            if (*abort_flag) {
+                // let issued MMAs retire before tensor memory is released
+                tc_commit(smem_u32(&ctl->mma_drain));
+                int dummy = 0;
+                mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue warps
+        const int q = warp & 3;  // tensor-memory lane quadrant this warp may read
+        const uint32_t buf0 = s_epi + (warp - 2) * 2 * kEpiBufBytes;
+        const bool reduce = p.k_splits > 1;
+        uint32_t tile_it = 0, chunk_it = 0;
+        for (uint32_t it = 0;; ++it) {
+            const int r = it % kRing;
+            if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                if (lane == 0) report_timeout(p, 6);
+                break;
+            }
+            const int u = ctl->ring[r];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+            if (u < 0) break;
+            const int t = u / p.k_splits;
+            const int tm = t / p.tiles_n, tn = t % p.tiles_n;
+            const uint32_t acc = tile_it & 1;
+            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
+                if (lane == 0) report_timeout(p, 7);
+                break;
+            }
+            tc_fence_after();
+            const int row0 = tm * BM + q * 32;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c, ++chunk_it) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c * 32, v);
+                tmem_ld_wait();
+                const uint32_t buf = buf0 + (chunk_it & 1) * kEpiBufBytes;
+                if (lane == 0) bulk_wait_read<1>();  // the store that last used this buffer has read it
+                __syncwarp();
+                const uint32_t rowaddr = buf + lane * 128;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t a = rowaddr + ((j ^ (lane & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v[4 * j]), "r"(v[4 * j + 1]),
+                                 "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
+                                 : "memory");
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    const int x = tn * BN + c * 32;
+                    if (x < p.N && row0 < p.M) {
+                        if (reduce) tma_reduce_add_2d(&tm_c, buf, x, row0);
+                        else tma_store_2d(&tm_c, buf, x, row0);
+                    }
+                    bulk_commit();
+                }
+            }
+            // accumulator fully read: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+                if (q == 0) {
+                    p.tile_owner[u] = my_sm;
+                    atomicAdd(&p.tile_count[u], 1);
+                }
+            }
+            ++tile_it;
+        }
+        if (lane == 0) bulk_wait<0>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// 2-D row-major tensor of `rows` x `cols` elements, box = box_cols x box_rows, 128-byte swizzle.
+static bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const void* ptr, uint64_t rows,
+                      uint64_t cols, uint32_t box_cols, uint32_t box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(tm, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+static ag_status launch(const ag_plan* plan, const GemmParams& gp, cudaStream_t stream) {
+    using C = Cfg<BN>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(k_gemm_persistent<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    k_gemm_persistent<BN><<<plan->lay.n_sm, kThreads, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);
+    count_launch();
+    AG_CUDA(cudaGetLastError());
+    return AG_OK;
+}
+
+}  // namespace ag
+
+using namespace ag;
+
+extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, int M, int N, int K,
+                                     const ag_plan* plan, void* cuda_stream) {
+    if (!A || !B || !Cout || !plan) return AG_ERR_ARG;
+    const int32_t* h = plan->header;
+    if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
+    if (h[H_TILE_M] != BM || (h[H_TILE_N] != 64 && h[H_TILE_N] != 128 && h[H_TILE_N] != 256)) return AG_ERR_ARG;
+    if (plan->policy.k_unit != BK) return AG_ERR_ARG;
+    if ((K % 8) || (N % 8)) return AG_ERR_ARG;
+    if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    int dev = 0, n_sm = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    if (n_sm != plan->lay.n_sm) return AG_ERR_ARG;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const int BN = h[H_TILE_N];
+    if (plan->tm_a_ptr != A || plan->tm_b_ptr != B || plan->tm_c_ptr != Cout) {
+        if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, BK, BM)) return AG_ERR_CUDA;
+        if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, BK)) return AG_ERR_CUDA;
+        if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
+        plan->tm_a_ptr = A; plan->tm_b_ptr = B; plan->tm_c_ptr = Cout;
+    }
+    if (h[H_KSPLITS] > 1) AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * (size_t)M * (size_t)N, stream));
+    GemmParams gp;
+    gp.image = plan->d_image;
+    gp.ctrl = plan->d_ctrl;
+    gp.tile_owner = plan->d_tile_owner;
+    gp.tile_count = plan->d_tile_count;
+    gp.M = M; gp.N = N; gp.K = K;
+    gp.b = plan->lay.b; gp.n_units = plan->lay.n_units; gp.n_sm = plan->lay.n_sm;
+    gp.tiles_n = h[H_TILES_N]; gp.k_splits = h[H_KSPLITS];
+    gp.kslabs_total = plan->kslabs_total; gp.kslabs_per_split = plan->kslabs_per_split;
+    gp.static_assign = h[H_STATIC];
+    gp.epoch = ++plan->epoch;
+    gp.wait_limit_ns = kWaitLimitNs;
+    if (BN == 256) return launch<256>(plan, gp, stream);
+    if (BN == 128) return launch<128>(plan, gp, stream);
+    return launch<64>(plan, gp, stream);
+}

@@ -1,0 +1,89 @@
+// Host-side internals shared by the translation units of the library.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "../../include/asymgemm.h"
+
+namespace ag {
+
+constexpr int32_t kPlanMagic = 0x41475031;
+constexpr int kHeaderWords = 16;
+
+// Header word indices of the plan image.
+enum { H_MAGIC = 0, H_KIND, H_NSM, H_B, H_NDIE, H_NUNITS, H_TILES_M, H_TILES_N, H_KSPLITS, H_TILE_M, H_TILE_N,
+       H_M, H_N, H_K, H_STATIC, H_ZERO };
+
+// Offsets (in int32 words) of the arrays inside the plan image, derived from b, n_units, n_sm.
+struct PlanLayout {
+    int b, n_units, n_sm;
+    __host__ __device__ int sm_list() const { return kHeaderWords; }
+    __host__ __device__ int sm_die() const { return sm_list() + b; }
+    __host__ __device__ int rank_in_die() const { return sm_die() + b; }
+    __host__ __device__ int die_sm_count() const { return rank_in_die() + b; }
+    __host__ __device__ int die_q_off() const { return die_sm_count() + 2; }
+    __host__ __device__ int die_q() const { return die_q_off() + 3; }
+    __host__ __device__ int sm_q_off() const { return die_q() + n_units; }
+    __host__ __device__ int sm_q() const { return sm_q_off() + b + 1; }
+    __host__ __device__ int smid_to_slot() const { return sm_q() + n_units; }
+    __host__ __device__ int total() const { return smid_to_slot() + n_sm; }
+};
+
+// Mutable per-plan control block on the device (zeroed at creation, self-resetting by epoch).
+struct PlanCtrl {
+    unsigned long long die_head[2];  // (epoch << 32) | next index, dynamic mode
+    int status;                      // ag_status of the last launch (0 = ok)
+    int status_info;                 // where the kernel gave up (role << 16 | smid)
+    unsigned int adopted;            // lists run by a block other than the one pinned to their SM
+    unsigned int pad;
+    unsigned int claimed[AG_MAX_SM]; // epoch of the launch whose block took this slot
+};
+
+}  // namespace ag
+
+struct ag_affinity_map {
+    const void* base;        // device pointer that was probed
+    size_t bytes;
+    size_t n_chunks;
+    uint8_t* d_die_of_chunk; // device, one byte per chunk
+    std::vector<uint8_t> h_die_of_chunk;
+    std::vector<uint32_t> h_cycles;  // min latency per chunk (empty for tables given by the caller)
+    int ref_sm[2];
+    uint32_t threshold;
+};
+
+struct ag_plan {
+    ag::PlanLayout lay;
+    int32_t header[ag::kHeaderWords];
+    ag_policy policy;
+    int32_t* d_image;          // device: the plan image (export layout)
+    ag::PlanCtrl* d_ctrl;      // device
+    int32_t* d_tile_owner;     // device [n_units]
+    int32_t* d_tile_count;     // device [n_units]
+    long long* d_margins;      // device [n_units] (affinity only, else null)
+    std::vector<int32_t> h_image;
+    mutable uint32_t epoch;
+    int kslabs_total;
+    int kslabs_per_split;
+    // tensor-map cache for the last (A, B, C) triple
+    mutable const void* tm_a_ptr; mutable const void* tm_b_ptr; mutable void* tm_c_ptr;
+    mutable CUtensorMap tm_a, tm_b, tm_c;
+};
+
+namespace ag {
+extern thread_local int g_last_cuda_error;
+extern std::atomic<unsigned long long> g_launch_count;
+inline void count_launch(int n = 1) { g_launch_count.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+ag_status check_arch();              // AG_OK on compute capability 10.x
+ag_status cuda_fail(cudaError_t e);  // records e, returns AG_ERR_CUDA (or AG_ERR_NOMEM)
+}  // namespace ag
+
+#define AG_CUDA(expr)                                         \
+    do {                                                      \
+        cudaError_t e__ = (expr);                             \
+        if (e__ != cudaSuccess) return ag::cuda_fail(e__);    \
+    } while (0)

@@ -1,0 +1,710 @@
+// topo_discover and affinity_probe: per-chip discovery of compute and memory asymmetry.
+//
+//   census           every SM reports %smid once (grid = #SMs, one block per SM)
+//   cluster probing  Section 5.1.1: thread-block clusters of size 3..8 are co-scheduled on one
+//                    GPC; SM ids seen together are merged (union-find); SMs never seen are "random"
+//   latency probing  Section 6.1.1 + appendix (HBM latency kernel): single thread, invalidate the
+//                    L2 line, L1-bypassing load, SM cycle counter; run from every SM it splits
+//                    the SMs into two partitions (dies)
+//   bandwidth probe  Section 5.1.2: SMs of one GPC share its crossbar port to L2; a random TPC
+//                    belongs to the GPC whose known SMs it slows down
+//   affinity probe   Section 6.1: chunk -> die from the two latency tiers, 4 KB chunks
+//
+// Pinning: a kernel cannot choose its SMs, so every probe launches one block per SM and lets
+// the blocks that landed on the wanted SMs work.  The others stay resident (bounded) until the
+// wanted SMs have checked in, so that all blocks sit on distinct SMs.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <numeric>
+#include <vector>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace ag {
+
+constexpr int kPinSmem = 120 * 1024;  // > half of an SM's shared memory: at most one block per SM
+constexpr int kRefChunks = 64;        // reference chunks for the SM -> die probe
+constexpr int kLatReps = 8;           // min over this many timed loads
+
+struct PinCtrl {
+    unsigned int arrived;   // members that have checked in
+    unsigned int pad[3];
+    unsigned long long t_start[AG_MAX_SM];
+    unsigned long long t_end[AG_MAX_SM];
+};
+
+// Members check in; everybody then waits (at most wait_ns) until all members are there.
+__device__ inline void pin_rendezvous(PinCtrl* pc, bool member, unsigned int n_members, unsigned long long wait_ns) {
+    if (threadIdx.x == 0) {
+        if (member) atomicAdd(&pc->arrived, 1u);
+        const unsigned long long t0 = globaltimer_ns();
+        while (*reinterpret_cast<volatile unsigned int*>(&pc->arrived) < n_members) {
+            if (globaltimer_ns() - t0 > wait_ns) break;
+            __nanosleep(100);
+        }
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ unsigned long long clock64_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t)::"memory");
+    return t;
+}
+
+// One timed L1-bypassing load; the add that consumes the value sits between the load and the
+// second clock read, so the clock is read only after the data has arrived.
+__device__ __forceinline__ uint32_t timed_load_cg(const void* p, uint32_t& sink) {
+    const unsigned long long t0 = clock64_now();
+    uint32_t v = ld_cg_u32(p);
+    asm volatile("add.u32 %0, %0, %1;" : "+r"(sink) : "r"(v) : "memory");
+    const unsigned long long t1 = clock64_now();
+    return (uint32_t)(t1 - t0);
+}
+
+// ---- census ---------------------------------------------------------------------------------
+__global__ void k_census(PinCtrl* pc, int* count, unsigned int n_blocks) {
+    if (threadIdx.x == 0) atomicAdd(&count[smid()], 1);
+    pin_rendezvous(pc, true, n_blocks, 100000ull);
+}
+
+// ---- cluster probe ---------------------------------------------------------------------------
+__global__ void k_cluster_probe(int* smid_of_block) {
+    if (threadIdx.x == 0) {
+        smid_of_block[blockIdx.x] = (int)smid();
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 20000ull) __nanosleep(500);  // stay a while so clusters spread out
+    }
+}
+
+// ---- latency probe from one SM -------------------------------------------------------------
+// mode 0: invalidate the L2 line first (HBM latency).  mode 1: plain timed load (whatever level
+// holds the line).  out[r] = min over reps; the 128-byte line is saved and written back.
+__global__ void k_latency_from_sm(PinCtrl* pc, int target_sm, uint8_t* buf, const long long* line_off, int n_lines,
+                                  int reps, int mode, uint32_t* out) {
+    const bool member = ((int)smid() == target_sm);
+    pin_rendezvous(pc, member, 1, 100000ull);
+    if (!member || threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    uint32_t sink = 0;
+    for (int r = 0; r < n_lines; ++r) {
+        uint8_t* line = buf + line_off[r];
+        uint32_t best = 0xffffffffu;
+        for (int k = 0; k < reps; ++k) {
+            uint32_t saved = 0;
+            if (mode == 0) {
+                saved = ld_cg_u32(line + lane * 4);
+                __syncwarp();
+                if (lane == 0) discard_l2_128(line);
+                __syncwarp();
+            }
+            if (lane == 0) {
+                sink += ld_cg_u32(line + 256);  // another line of the same chunk: warms the address translation
+                const uint32_t dt = timed_load_cg(line, sink);
+                best = min(best, dt);
+            }
+            __syncwarp();
+            if (mode == 0) {
+                reinterpret_cast<uint32_t*>(line)[lane] = saved;
+                __threadfence();
+            }
+        }
+        if (lane == 0) out[r] = best;
+    }
+    if (lane == 0 && sink == 0x12345678u) out[0] = sink;  // keep the loads alive
+}
+
+// ---- L2 bandwidth of a set of SMs ----------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+k_l2_bandwidth(PinCtrl* pc, const unsigned long long* member_mask, unsigned int n_members, const uint4* buf,
+               size_t slice_vec, int passes, unsigned int* sink_out) {
+    const int sm = (int)smid();
+    const bool member = (member_mask[sm >> 6] >> (sm & 63)) & 1ull;
+    pin_rendezvous(pc, member, n_members, 200000ull);
+    if (!member) return;
+    // each member streams its own slice (warm-up pass untimed, then `passes` timed passes)
+    const uint4* slice = buf + (size_t)(sm % 64) * slice_vec;
+    unsigned int acc = 0;
+    for (size_t i = threadIdx.x; i < slice_vec; i += blockDim.x) acc += ld_cg_u128(slice + i).x;
+    __syncthreads();
+    unsigned long long t0 = 0;
+    if (threadIdx.x == 0) t0 = globaltimer_ns();
+    for (int p = 0; p < passes; ++p)
+        for (size_t i = threadIdx.x; i < slice_vec; i += blockDim.x) {
+            const uint4 v = ld_cg_u128(slice + i);
+            acc += v.x ^ v.w;
+        }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        pc->t_start[sm] = t0;
+        pc->t_end[sm] = globaltimer_ns();
+    }
+    if (acc == 0x9e3779b9u) sink_out[0] = acc;
+}
+
+// ---- affinity probe over a buffer -----------------------------------------------------------------
+// Members (the SMs of one die) split the chunks round-robin; one warp per SM.  Per chunk: a few
+// 128-byte lines, each saved, invalidated in L2, loaded with a timed L1-bypassing load, restored.
+__global__ void k_affinity_probe(PinCtrl* pc, const int* member_rank /*[n_sm], -1 = not a member*/,
+                                 unsigned int n_members, uint8_t* buf, size_t n_chunks, int lines_per_chunk,
+                                 int reps, uint32_t* cycles) {
+    const int rank = member_rank[smid()];
+    pin_rendezvous(pc, rank >= 0, n_members, 200000ull);
+    if (rank < 0 || threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    uint32_t sink = 0;
+    for (size_t c = (size_t)rank; c < n_chunks; c += n_members) {
+        uint8_t* chunk = buf + c * AG_CHUNK_BYTES;
+        uint8_t* partner = buf + (c ^ 1) * AG_CHUNK_BYTES;  // other chunk of the aligned pair: same large page
+        if ((c ^ 1) >= n_chunks) partner = chunk + 3968;
+        uint32_t best = 0xffffffffu;
+        for (int l = 0; l < lines_per_chunk; ++l) {
+            uint8_t* line = chunk + ((l * 1152 + 128) % AG_CHUNK_BYTES);
+            for (int k = 0; k < reps; ++k) {
+                const uint32_t saved = ld_cg_u32(line + lane * 4);
+                __syncwarp();
+                if (lane == 0) {
+                    discard_l2_128(line);
+                    sink += ld_cg_u32(partner);  // translation for this large page is now cached
+                    best = min(best, timed_load_cg(line, sink));
+                }
+                __syncwarp();
+                reinterpret_cast<uint32_t*>(line)[lane] = saved;
+                __threadfence();
+            }
+        }
+        if (lane == 0) cycles[c] = best;
+    }
+    if (lane == 0 && sink == 0x12345678u) cycles[0] = sink;
+}
+
+// ---- host helpers ------------------------------------------------------------------------------------
+struct UnionFind {
+    std::vector<int> p;
+    explicit UnionFind(int n) : p(n) { std::iota(p.begin(), p.end(), 0); }
+    int find(int x) { while (p[x] != x) { p[x] = p[p[x]]; x = p[x]; } return x; }
+    void unite(int a, int b) { a = find(a); b = find(b); if (a != b) p[std::max(a, b)] = std::min(a, b); }
+};
+
+// 1-D two-means started at the extremes; returns false if the tiers are not clearly apart.
+static bool two_means(const std::vector<uint32_t>& v, double& lo, double& hi, double& thr) {
+    if (v.size() < 2) return false;
+    {
+        // start from the 5th / 95th percentile so that a stray slow sample cannot own a cluster
+        std::vector<uint32_t> sorted(v);
+        std::sort(sorted.begin(), sorted.end());
+        lo = sorted[sorted.size() / 20];
+        hi = sorted[sorted.size() - 1 - sorted.size() / 20];
+    }
+    if (hi <= lo) return false;
+    for (int it = 0; it < 32; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        double s0 = 0, s1 = 0;
+        size_t n0 = 0, n1 = 0;
+        for (uint32_t x : v) {
+            if (x <= mid) { s0 += x; ++n0; } else { s1 += x; ++n1; }
+        }
+        if (!n0 || !n1) return false;
+        const double nlo = s0 / n0, nhi = s1 / n1;
+        if (fabs(nlo - lo) < 0.5 && fabs(nhi - hi) < 0.5) { lo = nlo; hi = nhi; break; }
+        lo = nlo; hi = nhi;
+    }
+    thr = 0.5 * (lo + hi);
+    return hi > 1.15 * lo;  // the paper's tiers are 34 % (H200) and 67 % (B200) apart
+}
+
+static void finish_counts(ag_topo_map* m) {
+    memset(m->die_sm_count, 0, sizeof m->die_sm_count);
+    memset(m->gpc_sm_count, 0, sizeof m->gpc_sm_count);
+    m->n_unplaced = 0;
+    for (int s = 0; s < m->n_sm; ++s) {
+        m->die_sm_count[m->die[s] & 1]++;
+        if (m->gpc[s] >= 0) m->gpc_sm_count[m->gpc[s]]++; else m->n_unplaced++;
+    }
+    for (int g = 0; g < m->n_gpc; ++g) {
+        int c[2] = {0, 0};
+        for (int s = 0; s < m->n_sm; ++s)
+            if (m->gpc[s] == g) c[m->die[s] & 1]++;
+        m->gpc_die[g] = c[1] > c[0] ? 1 : 0;
+    }
+}
+
+}  // namespace ag
+
+using namespace ag;
+
+extern "C" ag_status ag_topo_from_observations(int32_t n_sm, const int32_t* cluster_sm, const int32_t* cluster_off,
+                                               int32_t n_clusters, const uint32_t* lat, int32_t n_ref,
+                                               ag_topo_map* map) {
+    if (!map || n_sm <= 0 || n_sm > AG_MAX_SM || n_clusters < 0 || (n_clusters > 0 && (!cluster_sm || !cluster_off)))
+        return AG_ERR_ARG;
+    memset(map, 0, sizeof *map);
+    map->n_sm = n_sm;
+    map->n_tpc = (n_sm + 1) / 2;
+    map->n_die = 2;
+    for (int s = 0; s < n_sm; ++s) {
+        map->tpc[s] = s / 2;  // two consecutive SM ids form a TPC (Section 5.1.2)
+        map->gpc[s] = -1;
+        map->is_random[s] = 1;
+    }
+    // GPC classes: SMs seen in one cluster share a GPC
+    UnionFind uf(n_sm);
+    std::vector<char> seen(n_sm, 0);
+    for (int c = 0; c < n_clusters; ++c) {
+        const int lo = cluster_off[c], hi = cluster_off[c + 1];
+        if (hi - lo < 3) continue;  // pairs say nothing beyond the TPC
+        for (int i = lo; i < hi; ++i) {
+            const int s = cluster_sm[i];
+            if (s < 0 || s >= n_sm) return AG_ERR_ARG;
+            seen[s] = 1;
+            uf.unite(cluster_sm[lo], s);
+        }
+    }
+    int n_gpc = 0;
+    std::vector<int> root_gpc(n_sm, -1);
+    for (int s = 0; s < n_sm; ++s) {
+        if (!seen[s]) continue;
+        map->is_random[s] = 0;
+        const int r = uf.find(s);
+        if (root_gpc[r] < 0) {
+            if (n_gpc >= AG_MAX_GPC) return AG_ERR_ARG;
+            root_gpc[r] = n_gpc++;
+        }
+        map->gpc[s] = root_gpc[r];
+    }
+    map->n_gpc = n_gpc;
+    if (n_clusters > 0) map->flags |= AG_TOPO_CLUSTER;
+    // dies: near/far pattern of every SM over the reference chunks, compared with SM 0's
+    if (lat && n_ref > 0) {
+        std::vector<uint32_t> all(lat, lat + (size_t)n_sm * n_ref);
+        double lo, hi, thr;
+        if (!two_means(all, lo, hi, thr)) return AG_ERR_NOISY_PROBE;
+        map->lat_near_cycles = (uint32_t)(lo + 0.5);
+        map->lat_far_cycles = (uint32_t)(hi + 0.5);
+        map->lat_threshold = (uint32_t)(thr + 0.5);
+        for (int s = 0; s < n_sm; ++s) {
+            int same = 0;
+            for (int r = 0; r < n_ref; ++r)
+                same += ((lat[(size_t)s * n_ref + r] > thr) == (lat[r] > thr));
+            if (same * 4 > n_ref && same * 4 < 3 * n_ref) return AG_ERR_NOISY_PROBE;
+            map->die[s] = same * 2 >= n_ref ? 0 : 1;
+        }
+        map->flags |= AG_TOPO_LATENCY;
+    }
+    finish_counts(map);
+    return AG_OK;
+}
+
+extern "C" int32_t ag_topo_place_by_gain(const double* gain, int32_t n, double solo_bw) {
+    if (!gain || n <= 0 || solo_bw <= 0) return -1;
+    int best = 0;
+    for (int i = 1; i < n; ++i)
+        if (gain[i] < gain[best]) best = i;
+    double runner = 1e300;
+    for (int i = 0; i < n; ++i)
+        if (i != best) runner = std::min(runner, gain[i]);
+    // contended: clearly less than one TPC's own bandwidth; the others: close to it
+    if (gain[best] < 0.80 * solo_bw && (n == 1 || runner > gain[best] + 0.10 * solo_bw)) return best;
+    return -1;
+}
+
+namespace {
+
+struct Scratch {
+    PinCtrl* pc = nullptr;
+    int* d_int = nullptr;
+    uint8_t* ref = nullptr;
+    long long* d_off = nullptr;
+    uint32_t* d_out = nullptr;
+    unsigned long long* d_mask = nullptr;
+    uint4* bw_buf = nullptr;
+    unsigned int* d_sink = nullptr;
+    ~Scratch() {
+        cudaFree(pc); cudaFree(d_int); cudaFree(ref); cudaFree(d_off); cudaFree(d_out); cudaFree(d_mask);
+        cudaFree(bw_buf); cudaFree(d_sink);
+    }
+};
+
+ag_status set_pin_smem() {
+    static bool done = false;
+    if (done) return AG_OK;
+    AG_CUDA(cudaFuncSetAttribute(k_census, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+    AG_CUDA(cudaFuncSetAttribute(k_cluster_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+    AG_CUDA(cudaFuncSetAttribute(k_latency_from_sm, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+    AG_CUDA(cudaFuncSetAttribute(k_l2_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+    AG_CUDA(cudaFuncSetAttribute(k_affinity_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+    done = true;
+    return AG_OK;
+}
+
+// aggregate L2 read bandwidth (bytes/s) of the SMs in `mask`, best of `tries`
+ag_status measure_bw(Scratch& sc, int n_sm, const unsigned long long mask[4], size_t slice_vec, int passes, int tries,
+                     double* bw) {
+    unsigned int n_members = 0;
+    for (int s = 0; s < n_sm; ++s) n_members += (mask[s >> 6] >> (s & 63)) & 1ull;
+    AG_CUDA(cudaMemcpy(sc.d_mask, mask, 4 * sizeof(unsigned long long), cudaMemcpyHostToDevice));
+    double best = 0;
+    std::vector<PinCtrl> h(1);
+    for (int t = 0; t < tries; ++t) {
+        AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
+        k_l2_bandwidth<<<n_sm, 512, kPinSmem>>>(sc.pc, sc.d_mask, n_members, sc.bw_buf, slice_vec, passes, sc.d_sink);
+        count_launch();
+        AG_CUDA(cudaGetLastError());
+        AG_CUDA(cudaDeviceSynchronize());
+        AG_CUDA(cudaMemcpy(h.data(), sc.pc, sizeof(PinCtrl), cudaMemcpyDeviceToHost));
+        unsigned long long t0 = ~0ull, t1 = 0;
+        unsigned int got = 0;
+        for (int s = 0; s < n_sm; ++s)
+            if ((mask[s >> 6] >> (s & 63)) & 1ull) {
+                if (h[0].t_end[s] == 0) continue;
+                ++got;
+                t0 = std::min(t0, h[0].t_start[s]);
+                t1 = std::max(t1, h[0].t_end[s]);
+            }
+        if (got != n_members || t1 <= t0) continue;  // an SM of the set got no block: try again
+        const double bytes = (double)n_members * passes * slice_vec * 16.0;
+        best = std::max(best, bytes / ((double)(t1 - t0) * 1e-9));
+    }
+    *bw = best;
+    return best > 0 ? AG_OK : AG_ERR_UNMANNED_SM;
+}
+
+ag_status latency_rows(Scratch& sc, int n_sm, const std::vector<int>& sms, int n_lines, int mode, int reps,
+                       std::vector<uint32_t>& out /* sms.size() x n_lines */) {
+    out.assign(sms.size() * (size_t)n_lines, 0);
+    for (size_t i = 0; i < sms.size(); ++i) {
+        bool ok = false;
+        for (int attempt = 0; attempt < 3 && !ok; ++attempt) {
+            AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
+            AG_CUDA(cudaMemset(sc.d_out, 0, sizeof(uint32_t) * n_lines));
+            k_latency_from_sm<<<n_sm, 32, kPinSmem>>>(sc.pc, sms[i], sc.ref, sc.d_off, n_lines, reps, mode, sc.d_out);
+            count_launch();
+            AG_CUDA(cudaGetLastError());
+            AG_CUDA(cudaDeviceSynchronize());
+            AG_CUDA(cudaMemcpy(&out[i * n_lines], sc.d_out, sizeof(uint32_t) * n_lines, cudaMemcpyDeviceToHost));
+            ok = out[i * n_lines] != 0;  // zero: no block landed on that SM
+        }
+        if (!ok) return AG_ERR_UNMANNED_SM;
+    }
+    return AG_OK;
+}
+
+}  // namespace
+
+extern "C" ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases) {
+    if (!map) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    st = set_pin_smem();
+    if (st != AG_OK) return st;
+    int dev = 0, n_sm = 0, clock_khz = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    AG_CUDA(cudaDeviceGetAttribute(&clock_khz, cudaDevAttrClockRate, dev));
+    if (n_sm > AG_MAX_SM) return AG_ERR_ARG;
+
+    Scratch sc;
+    const size_t ref_bytes = 8u << 20;
+    AG_CUDA(cudaMalloc(&sc.pc, sizeof(PinCtrl)));
+    AG_CUDA(cudaMalloc(&sc.d_int, sizeof(int) * 16384));
+    AG_CUDA(cudaMalloc(&sc.ref, ref_bytes));
+    AG_CUDA(cudaMemset(sc.ref, 0, ref_bytes));
+    AG_CUDA(cudaMalloc(&sc.d_off, sizeof(long long) * 1024));
+    AG_CUDA(cudaMalloc(&sc.d_out, sizeof(uint32_t) * 1024));
+    AG_CUDA(cudaMalloc(&sc.d_mask, 4 * sizeof(unsigned long long)));
+    AG_CUDA(cudaMalloc(&sc.d_sink, 64));
+
+    // ---- census: every SM id exactly once
+    AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
+    AG_CUDA(cudaMemset(sc.d_int, 0, sizeof(int) * AG_MAX_SM));
+    k_census<<<n_sm, 32, kPinSmem>>>(sc.pc, sc.d_int, (unsigned int)n_sm);
+    count_launch();
+    AG_CUDA(cudaGetLastError());
+    AG_CUDA(cudaDeviceSynchronize());
+    std::vector<int> cnt(AG_MAX_SM);
+    AG_CUDA(cudaMemcpy(cnt.data(), sc.d_int, sizeof(int) * AG_MAX_SM, cudaMemcpyDeviceToHost));
+    for (int s = 0; s < AG_MAX_SM; ++s)
+        if (cnt[s] != (s < n_sm ? 1 : 0)) return AG_ERR_UNMANNED_SM;
+
+    // ---- cluster probing, sizes 3..8
+    std::vector<int32_t> cl_sm, cl_off(1, 0);
+    if (phases & AG_TOPO_CLUSTER) {
+        for (int rep = 0; rep < 3; ++rep)
+            for (int cs = 3; cs <= 8; ++cs) {
+                const int n_clusters = std::max(1, (2 * n_sm) / cs);
+                const int grid = n_clusters * cs;
+                if (grid > 16384) continue;
+                cudaLaunchConfig_t cfg;
+                memset(&cfg, 0, sizeof cfg);
+                cfg.gridDim = dim3(grid);
+                cfg.blockDim = dim3(32);
+                cfg.dynamicSmemBytes = kPinSmem;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = cs;
+                attr[0].val.clusterDim.y = 1;
+                attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                AG_CUDA(cudaMemset(sc.d_int, 0xFF, sizeof(int) * grid));
+                cudaError_t e = cudaLaunchKernelEx(&cfg, k_cluster_probe, sc.d_int);
+                if (e != cudaSuccess) { cudaGetLastError(); continue; }  // this cluster size cannot be placed
+                count_launch();
+                AG_CUDA(cudaDeviceSynchronize());
+                std::vector<int> ids(grid);
+                AG_CUDA(cudaMemcpy(ids.data(), sc.d_int, sizeof(int) * grid, cudaMemcpyDeviceToHost));
+                for (int c = 0; c < n_clusters; ++c) {
+                    for (int i = 0; i < cs; ++i) cl_sm.push_back(ids[c * cs + i]);
+                    cl_off.push_back((int32_t)cl_sm.size());
+                }
+            }
+    }
+
+    // ---- latency from every SM to the reference chunks
+    std::vector<uint32_t> lat;
+    std::vector<long long> offs(kRefChunks);
+    if (phases & AG_TOPO_LATENCY) {
+        const long long n_chunks = (long long)(ref_bytes / AG_CHUNK_BYTES);
+        for (int r = 0; r < kRefChunks; ++r) offs[r] = ((r * 29LL + 3) % n_chunks) * AG_CHUNK_BYTES + 512;
+        AG_CUDA(cudaMemcpy(sc.d_off, offs.data(), sizeof(long long) * kRefChunks, cudaMemcpyHostToDevice));
+        std::vector<int> all(n_sm);
+        std::iota(all.begin(), all.end(), 0);
+        st = latency_rows(sc, n_sm, all, kRefChunks, 0, kLatReps, lat);
+        if (st != AG_OK) return st;
+    }
+    st = ag_topo_from_observations(n_sm, cl_sm.data(), cl_off.data(), (int32_t)cl_off.size() - 1,
+                                   lat.empty() ? nullptr : lat.data(), lat.empty() ? 0 : kRefChunks, map);
+    if (st != AG_OK) return st;
+    map->device = dev;
+    map->sm_clock_khz = (uint32_t)clock_khz;
+    map->flags |= AG_TOPO_CENSUS;
+
+    // ---- L2-hit latency, same-die and other-die reader (appendix, L2 latency kernel)
+    if ((phases & AG_TOPO_LATENCY) && map->die_sm_count[0] > 0 && map->die_sm_count[1] > 0) {
+        int other = -1;
+        for (int s = 0; s < n_sm && other < 0; ++s)
+            if (map->die[s] == 1) other = s;
+        // lines that are near for die 0
+        std::vector<long long> near_off;
+        for (int r = 0; r < kRefChunks; ++r)
+            if (lat[r] <= map->lat_threshold) near_off.push_back(offs[r] + 1024);
+        if (near_off.size() >= 4 && other >= 0) {
+            const int n = (int)near_off.size();
+            AG_CUDA(cudaMemcpy(sc.d_off, near_off.data(), sizeof(long long) * n, cudaMemcpyHostToDevice));
+            std::vector<uint32_t> tmp, nearv, farv;
+            st = latency_rows(sc, n_sm, std::vector<int>{0}, n, 1, 1, tmp);       // SM 0 caches the lines in its L2
+            if (st == AG_OK) st = latency_rows(sc, n_sm, std::vector<int>{0}, n, 1, 1, nearv);   // local hit
+            if (st == AG_OK) st = latency_rows(sc, n_sm, std::vector<int>{other}, n, 1, 1, farv);  // other-die reader
+            if (st != AG_OK) return st;
+            std::sort(nearv.begin(), nearv.end());
+            std::sort(farv.begin(), farv.end());
+            map->l2_near_cycles = nearv[n / 2];
+            map->l2_far_cycles = farv[n / 2];
+        }
+    }
+
+    // ---- place the random TPCs by L2-bandwidth contention
+    if ((phases & AG_TOPO_BANDWIDTH) && (map->flags & AG_TOPO_CLUSTER) && (map->flags & AG_TOPO_LATENCY) &&
+        map->n_unplaced > 0 && map->n_gpc > 0) {
+        const size_t slice_bytes = 1u << 20;  // per-SM slice: larger than L1, 64 slices fit well inside L2
+        const size_t slice_vec = slice_bytes / 16;
+        AG_CUDA(cudaMalloc(&sc.bw_buf, slice_bytes * 64));
+        AG_CUDA(cudaMemset(sc.bw_buf, 1, slice_bytes * 64));
+        const int passes = 8, tries = 3;
+        std::vector<double> base_bw(map->n_gpc, -1.0);
+        auto mask_of_gpc = [&](int g, unsigned long long m[4]) {
+            m[0] = m[1] = m[2] = m[3] = 0;
+            for (int s = 0; s < n_sm; ++s)
+                if (map->gpc[s] == g && !map->is_random[s]) m[s >> 6] |= 1ull << (s & 63);
+        };
+        for (int t = 0; t < map->n_tpc; ++t) {
+            const int s0 = 2 * t, s1 = 2 * t + 1;
+            if (s0 >= n_sm || map->gpc[s0] >= 0) continue;
+            unsigned long long m[4] = {0, 0, 0, 0};
+            m[s0 >> 6] |= 1ull << (s0 & 63);
+            if (s1 < n_sm) m[s1 >> 6] |= 1ull << (s1 & 63);
+            double solo = 0;
+            if (measure_bw(sc, n_sm, m, slice_vec, passes, tries, &solo) != AG_OK) continue;
+            std::vector<int> cands;
+            std::vector<double> gains;
+            for (int g = 0; g < map->n_gpc; ++g) {
+                if (map->gpc_die[g] != map->die[s0]) continue;  // a TPC sits on the die its latency shows
+                unsigned long long mg[4];
+                mask_of_gpc(g, mg);
+                if (base_bw[g] < 0 && measure_bw(sc, n_sm, mg, slice_vec, passes, tries, &base_bw[g]) != AG_OK) continue;
+                for (int i = 0; i < 4; ++i) mg[i] |= m[i];
+                double with = 0;
+                if (measure_bw(sc, n_sm, mg, slice_vec, passes, tries, &with) != AG_OK) continue;
+                cands.push_back(g);
+                gains.push_back(with - base_bw[g]);
+            }
+            const int pick = ag_topo_place_by_gain(gains.data(), (int)gains.size(), solo);
+            if (pick >= 0) {
+                map->gpc[s0] = cands[pick];
+                if (s1 < n_sm) map->gpc[s1] = cands[pick];
+            }
+        }
+        map->flags |= AG_TOPO_BANDWIDTH;
+        finish_counts(map);
+    }
+    return AG_OK;
+}
+
+extern "C" ag_status topo_discover(ag_topo_map* map) {
+    return ag_topo_discover_phases(map, AG_TOPO_CENSUS | AG_TOPO_CLUSTER | AG_TOPO_LATENCY | AG_TOPO_BANDWIDTH);
+}
+
+// ---- affinity --------------------------------------------------------------------------------------------
+static ag_status probe_from_die(uint8_t* buf, size_t n_chunks, const ag_topo_map* map, int die,
+                                std::vector<uint32_t>& cycles, int ref_sm[2]) {
+    ag_status st = set_pin_smem();
+    if (st != AG_OK) return st;
+    const int n_sm = map->n_sm;
+    std::vector<int> rank(AG_MAX_SM, -1);
+    unsigned int n_members = 0;
+    for (int s = 0; s < n_sm; ++s)
+        if (map->die[s] == die) {
+            if (ref_sm[die] < 0) ref_sm[die] = s;
+            rank[s] = (int)n_members++;
+        }
+    if (n_members == 0) return AG_ERR_ARG;
+    PinCtrl* pc = nullptr;
+    int* d_rank = nullptr;
+    uint32_t* d_cycles = nullptr;
+    cudaError_t e = cudaSuccess;
+    do {
+        if ((e = cudaMalloc(&pc, sizeof(PinCtrl))) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_rank, sizeof(int) * AG_MAX_SM)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_cycles, sizeof(uint32_t) * n_chunks)) != cudaSuccess) break;
+        if ((e = cudaMemset(pc, 0, sizeof(PinCtrl))) != cudaSuccess) break;
+        if ((e = cudaMemset(d_cycles, 0, sizeof(uint32_t) * n_chunks)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(d_rank, rank.data(), sizeof(int) * AG_MAX_SM, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        k_affinity_probe<<<n_sm, 32, kPinSmem>>>(pc, d_rank, n_members, buf, n_chunks, 3, 2, d_cycles);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) break;
+        if ((e = cudaDeviceSynchronize()) != cudaSuccess) break;
+        cycles.resize(n_chunks);
+        e = cudaMemcpy(cycles.data(), d_cycles, sizeof(uint32_t) * n_chunks, cudaMemcpyDeviceToHost);
+    } while (0);
+    cudaFree(pc);
+    cudaFree(d_rank);
+    cudaFree(d_cycles);
+    if (e != cudaSuccess) return cuda_fail(e);
+    for (uint32_t c : cycles)
+        if (c == 0) return AG_ERR_UNMANNED_SM;  // a member SM got no block: its chunks were not probed
+    return AG_OK;
+}
+
+static ag_status classify(const std::vector<uint32_t>& cycles, int near_die, std::vector<uint8_t>& table,
+                          uint32_t* threshold) {
+    double lo, hi, thr;
+    if (!two_means(cycles, lo, hi, thr)) return AG_ERR_NOISY_PROBE;
+    table.resize(cycles.size());
+    size_t ambiguous = 0;
+    for (size_t i = 0; i < cycles.size(); ++i) {
+        table[i] = (uint8_t)((cycles[i] > thr) ? 1 - near_die : near_die);
+        if (fabs((double)cycles[i] - thr) < 0.05 * thr) ++ambiguous;
+    }
+    *threshold = (uint32_t)(thr + 0.5);
+    if (ambiguous * 100 > cycles.size()) return AG_ERR_NOISY_PROBE;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_affinity_from_table(const void* buf, size_t bytes, const uint8_t* die_of_chunk,
+                                            size_t n_chunks, ag_affinity_map** out) {
+    if (!out || !die_of_chunk || n_chunks == 0 || bytes != n_chunks * AG_CHUNK_BYTES) return AG_ERR_ARG;
+    *out = nullptr;
+    ag_affinity_map* a = new (std::nothrow) ag_affinity_map();
+    if (!a) return AG_ERR_NOMEM;
+    a->base = buf;
+    a->bytes = bytes;
+    a->n_chunks = n_chunks;
+    a->d_die_of_chunk = nullptr;
+    a->h_die_of_chunk.assign(die_of_chunk, die_of_chunk + n_chunks);
+    for (auto& v : a->h_die_of_chunk) v = v ? 1 : 0;
+    a->ref_sm[0] = a->ref_sm[1] = -1;
+    a->threshold = 0;
+    cudaError_t e = cudaMalloc(&a->d_die_of_chunk, n_chunks);
+    if (e == cudaSuccess) e = cudaMemcpy(a->d_die_of_chunk, a->h_die_of_chunk.data(), n_chunks, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        ag_affinity_destroy(a);
+        return cuda_fail(e);
+    }
+    *out = a;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_affinity_probe_with_map(void* buf, size_t bytes, const ag_topo_map* map,
+                                                ag_affinity_map** out) {
+    if (!buf || !map || !out || bytes == 0 || (bytes % AG_CHUNK_BYTES) || ((uintptr_t)buf % AG_CHUNK_BYTES))
+        return AG_ERR_ARG;
+    *out = nullptr;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    if (!(map->flags & AG_TOPO_LATENCY)) return AG_ERR_ARG;
+    const size_t n_chunks = bytes / AG_CHUNK_BYTES;
+    std::vector<uint32_t> cycles;
+    int ref_sm[2] = {-1, -1};
+    st = probe_from_die((uint8_t*)buf, n_chunks, map, 0, cycles, ref_sm);
+    if (st != AG_OK) return st;
+    std::vector<uint8_t> table;
+    uint32_t thr = 0;
+    st = classify(cycles, 0, table, &thr);
+    if (st != AG_OK) return st;
+    st = ag_affinity_from_table(buf, bytes, table.data(), n_chunks, out);
+    if (st != AG_OK) return st;
+    (*out)->h_cycles.swap(cycles);
+    (*out)->ref_sm[0] = ref_sm[0];
+    (*out)->threshold = thr;
+    return AG_OK;
+}
+
+extern "C" ag_status affinity_probe(void* buf, size_t bytes, ag_affinity_map** out) {
+    ag_topo_map map;
+    ag_status st = ag_topo_discover_phases(&map, AG_TOPO_CENSUS | AG_TOPO_LATENCY);
+    if (st != AG_OK) return st;
+    return ag_affinity_probe_with_map(buf, bytes, &map, out);
+}
+
+extern "C" ag_status ag_affinity_check_complement(const ag_affinity_map* amap, const ag_topo_map* map,
+                                                  size_t* mismatches) {
+    if (!amap || !map || !mismatches) return AG_ERR_ARG;
+    std::vector<uint32_t> cycles;
+    int ref_sm[2] = {-1, -1};
+    ag_status st = probe_from_die((uint8_t*)amap->base, amap->n_chunks, map, 1, cycles, ref_sm);
+    if (st != AG_OK) return st;
+    std::vector<uint8_t> table;
+    uint32_t thr = 0;
+    st = classify(cycles, 1, table, &thr);
+    if (st != AG_OK) return st;
+    size_t bad = 0;
+    for (size_t i = 0; i < table.size(); ++i) bad += table[i] != amap->h_die_of_chunk[i];
+    *mismatches = bad;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_affinity_export(const ag_affinity_map* amap, uint8_t* die_of_chunk, size_t cap,
+                                        size_t* n_chunks) {
+    if (!amap) return AG_ERR_ARG;
+    if (n_chunks) *n_chunks = amap->n_chunks;
+    if (!die_of_chunk) return n_chunks ? AG_OK : AG_ERR_ARG;
+    if (cap < amap->n_chunks) return AG_ERR_ARG;
+    memcpy(die_of_chunk, amap->h_die_of_chunk.data(), amap->n_chunks);
+    return AG_OK;
+}
+
+extern "C" ag_status ag_affinity_cycles(const ag_affinity_map* amap, uint32_t* cycles, size_t cap) {
+    if (!amap || !cycles || amap->h_cycles.empty() || cap < amap->n_chunks) return AG_ERR_ARG;
+    memcpy(cycles, amap->h_cycles.data(), amap->n_chunks * sizeof(uint32_t));
+    return AG_OK;
+}
+
+extern "C" void ag_affinity_destroy(ag_affinity_map* amap) {
+    if (!amap) return;
+    cudaFree(amap->d_die_of_chunk);
+    delete amap;
+}

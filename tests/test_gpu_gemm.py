@@ -1,0 +1,139 @@
+"""gemm_persistent through the C ABI against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gemm as og
+from paper_2609_24270_b200 import binding as ag
+from paper_2609_24270_b200 import inputs
+from tests.gpu_util import check_close, device_topo, run_gemm, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def plan_for(M, N, K, b=None, **kw):
+    topo = device_topo()
+    b = topo.n_sm if b is None else b
+    return ag.sched_build(topo, None, b, ag.make_policy(M=M, N=N, K=K, **kw))
+
+
+@pytest.mark.parametrize("shape", [(128, 256, 64), (128, 256, 256), (256, 512, 128), (1024, 1024, 1024)])
+def test_integer_inputs_bit_exact(shape):
+    """Entries in {-2..2}: every partial sum is a small integer, so fp32 accumulation is exact in
+    any order and the result must equal the oracle bit for bit.  Pins tile indexing, swizzles,
+    k-slab order and epilogue addressing."""
+    M, N, K = shape
+    A = inputs.small_int_bf16(M, K, seed=1)
+    B = inputs.small_int_bf16(K, N, seed=2)
+    plan = plan_for(M, N, K)
+    C = run_gemm(A, B, plan)
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+
+
+def test_one_hot_localises_addressing():
+    M, N, K = 256, 512, 192
+    B = inputs.uniform_bf16(K, N, seed=8)
+    A = np.zeros((M, K), dtype=np.float32)
+    A[130, 77] = 1.0
+    A[5, 191] = 2.0
+    Ab = inputs.f32_to_bf16_bits(A)
+    C = run_gemm(Ab, B, plan_for(M, N, K))
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(Ab, B))
+
+
+@pytest.mark.parametrize("shape", [(1024, 1024, 1024), (1000, 1000, 1000), (333, 776, 520), (1, 8, 8), (129, 264, 72),
+                                   (2048, 2304, 1536)])
+def test_uniform_inputs_within_tolerance(shape):
+    M, N, K = shape
+    A, B = inputs.gemm_inputs(M, N, K)
+    C = run_gemm(A, B, plan_for(M, N, K, kind=ag.AG_DIE_COMPACT, raster_group=2))
+    check_close(C, og.gemm_blocked(A, B))
+
+
+@pytest.mark.parametrize("tile_n", [64, 128, 256])
+@pytest.mark.parametrize("k_splits", [1, 4])
+def test_tile_widths_and_split_k(tile_n, k_splits):
+    M, N, K = 512, 768, 1024
+    A, B = inputs.gemm_inputs(M, N, K, seed=77)
+    C = run_gemm(A, B, plan_for(M, N, K, tile_n=tile_n, k_splits=k_splits))
+    check_close(C, og.gemm_blocked(A, B))
+    Ai, Bi = inputs.small_int_bf16(M, K, 3), inputs.small_int_bf16(K, N, 4)
+    Ci = run_gemm(Ai, Bi, plan_for(M, N, K, tile_n=tile_n, k_splits=k_splits))
+    assert np.array_equal(Ci.astype(np.float64), og.gemm_blocked(Ai, Bi))
+
+
+@pytest.mark.parametrize("kind", [ag.AG_OBLIVIOUS, ag.AG_DIE_COMPACT])
+@pytest.mark.parametrize("b", [1, 16, 37, 74, 148])
+@pytest.mark.parametrize("static", [1, 0])
+def test_sm_budgets_policies_and_dynamic_queues(kind, b, static):
+    M, N, K = 1024, 1536, 512
+    A, B = inputs.small_int_bf16(M, K, 5), inputs.small_int_bf16(K, N, 6)
+    plan = plan_for(M, N, K, b=b, kind=kind, static_assign=static, seed=0)
+    plan.reset_record()
+    C = run_gemm(A, B, plan)
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+    owner, count = plan.tile_record()
+    assert (count == 1).all()                               # every unit ran exactly once
+    p = plan.parsed()
+    assert set(owner) <= set(p["sm_list"])                  # only planned SMs did any work
+    if static:
+        want = np.empty(p["n_units"], dtype=np.int32)
+        for slot in range(b):
+            want[p["sm_q"][p["sm_q_off"][slot]:p["sm_q_off"][slot + 1]]] = p["sm_list"][slot]
+        assert np.array_equal(owner, want)                  # the SM the plan names ran the unit
+
+
+def test_random_subset_and_repeat_launches():
+    M, N, K = 1024, 1024, 256
+    A, B = inputs.small_int_bf16(M, K, 9), inputs.small_int_bf16(K, N, 10)
+    want = og.gemm_blocked(A, B)
+    plan = plan_for(M, N, K, b=32, seed=5)
+    dA, dB = to_dev_bf16(A), to_dev_bf16(B)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    for _ in range(5):                                      # epochs: claim flags reset themselves
+        dC.fill_(float("nan"))
+        ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), want)
+
+
+def test_non_default_stream():
+    M, N, K = 512, 512, 512
+    A, B = inputs.gemm_inputs(M, N, K, seed=4)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        C = run_gemm(A, B, plan_for(M, N, K), stream=s)
+    check_close(C, og.gemm_blocked(A, B))
+
+
+def test_rejects_mismatched_shapes_and_alignment():
+    plan = plan_for(256, 256, 256)
+    t = torch.zeros(1 << 20, dtype=torch.int16, device="cuda")
+    c = torch.zeros(1 << 20, dtype=torch.float32, device="cuda")
+    L = ag.lib()
+    assert L.gemm_persistent(t.data_ptr(), t.data_ptr(), c.data_ptr(), 256, 256, 128, plan.handle, None) == ag.AG_ERR_ARG
+    assert L.gemm_persistent(t.data_ptr() + 2, t.data_ptr(), c.data_ptr(), 256, 256, 256, plan.handle, None) == ag.AG_ERR_ARG
+    with pytest.raises(ag.AgError):
+        p2 = plan_for(256, 252, 256)
+        ag.gemm_persistent(t.data_ptr(), t.data_ptr(), c.data_ptr(), 256, 252, 256, p2)
+
+
+def test_full_size_sampled_against_oracle():
+    """8192^3 in the bench's launch configuration; the oracle computes sampled entries one by
+    one and one full 128 x 256 tile."""
+    M = N = K = 8192
+    A, B = inputs.gemm_inputs(M, N, K)
+    plan = plan_for(M, N, K, kind=ag.AG_DIE_COMPACT, raster_group=8)
+    C = run_gemm(A, B, plan)
+    rng = np.random.default_rng(0)
+    rows, cols = rng.integers(0, M, 200), rng.integers(0, N, 200)
+    rows[:4], cols[:4] = [0, M - 1, 0, M - 1], [0, 0, N - 1, N - 1]
+    ref = og.gemm_entries(A, B, rows, cols)
+    got = C[rows, cols].astype(np.float64)
+    assert np.abs(got - ref).max() <= 1e-2
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-4
+    blk = og.gemm_block(A, B, 8064, 8192, 7936, 8192)       # the last tile
+    check_close(C[8064:8192, 7936:8192], blk)
+    owner, count = plan.tile_record()
+    assert (count == 1).all()

@@ -1,0 +1,81 @@
+"""topo_discover / affinity_probe on the real chip: no CPU oracle exists for a measurement, so
+the maps are pinned by the structure the paper reports for B200 and by self-consistency."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_24270_b200 import binding as ag
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def topo():
+    return ag.topo_discover()
+
+
+def test_census_and_tpc_pairs(topo):
+    m = topo.as_dict()
+    assert m["n_sm"] == torch.cuda.get_device_properties(0).multi_processor_count
+    assert m["tpc"] == [s // 2 for s in range(m["n_sm"])]
+    assert m["flags"] & ag.AG_TOPO_CENSUS
+
+
+def test_die_split(topo):
+    m = topo.as_dict()
+    n0, n1 = m["die_sm_count"]
+    assert n0 + n1 == m["n_sm"] and m["die"][0] == 0
+    assert abs(n0 - n1) <= 8                                 # B200 partitions differ by at most 8 SMs (Section 6.1.1)
+    for t in range(m["n_sm"] // 2):                          # both SMs of a TPC sit on one die
+        assert m["die"][2 * t] == m["die"][2 * t + 1]
+    # latency tiers: far/near about 1.67 on B200 (552 -> 920 cycles); a band, not an equality
+    ratio = m["lat_far_cycles"] / m["lat_near_cycles"]
+    assert 1.25 < ratio < 2.3, (m["lat_near_cycles"], m["lat_far_cycles"])
+    if m["l2_near_cycles"]:
+        assert 1.3 < m["l2_far_cycles"] / m["l2_near_cycles"] < 3.0
+
+
+def test_gpc_classes(topo):
+    m = topo.as_dict()
+    if not (m["flags"] & ag.AG_TOPO_CLUSTER) or m["n_gpc"] == 0:
+        pytest.skip("cluster probing gave no classes on this device")
+    assert m["n_gpc"] == 8                                   # 2 dies x 4 GPCs (Table 1)
+    for g in range(m["n_gpc"]):
+        members = [s for s in range(m["n_sm"]) if m["gpc"][s] == g]
+        assert 2 <= len(members) <= 20                       # at most 10 TPCs per GPC
+        assert len({m["die"][s] for s in members}) == 1      # GPC classes nest inside die classes
+    assert sum(1 for g in range(8) if m["gpc_die"][g] == 0) == 4
+    for t in range(m["n_sm"] // 2):
+        assert m["gpc"][2 * t] == m["gpc"][2 * t + 1]
+    normal = [s for s in range(m["n_sm"]) if not m["is_random"][s]]
+    assert all(m["gpc"][s] >= 0 for s in normal)
+
+
+def test_discovery_is_repeatable(topo):
+    again = ag.topo_discover(ag.AG_TOPO_CENSUS | ag.AG_TOPO_CLUSTER | ag.AG_TOPO_LATENCY).as_dict()
+    m = topo.as_dict()
+    assert again["die"] == m["die"]
+    assert again["is_random"] == m["is_random"]
+    same_class = lambda g: {(a, b) for a in range(0, m["n_sm"], 7) for b in range(0, m["n_sm"], 5)
+                            if g[a] >= 0 and g[a] == g[b]}
+    normal_gpc = [g if not r else -1 for g, r in zip(m["gpc"], m["is_random"])]
+    assert same_class(again["gpc"]) == same_class(normal_gpc)
+
+
+def test_affinity_probe_structure_and_content_preserved(topo):
+    nbytes = 64 << 20
+    buf = torch.arange(nbytes // 4, dtype=torch.int32, device="cuda")
+    before = buf.clone()
+    amap = ag.affinity_probe(buf.data_ptr(), nbytes, topo)
+    torch.cuda.synchronize()
+    assert torch.equal(buf, before)                          # probed lines are saved and written back
+    t = amap.export()
+    assert t.size == nbytes // 4096 and set(np.unique(t)) == {0, 1}
+    assert abs(t.mean() - 0.5) < 0.02                        # interleaved across the two dies
+    base_chunk = (buf.data_ptr() // 4096) & 1
+    pairs = t[base_chunk:].copy()
+    pairs = pairs[: (pairs.size // 2) * 2].reshape(-1, 2)
+    assert (pairs[:, 0] != pairs[:, 1]).mean() > 0.99        # each aligned pair of 4 KB pages: one per die (Section 7.1.1)
+    assert amap.check_complement(topo) <= t.size // 200      # a die-1 SM sees the opposite tiers
+    again = ag.affinity_probe(buf.data_ptr(), nbytes, topo).export()
+    assert (again != t).sum() <= t.size // 200               # repeatable
