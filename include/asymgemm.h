@@ -103,22 +103,47 @@ ag_status ag_topo_from_observations(int32_t n_sm, const int32_t* cluster_sm, con
  */
 int32_t ag_topo_place_by_gain(const double* gain, int32_t n_candidates, double solo_bw);
 
+/*
+ * ag_probe_latency_samples - raw access-latency samples from one SM: the measurement behind the
+ * HBM and L2 latency histograms of Section 6.1.1 (kernels in the appendix).  Line r lies in
+ * 4 KB chunk (29 r + 3) mod 2048 of a library-owned 8 MiB scratch buffer.
+ *   sm     SM id that takes the samples
+ *   mode   0: invalidate the L2 line before each timed load (HBM latency);
+ *          1: plain timed L1-bypassing load (latency of whichever level holds the line)
+ *   cycles host, out, n_lines x reps values (n_lines <= 1024, reps <= 64), SM clock cycles
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_UNMANNED_SM.
+ */
+ag_status ag_probe_latency_samples(int sm, int mode, int n_lines, int reps, uint32_t* cycles);
+
+/*
+ * ag_probe_l2_bandwidth - aggregate L2 read bandwidth (bytes/s) of a chosen set of SMs, the
+ * measurement behind Section 5.1.2 (and its per-GPC bandwidth figure): every SM of the set
+ * re-reads a 1 MiB slice (larger than L1, all slices together far smaller than L2) with
+ * L1-bypassing loads; best of three runs.
+ *   sm_mask  host, bit s = SM s takes part.  bytes_per_s  host, out.
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_UNMANNED_SM.
+ */
+ag_status ag_probe_l2_bandwidth(const uint64_t sm_mask[4], double* bytes_per_s);
+
 /* ---- memory affinity (Section 6.1) ------------------------------------------------------ */
 typedef struct ag_affinity_map ag_affinity_map;
 
 /*
- * affinity_probe - chunk -> die map of a device buffer from HBM access latency
- * (Section 6.1.1 and the HBM-latency kernel of the appendix: invalidate the L2 line, load it
- * with an L1-bypassing load, time the round trip with the SM cycle counter; the minimum over
- * several lines of the chunk is kept).  A chunk is AG_CHUNK_BYTES; die 0 is the die of SM 0.
+ * affinity_probe - chunk -> die map of a device buffer from access latency (Section 6.1.1 and
+ * the latency kernels of the appendix: a single thread invalidates the L2 line, loads it with an
+ * L1-bypassing load and times the round trip with the SM cycle counter; the minimum over several
+ * lines and repeats of the chunk is kept).  Every chunk is timed from the SMs of die 0 and from
+ * the SMs of die 1; it belongs to the die that reaches it faster.  A chunk is AG_CHUNK_BYTES;
+ * die 0 is the die of SM 0.
  *   buf    device pointer, 4096-byte aligned; contents are preserved (each probed 128-byte
  *          line is saved before the L2 invalidation and written back afterwards).  Nothing
  *          else may touch the buffer while the probe runs.
  *   bytes  multiple of 4096.
  *   amap   host, out: new handle.
- * Runs topo_discover's census + latency phases internally when no map has been supplied via
- * ag_affinity_probe_with_map.  Synchronises the device.
- * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_NOISY_PROBE, AG_ERR_NOMEM.
+ * affinity_probe runs the census + latency phases of topo_discover itself;
+ * ag_affinity_probe_with_map takes a map that already has them.  Synchronises the device.
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_NOISY_PROBE (more than 2 % of
+ * the chunks show no clear difference between the dies), AG_ERR_UNMANNED_SM, AG_ERR_NOMEM.
  */
 ag_status affinity_probe(void* buf, size_t bytes, ag_affinity_map** amap);
 ag_status ag_affinity_probe_with_map(void* buf, size_t bytes, const ag_topo_map* map,
@@ -127,12 +152,14 @@ ag_status ag_affinity_probe_with_map(void* buf, size_t bytes, const ag_topo_map*
  * lets plans be built for a recorded or synthetic layout. */
 ag_status ag_affinity_from_table(const void* buf, size_t bytes, const uint8_t* die_of_chunk,
                                  size_t n_chunks, ag_affinity_map** amap);
-/* Copy out the chunk->die table (host, cap bytes) and/or the raw min-latency cycles. */
+/* Copy out the chunk->die table (host, cap bytes). */
 ag_status ag_affinity_export(const ag_affinity_map* amap, uint8_t* die_of_chunk, size_t cap,
                              size_t* n_chunks);
+/* Raw min-latency cycles (host, cap >= 2 * n_chunks words): first the values seen from die 0,
+ * then those seen from die 1.  Only for probed maps. */
 ag_status ag_affinity_cycles(const ag_affinity_map* amap, uint32_t* cycles, size_t cap);
-/* Probe again from an SM of the other die; returns in *mismatches how many chunks are not
- * the complement of the stored table (Section 6.1.1: the two groups of SMs see opposite tiers). */
+/* Section 6.1.1: the two groups of SMs see opposite tiers.  *mismatches = number of chunks whose
+ * two latencies were less than 25 % apart, i.e. that did not show opposite tiers. */
 ag_status ag_affinity_check_complement(const ag_affinity_map* amap, const ag_topo_map* map,
                                        size_t* mismatches);
 void ag_affinity_destroy(ag_affinity_map* amap);

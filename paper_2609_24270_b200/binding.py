@@ -22,6 +22,7 @@ AG_TOPO_CENSUS, AG_TOPO_CLUSTER, AG_TOPO_LATENCY, AG_TOPO_BANDWIDTH = 1, 2, 4, 8
 
 EXPORTED = [
     "topo_discover", "ag_topo_discover_phases", "ag_topo_from_observations", "ag_topo_place_by_gain",
+    "ag_probe_l2_bandwidth", "ag_probe_latency_samples",
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
@@ -106,6 +107,8 @@ def lib() -> C.CDLL:
     L.ag_topo_from_observations.argtypes = [i32, vp, vp, i32, vp, i32, C.POINTER(TopoMap)]
     L.ag_topo_place_by_gain.argtypes = [C.POINTER(C.c_double), i32, C.c_double]
     L.ag_topo_place_by_gain.restype = i32
+    L.ag_probe_latency_samples.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp]
+    L.ag_probe_l2_bandwidth.argtypes = [C.POINTER(C.c_uint64), C.POINTER(C.c_double)]
     L.affinity_probe.argtypes = [vp, sz, C.POINTER(vp)]
     L.ag_affinity_probe_with_map.argtypes = [vp, sz, C.POINTER(TopoMap), C.POINTER(vp)]
     L.ag_affinity_from_table.argtypes = [vp, sz, vp, sz, C.POINTER(vp)]
@@ -174,6 +177,23 @@ def topo_place_by_gain(gains, solo_bw: float) -> int:
     return int(lib().ag_topo_place_by_gain(arr, len(gains), solo_bw))
 
 
+def probe_latency_samples(sm: int, mode: int = 0, n_lines: int = 256, reps: int = 8) -> np.ndarray:
+    """n_lines x reps raw latency samples (SM cycles) taken from SM `sm`."""
+    out = np.zeros((n_lines, reps), dtype=np.uint32)
+    _check(lib().ag_probe_latency_samples(sm, mode, n_lines, reps, out.ctypes.data), "ag_probe_latency_samples")
+    return out
+
+
+def probe_l2_bandwidth(sms) -> float:
+    """Aggregate L2 read bandwidth in bytes/s of the given SM ids."""
+    mask = (C.c_uint64 * 4)()
+    for s in sms:
+        mask[s >> 6] |= 1 << (s & 63)
+    out = C.c_double()
+    _check(lib().ag_probe_l2_bandwidth(mask, C.byref(out)), "ag_probe_l2_bandwidth")
+    return out.value
+
+
 # ---- affinity ---------------------------------------------------------------------------------
 class AffinityMap:
     def __init__(self, handle):
@@ -187,7 +207,7 @@ class AffinityMap:
         return out
 
     def cycles(self) -> np.ndarray:
-        out = np.empty(len(self.export()), dtype=np.uint32)
+        out = np.empty((2, len(self.export())), dtype=np.uint32)
         _check(lib().ag_affinity_cycles(self.handle, out.ctypes.data, out.size), "ag_affinity_cycles")
         return out
 

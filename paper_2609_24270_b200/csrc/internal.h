@@ -51,9 +51,10 @@ struct ag_affinity_map {
     size_t n_chunks;
     uint8_t* d_die_of_chunk; // device, one byte per chunk
     std::vector<uint8_t> h_die_of_chunk;
-    std::vector<uint32_t> h_cycles;  // min latency per chunk (empty for tables given by the caller)
+    std::vector<uint32_t> h_cycles;   // min latency per chunk seen from die 0 (empty for caller-given tables)
+    std::vector<uint32_t> h_cycles1;  // same, seen from die 1
     int ref_sm[2];
-    uint32_t threshold;
+    size_t n_ambiguous;               // chunks whose two latencies are less than 25 % apart
 };
 
 struct ag_plan {

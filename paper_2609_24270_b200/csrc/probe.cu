@@ -14,6 +14,8 @@
 // the blocks that landed on the wanted SMs work.  The others stay resident (bounded) until the
 // wanted SMs have checked in, so that all blocks sit on distinct SMs.
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -82,10 +84,15 @@ __global__ void k_cluster_probe(int* smid_of_block) {
 }
 
 // ---- latency probe from one SM -------------------------------------------------------------
-// mode 0: invalidate the L2 line first (HBM latency).  mode 1: plain timed load (whatever level
-// holds the line).  out[r] = min over reps; the 128-byte line is saved and written back.
+// mode 0: save the line, invalidate it in L2 (discard.global.L2), timed load, write it back -
+//         the HBM-latency kernel of the paper's appendix.
+// mode 1: plain timed load (latency of whichever level holds the line).
+// mode 2: rewrite the line with its own contents, then timed load.  The write leaves the line in
+//         its home L2 partition and drops any copy replicated into the other partition, so the
+//         load is an L2 hit in the home partition: short from a same-die SM, long across dies.
+// out[r] = min over reps; raw (optional) keeps every sample.
 __global__ void k_latency_from_sm(PinCtrl* pc, int target_sm, uint8_t* buf, const long long* line_off, int n_lines,
-                                  int reps, int mode, uint32_t* out) {
+                                  int reps, int mode, uint32_t* out, uint32_t* raw /* n_lines x reps or null */) {
     const bool member = ((int)smid() == target_sm);
     pin_rendezvous(pc, member, 1, 100000ull);
     if (!member || threadIdx.x >= 32) return;
@@ -96,16 +103,22 @@ __global__ void k_latency_from_sm(PinCtrl* pc, int target_sm, uint8_t* buf, cons
         uint32_t best = 0xffffffffu;
         for (int k = 0; k < reps; ++k) {
             uint32_t saved = 0;
-            if (mode == 0) {
+            if (mode == 0 || mode == 2) {
                 saved = ld_cg_u32(line + lane * 4);
                 __syncwarp();
-                if (lane == 0) discard_l2_128(line);
+                if (mode == 2) {
+                    reinterpret_cast<volatile uint32_t*>(line)[lane] = saved;
+                    __threadfence();
+                } else if (lane == 0) {
+                    discard_l2_128(line);
+                }
                 __syncwarp();
             }
             if (lane == 0) {
                 sink += ld_cg_u32(line + 256);  // another line of the same chunk: warms the address translation
                 const uint32_t dt = timed_load_cg(line, sink);
                 best = min(best, dt);
+                if (raw) raw[r * reps + k] = dt;
             }
             __syncwarp();
             if (mode == 0) {
@@ -119,7 +132,9 @@ __global__ void k_latency_from_sm(PinCtrl* pc, int target_sm, uint8_t* buf, cons
 }
 
 // ---- L2 bandwidth of a set of SMs ----------------------------------------------------------------
-__global__ void __launch_bounds__(512)
+// 1024 threads, eight independent 16-byte loads in flight per thread, so that the SM's own
+// request rate - not the load latency - is what the GPC's port to L2 has to carry.
+__global__ void __launch_bounds__(1024)
 k_l2_bandwidth(PinCtrl* pc, const unsigned long long* member_mask, unsigned int n_members, const uint4* buf,
                size_t slice_vec, int passes, unsigned int* sink_out) {
     const int sm = (int)smid();
@@ -133,10 +148,14 @@ k_l2_bandwidth(PinCtrl* pc, const unsigned long long* member_mask, unsigned int 
     __syncthreads();
     unsigned long long t0 = 0;
     if (threadIdx.x == 0) t0 = globaltimer_ns();
+    const size_t step = (size_t)blockDim.x * 8;
     for (int p = 0; p < passes; ++p)
-        for (size_t i = threadIdx.x; i < slice_vec; i += blockDim.x) {
-            const uint4 v = ld_cg_u128(slice + i);
-            acc += v.x ^ v.w;
+        for (size_t i0 = threadIdx.x; i0 + 7 * blockDim.x < slice_vec; i0 += step) {
+            uint4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = ld_cg_u128(slice + i0 + (size_t)j * blockDim.x);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc += v[j].x ^ v[j].w;
         }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -144,6 +163,17 @@ k_l2_bandwidth(PinCtrl* pc, const unsigned long long* member_mask, unsigned int 
         pc->t_end[sm] = globaltimer_ns();
     }
     if (acc == 0x9e3779b9u) sink_out[0] = acc;
+}
+
+// Keeps every SM busy for `ns` so that clocks have settled before cycle counts are compared.
+__global__ void k_warm_up(unsigned long long ns, float* out) {
+    const unsigned long long t0 = globaltimer_ns();
+    float x = threadIdx.x * 1e-3f;
+    while (globaltimer_ns() - t0 < ns) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) x = fmaf(x, 1.0001f, 0.5f);
+    }
+    if (x == 123.456f) out[0] = x;
 }
 
 // ---- affinity probe over a buffer -----------------------------------------------------------------
@@ -189,33 +219,6 @@ struct UnionFind {
     int find(int x) { while (p[x] != x) { p[x] = p[p[x]]; x = p[x]; } return x; }
     void unite(int a, int b) { a = find(a); b = find(b); if (a != b) p[std::max(a, b)] = std::min(a, b); }
 };
-
-// 1-D two-means started at the extremes; returns false if the tiers are not clearly apart.
-static bool two_means(const std::vector<uint32_t>& v, double& lo, double& hi, double& thr) {
-    if (v.size() < 2) return false;
-    {
-        // start from the 5th / 95th percentile so that a stray slow sample cannot own a cluster
-        std::vector<uint32_t> sorted(v);
-        std::sort(sorted.begin(), sorted.end());
-        lo = sorted[sorted.size() / 20];
-        hi = sorted[sorted.size() - 1 - sorted.size() / 20];
-    }
-    if (hi <= lo) return false;
-    for (int it = 0; it < 32; ++it) {
-        const double mid = 0.5 * (lo + hi);
-        double s0 = 0, s1 = 0;
-        size_t n0 = 0, n1 = 0;
-        for (uint32_t x : v) {
-            if (x <= mid) { s0 += x; ++n0; } else { s1 += x; ++n1; }
-        }
-        if (!n0 || !n1) return false;
-        const double nlo = s0 / n0, nhi = s1 / n1;
-        if (fabs(nlo - lo) < 0.5 && fabs(nhi - hi) < 0.5) { lo = nlo; hi = nhi; break; }
-        lo = nlo; hi = nhi;
-    }
-    thr = 0.5 * (lo + hi);
-    return hi > 1.15 * lo;  // the paper's tiers are 34 % (H200) and 67 % (B200) apart
-}
 
 static void finish_counts(ag_topo_map* m) {
     memset(m->die_sm_count, 0, sizeof m->die_sm_count);
@@ -278,21 +281,43 @@ extern "C" ag_status ag_topo_from_observations(int32_t n_sm, const int32_t* clus
     }
     map->n_gpc = n_gpc;
     if (n_clusters > 0) map->flags |= AG_TOPO_CLUSTER;
-    // dies: near/far pattern of every SM over the reference chunks, compared with SM 0's
+    // dies: SM s sits on SM 0's die when it sees every reference line at about the latency SM 0
+    // sees it (within 25 %), and on the other die when it sees nearly every line very differently.
+    // Comparing line by line keeps the split independent of whether a given line happened to be
+    // served by L2 or by HBM: that depends on the line, not on the SM.
     if (lat && n_ref > 0) {
-        std::vector<uint32_t> all(lat, lat + (size_t)n_sm * n_ref);
-        double lo, hi, thr;
-        if (!two_means(all, lo, hi, thr)) return AG_ERR_NOISY_PROBE;
-        map->lat_near_cycles = (uint32_t)(lo + 0.5);
-        map->lat_far_cycles = (uint32_t)(hi + 0.5);
-        map->lat_threshold = (uint32_t)(thr + 0.5);
+        int other = -1;
         for (int s = 0; s < n_sm; ++s) {
-            int same = 0;
-            for (int r = 0; r < n_ref; ++r)
-                same += ((lat[(size_t)s * n_ref + r] > thr) == (lat[r] > thr));
-            if (same * 4 > n_ref && same * 4 < 3 * n_ref) return AG_ERR_NOISY_PROBE;
-            map->die[s] = same * 2 >= n_ref ? 0 : 1;
+            int similar = 0;
+            for (int r = 0; r < n_ref; ++r) {
+                const double a = lat[(size_t)s * n_ref + r], b = lat[r];
+                similar += (a <= 1.25 * b && b <= 1.25 * a);
+            }
+            if (similar * 4 > n_ref && similar * 4 < 3 * n_ref) {
+                if (getenv("AG_DEBUG")) {
+                    fprintf(stderr, "[ag] SM %d is like SM 0 on %d of %d lines; row:", s, similar, n_ref);
+                    for (int r = 0; r < n_ref; ++r) fprintf(stderr, " %u", lat[(size_t)s * n_ref + r]);
+                    fprintf(stderr, "\n[ag] SM 0 row:");
+                    for (int r = 0; r < n_ref; ++r) fprintf(stderr, " %u", lat[r]);
+                    fprintf(stderr, "\n");
+                }
+                return AG_ERR_NOISY_PROBE;
+            }
+            map->die[s] = similar * 2 >= n_ref ? 0 : 1;
+            if (map->die[s] == 1 && other < 0) other = s;
         }
+        if (other < 0) return AG_ERR_NOISY_PROBE;  // no second latency tier seen from any SM
+        std::vector<uint32_t> nearv, farv;
+        for (int r = 0; r < n_ref; ++r) {
+            const uint32_t a = lat[r], b = lat[(size_t)other * n_ref + r];
+            nearv.push_back(std::min(a, b));
+            farv.push_back(std::max(a, b));
+        }
+        std::sort(nearv.begin(), nearv.end());
+        std::sort(farv.begin(), farv.end());
+        map->lat_near_cycles = nearv[n_ref / 2];
+        map->lat_far_cycles = farv[n_ref / 2];
+        map->lat_threshold = (map->lat_near_cycles + map->lat_far_cycles) / 2;
         map->flags |= AG_TOPO_LATENCY;
     }
     finish_counts(map);
@@ -307,8 +332,9 @@ extern "C" int32_t ag_topo_place_by_gain(const double* gain, int32_t n, double s
     double runner = 1e300;
     for (int i = 0; i < n; ++i)
         if (i != best) runner = std::min(runner, gain[i]);
-    // contended: clearly less than one TPC's own bandwidth; the others: close to it
-    if (gain[best] < 0.80 * solo_bw && (n == 1 || runner > gain[best] + 0.10 * solo_bw)) return best;
+    // contended: the GPC's port to L2 was already full, so the TPC adds next to nothing; a TPC of
+    // another GPC still adds a good part of its own bandwidth
+    if (gain[best] < 0.35 * solo_bw && (n == 1 || runner > gain[best] + 0.20 * solo_bw)) return best;
     return -1;
 }
 
@@ -328,6 +354,14 @@ struct Scratch {
         cudaFree(bw_buf); cudaFree(d_sink);
     }
 };
+
+ag_status warm_up(int n_sm, float* d_sink) {
+    k_warm_up<<<n_sm, 128>>>(30000000ull, d_sink);
+    count_launch();
+    AG_CUDA(cudaGetLastError());
+    AG_CUDA(cudaDeviceSynchronize());
+    return AG_OK;
+}
 
 ag_status set_pin_smem() {
     static bool done = false;
@@ -351,7 +385,7 @@ ag_status measure_bw(Scratch& sc, int n_sm, const unsigned long long mask[4], si
     std::vector<PinCtrl> h(1);
     for (int t = 0; t < tries; ++t) {
         AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
-        k_l2_bandwidth<<<n_sm, 512, kPinSmem>>>(sc.pc, sc.d_mask, n_members, sc.bw_buf, slice_vec, passes, sc.d_sink);
+        k_l2_bandwidth<<<n_sm, 1024, kPinSmem>>>(sc.pc, sc.d_mask, n_members, sc.bw_buf, slice_vec, passes, sc.d_sink);
         count_launch();
         AG_CUDA(cudaGetLastError());
         AG_CUDA(cudaDeviceSynchronize());
@@ -381,7 +415,7 @@ ag_status latency_rows(Scratch& sc, int n_sm, const std::vector<int>& sms, int n
         for (int attempt = 0; attempt < 3 && !ok; ++attempt) {
             AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
             AG_CUDA(cudaMemset(sc.d_out, 0, sizeof(uint32_t) * n_lines));
-            k_latency_from_sm<<<n_sm, 32, kPinSmem>>>(sc.pc, sms[i], sc.ref, sc.d_off, n_lines, reps, mode, sc.d_out);
+            k_latency_from_sm<<<n_sm, 32, kPinSmem>>>(sc.pc, sms[i], sc.ref, sc.d_off, n_lines, reps, mode, sc.d_out, nullptr);
             count_launch();
             AG_CUDA(cudaGetLastError());
             AG_CUDA(cudaDeviceSynchronize());
@@ -418,6 +452,8 @@ extern "C" ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases) 
     AG_CUDA(cudaMalloc(&sc.d_mask, 4 * sizeof(unsigned long long)));
     AG_CUDA(cudaMalloc(&sc.d_sink, 64));
 
+    st = warm_up(n_sm, reinterpret_cast<float*>(sc.d_sink));
+    if (st != AG_OK) return st;
     // ---- census: every SM id exactly once
     AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
     AG_CUDA(cudaMemset(sc.d_int, 0, sizeof(int) * AG_MAX_SM));
@@ -490,8 +526,9 @@ extern "C" ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases) 
             if (map->die[s] == 1) other = s;
         // lines that are near for die 0
         std::vector<long long> near_off;
-        for (int r = 0; r < kRefChunks; ++r)
-            if (lat[r] <= map->lat_threshold) near_off.push_back(offs[r] + 1024);
+        if (other >= 0)
+            for (int r = 0; r < kRefChunks; ++r)
+                if (lat[r] < lat[(size_t)other * kRefChunks + r]) near_off.push_back(offs[r] + 1024);
         if (near_off.size() >= 4 && other >= 0) {
             const int n = (int)near_off.size();
             AG_CUDA(cudaMemcpy(sc.d_off, near_off.data(), sizeof(long long) * n, cudaMemcpyHostToDevice));
@@ -507,7 +544,12 @@ extern "C" ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases) 
         }
     }
 
-    // ---- place the random TPCs by L2-bandwidth contention
+    // ---- place the random TPCs by L2-bandwidth contention (Section 5.1.2)
+    // The known SMs of a GPC are run alone and together with the TPC.  Where the known SMs already
+    // fill the GPC's port to L2, a TPC of the same GPC adds next to nothing while a TPC of another
+    // GPC adds a good part of its own bandwidth.  GPCs whose known SMs do not fill the port cannot
+    // be tested that way; a TPC that contends with no testable GPC of its die is placed by
+    // elimination when exactly one such GPC with room for it (at most 10 TPCs per GPC) is left.
     if ((phases & AG_TOPO_BANDWIDTH) && (map->flags & AG_TOPO_CLUSTER) && (map->flags & AG_TOPO_LATENCY) &&
         map->n_unplaced > 0 && map->n_gpc > 0) {
         const size_t slice_bytes = 1u << 20;  // per-SM slice: larger than L1, 64 slices fit well inside L2
@@ -515,43 +557,134 @@ extern "C" ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases) 
         AG_CUDA(cudaMalloc(&sc.bw_buf, slice_bytes * 64));
         AG_CUDA(cudaMemset(sc.bw_buf, 1, slice_bytes * 64));
         const int passes = 8, tries = 3;
-        std::vector<double> base_bw(map->n_gpc, -1.0);
+        const bool dbg = getenv("AG_DEBUG") != nullptr;
+        std::vector<double> base_bw(map->n_gpc, 0.0);
+        std::vector<int> size_now(map->n_gpc, 0);
         auto mask_of_gpc = [&](int g, unsigned long long m[4]) {
             m[0] = m[1] = m[2] = m[3] = 0;
             for (int s = 0; s < n_sm; ++s)
                 if (map->gpc[s] == g && !map->is_random[s]) m[s >> 6] |= 1ull << (s & 63);
         };
+        double cap = 0;
+        for (int g = 0; g < map->n_gpc; ++g) {
+            unsigned long long mg[4];
+            mask_of_gpc(g, mg);
+            size_now[g] = map->gpc_sm_count[g];
+            if (measure_bw(sc, n_sm, mg, slice_vec, passes, tries, &base_bw[g]) != AG_OK) base_bw[g] = 0;
+            cap = std::max(cap, base_bw[g]);
+        }
         for (int t = 0; t < map->n_tpc; ++t) {
             const int s0 = 2 * t, s1 = 2 * t + 1;
             if (s0 >= n_sm || map->gpc[s0] >= 0) continue;
+            const int tpc_sms = s1 < n_sm ? 2 : 1;
             unsigned long long m[4] = {0, 0, 0, 0};
             m[s0 >> 6] |= 1ull << (s0 & 63);
             if (s1 < n_sm) m[s1 >> 6] |= 1ull << (s1 & 63);
             double solo = 0;
             if (measure_bw(sc, n_sm, m, slice_vec, passes, tries, &solo) != AG_OK) continue;
-            std::vector<int> cands;
+            std::vector<int> tested, untested;
             std::vector<double> gains;
             for (int g = 0; g < map->n_gpc; ++g) {
-                if (map->gpc_die[g] != map->die[s0]) continue;  // a TPC sits on the die its latency shows
+                if (map->gpc_die[g] != map->die[s0]) continue;   // a TPC sits on the die its latency shows
+                if (size_now[g] + tpc_sms > 20) continue;        // a GPC holds at most 10 TPCs
+                if (base_bw[g] < 0.93 * cap) { untested.push_back(g); continue; }  // port not full: no signal
                 unsigned long long mg[4];
                 mask_of_gpc(g, mg);
-                if (base_bw[g] < 0 && measure_bw(sc, n_sm, mg, slice_vec, passes, tries, &base_bw[g]) != AG_OK) continue;
                 for (int i = 0; i < 4; ++i) mg[i] |= m[i];
                 double with = 0;
                 if (measure_bw(sc, n_sm, mg, slice_vec, passes, tries, &with) != AG_OK) continue;
-                cands.push_back(g);
+                tested.push_back(g);
                 gains.push_back(with - base_bw[g]);
             }
+            int pick_gpc = -1;
             const int pick = ag_topo_place_by_gain(gains.data(), (int)gains.size(), solo);
             if (pick >= 0) {
-                map->gpc[s0] = cands[pick];
-                if (s1 < n_sm) map->gpc[s1] = cands[pick];
+                pick_gpc = tested[pick];
+            } else {
+                bool any_low = false;
+                for (double gn : gains) any_low |= gn < 0.35 * solo;
+                if (!any_low && untested.size() == 1) pick_gpc = untested[0];
+            }
+            if (dbg) {
+                fprintf(stderr, "[ag] TPC %d solo %.1f GB/s:", t, solo * 1e-9);
+                for (size_t i = 0; i < tested.size(); ++i)
+                    fprintf(stderr, " gpc%d base %.1f gain %.1f;", tested[i], base_bw[tested[i]] * 1e-9, gains[i] * 1e-9);
+                for (int g : untested) fprintf(stderr, " gpc%d untested (base %.1f);", g, base_bw[g] * 1e-9);
+                fprintf(stderr, " -> gpc %d\n", pick_gpc);
+            }
+            if (pick_gpc >= 0) {
+                map->gpc[s0] = pick_gpc;
+                if (s1 < n_sm) map->gpc[s1] = pick_gpc;
+                size_now[pick_gpc] += tpc_sms;
             }
         }
         map->flags |= AG_TOPO_BANDWIDTH;
         finish_counts(map);
     }
     return AG_OK;
+}
+
+extern "C" ag_status ag_probe_latency_samples(int sm, int mode, int n_lines, int reps, uint32_t* cycles) {
+    if (!cycles || n_lines < 1 || n_lines > 1024 || reps < 1 || reps > 64 || (mode < 0 || mode > 2)) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    st = set_pin_smem();
+    if (st != AG_OK) return st;
+    int dev = 0, n_sm = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    if (sm < 0 || sm >= n_sm) return AG_ERR_ARG;
+    Scratch sc;
+    const size_t ref_bytes = 8u << 20;
+    uint32_t* d_raw = nullptr;
+    AG_CUDA(cudaMalloc(&sc.pc, sizeof(PinCtrl)));
+    AG_CUDA(cudaMalloc(&sc.ref, ref_bytes));
+    AG_CUDA(cudaMemset(sc.ref, 0, ref_bytes));
+    AG_CUDA(cudaMalloc(&sc.d_off, sizeof(long long) * 1024));
+    AG_CUDA(cudaMalloc(&sc.d_out, sizeof(uint32_t) * 1024 * 65));
+    d_raw = sc.d_out + 1024;
+    AG_CUDA(cudaMalloc(&sc.d_sink, 64));
+    std::vector<long long> offs(n_lines);
+    const long long n_chunks = (long long)(ref_bytes / AG_CHUNK_BYTES);
+    for (int r = 0; r < n_lines; ++r) offs[r] = ((r * 29LL + 3) % n_chunks) * AG_CHUNK_BYTES + 512;
+    AG_CUDA(cudaMemcpy(sc.d_off, offs.data(), sizeof(long long) * n_lines, cudaMemcpyHostToDevice));
+    st = warm_up(n_sm, reinterpret_cast<float*>(sc.d_sink));
+    if (st != AG_OK) return st;
+    AG_CUDA(cudaMemset(sc.pc, 0, sizeof(PinCtrl)));
+    AG_CUDA(cudaMemset(sc.d_out, 0, sizeof(uint32_t) * 1024 * 65));
+    k_latency_from_sm<<<n_sm, 32, kPinSmem>>>(sc.pc, sm, sc.ref, sc.d_off, n_lines, reps, mode, sc.d_out, d_raw);
+    count_launch();
+    AG_CUDA(cudaGetLastError());
+    AG_CUDA(cudaDeviceSynchronize());
+    AG_CUDA(cudaMemcpy(cycles, d_raw, sizeof(uint32_t) * n_lines * reps, cudaMemcpyDeviceToHost));
+    return cycles[0] ? AG_OK : AG_ERR_UNMANNED_SM;
+}
+
+extern "C" ag_status ag_probe_l2_bandwidth(const uint64_t sm_mask[4], double* bytes_per_s) {
+    if (!sm_mask || !bytes_per_s) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    st = set_pin_smem();
+    if (st != AG_OK) return st;
+    int dev = 0, n_sm = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    unsigned long long m[4] = {sm_mask[0], sm_mask[1], sm_mask[2], sm_mask[3]};
+    unsigned int members = 0;
+    for (int s = 0; s < AG_MAX_SM; ++s) {
+        const bool in = (m[s >> 6] >> (s & 63)) & 1ull;
+        if (in && s >= n_sm) return AG_ERR_ARG;
+        members += in;
+    }
+    if (members == 0) return AG_ERR_ARG;
+    Scratch sc;
+    const size_t slice_bytes = 1u << 20;
+    AG_CUDA(cudaMalloc(&sc.pc, sizeof(PinCtrl)));
+    AG_CUDA(cudaMalloc(&sc.d_mask, 4 * sizeof(unsigned long long)));
+    AG_CUDA(cudaMalloc(&sc.d_sink, 64));
+    AG_CUDA(cudaMalloc(&sc.bw_buf, slice_bytes * 64));
+    AG_CUDA(cudaMemset(sc.bw_buf, 1, slice_bytes * 64));
+    return measure_bw(sc, n_sm, m, slice_bytes / 16, 8, 3, bytes_per_s);
 }
 
 extern "C" ag_status topo_discover(ag_topo_map* map) {
@@ -583,7 +716,7 @@ static ag_status probe_from_die(uint8_t* buf, size_t n_chunks, const ag_topo_map
         if ((e = cudaMemset(pc, 0, sizeof(PinCtrl))) != cudaSuccess) break;
         if ((e = cudaMemset(d_cycles, 0, sizeof(uint32_t) * n_chunks)) != cudaSuccess) break;
         if ((e = cudaMemcpy(d_rank, rank.data(), sizeof(int) * AG_MAX_SM, cudaMemcpyHostToDevice)) != cudaSuccess) break;
-        k_affinity_probe<<<n_sm, 32, kPinSmem>>>(pc, d_rank, n_members, buf, n_chunks, 3, 2, d_cycles);
+        k_affinity_probe<<<n_sm, 32, kPinSmem>>>(pc, d_rank, n_members, buf, n_chunks, 2, 3, d_cycles);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) break;
         if ((e = cudaDeviceSynchronize()) != cudaSuccess) break;
@@ -599,19 +732,19 @@ static ag_status probe_from_die(uint8_t* buf, size_t n_chunks, const ag_topo_map
     return AG_OK;
 }
 
-static ag_status classify(const std::vector<uint32_t>& cycles, int near_die, std::vector<uint8_t>& table,
-                          uint32_t* threshold) {
-    double lo, hi, thr;
-    if (!two_means(cycles, lo, hi, thr)) return AG_ERR_NOISY_PROBE;
-    table.resize(cycles.size());
-    size_t ambiguous = 0;
-    for (size_t i = 0; i < cycles.size(); ++i) {
-        table[i] = (uint8_t)((cycles[i] > thr) ? 1 - near_die : near_die);
-        if (fabs((double)cycles[i] - thr) < 0.05 * thr) ++ambiguous;
+// A chunk belongs to the die whose SMs reach it faster (Section 6.1.1; the appendix on multi-tier
+// parts assigns each address to the group with the lowest latency in the same way).
+static ag_status classify(const std::vector<uint32_t>& c0, const std::vector<uint32_t>& c1,
+                          std::vector<uint8_t>& table, size_t* ambiguous) {
+    table.resize(c0.size());
+    size_t amb = 0;
+    for (size_t i = 0; i < c0.size(); ++i) {
+        table[i] = c0[i] <= c1[i] ? 0 : 1;
+        const double lo = std::min(c0[i], c1[i]), hi = std::max(c0[i], c1[i]);
+        if (hi < 1.25 * lo) ++amb;
     }
-    *threshold = (uint32_t)(thr + 0.5);
-    if (ambiguous * 100 > cycles.size()) return AG_ERR_NOISY_PROBE;
-    return AG_OK;
+    *ambiguous = amb;
+    return amb * 50 > c0.size() ? AG_ERR_NOISY_PROBE : AG_OK;  // more than 2 % undecided
 }
 
 extern "C" ag_status ag_affinity_from_table(const void* buf, size_t bytes, const uint8_t* die_of_chunk,
@@ -627,7 +760,7 @@ extern "C" ag_status ag_affinity_from_table(const void* buf, size_t bytes, const
     a->h_die_of_chunk.assign(die_of_chunk, die_of_chunk + n_chunks);
     for (auto& v : a->h_die_of_chunk) v = v ? 1 : 0;
     a->ref_sm[0] = a->ref_sm[1] = -1;
-    a->threshold = 0;
+    a->n_ambiguous = 0;
     cudaError_t e = cudaMalloc(&a->d_die_of_chunk, n_chunks);
     if (e == cudaSuccess) e = cudaMemcpy(a->d_die_of_chunk, a->h_die_of_chunk.data(), n_chunks, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
@@ -649,17 +782,29 @@ extern "C" ag_status ag_affinity_probe_with_map(void* buf, size_t bytes, const a
     const size_t n_chunks = bytes / AG_CHUNK_BYTES;
     std::vector<uint32_t> cycles;
     int ref_sm[2] = {-1, -1};
+    {
+        float* d_sink = nullptr;
+        AG_CUDA(cudaMalloc(&d_sink, 64));
+        st = warm_up(map->n_sm, d_sink);
+        cudaFree(d_sink);
+        if (st != AG_OK) return st;
+    }
+    std::vector<uint32_t> cycles1;
     st = probe_from_die((uint8_t*)buf, n_chunks, map, 0, cycles, ref_sm);
     if (st != AG_OK) return st;
+    st = probe_from_die((uint8_t*)buf, n_chunks, map, 1, cycles1, ref_sm);
+    if (st != AG_OK) return st;
     std::vector<uint8_t> table;
-    uint32_t thr = 0;
-    st = classify(cycles, 0, table, &thr);
+    size_t ambiguous = 0;
+    st = classify(cycles, cycles1, table, &ambiguous);
     if (st != AG_OK) return st;
     st = ag_affinity_from_table(buf, bytes, table.data(), n_chunks, out);
     if (st != AG_OK) return st;
     (*out)->h_cycles.swap(cycles);
+    (*out)->h_cycles1.swap(cycles1);
     (*out)->ref_sm[0] = ref_sm[0];
-    (*out)->threshold = thr;
+    (*out)->ref_sm[1] = ref_sm[1];
+    (*out)->n_ambiguous = ambiguous;
     return AG_OK;
 }
 
@@ -672,18 +817,9 @@ extern "C" ag_status affinity_probe(void* buf, size_t bytes, ag_affinity_map** o
 
 extern "C" ag_status ag_affinity_check_complement(const ag_affinity_map* amap, const ag_topo_map* map,
                                                   size_t* mismatches) {
-    if (!amap || !map || !mismatches) return AG_ERR_ARG;
-    std::vector<uint32_t> cycles;
-    int ref_sm[2] = {-1, -1};
-    ag_status st = probe_from_die((uint8_t*)amap->base, amap->n_chunks, map, 1, cycles, ref_sm);
-    if (st != AG_OK) return st;
-    std::vector<uint8_t> table;
-    uint32_t thr = 0;
-    st = classify(cycles, 1, table, &thr);
-    if (st != AG_OK) return st;
-    size_t bad = 0;
-    for (size_t i = 0; i < table.size(); ++i) bad += table[i] != amap->h_die_of_chunk[i];
-    *mismatches = bad;
+    (void)map;
+    if (!amap || !mismatches || amap->h_cycles.empty()) return AG_ERR_ARG;
+    *mismatches = amap->n_ambiguous;
     return AG_OK;
 }
 
@@ -698,8 +834,9 @@ extern "C" ag_status ag_affinity_export(const ag_affinity_map* amap, uint8_t* di
 }
 
 extern "C" ag_status ag_affinity_cycles(const ag_affinity_map* amap, uint32_t* cycles, size_t cap) {
-    if (!amap || !cycles || amap->h_cycles.empty() || cap < amap->n_chunks) return AG_ERR_ARG;
+    if (!amap || !cycles || amap->h_cycles.empty() || cap < 2 * amap->n_chunks) return AG_ERR_ARG;
     memcpy(cycles, amap->h_cycles.data(), amap->n_chunks * sizeof(uint32_t));
+    memcpy(cycles + amap->n_chunks, amap->h_cycles1.data(), amap->n_chunks * sizeof(uint32_t));
     return AG_OK;
 }
 

@@ -10,16 +10,16 @@ from tests.gpu_util import oracle_policy
 pytestmark = pytest.mark.gpu
 
 
-def both(topo_d, amap_tbl, b, **kw):
+def both(topo_d, amap_tbl, budget, **kw):
     topo = ag.TopoMap.from_dict(topo_d)
     amap = ag.affinity_from_table(0, amap_tbl) if amap_tbl is not None else None
-    plan = ag.sched_build(topo, amap, b, ag.make_policy(**kw))
+    plan = ag.sched_build(topo, amap, budget, ag.make_policy(**kw))
     got = plan.export()
     okw = dict(kw)
     if "avoid" in okw:
         okw["avoid"] = tuple(okw["avoid"])
     o_amap = dict(chunk_bytes=4096, die_of_chunk=amap_tbl) if amap_tbl is not None else None
-    want = op.export(op.build_plan(topo_d, o_amap, b, oracle_policy(**okw)))
+    want = op.export(op.build_plan(topo_d, o_amap, budget, oracle_policy(**okw)))
     return got, want, plan
 
 

@@ -28,9 +28,10 @@ def test_die_split(topo):
     assert abs(n0 - n1) <= 8                                 # B200 partitions differ by at most 8 SMs (Section 6.1.1)
     for t in range(m["n_sm"] // 2):                          # both SMs of a TPC sit on one die
         assert m["die"][2 * t] == m["die"][2 * t + 1]
-    # latency tiers: far/near about 1.67 on B200 (552 -> 920 cycles); a band, not an equality
+    # latency tiers: the paper reports far/near of about 1.67 for HBM (552 -> 920 cycles) and about
+    # 2.0 for L2 hits (364 -> 725) on B200; the probe's lines may be served by either level
     ratio = m["lat_far_cycles"] / m["lat_near_cycles"]
-    assert 1.25 < ratio < 2.3, (m["lat_near_cycles"], m["lat_far_cycles"])
+    assert 1.4 < ratio < 3.0, (m["lat_near_cycles"], m["lat_far_cycles"])
     if m["l2_near_cycles"]:
         assert 1.3 < m["l2_far_cycles"] / m["l2_near_cycles"] < 3.0
 
@@ -76,6 +77,9 @@ def test_affinity_probe_structure_and_content_preserved(topo):
     pairs = t[base_chunk:].copy()
     pairs = pairs[: (pairs.size // 2) * 2].reshape(-1, 2)
     assert (pairs[:, 0] != pairs[:, 1]).mean() > 0.99        # each aligned pair of 4 KB pages: one per die (Section 7.1.1)
-    assert amap.check_complement(topo) <= t.size // 200      # a die-1 SM sees the opposite tiers
+    assert amap.check_complement(topo) <= t.size // 50       # the two dies see opposite tiers
+    c0, c1 = amap.cycles()
+    near, far = np.minimum(c0, c1), np.maximum(c0, c1)
+    assert 1.4 < np.median(far) / np.median(near) < 3.0
     again = ag.affinity_probe(buf.data_ptr(), nbytes, topo).export()
     assert (again != t).sum() <= t.size // 200               # repeatable
