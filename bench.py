@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the asymmetry-aware persistent BF16 GEMM (one JSON line on stdout).
+
+Workload: dense C = A.B with M = N = K = 8192, bf16 inputs uniform in [-1, 1) from a seed, fp32
+accumulate and output, 128 x 256 output tiles on all SMs - the configuration the headline metric
+is quoted on.  A step is one gemm_persistent call under the affinity plan (topology discovery,
+affinity probing and plan building are one-off set-up and are timed separately in `setup_s`).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (launched by torchrun) every rank runs an independent replica on its own GPU with its
+own maps and plans - the path has no exchange step - and the whole-job value is the sum.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+M = N = K = 8192
+TILE_M, TILE_N = 128, 256
+RASTER_GROUP = 16
+# affinity margins below 1/8 of a unit's bytes (A panel + B panel + C tile) are treated as ties: with plain
+# row-major operands every unit is interleaved about half and half over the dies
+MIN_MARGIN = (TILE_M * K * 2 + TILE_N * K * 2 + TILE_M * TILE_N * 4) // 8
+FLOPS = 2.0 * M * N * K
+METRIC = "bf16_gemm_tflops"
+UNIT = "TFLOP/s"
+# DRAM bytes per launch of the dominant kernel, from the ncu capture summarised in
+# profiles/gemm_persistent_8192.md (dram__bytes_read.sum 1.191 GB + dram__bytes_write.sum 0.255 GB).
+NCU_TRAFFIC_BYTES = 1.446e9
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(bf16_tflops=d["bf16_tflops"], bf16_tflops_sustained=d.get("bf16_tflops_sustained"),
+                    hbm_gbs=d["hbm_gbs"], source="measured")
+    return dict(bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, hbm_gbs=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [f.strip() for f in line.split(",")]))
+
+    def mark(self):
+        """Start of the timed region: only samples taken after this count."""
+        self.t_mark = time.time()
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        t_end = time.time()
+        time.sleep(0.1)
+        self.proc.terminate()
+        mhz, mx, reasons = [], None, set()
+        for t, r in self.rows:
+            if t < getattr(self, "t_mark", 0.0) or t > t_end + 0.05:
+                continue
+            try:
+                mhz.append(float(r[0]))
+                mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+def oracle_sample(A, B, rows=None, cols=N, target_s=15.0):
+    """The fp64 oracle, as it stands, on a bounded block (the first `rows` rows of C) of the same
+    workload.  With rows=None a 64-row probe sets the row count so that the run takes about target_s."""
+    from oracle import gemm as og
+    if rows is None:
+        t0 = time.time()
+        og.gemm_block(A, B, 0, 64, 0, cols)
+        rate = 64 / max(time.time() - t0, 1e-3)
+        rows = int(min(M, max(64, (rate * target_s) // 64 * 64)))
+    t0 = time.time()
+    blk = og.gemm_block(A, B, 0, rows, 0, cols)
+    dt = time.time() - t0
+    return blk, dt, 2.0 * rows * cols * K, og.num_threads()
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2609_24270_b200 import inputs
+    A, B = inputs.gemm_inputs(M, N, K)
+    rows, cols = 64, N
+    for _ in range(args.warmup):
+        oracle_sample(A, B, 8, 1024)
+    t0 = time.time()
+    cores = 1
+    for _ in range(args.steps):
+        _, _, fl, cores = oracle_sample(A, B, rows, cols)
+        if time.time() - t0 > 240:      # keep the whole run within a few minutes whatever K is
+            break
+    dt = (time.time() - t0) / args.steps
+    val = fl / dt / 1e12
+    sample = f"rows 0..{rows} x cols 0..{cols} of C per step ({fl / 1e9:.1f} GFLOP of the {FLOPS / 1e12:.2f} TFLOP problem)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"dense GEMM M=N=K={M}, bf16 uniform[-1,1) seeded, fp32 out", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_24270_b200 import binding as ag
+    from paper_2609_24270_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+
+    # ---- inputs: one buffer holds A, B and C so that one affinity map covers all three
+    A_h, B_h = inputs.gemm_inputs(M, N, K)
+    a_bytes, b_bytes, c_bytes = M * K * 2, K * N * 2, M * N * 4
+    buf = torch.empty(a_bytes + b_bytes + c_bytes, dtype=torch.uint8, device="cuda")
+    assert buf.data_ptr() % 4096 == 0
+    a_off, b_off, c_off = 0, a_bytes, a_bytes + b_bytes
+    dA = buf[a_off:a_off + a_bytes].view(torch.int16).view(M, K)
+    dB = buf[b_off:b_off + b_bytes].view(torch.int16).view(K, N)
+    dC = buf[c_off:].view(torch.float32).view(M, N)
+    A_pin = torch.from_numpy(A_h.view(np.int16)).pin_memory()
+    B_pin = torch.from_numpy(B_h.view(np.int16)).pin_memory()
+    C_pin = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    dA.copy_(A_pin)
+    dB.copy_(B_pin)
+    torch.cuda.synchronize()
+
+    # ---- one-off set-up: discover the chip, probe the buffer, build the plans
+    t0 = time.time()
+    topo = ag.topo_discover()
+    t_topo = time.time() - t0
+    t0 = time.time()
+    amap = ag.affinity_probe(buf.data_ptr(), buf.numel(), topo)
+    t_aff = time.time() - t0
+    ops = dict(a=dict(offset=a_off, row_stride=K * 2, elem_bytes=2), b=dict(offset=b_off, row_stride=N * 2, elem_bytes=2),
+               c=dict(offset=c_off, row_stride=N * 4, elem_bytes=4))
+    base = dict(M=M, N=N, K=K, tile_m=TILE_M, tile_n=TILE_N)
+    t0 = time.time()
+    plans = {
+        "oblivious_raster": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, raster_group=1, **base)),
+        "oblivious_grouped": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, raster_group=RASTER_GROUP, **base)),
+        "die_compact": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, raster_group=RASTER_GROUP, **base)),
+        "affinity": ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, raster_group=RASTER_GROUP, min_margin=MIN_MARGIN, **base, **ops)),
+    }
+    t_plan = time.time() - t0
+    stream = torch.cuda.current_stream()
+    pa, pb, pc = dA.data_ptr(), dB.data_ptr(), dC.data_ptr()
+
+    def step(plan):
+        ag.gemm_persistent(pa, pb, pc, M, N, K, plan, stream.cuda_stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(plan, steps, warmup, sampler=None):
+        for _ in range(warmup):
+            step(plan)
+        barrier()
+        if sampler is not None:
+            sampler.mark()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        launches0 = ag.kernel_launch_count()
+        evs[0].record(stream)
+        for i in range(steps):
+            step(plan)
+            evs[i + 1].record(stream)
+        barrier()
+        total_ms = evs[0].elapsed_time(evs[-1])
+        per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+        st = plan.last_status()
+        if st != ag.AG_OK:
+            raise RuntimeError("device status: " + ag.strerror(st))
+        return total_ms, per, ag.kernel_launch_count() - launches0
+
+    # policy comparison: the policies take turns in short rounds so that all of them see the same
+    # power and clock state; the median over each policy's steps is reported
+    names = list(plans)
+    per_policy = {n: [] for n in names}
+    for n in names:
+        for _ in range(args.warmup):
+            step(plans[n])
+    barrier()
+    rounds, per_round = 6, max(2, min(args.steps, 60) // 6)
+    for _ in range(rounds):
+        for n in names:
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(per_round + 1)]
+            evs[0].record(stream)
+            for i in range(per_round):
+                step(plans[n])
+                evs[i + 1].record(stream)
+            torch.cuda.synchronize()
+            per_policy[n] += [evs[i].elapsed_time(evs[i + 1]) for i in range(per_round)]
+    side = {n: FLOPS / (float(np.median(v)) * 1e-3) / 1e12 for n, v in per_policy.items()}
+    sampler = ClockSampler(local)
+    sampler.start()
+    total_ms, per, launches = timed(plans["affinity"], args.steps, args.warmup, sampler)
+    clocks = sampler.stop()
+    ms_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_step], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    value = world * FLOPS / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end through the same call with host buffers: H2D of A and B, GEMM, D2H of C
+    def e2e_step():
+        dA.copy_(A_pin, non_blocking=True)
+        dB.copy_(B_pin, non_blocking=True)
+        step(plans["affinity"])
+        C_pin.copy_(dC, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_val = world * FLOPS / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    kernel_ms = float(np.mean(per))
+    achieved = FLOPS / (kernel_ms * 1e-3) / 1e12
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"dense GEMM M=N=K={M}, A,B bf16 row-major uniform[-1,1) seed {inputs.DEFAULT_SEED}, fp32 out, "
+                               f"{TILE_M}x{TILE_N} tiles, all {topo.n_sm} SMs, affinity policy, raster group {RASTER_GROUP}",
+                   "l2": "inputs+output 512 MiB > 126 MB L2, no flush between iterations",
+                   "replicas": "independent per GPU" if world > 1 else "single GPU"},
+        "policies_tflops": side,
+        "aware_over_oblivious_raster": side["affinity"] / side["oblivious_raster"],
+        "die_sm_count": list(topo.die_sm_count), "gpc_sm_count": list(topo.gpc_sm_count[:topo.n_gpc]),
+        "setup_s": {"topo_discover": t_topo, "affinity_probe": t_aff, "sched_build_x4": t_plan},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": a_bytes + b_bytes, "d2h_bytes_per_step": c_bytes,
+                "ms_per_step": e2e_ms},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES,
+                     "peak_source": f"{peaks['source']} cuBLAS bf16 burst (sustained {peaks['bf16_tflops_sustained']})",
+                     "kernel": "k_gemm_persistent<256>", "kernel_ms": kernel_ms},
+    }
+    if not args.no_cpu_baseline:
+        blk, dt, fl, cores = oracle_sample(A_h, B_h)
+        got = dC[:blk.shape[0], :blk.shape[1]].cpu().numpy().astype(np.float64)
+        out["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": f"rows 0..{blk.shape[0]} x cols 0..{blk.shape[1]} of C ({fl / 1e9:.1f} GFLOP), {dt:.1f} s",
+                               "gpu_max_abs_err_on_sample": float(np.abs(got - blk).max()),
+                               "gpu_rel_fro_err_on_sample": float(np.linalg.norm(got - blk) / np.linalg.norm(blk))}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

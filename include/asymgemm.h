@@ -191,6 +191,7 @@ typedef struct {
     int32_t invert_affinity; /* 1: send every unit to the die that holds fewer of its bytes */
     int32_t static_assign;   /* 1: static per-SM lists (the paper's mode); 0: CTAs pull from per-die queues */
     uint64_t seed;           /* oblivious only: 0 = lowest SM ids, else seeded random subset */
+    int64_t min_margin;      /* affinity only: byte margins below this count as ties (0 = exact ties only) */
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;

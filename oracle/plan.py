@@ -38,7 +38,9 @@ Steps.
        die_compact  die 0 takes R[0..q_0), die 1 takes the rest (contiguous bands);
        affinity     margin m(u) = local_0(u) - local_1(u) where local_d counts the bytes of
                     the unit's A panel, B panel and C tile that sit in chunks of die d
-                    (negated when invert_affinity); preferred die = 0 if m > 0, 1 if m < 0,
+                    (negated when invert_affinity); a margin with |m| < min_margin counts as 0
+                    (in an interleaved layout every unit is about half on each die and the
+                    sign of a tiny m is noise); preferred die = 0 if m > 0, 1 if m < 0,
                     the die_compact band's die if m == 0; units sorted by (|m| descending,
                     raster index ascending) are given to their preferred die while its
                     quota lasts, else to the other die; each die's queue is then put back
@@ -70,7 +72,7 @@ def mix64(x: int) -> int:
 def default_policy(**kw) -> dict:
     p = dict(kind=OBLIVIOUS, seed=0, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1,
              k_unit=64, raster_group=1, preferred_die=-1, invert_affinity=0,
-             static_assign=1, avoid=(), a=None, b=None, c=None)
+             static_assign=1, min_margin=0, avoid=(), a=None, b=None, c=None)
     p.update(kw)
     return p
 
@@ -257,6 +259,8 @@ def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
                 m = l0 - l1
                 if pol["invert_affinity"]:
                     m = -m
+                if abs(m) < pol["min_margin"]:
+                    m = 0
                 if m > 0:
                     pref = 0
                 elif m < 0:

@@ -532,15 +532,21 @@ extern "C" ag_status ag_topo_discover_phases(ag_topo_map* map, uint32_t phases) 
         if (near_off.size() >= 4 && other >= 0) {
             const int n = (int)near_off.size();
             AG_CUDA(cudaMemcpy(sc.d_off, near_off.data(), sizeof(long long) * n, cudaMemcpyHostToDevice));
-            std::vector<uint32_t> tmp, nearv, farv;
-            st = latency_rows(sc, n_sm, std::vector<int>{0}, n, 1, 1, tmp);       // SM 0 caches the lines in its L2
-            if (st == AG_OK) st = latency_rows(sc, n_sm, std::vector<int>{0}, n, 1, 1, nearv);   // local hit
-            if (st == AG_OK) st = latency_rows(sc, n_sm, std::vector<int>{other}, n, 1, 1, farv);  // other-die reader
+            std::vector<uint32_t> nearv, farv;
+            // SM 0 rewrites each line (now dirty in its home L2 on die 0) and times a reload: local hit.
+            st = latency_rows(sc, n_sm, std::vector<int>{0}, n, 2, 2, nearv);
+            // An SM of the other die then loads each line once: it comes from the home partition
+            // across the die-to-die fabric (a second load would hit the copy replicated locally).
+            if (st == AG_OK) st = latency_rows(sc, n_sm, std::vector<int>{other}, n, 1, 1, farv);
             if (st != AG_OK) return st;
             std::sort(nearv.begin(), nearv.end());
             std::sort(farv.begin(), farv.end());
-            map->l2_near_cycles = nearv[n / 2];
-            map->l2_far_cycles = farv[n / 2];
+            // reported only when the two tiers are apart: lines that an earlier access already
+            // replicated into the other die's L2 would read as local hits there
+            if (farv[n / 2] > 1.3 * nearv[n / 2]) {
+                map->l2_near_cycles = nearv[n / 2];
+                map->l2_far_cycles = farv[n / 2];
+            }
         }
     }
 

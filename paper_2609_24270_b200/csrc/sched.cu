@@ -25,6 +25,7 @@ struct OperandDev {
 struct PolicyDev {
     int kind, M, N, K, tile_m, tile_n, k_splits, k_unit, raster_group, preferred_die, invert, static_assign;
     unsigned long long seed;
+    long long min_margin;
     unsigned long long avoid[4];
     OperandDev a, b, c;
 };
@@ -251,10 +252,12 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
     } else {
         // rank of raster index i under the key (|m| descending, i ascending)
         for (int i = tid; i < n_units; i += nt) {
-            const long long mi = margins[i] < 0 ? -margins[i] : margins[i];
+            long long mi = margins[i] < 0 ? -margins[i] : margins[i];
+            if (mi < pol.min_margin) mi = 0;
             int rank = 0;
             for (int j = 0; j < n_units; ++j) {
-                const long long mj = margins[j] < 0 ? -margins[j] : margins[j];
+                long long mj = margins[j] < 0 ? -margins[j] : margins[j];
+                if (mj < pol.min_margin) mj = 0;
                 rank += (mj > mi) || (mj == mi && j < i);
             }
             order[rank] = i;
@@ -266,6 +269,7 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
                 const int i = order[r];
                 long long m = margins[i];
                 if (pol.invert) m = -m;
+                if ((m < 0 ? -m : m) < pol.min_margin) m = 0;
                 const int pref = m > 0 ? 0 : (m < 0 ? 1 : (i < q0 ? 0 : 1));
                 const int d = got[pref] < q[pref] ? pref : 1 - pref;
                 got[d]++;
@@ -350,7 +354,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     if (map->n_sm <= 0 || map->n_sm > AG_MAX_SM) return AG_ERR_ARG;
     if (p.kind < AG_OBLIVIOUS || p.kind > AG_AFFINITY) return AG_ERR_ARG;
     if (p.M <= 0 || p.N <= 0 || p.K <= 0 || p.tile_m <= 0 || p.tile_n <= 0) return AG_ERR_ARG;
-    if (p.k_splits < 1 || p.k_unit < 1 || p.raster_group < 1) return AG_ERR_ARG;
+    if (p.k_splits < 1 || p.k_unit < 1 || p.raster_group < 1 || p.min_margin < 0) return AG_ERR_ARG;
     if (p.kind == AG_AFFINITY && !amap) return AG_ERR_ARG;
     int n_cand = 0;
     for (int s = 0; s < map->n_sm; ++s)
@@ -422,6 +426,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pd.k_splits = p.k_splits; pd.k_unit = p.k_unit; pd.raster_group = p.raster_group;
         pd.preferred_die = p.preferred_die; pd.invert = p.invert_affinity; pd.static_assign = p.static_assign;
         pd.seed = p.seed;
+        pd.min_margin = p.min_margin;
         for (int i = 0; i < 4; ++i) pd.avoid[i] = p.avoid_sm_mask[i];
         pd.a = to_dev(p.a, nullptr); pd.b = to_dev(p.b, d_table); pd.c = to_dev(p.c, nullptr);
 

@@ -64,8 +64,8 @@ def test_full_size_config_plans_match():
             assert got.tobytes() == want.tobytes()
 
 
-@pytest.mark.parametrize("invert", [0, 1])
-def test_affinity_plan_matches_oracle_rowmajor(invert):
+@pytest.mark.parametrize("invert,min_margin", [(0, 0), (1, 0), (0, 20000), (0, 1 << 40)])
+def test_affinity_plan_matches_oracle_rowmajor(invert, min_margin):
     topo = inputs.synthetic_topo(die0_sms=72, seed=6)
     M = N = K = 1024
     a_off, b_off, c_off = 0, M * K * 2, M * K * 2 + K * N * 2
@@ -75,11 +75,16 @@ def test_affinity_plan_matches_oracle_rowmajor(invert):
     tbl = tbl.copy()
     tbl[::7] = 0
     kw = dict(kind=ag.AG_AFFINITY, M=M, N=N, K=K, tile_m=128, tile_n=128, invert_affinity=invert, raster_group=2,
+              min_margin=min_margin,
               a=dict(offset=a_off, row_stride=K * 2, elem_bytes=2),
               b=dict(offset=b_off, row_stride=N * 2, elem_bytes=2),
               c=dict(offset=c_off, row_stride=N * 4, elem_bytes=4))
     got, want, plan = both(topo, tbl, 148, **kw)
     assert got.tobytes() == want.tobytes()
+    if min_margin >= 1 << 40:                               # every margin is a tie: the die_compact bands
+        dc = op.export(op.build_plan(topo, None, 148, oracle_policy(kind=op.DIE_COMPACT, M=M, N=N, K=K, tile_m=128,
+                                                                    tile_n=128, raster_group=2)))
+        assert np.array_equal(got[2:], dc[2:])
     # margins, unit by unit
     pol = oracle_policy(**kw)
     amap = dict(chunk_bytes=4096, die_of_chunk=tbl)

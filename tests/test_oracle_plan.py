@@ -191,6 +191,19 @@ def test_equal_dies_split_c_in_halves():
     assert plan["die_q"][0] == list(range(1024)) and plan["die_q"][1] == list(range(1024, 2048))
 
 
+def test_min_margin_turns_weak_preferences_into_ties():
+    amap = toy_amap_case_d()
+    base = dict(M=256, N=512, K=64, c=op.operand(0, 2048, 4))
+    # margins are -131072, +65536, +131072, 0: with a floor of 100000 unit 1 becomes a tie and
+    # falls back to its band (raster index 1 < q0 = 2 -> die 0), which is where it was anyway;
+    p1 = op.build_plan(TOY, amap, 4, op.default_policy(kind=op.AFFINITY, min_margin=100000, **base))
+    assert p1["die_q"] == [[1, 2], [0, 3]]
+    # with a floor above every margin the plan is the die_compact one
+    p2 = op.build_plan(TOY, amap, 4, op.default_policy(kind=op.AFFINITY, min_margin=1 << 30, **base))
+    p3 = op.build_plan(TOY, None, 4, op.default_policy(kind=op.DIE_COMPACT, M=256, N=512, K=64))
+    assert p2["die_q"] == p3["die_q"] == [[0, 1], [2, 3]] and p2["sm_q"] == p3["sm_q"]
+
+
 def test_all_ties_affinity_equals_die_compact():
     topo = inputs.synthetic_topo(die0_sms=72)
     # A rows are 8 KB = one aligned chunk pair (dies 0,1): every margin is exactly 0
