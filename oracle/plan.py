@@ -313,23 +313,69 @@ def export(plan: dict) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------- die-view packing
-def build_page_table(unit_die: list[int], pages_per_unit: int, amap: dict) -> list[int]:
-    """Indirect allocation by remapping (Section 7.1.1, Eq. 1): logical page j of the
-    packed operand lives in one of the two physical chunks (2j, 2j+1); the one whose
-    measured die equals the die that owns the page's unit is taken.  The measured
-    chunk->die bit replaces the parity-of-masked-physical-address selector of Eq. 1,
-    which needs a physical base address that an unmodified driver does not expose.
-    If both chunks of a pair sit on the same die (the pair rule fails), chunk 2j is used.
+def build_page_table(page_die, amap: dict) -> list[int]:
+    """Indirect allocation by remapping (Section 7.1.1, Eq. 1 of the remapping appendix).
+
+    The packed buffer is read as aligned pairs of 4 KB chunks (2p, 2p+1); by the pair rule one
+    chunk of every pair sits on each die.  Two logical views are laid over the buffer, one per die:
+    page p of view d is the chunk of pair p that sits on die d.  Logical weight page j (owned by a
+    work unit that the plan gave to die ``page_die[j]``) takes the next free page of that die's
+    view.  The measured chunk->die bit replaces the parity-of-masked-physical-address selector of
+    Eq. 1, which needs a physical base address that an unmodified driver does not expose.
+    Where a pair has both chunks on one die x (the pair rule fails), view x takes the even chunk
+    and the other view the odd one, so that no chunk is used twice.
     """
     doc = amap["die_of_chunk"]
+    nxt = [0, 0]
     table = []
-    for u, d in enumerate(unit_die):
-        for p in range(pages_per_unit):
-            j = u * pages_per_unit + p
-            if int(doc[2 * j]) == d:
-                table.append(2 * j)
-            elif int(doc[2 * j + 1]) == d:
-                table.append(2 * j + 1)
-            else:
-                table.append(2 * j)
+    for d in page_die:
+        d = int(d)
+        pair = nxt[d]
+        nxt[d] += 1
+        # even chunk if it sits on die d, else the odd one (also right when the pair rule fails:
+        # both chunks on die x -> view x gets the even chunk, the other view the odd one)
+        table.append(2 * pair + (0 if int(doc[2 * pair]) == d else 1))
     return table
+
+
+def page_die_from_plan(plan: dict, K: int, k_unit: int = 64) -> list[int]:
+    """Die of every logical weight page (tn, k16), j = tn * ceil(K/16) + k16: the die whose queue
+    holds the unit (tn, ks) whose k-range contains the page."""
+    unit_die = {}
+    for d in (0, 1):
+        for u in plan["die_q"][d]:
+            unit_die[u] = d
+    ksp = plan["k_splits"]
+    n_slab = -(-K // k_unit)
+    per = -(-n_slab // ksp)
+    ppt = -(-K // 16)
+    out = []
+    for tn in range(plan["tiles_n"]):
+        for k16 in range(ppt):
+            ks = (k16 * 16 // k_unit) // per
+            out.append(unit_die[tn * ksp + ks])
+    return out
+
+
+def pack_weights(B_bits: np.ndarray, page_table: list[int], n_chunks: int, tile_n: int = 128) -> np.ndarray:
+    """Packed image (uint16, n_chunks x 2048) of the K x N bf16 weights.
+
+    Logical page (tn, k16) holds W[n][k] for n in [tn*128, tn*128+128), k in [k16*16, k16*16+16)
+    as 8 x 8 blocks ("core matrices", 8 rows n x 16 bytes of k, 128 bytes each, row-major inside):
+    element (n, k) of the page sits at byte (n//8)*256 + (k//8)*128 + (n%8)*16 + (k%8)*2.
+    Out-of-range n or k are zeros; chunks no page maps to stay zero.
+    """
+    K, N = B_bits.shape
+    ppt = -(-K // 16)
+    tiles_n = -(-N // tile_n)
+    out = np.zeros((n_chunks, 2048), dtype=np.uint16)
+    for tn in range(tiles_n):
+        for k16 in range(ppt):
+            page = np.zeros((tile_n, 16), dtype=np.uint16)
+            k0, n0 = k16 * 16, tn * tile_n
+            blk = B_bits[k0:min(K, k0 + 16), n0:min(N, n0 + tile_n)]       # [k][n]
+            page[:blk.shape[1], :blk.shape[0]] = blk.T
+            # (n//8, n%8, k//8, k%8) -> (n//8, k//8, n%8, k%8)
+            img = page.reshape(tile_n // 8, 8, 2, 8).transpose(0, 2, 1, 3).reshape(-1)
+            out[page_table[tn * ppt + k16]] = img
+    return out

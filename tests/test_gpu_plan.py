@@ -130,7 +130,7 @@ def test_paged_weights_affinity_recovers_packing_plan():
             unit_die[u] = d
     n_log = 16 * 64
     tbl = inputs.synthetic_chunk_die(2 * n_log, seed=5)
-    table = op.build_page_table(unit_die, 32, dict(chunk_bytes=4096, die_of_chunk=tbl))
+    table = op.build_page_table(op.page_die_from_plan(plan_d, 1024), dict(chunk_bytes=4096, die_of_chunk=tbl))
     bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=table)
     for inv in (0, 1):
         got, want, _ = both(topo, tbl, 148, kind=ag.AG_AFFINITY, invert_affinity=inv, b=bop, **kw)

@@ -236,7 +236,10 @@ def test_packing_by_plan_is_recovered_by_affinity():
     amap = dict(chunk_bytes=4096, die_of_chunk=inputs.synthetic_chunk_die(2 * n_log, seed=5))
     doc = amap["die_of_chunk"]
     assert all(doc[2 * j] != doc[2 * j + 1] for j in range(n_log))      # pair rule of Section 7.1.1
-    table = op.build_page_table(unit_die, pages_per_unit, amap)
+    page_die = op.page_die_from_plan(plan_d, 1024)
+    assert page_die == [d for d in unit_die for _ in range(pages_per_unit)]
+    table = op.build_page_table(page_die, amap)
+    assert len(set(table)) == len(table) and max(table) < 2 * max(page_die.count(0), page_die.count(1))
     assert all(int(doc[table[u * pages_per_unit + p]]) == unit_die[u]
                for u in range(plan_d["n_units"]) for p in range(pages_per_unit))
     bop = op.operand(0, 0, 2, layout=op.LAYOUT_PAGED, page_table=table)
@@ -251,6 +254,27 @@ def test_packing_by_plan_is_recovered_by_affinity():
     check_invariants(topo, plan_i, pi, 148)
 
 
+def test_page_table_views_share_pairs_and_survive_broken_pairs():
+    doc = np.array([0, 1, 1, 0, 1, 1, 0, 0, 1, 0], dtype=np.uint8)      # pairs 2 and 3 break the pair rule
+    amap = dict(chunk_bytes=4096, die_of_chunk=doc)
+    table = op.build_page_table([0, 1, 1, 0, 0, 1, 1, 0], amap)
+    # view 0 pages -> pairs 0,1,2,3 ; view 1 pages -> pairs 0,1,2,3
+    assert table == [0, 1, 2, 3, 5, 4, 7, 6]
+    assert len(set(table)) == 8
+
+
+def test_packed_page_layout_by_hand():
+    K, N = 32, 128
+    B = np.arange(K * N, dtype=np.uint16).reshape(K, N)                 # B[k][n] = k*128 + n
+    img = op.pack_weights(B, [3, 1], n_chunks=4)
+    assert not img[0].any() and not img[2].any()
+    page0 = img[3]                                                       # k16 = 0
+    # element (n, k) at halfword (n//8)*128 + (k//8)*64 + (n%8)*8 + (k%8)
+    for n, k in ((0, 0), (1, 0), (0, 1), (7, 7), (8, 0), (0, 8), (127, 15), (77, 13)):
+        assert page0[(n // 8) * 128 + (k // 8) * 64 + (n % 8) * 8 + (k % 8)] == k * 128 + n
+    assert img[1][(5 // 8) * 128 + (9 // 8) * 64 + 5 * 8 + 1] == (16 + 9) * 128 + 5   # k16 = 1
+
+
 def test_page_table_matches_printed_remap_formula():
     """Eq. 1 (appendix on address remapping): page_phys = 2j + [parity((page_start + 2j) & MASK) xor P]
     when a chunk's die is parity((page_start + chunk) & MASK) and bit 0 is in MASK."""
@@ -260,6 +284,6 @@ def test_page_table_matches_printed_remap_formula():
     doc = np.array([par((start + c) & MASK) for c in range(2 * n_log)], dtype=np.uint8)
     amap = dict(chunk_bytes=4096, die_of_chunk=doc)
     for P in (0, 1):
-        table = op.build_page_table([P] * n_log, 1, amap)
+        table = op.build_page_table([P] * n_log, amap)
         want = [2 * j + (par((start + 2 * j) & MASK) ^ P) for j in range(n_log)]
         assert table == want
