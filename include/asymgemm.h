@@ -183,7 +183,7 @@ typedef struct {
 typedef struct {
     int32_t kind;            /* AG_OBLIVIOUS | AG_DIE_COMPACT | AG_AFFINITY */
     int32_t M, N, K;
-    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}; skinny kernel: M<=... x 128 */
+    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}; decode-shaped kernel: {16,32} x 128 */
     int32_t k_splits;        /* >= 1, runs of whole k-slabs */
     int32_t k_unit;          /* elements per k-slab (64) */
     int32_t raster_group;    /* tile rows per raster group (>= 1) */
@@ -243,6 +243,45 @@ void ag_plan_destroy(ag_plan* plan);
  */
 ag_status gemm_persistent(const void* A, const void* B, void* C, int M, int N, int K,
                           const ag_plan* plan, void* cuda_stream);
+
+/* ---- die-local packed weights for decode-shaped GEMMs (Section 7.1.1) ------------------------ */
+typedef struct ag_packed_weights ag_packed_weights;
+
+/*
+ * ag_pack_weights - indirect allocation by remapping (Section 7.1.1 and the remapping appendix,
+ * Eq. 1): copy the K x N weights into 4 KB pages of [128 columns x 16 k] elements and store
+ * every page in a chunk of the die that the plan gave the page's work unit to.  The destination
+ * is read as aligned chunk pairs; two logical views (one per die) are laid over it and page p of
+ * view d is the chunk of pair p that the affinity map places on die d (the measured bit stands in
+ * for the parity-of-masked-physical-address selector of Eq. 1).  Inside a page element (n, k) sits
+ * at byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2, the order the MMA reads without swizzle.
+ *   B      device, K x N bf16 row-major
+ *   plan   a plan with tile_n = 128 and one tile row (M <= tile_m <= 32), K % 64 == 0
+ *   amap   affinity map of exactly (dst, dst_bytes), else AG_ERR_STALE_AMAP
+ *   dst    device, 4096-aligned; needs 2 * max(pages of die 0, pages of die 1) chunks
+ *   out    host, out: handle holding the page table (device + host copy)
+ * Synchronises the device.  Errors: AG_ERR_ARG, AG_ERR_STALE_AMAP, AG_ERR_CUDA, AG_ERR_NOMEM.
+ */
+ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
+                          void* dst, size_t dst_bytes, ag_packed_weights** out);
+/* Page table (host, cap entries): chunk index in dst of logical page (tn, k16) = tn * (K/16) + k16;
+ * feed it to ag_operand_desc.page_table to build an affinity plan over the packed weights. */
+ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* out, size_t cap, size_t* n_pages);
+void ag_packed_destroy(ag_packed_weights* w);
+
+/*
+ * gemm_persistent_packed - C = A * B for M <= 32 with the weights taken from a packed buffer
+ * (Section 7.1.2 on top of Section 7.1.1: each block reads the pages of its units, which the
+ * packing put on the block's own die when plan and packing agree).  gemm_persistent handles the
+ * same shapes with row-major B.
+ *   A  device, M x K bf16 row-major, 16-byte aligned;  C  device, M x N fp32 row-major, overwritten
+ *   plan  tile_m in {16, 32} (M <= tile_m), tile_n = 128, same N, K as the packing; with
+ *         k_splits > 1 the partial sums go through the plan's workspace and are added in
+ *         ascending split order by the block that finishes a tile last (deterministic)
+ * Asynchronous on cuda_stream.  Errors as gemm_persistent.
+ */
+ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* C, int M, int N, int K,
+                                 const ag_plan* plan, void* cuda_stream);
 
 const char* ag_strerror(ag_status s);
 /* Last CUDA error code seen by the calling thread inside the library (0 = none). */

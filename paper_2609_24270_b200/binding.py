@@ -26,7 +26,8 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_strerror", "ag_last_cuda_error",
+    "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
+    "ag_packed_destroy", "gemm_persistent_packed", "ag_strerror", "ag_last_cuda_error",
     "ag_kernel_launch_count",
 ]
 
@@ -127,6 +128,11 @@ def lib() -> C.CDLL:
     L.ag_plan_destroy.argtypes = [vp]
     L.ag_plan_destroy.restype = None
     L.gemm_persistent.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.ag_pack_weights.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, sz, C.POINTER(vp)]
+    L.ag_packed_page_table.argtypes = [vp, vp, sz, C.POINTER(sz)]
+    L.ag_packed_destroy.argtypes = [vp]
+    L.ag_packed_destroy.restype = None
+    L.gemm_persistent_packed.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.ag_strerror.argtypes = [C.c_int]
     L.ag_strerror.restype = C.c_char_p
     L.ag_last_cuda_error.restype = C.c_int
@@ -339,3 +345,38 @@ def sched_build(topo: TopoMap, amap: AffinityMap | None, sm_budget: int, policy:
 def gemm_persistent(a_ptr: int, b_ptr: int, c_ptr: int, M: int, N: int, K: int, plan: Plan, stream: int = 0):
     """Raw device pointers in, asynchronous on `stream` (a cudaStream_t value, 0 = default)."""
     _check(lib().gemm_persistent(a_ptr, b_ptr, c_ptr, M, N, K, plan.handle, stream), "gemm_persistent")
+
+
+class PackedWeights:
+    def __init__(self, handle):
+        self.handle = handle
+
+    def page_table(self) -> np.ndarray:
+        n = C.c_size_t()
+        _check(lib().ag_packed_page_table(self.handle, None, 0, C.byref(n)), "ag_packed_page_table")
+        out = np.empty(n.value, dtype=np.int32)
+        _check(lib().ag_packed_page_table(self.handle, out.ctypes.data, out.size, C.byref(n)), "ag_packed_page_table")
+        return out
+
+    def destroy(self):
+        if self.handle:
+            lib().ag_packed_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def pack_weights(b_ptr: int, K: int, N: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int) -> PackedWeights:
+    h = C.c_void_p()
+    _check(lib().ag_pack_weights(b_ptr, K, N, plan.handle, amap.handle, dst_ptr, dst_bytes, C.byref(h)), "ag_pack_weights")
+    return PackedWeights(h)
+
+
+def gemm_persistent_packed(a_ptr: int, packed: PackedWeights, c_ptr: int, M: int, N: int, K: int, plan: Plan,
+                           stream: int = 0):
+    _check(lib().gemm_persistent_packed(a_ptr, packed.handle, c_ptr, M, N, K, plan.handle, stream),
+           "gemm_persistent_packed")

@@ -13,18 +13,13 @@
 
 #include <mutex>
 
-#include "internal.h"
-#include "ptx.cuh"
+#include "persist.cuh"
 
 namespace ag {
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int kThreads = 192;
-constexpr int kRing = 8;            // depth of the unit-id ring between the scheduler and its consumers
-constexpr int kEpiWarps = 4;
 constexpr int kEpiBufBytes = 32 * 32 * 4;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s
 
 template <int BN>
 struct Cfg {
@@ -37,19 +32,6 @@ struct Cfg {
     static constexpr int stages = budget / stage_bytes > 8 ? 8 : budget / stage_bytes;
     static constexpr int smem_bytes = stages * stage_bytes + epi_bytes + bar_bytes + 1024;
     static constexpr int tmem_cols = 2 * BN < 32 ? 32 : 2 * BN;  // power of two for BN in {64,128,256}
-};
-
-struct GemmParams {
-    const int32_t* image;   // plan image (device)
-    PlanCtrl* ctrl;
-    int32_t* tile_owner;
-    int32_t* tile_count;
-    int M, N, K;
-    int b, n_units, n_sm;
-    int tiles_n, k_splits, kslabs_total, kslabs_per_split;
-    int static_assign;
-    unsigned int epoch;
-    unsigned long long wait_limit_ns;
 };
 
 struct SharedCtl {
@@ -66,32 +48,10 @@ struct SharedCtl {
     int member;
 };
 
-__device__ __forceinline__ void report_timeout(const GemmParams& p, int role) {
-    if (atomicCAS(&p.ctrl->status, 0, (int)AG_ERR_TIMEOUT) == 0) p.ctrl->status_info = (role << 16) | (int)smid();
-}
-
-// Dynamic mode: take the next index of die d's queue; the 64-bit head carries the epoch of the
-// launch that last touched it, so it resets itself.  Returns -1 when the queue is drained.
-__device__ inline int pop_queue(unsigned long long* head, unsigned int epoch, int len) {
-    for (int tries = 0; tries < 100000; ++tries) {
-        unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(head);
-        if ((unsigned int)(cur >> 32) != epoch) {
-            if (len <= 0) return -1;
-            const unsigned long long nv = ((unsigned long long)epoch << 32) | 1ull;
-            if (atomicCAS(head, cur, nv) == cur) return 0;
-            continue;
-        }
-        const int idx = (int)(cur & 0xffffffffull);
-        if (idx >= len) return -1;
-        if (atomicCAS(head, cur, cur + 1) == cur) return idx;
-    }
-    return -1;
-}
-
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                  const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
+                  const __grid_constant__ CUtensorMap tm_c, const PersistParams p) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -103,30 +63,10 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const PlanLayout lay{p.b, p.n_units, p.n_sm};
     const int my_sm = (int)smid();
-    const int slot = p.image[lay.smid_to_slot() + my_sm];
-
-    if (slot < 0) {
-        // Not in the plan.  Stay resident until every planned SM has a block (or ~40 us pass), so
-        // that blocks still being placed can only land on SMs that have none yet.
-        const uint64_t t0 = globaltimer_ns();
-        while (true) {
-            int ok = 1;
-            for (int i = tid; i < p.b; i += kThreads)
-                ok &= (*reinterpret_cast<volatile unsigned int*>(&p.ctrl->claimed[i]) == p.epoch);
-            if (__syncthreads_and(ok)) break;
-            if (globaltimer_ns() - t0 > 40000ull) break;
-            __nanosleep(200);
-        }
-        return;
-    }
-    if (tid == 0) {
-        ctl->member = atomicMax(&p.ctrl->claimed[slot], p.epoch) < p.epoch;
-        ctl->abort_flag = 0;
-    }
-    __syncthreads();
-    if (!ctl->member) return;  // a second block on an SM whose slot is already taken
+    if (tid == 0) ctl->abort_flag = 0;
+    const int slot = join_plan(p, &ctl->member);
+    if (slot < 0) return;
 
     if (tid == 0) {
         for (int i = 0; i < C::stages; ++i) {
@@ -160,44 +100,11 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     if (warp == 0) {
         // ------------------------------------------------ scheduler + TMA producer (one lane)
         if (lane == 0) {
-            const int my_die = p.image[lay.sm_die() + slot];
-            int cur_slot = slot, idx = 0;
-            int list_off = p.image[lay.sm_q_off() + slot], list_len = p.image[lay.sm_q_off() + slot + 1] - list_off;
-            int scan = 0;          // static mode: next slot to look at for adoption
-            int dyn_die = my_die;  // dynamic mode: queue being drained
+            UnitSource src(p, slot);
             uint32_t it = 0, kit = 0;
             bool ok = true;
             while (ok) {
-                int u = -1;
-                if (p.static_assign) {
-                    while (true) {
-                        if (idx < list_len) { u = p.image[lay.sm_q() + list_off + idx++]; break; }
-                        // own list done: run the list of any planned SM that never got a block
-                        bool adopted = false;
-                        for (; scan < p.b; ++scan) {
-                            if (*reinterpret_cast<volatile unsigned int*>(&p.ctrl->claimed[scan]) == p.epoch) continue;
-                            if (atomicMax(&p.ctrl->claimed[scan], p.epoch) < p.epoch) {
-                                cur_slot = scan;
-                                list_off = p.image[lay.sm_q_off() + cur_slot];
-                                list_len = p.image[lay.sm_q_off() + cur_slot + 1] - list_off;
-                                idx = 0;
-                                atomicAdd(&p.ctrl->adopted, 1u);
-                                adopted = true;
-                                ++scan;
-                                break;
-                            }
-                        }
-                        if (!adopted) break;
-                    }
-                } else {
-                    for (int t = 0; t < 2 && u < 0; ++t) {
-                        const int q_off = p.image[lay.die_q_off() + dyn_die];
-                        const int q_len = p.image[lay.die_q_off() + dyn_die + 1] - q_off;
-                        const int e = pop_queue(&p.ctrl->die_head[dyn_die], p.epoch, q_len);
-                        if (e >= 0) u = p.image[lay.die_q() + q_off + e];
-                        else dyn_die ^= 1;  // own die drained: help the other one
-                    }
-                }
+                const int u = src.next();
                 const int r = it % kRing;
                 if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 1);
@@ -367,11 +274,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode() {
+EncodeTiledFn get_encode_tiled() {
     static EncodeTiledFn fn = nullptr;
     static std::once_flag once;
     std::call_once(once, [] {
@@ -384,10 +287,9 @@ static EncodeTiledFn get_encode() {
     return fn;
 }
 
-// 2-D row-major tensor of `rows` x `cols` elements, box = box_cols x box_rows, 128-byte swizzle.
-static bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const void* ptr, uint64_t rows,
-                      uint64_t cols, uint32_t box_cols, uint32_t box_rows) {
-    EncodeTiledFn enc = get_encode();
+bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const void* ptr, uint64_t rows,
+               uint64_t cols, uint32_t box_cols, uint32_t box_rows) {
+    EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
@@ -399,7 +301,7 @@ static bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, c
 }
 
 template <int BN>
-static ag_status launch(const ag_plan* plan, const GemmParams& gp, cudaStream_t stream) {
+static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream_t stream) {
     using C = Cfg<BN>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -415,12 +317,20 @@ static ag_status launch(const ag_plan* plan, const GemmParams& gp, cudaStream_t 
 
 }  // namespace ag
 
+namespace ag {
+ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
+                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream);
+}
+
 using namespace ag;
 
 extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, int M, int N, int K,
                                      const ag_plan* plan, void* cuda_stream) {
     if (!A || !B || !Cout || !plan) return AG_ERR_ARG;
     const int32_t* h = plan->header;
+    if (h[H_TILE_M] <= 32)  // decode-shaped plan: weights on the MMA's M side, split-K through the plan's scratch
+        return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
+                                    reinterpret_cast<cudaStream_t>(cuda_stream));
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_M] != BM || (h[H_TILE_N] != 64 && h[H_TILE_N] != 128 && h[H_TILE_N] != 256)) return AG_ERR_ARG;
     if (plan->policy.k_unit != BK) return AG_ERR_ARG;
@@ -441,18 +351,7 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
         plan->tm_a_ptr = A; plan->tm_b_ptr = B; plan->tm_c_ptr = Cout;
     }
     if (h[H_KSPLITS] > 1) AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * (size_t)M * (size_t)N, stream));
-    GemmParams gp;
-    gp.image = plan->d_image;
-    gp.ctrl = plan->d_ctrl;
-    gp.tile_owner = plan->d_tile_owner;
-    gp.tile_count = plan->d_tile_count;
-    gp.M = M; gp.N = N; gp.K = K;
-    gp.b = plan->lay.b; gp.n_units = plan->lay.n_units; gp.n_sm = plan->lay.n_sm;
-    gp.tiles_n = h[H_TILES_N]; gp.k_splits = h[H_KSPLITS];
-    gp.kslabs_total = plan->kslabs_total; gp.kslabs_per_split = plan->kslabs_per_split;
-    gp.static_assign = h[H_STATIC];
-    gp.epoch = ++plan->epoch;
-    gp.wait_limit_ns = kWaitLimitNs;
+    const PersistParams gp = make_persist_params(plan, M, N, K);
     if (BN == 256) return launch<256>(plan, gp, stream);
     if (BN == 128) return launch<128>(plan, gp, stream);
     return launch<64>(plan, gp, stream);

@@ -1,0 +1,432 @@
+// Decode-shaped (skinny) persistent GEMM: C[M x N] = A[M x K] * B[K x N] with M <= 32.  The
+// weights B are the work: every unit streams a 128-column weight tile over a run of k-slabs, so
+// the kernel is HBM bound.  The MMA is turned around: the weight tile is the M = 128 operand,
+// the activations are the N = 16 or 32 operand, D[n][m] accumulates in tensor memory.
+//
+// Weights come either row-major (K x N, consumed in place as an MN-major operand through TMA) or
+// packed by ag_pack_weights: 4 KB pages of [128 n x 16 k] elements, each page already in the
+// MMA's no-swizzle core-matrix order and stored in a chunk of the die that owns its work unit
+// (indirect allocation by remapping, Section 7.1.1 of the paper).  A packed page is fetched with
+// one 4 KB bulk copy whose source address comes from the page table.
+//
+// Split-K units write partial sums to a scratch workspace; the block that completes a tile's
+// last split adds them in ascending split order (deterministic) and writes C.
+#include <string.h>
+
+#include <mutex>
+#include <new>
+
+#include "persist.cuh"
+
+namespace ag {
+
+constexpr int SK_BN = 128;     // weight columns per unit
+constexpr int SK_BK = 64;      // k-slab
+constexpr int SK_STAGES = 10;
+constexpr int SK_W_BYTES = SK_BN * SK_BK * 2;      // 16 KB of weights per stage
+constexpr int SK_A_BYTES = 32 * SK_BK * 2;         // room for 32 activation rows
+constexpr int SK_STAGE_BYTES = SK_W_BYTES + SK_A_BYTES;
+constexpr int SK_SMEM_BYTES = SK_STAGES * SK_STAGE_BYTES + 1024 + 1024;
+constexpr int SK_TMEM_COLS = 64;                   // two accumulators of 32 columns
+
+struct SkinnyCtl {
+    uint64_t full[SK_STAGES];
+    uint64_t empty[SK_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t sched_full[kRing];
+    uint64_t sched_empty[kRing];
+    uint64_t mma_drain;
+    int ring[kRing];
+    uint32_t tmem_base;
+    int abort_flag;
+    int member;
+};
+
+struct SkinnyArgs {
+    const uint8_t* packed;        // packed weights base (PACKED) or null
+    const int32_t* page_table;    // device (PACKED)
+    int pages_per_tile;
+    float* C;
+    float* partial;               // [k_splits][M][N] or null when k_splits == 1
+    int* sem;                     // [tiles_n * 4]: one arrival counter per 32-column quarter of a tile
+};
+
+template <int NM, bool PACKED>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+              const PersistParams p, const SkinnyArgs x) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + SK_STAGES * SK_STAGE_BYTES);
+    volatile int* abort_flag = &ctl->abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int my_sm = (int)smid();
+    if (tid == 0) ctl->abort_flag = 0;
+    const int slot = join_plan(p, &ctl->member);
+    if (slot < 0) return;
+
+    if (tid == 0) {
+        for (int i = 0; i < SK_STAGES; ++i) {
+            mbar_init(smem_u32(&ctl->full[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), kEpiWarps);
+        }
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(smem_u32(&ctl->sched_full[i]), 1);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps);
+        }
+        mbar_init(smem_u32(&ctl->mma_drain), 1);
+        mbar_fence_init();
+        prefetch_tmap(&tm_a);
+        if (!PACKED) prefetch_tmap(&tm_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), SK_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const uint64_t limit = p.wait_limit_ns;
+    constexpr uint32_t kTxBytes = SK_W_BYTES + NM * SK_BK * 2;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            UnitSource src(p, slot);
+            uint32_t it = 0, kit = 0;
+            bool ok = true;
+            while (ok) {
+                const int u = src.next();
+                const int r = it % kRing;
+                if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                    report_timeout(p, 1);
+                    ok = false;
+                    break;
+                }
+                ctl->ring[r] = u;
+                mbar_arrive(smem_u32(&ctl->sched_full[r]));
+                ++it;
+                if (u < 0) break;
+                const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
+                const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
+                const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+                for (int s = s0; s < s1; ++s, ++kit) {
+                    const int st = kit % SK_STAGES;
+                    if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / SK_STAGES) & 1) ^ 1, abort_flag, limit)) {
+                        report_timeout(p, 2);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&ctl->full[st]);
+                    const uint32_t sw = base + st * SK_STAGE_BYTES, sa = sw + SK_W_BYTES;
+                    mbar_expect_tx(bar, kTxBytes);
+                    if (PACKED) {
+                        const int32_t* pt = x.page_table + (size_t)tn * x.pages_per_tile + s * 4;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            bulk_load(sw + i * 4096, x.packed + (size_t)pt[i] * AG_CHUNK_BYTES, 4096, bar);
+                    } else {
+                        tma_load_2d(sw, &tm_w, bar, tn * SK_BN, s * SK_BK);
+                        tma_load_2d(sw + 8192, &tm_w, bar, tn * SK_BN + 64, s * SK_BK);
+                    }
+                    tma_load_2d(sa, &tm_a, bar, s * SK_BK, 0);
+                }
+            }
+            if (!ok) {
+                const uint32_t n_out = kit < (uint32_t)SK_STAGES ? kit : (uint32_t)SK_STAGES;
+                for (uint32_t j = 0; j < n_out; ++j) {
+                    const uint32_t k2 = kit - 1 - j;
+                    int dummy = 0;
+                    mbar_wait(smem_u32(&ctl->full[k2 % SK_STAGES]), (k2 / SK_STAGES) & 1, &dummy, 2000000ull);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(128, NM, PACKED ? 0 : 1, 0);
+            uint32_t kit = 0, tile_it = 0;
+            bool ok = true;
+            for (uint32_t it = 0; ok; ++it) {
+                const int r = it % kRing;
+                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    report_timeout(p, 3);
+                    break;
+                }
+                const int u = ctl->ring[r];
+                mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                if (u < 0) break;
+                const int ks = u % p.k_splits;
+                const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
+                const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+                const uint32_t acc = tile_it & 1;
+                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
+                    report_timeout(p, 4);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * 32;
+                for (int s = s0; s < s1; ++s, ++kit) {
+                    const int st = kit % SK_STAGES;
+                    if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / SK_STAGES) & 1, abort_flag, limit)) {
+                        report_timeout(p, 5);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sw = base + st * SK_STAGE_BYTES, sa = sw + SK_W_BYTES;
+#pragma unroll
+                    for (int k4 = 0; k4 < SK_BK / 16; ++k4) {
+                        // weights: packed page = no swizzle, 16-byte k chunks 128 B apart (LBO), 8-row groups
+                        // 256 B apart (SBO); row-major = MN-major, 128-byte swizzle, as B in the dense kernel
+                        const uint64_t dw = PACKED ? make_smem_desc(sw + k4 * 4096, 128, 256, 0)
+                                                   : make_smem_desc(sw + k4 * 2048, 8192, 1024, 2);
+                        const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
+                        tc_mma_f16(d_tmem, dw, da, idesc, (s > s0 || k4 > 0) ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->empty[st]));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                ++tile_it;
+            }
+            if (*abort_flag) {
+                tc_commit(smem_u32(&ctl->mma_drain));
+                int dummy = 0;
+                mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue: lane = weight column n, registers = rows m
+        const int q = warp & 3;
+        uint32_t tile_it = 0;
+        for (uint32_t it = 0;; ++it) {
+            const int r = it % kRing;
+            if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                if (lane == 0) report_timeout(p, 6);
+                break;
+            }
+            const int u = ctl->ring[r];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+            if (u < 0) break;
+            const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
+            const uint32_t acc = tile_it & 1;
+            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
+                if (lane == 0) report_timeout(p, 7);
+                break;
+            }
+            tc_fence_after();
+            uint32_t v[NM];
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 32;
+            if constexpr (NM == 16) tmem_ld_32x16(taddr, v); else tmem_ld_32x32(taddr, v);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+            const int n = tn * SK_BN + q * 32 + lane;
+            float* out = p.k_splits > 1 ? x.partial + (size_t)ks * p.M * p.N : x.C;
+            if (n < p.N) {
+#pragma unroll
+                for (int m = 0; m < NM; ++m)
+                    if (m < p.M) out[(size_t)m * p.N + n] = __uint_as_float(v[m]);
+            }
+            if (p.k_splits > 1) {
+                // Each epilogue warp owns 32 columns of the tile and keeps its own arrival counter: the
+                // warp that completes the last of the k_splits partial sums of those columns adds them
+                // in ascending split order.  No barrier between warps is needed.
+                __threadfence();
+                __syncwarp();
+                int last = 0;
+                if (lane == 0) last = atomicAdd(&x.sem[tn * 4 + q], 1) == p.k_splits - 1;
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    __threadfence();
+                    if (n < p.N) {
+                        for (int m = 0; m < p.M; ++m) {
+                            float s = 0.f;
+                            for (int k = 0; k < p.k_splits; ++k)
+                                s += __ldcg(x.partial + ((size_t)k * p.M + m) * p.N + n);
+                            x.C[(size_t)m * p.N + n] = s;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) x.sem[tn * 4 + q] = 0;  // ready for the next launch
+                }
+            }
+            if (lane == 0 && q == 0) {
+                p.tile_owner[u] = my_sm;
+                atomicAdd(&p.tile_count[u], 1);
+            }
+            ++tile_it;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, SK_TMEM_COLS);
+    }
+}
+
+// One block per logical page: gathers W[n][k] = B[k][n] for 128 n x 16 k and writes the 4 KB page in
+// core-matrix order into its chunk.
+__global__ void k_pack_weights(const uint16_t* __restrict__ B, int K, int N, int pages_per_tile,
+                               const int32_t* __restrict__ page_table, uint8_t* __restrict__ dst) {
+    const int page = blockIdx.x;
+    const int tn = page / pages_per_tile, k16 = page % pages_per_tile;
+    const int n_local = threadIdx.x;  // 128 threads
+    const int n = tn * SK_BN + n_local;
+    uint16_t v[16];
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+        const int k = k16 * 16 + kk;
+        v[kk] = (n < N && k < K) ? B[(size_t)k * N + n] : (uint16_t)0;
+    }
+    uint8_t* out = dst + (size_t)page_table[page] * AG_CHUNK_BYTES + (n_local / 8) * 256 + (n_local % 8) * 16;
+    uint4 lo, hi;
+    lo.x = v[0] | (v[1] << 16); lo.y = v[2] | (v[3] << 16); lo.z = v[4] | (v[5] << 16); lo.w = v[6] | (v[7] << 16);
+    hi.x = v[8] | (v[9] << 16); hi.y = v[10] | (v[11] << 16); hi.z = v[12] | (v[13] << 16); hi.w = v[14] | (v[15] << 16);
+    *reinterpret_cast<uint4*>(out) = lo;
+    *reinterpret_cast<uint4*>(out + 128) = hi;
+}
+
+template <int NM, bool PACKED>
+static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, const CUtensorMap& tm_w,
+                               const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream) {
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(k_gemm_skinny<NM, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SK_SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    k_gemm_skinny<NM, PACKED><<<plan->lay.n_sm, kThreads, SK_SMEM_BYTES, stream>>>(tm_a, tm_w, gp, x);
+    count_launch();
+    AG_CUDA(cudaGetLastError());
+    return AG_OK;
+}
+
+// Shared host path of the two skinny entry points.
+ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
+                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream) {
+    const int32_t* h = plan->header;
+    if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
+    if (h[H_TILE_N] != SK_BN || (h[H_TILE_M] != 16 && h[H_TILE_M] != 32) || M > h[H_TILE_M]) return AG_ERR_ARG;
+    if (plan->policy.k_unit != SK_BK || (K % 8) || (N % 8)) return AG_ERR_ARG;
+    if (((uintptr_t)A | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
+    if (h[H_KSPLITS] > 1 && (!partial || !sem)) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    int dev = 0, n_sm = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    if (n_sm != plan->lay.n_sm) return AG_ERR_ARG;
+    const int NM = h[H_TILE_M];
+    CUtensorMap tm_a, tm_w;
+    memset(&tm_w, 0, sizeof tm_w);
+    if (!encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, SK_BK, NM)) return AG_ERR_CUDA;
+    SkinnyArgs x;
+    memset(&x, 0, sizeof x);
+    x.C = (float*)Cout;
+    x.partial = h[H_KSPLITS] > 1 ? partial : nullptr;
+    x.sem = sem;
+    if (W) {
+        if (W->K != K || W->N != N || (K % SK_BK)) return AG_ERR_ARG;
+        x.packed = W->dst;
+        x.page_table = W->d_page_table;
+        x.pages_per_tile = W->pages_per_tile;
+    } else {
+        if (!B_rowmajor || ((uintptr_t)B_rowmajor & 15u)) return AG_ERR_ARG;
+        if (!encode_2d(&tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_rowmajor, K, N, 64, SK_BK)) return AG_ERR_CUDA;
+    }
+    const PersistParams gp = make_persist_params(plan, M, N, K);
+    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream)
+                           : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream);
+    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, gp, x, stream)
+             : launch_skinny<32, false>(plan, tm_a, tm_w, gp, x, stream);
+}
+
+}  // namespace ag
+
+using namespace ag;
+
+extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
+                                     void* dst, size_t dst_bytes, ag_packed_weights** out) {
+    if (!B || !plan || !amap || !dst || !out || K <= 0 || N <= 0) return AG_ERR_ARG;
+    *out = nullptr;
+    const int32_t* h = plan->header;
+    if (h[H_TILE_N] != SK_BN || h[H_N] != N || h[H_K] != K || h[H_TILES_M] != 1 || (K % SK_BK)) return AG_ERR_ARG;
+    if (amap->base != dst || amap->bytes != dst_bytes) return AG_ERR_STALE_AMAP;
+    const int tiles_n = h[H_TILES_N], ksp = h[H_KSPLITS];
+    const int ppt = K / 16;
+    const size_t n_pages = (size_t)tiles_n * ppt;
+    // die of every unit from the plan's die queues
+    const PlanLayout& lay = plan->lay;
+    const int32_t* img = plan->h_image.data();
+    std::vector<uint8_t> unit_die(lay.n_units, 0);
+    for (int e = img[lay.die_q_off() + 1]; e < lay.n_units; ++e) unit_die[img[lay.die_q() + e]] = 1;
+    // two logical views over the chunk pairs: page p of view d = the chunk of pair p that sits on die d
+    ag_packed_weights* w = new (std::nothrow) ag_packed_weights();
+    if (!w) return AG_ERR_NOMEM;
+    w->K = K; w->N = N; w->tiles_n = tiles_n; w->pages_per_tile = ppt; w->n_pages = n_pages;
+    w->dst = (const uint8_t*)dst; w->dst_bytes = dst_bytes; w->d_page_table = nullptr;
+    w->h_page_table.resize(n_pages);
+    size_t next[2] = {0, 0};
+    const int per = plan->kslabs_per_split;
+    for (int tn = 0; tn < tiles_n; ++tn)
+        for (int k16 = 0; k16 < ppt; ++k16) {
+            const int ks = (k16 * 16 / SK_BK) / per;
+            const int d = unit_die[(size_t)tn * ksp + ks];
+            const size_t pair = next[d]++;
+            if (2 * pair + 1 >= amap->n_chunks) {
+                delete w;
+                return AG_ERR_ARG;  // destination too small for this die's view
+            }
+            w->h_page_table[(size_t)tn * ppt + k16] = (int32_t)(2 * pair + (amap->h_die_of_chunk[2 * pair] == d ? 0 : 1));
+        }
+    cudaError_t e = cudaMalloc(&w->d_page_table, sizeof(int32_t) * n_pages);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(w->d_page_table, w->h_page_table.data(), sizeof(int32_t) * n_pages, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        k_pack_weights<<<(unsigned)n_pages, 128>>>((const uint16_t*)B, K, N, ppt, w->d_page_table, (uint8_t*)dst);
+        count_launch();
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        cudaFree(w->d_page_table);
+        delete w;
+        return cuda_fail(e);
+    }
+    *out = w;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* outp, size_t cap, size_t* n_pages) {
+    if (!w) return AG_ERR_ARG;
+    if (n_pages) *n_pages = w->n_pages;
+    if (!outp) return n_pages ? AG_OK : AG_ERR_ARG;
+    if (cap < w->n_pages) return AG_ERR_ARG;
+    memcpy(outp, w->h_page_table.data(), w->n_pages * sizeof(int32_t));
+    return AG_OK;
+}
+
+extern "C" void ag_packed_destroy(ag_packed_weights* w) {
+    if (!w) return;
+    cudaFree(w->d_page_table);
+    delete w;
+}
+
+extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* Cout, int M, int N, int K,
+                                            const ag_plan* plan, void* cuda_stream) {
+    if (!A || !W || !Cout || !plan) return AG_ERR_ARG;
+    return gemm_skinny_dispatch(A, nullptr, W, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
+                                reinterpret_cast<cudaStream_t>(cuda_stream));
+}

@@ -66,6 +66,8 @@ struct ag_plan {
     int32_t* d_tile_owner;     // device [n_units]
     int32_t* d_tile_count;     // device [n_units]
     long long* d_margins;      // device [n_units] (affinity only, else null)
+    float* d_partial;          // device [k_splits][M][N] split-K partial sums (skinny plans with k_splits > 1)
+    int* d_sem;                // device [4 * tiles_n] arrival counters for the split-K reduction
     std::vector<int32_t> h_image;
     mutable uint32_t epoch;
     int kslabs_total;
@@ -73,6 +75,15 @@ struct ag_plan {
     // tensor-map cache for the last (A, B, C) triple
     mutable const void* tm_a_ptr; mutable const void* tm_b_ptr; mutable void* tm_c_ptr;
     mutable CUtensorMap tm_a, tm_b, tm_c;
+};
+
+struct ag_packed_weights {
+    int K, N, tiles_n, pages_per_tile;   // pages_per_tile = K / 16
+    size_t n_pages;
+    const uint8_t* dst;                  // device: packed buffer (the probed buffer)
+    size_t dst_bytes;
+    int32_t* d_page_table;               // device [n_pages]: chunk index of each logical page
+    std::vector<int32_t> h_page_table;
 };
 
 namespace ag {

@@ -391,6 +391,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     pl->policy.a.page_table = pl->policy.b.page_table = pl->policy.c.page_table = nullptr;
     pl->d_image = nullptr; pl->d_ctrl = nullptr; pl->d_tile_owner = nullptr; pl->d_tile_count = nullptr;
     pl->d_margins = nullptr;
+    pl->d_partial = nullptr; pl->d_sem = nullptr;
     pl->epoch = 0;
     pl->kslabs_total = n_slab;
     pl->kslabs_per_split = per;
@@ -412,6 +413,12 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         TRY(cudaMalloc(&pl->d_tile_count, sizeof(int32_t) * n_units));
         TRY(cudaMemset(pl->d_tile_owner, 0xFF, sizeof(int32_t) * n_units));
         TRY(cudaMemset(pl->d_tile_count, 0, sizeof(int32_t) * n_units));
+        if (p.tile_m <= 32 && p.k_splits > 1) {
+            // decode-shaped plans: split-K partial sums and per-tile arrival counters
+            TRY(cudaMalloc(&pl->d_partial, sizeof(float) * (size_t)p.k_splits * p.M * p.N));
+            TRY(cudaMalloc(&pl->d_sem, sizeof(int) * (size_t)tiles_n * 4));
+            TRY(cudaMemset(pl->d_sem, 0, sizeof(int) * (size_t)tiles_n * 4));
+        }
         TRY(cudaMalloc(&d_topo, sizeof(ag_topo_map)));
         TRY(cudaMemcpy(d_topo, map, sizeof(ag_topo_map), cudaMemcpyHostToDevice));
         TRY(cudaMalloc(&d_order, sizeof(int32_t) * n_units));
@@ -519,5 +526,7 @@ extern "C" void ag_plan_destroy(ag_plan* plan) {
     cudaFree(plan->d_tile_owner);
     cudaFree(plan->d_tile_count);
     cudaFree(plan->d_margins);
+    cudaFree(plan->d_partial);
+    cudaFree(plan->d_sem);
     delete plan;
 }

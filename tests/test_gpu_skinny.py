@@ -1,0 +1,134 @@
+"""Decode-shaped GEMM (M <= 32): row-major and die-packed weights against the fp64 oracle, the
+packing against the oracle's page table and page layout."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gemm as og
+from oracle import plan as op
+from paper_2609_24270_b200 import binding as ag
+from paper_2609_24270_b200 import inputs
+from tests.gpu_util import check_close, device_topo, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def run_rowmajor(A, B, plan):
+    M, K = A.shape
+    N = B.shape[1]
+    dA, dB = to_dev_bf16(A), to_dev_bf16(B)
+    dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK
+    return dC.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,tile_m", [(16, 16), (32, 32), (5, 16), (20, 32), (1, 16)])
+@pytest.mark.parametrize("k_splits", [1, 4])
+def test_rowmajor_weights_integer_exact(M, tile_m, k_splits):
+    N, K = 1024, 1024
+    A, B = inputs.small_int_bf16(M, K, 11), inputs.small_int_bf16(K, N, 12)
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=tile_m,
+                                                                tile_n=128, k_splits=k_splits))
+    plan.reset_record()
+    for _ in range(2):                                      # second launch: arrival counters reset themselves
+        C = run_rowmajor(A, B, plan)
+        assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+    owner, count = plan.tile_record()
+    assert (count == 2).all()
+
+
+@pytest.mark.parametrize("shape", [(16, 8192, 8192, 16), (32, 4096, 4096, 8), (16, 1000, 520, 2), (7, 264, 72, 1)])
+def test_rowmajor_weights_uniform(shape):
+    M, N, K, ksp = shape
+    A, B = inputs.gemm_inputs(M, N, K, seed=31)
+    topo = device_topo()
+    for b in (37, topo.n_sm):
+        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
+                                                            tile_m=16 if M <= 16 else 32, tile_n=128, k_splits=ksp))
+        check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
+
+
+def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False):
+    topo = device_topo()
+    b = topo.n_sm if b is None else b
+    if integer:
+        A, B = inputs.small_int_bf16(M, K, seed), inputs.small_int_bf16(K, N, seed + 1)
+    else:
+        A, B = inputs.gemm_inputs(M, N, K, seed=seed)
+    kw = dict(M=M, N=N, K=K, tile_m=16 if M <= 16 else 32, tile_n=128, k_splits=ksp)
+    plan_d = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+    dst_bytes = 2 * K * N * 2 + (8 << 20)                    # two views, head-room for an uneven die split
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    dB = to_dev_bf16(B)
+    packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes)
+    return topo, A, B, kw, plan_d, dst, amap, packed
+
+
+def test_packing_matches_oracle_table_and_layout():
+    M, N, K, ksp = 16, 1024, 512, 2
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp)
+    tbl = amap.export()
+    o_plan = op.build_plan(topo.as_dict(), None, topo.n_sm, op.default_policy(kind=op.DIE_COMPACT, **kw))
+    assert plan_d.export().tobytes() == op.export(o_plan).tobytes()
+    page_die = op.page_die_from_plan(o_plan, K)
+    want_table = op.build_page_table(page_die, dict(chunk_bytes=4096, die_of_chunk=tbl))
+    got_table = packed.page_table()
+    assert np.array_equal(got_table, np.array(want_table, dtype=np.int32))
+    # every page sits on the die of its unit wherever the pair rule holds
+    on_die = tbl[got_table] == np.array(page_die)
+    assert on_die.mean() > 0.99
+    n_chunks = int(got_table.max()) + 1
+    want_img = op.pack_weights(B, want_table, n_chunks)
+    got_img = dst[: n_chunks * 4096].cpu().numpy().view(np.uint16).reshape(n_chunks, 2048)
+    assert np.array_equal(got_img, want_img)
+
+
+@pytest.mark.parametrize("M,N,K,ksp", [(16, 1024, 1024, 1), (16, 2048, 2048, 4), (32, 1024, 512, 2), (9, 1096, 256, 1)])
+def test_packed_gemm_integer_exact(M, N, K, ksp):
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp, integer=True)
+    dA = to_dev_bf16(A)
+    dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan_d)
+        torch.cuda.synchronize()
+        assert plan_d.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), og.gemm_blocked(A, B))
+
+
+def test_packed_gemm_full_size_affinity_and_inverted_plans():
+    """M=16, N=K=8192 (the decode-shaped configuration): local and deliberately remote assignment
+    compute the same C; the affinity policy over the page table rebuilds the packing plan."""
+    M, N, K, ksp = 16, 8192, 8192, 16
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp)
+    table = packed.page_table()
+    bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=table)
+    plan_a = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, b=bop, **kw))
+    plan_i = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
+    pa, pd, pi = plan_a.parsed(), plan_d.parsed(), plan_i.parsed()
+    assert np.array_equal(pa["die_q"], pd["die_q"]) and np.array_equal(pa["sm_q"], pd["sm_q"])
+    assert not np.array_equal(pi["die_q"], pd["die_q"])
+    ref = og.gemm_blocked(A, B)
+    dA = to_dev_bf16(A)
+    for plan in (plan_d, plan_a, plan_i):
+        dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        check_close(dC.cpu().numpy(), ref)
+
+
+def test_packed_rejects_foreign_map_and_shapes():
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(16, 512, 256, 1)
+    other = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    h = ag.C.c_void_p()
+    st = ag.lib().ag_pack_weights(to_dev_bf16(B).data_ptr(), 256, 512, plan_d.handle, amap.handle, other.data_ptr(),
+                                  other.numel(), ag.C.byref(h))
+    assert st == ag.AG_ERR_STALE_AMAP
+    dA = to_dev_bf16(A)
+    dC = torch.zeros((16, 512), dtype=torch.float32, device="cuda")
+    assert ag.lib().gemm_persistent_packed(dA.data_ptr(), packed.handle, dC.data_ptr(), 16, 512, 128, plan_d.handle,
+                                           None) == ag.AG_ERR_ARG
