@@ -283,6 +283,34 @@ void ag_packed_destroy(ag_packed_weights* w);
 ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* C, int M, int N, int K,
                                  const ag_plan* plan, void* cuda_stream);
 
+/*
+ * gemm_persistent_noalloc - the decode-shaped gemm_persistent (M <= 32, row-major B) for callers
+ * that cannot allocate device memory when they need the result.  (The paper has no counterpart;
+ * this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: a serving process whose own memory pool already owns all of the GPU's free memory,
+ * so that cudaMalloc fails; a latency-bound request loop where an allocator call is not
+ * acceptable; code that runs after a framework has declared "no more allocations".  The split-K
+ * partial sums and arrival counters, which normally live in memory that sched_build attached to
+ * the plan, are placed instead in a fixed workspace that is part of the library image: 8 MiB +
+ * 16 KiB of device memory on every GPU the library is loaded on, held until the process exits.
+ * The call itself performs no cudaMalloc, cudaFree or any other allocating call.
+ *
+ * Limits: k_splits * M * N * 4 bytes <= 8 MiB (for example M = 16, N = 8192, k_splits = 16) and
+ * N <= 131072; larger problems are refused with AG_ERR_ARG, as are plans that are not
+ * decode-shaped (tile_m > 32).  Arguments are those of gemm_persistent; the plan may come from a
+ * sched_build done at start-up, when allocation was still allowed.
+ *
+ * The first call on each device looks up the workspace's device address; make that first call
+ * outside any stream capture.  All calls on a device share the one workspace, which keeps
+ * whatever the previous call left in it (the counters are cleared on the given stream at the
+ * start of every call): two calls whose kernels may run at the same time on one GPU - different
+ * streams, or different host threads - race on it and give wrong results.  Serialise them.
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA; device-side status via ag_last_status.
+ */
+ag_status gemm_persistent_noalloc(const void* A, const void* B, void* C, int M, int N, int K,
+                                  const ag_plan* plan, void* cuda_stream);
+
 const char* ag_strerror(ag_status s);
 /* Last CUDA error code seen by the calling thread inside the library (0 = none). */
 int ag_last_cuda_error(void);

@@ -27,7 +27,7 @@ EXPORTED = [
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
     "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
-    "ag_packed_destroy", "gemm_persistent_packed", "ag_strerror", "ag_last_cuda_error",
+    "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_strerror", "ag_last_cuda_error",
     "ag_kernel_launch_count",
 ]
 
@@ -133,6 +133,7 @@ def lib() -> C.CDLL:
     L.ag_packed_destroy.argtypes = [vp]
     L.ag_packed_destroy.restype = None
     L.gemm_persistent_packed.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.gemm_persistent_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.ag_strerror.argtypes = [C.c_int]
     L.ag_strerror.restype = C.c_char_p
     L.ag_last_cuda_error.restype = C.c_int
@@ -380,3 +381,10 @@ def gemm_persistent_packed(a_ptr: int, packed: PackedWeights, c_ptr: int, M: int
                            stream: int = 0):
     _check(lib().gemm_persistent_packed(a_ptr, packed.handle, c_ptr, M, N, K, plan.handle, stream),
            "gemm_persistent_packed")
+
+
+def gemm_persistent_noalloc(a_ptr: int, b_ptr: int, c_ptr: int, M: int, N: int, K: int, plan: Plan, stream: int = 0):
+    """Decode-shaped GEMM (M <= 32) that takes its split-K workspace from the library's built-in
+    device array instead of allocated memory; for callers that may not allocate.  Calls on one GPU
+    must not overlap.  Limits: k_splits * M * N * 4 <= 8 MiB, N <= 131072."""
+    _check(lib().gemm_persistent_noalloc(a_ptr, b_ptr, c_ptr, M, N, K, plan.handle, stream), "gemm_persistent_noalloc")

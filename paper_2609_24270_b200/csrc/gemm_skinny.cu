@@ -430,3 +430,55 @@ extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weigh
     return gemm_skinny_dispatch(A, nullptr, W, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
                                 reinterpret_cast<cudaStream_t>(cuda_stream));
 }
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the decode-shaped GEMM.
+//
+// Some callers must not allocate device memory at the moment they need the GEMM: an inference
+// server that has handed every free byte of the GPU to its own arena (cudaMalloc simply fails
+// there), a request loop with a latency budget that an allocator call would break, or code
+// running between other libraries' strict "no allocation after start-up" phases.  For them the
+// split-K workspace lives in the library image itself: a fixed array in device memory that exists
+// on every GPU from the moment the library is loaded there until the process ends.
+//
+// The array's name is only a host-side handle; the address the kernel needs is asked from the
+// runtime once per device (cudaGetSymbolAddress, with that device current) and remembered.
+constexpr size_t kNoAllocSemBytes = 16 * 1024;                   // 4096 arrival counters = 1024 tiles of 128 columns
+constexpr size_t kNoAllocPartialBytes = 8u * 1024 * 1024;        // 2 Mi fp32 partial sums
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocSemBytes + kNoAllocPartialBytes];
+
+namespace {
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[64] = {nullptr};   // device address of g_noalloc_scratch, per device ordinal
+}  // namespace
+
+extern "C" ag_status gemm_persistent_noalloc(const void* A, const void* B, void* Cout, int M, int N, int K,
+                                             const ag_plan* plan, void* cuda_stream) {
+    if (!A || !B || !Cout || !plan) return AG_ERR_ARG;
+    const int32_t* h = plan->header;
+    if (h[H_TILE_M] > 32) return AG_ERR_ARG;  // only decode-shaped plans use a workspace
+    const int ksp = h[H_KSPLITS], tiles_n = h[H_TILES_N];
+    // limits of the built-in workspace
+    if ((size_t)tiles_n * 4 * sizeof(int) > kNoAllocSemBytes) return AG_ERR_ARG;
+    if (ksp > 1 && (size_t)ksp * (size_t)M * (size_t)N * sizeof(float) > kNoAllocPartialBytes) return AG_ERR_ARG;
+    int dev = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return AG_ERR_ARG;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ptr[dev]) {
+            // first call on this device: resolve the array's device address (not an allocation)
+            void* ptr = nullptr;
+            AG_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+            g_noalloc_ptr[dev] = ptr;
+        }
+        scratch = g_noalloc_ptr[dev];
+    }
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int* sem = reinterpret_cast<int*>(scratch);
+    float* partial = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + kNoAllocSemBytes);
+    // the counters must start at zero; whatever an earlier call left behind is wiped on the same stream
+    AG_CUDA(cudaMemsetAsync(sem, 0, (size_t)tiles_n * 4 * sizeof(int), stream));
+    return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, partial, sem, stream);
+}

@@ -1,0 +1,53 @@
+"""The allocation-free entry point: a server that has reserved all GPU memory for its own pool,
+or a request loop that must not call an allocator, still gets the decode-shaped GEMM, because its
+split-K workspace is a fixed array inside the library.  Checked here against the ordinary entry
+point on the same inputs, twice in a row (the workspace is shared and keeps old contents)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_24270_b200 import binding as ag
+from paper_2609_24270_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_noalloc_matches_regular_entry_point_twice():
+    M, N, K, ksp = 16, 2048, 2048, 4
+    topo = ag.topo_discover(ag.AG_TOPO_CENSUS | ag.AG_TOPO_LATENCY)
+    A, B = inputs.gemm_inputs(M, N, K, seed=5)
+    A2, B2 = inputs.gemm_inputs(M, N, K, seed=9)
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16,
+                                                                tile_n=128, k_splits=ksp))
+    stream = torch.cuda.current_stream().cuda_stream
+    for a_bits, b_bits in ((A, B), (A2, B2)):                 # two calls in a row, different data
+        dA = torch.from_numpy(a_bits.view(np.int16).copy()).cuda()
+        dB = torch.from_numpy(b_bits.view(np.int16).copy()).cuda()
+        c_ref = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        c_new = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), c_ref.data_ptr(), M, N, K, plan, stream)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        ag.gemm_persistent_noalloc(dA.data_ptr(), dB.data_ptr(), c_new.data_ptr(), M, N, K, plan, stream)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        ref = c_ref.cpu().numpy().astype(np.float64)
+        got = c_new.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        # same tolerance as the GEMM parity tests: relative Frobenius <= 1e-4, max abs <= 1e-2
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-4
+        assert np.abs(got - ref).max() <= 1e-2
+
+
+def test_noalloc_refuses_problems_beyond_the_builtin_workspace():
+    topo = ag.topo_discover(ag.AG_TOPO_CENSUS | ag.AG_TOPO_LATENCY)
+    M, N, K, ksp = 32, 8192, 4096, 16                         # 32 * 8192 * 16 * 4 B = 16 MiB > 8 MiB
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=32,
+                                                                tile_n=128, k_splits=ksp))
+    t = torch.zeros(K * N, dtype=torch.int16, device="cuda")
+    c = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    st = ag.lib().gemm_persistent_noalloc(t.data_ptr(), t.data_ptr(), c.data_ptr(), M, N, K, plan.handle, None)
+    assert st == ag.AG_ERR_ARG
+    dense = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(M=256, N=256, K=256))
+    st = ag.lib().gemm_persistent_noalloc(t.data_ptr(), t.data_ptr(), c.data_ptr(), 256, 256, 256, dense.handle, None)
+    assert st == ag.AG_ERR_ARG
