@@ -192,6 +192,11 @@ typedef struct {
     int32_t static_assign;   /* 1: static per-SM lists (the paper's mode); 0: CTAs pull from per-die queues */
     uint64_t seed;           /* oblivious only: 0 = lowest SM ids, else seeded random subset */
     int64_t min_margin;      /* affinity only: byte margins below this count as ties (0 = exact ties only) */
+    int32_t splitk_in_memory; /* decode-shaped plans with k_splits > 1: 0 = partial sums go through a
+                                 workspace and are added in ascending split order (bit-reproducible);
+                                 1 = C is zeroed and every unit adds its partial sums with reductions in
+                                 memory (no workspace, no waiting; the order of the fp32 adds is not fixed) */
+    int32_t reserved0;
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;
@@ -276,8 +281,9 @@ void ag_packed_destroy(ag_packed_weights* w);
  * same shapes with row-major B.
  *   A  device, M x K bf16 row-major, 16-byte aligned;  C  device, M x N fp32 row-major, overwritten
  *   plan  tile_m in {16, 32} (M <= tile_m), tile_n = 128, same N, K as the packing; with
- *         k_splits > 1 the partial sums go through the plan's workspace and are added in
- *         ascending split order by the block that finishes a tile last (deterministic)
+ *         k_splits > 1 the partial sums either go through the plan's workspace and are added in
+ *         ascending split order by the block that finishes a tile last, or are added straight
+ *         into a zeroed C by reductions in memory (policy.splitk_in_memory)
  * Asynchronous on cuda_stream.  Errors as gemm_persistent.
  */
 ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* C, int M, int N, int K,

@@ -98,23 +98,26 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     const uint64_t limit = p.wait_limit_ns;
 
     if (warp == 0) {
-        // ------------------------------------------------ scheduler + TMA producer (one lane)
-        if (lane == 0) {
-            UnitSource src(p, slot);
-            uint32_t it = 0, kit = 0;
-            bool ok = true;
-            while (ok) {
-                const int u = src.next();
+        // ------------------------------------------------ scheduler (warp-collective) + TMA producer (lane 0)
+        UnitSource src(p, slot);
+        uint32_t it = 0, kit = 0;
+        int ok = 1;
+        while (ok) {
+            const int u = src.next(lane);
+            if (lane == 0) {
                 const int r = it % kRing;
                 if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 1);
-                    ok = false;
-                    break;
+                    ok = 0;
+                } else {
+                    ctl->ring[r] = u;
+                    mbar_arrive(smem_u32(&ctl->sched_full[r]));
                 }
-                ctl->ring[r] = u;
-                mbar_arrive(smem_u32(&ctl->sched_full[r]));
-                ++it;
-                if (u < 0) break;
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ++it;
+            if (!ok || u < 0) break;
+            if (lane == 0) {
                 const int ks = u % p.k_splits, t = u / p.k_splits;
                 const int tm = t / p.tiles_n, tn = t % p.tiles_n;
                 const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
@@ -123,7 +126,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                     const int st = kit % C::stages;
                     if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / C::stages) & 1) ^ 1, abort_flag, limit)) {
                         report_timeout(p, 2);
-                        ok = false;
+                        ok = 0;
                         break;
                     }
                     const uint32_t bar = smem_u32(&ctl->full[st]);
@@ -134,14 +137,15 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                     for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tm_b, bar, tn * BN + j * 64, s * BK);
                 }
             }
-            if (!ok) {
-                // gave up: let the copies already in flight land before the block leaves
-                const uint32_t n_out = kit < (uint32_t)C::stages ? kit : (uint32_t)C::stages;
-                for (uint32_t j = 0; j < n_out; ++j) {
-                    const uint32_t k2 = kit - 1 - j;
-                    int dummy = 0;
-                    mbar_wait(smem_u32(&ctl->full[k2 % C::stages]), (k2 / C::stages) & 1, &dummy, 2000000ull);
-                }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+        if (!ok && lane == 0) {
+            // gave up: let the copies already in flight land before the block leaves
+            const uint32_t n_out = kit < (uint32_t)C::stages ? kit : (uint32_t)C::stages;
+            for (uint32_t j = 0; j < n_out; ++j) {
+                const uint32_t k2 = kit - 1 - j;
+                int dummy = 0;
+                mbar_wait(smem_u32(&ctl->full[k2 % C::stages]), (k2 / C::stages) & 1, &dummy, 2000000ull);
             }
         }
     } else if (warp == 1) {

@@ -22,12 +22,18 @@ namespace ag {
 
 constexpr int SK_BN = 128;     // weight columns per unit
 constexpr int SK_BK = 64;      // k-slab
-constexpr int SK_STAGES = 10;
+// Six stages (about 110 KB in flight per SM) already cover bandwidth x latency several times; a deeper
+// ring only lengthens the queues in the memory system, and with them every dependent round trip
+// (fence, arrival atomic, reduction loads).
+constexpr int SK_STAGES = 6;
 constexpr int SK_W_BYTES = SK_BN * SK_BK * 2;      // 16 KB of weights per stage
 constexpr int SK_A_BYTES = 32 * SK_BK * 2;         // room for 32 activation rows
 constexpr int SK_STAGE_BYTES = SK_W_BYTES + SK_A_BYTES;
 constexpr int SK_SMEM_BYTES = SK_STAGES * SK_STAGE_BYTES + 1024 + 1024;
-constexpr int SK_TMEM_COLS = 64;                   // two accumulators of 32 columns
+// An MMA with so few columns finishes its arithmetic in a few cycles but a following MMA that adds to the
+// same accumulator has to wait for its result (measured: ~370 cycles per dependent K=16 step).  The
+// k-steps of a unit therefore rotate over SK_ACCS independent accumulators, summed in the epilogue.
+constexpr int SK_ACCS = 8;
 
 struct SkinnyCtl {
     uint64_t full[SK_STAGES];
@@ -61,6 +67,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
     SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + SK_STAGES * SK_STAGE_BYTES);
+    constexpr uint32_t kAccCols = SK_ACCS * NM;          // columns of one accumulator set
+    constexpr uint32_t kTmemCols = 2 * kAccCols;         // two sets: 256 (NM = 16) or 512 (NM = 32) columns
     volatile int* abort_flag = &ctl->abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int my_sm = (int)smid();
@@ -87,7 +95,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         if (!PACKED) prefetch_tmap(&tm_w);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&ctl->tmem_base), SK_TMEM_COLS);
+        tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -98,54 +106,73 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     constexpr uint32_t kTxBytes = SK_W_BYTES + NM * SK_BK * 2;
 
     if (warp == 0) {
-        if (lane == 0) {
-            UnitSource src(p, slot);
-            uint32_t it = 0, kit = 0;
-            bool ok = true;
-            while (ok) {
-                const int u = src.next();
+        // ------------------------------------------------ scheduler + producer.  Lane 0 waits and issues
+        // the copies; for packed weights all 32 lanes fetch the page-table entries of the next eight
+        // k-slabs (32 pages) with one load each, so the issuing lane never waits on a table lookup.
+        UnitSource src(p, slot);
+        const uint64_t stream_policy = l2_policy_evict_first();  // weights are read once: do not keep them in L2
+        uint32_t it = 0, kit = 0;
+        int ok = 1;
+        while (ok) {
+            const int u = src.next(lane);
+            if (lane == 0) {
                 const int r = it % kRing;
                 if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 1);
-                    ok = false;
-                    break;
-                }
-                ctl->ring[r] = u;
-                mbar_arrive(smem_u32(&ctl->sched_full[r]));
-                ++it;
-                if (u < 0) break;
-                const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
-                const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
-                const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
-                for (int s = s0; s < s1; ++s, ++kit) {
-                    const int st = kit % SK_STAGES;
-                    if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / SK_STAGES) & 1) ^ 1, abort_flag, limit)) {
-                        report_timeout(p, 2);
-                        ok = false;
-                        break;
-                    }
-                    const uint32_t bar = smem_u32(&ctl->full[st]);
-                    const uint32_t sw = base + st * SK_STAGE_BYTES, sa = sw + SK_W_BYTES;
-                    mbar_expect_tx(bar, kTxBytes);
-                    if (PACKED) {
-                        const int32_t* pt = x.page_table + (size_t)tn * x.pages_per_tile + s * 4;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            bulk_load(sw + i * 4096, x.packed + (size_t)pt[i] * AG_CHUNK_BYTES, 4096, bar);
-                    } else {
-                        tma_load_2d(sw, &tm_w, bar, tn * SK_BN, s * SK_BK);
-                        tma_load_2d(sw + 8192, &tm_w, bar, tn * SK_BN + 64, s * SK_BK);
-                    }
-                    tma_load_2d(sa, &tm_a, bar, s * SK_BK, 0);
+                    ok = 0;
+                } else {
+                    ctl->ring[r] = u;
+                    mbar_arrive(smem_u32(&ctl->sched_full[r]));
                 }
             }
-            if (!ok) {
-                const uint32_t n_out = kit < (uint32_t)SK_STAGES ? kit : (uint32_t)SK_STAGES;
-                for (uint32_t j = 0; j < n_out; ++j) {
-                    const uint32_t k2 = kit - 1 - j;
-                    int dummy = 0;
-                    mbar_wait(smem_u32(&ctl->full[k2 % SK_STAGES]), (k2 / SK_STAGES) & 1, &dummy, 2000000ull);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ++it;
+            if (!ok || u < 0) break;
+            const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
+            const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
+            const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+            for (int sb = s0; sb < s1 && ok; sb += 8) {
+                int my_page = 0;
+                if (PACKED) {
+                    const int pg = sb * 4 + lane;
+                    if (pg < s1 * 4) my_page = x.page_table[(size_t)tn * x.pages_per_tile + pg];
                 }
+                const int se = min(s1, sb + 8);
+                for (int s = sb; s < se; ++s, ++kit) {
+                    const int st = kit % SK_STAGES;
+                    const uint32_t bar = smem_u32(&ctl->full[st]);
+                    const uint32_t sw = base + st * SK_STAGE_BYTES, sa = sw + SK_W_BYTES;
+                    if (lane == 0) {
+                        if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / SK_STAGES) & 1) ^ 1, abort_flag, limit)) {
+                            report_timeout(p, 2);
+                            ok = 0;
+                        } else {
+                            mbar_expect_tx(bar, kTxBytes);
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    if (PACKED) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + i);
+                            if (lane == 0) bulk_load_hint(sw + i * 4096, x.packed + (size_t)page * AG_CHUNK_BYTES, 4096, bar, stream_policy);
+                        }
+                    } else if (lane == 0) {
+                        tma_load_2d_hint(sw, &tm_w, bar, tn * SK_BN, s * SK_BK, stream_policy);
+                        tma_load_2d_hint(sw + 8192, &tm_w, bar, tn * SK_BN + 64, s * SK_BK, stream_policy);
+                    }
+                    if (lane == 0) tma_load_2d(sa, &tm_a, bar, s * SK_BK, 0);
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            // gave up: let the copies already in flight land before the block leaves
+            const uint32_t n_out = kit < (uint32_t)SK_STAGES ? kit : (uint32_t)SK_STAGES;
+            for (uint32_t j = 0; j < n_out; ++j) {
+                const uint32_t k2 = kit - 1 - j;
+                int dummy = 0;
+                mbar_wait(smem_u32(&ctl->full[k2 % SK_STAGES]), (k2 / SK_STAGES) & 1, &dummy, 2000000ull);
             }
         }
     } else if (warp == 1) {
@@ -171,7 +198,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * 32;
+                const uint32_t d_tmem = tmem_base + acc * kAccCols;
                 for (int s = s0; s < s1; ++s, ++kit) {
                     const int st = kit % SK_STAGES;
                     if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / SK_STAGES) & 1, abort_flag, limit)) {
@@ -188,7 +215,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         const uint64_t dw = PACKED ? make_smem_desc(sw + k4 * 4096, 128, 256, 0)
                                                    : make_smem_desc(sw + k4 * 2048, 8192, 1024, 2);
                         const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
-                        tc_mma_f16(d_tmem, dw, da, idesc, (s > s0 || k4 > 0) ? 1u : 0u);
+                        const int step = (s - s0) * 4 + k4;  // k-step of this unit -> accumulator step mod SK_ACCS
+                        tc_mma_f16(d_tmem + (step & (SK_ACCS - 1)) * NM, dw, da, idesc, step >= SK_ACCS ? 1u : 0u);
                     }
                     tc_commit(smem_u32(&ctl->empty[st]));
                 }
@@ -204,74 +232,143 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------ epilogue: lane = weight column n, registers = rows m
+        // Split-K hand-off, software-pipelined so that no memory round trip sits between two units:
+        //   unit i    its partial sums are stored;
+        //   unit i-1  (stores acknowledged long ago) fence, then the arrival counter of its 32 columns
+        //             is bumped with an atomic whose result is not looked at yet;
+        //   unit i-2  the atomic's result is read: the warp that completed the last of the k_splits
+        //             partial sums adds them in ascending split order and writes C.
+        // Each epilogue warp owns 32 columns of a tile and its own counter; no barrier between warps.
         const int q = warp & 3;
-        uint32_t tile_it = 0;
-        for (uint32_t it = 0;; ++it) {
+        uint32_t tile_it = 0, it = 0;
+        int st_tn = -1;              // unit whose partial sums are stored but not yet announced
+        int at_tn = -1;              // unit whose arrival atomic is in flight
+        int oldA = 0, oldB = 0;      // results of the arrival atomics (lane 0), used one unit later
+
+        auto reduce_columns = [&](int tn) {
+            __threadfence();
+            // lane = (row group lane/8, four columns); the k_splits loads of one output quad are in flight
+            // together and are added in ascending split order
+            const int nq = tn * SK_BN + q * 32 + (lane & 7) * 4;
+            if (nq < p.N) {
+                for (int m = lane >> 3; m < p.M; m += 4) {
+                    float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int k0 = 0; k0 < p.k_splits; k0 += 16) {
+                        float4 t[16];
+#pragma unroll
+                        for (int k = 0; k < 16; ++k)
+                            if (k0 + k < p.k_splits)
+                                t[k] = __ldcg(reinterpret_cast<const float4*>(
+                                    x.partial + ((size_t)(k0 + k) * p.M + m) * p.N + nq));
+#pragma unroll
+                        for (int k = 0; k < 16; ++k)
+                            if (k0 + k < p.k_splits) {
+                                acc4.x += t[k].x; acc4.y += t[k].y; acc4.z += t[k].z; acc4.w += t[k].w;
+                            }
+                    }
+                    *reinterpret_cast<float4*>(x.C + (size_t)m * p.N + nq) = acc4;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) x.sem[tn * 4 + q] = 0;  // ready for the next launch
+        };
+        // announce the stored unit (atomic result lands in old_new), resolve the one announced before
+        auto hand_off = [&](int& old_use, int& old_new) {
+            const int announce = st_tn, resolve = at_tn;
+            if (announce >= 0) {
+                __threadfence();
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("atom.global.add.u32 %0, [%1], 1;" : "=r"(old_new) : "l"(x.sem + announce * 4 + q) : "memory");
+            }
+            if (resolve >= 0) {
+                const int last = __shfl_sync(0xffffffffu, old_use == p.k_splits - 1, 0);
+                if (last) reduce_columns(resolve);
+            }
+            at_tn = announce;
+            st_tn = -1;
+        };
+        // one unit; returns false when the list is finished (or a wait ran out)
+        auto one_unit = [&](int& old_use, int& old_new) -> bool {
             const int r = it % kRing;
             if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 6);
-                break;
+                return false;
             }
             const int u = ctl->ring[r];
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
-            if (u < 0) break;
+            ++it;
+            if (u < 0) return false;
             const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
             const uint32_t acc = tile_it & 1;
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 7);
-                break;
+                return false;
             }
             tc_fence_after();
-            uint32_t v[NM];
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 32;
-            if constexpr (NM == 16) tmem_ld_32x16(taddr, v); else tmem_ld_32x32(taddr, v);
-            tmem_ld_wait();
+            // sum the accumulators that this unit used
+            const int s0e = min(p.kslabs_total, ks * p.kslabs_per_split);
+            const int s1e = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+            const int n_used = min(SK_ACCS, (s1e - s0e) * 4);
+            float sum[NM];
+#pragma unroll
+            for (int m = 0; m < NM; ++m) sum[m] = 0.f;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
+            for (int j = 0; j < n_used; ++j) {
+                uint32_t v[NM];
+                if constexpr (NM == 16) tmem_ld_32x16(taddr + j * NM, v); else tmem_ld_32x32(taddr + j * NM, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int m = 0; m < NM; ++m) sum[m] += __uint_as_float(v[m]);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+            ++tile_it;
             const int n = tn * SK_BN + q * 32 + lane;
-            float* out = p.k_splits > 1 ? x.partial + (size_t)ks * p.M * p.N : x.C;
-            if (n < p.N) {
+            if (p.k_splits > 1 && x.partial == nullptr) {
+                // in-memory reduction: C was zeroed before the launch, every unit adds its partial sums
+                // with reductions that L2 carries out; nothing comes back, so nothing is waited for
+                if (n < p.N) {
 #pragma unroll
-                for (int m = 0; m < NM; ++m)
-                    if (m < p.M) out[(size_t)m * p.N + n] = __uint_as_float(v[m]);
-            }
-            if (p.k_splits > 1) {
-                // Each epilogue warp owns 32 columns of the tile and keeps its own arrival counter: the
-                // warp that completes the last of the k_splits partial sums of those columns adds them
-                // in ascending split order.  No barrier between warps is needed.
-                __threadfence();
-                __syncwarp();
-                int last = 0;
-                if (lane == 0) last = atomicAdd(&x.sem[tn * 4 + q], 1) == p.k_splits - 1;
-                last = __shfl_sync(0xffffffffu, last, 0);
-                if (last) {
-                    __threadfence();
-                    if (n < p.N) {
-                        for (int m = 0; m < p.M; ++m) {
-                            float s = 0.f;
-                            for (int k = 0; k < p.k_splits; ++k)
-                                s += __ldcg(x.partial + ((size_t)k * p.M + m) * p.N + n);
-                            x.C[(size_t)m * p.N + n] = s;
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) x.sem[tn * 4 + q] = 0;  // ready for the next launch
+                    for (int m = 0; m < NM; ++m)
+                        if (m < p.M) atomicAdd(x.C + (size_t)m * p.N + n, sum[m]);
                 }
+            } else {
+                if (p.k_splits > 1) hand_off(old_use, old_new);
+                float* out = p.k_splits > 1 ? x.partial + (size_t)ks * p.M * p.N : x.C;
+                if (n < p.N) {
+#pragma unroll
+                    for (int m = 0; m < NM; ++m)
+                        if (m < p.M) out[(size_t)m * p.N + n] = sum[m];
+                }
+                if (p.k_splits > 1) st_tn = tn;
             }
             if (lane == 0 && q == 0) {
                 p.tile_owner[u] = my_sm;
                 atomicAdd(&p.tile_count[u], 1);
             }
-            ++tile_it;
+            return true;
+        };
+        // two copies of the step with the roles of oldA / oldB swapped: the atomic's result register is
+        // never copied, so nothing waits for it before the step that needs it
+        int which = 0;
+        while (true) {
+            if (!one_unit(oldA, oldB)) { which = 0; break; }
+            if (!one_unit(oldB, oldA)) { which = 1; break; }
+        }
+        if (p.k_splits > 1 && x.partial != nullptr && !*abort_flag) {
+            // drain: `which` = 0 means the atomic in flight wrote oldA (next result goes to oldB)
+            if (which == 0) { hand_off(oldA, oldB); hand_off(oldB, oldA); }
+            else            { hand_off(oldB, oldA); hand_off(oldA, oldB); }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, SK_TMEM_COLS);
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -321,7 +418,6 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     if (h[H_TILE_N] != SK_BN || (h[H_TILE_M] != 16 && h[H_TILE_M] != 32) || M > h[H_TILE_M]) return AG_ERR_ARG;
     if (plan->policy.k_unit != SK_BK || (K % 8) || (N % 8)) return AG_ERR_ARG;
     if (((uintptr_t)A | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
-    if (h[H_KSPLITS] > 1 && (!partial || !sem)) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
     int dev = 0, n_sm = 0;
@@ -346,6 +442,8 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
         if (!B_rowmajor || ((uintptr_t)B_rowmajor & 15u)) return AG_ERR_ARG;
         if (!encode_2d(&tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_rowmajor, K, N, 64, SK_BK)) return AG_ERR_CUDA;
     }
+    if (h[H_KSPLITS] > 1 && !x.partial)  // in-memory reduction mode: the adds need a zeroed C
+        AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * (size_t)M * (size_t)N, stream));
     const PersistParams gp = make_persist_params(plan, M, N, K);
     if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream)
                            : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream);

@@ -72,7 +72,8 @@ __device__ inline int join_plan(const PersistParams& p, int* s_member) {
     return *s_member ? slot : -1;
 }
 
-// Source of work units for one block; lives in the registers of the scheduler lane.
+// Source of work units for one block.  Warp-collective: every lane of the scheduler warp holds the
+// same state and calls next() together; atomics are done by lane 0 and broadcast.
 struct UnitSource {
     const PersistParams& p;
     PlanLayout lay;
@@ -86,35 +87,43 @@ struct UnitSource {
         dyn_die = p.image[lay.sm_die() + slot];
     }
     // next unit id, or -1 when there is nothing left for this block
-    __device__ int next() {
+    __device__ int next(int lane) {
         if (p.static_assign) {
             while (true) {
                 if (idx < list_len) return p.image[lay.sm_q() + list_off + idx++];
-                // own list done: run the list of any planned SM that never got a block
-                bool adopted = false;
-                for (; scan < p.b; ++scan) {
-                    if (*reinterpret_cast<volatile unsigned int*>(&p.ctrl->claimed[scan]) == p.epoch) continue;
-                    if (atomicMax(&p.ctrl->claimed[scan], p.epoch) < p.epoch) {
-                        list_off = p.image[lay.sm_q_off() + scan];
-                        list_len = p.image[lay.sm_q_off() + scan + 1] - list_off;
-                        idx = 0;
-                        atomicAdd(&p.ctrl->adopted, 1u);
-                        adopted = true;
-                        ++scan;
-                        break;
-                    }
+                // Own list done: look for a planned SM that never got a block and run its list.  The 32
+                // lanes check 32 claim flags at a time (a serial scan would cost one L2 round trip each).
+                int cand = -1;
+                for (; scan < p.b; scan += 32) {
+                    const int i = scan + lane;
+                    const bool unclaimed =
+                        i < p.b && *reinterpret_cast<volatile unsigned int*>(&p.ctrl->claimed[i]) != p.epoch;
+                    const unsigned m = __ballot_sync(0xffffffffu, unclaimed);
+                    if (m) { cand = scan + __ffs(m) - 1; break; }
                 }
-                if (!adopted) return -1;
+                if (cand < 0) return -1;
+                int got = 0;
+                if (lane == 0) got = atomicMax(&p.ctrl->claimed[cand], p.epoch) < p.epoch;
+                got = __shfl_sync(0xffffffffu, got, 0);
+                if (got) {
+                    list_off = p.image[lay.sm_q_off() + cand];
+                    list_len = p.image[lay.sm_q_off() + cand + 1] - list_off;
+                    idx = 0;
+                    if (lane == 0) atomicAdd(&p.ctrl->adopted, 1u);
+                }
             }
         }
-        for (int t = 0; t < 2; ++t) {
-            const int q_off = p.image[lay.die_q_off() + dyn_die];
-            const int q_len = p.image[lay.die_q_off() + dyn_die + 1] - q_off;
-            const int e = pop_queue(&p.ctrl->die_head[dyn_die], p.epoch, q_len);
-            if (e >= 0) return p.image[lay.die_q() + q_off + e];
-            dyn_die ^= 1;  // own die drained: help the other one
+        int u = -1;
+        if (lane == 0) {
+            for (int t = 0; t < 2 && u < 0; ++t) {
+                const int q_off = p.image[lay.die_q_off() + dyn_die];
+                const int q_len = p.image[lay.die_q_off() + dyn_die + 1] - q_off;
+                const int e = pop_queue(&p.ctrl->die_head[dyn_die], p.epoch, q_len);
+                if (e >= 0) u = p.image[lay.die_q() + q_off + e];
+                else dyn_die ^= 1;  // own die drained: help the other one
+            }
         }
-        return -1;
+        return __shfl_sync(0xffffffffu, u, 0);
     }
 };
 

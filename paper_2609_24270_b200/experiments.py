@@ -1,0 +1,265 @@
+"""Measurements for the workload configurations other than the headline one (which bench.py times).
+
+    python -m paper_2609_24270_b200.experiments --config 3 [--out results.jsonl]
+    python -m paper_2609_24270_b200.experiments --config 4
+    python -m paper_2609_24270_b200.experiments --config 5
+    python -m paper_2609_24270_b200.experiments --config raster      # raster-group sweep at 8192^3
+
+Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
+launches first, median of the timed launches.  torch is used for device memory, streams and events.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+import numpy as np
+import torch
+
+from . import binding as ag
+from . import inputs
+
+
+def emit(rec, fh):
+    line = json.dumps(rec)
+    print(line, flush=True)
+    if fh:
+        fh.write(line + "\n")
+        fh.flush()
+
+
+def dev_bf16(bits):
+    return torch.from_numpy(bits.view(np.int16).copy()).cuda()
+
+
+def time_launches(fn, warmup=3, iters=10, stream=None):
+    stream = stream or torch.cuda.current_stream()
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    evs[0].record(stream)
+    for i in range(iters):
+        fn()
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    return [evs[i].elapsed_time(evs[i + 1]) for i in range(iters)]
+
+
+def sm_set_summary(topo, plan):
+    p = plan.parsed()
+    sms = [int(s) for s in p["sm_list"]]
+    die = [int(d) for d in p["die_sm_count"]]
+    gpcs = np.bincount([topo.gpc[s] for s in sms if topo.gpc[s] >= 0], minlength=max(topo.n_gpc, 1))
+    return dict(die_sm_count=die, gpc_sm_count=[int(x) for x in gpcs])
+
+
+# ---------------------------------------------------------------------------------------------
+def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
+    """M=N=K=4096 on SM budgets; 32 seeded random subsets and the die_compact subset per budget."""
+    M = N = K = 4096
+    A, B = inputs.gemm_inputs(M, N, K)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    flops = 2.0 * M * N * K
+    for b in budgets:
+        res = {}
+        plans = {f"random_{s}": ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, seed=s, M=M, N=N, K=K,
+                                                                            raster_group=8))
+                 for s in range(1, n_subsets + 1)}
+        plans["lowest_ids"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, M=M, N=N, K=K, raster_group=8))
+        plans["die_compact"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
+                                                                            raster_group=8))
+        # two passes over all subsets so that clock drift is shared
+        acc = {n: [] for n in plans}
+        for _ in range(2):
+            for n, plan in plans.items():
+                acc[n] += time_launches(lambda: ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan),
+                                        warmup=2, iters=5)
+        for n in plans:
+            res[n] = flops / (float(np.median(acc[n])) * 1e-3) / 1e12
+            assert plans[n].last_status() == ag.AG_OK
+        rnd = [res[f"random_{s}"] for s in range(1, n_subsets + 1)]
+        rank = 1 + sum(1 for v in rnd if v > res["die_compact"])
+        emit(dict(config=3, workload="dense GEMM 4096^3 bf16, 128x256 tiles", sm_budget=b,
+                  random_subsets_tflops=dict(min=min(rnd), max=max(rnd), median=float(np.median(rnd)),
+                                             spread_max_over_min=max(rnd) / min(rnd)),
+                  lowest_ids_tflops=res["lowest_ids"], die_compact_tflops=res["die_compact"],
+                  die_compact_rank_among_33=rank, die_compact_set=sm_set_summary(topo, plans["die_compact"]),
+                  peak_scaled_tflops=2250.0 * b / topo.n_sm, all_tflops=rnd), fh)
+
+
+# ---------------------------------------------------------------------------------------------
+def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
+    """M=16, N=K=8192 decode-shaped GEMM, weights die-packed; die-local vs remote assignment."""
+    M, N, K, ksp = 16, 8192, 8192, 16
+    A = inputs.uniform_bf16(M, K, inputs.DEFAULT_SEED)
+    dA = dev_bf16(A)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    algo_bytes = K * N * 2 + M * K * 2 + M * N * 4
+    kw = dict(M=M, N=N, K=K, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=1)
+    Bs = [dev_bf16(inputs.uniform_bf16(K, N, inputs.DEFAULT_SEED + 1 + i)) for i in range(n_buffers)]
+    dst_bytes = 2 * K * N * 2 + (8 << 20)
+    for b in budgets:
+        plan_local = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+        dsts, packs = [], []
+        for i in range(n_buffers):                      # rotate buffers so that no launch finds its weights in L2
+            dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+            packs.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
+            dsts.append(dst)
+        table = packs[0][0].page_table()
+        page_owner = np.repeat(_unit_die(plan_local), K // 16 // ksp)      # pages of a unit are consecutive
+        on_die = float((packs[0][1].export()[table] == page_owner).mean())
+        bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=table)
+        local_set = plan_local.parsed()["sm_list"]
+        n0 = int(plan_local.parsed()["die_sm_count"][0])
+        if b < topo.n_sm and (n0 == 0 or n0 == b):
+            # all SMs on one die: the remote case runs the same units from SMs of the other die
+            other = 1 - (0 if n0 == b else 1)
+            plan_remote = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, preferred_die=other, **kw))
+        else:
+            plan_remote = ag.sched_build(topo, packs[0][1], b, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
+        plan_obl = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
+        out = {}
+        for name, plan in (("die_local", plan_local), ("remote", plan_remote)):
+            state = {"i": 0}
+
+            def run():
+                pk = packs[state["i"] % n_buffers][0]
+                state["i"] += 1
+                ag.gemm_persistent_packed(dA.data_ptr(), pk, dC.data_ptr(), M, N, K, plan)
+            ms = time_launches(run, warmup=4, iters=24)
+            assert plan.last_status() == ag.AG_OK
+            out[name] = algo_bytes / (float(np.median(ms)) * 1e-3) / 1e9
+        for name, plan in (("rowmajor_oblivious", plan_obl), ("rowmajor_die_compact", plan_local)):
+            state = {"i": 0}
+
+            def run2():
+                wb = Bs[state["i"] % n_buffers]
+                state["i"] += 1
+                ag.gemm_persistent(dA.data_ptr(), wb.data_ptr(), dC.data_ptr(), M, N, K, plan)
+            ms = time_launches(run2, warmup=4, iters=24)
+            out[name] = algo_bytes / (float(np.median(ms)) * 1e-3) / 1e9
+        emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
+                  sm_budget=b, gbs=out, local_over_remote=out["die_local"] / out["remote"],
+                  pages_on_owner_die=on_die, local_set=sm_set_summary(topo, plan_local),
+                  remote_set=sm_set_summary(topo, plan_remote), algo_bytes=algo_bytes,
+                  hbm_peak_measured_gbs=6534.1), fh)
+        del packs, dsts
+
+
+def _unit_die(plan):
+    p = plan.parsed()
+    ud = np.zeros(p["n_units"], dtype=np.uint8)
+    ud[p["die_q"][int(p["die_q_off"][1]):]] = 1
+    return ud
+
+
+# ---------------------------------------------------------------------------------------------
+def config5(fh, topo):
+    """Prefill-like GEMM (8192x4096x4096) and decode-like GEMM (32x4096x4096 over 8 weight matrices)
+    on two streams and disjoint SM partitions; die-split against oblivious (lowest ids / the rest)."""
+    Mp, Md, N, K = 8192, 32, 4096, 4096
+    Ap, Bp = inputs.gemm_inputs(Mp, N, K)
+    dAp, dBp = dev_bf16(Ap), dev_bf16(Bp)
+    dCp = torch.empty((Mp, N), dtype=torch.float32, device="cuda")
+    Ad = inputs.uniform_bf16(Md, K, 77)
+    dAd = dev_bf16(Ad)
+    Wd = [dev_bf16(inputs.uniform_bf16(K, N, 100 + i)) for i in range(8)]
+    dCd = torch.empty((Md, N), dtype=torch.float32, device="cuda")
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    flops_p = 2.0 * Mp * N * K
+    bytes_d = K * N * 2 + Md * K * 2 + Md * N * 4
+    pre_kw = dict(M=Mp, N=N, K=K, tile_m=128, tile_n=256, raster_group=8)
+    dec_kw = dict(M=Md, N=N, K=K, tile_m=32, tile_n=128, k_splits=8, splitk_in_memory=1)
+    for split in ((74, 74), (110, 38)):
+        for mode in ("die_split", "oblivious"):
+            kind = ag.AG_DIE_COMPACT if mode == "die_split" else ag.AG_OBLIVIOUS
+            plan_p = ag.sched_build(topo, None, split[0], ag.make_policy(kind=kind, preferred_die=0, **pre_kw))
+            taken = [int(s) for s in plan_p.parsed()["sm_list"]]
+            plan_d = ag.sched_build(topo, None, split[1], ag.make_policy(kind=kind, avoid=taken, **dec_kw))
+            n_pre, n_dec = 6, 6 * 8 * 4
+
+            def pre():
+                ag.gemm_persistent(dAp.data_ptr(), dBp.data_ptr(), dCp.data_ptr(), Mp, N, K, plan_p, s1.cuda_stream)
+
+            def dec(i):
+                ag.gemm_persistent(dAd.data_ptr(), Wd[i % 8].data_ptr(), dCd.data_ptr(), Md, N, K, plan_d, s2.cuda_stream)
+
+            def run(do_pre, do_dec):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                torch.cuda.synchronize()
+                if do_pre:
+                    ev[0].record(s1)
+                if do_dec:
+                    ev[2].record(s2)
+                # interleave the launches so that both streams are fed from the start
+                for i in range(max(n_pre, n_dec)):
+                    if do_pre and i < n_pre:
+                        pre()
+                    if do_dec and i < n_dec:
+                        dec(i)
+                if do_pre:
+                    ev[1].record(s1)
+                if do_dec:
+                    ev[3].record(s2)
+                torch.cuda.synchronize()
+                tp = ev[0].elapsed_time(ev[1]) / n_pre if do_pre else None
+                td = ev[2].elapsed_time(ev[3]) / n_dec if do_dec else None
+                return tp, td
+
+            for _ in range(2):
+                run(True, True)
+            alone_p = np.median([run(True, False)[0] for _ in range(3)])
+            alone_d = np.median([run(False, True)[1] for _ in range(3)])
+            both = [run(True, True) for _ in range(5)]
+            ov_p = np.median([x[0] for x in both])
+            ov_d = np.median([x[1] for x in both])
+            assert plan_p.last_status() == ag.AG_OK and plan_d.last_status() == ag.AG_OK
+            emit(dict(config=5, split=list(split), partition=mode,
+                      prefill_tflops=dict(alone=flops_p / (alone_p * 1e-3) / 1e12, overlapped=flops_p / (ov_p * 1e-3) / 1e12),
+                      decode_gbs=dict(alone=bytes_d / (alone_d * 1e-3) / 1e9, overlapped=bytes_d / (ov_d * 1e-3) / 1e9),
+                      prefill_set=sm_set_summary(topo, plan_p), decode_set=sm_set_summary(topo, plan_d),
+                      note="decode time per GEMM includes the hand-over between back-to-back launches"), fh)
+
+
+# ---------------------------------------------------------------------------------------------
+def raster(fh, topo):
+    M = N = K = 8192
+    A, B = inputs.gemm_inputs(M, N, K)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    flops = 2.0 * M * N * K
+    plans = {}
+    for g in (1, 2, 4, 8, 16, 32, 64):
+        for kind, name in ((ag.AG_OBLIVIOUS, "oblivious"), (ag.AG_DIE_COMPACT, "die_compact")):
+            for static in (1, 0):
+                plans[(g, name, static)] = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(
+                    kind=kind, M=M, N=N, K=K, raster_group=g, static_assign=static))
+    acc = {k: [] for k in plans}
+    for _ in range(3):
+        for k, plan in plans.items():
+            acc[k] += time_launches(lambda: ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan),
+                                    warmup=2, iters=6)
+    for (g, name, static), v in acc.items():
+        emit(dict(config="raster", raster_group=g, policy=name, static_assign=static,
+                  tflops=flops / (float(np.median(v)) * 1e-3) / 1e12), fh)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", required=True)
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args()
+    fh = open(args.out, "a") if args.out else None
+    topo = ag.topo_discover()
+    emit(dict(config="topology", n_sm=topo.n_sm, die_sm_count=list(topo.die_sm_count),
+              gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
+              lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
+    {"3": config3, "4": config4, "5": config5, "raster": raster}[args.config](fh, topo)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -41,14 +41,31 @@ def test_rowmajor_weights_integer_exact(M, tile_m, k_splits):
 
 
 @pytest.mark.parametrize("shape", [(16, 8192, 8192, 16), (32, 4096, 4096, 8), (16, 1000, 520, 2), (7, 264, 72, 1)])
-def test_rowmajor_weights_uniform(shape):
+@pytest.mark.parametrize("in_memory", [0, 1])
+def test_rowmajor_weights_uniform(shape, in_memory):
     M, N, K, ksp = shape
     A, B = inputs.gemm_inputs(M, N, K, seed=31)
     topo = device_topo()
     for b in (37, topo.n_sm):
-        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
+        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, splitk_in_memory=in_memory,
                                                             tile_m=16 if M <= 16 else 32, tile_n=128, k_splits=ksp))
-        check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
+        for _ in range(2):
+            check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
+
+
+def test_in_memory_splitk_integer_exact_packed_and_rowmajor():
+    M, N, K, ksp = 16, 2048, 2048, 8
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp, integer=True)
+    plan_m = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, splitk_in_memory=1, **kw))
+    dA, dB = to_dev_bf16(A), to_dev_bf16(B)
+    ref = og.gemm_blocked(A, B)
+    for _ in range(2):
+        dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan_m)
+        torch.cuda.synchronize()
+        assert plan_m.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), ref)
+        assert np.array_equal(run_rowmajor(A, B, plan_m).astype(np.float64), ref)
 
 
 def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False):
