@@ -27,17 +27,18 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 M = N = K = 8192
-TILE_M, TILE_N = 128, 256
-RASTER_GROUP = 16
+TILE_M, TILE_N = 128, 256      # output tile of one thread block
+UNIT_M = 256                    # two blocks (a cluster pair, tcgen05 cta_group::2) share a 256 x 256 unit
+RASTER_GROUP = 8                # unit rows per raster group
 # affinity margins below 1/8 of a unit's bytes (A panel + B panel + C tile) are treated as ties: with plain
 # row-major operands every unit is interleaved about half and half over the dies
-MIN_MARGIN = (TILE_M * K * 2 + TILE_N * K * 2 + TILE_M * TILE_N * 4) // 8
+MIN_MARGIN = (UNIT_M * K * 2 + TILE_N * K * 2 + UNIT_M * TILE_N * 4) // 8
 FLOPS = 2.0 * M * N * K
 METRIC = "bf16_gemm_tflops"
 UNIT = "TFLOP/s"
 # DRAM bytes per launch of the dominant kernel, from the ncu capture summarised in
-# profiles/gemm_persistent_8192.md (dram__bytes_read.sum 1.191 GB + dram__bytes_write.sum 0.255 GB).
-NCU_TRAFFIC_BYTES = 1.446e9
+# profiles/gemm_persistent_pair_8192.md (dram__bytes_read.sum + dram__bytes_write.sum).
+NCU_TRAFFIC_BYTES = None
 
 
 def load_peaks():
@@ -155,7 +156,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2609_24270_b200 import binding as ag
-    from paper_2609_24270_b200 import inputs
+    from paper_2609_24270_b200 import inputs, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -190,13 +191,15 @@ def main():
     t_aff = time.time() - t0
     ops = dict(a=dict(offset=a_off, row_stride=K * 2, elem_bytes=2), b=dict(offset=b_off, row_stride=N * 2, elem_bytes=2),
                c=dict(offset=c_off, row_stride=N * 4, elem_bytes=4))
-    base = dict(M=M, N=N, K=K, tile_m=TILE_M, tile_n=TILE_N)
+    base = dict(M=M, N=N, K=K, tile_m=UNIT_M, tile_n=TILE_N)
+    single = dict(M=M, N=N, K=K, tile_m=TILE_M, tile_n=TILE_N)
     t0 = time.time()
     plans = {
         "oblivious_raster": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, raster_group=1, **base)),
         "oblivious_grouped": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, raster_group=RASTER_GROUP, **base)),
         "die_compact": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, raster_group=RASTER_GROUP, **base)),
         "affinity": ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, raster_group=RASTER_GROUP, min_margin=MIN_MARGIN, **base, **ops)),
+        "die_compact_one_cta_tiles": ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, raster_group=16, **single)),
     }
     t_plan = time.time() - t0
     stream = torch.cuda.current_stream()
@@ -250,16 +253,30 @@ def main():
             torch.cuda.synchronize()
             per_policy[n] += [evs[i].elapsed_time(evs[i + 1]) for i in range(per_round)]
     side = {n: FLOPS / (float(np.median(v)) * 1e-3) / 1e12 for n, v in per_policy.items()}
+    # context only: the vendor library's GEMM on the same operands in the same power state (not on the product path)
+    cublas_tflops = None
+    try:
+        tA, tB = dA.view(torch.bfloat16), dB.view(torch.bfloat16)
+        tC = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        for _ in range(args.warmup):
+            torch.mm(tA, tB, out=tC)
+        torch.cuda.synchronize()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(21)]
+        evs[0].record(stream)
+        for i in range(20):
+            torch.mm(tA, tB, out=tC)
+            evs[i + 1].record(stream)
+        torch.cuda.synchronize()
+        cublas_tflops = FLOPS / (float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(20)])) * 1e-3) / 1e12
+        del tC
+    except Exception:
+        pass
     sampler = ClockSampler(local)
     sampler.start()
     total_ms, per, launches = timed(plans["affinity"], args.steps, args.warmup, sampler)
     clocks = sampler.stop()
-    ms_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_step], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-    value = world * FLOPS / (ms_step * 1e-3) / 1e12
+    value, ms_step = replicas.job_throughput(total_ms / args.steps, FLOPS, "cuda")
+    value /= 1e12
 
     # ---- end to end through the same call with host buffers: H2D of A and B, GEMM, D2H of C
     def e2e_step():
@@ -278,12 +295,8 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_val = world * FLOPS / (e2e_ms * 1e-3) / 1e12
+    e2e_val, e2e_ms = replicas.job_throughput(e0.elapsed_time(e1) / e2e_steps, FLOPS, "cuda")
+    e2e_val /= 1e12
 
     if rank != 0:
         if world > 1:
@@ -297,10 +310,12 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"dense GEMM M=N=K={M}, A,B bf16 row-major uniform[-1,1) seed {inputs.DEFAULT_SEED}, fp32 out, "
-                               f"{TILE_M}x{TILE_N} tiles, all {topo.n_sm} SMs, affinity policy, raster group {RASTER_GROUP}",
+                               f"{TILE_M}x{TILE_N} tile per thread block (block pairs share 256x256 units), all {topo.n_sm} SMs, "
+                               f"affinity policy, raster group {RASTER_GROUP}",
                    "l2": "inputs+output 512 MiB > 126 MB L2, no flush between iterations",
                    "replicas": "independent per GPU" if world > 1 else "single GPU"},
         "policies_tflops": side,
+        "context_cublas_bf16_out_tflops_same_run": cublas_tflops,
         "aware_over_oblivious_raster": side["affinity"] / side["oblivious_raster"],
         "die_sm_count": list(topo.die_sm_count), "gpc_sm_count": list(topo.gpc_sm_count[:topo.n_gpc]),
         "setup_s": {"topo_discover": t_topo, "affinity_probe": t_aff, "sched_build_x4": t_plan},
@@ -311,7 +326,7 @@ def main():
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES,
                      "peak_source": f"{peaks['source']} cuBLAS bf16 burst (sustained {peaks['bf16_tflops_sustained']})",
-                     "kernel": "k_gemm_persistent<256>", "kernel_ms": kernel_ms},
+                     "kernel": "k_gemm_persistent_pair", "kernel_ms": kernel_ms},
     }
     if not args.no_cpu_baseline:
         blk, dt, fl, cores = oracle_sample(A_h, B_h)

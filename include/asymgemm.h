@@ -103,6 +103,12 @@ ag_status ag_topo_from_observations(int32_t n_sm, const int32_t* cluster_sm, con
  */
 int32_t ag_topo_place_by_gain(const double* gain, int32_t n_candidates, double solo_bw);
 
+/* Keep a map in a file / read it back (the paper budgets up to a minute per GPU for discovery,
+ * Section 5.1.2).  Loading checks the file's magic, size and internal consistency; a map belongs
+ * to the GPU it was measured on (map->device).  Errors: AG_ERR_ARG. */
+ag_status ag_topo_save(const ag_topo_map* map, const char* path);
+ag_status ag_topo_load(const char* path, ag_topo_map* map);
+
 /*
  * ag_probe_latency_samples - raw access-latency samples from one SM: the measurement behind the
  * HBM and L2 latency histograms of Section 6.1.1 (kernels in the appendix).  Line r lies in
@@ -183,7 +189,8 @@ typedef struct {
 typedef struct {
     int32_t kind;            /* AG_OBLIVIOUS | AG_DIE_COMPACT | AG_AFFINITY */
     int32_t M, N, K;
-    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}; decode-shaped kernel: {16,32} x 128 */
+    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}, or 256 x 256 (two thread blocks per unit, only
+                                for plans that use every SM); decode-shaped kernel: {16,32} x 128 */
     int32_t k_splits;        /* >= 1, runs of whole k-slabs */
     int32_t k_unit;          /* elements per k-slab (64) */
     int32_t raster_group;    /* tile rows per raster group (>= 1) */
@@ -316,6 +323,14 @@ ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void
  */
 ag_status gemm_persistent_noalloc(const void* A, const void* B, void* C, int M, int N, int K,
                                   const ag_plan* plan, void* cuda_stream);
+
+/*
+ * ag_wait_probe - self test of the bounded device-side wait that every kernel of this library
+ * uses: one thread waits on a barrier that nothing signals, gives up after limit_ns
+ * (<= 1 second) and the call returns AG_ERR_TIMEOUT, with the time actually waited in *waited_ns
+ * (host, may be NULL).  The device stays usable.  Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA.
+ */
+ag_status ag_wait_probe(uint64_t limit_ns, uint64_t* waited_ns);
 
 const char* ag_strerror(ag_status s);
 /* Last CUDA error code seen by the calling thread inside the library (0 = none). */

@@ -35,7 +35,11 @@ Steps.
      descending order of (n_u * n_d mod b), tie -> lower die id.
   5. unit -> die:
        oblivious    R[i] goes to S[i mod b]; the unit's die is that SM's die;
-       die_compact  die 0 takes R[0..q_0), die 1 takes the rest (contiguous bands);
+       die_compact  every raster group (g tile rows) is cut in two in raster order: die 0 takes the
+                    first part, die 1 the rest, the cut placed so that after x units of the raster
+                    die 0 holds floor(x * q_0 / n_u) of them.  Both dies walk through the raster
+                    together and share the row panels of the group they are in, while each keeps its
+                    own column panels; with one single group this is two contiguous bands;
        affinity     margin m(u) = local_0(u) - local_1(u) where local_d counts the bytes of
                     the unit's A panel, B panel and C tile that sit in chunks of die d
                     (negated when invert_affinity); a margin with |m| < min_margin counts as 0
@@ -159,6 +163,15 @@ def quotas(n_u: int, n_d: list[int], b: int) -> list[int]:
 
 
 # ----------------------------------------------------------------------------- step 5 helpers
+def band_die(i: int, n_u: int, q0: int, group_len: int) -> int:
+    """Die that the die_compact rule gives raster index i (see step 5)."""
+    start = (i // group_len) * group_len
+    end = min(n_u, start + group_len)
+    cut = (end * q0) // n_u - (start * q0) // n_u       # die-0 units inside this raster group
+    return 0 if i - start < cut else 1
+
+
+
 def k_range(pol: dict, ks: int) -> tuple[int, int]:
     """Element range [k0, k1) of split ks: whole k-slabs, the first splits take the longer runs."""
     K, ku = pol["K"], pol["k_unit"]
@@ -248,8 +261,11 @@ def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
             sm_q[slot].append(u)
             die_q[sm_die[slot]].append(u)
     else:
+        group_len = max(1, pol["raster_group"]) * tiles_n * ksp
         if pol["kind"] == DIE_COMPACT:
-            die_q = [R[:q[0]], R[q[0]:]]
+            die_q = [[], []]
+            for i, u in enumerate(R):
+                die_q[band_die(i, n_u, q[0], group_len)].append(u)
         else:
             if amap is None:
                 raise ValueError("affinity policy needs an affinity map")
@@ -266,7 +282,7 @@ def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
                 elif m < 0:
                     pref = 1
                 else:
-                    pref = 0 if i < q[0] else 1
+                    pref = band_die(i, n_u, q[0], group_len)
                 items.append((-abs(m), i, u, pref))
             items.sort()
             got = [[], []]

@@ -27,7 +27,8 @@ EXPORTED = [
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
     "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
-    "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_strerror", "ag_last_cuda_error",
+    "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
+    "ag_topo_load", "ag_strerror", "ag_last_cuda_error",
     "ag_kernel_launch_count",
 ]
 
@@ -135,6 +136,9 @@ def lib() -> C.CDLL:
     L.ag_packed_destroy.restype = None
     L.gemm_persistent_packed.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.gemm_persistent_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.ag_wait_probe.argtypes = [C.c_uint64, C.POINTER(C.c_uint64)]
+    L.ag_topo_save.argtypes = [C.POINTER(TopoMap), C.c_char_p]
+    L.ag_topo_load.argtypes = [C.c_char_p, C.POINTER(TopoMap)]
     L.ag_strerror.argtypes = [C.c_int]
     L.ag_strerror.restype = C.c_char_p
     L.ag_last_cuda_error.restype = C.c_int
@@ -179,6 +183,23 @@ def topo_from_observations(n_sm: int, clusters: list[list[int]], lat: np.ndarray
     _check(lib().ag_topo_from_observations(n_sm, flat.ctypes.data if len(flat) else None, off.ctypes.data,
                                            len(clusters), lp, n_ref, C.byref(m)), "ag_topo_from_observations")
     return m
+
+
+def topo_save(topo: TopoMap, path: str):
+    _check(lib().ag_topo_save(C.byref(topo), path.encode()), "ag_topo_save")
+
+
+def topo_load(path: str) -> TopoMap:
+    m = TopoMap()
+    _check(lib().ag_topo_load(path.encode(), C.byref(m)), "ag_topo_load")
+    return m
+
+
+def wait_probe(limit_ns: int):
+    """Returns (status, waited_ns) of a device-side wait that is designed to run out."""
+    w = C.c_uint64()
+    st = lib().ag_wait_probe(limit_ns, C.byref(w))
+    return int(st), int(w.value)
 
 
 def topo_place_by_gain(gains, solo_bw: float) -> int:

@@ -324,6 +324,8 @@ static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream
 namespace ag {
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
                                int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream);
+ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, int N, int K, const ag_plan* plan,
+                             cudaStream_t stream);
 }
 
 using namespace ag;
@@ -336,6 +338,8 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
         return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
                                     reinterpret_cast<cudaStream_t>(cuda_stream));
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
+    if (h[H_TILE_M] == 256)  // 256 x 256 units: pairs of blocks, full-chip plans only
+        return gemm_pair_dispatch(A, B, Cout, M, N, K, plan, reinterpret_cast<cudaStream_t>(cuda_stream));
     if (h[H_TILE_M] != BM || (h[H_TILE_N] != 64 && h[H_TILE_N] != 128 && h[H_TILE_N] != 256)) return AG_ERR_ARG;
     if (plan->policy.k_unit != BK) return AG_ERR_ARG;
     if ((K % 8) || (N % 8)) return AG_ERR_ARG;

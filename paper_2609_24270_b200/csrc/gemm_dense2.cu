@@ -1,0 +1,383 @@
+// Two-CTA variant of the persistent dense GEMM (tcgen05 cta_group::2) for plans that use every SM.
+//
+// Two thread blocks form a cluster and compute one 256 x 256 output unit together: block r of
+// the pair holds rows [128 r, 128 r + 128) of the A tile and columns [128 r, 128 r + 128) of the
+// B tile in its own shared memory, the leader block (rank 0) issues one MMA per K = 16 step for
+// both, and every block ends up with its 128 x 256 part of the result in its own tensor memory.
+// Per SM a k-slab costs 32 KB of copies instead of 48 KB, which matters because a single SM's
+// TMA unit keeps only ~32 KB of copies in flight: the one-CTA kernel waits for data a fifth of
+// the time, this one does not.
+//
+// Pinning (Section 7.1.2 of the paper) works as in the one-CTA kernel: every block reads %smid and
+// takes the plan slot of its SM.  The two blocks of a pair tell each other their slots and walk the
+// two task lists in alternation, so every list of the plan is still run exactly once.  No copy is
+// multicast: each block loads its own halves; only the "stage is free" and "accumulator is ready"
+// signals of tcgen05.commit go to both blocks.
+#include <string.h>
+
+#include <mutex>
+
+#include "persist.cuh"
+
+namespace ag {
+
+constexpr int P_BM = 128;        // rows per block (256 per pair)
+constexpr int P_BN = 256;        // columns of the unit
+constexpr int P_BNH = 128;       // B columns held by one block
+constexpr int P_BK = 64;
+constexpr int P_STAGES = 6;
+constexpr int P_A_BYTES = P_BM * P_BK * 2;     // 16 KB
+constexpr int P_B_BYTES = P_BK * P_BNH * 2;    // 16 KB
+constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES;
+constexpr int P_EPI_BUF = 32 * 32 * 4;
+constexpr int P_EPI_BYTES = kEpiWarps * 2 * P_EPI_BUF;
+constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_EPI_BYTES + 1024 + 1024;
+constexpr int P_TMEM_COLS = 512;
+
+struct PairCtl {
+    uint64_t full[P_STAGES];       // leader's copy collects the bytes of both blocks
+    uint64_t empty[P_STAGES];      // signalled in both blocks by the leader's commit
+    uint64_t tmem_full[2];         // signalled in both blocks by the leader's commit
+    uint64_t tmem_empty[2];        // leader's copy: 8 arrivals (4 epilogue warps of each block)
+    uint64_t sched_full[kRing];
+    uint64_t sched_empty[kRing];
+    uint64_t mma_drain;
+    int ring[kRing];
+    uint32_t tmem_base;
+    int abort_flag;
+    int member;
+    int peer_slot;                 // written by the other block of the pair
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+// copy into this block's shared memory, completion bytes reported to a barrier that may sit in the peer block
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive on the barrier at this offset in both blocks of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+}
+
+// Unit sequence of a pair: the two task lists in alternation, the lower slot first.
+struct PairSource {
+    const int32_t* image;
+    int off[2], len[2], pos;
+    __device__ PairSource(const PersistParams& p, int slot_a, int slot_b) : image(p.image), pos(0) {
+        const PlanLayout lay{p.b, p.n_units, p.n_sm};
+        const int lo = min(slot_a, slot_b), hi = max(slot_a, slot_b);
+        off[0] = lay.sm_q() + p.image[lay.sm_q_off() + lo];
+        len[0] = p.image[lay.sm_q_off() + lo + 1] - p.image[lay.sm_q_off() + lo];
+        off[1] = lay.sm_q() + p.image[lay.sm_q_off() + hi];
+        len[1] = p.image[lay.sm_q_off() + hi + 1] - p.image[lay.sm_q_off() + hi];
+    }
+    __device__ int next() {
+        const int common = 2 * min(len[0], len[1]);
+        int u = -1;
+        if (pos < common) {
+            u = image[off[pos & 1] + (pos >> 1)];
+        } else {
+            const int longer = len[0] >= len[1] ? 0 : 1;
+            const int i = (common >> 1) + (pos - common);
+            if (i < len[longer]) u = image[off[longer] + i];
+        }
+        ++pos;
+        return u;
+    }
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                       const __grid_constant__ CUtensorMap tm_c, const PersistParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t s_epi = base + P_STAGES * P_STAGE_BYTES;
+    PairCtl* ctl = reinterpret_cast<PairCtl*>(smem + P_STAGES * P_STAGE_BYTES + P_EPI_BYTES);
+    volatile int* abort_flag = &ctl->abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int my_sm = (int)smid();
+    const PlanLayout lay{p.b, p.n_units, p.n_sm};
+
+    // take the slot of this SM (every SM is planned: the host only launches this kernel for full-chip plans)
+    const int slot = p.image[lay.smid_to_slot() + my_sm];
+    if (tid == 0) {
+        ctl->abort_flag = 0;
+        ctl->member = slot >= 0 && atomicMax(&p.ctrl->claimed[slot], p.epoch) < p.epoch;
+        for (int i = 0; i < P_STAGES; ++i) {
+            mbar_init(smem_u32(&ctl->full[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), 2 * kEpiWarps);
+        }
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(smem_u32(&ctl->sched_full[i]), 1);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps);
+        }
+        mbar_init(smem_u32(&ctl->mma_drain), 1);
+        mbar_fence_init();
+        prefetch_tmap(&tm_a);
+        prefetch_tmap(&tm_b);
+        prefetch_tmap(&tm_c);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), P_TMEM_COLS);   // all 512 columns: both blocks get the same base
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // both blocks are running and have their barriers set up; then tell the peer which slot this block
+    // holds (-1: it has none) and meet again
+    cluster_sync();
+    if (tid == 0) st_cluster_u32(map_to_cta(smem_u32(&ctl->peer_slot), rank ^ 1u), (uint32_t)(ctl->member ? slot : -1));
+    cluster_sync();
+    const int peer_slot = ctl->peer_slot;
+    const bool active = ctl->member && peer_slot >= 0;
+    if (!active && tid == 0 && (ctl->member || peer_slot >= 0))
+        atomicCAS(&p.ctrl->status, 0, (int)AG_ERR_UNMANNED_SM);  // half a pair cannot run this kernel
+    const uint32_t tmem_base = ctl->tmem_base;
+    const uint64_t limit = p.wait_limit_ns;
+
+    if (active) {
+        if (warp == 0) {
+            // ------------------------------------------------ scheduler + TMA producer (lane 0)
+            if (lane == 0) {
+                PairSource src(p, slot, peer_slot);
+                uint32_t it = 0, kit = 0;
+                bool ok = true;
+                while (ok) {
+                    const int u = src.next();
+                    const int r = it % kRing;
+                    if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                        report_timeout(p, 1);
+                        ok = false;
+                        break;
+                    }
+                    ctl->ring[r] = u;
+                    mbar_arrive(smem_u32(&ctl->sched_full[r]));
+                    ++it;
+                    if (u < 0) break;
+                    const int tm = u / p.tiles_n, tn = u % p.tiles_n;
+                    for (int s = 0; s < p.kslabs_total; ++s, ++kit) {
+                        const int st = kit % P_STAGES;
+                        if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / P_STAGES) & 1) ^ 1, abort_flag, limit)) {
+                            report_timeout(p, 2);
+                            ok = false;
+                            break;
+                        }
+                        // the leader's barrier counts the bytes of both blocks
+                        const uint32_t bar_leader = map_to_cta(smem_u32(&ctl->full[st]), 0);
+                        if (leader) mbar_expect_tx(smem_u32(&ctl->full[st]), 2 * P_STAGE_BYTES);
+                        const uint32_t sa = base + st * P_STAGE_BYTES, sb = sa + P_A_BYTES;
+                        tma_load_2d_pair(sa, &tm_a, bar_leader, s * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
+                        tma_load_2d_pair(sb, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH, s * P_BK);
+                        tma_load_2d_pair(sb + P_BK * 128, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH + 64, s * P_BK);
+                    }
+                }
+            }
+        } else if (warp == 1) {
+            if (lane == 0) {
+                // ------------------------------------------------ MMA issuer (leader) / ring consumer (peer)
+                constexpr uint32_t idesc = make_idesc_bf16(2 * P_BM, P_BN, 0, 1);
+                uint32_t kit = 0, tile_it = 0;
+                bool ok = true;
+                for (uint32_t it = 0; ok; ++it) {
+                    const int r = it % kRing;
+                    if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                        report_timeout(p, 3);
+                        break;
+                    }
+                    const int u = ctl->ring[r];
+                    mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                    if (u < 0) break;
+                    if (!leader) continue;
+                    const uint32_t acc = tile_it & 1;
+                    if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
+                        report_timeout(p, 4);
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * P_BN;
+                    for (int s = 0; s < p.kslabs_total; ++s, ++kit) {
+                        const int st = kit % P_STAGES;
+                        if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / P_STAGES) & 1, abort_flag, limit)) {
+                            report_timeout(p, 5);
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t sa = base + st * P_STAGE_BYTES, sb = sa + P_A_BYTES;
+#pragma unroll
+                        for (int k4 = 0; k4 < P_BK / 16; ++k4) {
+                            const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
+                            const uint64_t db = make_smem_desc(sb + k4 * 2048, P_BK * 128, 1024, 2);
+                            tc_mma_f16_pair(d_tmem, da, db, idesc, (s > 0 || k4 > 0) ? 1u : 0u);
+                        }
+                        tc_commit_pair(smem_u32(&ctl->empty[st]));
+                    }
+                    if (!ok) break;
+                    tc_commit_pair(smem_u32(&ctl->tmem_full[acc]));
+                    ++tile_it;
+                }
+                if (leader && *abort_flag) {
+                    tc_commit(smem_u32(&ctl->mma_drain));
+                    int dummy = 0;
+                    mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                }
+            }
+        } else {
+            // ------------------------------------------------ epilogue warps: this block's 128 rows of the unit
+            const int q = warp & 3;
+            const uint32_t buf0 = s_epi + (warp - 2) * 2 * P_EPI_BUF;
+            uint32_t tile_it = 0, chunk_it = 0;
+            for (uint32_t it = 0;; ++it) {
+                const int r = it % kRing;
+                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 6);
+                    break;
+                }
+                const int u = ctl->ring[r];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                if (u < 0) break;
+                const int tm = u / p.tiles_n, tn = u % p.tiles_n;
+                const uint32_t acc = tile_it & 1;
+                if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 7);
+                    break;
+                }
+                tc_fence_after();
+                const int row0 = tm * 2 * P_BM + (int)rank * P_BM + q * 32;
+#pragma unroll 1
+                for (int c = 0; c < P_BN / 32; ++c, ++chunk_it) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * P_BN + c * 32, v);
+                    tmem_ld_wait();
+                    const uint32_t buf = buf0 + (chunk_it & 1) * P_EPI_BUF;
+                    if (lane == 0) bulk_wait_read<1>();
+                    __syncwarp();
+                    const uint32_t rowaddr = buf + lane * 128;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t a = rowaddr + ((j ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v[4 * j]), "r"(v[4 * j + 1]),
+                                     "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
+                                     : "memory");
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int x = tn * P_BN + c * 32;
+                        if (x < p.N && row0 < p.M) tma_store_2d(&tm_c, buf, x, row0);
+                        bulk_commit();
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    // the leader issues the MMAs for both blocks: it must know that both have read this accumulator
+                    mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[acc]), 0));
+                    if (q == 0 && leader) {
+                        p.tile_owner[u] = my_sm;
+                        atomicAdd(&p.tile_count[u], 1);
+                    }
+                }
+                ++tile_it;
+            }
+            if (lane == 0) bulk_wait<0>();
+        }
+    }
+    // nobody leaves while the peer may still signal this block's barriers or read its shared memory
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, P_TMEM_COLS);
+    }
+}
+
+ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, int N, int K, const ag_plan* plan,
+                             cudaStream_t stream) {
+    const int32_t* h = plan->header;
+    if (h[H_TILE_M] != 2 * P_BM || h[H_TILE_N] != P_BN || h[H_KSPLITS] != 1 || !h[H_STATIC]) return AG_ERR_ARG;
+    if (plan->policy.k_unit != P_BK || (K % 8) || (N % 8)) return AG_ERR_ARG;
+    if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    int dev = 0, n_sm = 0;
+    AG_CUDA(cudaGetDevice(&dev));
+    AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    // pairs need every SM: a block whose partner sits on an unplanned SM could not run
+    if (n_sm != plan->lay.n_sm || plan->lay.b != n_sm || (n_sm & 1)) return AG_ERR_ARG;
+    if (plan->tm_a_ptr != A || plan->tm_b_ptr != B || plan->tm_c_ptr != Cout) {
+        if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)) return AG_ERR_CUDA;
+        if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_BK)) return AG_ERR_CUDA;
+        if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
+        plan->tm_a_ptr = A; plan->tm_b_ptr = B; plan->tm_c_ptr = Cout;
+    }
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(k_gemm_persistent_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    const PersistParams gp = make_persist_params(plan, M, N, K);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(n_sm);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = P_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair, plan->tm_a, plan->tm_b, plan->tm_c, gp));
+    count_launch();
+    return AG_OK;
+}
+
+}  // namespace ag

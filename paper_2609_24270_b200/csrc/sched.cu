@@ -51,6 +51,15 @@ __device__ inline int raster_unit(int i, int tiles_m, int tiles_n, int ksp, int 
     return (tm * tiles_n + tn) * ksp + ks;
 }
 
+// die_compact rule: every raster group is cut in two, die 0 first; after x units of the raster die 0
+// holds floor(x * q0 / n_units) of them.
+__device__ inline int band_die(int i, int n_units, int q0, int group_len) {
+    const int start = (i / group_len) * group_len;
+    const int end = min(n_units, start + group_len);
+    const int cut = (int)(((long long)end * q0) / n_units - ((long long)start * q0) / n_units);
+    return (i - start) < cut ? 0 : 1;
+}
+
 __device__ inline bool avoided(const PolicyDev& p, int s) { return (p.avoid[s >> 6] >> (s & 63)) & 1ull; }
 
 // ---- steps 2, 3, 4 and the header: one thread -------------------------------------------------
@@ -244,11 +253,12 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
     __syncthreads();
     const int q0 = image[lay.die_q_off() + 1];
     const int q[2] = {q0, n_units - q0};
+    const int group_len = pol.raster_group * tiles_n * pol.k_splits;
 
     if (pol.kind == AG_OBLIVIOUS) {
         for (int i = tid; i < n_units; i += nt) die_of[i] = image[lay.sm_die() + (i % b)];
     } else if (pol.kind == AG_DIE_COMPACT) {
-        for (int i = tid; i < n_units; i += nt) die_of[i] = i < q0 ? 0 : 1;
+        for (int i = tid; i < n_units; i += nt) die_of[i] = band_die(i, n_units, q0, group_len);
     } else {
         // rank of raster index i under the key (|m| descending, i ascending)
         for (int i = tid; i < n_units; i += nt) {
@@ -270,7 +280,7 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
                 long long m = margins[i];
                 if (pol.invert) m = -m;
                 if ((m < 0 ? -m : m) < pol.min_margin) m = 0;
-                const int pref = m > 0 ? 0 : (m < 0 ? 1 : (i < q0 ? 0 : 1));
+                const int pref = m > 0 ? 0 : (m < 0 ? 1 : band_die(i, n_units, q0, group_len));
                 const int d = got[pref] < q[pref] ? pref : 1 - pref;
                 got[d]++;
                 die_of[i] = d;

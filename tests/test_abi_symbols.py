@@ -103,3 +103,22 @@ def test_bandwidth_gain_rule():
     assert ag.topo_place_by_gain([200e9, 195e9, 199e9, 205e9], 200e9) == -1
     # two equally contended candidates: ambiguous
     assert ag.topo_place_by_gain([60e9, 61e9, 200e9], 200e9) == -1
+
+
+def test_topo_map_file_roundtrip(tmp_path):
+    topo = inputs.synthetic_topo(die0_sms=72, seed=3)
+    m = ag.TopoMap.from_dict(topo)
+    path = str(tmp_path / "topo.bin")
+    ag.topo_save(m, path)
+    back = ag.topo_load(path)
+    assert bytes(back) == bytes(m)
+    # a truncated or foreign file is refused
+    blob = open(path, "rb").read()
+    open(path, "wb").write(blob[:-5])
+    with pytest.raises(ag.AgError):
+        ag.topo_load(path)
+    open(path, "wb").write(b"NOTATOPO" + blob[8:])
+    with pytest.raises(ag.AgError):
+        ag.topo_load(path)
+    with pytest.raises(ag.AgError):
+        ag.topo_load(str(tmp_path / "missing.bin"))

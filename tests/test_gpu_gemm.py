@@ -137,3 +137,42 @@ def test_full_size_sampled_against_oracle():
     check_close(C[8064:8192, 7936:8192], blk)
     owner, count = plan.tile_record()
     assert (count == 1).all()
+
+
+@pytest.mark.parametrize("shape", [(256, 256, 64), (512, 768, 256), (1024, 1024, 1024), (1000, 776, 520), (2048, 2304, 1536)])
+def test_two_cta_units_integer_exact(shape):
+    """256 x 256 units computed by pairs of thread blocks (full-chip plans)."""
+    M, N, K = shape
+    A, B = inputs.small_int_bf16(M, K, 21), inputs.small_int_bf16(K, N, 22)
+    plan = plan_for(M, N, K, tile_m=256, tile_n=256, kind=ag.AG_DIE_COMPACT, raster_group=2)
+    plan.reset_record()
+    for _ in range(2):
+        C = run_gemm(A, B, plan)
+        assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+    owner, count = plan.tile_record()
+    assert (count == 2).all() and set(owner) <= set(plan.parsed()["sm_list"])
+
+
+def test_two_cta_units_uniform_and_rejections():
+    M, N, K = 1024, 1536, 2048
+    A, B = inputs.gemm_inputs(M, N, K, seed=13)
+    C = run_gemm(A, B, plan_for(M, N, K, tile_m=256, tile_n=256))
+    check_close(C, og.gemm_blocked(A, B))
+    topo = device_topo()
+    sub = ag.sched_build(topo, None, topo.n_sm - 2, ag.make_policy(M=M, N=N, K=K, tile_m=256, tile_n=256))
+    dA, dB = to_dev_bf16(A), to_dev_bf16(B)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    st = ag.lib().gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, sub.handle, None)
+    assert st == ag.AG_ERR_ARG                              # pairs need every SM
+
+
+def test_bounded_wait_gives_up_and_leaves_the_device_usable():
+    """Every device-side wait of the library has a limit; here one is made to run out on purpose
+    (a barrier that nothing signals, 2 ms limit): the kernel returns AG_ERR_TIMEOUT, nothing hangs."""
+    st, waited = ag.wait_probe(2_000_000)
+    assert st == ag.AG_ERR_TIMEOUT
+    assert 2_000_000 <= waited < 200_000_000
+    assert ag.lib().ag_wait_probe(0, None) == ag.AG_ERR_ARG
+    A, B = inputs.small_int_bf16(256, 64, 1), inputs.small_int_bf16(64, 256, 2)
+    C = run_gemm(A, B, plan_for(256, 256, 64))               # the context still works
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))

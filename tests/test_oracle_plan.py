@@ -186,22 +186,36 @@ def test_die_compact_is_compact_and_gpc_balanced():
 
 def test_equal_dies_split_c_in_halves():
     topo = inputs.synthetic_topo(die0_sms=74)
-    pol = op.default_policy(kind=op.DIE_COMPACT, M=8192, N=8192, K=8192)
+    # one raster group over all 64 tile rows: two contiguous bands of the raster (tn outer): die 0
+    # owns the left half of C's columns, die 1 the right half
+    pol = op.default_policy(kind=op.DIE_COMPACT, M=8192, N=8192, K=8192, raster_group=64)
     plan = op.build_plan(topo, None, 148, pol)
-    assert plan["die_q"][0] == list(range(1024)) and plan["die_q"][1] == list(range(1024, 2048))
+    assert sorted(plan["die_q"][0]) == [tm * 32 + tn for tm in range(64) for tn in range(16)]
+    # groups of 8 tile rows: every group is cut the same way, so the dies advance together
+    pol = op.default_policy(kind=op.DIE_COMPACT, M=8192, N=8192, K=8192, raster_group=8)
+    plan = op.build_plan(topo, None, 148, pol)
+    assert sorted(plan["die_q"][0]) == [tm * 32 + tn for tm in range(64) for tn in range(16)]
+    assert plan["die_q"][0][:8] == [tm * 32 for tm in range(8)]
+    # unequal dies (70/78): the cut follows floor(x * q0 / n_u) and the quotas still hold exactly
+    topo = inputs.synthetic_topo(die0_sms=70, seed=2)
+    plan = op.build_plan(topo, None, 148, pol)
+    assert [len(q) for q in plan["die_q"]] == op.quotas(2048, [70, 78], 148)
+    per_group0 = [sum(1 for u in plan["die_q"][0] if u // 32 // 8 == g) for g in range(8)]
+    assert max(per_group0) - min(per_group0) <= 1
 
 
 def test_min_margin_turns_weak_preferences_into_ties():
     amap = toy_amap_case_d()
     base = dict(M=256, N=512, K=64, c=op.operand(0, 2048, 4))
     # margins are -131072, +65536, +131072, 0: with a floor of 100000 unit 1 becomes a tie and
-    # falls back to its band (raster index 1 < q0 = 2 -> die 0), which is where it was anyway;
+    # falls back to the die_compact rule (second unit of its tile row -> die 1); unit 3, also a
+    # tie for die 1, then finds die 1 full and goes to die 0
     p1 = op.build_plan(TOY, amap, 4, op.default_policy(kind=op.AFFINITY, min_margin=100000, **base))
-    assert p1["die_q"] == [[1, 2], [0, 3]]
+    assert p1["die_q"] == [[2, 3], [0, 1]]
     # with a floor above every margin the plan is the die_compact one
     p2 = op.build_plan(TOY, amap, 4, op.default_policy(kind=op.AFFINITY, min_margin=1 << 30, **base))
     p3 = op.build_plan(TOY, None, 4, op.default_policy(kind=op.DIE_COMPACT, M=256, N=512, K=64))
-    assert p2["die_q"] == p3["die_q"] == [[0, 1], [2, 3]] and p2["sm_q"] == p3["sm_q"]
+    assert p2["die_q"] == p3["die_q"] == [[0, 2], [1, 3]] and p2["sm_q"] == p3["sm_q"]
 
 
 def test_all_ties_affinity_equals_die_compact():
