@@ -189,8 +189,9 @@ typedef struct {
 typedef struct {
     int32_t kind;            /* AG_OBLIVIOUS | AG_DIE_COMPACT | AG_AFFINITY */
     int32_t M, N, K;
-    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}, or 256 x 256 (two thread blocks per unit, only
-                                for plans that use every SM); decode-shaped kernel: {16,32} x 128 */
+    int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}, or 256 x 256 (two thread blocks on the two SMs of a TPC
+                                share a unit; the plan's SM set must consist of whole TPCs, else AG_ERR_ARG);
+                                decode-shaped kernel: {16,32} x 128 */
     int32_t k_splits;        /* >= 1, runs of whole k-slabs */
     int32_t k_unit;          /* elements per k-slab (64) */
     int32_t raster_group;    /* tile rows per raster group (>= 1) */
@@ -203,7 +204,8 @@ typedef struct {
                                  workspace and are added in ascending split order (bit-reproducible);
                                  1 = C is zeroed and every unit adds its partial sums with reductions in
                                  memory (no workspace, no waiting; the order of the fp32 adds is not fixed) */
-    int32_t reserved0;
+    int32_t sm_select;       /* die_compact / affinity: 0 = primary die first (die-compact set); 1 = whole TPCs dealt
+                                round-robin over the GPCs of both dies (fewest SMs per GPC, Section 5.1.2) */
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;

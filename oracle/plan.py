@@ -29,7 +29,11 @@ Steps.
                            candidates, tie -> lower id), then the other; inside a die whole
                            TPCs dealt round-robin over that die's GPCs (ascending GPC id,
                            unplaced SMs with gpc < 0 form a last pseudo-GPC), ascending SM id
-                           inside a GPC, until b SMs are taken.
+                           inside a GPC, until b SMs are taken.  With sm_select = 1 ("GPC
+                           spread") the dies are not taken one after the other: whole TPCs
+                           are dealt round-robin over the GPCs of both dies, which keeps the
+                           number of SMs per GPC as low as the budget allows (SMs of one GPC
+                           share its port to L2, Section 5.1.2).
   3. per-die SM counts n_d and rank of each chosen SM inside its die (ascending id).
   4. quotas q_d = floor(n_u * n_d / b); leftover units go one each to the dies in
      descending order of (n_u * n_d mod b), tie -> lower die id.
@@ -76,7 +80,7 @@ def mix64(x: int) -> int:
 def default_policy(**kw) -> dict:
     p = dict(kind=OBLIVIOUS, seed=0, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1,
              k_unit=64, raster_group=1, preferred_die=-1, invert_affinity=0,
-             static_assign=1, min_margin=0, avoid=(), a=None, b=None, c=None)
+             static_assign=1, min_margin=0, sm_select=0, avoid=(), a=None, b=None, c=None)
     p.update(kw)
     return p
 
@@ -123,11 +127,12 @@ def select_sms(topo: dict, b: int, pol: dict) -> list[int]:
     else:
         primary = 0 if cnt[0] >= cnt[1] else 1
     S = []
-    for d in (primary, 1 - primary):
-        # candidate TPCs of this die, grouped by GPC key (gpc < 0 -> pseudo-GPC n_gpc)
+    die_passes = [(0, 1)] if pol.get("sm_select", 0) == 1 else [(primary,), (1 - primary,)]
+    for dies in die_passes:
+        # candidate TPCs of these dies, grouped by GPC key (gpc < 0 -> pseudo-GPC n_gpc)
         groups: dict[int, dict[int, list[int]]] = {}
         for s in cand:
-            if die[s] != d:
+            if die[s] not in dies:
                 continue
             key = int(gpc[s]) if gpc[s] >= 0 else n_gpc
             groups.setdefault(key, {}).setdefault(int(tpc[s]), []).append(s)

@@ -1,4 +1,5 @@
-// Two-CTA variant of the persistent dense GEMM (tcgen05 cta_group::2) for plans that use every SM.
+// Two-CTA variant of the persistent dense GEMM (tcgen05 cta_group::2) for plans whose SM set consists of
+// whole TPCs (both SMs of every chosen TPC), e.g. every full-chip plan and every die-compact set.
 //
 // Two thread blocks form a cluster and compute one 256 x 256 output unit together: block r of
 // the pair holds rows [128 r, 128 r + 128) of the A tile and columns [128 r, 128 r + 128) of the
@@ -135,7 +136,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const int my_sm = (int)smid();
     const PlanLayout lay{p.b, p.n_units, p.n_sm};
 
-    // take the slot of this SM (every SM is planned: the host only launches this kernel for full-chip plans)
+    // take the slot of this SM; a pair on an unplanned TPC has nothing to do and leaves after the hand-shake
     const int slot = p.image[lay.smid_to_slot() + my_sm];
     if (tid == 0) {
         ctl->abort_flag = 0;
@@ -347,8 +348,15 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, in
     int dev = 0, n_sm = 0;
     AG_CUDA(cudaGetDevice(&dev));
     AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-    // pairs need every SM: a block whose partner sits on an unplanned SM could not run
-    if (n_sm != plan->lay.n_sm || plan->lay.b != n_sm || (n_sm & 1)) return AG_ERR_ARG;
+    // A pair of blocks is co-scheduled on the two SMs of one TPC, so the plan must hold whole TPCs: a block
+    // whose partner sits on an unplanned SM could not run.  (Seeded random SM subsets do not qualify - the
+    // compute-side counterpart of the paper's point that equal SM counts are not equal capabilities.)
+    if (n_sm != plan->lay.n_sm || (n_sm & 1)) return AG_ERR_ARG;
+    {
+        const int32_t* slot_of = plan->h_image.data() + plan->lay.smid_to_slot();
+        for (int s = 0; s < n_sm; ++s)
+            if ((slot_of[s] >= 0) != (slot_of[s ^ 1] >= 0)) return AG_ERR_ARG;
+    }
     if (plan->tm_a_ptr != A || plan->tm_b_ptr != B || plan->tm_c_ptr != Cout) {
         if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)) return AG_ERR_CUDA;
         if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_BK)) return AG_ERR_CUDA;

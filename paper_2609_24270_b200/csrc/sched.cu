@@ -24,6 +24,7 @@ struct OperandDev {
 };
 struct PolicyDev {
     int kind, M, N, K, tile_m, tile_n, k_splits, k_unit, raster_group, preferred_die, invert, static_assign;
+    int sm_select, pad0;
     unsigned long long seed;
     long long min_margin;
     unsigned long long avoid[4];
@@ -91,8 +92,9 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
         int primary = (pol.preferred_die == 0 || pol.preferred_die == 1) ? pol.preferred_die
                                                                            : (cnt[0] >= cnt[1] ? 0 : 1);
         const int n_gpc = topo->n_gpc;
-        for (int pass_d = 0; pass_d < 2 && ns < b; ++pass_d) {
-            const int d = pass_d == 0 ? primary : 1 - primary;
+        const int n_pass = pol.sm_select == 1 ? 1 : 2;  // GPC spread: both dies in one round-robin
+        for (int pass_d = 0; pass_d < n_pass && ns < b; ++pass_d) {
+            const int d = pol.sm_select == 1 ? -1 : (pass_d == 0 ? primary : 1 - primary);
             for (int p = 0; ns < b; ++p) {
                 bool any = false;
                 for (int key = 0; key <= n_gpc && ns < b; ++key) {
@@ -100,7 +102,7 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
                     int nt = 0;
                     for (int i = 0; i < nc; ++i) {
                         const int s = cand[i];
-                        if (topo->die[s] != d) continue;
+                        if (d >= 0 && topo->die[s] != d) continue;
                         const int k = topo->gpc[s] >= 0 ? topo->gpc[s] : n_gpc;
                         if (k != key) continue;
                         const int t = topo->tpc[s];
@@ -120,7 +122,7 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
                     const int t = tpcs[p];
                     for (int i = 0; i < nc && ns < b; ++i) {
                         const int s = cand[i];
-                        if (topo->die[s] == d && topo->tpc[s] == t &&
+                        if ((d < 0 || topo->die[s] == d) && topo->tpc[s] == t &&
                             (topo->gpc[s] >= 0 ? topo->gpc[s] : n_gpc) == key)
                             S[ns++] = s;
                     }
@@ -365,6 +367,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     if (p.kind < AG_OBLIVIOUS || p.kind > AG_AFFINITY) return AG_ERR_ARG;
     if (p.M <= 0 || p.N <= 0 || p.K <= 0 || p.tile_m <= 0 || p.tile_n <= 0) return AG_ERR_ARG;
     if (p.k_splits < 1 || p.k_unit < 1 || p.raster_group < 1 || p.min_margin < 0) return AG_ERR_ARG;
+    if (p.sm_select < 0 || p.sm_select > 1) return AG_ERR_ARG;
     if (p.kind == AG_AFFINITY && !amap) return AG_ERR_ARG;
     int n_cand = 0;
     for (int s = 0; s < map->n_sm; ++s)
@@ -443,6 +446,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pd.k_splits = p.k_splits; pd.k_unit = p.k_unit; pd.raster_group = p.raster_group;
         pd.preferred_die = p.preferred_die; pd.invert = p.invert_affinity; pd.static_assign = p.static_assign;
         pd.seed = p.seed;
+        pd.sm_select = p.sm_select;
         pd.min_margin = p.min_margin;
         for (int i = 0; i < 4; ++i) pd.avoid[i] = p.avoid_sm_mask[i];
         pd.a = to_dev(p.a, nullptr); pd.b = to_dev(p.b, d_table); pd.c = to_dev(p.c, nullptr);

@@ -71,6 +71,13 @@ def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
         plans["lowest_ids"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, M=M, N=N, K=K, raster_group=8))
         plans["die_compact"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
                                                                             raster_group=8))
+        plans["gpc_spread"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
+                                                                           raster_group=8, sm_select=1))
+        # whole-TPC sets can also run block pairs (256 x 256 units); random subsets cannot
+        for name, sel in (("die_compact_pairs", 0), ("gpc_spread_pairs", 1)):
+            if b % 2 == 0:
+                plans[name] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=256,
+                                                                           tile_n=256, raster_group=4, sm_select=sel))
         # two passes over all subsets so that clock drift is shared
         acc = {n: [] for n in plans}
         for _ in range(2):
@@ -82,11 +89,15 @@ def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
             assert plans[n].last_status() == ag.AG_OK
         rnd = [res[f"random_{s}"] for s in range(1, n_subsets + 1)]
         rank = 1 + sum(1 for v in rnd if v > res["die_compact"])
+        rank_spread = 1 + sum(1 for v in rnd if v > res["gpc_spread"])
         emit(dict(config=3, workload="dense GEMM 4096^3 bf16, 128x256 tiles", sm_budget=b,
                   random_subsets_tflops=dict(min=min(rnd), max=max(rnd), median=float(np.median(rnd)),
                                              spread_max_over_min=max(rnd) / min(rnd)),
                   lowest_ids_tflops=res["lowest_ids"], die_compact_tflops=res["die_compact"],
                   die_compact_rank_among_33=rank, die_compact_set=sm_set_summary(topo, plans["die_compact"]),
+                  gpc_spread_tflops=res["gpc_spread"], gpc_spread_rank_among_33=rank_spread,
+                  gpc_spread_set=sm_set_summary(topo, plans["gpc_spread"]),
+                  die_compact_pairs_tflops=res.get("die_compact_pairs"), gpc_spread_pairs_tflops=res.get("gpc_spread_pairs"),
                   peak_scaled_tflops=2250.0 * b / topo.n_sm, all_tflops=rnd), fh)
 
 
@@ -172,7 +183,7 @@ def config5(fh, topo):
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     flops_p = 2.0 * Mp * N * K
     bytes_d = K * N * 2 + Md * K * 2 + Md * N * 4
-    pre_kw = dict(M=Mp, N=N, K=K, tile_m=128, tile_n=256, raster_group=8)
+    pre_kw = dict(M=Mp, N=N, K=K, tile_m=256, tile_n=256, raster_group=4)   # both partitions hold whole TPCs: block pairs
     dec_kw = dict(M=Md, N=N, K=K, tile_m=32, tile_n=128, k_splits=8, splitk_in_memory=1)
     for split in ((74, 74), (110, 38)):
         for mode in ("die_split", "oblivious"):

@@ -159,11 +159,24 @@ def test_two_cta_units_uniform_and_rejections():
     C = run_gemm(A, B, plan_for(M, N, K, tile_m=256, tile_n=256))
     check_close(C, og.gemm_blocked(A, B))
     topo = device_topo()
-    sub = ag.sched_build(topo, None, topo.n_sm - 2, ag.make_policy(M=M, N=N, K=K, tile_m=256, tile_n=256))
+    odd = ag.sched_build(topo, None, 37, ag.make_policy(M=M, N=N, K=K, tile_m=256, tile_n=256, seed=3))
     dA, dB = to_dev_bf16(A), to_dev_bf16(B)
     dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
-    st = ag.lib().gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, sub.handle, None)
-    assert st == ag.AG_ERR_ARG                              # pairs need every SM
+    st = ag.lib().gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, odd.handle, None)
+    assert st == ag.AG_ERR_ARG                              # a random subset is not made of whole TPCs
+
+
+@pytest.mark.parametrize("b,sm_select", [(16, 0), (64, 0), (74, 0), (64, 1), (100, 1)])
+def test_two_cta_units_on_sub_budgets_of_whole_tpcs(b, sm_select):
+    """Die-compact and GPC-spread sets hold whole TPCs, so block pairs can run on them."""
+    M, N, K = 1024, 1536, 512
+    A, B = inputs.small_int_bf16(M, K, 31), inputs.small_int_bf16(K, N, 32)
+    plan = plan_for(M, N, K, b=b, tile_m=256, tile_n=256, kind=ag.AG_DIE_COMPACT, sm_select=sm_select, raster_group=2)
+    plan.reset_record()
+    C = run_gemm(A, B, plan)
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+    owner, count = plan.tile_record()
+    assert (count == 1).all() and set(owner) <= set(plan.parsed()["sm_list"])
 
 
 def test_bounded_wait_gives_up_and_leaves_the_device_usable():

@@ -43,6 +43,14 @@ def test_seeded_random_subsets_match_oracle(seed, b):
     assert got.tobytes() == want.tobytes()
 
 
+@pytest.mark.parametrize("b", [16, 48, 64, 74, 111])
+def test_gpc_spread_selection_matches_oracle(b):
+    topo = inputs.synthetic_topo(die0_sms=70, seed=8)
+    for kind in (ag.AG_DIE_COMPACT,):
+        got, want, _ = both(topo, None, b, kind=kind, M=4096, N=4096, K=4096, raster_group=8, sm_select=1)
+        assert got.tobytes() == want.tobytes()
+
+
 def test_avoid_mask_and_unplaced_sms():
     topo = inputs.synthetic_topo(die0_sms=74, seed=4)
     topo["gpc"] = topo["gpc"].copy()

@@ -184,6 +184,24 @@ def test_die_compact_is_compact_and_gpc_balanced():
     assert all(topo["die"][s] == 0 for s in op.select_sms(topo, 32, pol0))
 
 
+def test_gpc_spread_selection_minimises_sms_per_gpc():
+    topo = inputs.synthetic_topo(die0_sms=70, seed=3)
+    for b in (16, 48, 64, 100):
+        pol = op.default_policy(kind=op.DIE_COMPACT, M=4096, N=4096, K=4096, sm_select=1)
+        S = op.select_sms(topo, b, pol)
+        assert len(S) == b and all((s ^ 1) in S for s in S)            # whole TPCs
+        per_gpc = np.bincount([topo["gpc"][s] for s in S], minlength=8)
+        sizes = np.bincount(topo["gpc"], minlength=8)
+        cap = -(-b // 16) * 2                                         # ceil(b / 8 GPCs) rounded up to a TPC
+        assert all(per_gpc[g] <= max(cap, 2) or per_gpc[g] == sizes[g] for g in range(8))
+        assert per_gpc.max() - per_gpc[per_gpc < sizes].min() <= 2
+        plan = op.build_plan(topo, None, b, pol)
+        check_invariants(topo, plan, pol, b)
+    # the die-compact set of the same budget sits in four GPCs only
+    S0 = op.select_sms(topo, 64, op.default_policy(kind=op.DIE_COMPACT, M=1, N=1, K=1))
+    assert len({topo["gpc"][s] for s in S0}) == 4
+
+
 def test_equal_dies_split_c_in_halves():
     topo = inputs.synthetic_topo(die0_sms=74)
     # one raster group over all 64 tile rows: two contiguous bands of the raster (tn outer): die 0
