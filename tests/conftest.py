@@ -12,6 +12,16 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """The shared libraries are build products (not in git): compile them when missing or stale.
+    nvcc cross-compiles for sm_100a without a GPU; gcc builds the oracle's C part."""
+    from oracle import build as oracle_build
+    from paper_2609_24270_b200 import build as lib_build
+    oracle_build.build()
+    lib_build.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
