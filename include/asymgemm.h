@@ -270,7 +270,9 @@ typedef struct ag_packed_weights ag_packed_weights;
  * for the parity-of-masked-physical-address selector of Eq. 1).  Inside a page element (n, k) sits
  * at byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2, the order the MMA reads without swizzle.
  *   B      device, K x N bf16 row-major
- *   plan   a plan with tile_n = 128 and one tile row (M <= tile_m <= 32), K % 64 == 0
+ *   plan   a decode-shaped plan (tile_n = 128, one tile row) or a dense plan with 256-column units
+ *          (tile_n = 256: two pages side by side per unit column); K % 64 == 0.  A page read by
+ *          units of both dies goes to the die that runs most of them (tie: die 0)
  *   amap   affinity map of exactly (dst, dst_bytes), else AG_ERR_STALE_AMAP
  *   dst    device, 4096-aligned; needs 2 * max(pages of die 0, pages of die 1) chunks
  *   out    host, out: handle holding the page table (device + host copy)
@@ -284,12 +286,14 @@ ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* out, size_t 
 void ag_packed_destroy(ag_packed_weights* w);
 
 /*
- * gemm_persistent_packed - C = A * B for M <= 32 with the weights taken from a packed buffer
+ * gemm_persistent_packed - C = A * B with the B operand taken from a packed buffer
  * (Section 7.1.2 on top of Section 7.1.1: each block reads the pages of its units, which the
- * packing put on the block's own die when plan and packing agree).  gemm_persistent handles the
- * same shapes with row-major B.
+ * packing put on the block's own die when plan and packing agree).  Decode-shaped plans
+ * (tile_m in {16, 32}, tile_n = 128, M <= tile_m) and dense plans of block pairs (256 x 256
+ * units, SM set of whole TPCs) are accepted; gemm_persistent handles the same shapes with
+ * row-major B.
  *   A  device, M x K bf16 row-major, 16-byte aligned;  C  device, M x N fp32 row-major, overwritten
- *   plan  tile_m in {16, 32} (M <= tile_m), tile_n = 128, same N, K as the packing; with
+ *   plan  same N, K (and tile_n) as the packing; decode-shaped plans: with
  *         k_splits > 1 the partial sums either go through the plan's workspace and are added in
  *         ascending split order by the block that finishes a tile last, or are added straight
  *         into a zeroed C by reductions in memory (policy.splitk_in_memory)

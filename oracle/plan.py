@@ -226,12 +226,15 @@ def unit_local_bytes(pol: dict, amap: dict, u: int) -> list[int]:
     add(pol["a"], r0, r1, k0, k1)                      # A panel: rows of the tile, k-range columns
     bop = pol["b"]
     if bop is not None and bop["layout"] == LAYOUT_PAGED:
-        # weights stored as pages of [16 k x tile_n] elements; logical page of (tn, k16)
+        # weights stored as 4 KB pages of [128 columns x 16 k] elements; logical page of
+        # (128-column block pc, k16) = pc * ceil(K/16) + k16; a unit column holds tile_n/128 blocks
         ppt = -(-pol["K"] // 16)
+        ppc = max(1, pol["tile_n"] // 128)
         cb = amap["chunk_bytes"]
-        for k16 in range(k0 // 16, -(-k1 // 16)):
-            phys = int(bop["page_table"][tn * ppt + k16])
-            tot[int(amap["die_of_chunk"][phys])] += cb
+        for pc in range(tn * ppc, (tn + 1) * ppc):
+            for k16 in range(k0 // 16, -(-k1 // 16)):
+                phys = int(bop["page_table"][pc * ppt + k16])
+                tot[int(amap["die_of_chunk"][phys])] += cb
     else:
         add(bop, k0, k1, c0, c1)                       # B panel: k-range rows, tile columns
     add(pol["c"], r0, r1, c0, c1)                      # C tile
@@ -360,28 +363,35 @@ def build_page_table(page_die, amap: dict) -> list[int]:
 
 
 def page_die_from_plan(plan: dict, K: int, k_unit: int = 64) -> list[int]:
-    """Die of every logical weight page (tn, k16), j = tn * ceil(K/16) + k16: the die whose queue
-    holds the unit (tn, ks) whose k-range contains the page."""
+    """Die that owns every logical weight page (pc, k16), j = pc * ceil(K/16) + k16, pc = index of the
+    128-column block: the die whose queue holds most of the units (tm, tn, ks) that read the page
+    (tn = pc // (tile_n/128), ks = the k-split containing k16; a tie goes to die 0).  Decode-shaped
+    plans have one tile row, so exactly one unit reads a page."""
     unit_die = {}
     for d in (0, 1):
         for u in plan["die_q"][d]:
             unit_die[u] = d
-    ksp = plan["k_splits"]
+    ksp, tiles_m, tiles_n = plan["k_splits"], plan["tiles_m"], plan["tiles_n"]
     n_slab = -(-K // k_unit)
     per = -(-n_slab // ksp)
     ppt = -(-K // 16)
+    ppc = max(1, plan["tile_n"] // 128)
     out = []
-    for tn in range(plan["tiles_n"]):
+    for pc in range(tiles_n * ppc):
+        tn = pc // ppc
         for k16 in range(ppt):
             ks = (k16 * 16 // k_unit) // per
-            out.append(unit_die[tn * ksp + ks])
+            votes = [0, 0]
+            for tm in range(tiles_m):
+                votes[unit_die[(tm * tiles_n + tn) * ksp + ks]] += 1
+            out.append(0 if votes[0] >= votes[1] else 1)
     return out
 
 
 def pack_weights(B_bits: np.ndarray, page_table: list[int], n_chunks: int, tile_n: int = 128) -> np.ndarray:
-    """Packed image (uint16, n_chunks x 2048) of the K x N bf16 weights.
+    """Packed image (uint16, n_chunks x 2048) of the K x N bf16 weights (tile_n = page width, 128).
 
-    Logical page (tn, k16) holds W[n][k] for n in [tn*128, tn*128+128), k in [k16*16, k16*16+16)
+    Logical page (pc, k16) holds W[n][k] for n in [pc*128, pc*128+128), k in [k16*16, k16*16+16)
     as 8 x 8 blocks ("core matrices", 8 rows n x 16 bytes of k, 128 bytes each, row-major inside):
     element (n, k) of the page sits at byte (n//8)*256 + (k//8)*128 + (n%8)*16 + (k%8)*2.
     Out-of-range n or k are zeros; chunks no page maps to stay zero.

@@ -133,8 +133,13 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                     const uint32_t sa = s_stage + st * C::stage_bytes, sb = sa + C::a_bytes;
                     mbar_expect_tx(bar, C::stage_bytes);
                     tma_load_2d(sa, &tm_a, bar, s * BK, tm * BM);
+                    if (p.b_blocks) {
+                        // one copy for all 64-column blocks of the slab (B seen as [N/64][K][64])
+                        tma_load_3d(sb, &tm_b, bar, 0, s * BK, tn * (BN / 64));
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tm_b, bar, tn * BN + j * 64, s * BK);
+                        for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tm_b, bar, tn * BN + j * 64, s * BK);
+                    }
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -304,6 +309,18 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const vo
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool encode_b_blocks(CUtensorMap* tm, const void* ptr, uint64_t K, uint64_t N, uint32_t box_k, uint32_t n_blocks) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc || (N % 64)) return false;
+    cuuint64_t dims[3] = {64, K, N / 64};
+    cuuint64_t strides[2] = {N * 2, 128};
+    cuuint32_t box[3] = {64, box_k, n_blocks};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN>
 static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream_t stream) {
     using C = Cfg<BN>;
@@ -324,8 +341,8 @@ static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream
 namespace ag {
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
                                int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream);
-ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, int N, int K, const ag_plan* plan,
-                             cudaStream_t stream);
+ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
+                             const ag_plan* plan, cudaStream_t stream);
 }
 
 using namespace ag;
@@ -339,7 +356,7 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
                                     reinterpret_cast<cudaStream_t>(cuda_stream));
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_M] == 256)  // 256 x 256 units: pairs of blocks, full-chip plans only
-        return gemm_pair_dispatch(A, B, Cout, M, N, K, plan, reinterpret_cast<cudaStream_t>(cuda_stream));
+        return gemm_pair_dispatch(A, B, nullptr, Cout, M, N, K, plan, reinterpret_cast<cudaStream_t>(cuda_stream));
     if (h[H_TILE_M] != BM || (h[H_TILE_N] != 64 && h[H_TILE_N] != 128 && h[H_TILE_N] != 256)) return AG_ERR_ARG;
     if (plan->policy.k_unit != BK) return AG_ERR_ARG;
     if ((K % 8) || (N % 8)) return AG_ERR_ARG;
@@ -354,12 +371,17 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
     const int BN = h[H_TILE_N];
     if (plan->tm_a_ptr != A || plan->tm_b_ptr != B || plan->tm_c_ptr != Cout) {
         if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, BK, BM)) return AG_ERR_CUDA;
-        if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, BK)) return AG_ERR_CUDA;
+        if (N % 64 == 0) {
+            if (!encode_b_blocks(&plan->tm_b, B, K, N, BK, BN / 64)) return AG_ERR_CUDA;
+        } else if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, BK)) {
+            return AG_ERR_CUDA;
+        }
         if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
         plan->tm_a_ptr = A; plan->tm_b_ptr = B; plan->tm_c_ptr = Cout;
     }
     if (h[H_KSPLITS] > 1) AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * (size_t)M * (size_t)N, stream));
-    const PersistParams gp = make_persist_params(plan, M, N, K);
+    PersistParams gp = make_persist_params(plan, M, N, K);
+    gp.b_blocks = (N % 64 == 0) ? 1 : 0;
     if (BN == 256) return launch<256>(plan, gp, stream);
     if (BN == 128) return launch<128>(plan, gp, stream);
     return launch<64>(plan, gp, stream);

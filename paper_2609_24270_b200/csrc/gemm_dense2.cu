@@ -76,6 +76,13 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(x), "r"(y)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int x, int y,
+                                                 int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
 __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                                 uint32_t accumulate) {
     asm volatile(
@@ -120,9 +127,13 @@ struct PairSource {
     }
 };
 
+// PACKED_B: the B panels come from die-local 4 KB pages ([128 columns x 16 k], no-swizzle core-matrix order,
+// see ag_pack_weights): tm_b then describes the packed buffer as [chunk][16][128] and a page is one box.
+template <bool PACKED_B>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                       const __grid_constant__ CUtensorMap tm_c, const PersistParams p) {
+                       const __grid_constant__ CUtensorMap tm_c, const PersistParams p,
+                       const int32_t* __restrict__ page_table, const int pages_per_block) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -180,45 +191,80 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 
     if (active) {
         if (warp == 0) {
-            // ------------------------------------------------ scheduler + TMA producer (lane 0)
-            if (lane == 0) {
-                PairSource src(p, slot, peer_slot);
-                uint32_t it = 0, kit = 0;
-                bool ok = true;
-                while (ok) {
-                    const int u = src.next();
+            // ------------------------------------------------ scheduler + TMA producer.  Every lane walks the same
+            // unit sequence; lane 0 waits and issues.  For packed B the 32 lanes fetch the page-table entries of
+            // the next eight k-slabs with one load each.
+            PairSource src(p, slot, peer_slot);
+            uint32_t it = 0, kit = 0;
+            int ok = 1;
+            while (ok) {
+                const int u = src.next();
+                if (lane == 0) {
                     const int r = it % kRing;
                     if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                         report_timeout(p, 1);
-                        ok = false;
-                        break;
+                        ok = 0;
+                    } else {
+                        ctl->ring[r] = u;
+                        mbar_arrive(smem_u32(&ctl->sched_full[r]));
                     }
-                    ctl->ring[r] = u;
-                    mbar_arrive(smem_u32(&ctl->sched_full[r]));
-                    ++it;
-                    if (u < 0) break;
-                    const int tm = u / p.tiles_n, tn = u % p.tiles_n;
-                    for (int s = 0; s < p.kslabs_total; ++s, ++kit) {
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                ++it;
+                if (!ok || u < 0) break;
+                const int tm = u / p.tiles_n, tn = u % p.tiles_n;
+                // Packed B: the units of one raster group that share a column panel start their k loop at
+                // different k-slabs (the sum over k does not care where it starts), so that at any moment they
+                // read different 4 KB pages: a page sits in few L2 slices, and eight pairs asking for the same
+                // page at once queue up there.
+                const int n_blk = (p.kslabs_total + 7) / 8;
+                const int rot = PACKED_B ? ((tm & 7) * max(1, n_blk / 8)) % n_blk : 0;
+                for (int b8 = 0; b8 < n_blk && ok; ++b8) {
+                    const int sb = ((b8 + rot) % n_blk) * 8;
+                    int my_page = 0;
+                    if (PACKED_B) {
+                        const int pg = sb * 4 + lane;
+                        if (pg < p.kslabs_total * 4) my_page = page_table[(size_t)(tn * 2 + (int)rank) * pages_per_block + pg];
+                    }
+                    const int se = min(p.kslabs_total, sb + 8);
+                    for (int s = sb; s < se; ++s, ++kit) {
                         const int st = kit % P_STAGES;
-                        if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / P_STAGES) & 1) ^ 1, abort_flag, limit)) {
-                            report_timeout(p, 2);
-                            ok = false;
-                            break;
-                        }
                         // the leader's barrier counts the bytes of both blocks
                         const uint32_t bar_leader = map_to_cta(smem_u32(&ctl->full[st]), 0);
-                        if (leader) mbar_expect_tx(smem_u32(&ctl->full[st]), 2 * P_STAGE_BYTES);
-                        const uint32_t sa = base + st * P_STAGE_BYTES, sb = sa + P_A_BYTES;
-                        tma_load_2d_pair(sa, &tm_a, bar_leader, s * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
-                        tma_load_2d_pair(sb, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH, s * P_BK);
-                        tma_load_2d_pair(sb + P_BK * 128, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH + 64, s * P_BK);
+                        const uint32_t sa = base + st * P_STAGE_BYTES, sb_addr = sa + P_A_BYTES;
+                        if (lane == 0) {
+                            if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / P_STAGES) & 1) ^ 1, abort_flag, limit)) {
+                                report_timeout(p, 2);
+                                ok = 0;
+                            } else {
+                                if (leader) mbar_expect_tx(smem_u32(&ctl->full[st]), 2 * P_STAGE_BYTES);
+                                tma_load_2d_pair(sa, &tm_a, bar_leader, s * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
+                                if (!PACKED_B) {
+                                    if (p.b_blocks) {
+                                        // both 64-column blocks of this block's half with one copy
+                                        tma_load_3d_pair(sb_addr, &tm_b, bar_leader, 0, s * P_BK, tn * 4 + (int)rank * 2);
+                                    } else {
+                                        tma_load_2d_pair(sb_addr, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH, s * P_BK);
+                                        tma_load_2d_pair(sb_addr + P_BK * 128, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH + 64, s * P_BK);
+                                    }
+                                }
+                            }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!ok) break;
+                        if (PACKED_B) {
+                            // four lanes issue the four page copies of the slab in one instruction: a single
+                            // thread gets only one bulk copy out every ~150 cycles
+                            const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + (lane & 3));
+                            if (lane < 4) tma_load_3d_pair(sb_addr + lane * 4096, &tm_b, bar_leader, 0, 0, page);
+                        }
                     }
                 }
             }
         } else if (warp == 1) {
             if (lane == 0) {
                 // ------------------------------------------------ MMA issuer (leader) / ring consumer (peer)
-                constexpr uint32_t idesc = make_idesc_bf16(2 * P_BM, P_BN, 0, 1);
+                constexpr uint32_t idesc = make_idesc_bf16(2 * P_BM, P_BN, 0, PACKED_B ? 0 : 1);
                 uint32_t kit = 0, tile_it = 0;
                 bool ok = true;
                 for (uint32_t it = 0; ok; ++it) {
@@ -250,7 +296,10 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 #pragma unroll
                         for (int k4 = 0; k4 < P_BK / 16; ++k4) {
                             const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
-                            const uint64_t db = make_smem_desc(sb + k4 * 2048, P_BK * 128, 1024, 2);
+                            // B: row-major source = N-major, 128-byte swizzle; packed page = K-major, no swizzle,
+                            // 16-byte k chunks 128 B apart (LBO), 8-column groups 256 B apart (SBO)
+                            const uint64_t db = PACKED_B ? make_smem_desc(sb + k4 * 4096, 128, 256, 0)
+                                                         : make_smem_desc(sb + k4 * 2048, P_BK * 128, 1024, 2);
                             tc_mma_f16_pair(d_tmem, da, db, idesc, (s > 0 || k4 > 0) ? 1u : 0u);
                         }
                         tc_commit_pair(smem_u32(&ctl->empty[st]));
@@ -337,12 +386,18 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     }
 }
 
-ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, int N, int K, const ag_plan* plan,
-                             cudaStream_t stream) {
+ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
+                             const ag_plan* plan, cudaStream_t stream) {
     const int32_t* h = plan->header;
+    if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_M] != 2 * P_BM || h[H_TILE_N] != P_BN || h[H_KSPLITS] != 1 || !h[H_STATIC]) return AG_ERR_ARG;
     if (plan->policy.k_unit != P_BK || (K % 8) || (N % 8)) return AG_ERR_ARG;
-    if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
+    if (((uintptr_t)A | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
+    if (W) {
+        if (W->K != K || W->N != N || (K % P_BK) || W->tiles_n != 2 * h[H_TILES_N]) return AG_ERR_ARG;
+    } else if (!B || ((uintptr_t)B & 15u)) {
+        return AG_ERR_ARG;
+    }
     ag_status st = check_arch();
     if (st != AG_OK) return st;
     int dev = 0, n_sm = 0;
@@ -357,19 +412,25 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, in
         for (int s = 0; s < n_sm; ++s)
             if ((slot_of[s] >= 0) != (slot_of[s ^ 1] >= 0)) return AG_ERR_ARG;
     }
-    if (plan->tm_a_ptr != A || plan->tm_b_ptr != B || plan->tm_c_ptr != Cout) {
+    const void* b_key = W ? (const void*)W : B;
+    if (plan->tm_a_ptr != A || plan->tm_b_ptr != b_key || plan->tm_c_ptr != Cout) {
         if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)) return AG_ERR_CUDA;
-        if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_BK)) return AG_ERR_CUDA;
+        if (W) plan->tm_b = W->tm_pages;
+        else if (N % 64 == 0) { if (!encode_b_blocks(&plan->tm_b, B, K, N, P_BK, 2)) return AG_ERR_CUDA; }
+        else if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_BK)) return AG_ERR_CUDA;
         if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
-        plan->tm_a_ptr = A; plan->tm_b_ptr = B; plan->tm_c_ptr = Cout;
+        plan->tm_a_ptr = A; plan->tm_b_ptr = b_key; plan->tm_c_ptr = Cout;
     }
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(k_gemm_persistent_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        attr_err = cudaFuncSetAttribute(k_gemm_persistent_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(k_gemm_persistent_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    const PersistParams gp = make_persist_params(plan, M, N, K);
+    PersistParams gp = make_persist_params(plan, M, N, K);
+    gp.b_blocks = (!W && N % 64 == 0) ? 1 : 0;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(n_sm);
@@ -383,7 +444,10 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, void* Cout, int M, in
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair, plan->tm_a, plan->tm_b, plan->tm_c, gp));
+    const int32_t* table = W ? W->d_page_table : nullptr;
+    const int ppb = W ? W->pages_per_tile : 0;
+    if (W) AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb));
+    else AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb));
     count_launch();
     return AG_OK;
 }

@@ -153,14 +153,19 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) break;
                     if (PACKED) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + i);
-                            if (lane == 0) bulk_load_hint(sw + i * 4096, x.packed + (size_t)page * AG_CHUNK_BYTES, 4096, bar, stream_policy);
-                        }
+                        // four lanes issue the four page copies of the slab in one instruction (a single thread
+                        // gets only one bulk copy out every ~150 cycles)
+                        const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + (lane & 3));
+                        if (lane < 4)
+                            bulk_load_hint(sw + lane * 4096, x.packed + (size_t)page * AG_CHUNK_BYTES, 4096, bar, stream_policy);
                     } else if (lane == 0) {
-                        tma_load_2d_hint(sw, &tm_w, bar, tn * SK_BN, s * SK_BK, stream_policy);
-                        tma_load_2d_hint(sw + 8192, &tm_w, bar, tn * SK_BN + 64, s * SK_BK, stream_policy);
+                        if (p.b_blocks) {
+                            // both 64-column blocks with one copy (B seen as [N/64][K][64])
+                            tma_load_3d_hint(sw, &tm_w, bar, 0, s * SK_BK, tn * 2, stream_policy);
+                        } else {
+                            tma_load_2d_hint(sw, &tm_w, bar, tn * SK_BN, s * SK_BK, stream_policy);
+                            tma_load_2d_hint(sw + 8192, &tm_w, bar, tn * SK_BN + 64, s * SK_BK, stream_policy);
+                        }
                     }
                     if (lane == 0) tma_load_2d(sa, &tm_a, bar, s * SK_BK, 0);
                 }
@@ -434,17 +439,22 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     x.partial = h[H_KSPLITS] > 1 ? partial : nullptr;
     x.sem = sem;
     if (W) {
-        if (W->K != K || W->N != N || (K % SK_BK)) return AG_ERR_ARG;
+        if (W->K != K || W->N != N || (K % SK_BK) || W->tiles_n != h[H_TILES_N]) return AG_ERR_ARG;
         x.packed = W->dst;
         x.page_table = W->d_page_table;
         x.pages_per_tile = W->pages_per_tile;
     } else {
         if (!B_rowmajor || ((uintptr_t)B_rowmajor & 15u)) return AG_ERR_ARG;
-        if (!encode_2d(&tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_rowmajor, K, N, 64, SK_BK)) return AG_ERR_CUDA;
+        if (N % 64 == 0) {
+            if (!encode_b_blocks(&tm_w, B_rowmajor, K, N, SK_BK, 2)) return AG_ERR_CUDA;
+        } else if (!encode_2d(&tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_rowmajor, K, N, 64, SK_BK)) {
+            return AG_ERR_CUDA;
+        }
     }
     if (h[H_KSPLITS] > 1 && !x.partial)  // in-memory reduction mode: the adds need a zeroed C
         AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * (size_t)M * (size_t)N, stream));
-    const PersistParams gp = make_persist_params(plan, M, N, K);
+    PersistParams gp = make_persist_params(plan, M, N, K);
+    gp.b_blocks = (!W && N % 64 == 0) ? 1 : 0;
     if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream)
                            : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream);
     return W ? launch_skinny<32, true>(plan, tm_a, tm_w, gp, x, stream)
@@ -460,35 +470,57 @@ extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan*
     if (!B || !plan || !amap || !dst || !out || K <= 0 || N <= 0) return AG_ERR_ARG;
     *out = nullptr;
     const int32_t* h = plan->header;
-    if (h[H_TILE_N] != SK_BN || h[H_N] != N || h[H_K] != K || h[H_TILES_M] != 1 || (K % SK_BK)) return AG_ERR_ARG;
+    if ((h[H_TILE_N] != 128 && h[H_TILE_N] != 256) || h[H_N] != N || h[H_K] != K || (K % SK_BK)) return AG_ERR_ARG;
     if (amap->base != dst || amap->bytes != dst_bytes) return AG_ERR_STALE_AMAP;
-    const int tiles_n = h[H_TILES_N], ksp = h[H_KSPLITS];
+    const int tiles_m = h[H_TILES_M], tiles_n = h[H_TILES_N], ksp = h[H_KSPLITS];
+    const int ppc = h[H_TILE_N] / 128;          // 128-column blocks per unit column
+    const int n_blocks = tiles_n * ppc;
     const int ppt = K / 16;
-    const size_t n_pages = (size_t)tiles_n * ppt;
+    const size_t n_pages = (size_t)n_blocks * ppt;
     // die of every unit from the plan's die queues
     const PlanLayout& lay = plan->lay;
     const int32_t* img = plan->h_image.data();
     std::vector<uint8_t> unit_die(lay.n_units, 0);
     for (int e = img[lay.die_q_off() + 1]; e < lay.n_units; ++e) unit_die[img[lay.die_q() + e]] = 1;
-    // two logical views over the chunk pairs: page p of view d = the chunk of pair p that sits on die d
+    // two logical views over the chunk pairs: page p of view d = the chunk of pair p that sits on die d;
+    // a page goes to the view of the die that runs most of the units reading it (tie -> die 0)
     ag_packed_weights* w = new (std::nothrow) ag_packed_weights();
     if (!w) return AG_ERR_NOMEM;
-    w->K = K; w->N = N; w->tiles_n = tiles_n; w->pages_per_tile = ppt; w->n_pages = n_pages;
+    w->K = K; w->N = N; w->tiles_n = n_blocks; w->pages_per_tile = ppt; w->n_pages = n_pages;
     w->dst = (const uint8_t*)dst; w->dst_bytes = dst_bytes; w->d_page_table = nullptr;
     w->h_page_table.resize(n_pages);
     size_t next[2] = {0, 0};
     const int per = plan->kslabs_per_split;
-    for (int tn = 0; tn < tiles_n; ++tn)
+    for (int pc = 0; pc < n_blocks; ++pc) {
+        const int tn = pc / ppc;
         for (int k16 = 0; k16 < ppt; ++k16) {
             const int ks = (k16 * 16 / SK_BK) / per;
-            const int d = unit_die[(size_t)tn * ksp + ks];
+            int votes[2] = {0, 0};
+            for (int tm = 0; tm < tiles_m; ++tm) votes[unit_die[((size_t)tm * tiles_n + tn) * ksp + ks]]++;
+            const int d = votes[0] >= votes[1] ? 0 : 1;
             const size_t pair = next[d]++;
             if (2 * pair + 1 >= amap->n_chunks) {
                 delete w;
                 return AG_ERR_ARG;  // destination too small for this die's view
             }
-            w->h_page_table[(size_t)tn * ppt + k16] = (int32_t)(2 * pair + (amap->h_die_of_chunk[2 * pair] == d ? 0 : 1));
+            w->h_page_table[(size_t)pc * ppt + k16] = (int32_t)(2 * pair + (amap->h_die_of_chunk[2 * pair] == d ? 0 : 1));
         }
+    }
+    {
+        // the packed buffer as a 3-D tensor [chunk][16 rows][128 bf16]: one box of (128, 16, 1) is one page,
+        // landing in shared memory in the page's own byte order (no swizzle)
+        EncodeTiledFn enc = get_encode_tiled();
+        cuuint64_t dims[3] = {128, 16, (cuuint64_t)amap->n_chunks};
+        cuuint64_t strides[2] = {256, AG_CHUNK_BYTES};
+        cuuint32_t box[3] = {128, 16, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (!enc || enc(&w->tm_pages, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, dst, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            delete w;
+            return AG_ERR_CUDA;
+        }
+    }
     cudaError_t e = cudaMalloc(&w->d_page_table, sizeof(int32_t) * n_pages);
     if (e == cudaSuccess)
         e = cudaMemcpy(w->d_page_table, w->h_page_table.data(), sizeof(int32_t) * n_pages, cudaMemcpyHostToDevice);
@@ -522,9 +554,16 @@ extern "C" void ag_packed_destroy(ag_packed_weights* w) {
     delete w;
 }
 
+namespace ag {
+ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
+                             const ag_plan* plan, cudaStream_t stream);
+}
+
 extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* Cout, int M, int N, int K,
                                             const ag_plan* plan, void* cuda_stream) {
     if (!A || !W || !Cout || !plan) return AG_ERR_ARG;
+    if (plan->header[H_TILE_M] == 256)  // dense plan of block pairs over packed B panels
+        return gemm_pair_dispatch(A, nullptr, W, Cout, M, N, K, plan, reinterpret_cast<cudaStream_t>(cuda_stream));
     return gemm_skinny_dispatch(A, nullptr, W, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
                                 reinterpret_cast<cudaStream_t>(cuda_stream));
 }

@@ -78,8 +78,11 @@ struct ag_plan {
 };
 
 struct ag_packed_weights {
-    int K, N, tiles_n, pages_per_tile;   // pages_per_tile = K / 16
+    int K, N;
+    int tiles_n;                         // number of 128-column blocks
+    int pages_per_tile;                  // pages per column block = K / 16
     size_t n_pages;
+    CUtensorMap tm_pages;                // dst seen as [chunk][16 rows][128 bf16]: one box = one 4 KB page
     const uint8_t* dst;                  // device: packed buffer (the probed buffer)
     size_t dst_bytes;
     int32_t* d_page_table;               // device [n_pages]: chunk index of each logical page

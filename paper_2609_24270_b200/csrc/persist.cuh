@@ -24,6 +24,7 @@ struct PersistParams {
     int static_assign;
     unsigned int epoch;
     unsigned long long wait_limit_ns;
+    int b_blocks;           // 1: tm_b is the 3-D [N/64][K][64] view of B (one copy per k-slab)
 };
 
 __device__ __forceinline__ void report_timeout(const PersistParams& p, int role) {
@@ -141,6 +142,7 @@ inline PersistParams make_persist_params(const ag_plan* plan, int M, int N, int 
     gp.static_assign = plan->header[H_STATIC];
     gp.epoch = ++plan->epoch;
     gp.wait_limit_ns = kWaitLimitNs;
+    gp.b_blocks = 0;
     return gp;
 }
 
@@ -151,5 +153,8 @@ EncodeTiledFn get_encode_tiled();
 // 2-D row-major tensor of `rows` x `cols` elements, box = box_cols x box_rows, 128-byte swizzle.
 bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const void* ptr, uint64_t rows,
                uint64_t cols, uint32_t box_cols, uint32_t box_rows);
+// Row-major K x N bf16 matrix (N % 64 == 0) seen as [N/64][K][64]: one box of (64, box_k, n_blocks) brings
+// n_blocks 64-column blocks of a k-slab with a single copy, each block laid out as a separate 2-D box would be.
+bool encode_b_blocks(CUtensorMap* tm, const void* ptr, uint64_t K, uint64_t N, uint32_t box_k, uint32_t n_blocks);
 
 }  // namespace ag

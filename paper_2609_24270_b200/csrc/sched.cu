@@ -214,11 +214,14 @@ __global__ void k_score_units(PolicyDev pol, int n_units, int tiles_m, int tiles
         }
     if (pol.b.present) {
         if (pol.b.layout == AG_LAYOUT_PAGED) {
+            // 4 KB pages of [128 columns x 16 k]; a unit column holds tile_n / 128 column blocks
             const int ppt = (pol.K + 15) / 16;
-            for (int k16 = k0 / 16 + lane; k16 < (k1 + 15) / 16; k16 += 32) {
-                const int phys = pol.b.page_table[(long long)tn * ppt + k16];
-                if (doc[phys]) l1 += AG_CHUNK_BYTES; else l0 += AG_CHUNK_BYTES;
-            }
+            const int ppc = max(1, pol.tile_n / 128);
+            for (int pc = tn * ppc; pc < (tn + 1) * ppc; ++pc)
+                for (int k16 = k0 / 16 + lane; k16 < (k1 + 15) / 16; k16 += 32) {
+                    const int phys = pol.b.page_table[(long long)pc * ppt + k16];
+                    if (doc[phys]) l1 += AG_CHUNK_BYTES; else l0 += AG_CHUNK_BYTES;
+                }
         } else {
             for (int k = k0 + lane; k < k1; k += 32) {
                 const long long base = pol.b.offset + (long long)k * pol.b.row_stride;
@@ -386,7 +389,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
             return AG_ERR_ARG;
         if (!operand_in_range(p.b, p.K, p.N, amap->bytes)) return AG_ERR_ARG;
         if (p.b.present && p.b.layout == AG_LAYOUT_PAGED) {
-            const long long need = tiles_n * ((p.K + 15) / 16);
+            const long long need = tiles_n * (p.tile_n >= 128 ? p.tile_n / 128 : 1) * ((p.K + 15) / 16);
             if (p.b.n_pages < need) return AG_ERR_ARG;
             for (long long i = 0; i < need; ++i)
                 if (p.b.page_table[i] < 0 || (size_t)p.b.page_table[i] >= amap->n_chunks) return AG_ERR_ARG;

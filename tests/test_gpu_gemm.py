@@ -189,3 +189,60 @@ def test_bounded_wait_gives_up_and_leaves_the_device_usable():
     A, B = inputs.small_int_bf16(256, 64, 1), inputs.small_int_bf16(64, 256, 2)
     C = run_gemm(A, B, plan_for(256, 256, 64))               # the context still works
     assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+
+
+def packed_dense_setup(M, N, K, raster_group=2, integer=True, seed=51):
+    topo = device_topo()
+    if integer:
+        A, B = inputs.small_int_bf16(M, K, seed), inputs.small_int_bf16(K, N, seed + 1)
+    else:
+        A, B = inputs.gemm_inputs(M, N, K, seed=seed)
+    kw = dict(M=M, N=N, K=K, tile_m=256, tile_n=256, raster_group=raster_group)
+    plan_d = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+    dst_bytes = 2 * K * ((N + 255) // 256 * 256) * 2 + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    dB = to_dev_bf16(B)
+    packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes)
+    return topo, A, B, kw, plan_d, dst, amap, packed
+
+
+@pytest.mark.parametrize("shape", [(256, 256, 64), (1024, 1024, 512), (1000, 776, 192), (2048, 2304, 1536)])
+def test_block_pairs_over_die_packed_b_integer_exact(shape):
+    M, N, K = shape
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_dense_setup(M, N, K)
+    dA = to_dev_bf16(A)
+    ref = og.gemm_blocked(A, B)
+    for _ in range(2):
+        dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan_d)
+        torch.cuda.synchronize()
+        assert plan_d.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), ref)
+
+
+def test_die_packed_b_pages_and_affinity_plan_match_oracle():
+    from oracle import plan as op
+    M, N, K = 2048, 2048, 256
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_dense_setup(M, N, K, raster_group=4, integer=False)
+    tbl = amap.export()
+    o_plan = op.build_plan(topo.as_dict(), None, topo.n_sm, op.default_policy(kind=op.DIE_COMPACT, **kw))
+    page_die = op.page_die_from_plan(o_plan, K)
+    want_table = op.build_page_table(page_die, dict(chunk_bytes=4096, die_of_chunk=tbl))
+    got_table = packed.page_table()
+    assert np.array_equal(got_table, np.array(want_table, dtype=np.int32))
+    n_chunks = int(got_table.max()) + 1
+    got_img = dst[: n_chunks * 4096].cpu().numpy().view(np.uint16).reshape(n_chunks, 2048)
+    assert np.array_equal(got_img, op.pack_weights(B, want_table, n_chunks))
+    # affinity over the packed B panels: bytewise equal to the oracle's plan, and the GEMM under it is right
+    bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=got_table)
+    plan_a = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, b=bop, **kw))
+    o_aff = op.build_plan(topo.as_dict(), dict(chunk_bytes=4096, die_of_chunk=tbl), topo.n_sm,
+                          op.default_policy(kind=op.AFFINITY, b=op.operand(0, 0, 2, op.LAYOUT_PAGED, want_table), **kw))
+    assert plan_a.export().tobytes() == op.export(o_aff).tobytes()
+    dA = to_dev_bf16(A)
+    dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan_a)
+    torch.cuda.synchronize()
+    assert plan_a.last_status() == ag.AG_OK
+    check_close(dC.cpu().numpy(), og.gemm_blocked(A, B))

@@ -286,6 +286,32 @@ def test_packing_by_plan_is_recovered_by_affinity():
     check_invariants(topo, plan_i, pi, 148)
 
 
+def test_page_owner_for_dense_plans_is_the_majority_die_of_the_column():
+    topo = inputs.synthetic_topo(die0_sms=70, seed=4)
+    kw = dict(M=2048, N=2048, K=256, tile_m=256, tile_n=256, raster_group=4)
+    plan = op.build_plan(topo, None, 148, op.default_policy(kind=op.DIE_COMPACT, **kw))
+    pd = op.page_die_from_plan(plan, 256)
+    ppt, ppc = 16, 2
+    assert len(pd) == 8 * ppc * ppt
+    unit_die = {u: d for d in (0, 1) for u in plan["die_q"][d]}
+    for tn in range(8):
+        votes = [sum(1 for tm in range(8) if unit_die[tm * 8 + tn] == d) for d in (0, 1)]
+        want = 0 if votes[0] >= votes[1] else 1
+        assert set(pd[tn * ppc * ppt:(tn + 1) * ppc * ppt]) == {want}
+    # die 0 (70 of 148 SMs) owns the left columns, die 1 the right ones
+    owners = [pd[tn * ppc * ppt] for tn in range(8)]
+    assert owners == sorted(owners) and owners[0] == 0 and owners[-1] == 1
+    # an affinity plan over such a packing keeps every unit of a column on the column's die
+    n_pages = len(pd)
+    amap = dict(chunk_bytes=4096, die_of_chunk=inputs.synthetic_chunk_die(2 * n_pages, seed=6))
+    table = op.build_page_table(pd, amap)
+    bop = op.operand(0, 0, 2, layout=op.LAYOUT_PAGED, page_table=table)
+    pa = op.build_plan(topo, amap, 148, op.default_policy(kind=op.AFFINITY, b=bop, **kw))
+    die_a = {u: d for d in (0, 1) for u in pa["die_q"][d]}
+    agree = sum(1 for u in range(64) if die_a[u] == owners[u % 8])
+    assert agree >= 56                                      # quotas may move a few units of the cut column
+
+
 def test_page_table_views_share_pairs_and_survive_broken_pairs():
     doc = np.array([0, 1, 1, 0, 1, 1, 0, 0, 1, 0], dtype=np.uint8)      # pairs 2 and 3 break the pair rule
     amap = dict(chunk_bytes=4096, die_of_chunk=doc)
