@@ -168,6 +168,16 @@ ag_status ag_affinity_cycles(const ag_affinity_map* amap, uint32_t* cycles, size
  * two latencies were less than 25 % apart, i.e. that did not show opposite tiers. */
 ag_status ag_affinity_check_complement(const ag_affinity_map* amap, const ag_topo_map* map,
                                        size_t* mismatches);
+/*
+ * ag_affinity_fit_hash - partition-hash recovery (Section 6.1.2) from a measured map: which of the
+ * nine chunk-index bits inside a 2 MiB page (address bits 12..20) take part in the XOR (parity)
+ * hash.  Bit b of *mask is set when flipping chunk-index bit b changes the die of most chunks.
+ * *violations (host, may be NULL) = chunks whose die is not parity(index-in-page & mask) ^ c for
+ * the best per-page constant c (measurement noise, or a layout that is not such a hash).  Address
+ * bits above 20 are not visible without physical addresses; they end up in the per-page constants.
+ * Needs a map of at least 4 MiB.  Errors: AG_ERR_ARG.
+ */
+ag_status ag_affinity_fit_hash(const ag_affinity_map* amap, uint32_t* mask, size_t* violations);
 void ag_affinity_destroy(ag_affinity_map* amap);
 
 /* ---- plan (Section 7.1.2) ------------------------------------------------------------ */

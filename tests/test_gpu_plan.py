@@ -153,3 +153,16 @@ def test_bad_arguments():
         assert e.value.status == ag.AG_ERR_ARG
     with pytest.raises(ag.AgError):
         ag.sched_build(topo, None, 149, ag.make_policy(M=128, N=128, K=128))
+
+
+def test_hash_fit_recovers_a_synthetic_xor_mask():
+    """Section 6.1.2 on a made-up layout: die = parity(chunk index in page & mask) ^ per-page constant."""
+    for mask in (0x1EF, 0x1B5, 0x001):
+        tbl = inputs.synthetic_chunk_die(8192, seed=3, mask_bits=mask)
+        amap = ag.affinity_from_table(0, tbl)
+        got, violations = amap.fit_hash()
+        assert got == (mask | 1) and violations == 0
+    noisy = inputs.synthetic_chunk_die(8192, seed=3, mask_bits=0x1EF).copy()
+    noisy[::97] ^= 1
+    got, violations = ag.affinity_from_table(0, noisy).fit_hash()
+    assert got == 0x1EF and 0 < violations <= 8192 // 97 + 1
