@@ -119,12 +119,13 @@ def test_rejects_mismatched_shapes_and_alignment():
         ag.gemm_persistent(t.data_ptr(), t.data_ptr(), c.data_ptr(), 256, 252, 256, p2)
 
 
-def test_full_size_sampled_against_oracle():
-    """8192^3 in the bench's launch configuration; the oracle computes sampled entries one by
-    one and one full 128 x 256 tile."""
+def test_full_size_one_block_tiles_sampled_against_oracle():
+    """8192^3 with one 128 x 256 tile per block (the kernel used for arbitrary SM sets); the
+    headline configuration with block pairs is covered in test_gpu_fullsize.py."""
     M = N = K = 8192
     A, B = inputs.gemm_inputs(M, N, K)
-    plan = plan_for(M, N, K, kind=ag.AG_DIE_COMPACT, raster_group=8)
+    plan = plan_for(M, N, K, kind=ag.AG_DIE_COMPACT, raster_group=16)
+    plan.reset_record()
     C = run_gemm(A, B, plan)
     rng = np.random.default_rng(0)
     rows, cols = rng.integers(0, M, 200), rng.integers(0, N, 200)
