@@ -312,6 +312,41 @@ void ag_packed_destroy(ag_packed_weights* w);
 ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* C, int M, int N, int K,
                                  const ag_plan* plan, void* cuda_stream);
 
+/* ---- grouped (MoE-shaped) decode GEMM --------------------------------------------------------
+ * The paper's best full-GPU result is a grouped GEMM (Section 7.1.2 and its workload appendix: G
+ * experts, expert g multiplies its M_g routed rows by its own K x N weights).  Built here for the
+ * decode-shaped case (M_g <= 32): the plan sees the experts side by side as one problem with
+ * N = G * N_expert columns, so the die-compact rule gives each die a run of experts, and
+ * ag_pack_weights_grouped puts every expert's weights on the die that runs it.
+ */
+typedef struct ag_group_desc ag_group_desc;
+/*
+ *   A_all  device, stacked activations: sum(rows) x K bf16 row-major, expert g owns rows
+ *          [sum(rows[0..g)), + rows[g])
+ *   C_all  device, stacked outputs: sum(rows) x N_expert fp32 row-major, same row ranges
+ *   rows   host [G], 0 <= rows[g] <= tile_m
+ *   B_list host array of G device pointers (K x N_expert bf16 row-major each), or NULL when only
+ *          packed weights will be used
+ *   N_expert % 128 == 0, K % 8 == 0, tile_m in {16, 32}
+ * Errors: AG_ERR_ARG, AG_ERR_CUDA, AG_ERR_NOMEM.
+ */
+ag_status ag_group_desc_create(const void* A_all, void* C_all, const int32_t* rows, int G,
+                               const void* const* B_list, int N_expert, int K, int tile_m,
+                               ag_group_desc** out);
+void ag_group_desc_destroy(ag_group_desc* d);
+/* As ag_pack_weights for G weight matrices; plan: N = G * N_expert, tile_n = 128, one tile row. */
+ag_status ag_pack_weights_grouped(const void* const* B_list, int G, int K, int N_expert, const ag_plan* plan,
+                                  const ag_affinity_map* amap, void* dst, size_t dst_bytes,
+                                  ag_packed_weights** out);
+/*
+ * gemm_persistent_grouped - C_g = A_g * B_g for all experts in one persistent launch.
+ *   W     packed weights from ag_pack_weights_grouped, or NULL to read the row-major B_list
+ *   plan  M = max rows of an expert (<= tile_m), N = G * N_expert, K, tile_n = 128
+ * Asynchronous on cuda_stream; split-K modes as gemm_persistent_packed.  Errors as gemm_persistent.
+ */
+ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weights* W, const ag_plan* plan,
+                                  void* cuda_stream);
+
 /*
  * gemm_persistent_noalloc - the decode-shaped gemm_persistent (M <= 32, row-major B) for callers
  * that cannot allocate device memory when they need the result.  (The paper has no counterpart;

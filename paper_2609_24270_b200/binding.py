@@ -28,7 +28,8 @@ EXPORTED = [
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
     "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
-    "ag_topo_load", "ag_strerror", "ag_last_cuda_error",
+    "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
+    "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
     "ag_kernel_launch_count",
 ]
 
@@ -140,6 +141,11 @@ def lib() -> C.CDLL:
     L.ag_wait_probe.argtypes = [C.c_uint64, C.POINTER(C.c_uint64)]
     L.ag_topo_save.argtypes = [C.POINTER(TopoMap), C.c_char_p]
     L.ag_topo_load.argtypes = [C.c_char_p, C.POINTER(TopoMap)]
+    L.ag_group_desc_create.argtypes = [vp, vp, vp, C.c_int, vp, C.c_int, C.c_int, C.c_int, C.POINTER(vp)]
+    L.ag_group_desc_destroy.argtypes = [vp]
+    L.ag_group_desc_destroy.restype = None
+    L.ag_pack_weights_grouped.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, vp, vp, sz, C.POINTER(vp)]
+    L.gemm_persistent_grouped.argtypes = [vp, vp, vp, vp]
     L.ag_strerror.argtypes = [C.c_int]
     L.ag_strerror.restype = C.c_char_p
     L.ag_last_cuda_error.restype = C.c_int
@@ -419,3 +425,40 @@ def gemm_persistent_noalloc(a_ptr: int, b_ptr: int, c_ptr: int, M: int, N: int, 
     device array instead of allocated memory; for callers that may not allocate.  Calls on one GPU
     must not overlap.  Limits: k_splits * M * N * 4 <= 8 MiB, N <= 131072."""
     _check(lib().gemm_persistent_noalloc(a_ptr, b_ptr, c_ptr, M, N, K, plan.handle, stream), "gemm_persistent_noalloc")
+
+
+class GroupDesc:
+    """Stacked activations / outputs and per-expert weights of a grouped decode GEMM."""
+
+    def __init__(self, a_ptr: int, c_ptr: int, rows, b_ptrs, n_expert: int, K: int, tile_m: int):
+        r = np.ascontiguousarray(rows, dtype=np.int32)
+        bl = (C.c_void_p * len(b_ptrs))(*b_ptrs) if b_ptrs is not None else None
+        h = C.c_void_p()
+        _check(lib().ag_group_desc_create(a_ptr, c_ptr, r.ctypes.data, r.size, bl, n_expert, K, tile_m, C.byref(h)),
+               "ag_group_desc_create")
+        self.handle = h
+
+    def destroy(self):
+        if self.handle:
+            lib().ag_group_desc_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def pack_weights_grouped(b_ptrs, K: int, n_expert: int, plan: Plan, amap: AffinityMap, dst_ptr: int,
+                         dst_bytes: int) -> PackedWeights:
+    bl = (C.c_void_p * len(b_ptrs))(*b_ptrs)
+    h = C.c_void_p()
+    _check(lib().ag_pack_weights_grouped(bl, len(b_ptrs), K, n_expert, plan.handle, amap.handle, dst_ptr, dst_bytes,
+                                         C.byref(h)), "ag_pack_weights_grouped")
+    return PackedWeights(h)
+
+
+def gemm_persistent_grouped(desc: GroupDesc, packed, plan: Plan, stream: int = 0):
+    _check(lib().gemm_persistent_grouped(desc.handle, packed.handle if packed is not None else None, plan.handle, stream),
+           "gemm_persistent_grouped")

@@ -338,13 +338,6 @@ static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream
 
 }  // namespace ag
 
-namespace ag {
-ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
-                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream);
-ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
-                             const ag_plan* plan, cudaStream_t stream);
-}
-
 using namespace ag;
 
 extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, int M, int N, int K,

@@ -56,7 +56,39 @@ struct SkinnyArgs {
     float* C;
     float* partial;               // [k_splits][M][N] or null when k_splits == 1
     int* sem;                     // [tiles_n * 4]: one arrival counter per 32-column quarter of a tile
+    // grouped (MoE-shaped) operation: the plan's N is G experts side by side, expert g = column tiles
+    // [g * tiles_per_group, (g + 1) * tiles_per_group); null / 0 when there is a single problem
+    const CUtensorMap* g_tm_a;    // device [G]: activations of expert g (rows of the stacked A)
+    const CUtensorMap* g_tm_w;    // device [G]: row-major weights of expert g (not PACKED)
+    const int* g_rows;            // device [G]
+    const int* g_row_off;         // device [G]
+    int tiles_per_group;
+    int n_group;                  // columns of one expert
 };
+
+// Where the output rows of column tile tn live: single problem = C itself; grouped = rows of expert g in the
+// stacked C (row stride = columns of one expert).
+struct OutView {
+    float* base;      // element (row 0, column 0 of the tile's problem)
+    int rows;         // valid rows
+    int ld;           // row stride in elements
+    int col0;         // first column of tile tn inside its problem
+    int n_cols;       // columns of the problem
+};
+__device__ __forceinline__ OutView out_view(const PersistParams& p, const SkinnyArgs& x, int tn) {
+    OutView v;
+    if (x.g_rows) {
+        const int g = tn / x.tiles_per_group, tl = tn - g * x.tiles_per_group;
+        v.base = x.C + (size_t)x.g_row_off[g] * x.n_group;
+        v.rows = x.g_rows[g];
+        v.ld = x.n_group;
+        v.col0 = tl * SK_BN;
+        v.n_cols = x.n_group;
+    } else {
+        v.base = x.C; v.rows = p.M; v.ld = p.N; v.col0 = tn * SK_BN; v.n_cols = p.N;
+    }
+    return v;
+}
 
 template <int NM, bool PACKED>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -129,6 +161,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             ++it;
             if (!ok || u < 0) break;
             const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
+            const int grp = x.tiles_per_group ? tn / x.tiles_per_group : 0;      // expert of this column tile
+            const int tl = x.tiles_per_group ? tn - grp * x.tiles_per_group : tn;  // tile inside the expert
             const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
             const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
             for (int sb = s0; sb < s1 && ok; sb += 8) {
@@ -159,15 +193,16 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         if (lane < 4)
                             bulk_load_hint(sw + lane * 4096, x.packed + (size_t)page * AG_CHUNK_BYTES, 4096, bar, stream_policy);
                     } else if (lane == 0) {
+                        const CUtensorMap* mw = x.g_tm_w ? &x.g_tm_w[grp] : &tm_w;
                         if (p.b_blocks) {
                             // both 64-column blocks with one copy (B seen as [N/64][K][64])
-                            tma_load_3d_hint(sw, &tm_w, bar, 0, s * SK_BK, tn * 2, stream_policy);
+                            tma_load_3d_hint(sw, mw, bar, 0, s * SK_BK, tl * 2, stream_policy);
                         } else {
-                            tma_load_2d_hint(sw, &tm_w, bar, tn * SK_BN, s * SK_BK, stream_policy);
-                            tma_load_2d_hint(sw + 8192, &tm_w, bar, tn * SK_BN + 64, s * SK_BK, stream_policy);
+                            tma_load_2d_hint(sw, mw, bar, tl * SK_BN, s * SK_BK, stream_policy);
+                            tma_load_2d_hint(sw + 8192, mw, bar, tl * SK_BN + 64, s * SK_BK, stream_policy);
                         }
                     }
-                    if (lane == 0) tma_load_2d(sa, &tm_a, bar, s * SK_BK, 0);
+                    if (lane == 0) tma_load_2d(sa, x.g_tm_a ? &x.g_tm_a[grp] : &tm_a, bar, s * SK_BK, 0);
                 }
             }
         }
@@ -255,8 +290,10 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             // lane = (row group lane/8, four columns); the k_splits loads of one output quad are in flight
             // together and are added in ascending split order
             const int nq = tn * SK_BN + q * 32 + (lane & 7) * 4;
-            if (nq < p.N) {
-                for (int m = lane >> 3; m < p.M; m += 4) {
+            const OutView ov = out_view(p, x, tn);
+            const int nlq = ov.col0 + q * 32 + (lane & 7) * 4;
+            if (nq < p.N && nlq < ov.n_cols) {
+                for (int m = lane >> 3; m < ov.rows; m += 4) {
                     float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int k0 = 0; k0 < p.k_splits; k0 += 16) {
                         float4 t[16];
@@ -271,7 +308,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                                 acc4.x += t[k].x; acc4.y += t[k].y; acc4.z += t[k].z; acc4.w += t[k].w;
                             }
                     }
-                    *reinterpret_cast<float4*>(x.C + (size_t)m * p.N + nq) = acc4;
+                    *reinterpret_cast<float4*>(ov.base + (size_t)m * ov.ld + nlq) = acc4;
                 }
             }
             __syncwarp();
@@ -331,24 +368,30 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
             ++tile_it;
-            const int n = tn * SK_BN + q * 32 + lane;
+            const int n = tn * SK_BN + q * 32 + lane;     // column in the plan's (possibly grouped) N
+            const OutView ov = out_view(p, x, tn);
+            const int nl = ov.col0 + q * 32 + lane;       // column inside the tile's problem
             if (p.k_splits > 1 && x.partial == nullptr) {
                 // in-memory reduction: C was zeroed before the launch, every unit adds its partial sums
                 // with reductions that L2 carries out; nothing comes back, so nothing is waited for
-                if (n < p.N) {
+                if (nl < ov.n_cols) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m)
-                        if (m < p.M) atomicAdd(x.C + (size_t)m * p.N + n, sum[m]);
+                        if (m < ov.rows) atomicAdd(ov.base + (size_t)m * ov.ld + nl, sum[m]);
                 }
-            } else {
-                if (p.k_splits > 1) hand_off(old_use, old_new);
-                float* out = p.k_splits > 1 ? x.partial + (size_t)ks * p.M * p.N : x.C;
+            } else if (p.k_splits > 1) {
+                hand_off(old_use, old_new);
+                float* out = x.partial + (size_t)ks * p.M * p.N;   // workspace rows: the plan's M bound, columns: the plan's N
                 if (n < p.N) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m)
                         if (m < p.M) out[(size_t)m * p.N + n] = sum[m];
                 }
-                if (p.k_splits > 1) st_tn = tn;
+                st_tn = tn;
+            } else if (nl < ov.n_cols) {
+#pragma unroll
+                for (int m = 0; m < NM; ++m)
+                    if (m < ov.rows) ov.base[(size_t)m * ov.ld + nl] = sum[m];
             }
             if (lane == 0 && q == 0) {
                 p.tile_owner[u] = my_sm;
@@ -417,7 +460,8 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
 
 // Shared host path of the two skinny entry points.
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
-                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream) {
+                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream,
+                               const ag_group_desc* grp) {
     const int32_t* h = plan->header;
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_N] != SK_BN || (h[H_TILE_M] != 16 && h[H_TILE_M] != 32) || M > h[H_TILE_M]) return AG_ERR_ARG;
@@ -432,9 +476,18 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     const int NM = h[H_TILE_M];
     CUtensorMap tm_a, tm_w;
     memset(&tm_w, 0, sizeof tm_w);
-    if (!encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, SK_BK, NM)) return AG_ERR_CUDA;
+    memset(&tm_a, 0, sizeof tm_a);
+    if (!grp && !encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, SK_BK, NM)) return AG_ERR_CUDA;
     SkinnyArgs x;
     memset(&x, 0, sizeof x);
+    if (grp) {
+        x.g_tm_a = grp->d_tm_a;
+        x.g_tm_w = W ? nullptr : grp->d_tm_w;
+        x.g_rows = grp->d_rows;
+        x.g_row_off = grp->d_row_off;
+        x.tiles_per_group = grp->N / SK_BN;
+        x.n_group = grp->N;
+    }
     x.C = (float*)Cout;
     x.partial = h[H_KSPLITS] > 1 ? partial : nullptr;
     x.sem = sem;
@@ -443,6 +496,8 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
         x.packed = W->dst;
         x.page_table = W->d_page_table;
         x.pages_per_tile = W->pages_per_tile;
+    } else if (grp) {
+        if (!grp->d_tm_w) return AG_ERR_ARG;  // the descriptor was made without row-major weights
     } else {
         if (!B_rowmajor || ((uintptr_t)B_rowmajor & 15u)) return AG_ERR_ARG;
         if (N % 64 == 0) {
@@ -451,10 +506,12 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
             return AG_ERR_CUDA;
         }
     }
-    if (h[H_KSPLITS] > 1 && !x.partial)  // in-memory reduction mode: the adds need a zeroed C
-        AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * (size_t)M * (size_t)N, stream));
+    if (h[H_KSPLITS] > 1 && !x.partial) {  // in-memory reduction mode: the adds need a zeroed C
+        const size_t c_elems = grp ? (size_t)grp->total_rows * (size_t)grp->N : (size_t)M * (size_t)N;
+        AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * c_elems, stream));
+    }
     PersistParams gp = make_persist_params(plan, M, N, K);
-    gp.b_blocks = (!W && N % 64 == 0) ? 1 : 0;
+    gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
     if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream)
                            : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream);
     return W ? launch_skinny<32, true>(plan, tm_a, tm_w, gp, x, stream)
@@ -465,9 +522,15 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
 
 using namespace ag;
 
-extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
-                                     void* dst, size_t dst_bytes, ag_packed_weights** out) {
-    if (!B || !plan || !amap || !dst || !out || K <= 0 || N <= 0) return AG_ERR_ARG;
+// Packs G source matrices (K x n_src each, row-major) side by side: the plan's N is G * n_src.  G = 1 is the
+// plain case.
+static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int N, const ag_plan* plan,
+                                   const ag_affinity_map* amap, void* dst, size_t dst_bytes, ag_packed_weights** out) {
+    if (!B_list || G < 1 || !plan || !amap || !dst || !out || K <= 0 || N <= 0 || (N % G)) return AG_ERR_ARG;
+    for (int g = 0; g < G; ++g)
+        if (!B_list[g]) return AG_ERR_ARG;
+    const int n_src = N / G;
+    if (G > 1 && (n_src % 128)) return AG_ERR_ARG;  // experts must start on a page-column boundary
     *out = nullptr;
     const int32_t* h = plan->header;
     if ((h[H_TILE_N] != 128 && h[H_TILE_N] != 256) || h[H_N] != N || h[H_K] != K || (K % SK_BK)) return AG_ERR_ARG;
@@ -524,8 +587,10 @@ extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan*
     cudaError_t e = cudaMalloc(&w->d_page_table, sizeof(int32_t) * n_pages);
     if (e == cudaSuccess)
         e = cudaMemcpy(w->d_page_table, w->h_page_table.data(), sizeof(int32_t) * n_pages, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) {
-        k_pack_weights<<<(unsigned)n_pages, 128>>>((const uint16_t*)B, K, N, ppt, w->d_page_table, (uint8_t*)dst);
+    const size_t pages_per_src = n_pages / G;
+    for (int g = 0; g < G && e == cudaSuccess; ++g) {
+        k_pack_weights<<<(unsigned)pages_per_src, 128>>>((const uint16_t*)B_list[g], K, n_src, ppt,
+                                                        w->d_page_table + (size_t)g * pages_per_src, (uint8_t*)dst);
         count_launch();
         e = cudaGetLastError();
     }
@@ -537,6 +602,101 @@ extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan*
     }
     *out = w;
     return AG_OK;
+}
+
+extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
+                                     void* dst, size_t dst_bytes, ag_packed_weights** out) {
+    const void* list[1] = {B};
+    return pack_weights_impl(list, 1, K, N, plan, amap, dst, dst_bytes, out);
+}
+
+extern "C" ag_status ag_pack_weights_grouped(const void* const* B_list, int G, int K, int N_expert, const ag_plan* plan,
+                                             const ag_affinity_map* amap, void* dst, size_t dst_bytes,
+                                             ag_packed_weights** out) {
+    if (G < 1 || N_expert <= 0 || (long long)G * N_expert > 0x7fffffff) return AG_ERR_ARG;
+    return pack_weights_impl(B_list, G, K, G * N_expert, plan, amap, dst, dst_bytes, out);
+}
+
+// ---- grouped (MoE-shaped) decode GEMM -------------------------------------------------------------------
+extern "C" void ag_group_desc_destroy(ag_group_desc* d) {
+    if (!d) return;
+    cudaFree(d->d_tm_a);
+    cudaFree(d->d_tm_w);
+    cudaFree(d->d_rows);
+    cudaFree(d->d_row_off);
+    delete d;
+}
+
+extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const int32_t* rows, int G,
+                                          const void* const* B_list, int N_expert, int K, int tile_m,
+                                          ag_group_desc** out) {
+    if (!A_all || !C_all || !rows || !out || G < 1 || G > 4096 || N_expert <= 0 || K <= 0) return AG_ERR_ARG;
+    if ((tile_m != 16 && tile_m != 32) || (N_expert % SK_BN) || (K % 8)) return AG_ERR_ARG;
+    if (((uintptr_t)A_all | (uintptr_t)C_all) & 15u) return AG_ERR_ARG;
+    *out = nullptr;
+    long long total = 0;
+    for (int g = 0; g < G; ++g) {
+        if (rows[g] < 0 || rows[g] > tile_m) return AG_ERR_ARG;
+        total += rows[g];
+    }
+    if (total < 1) return AG_ERR_ARG;
+    ag_group_desc* d = new (std::nothrow) ag_group_desc();
+    if (!d) return AG_ERR_NOMEM;
+    d->G = G; d->N = N_expert; d->K = K; d->tile_m = tile_m; d->total_rows = total;
+    d->A_all = A_all; d->C_all = C_all;
+    d->d_tm_a = nullptr; d->d_tm_w = nullptr; d->d_rows = nullptr; d->d_row_off = nullptr;
+    d->w_blocks = (N_expert % 64 == 0) ? 1 : 0;
+    d->rows.assign(rows, rows + G);
+    d->row_off.resize(G);
+    std::vector<CUtensorMap> ha(G), hw(B_list ? G : 0);
+    long long off = 0;
+    for (int g = 0; g < G; ++g) {
+        d->row_off[g] = (int)off;
+        // an expert without rows still gets a (one-row) view inside the buffer; nothing of it is stored
+        const long long first = std::min(off, total - 1);
+        const int n_rows = std::max(1, rows[g]);
+        const char* base = (const char*)A_all + (size_t)first * K * 2;
+        if (!encode_2d(&ha[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, (uint64_t)std::min<long long>(n_rows, total - first),
+                       K, SK_BK, tile_m)) {
+            delete d;
+            return AG_ERR_CUDA;
+        }
+        if (B_list) {
+            if (!B_list[g] || ((uintptr_t)B_list[g] & 15u)) { delete d; return AG_ERR_ARG; }
+            const bool ok = d->w_blocks ? encode_b_blocks(&hw[g], B_list[g], K, N_expert, SK_BK, 2)
+                                        : encode_2d(&hw[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_list[g], K, N_expert, 64, SK_BK);
+            if (!ok) { delete d; return AG_ERR_CUDA; }
+        }
+        off += rows[g];
+    }
+    cudaError_t e = cudaMalloc(&d->d_tm_a, sizeof(CUtensorMap) * G);
+    if (e == cudaSuccess) e = cudaMemcpy(d->d_tm_a, ha.data(), sizeof(CUtensorMap) * G, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && B_list) {
+        e = cudaMalloc(&d->d_tm_w, sizeof(CUtensorMap) * G);
+        if (e == cudaSuccess) e = cudaMemcpy(d->d_tm_w, hw.data(), sizeof(CUtensorMap) * G, cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) e = cudaMalloc(&d->d_rows, sizeof(int) * G);
+    if (e == cudaSuccess) e = cudaMemcpy(d->d_rows, d->rows.data(), sizeof(int) * G, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&d->d_row_off, sizeof(int) * G);
+    if (e == cudaSuccess) e = cudaMemcpy(d->d_row_off, d->row_off.data(), sizeof(int) * G, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        ag_group_desc_destroy(d);
+        return cuda_fail(e);
+    }
+    *out = d;
+    return AG_OK;
+}
+
+extern "C" ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weights* W, const ag_plan* plan,
+                                             void* cuda_stream) {
+    if (!d || !plan) return AG_ERR_ARG;
+    const int32_t* h = plan->header;
+    // the plan sees the experts side by side: N = G * N_expert, one tile row of at most tile_m rows
+    if (h[H_N] != d->G * d->N || h[H_K] != d->K || h[H_TILE_M] != d->tile_m || h[H_M] > d->tile_m) return AG_ERR_ARG;
+    for (int g = 0; g < d->G; ++g)
+        if (d->rows[g] > h[H_M]) return AG_ERR_ARG;
+    return gemm_skinny_dispatch(d->A_all, nullptr, W, d->C_all, h[H_M], h[H_N], h[H_K], plan, plan->d_partial, plan->d_sem,
+                                reinterpret_cast<cudaStream_t>(cuda_stream), d);
 }
 
 extern "C" ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* outp, size_t cap, size_t* n_pages) {
@@ -552,11 +712,6 @@ extern "C" void ag_packed_destroy(ag_packed_weights* w) {
     if (!w) return;
     cudaFree(w->d_page_table);
     delete w;
-}
-
-namespace ag {
-ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
-                             const ag_plan* plan, cudaStream_t stream);
 }
 
 extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weights* W, void* Cout, int M, int N, int K,

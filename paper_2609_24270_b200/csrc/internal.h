@@ -89,6 +89,21 @@ struct ag_packed_weights {
     std::vector<int32_t> h_page_table;
 };
 
+// Grouped (MoE-shaped) decode GEMM: G experts, expert g multiplies rows [row_off[g], row_off[g] + rows[g]) of the
+// stacked activations by its own K x N weights.
+struct ag_group_desc {
+    int G, N, K, tile_m;
+    long long total_rows;
+    const void* A_all;
+    void* C_all;
+    std::vector<int> rows, row_off;
+    CUtensorMap* d_tm_a;   // device [G]: activations of expert g
+    CUtensorMap* d_tm_w;   // device [G]: row-major weights of expert g (null when only packed weights are used)
+    int* d_rows;           // device [G]
+    int* d_row_off;        // device [G]
+    int w_blocks;          // 1: d_tm_w are the 3-D [N/64][K][64] views
+};
+
 namespace ag {
 extern thread_local int g_last_cuda_error;
 extern std::atomic<unsigned long long> g_launch_count;

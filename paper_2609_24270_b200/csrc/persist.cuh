@@ -157,4 +157,11 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const vo
 // n_blocks 64-column blocks of a k-slab with a single copy, each block laid out as a separate 2-D box would be.
 bool encode_b_blocks(CUtensorMap* tm, const void* ptr, uint64_t K, uint64_t N, uint32_t box_k, uint32_t n_blocks);
 
+// Host-side dispatchers of the kernel families (defined next to their kernels).
+ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
+                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream,
+                               const ag_group_desc* grp = nullptr);
+ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
+                             const ag_plan* plan, cudaStream_t stream);
+
 }  // namespace ag

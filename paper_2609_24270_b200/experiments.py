@@ -4,6 +4,7 @@
     python -m paper_2609_24270_b200.experiments --config 4
     python -m paper_2609_24270_b200.experiments --config 5
     python -m paper_2609_24270_b200.experiments --config raster      # raster-group sweep at 8192^3
+    python -m paper_2609_24270_b200.experiments --config groupgemm   # MoE-shaped grouped decode GEMM
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
 launches first, median of the timed launches.  torch is used for device memory, streams and events.
@@ -259,6 +260,67 @@ def raster(fh, topo):
                   tflops=flops / (float(np.median(v)) * 1e-3) / 1e12), fh)
 
 
+# ---------------------------------------------------------------------------------------------
+def time_queued(fn, warmup=3, iters=12):
+    """Median GPU time per call with the calls queued behind a device-side blocker, so that host-side
+    launch cost is not on the clock (the kernels here take tens of microseconds)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    s = torch.cuda.current_stream()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    torch.cuda._sleep(int(2e7))
+    evs[0].record(s)
+    for i in range(iters):
+        fn()
+        evs[i + 1].record(s)
+    torch.cuda.synchronize()
+    return float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(iters)]))
+
+
+def groupgemm(fh, topo, seeds=(1, 2)):
+    """The decode-shaped settings of the paper's GroupGEMM study (its workload appendix): (G, M) in
+    {(32, 20), (6, 20)}, (N, K) in {(6144, 7168), (7168, 3072), (4096, 4096), (4096, 2048)}, rows per
+    expert M_i = floor(M U_i), U_i ~ U(0.7, 1.3).  Random weights are made on the device (timing only;
+    parity is covered by the tests)."""
+    for G, M in ((32, 20), (6, 20)):
+        for N, K in ((6144, 7168), (7168, 3072), (4096, 4096), (4096, 2048)):
+            tiles = G * N // 128
+            ksp = 1
+            while tiles * ksp < 6 * topo.n_sm and K // 64 // (2 * ksp) >= 4:
+                ksp *= 2
+            Bs = [torch.randn((K, N), dtype=torch.bfloat16, device="cuda") for _ in range(G)]
+            w_bytes = G * K * N * 2
+            dst_bytes = 2 * w_bytes + (16 << 20)
+            dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+            for seed in seeds:
+                rows = inputs.group_rows(G, M, seed)
+                total = int(rows.sum())
+                dA = torch.randn((total, K), dtype=torch.bfloat16, device="cuda")
+                dC = torch.empty((total, N), dtype=torch.float32, device="cuda")
+                kw = dict(M=int(rows.max()), N=G * N, K=K, tile_m=32, tile_n=128, k_splits=ksp, splitk_in_memory=1)
+                plan_obl = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
+                plan_dc = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+                packed = ag.pack_weights_grouped([b.data_ptr() for b in Bs], K, N, plan_dc, amap, dst.data_ptr(), dst_bytes)
+                bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packed.page_table())
+                plan_rem = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
+                desc_rm = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, [b.data_ptr() for b in Bs], N, K, 32)
+                algo = w_bytes + total * K * 2 + total * N * 4
+                res = {}
+                for name, pk, plan in (("rowmajor_oblivious", None, plan_obl), ("rowmajor_die_compact", None, plan_dc),
+                                       ("packed_die_local", packed, plan_dc), ("packed_remote", packed, plan_rem)):
+                    ms = time_queued(lambda: ag.gemm_persistent_grouped(desc_rm, pk, plan))
+                    assert plan.last_status() == ag.AG_OK
+                    res[name] = algo / (ms * 1e-3) / 1e9
+                emit(dict(config="groupgemm", G=G, M=M, N=N, K=K, seed=seed, rows_total=total, k_splits=ksp,
+                          weight_gb=w_bytes / 1e9, gbs=res, local_over_remote=res["packed_die_local"] / res["packed_remote"],
+                          local_over_rowmajor_oblivious=res["packed_die_local"] / res["rowmajor_oblivious"]), fh)
+                del packed, desc_rm, dA, dC
+            del Bs, dst, amap
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -269,7 +331,7 @@ def main():
     emit(dict(config="topology", n_sm=topo.n_sm, die_sm_count=list(topo.die_sm_count),
               gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
-    {"3": config3, "4": config4, "5": config5, "raster": raster}[args.config](fh, topo)
+    {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm}[args.config](fh, topo)
 
 
 if __name__ == "__main__":

@@ -87,6 +87,14 @@ def gemm_inputs(M: int, N: int, K: int, seed: int = DEFAULT_SEED):
     return uniform_bf16(M, K, seed), uniform_bf16(K, N, seed + 1)
 
 
+def group_rows(G: int, M: int, seed: int) -> np.ndarray:
+    """Rows per expert of a grouped GEMM as in the paper's workload appendix: M_i = floor(M * U_i),
+    U_i uniform in [0.7, 1.3), drawn from the repo's counter-based mixer."""
+    h = mix64_np(np.arange(G, dtype=np.uint64) + mix64_np(np.array([seed], dtype=np.uint64))[0])
+    u = 0.7 + 0.6 * ((h >> np.uint64(40)).astype(np.float64) / float(1 << 24))
+    return np.floor(M * u).astype(np.int32)
+
+
 # ----------------------------------------------------------------------------
 # Synthetic chips and affinity maps for the CPU-side plan tests.
 # ----------------------------------------------------------------------------
