@@ -324,10 +324,11 @@ typedef struct ag_group_desc ag_group_desc;
  *   A_all  device, stacked activations: sum(rows) x K bf16 row-major, expert g owns rows
  *          [sum(rows[0..g)), + rows[g])
  *   C_all  device, stacked outputs: sum(rows) x N_expert fp32 row-major, same row ranges
- *   rows   host [G], 0 <= rows[g] <= tile_m
+ *   rows   host [G]; decode-shaped descriptors: 0 <= rows[g] <= tile_m; dense descriptors
+ *          (tile_m = 256, block pairs, N_expert % 256 == 0): any row count
  *   B_list host array of G device pointers (K x N_expert bf16 row-major each), or NULL when only
  *          packed weights will be used
- *   N_expert % 128 == 0, K % 8 == 0, tile_m in {16, 32}
+ *   N_expert % 128 == 0, K % 8 == 0, tile_m in {16, 32, 256}
  * Errors: AG_ERR_ARG, AG_ERR_CUDA, AG_ERR_NOMEM.
  */
 ag_status ag_group_desc_create(const void* A_all, void* C_all, const int32_t* rows, int G,
@@ -341,7 +342,9 @@ ag_status ag_pack_weights_grouped(const void* const* B_list, int G, int K, int N
 /*
  * gemm_persistent_grouped - C_g = A_g * B_g for all experts in one persistent launch.
  *   W     packed weights from ag_pack_weights_grouped, or NULL to read the row-major B_list
- *   plan  M = max rows of an expert (<= tile_m), N = G * N_expert, K, tile_n = 128
+ *   plan  M = max rows of an expert, N = G * N_expert, K; decode-shaped: tile_n = 128, M <= tile_m;
+ *         dense: tile_m = tile_n = 256, SM set of whole TPCs (units below an expert's last row are
+ *         skipped, so prefer static lists built from balanced row counts)
  * Asynchronous on cuda_stream; split-K modes as gemm_persistent_packed.  Errors as gemm_persistent.
  */
 ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weights* W, const ag_plan* plan,

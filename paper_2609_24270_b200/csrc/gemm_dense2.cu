@@ -100,11 +100,27 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
         : "memory");
 }
 
-// Unit sequence of a pair: the two task lists in alternation, the lower slot first.
+// Grouped (MoE-shaped) operation: the plan's N is G experts side by side (expert g = unit columns
+// [g * tiles_per_group, (g + 1) * tiles_per_group)), its M the largest row count; every expert has its own
+// A, B and C.  All pointers null / 0 for a single problem.
+struct GroupView {
+    const CUtensorMap* tm_a;   // device [G]
+    const CUtensorMap* tm_b;   // device [G] (row-major weights; unused with packed B)
+    const CUtensorMap* tm_c;   // device [G]
+    const int* rows;           // device [G]
+    int tiles_per_group;       // 256-column units per expert
+    int n_group;               // columns of one expert
+};
+
+// Unit sequence of a pair: the two task lists in alternation, the lower slot first.  In grouped operation
+// units that lie below an expert's last row are skipped here, so no role ever sees them.
 struct PairSource {
     const int32_t* image;
+    const int* g_rows;
+    int tiles_per_group, tiles_n;
     int off[2], len[2], pos;
-    __device__ PairSource(const PersistParams& p, int slot_a, int slot_b) : image(p.image), pos(0) {
+    __device__ PairSource(const PersistParams& p, int slot_a, int slot_b, const GroupView& gv)
+        : image(p.image), g_rows(gv.rows), tiles_per_group(gv.tiles_per_group), tiles_n(p.tiles_n), pos(0) {
         const PlanLayout lay{p.b, p.n_units, p.n_sm};
         const int lo = min(slot_a, slot_b), hi = max(slot_a, slot_b);
         off[0] = lay.sm_q() + p.image[lay.sm_q_off() + lo];
@@ -114,16 +130,20 @@ struct PairSource {
     }
     __device__ int next() {
         const int common = 2 * min(len[0], len[1]);
-        int u = -1;
-        if (pos < common) {
-            u = image[off[pos & 1] + (pos >> 1)];
-        } else {
-            const int longer = len[0] >= len[1] ? 0 : 1;
-            const int i = (common >> 1) + (pos - common);
-            if (i < len[longer]) u = image[off[longer] + i];
+        while (true) {
+            int u = -1;
+            if (pos < common) {
+                u = image[off[pos & 1] + (pos >> 1)];
+            } else {
+                const int longer = len[0] >= len[1] ? 0 : 1;
+                const int i = (common >> 1) + (pos - common);
+                if (i < len[longer]) u = image[off[longer] + i];
+            }
+            ++pos;
+            if (u < 0 || !g_rows) return u;
+            const int tm = u / tiles_n, g = (u % tiles_n) / tiles_per_group;
+            if (tm * 2 * 128 < g_rows[g]) return u;   // the expert has rows in this unit row
         }
-        ++pos;
-        return u;
     }
 };
 
@@ -133,7 +153,7 @@ template <bool PACKED_B>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                        const __grid_constant__ CUtensorMap tm_c, const PersistParams p,
-                       const int32_t* __restrict__ page_table, const int pages_per_block) {
+                       const int32_t* __restrict__ page_table, const int pages_per_block, const GroupView gv) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -194,7 +214,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
             // ------------------------------------------------ scheduler + TMA producer.  Every lane walks the same
             // unit sequence; lane 0 waits and issues.  For packed B the 32 lanes fetch the page-table entries of
             // the next eight k-slabs with one load each.
-            PairSource src(p, slot, peer_slot);
+            PairSource src(p, slot, peer_slot, gv);
             uint32_t it = 0, kit = 0;
             int ok = 1;
             while (ok) {
@@ -213,6 +233,10 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 ++it;
                 if (!ok || u < 0) break;
                 const int tm = u / p.tiles_n, tn = u % p.tiles_n;
+                const int grp = gv.rows ? tn / gv.tiles_per_group : 0;        // expert of this unit column
+                const int tl = gv.rows ? tn - grp * gv.tiles_per_group : tn;  // unit column inside the expert
+                const CUtensorMap* ma = gv.rows ? &gv.tm_a[grp] : &tm_a;
+                const CUtensorMap* mb = (gv.rows && !PACKED_B) ? &gv.tm_b[grp] : &tm_b;
                 // Packed B: the units of one raster group that share a column panel start their k loop at
                 // different k-slabs (the sum over k does not care where it starts), so that at any moment they
                 // read different 4 KB pages: a page sits in few L2 slices, and eight pairs asking for the same
@@ -238,14 +262,14 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                                 ok = 0;
                             } else {
                                 if (leader) mbar_expect_tx(smem_u32(&ctl->full[st]), 2 * P_STAGE_BYTES);
-                                tma_load_2d_pair(sa, &tm_a, bar_leader, s * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
+                                tma_load_2d_pair(sa, ma, bar_leader, s * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
                                 if (!PACKED_B) {
                                     if (p.b_blocks) {
                                         // both 64-column blocks of this block's half with one copy
-                                        tma_load_3d_pair(sb_addr, &tm_b, bar_leader, 0, s * P_BK, tn * 4 + (int)rank * 2);
+                                        tma_load_3d_pair(sb_addr, mb, bar_leader, 0, s * P_BK, tl * 4 + (int)rank * 2);
                                     } else {
-                                        tma_load_2d_pair(sb_addr, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH, s * P_BK);
-                                        tma_load_2d_pair(sb_addr + P_BK * 128, &tm_b, bar_leader, tn * P_BN + (int)rank * P_BNH + 64, s * P_BK);
+                                        tma_load_2d_pair(sb_addr, mb, bar_leader, tl * P_BN + (int)rank * P_BNH, s * P_BK);
+                                        tma_load_2d_pair(sb_addr + P_BK * 128, mb, bar_leader, tl * P_BN + (int)rank * P_BNH + 64, s * P_BK);
                                     }
                                 }
                             }
@@ -337,6 +361,10 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 }
                 tc_fence_after();
                 const int row0 = tm * 2 * P_BM + (int)rank * P_BM + q * 32;
+                const int grp = gv.rows ? tn / gv.tiles_per_group : 0;
+                const int tl = gv.rows ? tn - grp * gv.tiles_per_group : tn;
+                const CUtensorMap* mc = gv.rows ? &gv.tm_c[grp] : &tm_c;
+                const int m_rows = gv.rows ? gv.rows[grp] : p.M, n_cols = gv.rows ? gv.n_group : p.N;
 #pragma unroll 1
                 for (int c = 0; c < P_BN / 32; ++c, ++chunk_it) {
                     uint32_t v[32];
@@ -356,8 +384,8 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        const int x = tn * P_BN + c * 32;
-                        if (x < p.N && row0 < p.M) tma_store_2d(&tm_c, buf, x, row0);
+                        const int x = tl * P_BN + c * 32;
+                        if (x < n_cols && row0 < m_rows) tma_store_2d(mc, buf, x, row0);
                         bulk_commit();
                     }
                 }
@@ -387,7 +415,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 }
 
 ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
-                             const ag_plan* plan, cudaStream_t stream) {
+                             const ag_plan* plan, cudaStream_t stream, const ag_group_desc* grp) {
     const int32_t* h = plan->header;
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_M] != 2 * P_BM || h[H_TILE_N] != P_BN || h[H_KSPLITS] != 1 || !h[H_STATIC]) return AG_ERR_ARG;
@@ -395,9 +423,12 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     if (((uintptr_t)A | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
     if (W) {
         if (W->K != K || W->N != N || (K % P_BK) || W->tiles_n != 2 * h[H_TILES_N]) return AG_ERR_ARG;
+    } else if (grp) {
+        if (!grp->d_tm_w) return AG_ERR_ARG;
     } else if (!B || ((uintptr_t)B & 15u)) {
         return AG_ERR_ARG;
     }
+    if (grp && (!grp->d_tm_c || (grp->N % P_BN))) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
     int dev = 0, n_sm = 0;
@@ -413,7 +444,9 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
             if ((slot_of[s] >= 0) != (slot_of[s ^ 1] >= 0)) return AG_ERR_ARG;
     }
     const void* b_key = W ? (const void*)W : B;
-    if (plan->tm_a_ptr != A || plan->tm_b_ptr != b_key || plan->tm_c_ptr != Cout) {
+    if (grp) {
+        if (W) { plan->tm_b = W->tm_pages; plan->tm_b_ptr = nullptr; }   // the other maps come from the descriptor
+    } else if (plan->tm_a_ptr != A || plan->tm_b_ptr != b_key || plan->tm_c_ptr != Cout) {
         if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)) return AG_ERR_CUDA;
         if (W) plan->tm_b = W->tm_pages;
         else if (N % 64 == 0) { if (!encode_b_blocks(&plan->tm_b, B, K, N, P_BK, 2)) return AG_ERR_CUDA; }
@@ -430,7 +463,13 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
     PersistParams gp = make_persist_params(plan, M, N, K);
-    gp.b_blocks = (!W && N % 64 == 0) ? 1 : 0;
+    gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
+    GroupView gv;
+    memset(&gv, 0, sizeof gv);
+    if (grp) {
+        gv.tm_a = grp->d_tm_a; gv.tm_b = grp->d_tm_w; gv.tm_c = grp->d_tm_c; gv.rows = grp->d_rows;
+        gv.tiles_per_group = grp->N / P_BN; gv.n_group = grp->N;
+    }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(n_sm);
@@ -446,8 +485,8 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     cfg.numAttrs = 1;
     const int32_t* table = W ? W->d_page_table : nullptr;
     const int ppb = W ? W->pages_per_tile : 0;
-    if (W) AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb));
-    else AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb));
+    if (W) AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb, gv));
+    else AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb, gv));
     count_launch();
     return AG_OK;
 }

@@ -622,6 +622,7 @@ extern "C" void ag_group_desc_destroy(ag_group_desc* d) {
     if (!d) return;
     cudaFree(d->d_tm_a);
     cudaFree(d->d_tm_w);
+    cudaFree(d->d_tm_c);
     cudaFree(d->d_rows);
     cudaFree(d->d_row_off);
     delete d;
@@ -631,12 +632,13 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
                                           const void* const* B_list, int N_expert, int K, int tile_m,
                                           ag_group_desc** out) {
     if (!A_all || !C_all || !rows || !out || G < 1 || G > 4096 || N_expert <= 0 || K <= 0) return AG_ERR_ARG;
-    if ((tile_m != 16 && tile_m != 32) || (N_expert % SK_BN) || (K % 8)) return AG_ERR_ARG;
+    const bool dense = tile_m == 256;  // block pairs, 256 x 256 units; else decode-shaped (rows <= tile_m)
+    if ((tile_m != 16 && tile_m != 32 && !dense) || (N_expert % (dense ? 256 : SK_BN)) || (K % 8)) return AG_ERR_ARG;
     if (((uintptr_t)A_all | (uintptr_t)C_all) & 15u) return AG_ERR_ARG;
     *out = nullptr;
     long long total = 0;
     for (int g = 0; g < G; ++g) {
-        if (rows[g] < 0 || rows[g] > tile_m) return AG_ERR_ARG;
+        if (rows[g] < 0 || (!dense && rows[g] > tile_m)) return AG_ERR_ARG;
         total += rows[g];
     }
     if (total < 1) return AG_ERR_ARG;
@@ -644,11 +646,12 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
     if (!d) return AG_ERR_NOMEM;
     d->G = G; d->N = N_expert; d->K = K; d->tile_m = tile_m; d->total_rows = total;
     d->A_all = A_all; d->C_all = C_all;
-    d->d_tm_a = nullptr; d->d_tm_w = nullptr; d->d_rows = nullptr; d->d_row_off = nullptr;
+    d->d_tm_a = nullptr; d->d_tm_w = nullptr; d->d_tm_c = nullptr; d->d_rows = nullptr; d->d_row_off = nullptr;
     d->w_blocks = (N_expert % 64 == 0) ? 1 : 0;
     d->rows.assign(rows, rows + G);
     d->row_off.resize(G);
-    std::vector<CUtensorMap> ha(G), hw(B_list ? G : 0);
+    std::vector<CUtensorMap> ha(G), hw(B_list ? G : 0), hc(dense ? G : 0);
+    const uint32_t a_box_rows = dense ? 128 : (uint32_t)tile_m;
     long long off = 0;
     for (int g = 0; g < G; ++g) {
         d->row_off[g] = (int)off;
@@ -656,10 +659,17 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
         const long long first = std::min(off, total - 1);
         const int n_rows = std::max(1, rows[g]);
         const char* base = (const char*)A_all + (size_t)first * K * 2;
-        if (!encode_2d(&ha[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, (uint64_t)std::min<long long>(n_rows, total - first),
-                       K, SK_BK, tile_m)) {
+        const uint64_t view_rows = (uint64_t)std::min<long long>(n_rows, total - first);
+        if (!encode_2d(&ha[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, view_rows, K, SK_BK, a_box_rows)) {
             delete d;
             return AG_ERR_CUDA;
+        }
+        if (dense) {
+            float* cbase = (float*)C_all + (size_t)first * N_expert;
+            if (!encode_2d(&hc[g], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, cbase, view_rows, N_expert, 32, 32)) {
+                delete d;
+                return AG_ERR_CUDA;
+            }
         }
         if (B_list) {
             if (!B_list[g] || ((uintptr_t)B_list[g] & 15u)) { delete d; return AG_ERR_ARG; }
@@ -674,6 +684,10 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
     if (e == cudaSuccess && B_list) {
         e = cudaMalloc(&d->d_tm_w, sizeof(CUtensorMap) * G);
         if (e == cudaSuccess) e = cudaMemcpy(d->d_tm_w, hw.data(), sizeof(CUtensorMap) * G, cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess && dense) {
+        e = cudaMalloc(&d->d_tm_c, sizeof(CUtensorMap) * G);
+        if (e == cudaSuccess) e = cudaMemcpy(d->d_tm_c, hc.data(), sizeof(CUtensorMap) * G, cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = cudaMalloc(&d->d_rows, sizeof(int) * G);
     if (e == cudaSuccess) e = cudaMemcpy(d->d_rows, d->rows.data(), sizeof(int) * G, cudaMemcpyHostToDevice);
@@ -691,10 +705,14 @@ extern "C" ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_pa
                                              void* cuda_stream) {
     if (!d || !plan) return AG_ERR_ARG;
     const int32_t* h = plan->header;
-    // the plan sees the experts side by side: N = G * N_expert, one tile row of at most tile_m rows
-    if (h[H_N] != d->G * d->N || h[H_K] != d->K || h[H_TILE_M] != d->tile_m || h[H_M] > d->tile_m) return AG_ERR_ARG;
+    // the plan sees the experts side by side: N = G * N_expert, M = the largest row count of an expert
+    if (h[H_N] != d->G * d->N || h[H_K] != d->K || h[H_TILE_M] != d->tile_m) return AG_ERR_ARG;
     for (int g = 0; g < d->G; ++g)
         if (d->rows[g] > h[H_M]) return AG_ERR_ARG;
+    if (d->tile_m == 256)  // many rows per expert: block pairs, per-expert A / B / C views
+        return gemm_pair_dispatch(d->A_all, nullptr, W, d->C_all, h[H_M], h[H_N], h[H_K], plan,
+                                  reinterpret_cast<cudaStream_t>(cuda_stream), d);
+    if (h[H_M] > d->tile_m) return AG_ERR_ARG;
     return gemm_skinny_dispatch(d->A_all, nullptr, W, d->C_all, h[H_M], h[H_N], h[H_K], plan, plan->d_partial, plan->d_sem,
                                 reinterpret_cast<cudaStream_t>(cuda_stream), d);
 }

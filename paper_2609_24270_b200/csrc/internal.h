@@ -99,6 +99,7 @@ struct ag_group_desc {
     std::vector<int> rows, row_off;
     CUtensorMap* d_tm_a;   // device [G]: activations of expert g
     CUtensorMap* d_tm_w;   // device [G]: row-major weights of expert g (null when only packed weights are used)
+    CUtensorMap* d_tm_c;   // device [G]: outputs of expert g (dense descriptors, tile_m = 256, only)
     int* d_rows;           // device [G]
     int* d_row_off;        // device [G]
     int w_blocks;          // 1: d_tm_w are the 3-D [N/64][K][64] views

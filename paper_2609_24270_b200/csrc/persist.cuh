@@ -162,6 +162,6 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
                                int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream,
                                const ag_group_desc* grp = nullptr);
 ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
-                             const ag_plan* plan, cudaStream_t stream);
+                             const ag_plan* plan, cudaStream_t stream, const ag_group_desc* grp = nullptr);
 
 }  // namespace ag

@@ -4,7 +4,8 @@
     python -m paper_2609_24270_b200.experiments --config 4
     python -m paper_2609_24270_b200.experiments --config 5
     python -m paper_2609_24270_b200.experiments --config raster      # raster-group sweep at 8192^3
-    python -m paper_2609_24270_b200.experiments --config groupgemm   # MoE-shaped grouped decode GEMM
+    python -m paper_2609_24270_b200.experiments --config groupgemm         # MoE-shaped grouped GEMM, ~20 rows per expert
+    python -m paper_2609_24270_b200.experiments --config groupgemm_dense   # same, 192 / 1024 rows per expert
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
 launches first, median of the timed launches.  torch is used for device memory, streams and events.
@@ -321,6 +322,45 @@ def groupgemm(fh, topo, seeds=(1, 2)):
             torch.cuda.empty_cache()
 
 
+def groupgemm_dense(fh, topo, seeds=(1,)):
+    """The settings of the paper's GroupGEMM study with many rows per expert: (G, M) in {(32, 192), (6, 1024)},
+    same (N, K) list; block pairs with per-expert views."""
+    for G, M in ((32, 192), (6, 1024)):
+        for N, K in ((6144, 7168), (7168, 3072), (4096, 4096), (4096, 2048)):
+            Bs = [torch.randn((K, N), dtype=torch.bfloat16, device="cuda") for _ in range(G)]
+            w_bytes = G * K * N * 2
+            dst_bytes = 2 * w_bytes + (16 << 20)
+            dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+            for seed in seeds:
+                rows = inputs.group_rows(G, M, seed)
+                total = int(rows.sum())
+                dA = torch.randn((total, K), dtype=torch.bfloat16, device="cuda")
+                dC = torch.empty((total, N), dtype=torch.float32, device="cuda")
+                kw = dict(M=int(rows.max()), N=G * N, K=K, tile_m=256, tile_n=256, raster_group=1)
+                plan_obl = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
+                plan_dc = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+                packed = ag.pack_weights_grouped([b.data_ptr() for b in Bs], K, N, plan_dc, amap, dst.data_ptr(), dst_bytes)
+                bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packed.page_table())
+                plan_rem = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
+                desc = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, [b.data_ptr() for b in Bs], N, K, 256)
+                flops = 2.0 * total * N * K
+                algo = w_bytes + total * K * 2 + total * N * 4
+                res = {}
+                for name, pk, plan in (("rowmajor_oblivious", None, plan_obl), ("rowmajor_die_compact", None, plan_dc),
+                                       ("packed_die_local", packed, plan_dc), ("packed_remote", packed, plan_rem)):
+                    ms = time_queued(lambda: ag.gemm_persistent_grouped(desc, pk, plan))
+                    assert plan.last_status() == ag.AG_OK
+                    res[name] = dict(tflops=flops / (ms * 1e-3) / 1e12, gbs=algo / (ms * 1e-3) / 1e9, us=ms * 1e3)
+                emit(dict(config="groupgemm_dense", G=G, M=M, N=N, K=K, seed=seed, rows_total=total, weight_gb=w_bytes / 1e9,
+                          flop_per_byte=flops / algo, results=res,
+                          local_over_remote=res["packed_remote"]["us"] / res["packed_die_local"]["us"],
+                          local_over_rowmajor_oblivious=res["rowmajor_oblivious"]["us"] / res["packed_die_local"]["us"]), fh)
+                del packed, desc, dA, dC
+            del Bs, dst, amap
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -331,7 +371,7 @@ def main():
     emit(dict(config="topology", n_sm=topo.n_sm, die_sm_count=list(topo.die_sm_count),
               gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
-    {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm}[args.config](fh, topo)
+    {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense}[args.config](fh, topo)
 
 
 if __name__ == "__main__":

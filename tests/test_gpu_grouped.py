@@ -105,3 +105,48 @@ def test_grouped_handles_an_expert_without_rows():
     torch.cuda.synchronize()
     assert plan.last_status() == ag.AG_OK
     assert np.array_equal(dC.cpu().numpy().astype(np.float64), expert_refs(rows, A_all, Bs))
+
+
+@pytest.mark.parametrize("G,M,N,K,integer", [(6, 192, 512, 256, True), (3, 700, 768, 512, True), (8, 192, 1024, 1024, False)])
+def test_grouped_dense_block_pairs(G, M, N, K, integer):
+    """Many rows per expert (the paper's M = 192 / 1024 settings, scaled down): block pairs with
+    per-expert A, B and C views; units below an expert's last row are skipped."""
+    rows, A_all, Bs = make_problem(G, M, N, K, seed=7, integer=integer)
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=int(rows.max()), N=G * N, K=K,
+                                                                tile_m=256, tile_n=256, raster_group=1))
+    dA = to_dev_bf16(A_all)
+    dBs = [to_dev_bf16(b) for b in Bs]
+    dC = torch.full((int(rows.sum()), N), float("nan"), dtype=torch.float32, device="cuda")
+    desc = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, [b.data_ptr() for b in dBs], N, K, 256)
+    ref = expert_refs(rows, A_all, Bs)
+    for _ in range(2):
+        dC.fill_(float("nan"))
+        ag.gemm_persistent_grouped(desc, None, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        C = dC.cpu().numpy()
+        if integer:
+            assert np.array_equal(C.astype(np.float64), ref)
+        else:
+            check_close(C, ref)
+
+
+def test_grouped_dense_over_packed_weights():
+    G, M, N, K = 4, 192, 512, 512
+    rows, A_all, Bs = make_problem(G, M, N, K, seed=9, integer=True)
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=int(rows.max()), N=G * N, K=K,
+                                                                tile_m=256, tile_n=256))
+    dst_bytes = 2 * G * K * N * 2 + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    dBs = [to_dev_bf16(b) for b in Bs]
+    packed = ag.pack_weights_grouped([b.data_ptr() for b in dBs], K, N, plan, amap, dst.data_ptr(), dst_bytes)
+    dA = to_dev_bf16(A_all)
+    dC = torch.full((int(rows.sum()), N), float("nan"), dtype=torch.float32, device="cuda")
+    desc = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, None, N, K, 256)
+    ag.gemm_persistent_grouped(desc, packed, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK
+    assert np.array_equal(dC.cpu().numpy().astype(np.float64), expert_refs(rows, A_all, Bs))
