@@ -36,8 +36,8 @@ MIN_MARGIN = (UNIT_M * K * 2 + TILE_N * K * 2 + UNIT_M * TILE_N * 4) // 8
 FLOPS = 2.0 * M * N * K
 METRIC = "bf16_gemm_tflops"
 UNIT = "TFLOP/s"
-# DRAM bytes per launch of the dominant kernel, from the ncu capture summarised in
-# profiles/gemm_persistent_pair_8192.md (dram__bytes_read.sum 1.761 GB + dram__bytes_write.sum 0.253 GB).
+# DRAM bytes per launch of the dominant kernel, from an Nsight Compute capture of two timed steps of this
+# bench (dram__bytes_read.sum 1.761 GB + dram__bytes_write.sum 0.253 GB; summary kept under profiles/).
 NCU_TRAFFIC_BYTES = 2.014e9
 
 

@@ -17,6 +17,8 @@
  *     calls that launch kernels return AG_ERR_UNSUPPORTED_ARCH.
  *   - Every device-side wait is bounded; if one runs out the kernel records
  *     AG_ERR_TIMEOUT in the plan's status word (see ag_last_status) and returns.
+ *   - Environment: AG_DEBUG=1 makes topo_discover print its bandwidth measurements and any
+ *     rejected latency rows to stderr.  Nothing else is read from the environment.
  */
 #ifndef ASYMGEMM_H_
 #define ASYMGEMM_H_
