@@ -16,13 +16,15 @@ def _free_port():
         return s.getsockname()[1]
 
 
-def _worker(rank, world, port, out):
+def _worker(rank, world, port):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
         ms = [0.8, 1.25][rank]                                  # rank 1 is the slow replica
         value, job_ms = replicas.job_throughput(ms, 1.0e12)
-        out[rank] = (value, job_ms, replicas.slowest_rank_ms(ms))
+        # every rank sees the slowest rank's time and the work of both ranks (a failed assert fails the spawn)
+        assert abs(job_ms - 1.25) < 1e-12 and abs(replicas.slowest_rank_ms(ms) - 1.25) < 1e-12
+        assert abs(value - 2 * 1.0e12 / 1.25e-3) < 1e-3
         dist.barrier()
     finally:
         dist.destroy_process_group()
@@ -30,13 +32,7 @@ def _worker(rank, world, port, out):
 
 def test_two_replicas_take_the_slowest_ranks_time():
     world, port = 2, _free_port()
-    with mp.Manager() as mgr:
-        out = mgr.dict()
-        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
-        for rank in range(world):
-            value, job_ms, mx = out[rank]
-            assert job_ms == pytest.approx(1.25) and mx == pytest.approx(1.25)
-            assert value == pytest.approx(2 * 1.0e12 / 1.25e-3)
+    mp.spawn(_worker, args=(world, port), nprocs=world, join=True)
 
 
 def test_single_process_is_identity():
