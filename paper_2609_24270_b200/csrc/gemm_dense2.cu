@@ -12,8 +12,8 @@
 // Pinning (Section 7.1.2 of the paper) works as in the one-CTA kernel: every block reads %smid and
 // takes the plan slot of its SM.  The two blocks of a pair tell each other their slots and walk the
 // two task lists in alternation, so every list of the plan is still run exactly once.  No copy is
-// multicast: each block loads its own halves; only the "stage is free" and "accumulator is ready"
-// signals of tcgen05.commit go to both blocks.
+// shared between blocks: each block loads its own halves; only the "stage is free" and "accumulator is
+// ready" signals of tcgen05.commit go to both blocks.
 #include <string.h>
 
 #include <mutex>
@@ -91,13 +91,12 @@ __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// arrive on the barrier at this offset in both blocks of the pair once the MMAs issued so far are done
+// arrive on the barrier at this offset in both blocks of the pair once the MMAs issued so far are done:
+// one commit for the leader's own barrier, one for the peer's (addressed through the cluster window)
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-    const uint16_t mask = 3;
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"(mask)
-        : "memory");
+    const uint32_t own = map_to_cta(bar, 0), peer = map_to_cta(bar, 1);
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(own) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer) : "memory");
 }
 
 // Grouped (MoE-shaped) operation: the plan's N is G experts side by side (expert g = unit columns
