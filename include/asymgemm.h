@@ -250,6 +250,17 @@ ag_status ag_plan_margins(const ag_plan* plan, int64_t* out, size_t cap);
  * (host arrays of n_units entries, either may be NULL); ag_plan_reset_record zeroes the counts. */
 ag_status ag_plan_tile_record(const ag_plan* plan, int32_t* owner_sm, int32_t* run_count, size_t cap);
 ag_status ag_plan_reset_record(ag_plan* plan);
+/*
+ * ag_plan_set_grid - launch fewer thread blocks than the device has SMs (blocks = 0 restores one
+ * block per SM), e.g. when part of the GPU is known to be busy.  Planned SMs that get no block are
+ * then "unmanned": with static lists, a block that has finished its own list takes over the list
+ * of an unmanned SM (Section 7.1.2 plans per SM; the take-over keeps the plan complete), with
+ * dynamic queues the per-die queues are simply drained by fewer blocks.  Not available for plans of
+ * block pairs (tile_m = 256).  ag_plan_adopted reports how many lists have been taken over since the
+ * plan was built.  Errors: AG_ERR_ARG.
+ */
+ag_status ag_plan_set_grid(ag_plan* plan, int blocks);
+ag_status ag_plan_adopted(const ag_plan* plan, uint32_t* n_lists);
 /* Device status word of the most recent launch (call after synchronising its stream). */
 ag_status ag_last_status(const ag_plan* plan);
 void ag_plan_destroy(ag_plan* plan);

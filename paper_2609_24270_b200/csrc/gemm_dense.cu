@@ -330,7 +330,7 @@ static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream
         attr_err = cudaFuncSetAttribute(k_gemm_persistent<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    k_gemm_persistent<BN><<<plan->lay.n_sm, kThreads, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);
+    k_gemm_persistent<BN><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, kThreads, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);
     count_launch();
     AG_CUDA(cudaGetLastError());
     return AG_OK;

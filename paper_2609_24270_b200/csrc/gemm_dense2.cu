@@ -436,7 +436,7 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     // A pair of blocks is co-scheduled on the two SMs of one TPC, so the plan must hold whole TPCs: a block
     // whose partner sits on an unplanned SM could not run.  (Seeded random SM subsets do not qualify - the
     // compute-side counterpart of the paper's point that equal SM counts are not equal capabilities.)
-    if (n_sm != plan->lay.n_sm || (n_sm & 1)) return AG_ERR_ARG;
+    if (n_sm != plan->lay.n_sm || (n_sm & 1) || plan->grid_blocks != 0) return AG_ERR_ARG;  // pairs: always one block per SM
     {
         const int32_t* slot_of = plan->h_image.data() + plan->lay.smid_to_slot();
         for (int s = 0; s < n_sm; ++s)

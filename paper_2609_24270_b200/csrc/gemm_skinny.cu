@@ -452,7 +452,7 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
                                         SK_SMEM_BYTES);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    k_gemm_skinny<NM, PACKED><<<plan->lay.n_sm, kThreads, SK_SMEM_BYTES, stream>>>(tm_a, tm_w, gp, x);
+    k_gemm_skinny<NM, PACKED><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, kThreads, SK_SMEM_BYTES, stream>>>(tm_a, tm_w, gp, x);
     count_launch();
     AG_CUDA(cudaGetLastError());
     return AG_OK;

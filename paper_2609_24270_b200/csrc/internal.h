@@ -70,6 +70,7 @@ struct ag_plan {
     int* d_sem;                // device [4 * tiles_n] arrival counters for the split-K reduction
     std::vector<int32_t> h_image;
     mutable uint32_t epoch;
+    int grid_blocks;           // 0: one block per SM; else launch this many blocks (one-block and decode-shaped kernels)
     int kslabs_total;
     int kslabs_per_split;
     // tensor-map cache for the last (A, B, C) triple

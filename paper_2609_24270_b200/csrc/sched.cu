@@ -409,6 +409,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     pl->d_margins = nullptr;
     pl->d_partial = nullptr; pl->d_sem = nullptr;
     pl->epoch = 0;
+    pl->grid_blocks = 0;
     pl->kslabs_total = n_slab;
     pl->kslabs_per_split = per;
     pl->tm_a_ptr = pl->tm_b_ptr = nullptr; pl->tm_c_ptr = nullptr;
@@ -520,18 +521,34 @@ extern "C" ag_status ag_plan_reset_record(ag_plan* plan) {
     return AG_OK;
 }
 
+extern "C" ag_status ag_plan_set_grid(ag_plan* plan, int blocks) {
+    if (!plan || blocks < 0 || blocks > plan->lay.n_sm) return AG_ERR_ARG;
+    plan->grid_blocks = blocks;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_plan_adopted(const ag_plan* plan, uint32_t* n_lists) {
+    if (!plan || !n_lists) return AG_ERR_ARG;
+    PlanCtrl c;
+    AG_CUDA(cudaMemcpy(&c, plan->d_ctrl, sizeof(int) * 8, cudaMemcpyDeviceToHost));
+    *n_lists = c.adopted;
+    return AG_OK;
+}
+
 extern "C" ag_status ag_last_status(const ag_plan* plan) {
     if (!plan) return AG_ERR_ARG;
     PlanCtrl c;
     AG_CUDA(cudaMemcpy(&c, plan->d_ctrl, sizeof(int) * 8, cudaMemcpyDeviceToHost));
     if (c.status != 0) return (ag_status)c.status;
-    // every slot of the plan must have been taken by a block of the last launch
     if (plan->epoch != 0) {
         std::vector<unsigned int> claimed(plan->lay.b);
         AG_CUDA(cudaMemcpy(claimed.data(), (const char*)plan->d_ctrl + offsetof(PlanCtrl, claimed),
                            sizeof(unsigned int) * plan->lay.b, cudaMemcpyDeviceToHost));
-        for (int i = 0; i < plan->lay.b; ++i)
-            if (claimed[i] != plan->epoch) return AG_ERR_UNMANNED_SM;
+        int n_claimed = 0;
+        for (int i = 0; i < plan->lay.b; ++i) n_claimed += claimed[i] == plan->epoch;
+        // static lists: every list must have been run by somebody (its own SM's block or one that took it over);
+        // dynamic queues: any block drains them, so one is enough
+        if (plan->header[H_STATIC] ? n_claimed != plan->lay.b : n_claimed == 0) return AG_ERR_UNMANNED_SM;
     }
     return AG_OK;
 }

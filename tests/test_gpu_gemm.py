@@ -247,3 +247,27 @@ def test_die_packed_b_pages_and_affinity_plan_match_oracle():
     torch.cuda.synchronize()
     assert plan_a.last_status() == ag.AG_OK
     check_close(dC.cpu().numpy(), og.gemm_blocked(A, B))
+
+
+@pytest.mark.parametrize("blocks", [100, 37, 1])
+@pytest.mark.parametrize("static", [1, 0])
+def test_fewer_blocks_than_planned_sms_still_complete_the_plan(blocks, static):
+    """Planned SMs that get no thread block: their lists are taken over (static) or the queues are
+    drained by the blocks that exist (dynamic).  Every unit still runs exactly once."""
+    M, N, K = 1024, 1536, 256
+    A, B = inputs.small_int_bf16(M, K, 41), inputs.small_int_bf16(K, N, 42)
+    plan = plan_for(M, N, K, kind=ag.AG_DIE_COMPACT, static_assign=static, tile_n=128)
+    plan.set_grid(blocks)
+    plan.reset_record()
+    C = run_gemm(A, B, plan)
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+    owner, count = plan.tile_record()
+    assert (count == 1).all() and len(set(owner)) <= blocks
+    if static:
+        p = plan.parsed()
+        with_work = sum(1 for s in range(p["b"]) if p["sm_q_off"][s + 1] > p["sm_q_off"][s])
+        assert plan.adopted() >= min(with_work, p["b"]) - blocks   # at least the lists nobody was there for
+    pair = plan_for(M, N, K, tile_m=256, tile_n=256)
+    with pytest.raises(ag.AgError):
+        pair.set_grid(64)
+        run_gemm(A, B, pair)
