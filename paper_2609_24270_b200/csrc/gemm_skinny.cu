@@ -13,6 +13,7 @@
 // last split adds them in ascending split order (deterministic) and writes C.
 #include <string.h>
 
+#include <algorithm>
 #include <mutex>
 #include <new>
 
@@ -284,6 +285,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         int st_tn = -1;              // unit whose partial sums are stored but not yet announced
         int at_tn = -1;              // unit whose arrival atomic is in flight
         int oldA = 0, oldB = 0;      // results of the arrival atomics (lane 0), used one unit later
+        bool zero_done = false;      // in-memory split-K: the zeroing of C is known to be complete
 
         auto reduce_columns = [&](int tn) {
             __threadfence();
@@ -372,8 +374,14 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const OutView ov = out_view(p, x, tn);
             const int nl = ov.col0 + q * 32 + lane;       // column inside the tile's problem
             if (p.k_splits > 1 && x.partial == nullptr) {
-                // in-memory reduction: C was zeroed before the launch, every unit adds its partial sums
-                // with reductions that L2 carries out; nothing comes back, so nothing is waited for
+                // in-memory reduction: C is zeroed by the kernel launched just before this one, every unit adds
+                // its partial sums with reductions that L2 carries out; nothing comes back, so nothing is
+                // waited for.  This kernel may have started while the zeroing was still running (programmatic
+                // dependent launch): make sure it is complete before the first add.
+                if (!zero_done) {
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    zero_done = true;
+                }
                 if (nl < ov.n_cols) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m)
@@ -420,6 +428,14 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     }
 }
 
+// Zeroes C for the in-memory split-K mode.  Its dependents (the GEMM launched right after it) are released at
+// once, so the GEMM's start-up overlaps the zeroing; the GEMM waits for this kernel only before its first add.
+__global__ void k_zero_f32(float4* __restrict__ p, size_t n_vec) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x)
+        p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // One block per logical page: gathers W[n][k] = B[k][n] for 128 n x 16 k and writes the 4 KB page in
 // core-matrix order into its chunk.
 __global__ void k_pack_weights(const uint16_t* __restrict__ B, int K, int N, int pages_per_tile,
@@ -444,7 +460,7 @@ __global__ void k_pack_weights(const uint16_t* __restrict__ B, int K, int N, int
 
 template <int NM, bool PACKED>
 static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, const CUtensorMap& tm_w,
-                               const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream) {
+                               const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream, bool after_zeroing) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
@@ -452,9 +468,19 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
                                         SK_SMEM_BYTES);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    k_gemm_skinny<NM, PACKED><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, kThreads, SK_SMEM_BYTES, stream>>>(tm_a, tm_w, gp, x);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = SK_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_zeroing ? 1 : 0;   // may start while the zeroing kernel before it is still running
+    AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_skinny<NM, PACKED>, tm_a, tm_w, gp, x));
     count_launch();
-    AG_CUDA(cudaGetLastError());
     return AG_OK;
 }
 
@@ -506,16 +532,21 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
             return AG_ERR_CUDA;
         }
     }
-    if (h[H_KSPLITS] > 1 && !x.partial) {  // in-memory reduction mode: the adds need a zeroed C
+    const bool zeroing = h[H_KSPLITS] > 1 && !x.partial;
+    if (zeroing) {  // in-memory reduction mode: the adds need a zeroed C (N % 8 == 0 and 16-byte alignment: whole float4s)
         const size_t c_elems = grp ? (size_t)grp->total_rows * (size_t)grp->N : (size_t)M * (size_t)N;
-        AG_CUDA(cudaMemsetAsync(Cout, 0, sizeof(float) * c_elems, stream));
+        const size_t n_vec = c_elems / 4;
+        const unsigned blocks = (unsigned)std::min<size_t>(148, (n_vec + 255) / 256);
+        k_zero_f32<<<blocks, 256, 0, stream>>>((float4*)Cout, n_vec);
+        count_launch();
+        AG_CUDA(cudaGetLastError());
     }
     PersistParams gp = make_persist_params(plan, M, N, K);
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
-    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream)
-                           : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream);
-    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, gp, x, stream)
-             : launch_skinny<32, false>(plan, tm_a, tm_w, gp, x, stream);
+    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream, zeroing)
+                           : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream, zeroing);
+    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, gp, x, stream, zeroing)
+             : launch_skinny<32, false>(plan, tm_a, tm_w, gp, x, stream, zeroing);
 }
 
 }  // namespace ag
