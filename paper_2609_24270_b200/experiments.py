@@ -35,18 +35,23 @@ def dev_bf16(bits):
     return torch.from_numpy(bits.view(np.int16).copy()).cuda()
 
 
-def time_launches(fn, warmup=3, iters=10, stream=None):
+def time_launches(fn, warmup=3, iters=10, stream=None, batches=3):
+    """Per-launch times in ms: `batches` batches of `iters` back-to-back launches, each batch bracketed by one
+    event pair (an event pair around every single launch would add several microseconds to each)."""
     stream = stream or torch.cuda.current_stream()
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
-    evs[0].record(stream)
-    for i in range(iters):
-        fn()
-        evs[i + 1].record(stream)
-    torch.cuda.synchronize()
-    return [evs[i].elapsed_time(evs[i + 1]) for i in range(iters)]
+    out = []
+    for _ in range(batches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(iters):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1) / iters)
+    return out
 
 
 def sm_set_summary(topo, plan):
@@ -143,9 +148,9 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
                 pk = packs[state["i"] % n_buffers][0]
                 state["i"] += 1
                 ag.gemm_persistent_packed(dA.data_ptr(), pk, dC.data_ptr(), M, N, K, plan)
-            ms = time_launches(run, warmup=4, iters=24)
+            ms = time_queued(run, warmup=4, iters=24)
             assert plan.last_status() == ag.AG_OK
-            out[name] = algo_bytes / (float(np.median(ms)) * 1e-3) / 1e9
+            out[name] = algo_bytes / (ms * 1e-3) / 1e9
         for name, plan in (("rowmajor_oblivious", plan_obl), ("rowmajor_die_compact", plan_local)):
             state = {"i": 0}
 
@@ -153,8 +158,8 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
                 wb = Bs[state["i"] % n_buffers]
                 state["i"] += 1
                 ag.gemm_persistent(dA.data_ptr(), wb.data_ptr(), dC.data_ptr(), M, N, K, plan)
-            ms = time_launches(run2, warmup=4, iters=24)
-            out[name] = algo_bytes / (float(np.median(ms)) * 1e-3) / 1e9
+            ms = time_queued(run2, warmup=4, iters=24)
+            out[name] = algo_bytes / (ms * 1e-3) / 1e9
         emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
                   sm_budget=b, gbs=out, local_over_remote=out["die_local"] / out["remote"],
                   pages_on_owner_die=on_die, local_set=sm_set_summary(topo, plan_local),
@@ -262,21 +267,25 @@ def raster(fh, topo):
 
 
 # ---------------------------------------------------------------------------------------------
-def time_queued(fn, warmup=3, iters=12):
-    """Median GPU time per call with the calls queued behind a device-side blocker, so that host-side
-    launch cost is not on the clock (the kernels here take tens of microseconds)."""
+def time_queued(fn, warmup=3, iters=16, batches=3):
+    """Median GPU time per call in ms.  The calls of a batch are queued behind a device-side blocker, so that
+    host-side launch cost is not on the clock (the kernels here take tens of microseconds), and the batch is
+    bracketed by one event pair."""
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
     s = torch.cuda.current_stream()
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
-    torch.cuda._sleep(int(2e7))
-    evs[0].record(s)
-    for i in range(iters):
-        fn()
-        evs[i + 1].record(s)
-    torch.cuda.synchronize()
-    return float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(iters)]))
+    out = []
+    for _ in range(batches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(2e7))
+        e0.record(s)
+        for _ in range(iters):
+            fn()
+        e1.record(s)
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1) / iters)
+    return float(np.median(out))
 
 
 def groupgemm(fh, topo, seeds=(1, 2)):
