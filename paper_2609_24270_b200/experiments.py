@@ -73,13 +73,13 @@ def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
     for b in budgets:
         res = {}
         plans = {f"random_{s}": ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, seed=s, M=M, N=N, K=K,
-                                                                            raster_group=8))
+                                                                            raster_group=4))
                  for s in range(1, n_subsets + 1)}
-        plans["lowest_ids"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, M=M, N=N, K=K, raster_group=8))
+        plans["lowest_ids"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, M=M, N=N, K=K, raster_group=4))
         plans["die_compact"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
-                                                                            raster_group=8))
+                                                                            raster_group=4))
         plans["gpc_spread"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K,
-                                                                           raster_group=8, sm_select=1))
+                                                                           raster_group=4, sm_select=1))
         # whole-TPC sets can also run block pairs (256 x 256 units); random subsets cannot
         for name, sel in (("die_compact_pairs", 0), ("gpc_spread_pairs", 1)):
             if b % 2 == 0:
