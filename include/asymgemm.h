@@ -218,6 +218,10 @@ typedef struct {
                                  memory (no workspace, no waiting; the order of the fp32 adds is not fixed) */
     int32_t sm_select;       /* die_compact / affinity: 0 = primary die first (die-compact set); 1 = whole TPCs dealt
                                 round-robin over the GPCs of both dies (fewest SMs per GPC, Section 5.1.2) */
+    int32_t pair_lists;      /* 1: static lists are dealt to TPCs instead of SMs (entry i of a die's queue -> TPC i mod P,
+                                lower SM in even rounds, upper SM in odd ones), so that the two lists of a TPC together
+                                hold a fair share; for plans of block pairs.  Needs whole TPCs, else AG_ERR_ARG */
+    int32_t reserved1;
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;

@@ -53,7 +53,13 @@ Steps.
                     raster index ascending) are given to their preferred die while its
                     quota lasts, else to the other die; each die's queue is then put back
                     in raster order.
-  6. static lists: entry i of die d's queue goes to the SM of rank (i mod n_d) in d.
+  6. static lists: entry i of die d's queue goes to the SM of rank (i mod n_d) in d.  With
+     pair_lists = 1 (plans whose 256-row units are run by the two SMs of a TPC together) the
+     entries are dealt to TPCs instead: with P = n_d / 2 TPCs in the die, entry i goes to TPC
+     (i mod P) - ranks 2(i mod P) and 2(i mod P)+1 - to its lower SM when (i div P) is even,
+     else to its upper SM, so that the two lists of a TPC together hold a fair share of the
+     die's work.  (Oblivious plans deal the whole raster the same way over all chosen SMs.)
+     Every chosen TPC must be whole and n_d even.
   7. export: flat int32 words (see ``export``).
 """
 from __future__ import annotations
@@ -80,7 +86,7 @@ def mix64(x: int) -> int:
 def default_policy(**kw) -> dict:
     p = dict(kind=OBLIVIOUS, seed=0, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1,
              k_unit=64, raster_group=1, preferred_die=-1, invert_affinity=0,
-             static_assign=1, min_margin=0, sm_select=0, avoid=(), a=None, b=None, c=None)
+             static_assign=1, min_margin=0, sm_select=0, pair_lists=0, avoid=(), a=None, b=None, c=None)
     p.update(kw)
     return p
 
@@ -262,10 +268,22 @@ def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
     q = quotas(n_u, n_d, b)
 
     sm_q = [[] for _ in S]
+    pair_lists = pol.get("pair_lists", 0)
+    if pair_lists:
+        tpc = topo["tpc"]
+        groups = [list(range(b))] if pol["kind"] == OBLIVIOUS else slots_of_die
+        for slots in groups:
+            if len(slots) % 2 or any(tpc[S[slots[2 * j]]] != tpc[S[slots[2 * j + 1]]] for j in range(len(slots) // 2)):
+                raise ValueError("pair_lists needs whole TPCs")
+
+    def pair_slot(slots, i):
+        P = len(slots) // 2
+        return slots[2 * (i % P) + ((i // P) & 1)]
+
     if pol["kind"] == OBLIVIOUS:
         die_q = [[], []]
         for i, u in enumerate(R):
-            slot = i % b
+            slot = pair_slot(list(range(b)), i) if pair_lists else i % b
             sm_q[slot].append(u)
             die_q[sm_die[slot]].append(u)
     else:
@@ -300,7 +318,8 @@ def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
             die_q = [[u for _, u in sorted(g)] for g in got]
         for d in (0, 1):
             for i, u in enumerate(die_q[d]):
-                sm_q[slots_of_die[d][i % n_d[d]]].append(u)
+                slot = pair_slot(slots_of_die[d], i) if pair_lists else slots_of_die[d][i % n_d[d]]
+                sm_q[slot].append(u)
 
     smid_to_slot = [-1] * topo["n_sm"]
     for i, s in enumerate(S):

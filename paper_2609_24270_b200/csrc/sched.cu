@@ -24,7 +24,7 @@ struct OperandDev {
 };
 struct PolicyDev {
     int kind, M, N, K, tile_m, tile_n, k_splits, k_unit, raster_group, preferred_die, invert, static_assign;
-    int sm_select, pad0;
+    int sm_select, pair_lists;
     unsigned long long seed;
     long long min_margin;
     unsigned long long avoid[4];
@@ -261,7 +261,11 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
     const int group_len = pol.raster_group * tiles_n * pol.k_splits;
 
     if (pol.kind == AG_OBLIVIOUS) {
-        for (int i = tid; i < n_units; i += nt) die_of[i] = image[lay.sm_die() + (i % b)];
+        for (int i = tid; i < n_units; i += nt) {
+            const int P = b / 2;
+            const int slot = (pol.pair_lists && P > 0) ? 2 * (i % P) + ((i / P) & 1) : i % b;
+            die_of[i] = image[lay.sm_die() + slot];
+        }
     } else if (pol.kind == AG_DIE_COMPACT) {
         for (int i = tid; i < n_units; i += nt) die_of[i] = band_die(i, n_units, q0, group_len);
     } else {
@@ -310,7 +314,16 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
         for (int s = 0; s < b; ++s) {
             image[lay.sm_q_off() + s] = off;
             int len;
-            if (pol.kind == AG_OBLIVIOUS) {
+            if (pol.pair_lists) {
+                // entries are dealt to TPCs: entry i -> TPC (i mod P), its lower SM when (i div P) is even
+                const int d = image[lay.sm_die() + s];
+                const int r = pol.kind == AG_OBLIVIOUS ? s : image[lay.rank_in_die() + s];
+                const int total = pol.kind == AG_OBLIVIOUS ? n_units : cnt[d];
+                const int P = (pol.kind == AG_OBLIVIOUS ? b : n_d[d]) / 2;
+                const int j = r >> 1, par = r & 1;
+                const int T = (P > 0 && j < P && total > j) ? (total - j + P - 1) / P : 0;  // rounds in which TPC j gets a unit
+                len = par ? T / 2 : (T + 1) / 2;
+            } else if (pol.kind == AG_OBLIVIOUS) {
                 len = n_units > s ? (n_units - s + b - 1) / b : 0;
             } else {
                 const int d = image[lay.sm_die() + s], r = image[lay.rank_in_die() + s];
@@ -322,17 +335,30 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
     }
     __syncthreads();
     if (pol.kind == AG_OBLIVIOUS) {
+        const int P = b / 2;
         for (int i = tid; i < n_units; i += nt) {
             const int u = raster_unit(i, tiles_m, tiles_n, pol.k_splits, pol.raster_group);
-            image[lay.sm_q() + image[lay.sm_q_off() + (i % b)] + i / b] = u;
+            if (pol.pair_lists && P > 0) {
+                const int t = i / P;
+                image[lay.sm_q() + image[lay.sm_q_off() + 2 * (i % P) + (t & 1)] + t / 2] = u;
+            } else {
+                image[lay.sm_q() + image[lay.sm_q_off() + (i % b)] + i / b] = u;
+            }
         }
     } else {
         const int len0 = image[lay.die_q_off() + 1];
         for (int e = tid; e < n_units; e += nt) {
             const int d = e < len0 ? 0 : 1;
             const int idx = d == 0 ? e : e - len0;
-            const int slot = slots_of_die[d][idx % n_d[d]];
-            image[lay.sm_q() + image[lay.sm_q_off() + slot] + idx / n_d[d]] = image[lay.die_q() + e];
+            const int P = n_d[d] / 2;
+            if (pol.pair_lists && P > 0) {
+                const int t = idx / P;
+                const int slot = slots_of_die[d][2 * (idx % P) + (t & 1)];
+                image[lay.sm_q() + image[lay.sm_q_off() + slot] + t / 2] = image[lay.die_q() + e];
+            } else {
+                const int slot = slots_of_die[d][idx % n_d[d]];
+                image[lay.sm_q() + image[lay.sm_q_off() + slot] + idx / n_d[d]] = image[lay.die_q() + e];
+            }
         }
     }
 }
@@ -451,6 +477,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pd.preferred_die = p.preferred_die; pd.invert = p.invert_affinity; pd.static_assign = p.static_assign;
         pd.seed = p.seed;
         pd.sm_select = p.sm_select;
+        pd.pair_lists = p.pair_lists ? 1 : 0;
         pd.min_margin = p.min_margin;
         for (int i = 0; i < 4; ++i) pd.avoid[i] = p.avoid_sm_mask[i];
         pd.a = to_dev(p.a, nullptr); pd.b = to_dev(p.b, d_table); pd.c = to_dev(p.c, nullptr);
@@ -475,6 +502,19 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pl->h_image.resize(pl->lay.total());
         TRY(cudaMemcpy(pl->h_image.data(), pl->d_image, image_bytes, cudaMemcpyDeviceToHost));
         memcpy(pl->header, pl->h_image.data(), sizeof pl->header);
+        if (p.pair_lists) {
+            // units were dealt to TPCs: every chosen TPC must be whole (both SMs chosen, adjacent in the die's ranks)
+            const int32_t* img = pl->h_image.data();
+            const int groups = p.kind == AG_OBLIVIOUS ? 1 : 2;
+            for (int d = 0; d < groups && st == AG_OK; ++d) {
+                std::vector<int> sms;
+                for (int i = 0; i < sm_budget; ++i)
+                    if (groups == 1 || img[pl->lay.sm_die() + i] == d) sms.push_back(img[pl->lay.sm_list() + i]);
+                if (sms.size() % 2) st = AG_ERR_ARG;
+                for (size_t j = 0; j + 1 < sms.size() && st == AG_OK; j += 2)
+                    if (map->tpc[sms[j]] != map->tpc[sms[j + 1]]) st = AG_ERR_ARG;
+            }
+        }
     }
 done:
 #undef TRY

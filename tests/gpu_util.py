@@ -46,6 +46,8 @@ def check_close(C_gpu, C_ref):
 def oracle_policy(**kw):
     """Oracle-side policy dict from the same keyword arguments as ag.make_policy."""
     d = dict(kw)
+    if d.get("pair_lists") is None:                      # same default as ag.make_policy
+        d["pair_lists"] = 1 if d.get("tile_m", 128) == 256 else 0
     for name in ("a", "b", "c"):
         o = d.get(name)
         if o is not None:

@@ -32,7 +32,7 @@ def test_struct_sizes_match_header_layout():
     # int32 x4 + 3 arrays of 256 int32 + 256 bytes + 2 + 32 + 32 int32 + 9 x 4 bytes
     assert ag.C.sizeof(ag.TopoMap) == 16 + 3 * 1024 + 256 + 4 * (2 + 32 + 32) + 36
     assert ag.C.sizeof(ag.OperandDesc) == 48
-    assert ag.C.sizeof(ag.Policy) == 12 * 4 + 8 + 8 + 8 + 32 + 3 * 48
+    assert ag.C.sizeof(ag.Policy) == 12 * 4 + 8 + 8 + 8 + 8 + 32 + 3 * 48
 
 
 def test_null_arguments_are_rejected_without_a_device():

@@ -160,11 +160,13 @@ def test_two_cta_units_uniform_and_rejections():
     C = run_gemm(A, B, plan_for(M, N, K, tile_m=256, tile_n=256))
     check_close(C, og.gemm_blocked(A, B))
     topo = device_topo()
-    odd = ag.sched_build(topo, None, 37, ag.make_policy(M=M, N=N, K=K, tile_m=256, tile_n=256, seed=3))
+    with pytest.raises(ag.AgError):                         # a random subset is not made of whole TPCs: no pair lists ...
+        ag.sched_build(topo, None, 37, ag.make_policy(M=M, N=N, K=K, tile_m=256, tile_n=256, seed=3))
+    odd = ag.sched_build(topo, None, 37, ag.make_policy(M=M, N=N, K=K, tile_m=256, tile_n=256, seed=3, pair_lists=0))
     dA, dB = to_dev_bf16(A), to_dev_bf16(B)
     dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
     st = ag.lib().gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, odd.handle, None)
-    assert st == ag.AG_ERR_ARG                              # a random subset is not made of whole TPCs
+    assert st == ag.AG_ERR_ARG                              # ... and no block pairs either
 
 
 @pytest.mark.parametrize("b,sm_select", [(16, 0), (64, 0), (74, 0), (64, 1), (100, 1)])
@@ -198,7 +200,7 @@ def packed_dense_setup(M, N, K, raster_group=2, integer=True, seed=51):
         A, B = inputs.small_int_bf16(M, K, seed), inputs.small_int_bf16(K, N, seed + 1)
     else:
         A, B = inputs.gemm_inputs(M, N, K, seed=seed)
-    kw = dict(M=M, N=N, K=K, tile_m=256, tile_n=256, raster_group=raster_group)
+    kw = dict(M=M, N=N, K=K, tile_m=256, tile_n=256, raster_group=raster_group, pair_lists=1)
     plan_d = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
     dst_bytes = 2 * K * ((N + 255) // 256 * 256) * 2 + (8 << 20)
     dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")

@@ -166,3 +166,16 @@ def test_hash_fit_recovers_a_synthetic_xor_mask():
     noisy[::97] ^= 1
     got, violations = ag.affinity_from_table(0, noisy).fit_hash()
     assert got == 0x1EF and 0 < violations <= 8192 // 97 + 1
+
+
+@pytest.mark.parametrize("kind", [ag.AG_OBLIVIOUS, ag.AG_DIE_COMPACT])
+@pytest.mark.parametrize("b", [16, 48, 74, 148])
+def test_pair_lists_match_oracle(kind, b):
+    topo = inputs.synthetic_topo(die0_sms=70, seed=13)
+    for sel in (0, 1):
+        got, want, _ = both(topo, None, b, kind=kind, M=4096, N=4096, K=4096, tile_m=256, tile_n=256, raster_group=4,
+                            sm_select=sel, pair_lists=1)
+        assert got.tobytes() == want.tobytes()
+    with pytest.raises(ag.AgError):
+        ag.sched_build(ag.TopoMap.from_dict(topo), None, 37, ag.make_policy(kind=ag.AG_OBLIVIOUS, seed=3, M=4096, N=4096,
+                                                                            K=4096, tile_m=256, tile_n=256, pair_lists=1))

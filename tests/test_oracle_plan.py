@@ -184,6 +184,36 @@ def test_die_compact_is_compact_and_gpc_balanced():
     assert all(topo["die"][s] == 0 for s in op.select_sms(topo, 32, pol0))
 
 
+def test_pair_lists_deal_units_to_tpcs():
+    toy8 = dict(n_sm=8, n_tpc=4, n_gpc=2, n_die=2, tpc=[0, 0, 1, 1, 2, 2, 3, 3], gpc=[0, 0, 0, 0, 1, 1, 1, 1],
+                die=[0, 0, 0, 0, 1, 1, 1, 1], is_random=[0] * 8, gpc_die=[0, 1])
+    # hand-derived: 10 units (2 x 5 tiles of 256 x 256), oblivious, 4 TPCs: entries 0..3 -> lower SMs 0,2,4,6;
+    # 4..7 -> upper SMs 1,3,5,7; 8,9 -> lower SMs 0,2
+    pol = op.default_policy(kind=op.OBLIVIOUS, M=512, N=1280, K=64, tile_m=256, tile_n=256, pair_lists=1)
+    plan = op.build_plan(toy8, None, 8, pol)
+    assert plan["sm_q"] == [[0, 8], [4], [1, 9], [5], [2], [6], [3], [7]]
+    check_invariants(toy8, plan, pol, 8)
+    # die_compact, 37 TPCs in one die of a synthetic chip: 256 units -> TPC totals 7 or 6 (ranks dealing: 8 and 6)
+    topo = inputs.synthetic_topo(die0_sms=74, seed=5)
+    for pair_lists, worst in ((1, 7), (0, 8)):
+        pol = op.default_policy(kind=op.DIE_COMPACT, M=4096, N=4096, K=4096, tile_m=256, tile_n=256, raster_group=4,
+                                pair_lists=pair_lists)
+        plan = op.build_plan(topo, None, 74, pol)
+        check_invariants(topo, plan, pol, 74)
+        per_tpc = [len(plan["sm_q"][2 * j]) + len(plan["sm_q"][2 * j + 1]) for j in range(37)]
+        assert max(per_tpc) == worst and sum(per_tpc) == 256
+        if pair_lists:   # the two lists of a TPC, taken in alternation (lower first), are the die queue entries j, j+P, ...
+            q = plan["die_q"][plan["sm_die"][0]]
+            j = 5
+            lo, hi = plan["sm_q"][2 * j], plan["sm_q"][2 * j + 1]
+            merged = [x for pair in zip(lo, hi + [None]) for x in pair if x is not None]
+            assert merged == q[j::37]
+    # half a TPC in the set: refused
+    with pytest.raises(ValueError):
+        op.build_plan(topo, None, 37, op.default_policy(kind=op.OBLIVIOUS, seed=3, M=4096, N=4096, K=4096, tile_m=256,
+                                                        tile_n=256, pair_lists=1))
+
+
 def test_gpc_spread_selection_minimises_sms_per_gpc():
     topo = inputs.synthetic_topo(die0_sms=70, seed=3)
     for b in (16, 48, 64, 100):
