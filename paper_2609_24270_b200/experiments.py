@@ -193,11 +193,12 @@ def config5(fh, topo):
     pre_kw = dict(M=Mp, N=N, K=K, tile_m=256, tile_n=256, raster_group=4)   # both partitions hold whole TPCs: block pairs
     dec_kw = dict(M=Md, N=N, K=K, tile_m=32, tile_n=128, k_splits=8, splitk_in_memory=1)
     for split in ((74, 74), (110, 38)):
-        for mode in ("die_split", "oblivious"):
-            kind = ag.AG_DIE_COMPACT if mode == "die_split" else ag.AG_OBLIVIOUS
-            plan_p = ag.sched_build(topo, None, split[0], ag.make_policy(kind=kind, preferred_die=0, **pre_kw))
+        for mode in ("die_split", "gpc_spread", "oblivious"):
+            kind = ag.AG_OBLIVIOUS if mode == "oblivious" else ag.AG_DIE_COMPACT
+            sel = 1 if mode == "gpc_spread" else 0      # whole TPCs dealt over the GPCs of both dies
+            plan_p = ag.sched_build(topo, None, split[0], ag.make_policy(kind=kind, preferred_die=0, sm_select=sel, **pre_kw))
             taken = [int(s) for s in plan_p.parsed()["sm_list"]]
-            plan_d = ag.sched_build(topo, None, split[1], ag.make_policy(kind=kind, avoid=taken, **dec_kw))
+            plan_d = ag.sched_build(topo, None, split[1], ag.make_policy(kind=kind, avoid=taken, sm_select=sel, **dec_kw))
             n_pre, n_dec = 6, 6 * 8 * 4
 
             def pre():
