@@ -37,8 +37,8 @@ FLOPS = 2.0 * M * N * K
 METRIC = "bf16_gemm_tflops"
 UNIT = "TFLOP/s"
 # DRAM bytes per launch of the dominant kernel, from an Nsight Compute capture of two timed steps of this
-# bench (dram__bytes_read.sum 1.761 GB + dram__bytes_write.sum 0.253 GB; summary kept under profiles/).
-NCU_TRAFFIC_BYTES = 2.014e9
+# bench (dram__bytes_read.sum 1.050 GB + dram__bytes_write.sum 0.251 GB; summary kept under profiles/).
+NCU_TRAFFIC_BYTES = 1.301e9
 
 
 def load_peaks():
