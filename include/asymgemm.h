@@ -17,6 +17,9 @@
  *     calls that launch kernels return AG_ERR_UNSUPPORTED_ARCH.
  *   - Every device-side wait is bounded; if one runs out the kernel records
  *     AG_ERR_TIMEOUT in the plan's status word (see ag_last_status) and returns.
+ *   - A handle (plan, affinity map, packed weights, group descriptor) may be used by one host
+ *     thread at a time; launches of one plan must not overlap on the device (use one plan per
+ *     stream).  Different plans may run concurrently on disjoint SM sets (avoid_sm_mask).
  *   - Environment: AG_DEBUG=1 makes topo_discover print its bandwidth measurements and any
  *     rejected latency rows to stderr.  Nothing else is read from the environment.
  */
@@ -188,8 +191,9 @@ enum { AG_LAYOUT_ROWMAJOR = 0, AG_LAYOUT_PAGED = 1 };
 
 typedef struct {
     int32_t present;        /* 0: operand not counted by the affinity policy */
-    int32_t layout;         /* AG_LAYOUT_ROWMAJOR: rows of row_stride bytes; AG_LAYOUT_PAGED: B only,
-                               pages of [16 k x tile_n] elements, page of (tn, k16) = tn*ceil(K/16)+k16 */
+    int32_t layout;         /* AG_LAYOUT_ROWMAJOR: rows of row_stride bytes; AG_LAYOUT_PAGED: B only, 4 KB pages of
+                               [128 columns x 16 k] elements, page of (pc, k16) = pc*ceil(K/16)+k16 with pc the index
+                               of the 128-column block (a unit column of width tile_n holds tile_n/128 blocks) */
     int64_t offset;         /* byte offset of element (0,0) from the probed buffer's base */
     int64_t row_stride;     /* bytes between rows (row-major) */
     int32_t elem_bytes;
@@ -275,8 +279,11 @@ void ag_plan_destroy(ag_plan* plan);
  * (Section 7.1.2); TMA feeds shared memory, tcgen05 MMAs accumulate in tensor memory in fp32.
  *   A  device, M x K bf16 row-major, 16-byte aligned, K % 8 == 0
  *   B  device, K x N bf16 row-major, 16-byte aligned, N % 8 == 0
- *   C  device, M x N fp32 row-major, 16-byte aligned; overwritten (zeroed first when the plan
- *      has k_splits > 1, partial sums are then added with reductions in memory)
+ *   C  device, M x N fp32 row-major, 16-byte aligned; overwritten.  Dense plans with k_splits > 1:
+ *      zeroed first, partial sums are then added with reductions in memory.  Decode-shaped plans
+ *      (tile_m <= 32): see policy.splitk_in_memory
+ *   the plan's tile shape selects the kernel: 256 x 256 units = pairs of thread blocks, 128 x
+ *      {64,128,256} = one block per tile (any SM set), {16,32} x 128 = decode-shaped (M <= tile_m)
  *   plan  built for the same M, N, K, else AG_ERR_ARG
  *   cuda_stream  a cudaStream_t (NULL = default stream).  Asynchronous.
  * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA.  Device-side trouble
@@ -307,8 +314,8 @@ typedef struct ag_packed_weights ag_packed_weights;
  */
 ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
                           void* dst, size_t dst_bytes, ag_packed_weights** out);
-/* Page table (host, cap entries): chunk index in dst of logical page (tn, k16) = tn * (K/16) + k16;
- * feed it to ag_operand_desc.page_table to build an affinity plan over the packed weights. */
+/* Page table (host, cap entries): chunk index in dst of logical page (pc, k16) = pc * (K/16) + k16, pc = index
+ * of the 128-column block; feed it to ag_operand_desc.page_table to build an affinity plan over the packed weights. */
 ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* out, size_t cap, size_t* n_pages);
 void ag_packed_destroy(ag_packed_weights* w);
 
