@@ -259,6 +259,16 @@ ag_status ag_plan_margins(const ag_plan* plan, int64_t* out, size_t cap);
 ag_status ag_plan_tile_record(const ag_plan* plan, int32_t* owner_sm, int32_t* run_count, size_t cap);
 ag_status ag_plan_reset_record(ag_plan* plan);
 /*
+ * ag_plan_trace / ag_plan_unit_times - per-unit timeline of the last launch, for load-balance and tail
+ * analysis (the paper profiles its kernels with hardware counters; this is the software counterpart).
+ * With tracing on, every kernel stamps the global nanosecond timer when a unit is handed to the block's
+ * pipeline (start) and when its last output has been issued (end); unit u's pair is returned in
+ * start_ns[u], end_ns[u] (host, cap >= n_units; 0 = the unit did not run).  Cost: two 8-byte stores per unit.
+ * Errors: AG_ERR_ARG (tracing off, small cap), AG_ERR_CUDA, AG_ERR_NOMEM.
+ */
+ag_status ag_plan_trace(ag_plan* plan, int on);
+ag_status ag_plan_unit_times(const ag_plan* plan, uint64_t* start_ns, uint64_t* end_ns, size_t cap);
+/*
  * ag_plan_set_grid - launch fewer thread blocks than the device has SMs (blocks = 0 restores one
  * block per SM), e.g. when part of the GPU is known to be busy.  Planned SMs that get no block are
  * then "unmanned": with static lists, a block that has finished its own list takes over the list

@@ -26,7 +26,7 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_plan_set_grid", "ag_plan_adopted", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
+    "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
@@ -128,6 +128,8 @@ def lib() -> C.CDLL:
     L.ag_plan_margins.argtypes = [vp, vp, sz]
     L.ag_plan_tile_record.argtypes = [vp, vp, vp, sz]
     L.ag_plan_reset_record.argtypes = [vp]
+    L.ag_plan_trace.argtypes = [vp, C.c_int]
+    L.ag_plan_unit_times.argtypes = [vp, vp, vp, sz]
     L.ag_plan_set_grid.argtypes = [vp, C.c_int]
     L.ag_plan_adopted.argtypes = [vp, C.POINTER(C.c_uint32)]
     L.ag_last_status.argtypes = [vp]
@@ -361,6 +363,17 @@ class Plan:
 
     def reset_record(self):
         _check(lib().ag_plan_reset_record(self.handle), "ag_plan_reset_record")
+
+    def trace(self, on: bool = True):
+        _check(lib().ag_plan_trace(self.handle, 1 if on else 0), "ag_plan_trace")
+
+    def unit_times(self):
+        """(start_ns, end_ns) per unit of the last launch (tracing must be on)."""
+        n_u = int(self.export()[5])
+        t0 = np.zeros(n_u, dtype=np.uint64)
+        t1 = np.zeros(n_u, dtype=np.uint64)
+        _check(lib().ag_plan_unit_times(self.handle, t0.ctypes.data, t1.ctypes.data, n_u), "ag_plan_unit_times")
+        return t0, t1
 
     def set_grid(self, blocks: int):
         _check(lib().ag_plan_set_grid(self.handle, blocks), "ag_plan_set_grid")

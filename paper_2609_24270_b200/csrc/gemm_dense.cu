@@ -111,6 +111,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                     ok = 0;
                 } else {
                     ctl->ring[r] = u;
+                    if (p.unit_times && u >= 0) p.unit_times[2 * u] = globaltimer_ns();
                     mbar_arrive(smem_u32(&ctl->sched_full[r]));
                 }
             }
@@ -267,6 +268,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
                 if (q == 0) {
                     p.tile_owner[u] = my_sm;
+                    if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
                     atomicAdd(&p.tile_count[u], 1);
                 }
             }

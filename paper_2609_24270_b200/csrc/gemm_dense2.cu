@@ -227,6 +227,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                         ok = 0;
                     } else {
                         ctl->ring[r] = u;
+                    if (p.unit_times && u >= 0) p.unit_times[2 * u] = globaltimer_ns();
                         mbar_arrive(smem_u32(&ctl->sched_full[r]));
                     }
                 }
@@ -397,6 +398,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                     mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[acc]), 0));
                     if (q == 0 && leader) {
                         p.tile_owner[u] = my_sm;
+                    if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
                         atomicAdd(&p.tile_count[u], 1);
                     }
                 }

@@ -155,6 +155,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                     ok = 0;
                 } else {
                     ctl->ring[r] = u;
+                    if (p.unit_times && u >= 0) p.unit_times[2 * u] = globaltimer_ns();
                     mbar_arrive(smem_u32(&ctl->sched_full[r]));
                 }
             }
@@ -403,6 +404,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             }
             if (lane == 0 && q == 0) {
                 p.tile_owner[u] = my_sm;
+                    if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
                 atomicAdd(&p.tile_count[u], 1);
             }
             return true;

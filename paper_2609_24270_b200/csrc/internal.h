@@ -65,6 +65,7 @@ struct ag_plan {
     ag::PlanCtrl* d_ctrl;      // device
     int32_t* d_tile_owner;     // device [n_units]
     int32_t* d_tile_count;     // device [n_units]
+    unsigned long long* d_unit_times;  // device [n_units][2], allocated by ag_plan_trace(plan, 1)
     long long* d_margins;      // device [n_units] (affinity only, else null)
     float* d_partial;          // device [k_splits][M][N] split-K partial sums (skinny plans with k_splits > 1)
     int* d_sem;                // device [4 * tiles_n] arrival counters for the split-K reduction

@@ -18,6 +18,7 @@ struct PersistParams {
     PlanCtrl* ctrl;
     int32_t* tile_owner;
     int32_t* tile_count;
+    unsigned long long* unit_times;   // [n_units][2] start / end in ns of the global timer, or null (tracing off)
     int M, N, K;
     int b, n_units, n_sm;
     int tiles_n, k_splits, kslabs_total, kslabs_per_split;
@@ -135,6 +136,7 @@ inline PersistParams make_persist_params(const ag_plan* plan, int M, int N, int 
     gp.ctrl = plan->d_ctrl;
     gp.tile_owner = plan->d_tile_owner;
     gp.tile_count = plan->d_tile_count;
+    gp.unit_times = plan->d_unit_times;
     gp.M = M; gp.N = N; gp.K = K;
     gp.b = plan->lay.b; gp.n_units = plan->lay.n_units; gp.n_sm = plan->lay.n_sm;
     gp.tiles_n = plan->header[H_TILES_N]; gp.k_splits = plan->header[H_KSPLITS];

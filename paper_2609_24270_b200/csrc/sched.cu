@@ -433,6 +433,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     pl->policy.a.page_table = pl->policy.b.page_table = pl->policy.c.page_table = nullptr;
     pl->d_image = nullptr; pl->d_ctrl = nullptr; pl->d_tile_owner = nullptr; pl->d_tile_count = nullptr;
     pl->d_margins = nullptr;
+    pl->d_unit_times = nullptr;
     pl->d_partial = nullptr; pl->d_sem = nullptr;
     pl->epoch = 0;
     pl->grid_blocks = 0;
@@ -561,6 +562,30 @@ extern "C" ag_status ag_plan_reset_record(ag_plan* plan) {
     return AG_OK;
 }
 
+extern "C" ag_status ag_plan_trace(ag_plan* plan, int on) {
+    if (!plan) return AG_ERR_ARG;
+    if (on && !plan->d_unit_times) {
+        AG_CUDA(cudaMalloc(&plan->d_unit_times, sizeof(unsigned long long) * 2 * plan->lay.n_units));
+        AG_CUDA(cudaMemset(plan->d_unit_times, 0, sizeof(unsigned long long) * 2 * plan->lay.n_units));
+    } else if (!on && plan->d_unit_times) {
+        AG_CUDA(cudaDeviceSynchronize());
+        cudaFree(plan->d_unit_times);
+        plan->d_unit_times = nullptr;
+    }
+    return AG_OK;
+}
+
+extern "C" ag_status ag_plan_unit_times(const ag_plan* plan, uint64_t* start_ns, uint64_t* end_ns, size_t cap) {
+    if (!plan || !plan->d_unit_times || !start_ns || !end_ns || cap < (size_t)plan->lay.n_units) return AG_ERR_ARG;
+    std::vector<unsigned long long> t(2 * (size_t)plan->lay.n_units);
+    AG_CUDA(cudaMemcpy(t.data(), plan->d_unit_times, sizeof(unsigned long long) * t.size(), cudaMemcpyDeviceToHost));
+    for (int u = 0; u < plan->lay.n_units; ++u) {
+        start_ns[u] = t[2 * (size_t)u];
+        end_ns[u] = t[2 * (size_t)u + 1];
+    }
+    return AG_OK;
+}
+
 extern "C" ag_status ag_plan_set_grid(ag_plan* plan, int blocks) {
     if (!plan || blocks < 0 || blocks > plan->lay.n_sm) return AG_ERR_ARG;
     plan->grid_blocks = blocks;
@@ -600,6 +625,7 @@ extern "C" void ag_plan_destroy(ag_plan* plan) {
     cudaFree(plan->d_tile_owner);
     cudaFree(plan->d_tile_count);
     cudaFree(plan->d_margins);
+    cudaFree(plan->d_unit_times);
     cudaFree(plan->d_partial);
     cudaFree(plan->d_sem);
     delete plan;

@@ -273,3 +273,25 @@ def test_fewer_blocks_than_planned_sms_still_complete_the_plan(blocks, static):
     with pytest.raises(ag.AgError):
         pair.set_grid(64)
         run_gemm(A, B, pair)
+
+
+@pytest.mark.parametrize("tile_m", [128, 256])
+def test_unit_timeline(tile_m):
+    M, N, K = 2048, 2048, 1024
+    A, B = inputs.small_int_bf16(M, K, 61), inputs.small_int_bf16(K, N, 62)
+    plan = plan_for(M, N, K, tile_m=tile_m, tile_n=256, kind=ag.AG_DIE_COMPACT)
+    with pytest.raises(ag.AgError):
+        plan.unit_times()                                   # tracing is off by default
+    plan.trace(True)
+    C = run_gemm(A, B, plan)
+    assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
+    t0, t1 = plan.unit_times()
+    assert (t0 > 0).all() and (t1 > t0).all()
+    span_us = (int(t1.max()) - int(t0.min())) / 1e3
+    assert 1.0 < span_us < 5000.0
+    # the units of one SM's list run one after the other
+    p = plan.parsed()
+    lst = p["sm_q"][p["sm_q_off"][0]:p["sm_q_off"][1]]
+    if tile_m == 128 and len(lst) > 1:
+        assert all(t1[lst[i]] <= t1[lst[i + 1]] for i in range(len(lst) - 1))
+    plan.trace(False)
