@@ -66,10 +66,19 @@ __device__ inline bool avoided(const PolicyDev& p, int s) { return (p.avoid[s >>
 // ---- steps 2, 3, 4 and the header: one thread -------------------------------------------------
 __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol, int b, int n_units,
                              int tiles_m, int tiles_n, int32_t* __restrict__ image, PlanLayout lay) {
+    // the chip's per-SM arrays go to shared memory first (one thread walking them in global memory costs milliseconds)
+    __shared__ short s_die[AG_MAX_SM], s_gpc[AG_MAX_SM], s_tpc[AG_MAX_SM];
+    for (int s = threadIdx.x; s < topo->n_sm; s += blockDim.x) {
+        s_die[s] = (short)topo->die[s];
+        s_gpc[s] = (short)topo->gpc[s];
+        s_tpc[s] = (short)topo->tpc[s];
+    }
+    __syncthreads();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     __shared__ int cand[AG_MAX_SM];
     __shared__ int S[AG_MAX_SM];
-    __shared__ int tpcs[AG_MAX_SM];
+    __shared__ short key_tpc[AG_MAX_GPC + 1][AG_MAX_SM / 2];
+    __shared__ int key_nt[AG_MAX_GPC + 1];
     const int n_sm = topo->n_sm;
     int nc = 0;
     for (int s = 0; s < n_sm; ++s)
@@ -88,42 +97,42 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
         for (int i = 0; i < b; ++i) S[ns++] = cand[i];
     } else {
         int cnt[2] = {0, 0};
-        for (int i = 0; i < nc; ++i) cnt[topo->die[cand[i]] & 1]++;
+        for (int i = 0; i < nc; ++i) cnt[s_die[cand[i]] & 1]++;
         int primary = (pol.preferred_die == 0 || pol.preferred_die == 1) ? pol.preferred_die
                                                                            : (cnt[0] >= cnt[1] ? 0 : 1);
         const int n_gpc = topo->n_gpc;
         const int n_pass = pol.sm_select == 1 ? 1 : 2;  // GPC spread: both dies in one round-robin
         for (int pass_d = 0; pass_d < n_pass && ns < b; ++pass_d) {
             const int d = pol.sm_select == 1 ? -1 : (pass_d == 0 ? primary : 1 - primary);
+            // distinct TPC ids of the candidates of every GPC key (unplaced SMs: key n_gpc), ascending, built once
+            for (int key = 0; key <= n_gpc; ++key) key_nt[key] = 0;
+            for (int i = 0; i < nc; ++i) {
+                const int s = cand[i];
+                if (d >= 0 && s_die[s] != d) continue;
+                const int key = s_gpc[s] >= 0 ? s_gpc[s] : n_gpc;
+                const int t = s_tpc[s];
+                short* lst = key_tpc[key];
+                int nt = key_nt[key], pos = 0;
+                bool dup = false;
+                for (; pos < nt; ++pos) {
+                    if (lst[pos] == t) { dup = true; break; }
+                    if (lst[pos] > t) break;
+                }
+                if (dup) continue;
+                for (int m = nt; m > pos; --m) lst[m] = lst[m - 1];
+                lst[pos] = (short)t;
+                key_nt[key] = nt + 1;
+            }
             for (int p = 0; ns < b; ++p) {
                 bool any = false;
                 for (int key = 0; key <= n_gpc && ns < b; ++key) {
-                    // distinct TPC ids of candidates in (die d, GPC key), ascending
-                    int nt = 0;
-                    for (int i = 0; i < nc; ++i) {
-                        const int s = cand[i];
-                        if (d >= 0 && topo->die[s] != d) continue;
-                        const int k = topo->gpc[s] >= 0 ? topo->gpc[s] : n_gpc;
-                        if (k != key) continue;
-                        const int t = topo->tpc[s];
-                        int pos = 0;
-                        bool dup = false;
-                        for (; pos < nt; ++pos) {
-                            if (tpcs[pos] == t) { dup = true; break; }
-                            if (tpcs[pos] > t) break;
-                        }
-                        if (dup) continue;
-                        for (int m = nt; m > pos; --m) tpcs[m] = tpcs[m - 1];
-                        tpcs[pos] = t;
-                        ++nt;
-                    }
-                    if (p >= nt) continue;
+                    if (p >= key_nt[key]) continue;
                     any = true;
-                    const int t = tpcs[p];
+                    const int t = key_tpc[key][p];
                     for (int i = 0; i < nc && ns < b; ++i) {
                         const int s = cand[i];
-                        if ((d < 0 || topo->die[s] == d) && topo->tpc[s] == t &&
-                            (topo->gpc[s] >= 0 ? topo->gpc[s] : n_gpc) == key)
+                        if ((d < 0 || s_die[s] == d) && s_tpc[s] == t &&
+                            (s_gpc[s] >= 0 ? s_gpc[s] : n_gpc) == key)
                             S[ns++] = s;
                     }
                 }
@@ -141,7 +150,7 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
     int n_d[2] = {0, 0};
     for (int s = 0; s < n_sm; ++s) image[lay.smid_to_slot() + s] = -1;
     for (int i = 0; i < ns; ++i) {
-        const int d = topo->die[S[i]] & 1;
+        const int d = s_die[S[i]] & 1;
         image[lay.sm_list() + i] = S[i];
         image[lay.sm_die() + i] = d;
         image[lay.rank_in_die() + i] = n_d[d]++;
