@@ -179,15 +179,18 @@ __global__ void k_warm_up(unsigned long long ns, float* out) {
 // ---- affinity probe over a buffer -----------------------------------------------------------------
 // Members (the SMs of one die) split the chunks round-robin; one warp per SM.  Per chunk: a few
 // 128-byte lines, each saved, invalidated in L2, loaded with a timed L1-bypassing load, restored.
+// With `list` (n_work chunk indices) only those chunks are probed and cycles[i] belongs to list[i]; without it
+// all n_work chunks of the buffer are probed and cycles[c] belongs to chunk c.
 __global__ void k_affinity_probe(PinCtrl* pc, const int* member_rank /*[n_sm], -1 = not a member*/,
-                                 unsigned int n_members, uint8_t* buf, size_t n_chunks, int lines_per_chunk,
-                                 int reps, uint32_t* cycles) {
+                                 unsigned int n_members, uint8_t* buf, size_t n_chunks, const uint32_t* list,
+                                 size_t n_work, int lines_per_chunk, int reps, uint32_t* cycles) {
     const int rank = member_rank[smid()];
     pin_rendezvous(pc, rank >= 0, n_members, 200000ull);
     if (rank < 0 || threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
     uint32_t sink = 0;
-    for (size_t c = (size_t)rank; c < n_chunks; c += n_members) {
+    for (size_t w = (size_t)rank; w < n_work; w += n_members) {
+        const size_t c = list ? (size_t)list[w] : w;
         uint8_t* chunk = buf + c * AG_CHUNK_BYTES;
         uint8_t* partner = buf + (c ^ 1) * AG_CHUNK_BYTES;  // other chunk of the aligned pair: same large page
         if ((c ^ 1) >= n_chunks) partner = chunk + 3968;
@@ -207,7 +210,7 @@ __global__ void k_affinity_probe(PinCtrl* pc, const int* member_rank /*[n_sm], -
                 __threadfence();
             }
         }
-        if (lane == 0) cycles[c] = best;
+        if (lane == 0) cycles[w] = best;
     }
     if (lane == 0 && sink == 0x12345678u) cycles[0] = sink;
 }
@@ -698,8 +701,11 @@ extern "C" ag_status topo_discover(ag_topo_map* map) {
 }
 
 // ---- affinity --------------------------------------------------------------------------------------------
+// Probes all chunks (list == nullptr) or the listed ones from the SMs of one die; cycles gets one entry per
+// probed chunk (in list order when a list is given).
 static ag_status probe_from_die(uint8_t* buf, size_t n_chunks, const ag_topo_map* map, int die,
-                                std::vector<uint32_t>& cycles, int ref_sm[2]) {
+                                std::vector<uint32_t>& cycles, int ref_sm[2],
+                                const std::vector<uint32_t>* list = nullptr, int lines = 2, int reps = 3) {
     ag_status st = set_pin_smem();
     if (st != AG_OK) return st;
     const int n_sm = map->n_sm;
@@ -714,24 +720,34 @@ static ag_status probe_from_die(uint8_t* buf, size_t n_chunks, const ag_topo_map
     PinCtrl* pc = nullptr;
     int* d_rank = nullptr;
     uint32_t* d_cycles = nullptr;
+    uint32_t* d_list = nullptr;
+    const size_t n_work = list ? list->size() : n_chunks;
+    if (n_work < n_members) n_members = (unsigned int)std::max<size_t>(1, n_work);  // fewer chunks than SMs: fewer workers
+    for (int s = 0; s < n_sm; ++s)
+        if (rank[s] >= (int)n_members) rank[s] = -1;
     cudaError_t e = cudaSuccess;
     do {
         if ((e = cudaMalloc(&pc, sizeof(PinCtrl))) != cudaSuccess) break;
         if ((e = cudaMalloc(&d_rank, sizeof(int) * AG_MAX_SM)) != cudaSuccess) break;
-        if ((e = cudaMalloc(&d_cycles, sizeof(uint32_t) * n_chunks)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_cycles, sizeof(uint32_t) * n_work)) != cudaSuccess) break;
+        if (list) {
+            if ((e = cudaMalloc(&d_list, sizeof(uint32_t) * n_work)) != cudaSuccess) break;
+            if ((e = cudaMemcpy(d_list, list->data(), sizeof(uint32_t) * n_work, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        }
         if ((e = cudaMemset(pc, 0, sizeof(PinCtrl))) != cudaSuccess) break;
-        if ((e = cudaMemset(d_cycles, 0, sizeof(uint32_t) * n_chunks)) != cudaSuccess) break;
+        if ((e = cudaMemset(d_cycles, 0, sizeof(uint32_t) * n_work)) != cudaSuccess) break;
         if ((e = cudaMemcpy(d_rank, rank.data(), sizeof(int) * AG_MAX_SM, cudaMemcpyHostToDevice)) != cudaSuccess) break;
-        k_affinity_probe<<<n_sm, 32, kPinSmem>>>(pc, d_rank, n_members, buf, n_chunks, 2, 3, d_cycles);
+        k_affinity_probe<<<n_sm, 32, kPinSmem>>>(pc, d_rank, n_members, buf, n_chunks, d_list, n_work, lines, reps, d_cycles);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) break;
         if ((e = cudaDeviceSynchronize()) != cudaSuccess) break;
-        cycles.resize(n_chunks);
-        e = cudaMemcpy(cycles.data(), d_cycles, sizeof(uint32_t) * n_chunks, cudaMemcpyDeviceToHost);
+        cycles.resize(n_work);
+        e = cudaMemcpy(cycles.data(), d_cycles, sizeof(uint32_t) * n_work, cudaMemcpyDeviceToHost);
     } while (0);
     cudaFree(pc);
     cudaFree(d_rank);
     cudaFree(d_cycles);
+    cudaFree(d_list);
     if (e != cudaSuccess) return cuda_fail(e);
     for (uint32_t c : cycles)
         if (c == 0) return AG_ERR_UNMANNED_SM;  // a member SM got no block: its chunks were not probed
@@ -800,6 +816,26 @@ extern "C" ag_status ag_affinity_probe_with_map(void* buf, size_t bytes, const a
     if (st != AG_OK) return st;
     st = probe_from_die((uint8_t*)buf, n_chunks, map, 1, cycles1, ref_sm);
     if (st != AG_OK) return st;
+    // chunks whose two latencies are less than 25 % apart are probed once more, with more lines and repeats;
+    // the smaller of the old and the new value is kept for each die
+    {
+        std::vector<uint32_t> again;
+        for (size_t i = 0; i < n_chunks; ++i) {
+            const double lo = std::min(cycles[i], cycles1[i]), hi = std::max(cycles[i], cycles1[i]);
+            if (hi < 1.25 * lo) again.push_back((uint32_t)i);
+        }
+        if (!again.empty() && again.size() * 20 < n_chunks) {
+            std::vector<uint32_t> r0, r1;
+            int dummy[2] = {0, 0};
+            st = probe_from_die((uint8_t*)buf, n_chunks, map, 0, r0, dummy, &again, 6, 4);
+            if (st == AG_OK) st = probe_from_die((uint8_t*)buf, n_chunks, map, 1, r1, dummy, &again, 6, 4);
+            if (st != AG_OK) return st;
+            for (size_t k = 0; k < again.size(); ++k) {
+                cycles[again[k]] = std::min(cycles[again[k]], r0[k]);
+                cycles1[again[k]] = std::min(cycles1[again[k]], r1[k]);
+            }
+        }
+    }
     std::vector<uint8_t> table;
     size_t ambiguous = 0;
     st = classify(cycles, cycles1, table, &ambiguous);
