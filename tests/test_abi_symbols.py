@@ -122,3 +122,32 @@ def test_topo_map_file_roundtrip(tmp_path):
         ag.topo_load(path)
     with pytest.raises(ag.AgError):
         ag.topo_load(str(tmp_path / "missing.bin"))
+
+
+def test_ctypes_structs_match_the_header_as_a_c_compiler_sees_it(tmp_path):
+    """The header is plain C: compile it with gcc and compare sizes and field offsets with the binding."""
+    import subprocess
+    fields = {
+        "ag_topo_map": ["n_sm", "tpc", "gpc", "die", "is_random", "die_sm_count", "gpc_sm_count", "gpc_die",
+                        "lat_near_cycles", "l2_near_cycles", "n_unplaced", "device", "sm_clock_khz", "flags"],
+        "ag_operand_desc": ["present", "layout", "offset", "row_stride", "elem_bytes", "page_table", "n_pages"],
+        "ag_policy": ["kind", "M", "tile_m", "k_splits", "k_unit", "raster_group", "preferred_die", "invert_affinity",
+                      "static_assign", "seed", "min_margin", "splitk_in_memory", "sm_select", "pair_lists",
+                      "avoid_sm_mask", "a", "b", "c"],
+    }
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "asymgemm.h"', 'int main(void) {']
+    for sname, fl in fields.items():
+        lines.append(f'  printf("{sname} %zu\\n", sizeof({sname}));')
+        for f in fl:
+            lines.append(f'  printf("{sname}.{f} %zu\\n", offsetof({sname}, {f}));')
+    lines += ['  return 0;', '}']
+    src = tmp_path / "abi.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "abi"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    seen = dict(l.split() for l in subprocess.check_output([str(exe)], text=True).splitlines())
+    py = {"ag_topo_map": ag.TopoMap, "ag_operand_desc": ag.OperandDesc, "ag_policy": ag.Policy}
+    for sname, fl in fields.items():
+        assert int(seen[sname]) == ag.C.sizeof(py[sname]), sname
+        for f in fl:
+            assert int(seen[f"{sname}.{f}"]) == getattr(py[sname], f).offset, (sname, f)
