@@ -183,6 +183,17 @@ ag_status ag_affinity_check_complement(const ag_affinity_map* amap, const ag_top
  * Needs a map of at least 4 MiB.  Errors: AG_ERR_ARG.
  */
 ag_status ag_affinity_fit_hash(const ag_affinity_map* amap, uint32_t* mask, size_t* violations);
+/*
+ * ag_probe_die_bandwidth - local against remote memory bandwidth (Section 6.2.1: the 4 KB pages of a
+ * region are classified by partition and a read kernel is restricted to the local or the remote ones).
+ * The SMs of reader_die stream all chunks of the mapped buffer that belong to chunk_die (at least 1 GiB in
+ * total, several passes if needed; use a buffer well above the L2 size to measure HBM rather than L2).
+ *   bytes_per_s  host, out: best of three runs.
+ * Reads only; the buffer must be the one the map was probed on.  Synchronises the device.
+ * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_UNMANNED_SM.
+ */
+ag_status ag_probe_die_bandwidth(const ag_affinity_map* amap, const ag_topo_map* map, int reader_die,
+                                 int chunk_die, double* bytes_per_s);
 void ag_affinity_destroy(ag_affinity_map* amap);
 
 /* ---- plan (Section 7.1.2) ------------------------------------------------------------ */

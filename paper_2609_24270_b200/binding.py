@@ -24,7 +24,7 @@ EXPORTED = [
     "topo_discover", "ag_topo_discover_phases", "ag_topo_from_observations", "ag_topo_place_by_gain",
     "ag_probe_l2_bandwidth", "ag_probe_latency_samples",
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
-    "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_affinity_destroy",
+    "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
     "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
@@ -121,6 +121,7 @@ def lib() -> C.CDLL:
     L.ag_affinity_cycles.argtypes = [vp, vp, sz]
     L.ag_affinity_check_complement.argtypes = [vp, C.POINTER(TopoMap), C.POINTER(sz)]
     L.ag_affinity_fit_hash.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(sz)]
+    L.ag_probe_die_bandwidth.argtypes = [vp, C.POINTER(TopoMap), C.c_int, C.c_int, C.POINTER(C.c_double)]
     L.ag_affinity_destroy.argtypes = [vp]
     L.ag_affinity_destroy.restype = None
     L.sched_build.argtypes = [C.POINTER(TopoMap), vp, C.c_int, C.POINTER(Policy), C.POINTER(vp)]
@@ -256,6 +257,13 @@ class AffinityMap:
         n = C.c_size_t()
         _check(lib().ag_affinity_check_complement(self.handle, C.byref(topo), C.byref(n)), "ag_affinity_check_complement")
         return int(n.value)
+
+    def die_bandwidth(self, topo: TopoMap, reader_die: int, chunk_die: int) -> float:
+        """Bytes/s at which the SMs of reader_die stream the chunks of chunk_die."""
+        out = C.c_double()
+        _check(lib().ag_probe_die_bandwidth(self.handle, C.byref(topo), reader_die, chunk_die, C.byref(out)),
+               "ag_probe_die_bandwidth")
+        return out.value
 
     def fit_hash(self):
         """(mask over the 9 in-page chunk-index bits, number of chunks the fitted parity hash gets wrong)."""

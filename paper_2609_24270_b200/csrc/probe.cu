@@ -176,6 +176,43 @@ __global__ void k_warm_up(unsigned long long ns, float* out) {
     if (x == 123.456f) out[0] = x;
 }
 
+// ---- bandwidth of one die's SMs over the chunks of one die (Section 6.2.1) ---------------------------------
+// Members (the SMs of the reading die) split the listed chunks round-robin; every warp of a member streams whole
+// chunks with eight independent 16-byte L1-bypassing loads per lane (8 warps x 4 KB in flight per SM).
+__global__ void __launch_bounds__(256)
+k_die_bandwidth(PinCtrl* pc, const int* member_rank, unsigned int n_members, const uint8_t* buf,
+                const uint32_t* chunk_list, size_t n_list, int passes, unsigned int* sink_out) {
+    const int sm = (int)smid();
+    const int rank = member_rank[sm];
+    pin_rendezvous(pc, rank >= 0, n_members, 200000ull);
+    if (rank < 0) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    const size_t stride = (size_t)n_members * n_warps;
+    unsigned int acc = 0;
+    unsigned long long t0 = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) t0 = globaltimer_ns();
+    for (int p = 0; p < passes; ++p) {
+        size_t i = (size_t)rank * n_warps + warp;
+        uint32_t next = i < n_list ? chunk_list[i] : 0;
+        for (; i < n_list; i += stride) {
+            const uint4* chunk = reinterpret_cast<const uint4*>(buf + (size_t)next * AG_CHUNK_BYTES);
+            if (i + stride < n_list) next = chunk_list[i + stride];   // index of the following chunk: off the critical path
+            uint4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = ld_cg_u128(chunk + j * 32 + lane);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc += v[j].x ^ v[j].w;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        pc->t_start[sm] = t0;
+        pc->t_end[sm] = globaltimer_ns();
+    }
+    if (acc == 0x9e3779b9u) sink_out[0] = acc;
+}
+
 // ---- affinity probe over a buffer -----------------------------------------------------------------
 // Members (the SMs of one die) split the chunks round-robin; one warp per SM.  Per chunk: a few
 // 128-byte lines, each saved, invalidated in L2, loaded with a timed L1-bypassing load, restored.
@@ -374,6 +411,7 @@ ag_status set_pin_smem() {
     AG_CUDA(cudaFuncSetAttribute(k_latency_from_sm, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
     AG_CUDA(cudaFuncSetAttribute(k_l2_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
     AG_CUDA(cudaFuncSetAttribute(k_affinity_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+    AG_CUDA(cudaFuncSetAttribute(k_die_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
     done = true;
     return AG_OK;
 }
@@ -907,6 +945,69 @@ extern "C" ag_status ag_affinity_fit_hash(const ag_affinity_map* amap, uint32_t*
         *violations = bad;
     }
     return AG_OK;
+}
+
+extern "C" ag_status ag_probe_die_bandwidth(const ag_affinity_map* amap, const ag_topo_map* map, int reader_die,
+                                            int chunk_die, double* bytes_per_s) {
+    if (!amap || !map || !bytes_per_s || (reader_die | 1) != 1 || (chunk_die | 1) != 1 || !amap->base) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    st = set_pin_smem();
+    if (st != AG_OK) return st;
+    std::vector<uint32_t> list;
+    for (size_t c = 0; c < amap->n_chunks; ++c)
+        if (amap->h_die_of_chunk[c] == chunk_die) list.push_back((uint32_t)c);
+    if (list.empty()) return AG_ERR_ARG;
+    const int n_sm = map->n_sm;
+    std::vector<int> rank(AG_MAX_SM, -1);
+    unsigned int n_members = 0;
+    for (int s = 0; s < n_sm; ++s)
+        if (map->die[s] == reader_die) rank[s] = (int)n_members++;
+    if (n_members == 0) return AG_ERR_ARG;
+    PinCtrl* pc = nullptr;
+    int* d_rank = nullptr;
+    uint32_t* d_list = nullptr;
+    unsigned int* d_sink = nullptr;
+    cudaError_t e = cudaSuccess;
+    double best = 0;
+    do {
+        if ((e = cudaMalloc(&pc, sizeof(PinCtrl))) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_rank, sizeof(int) * AG_MAX_SM)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_list, sizeof(uint32_t) * list.size())) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_sink, 64)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(d_rank, rank.data(), sizeof(int) * AG_MAX_SM, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(d_list, list.data(), sizeof(uint32_t) * list.size(), cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        // enough passes to stream at least 1 GiB, so that the buffer cannot be served from L2 alone unless it is small
+        const size_t bytes_per_pass = list.size() * (size_t)AG_CHUNK_BYTES;
+        const int passes = (int)std::max<size_t>(1, (1ull << 30) / bytes_per_pass);
+        std::vector<PinCtrl> h(1);
+        for (int t = 0; t < 3 && e == cudaSuccess; ++t) {
+            if ((e = cudaMemset(pc, 0, sizeof(PinCtrl))) != cudaSuccess) break;
+            k_die_bandwidth<<<n_sm, 256, kPinSmem>>>(pc, d_rank, n_members, (const uint8_t*)amap->base, d_list, list.size(),
+                                                    passes, d_sink);
+            count_launch();
+            if ((e = cudaGetLastError()) != cudaSuccess) break;
+            if ((e = cudaDeviceSynchronize()) != cudaSuccess) break;
+            if ((e = cudaMemcpy(h.data(), pc, sizeof(PinCtrl), cudaMemcpyDeviceToHost)) != cudaSuccess) break;
+            unsigned long long t0 = ~0ull, t1 = 0;
+            unsigned int got = 0;
+            for (int s2 = 0; s2 < n_sm; ++s2)
+                if (rank[s2] >= 0 && h[0].t_end[s2]) {
+                    ++got;
+                    t0 = std::min(t0, h[0].t_start[s2]);
+                    t1 = std::max(t1, h[0].t_end[s2]);
+                }
+            if (got == n_members && t1 > t0)
+                best = std::max(best, (double)bytes_per_pass * passes / ((double)(t1 - t0) * 1e-9));
+        }
+    } while (0);
+    cudaFree(pc);
+    cudaFree(d_rank);
+    cudaFree(d_list);
+    cudaFree(d_sink);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *bytes_per_s = best;
+    return best > 0 ? AG_OK : AG_ERR_UNMANNED_SM;
 }
 
 extern "C" ag_status ag_affinity_export(const ag_affinity_map* amap, uint8_t* die_of_chunk, size_t cap,
