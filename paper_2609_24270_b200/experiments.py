@@ -6,6 +6,8 @@
     python -m paper_2609_24270_b200.experiments --config raster      # raster-group sweep at 8192^3
     python -m paper_2609_24270_b200.experiments --config groupgemm         # MoE-shaped grouped GEMM, ~20 rows per expert
     python -m paper_2609_24270_b200.experiments --config groupgemm_dense   # same, 192 / 1024 rows per expert
+    python -m paper_2609_24270_b200.experiments --config gpc_bandwidth     # L2 bandwidth of k SMs: one GPC vs spread
+    python -m paper_2609_24270_b200.experiments --config latency           # latency histograms from one SM per die
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
 launches first, median of the timed launches.  torch is used for device memory, streams and events.
@@ -371,6 +373,37 @@ def groupgemm_dense(fh, topo, seeds=(1,)):
             torch.cuda.empty_cache()
 
 
+def gpc_bandwidth(fh, topo):
+    """Section 5.1.2 (per-GPC L2 bandwidth figure): aggregate L2 read bandwidth of k SMs taken from one GPC
+    against k SMs spread over all GPCs."""
+    by_gpc = {g: [s for s in range(topo.n_sm) if topo.gpc[s] == g] for g in range(topo.n_gpc)}
+    biggest = max(by_gpc, key=lambda g: len(by_gpc[g]))
+    spread, i = [], 0
+    while len(spread) < len(by_gpc[biggest]):
+        for g in range(topo.n_gpc):
+            if 2 * i + 1 < len(by_gpc[g]):
+                spread += by_gpc[g][2 * i:2 * i + 2]
+        i += 1
+    for k in range(2, len(by_gpc[biggest]) + 1, 2):
+        emit(dict(config="gpc_bandwidth", n_sms=k, gpc=biggest,
+                  same_gpc_gbs=ag.probe_l2_bandwidth(by_gpc[biggest][:k]) / 1e9,
+                  spread_gbs=ag.probe_l2_bandwidth(spread[:k]) / 1e9), fh)
+
+
+def latency_histograms(fh, topo):
+    """Section 6.1.1 (latency histogram figures): samples from one SM of each die over 1024 lines; the first
+    sample of a line after the L2 invalidation is an HBM access, a plain reload is an L2 hit."""
+    sms = [0, next(s for s in range(topo.n_sm) if topo.die[s] == 1)]
+    edges = list(range(150, 1301, 50))
+    for sm in sms:
+        hbm = ag.probe_latency_samples(sm, mode=0, n_lines=1024, reps=1)[:, 0]
+        l2 = ag.probe_latency_samples(sm, mode=0, n_lines=1024, reps=4)[:, 1:].min(axis=1)   # later samples: served by L2
+        for name, v in (("first_touch_after_invalidate", hbm), ("repeat_after_invalidate", l2)):
+            hist, _ = np.histogram(v, bins=edges)
+            emit(dict(config="latency", sm=int(sm), die=int(topo.die[sm]), kind=name, bin_edges_cycles=edges,
+                      counts=[int(x) for x in hist], median=float(np.median(v))), fh)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -381,7 +414,8 @@ def main():
     emit(dict(config="topology", n_sm=topo.n_sm, die_sm_count=list(topo.die_sm_count),
               gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
-    {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense}[args.config](fh, topo)
+    {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
+     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms}[args.config](fh, topo)
 
 
 if __name__ == "__main__":
