@@ -335,6 +335,19 @@ typedef struct ag_packed_weights ag_packed_weights;
  */
 ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
                           void* dst, size_t dst_bytes, ag_packed_weights** out);
+/*
+ * ag_pack_weights_ex - ag_pack_weights / ag_pack_weights_grouped with options (G = 1: B_list holds one matrix).
+ *   flags  bit 0: keep the one-page-per-copy layout even where groups of four pages are possible.
+ * Grouped pages: when the map follows an XOR hash (ag_affinity_fit_hash) that uses chunk-index bits 0 and 1
+ * and leaves some bit f in 2..8 out, the chunks {q, q+a, q+F, q+F+a} (F = 2^f; a = 3 for q = 0 mod 4, a = 1
+ * for q = 1 mod 4; bit f of q clear) always sit on one die.  For decode-shaped plans the four pages of a
+ * k-slab are then stored in one such group and fetched with a single strided copy; groups whose measured
+ * chunks disagree are skipped.  ag_packed_info reports f (-1: single pages).
+ */
+ag_status ag_pack_weights_ex(const void* const* B_list, int G, int K, int N_expert, const ag_plan* plan,
+                             const ag_affinity_map* amap, void* dst, size_t dst_bytes, uint32_t flags,
+                             ag_packed_weights** out);
+ag_status ag_packed_info(const ag_packed_weights* w, int32_t* group_free_bit);
 /* Page table (host, cap entries): chunk index in dst of logical page (pc, k16) = pc * (K/16) + k16, pc = index
  * of the 128-column block; feed it to ag_operand_desc.page_table to build an affinity plan over the packed weights. */
 ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* out, size_t cap, size_t* n_pages);

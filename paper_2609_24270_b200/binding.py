@@ -26,7 +26,7 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_packed_page_table",
+    "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
@@ -138,6 +138,8 @@ def lib() -> C.CDLL:
     L.ag_plan_destroy.restype = None
     L.gemm_persistent.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.ag_pack_weights.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, sz, C.POINTER(vp)]
+    L.ag_pack_weights_ex.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, vp, vp, sz, C.c_uint32, C.POINTER(vp)]
+    L.ag_packed_info.argtypes = [vp, C.POINTER(C.c_int32)]
     L.ag_packed_page_table.argtypes = [vp, vp, sz, C.POINTER(sz)]
     L.ag_packed_destroy.argtypes = [vp]
     L.ag_packed_destroy.restype = None
@@ -422,6 +424,12 @@ class PackedWeights:
     def __init__(self, handle):
         self.handle = handle
 
+    def group_free_bit(self) -> int:
+        """>= 2: pages are stored in groups of four same-die chunks (one copy per k-slab); -1: single pages."""
+        f = C.c_int32()
+        _check(lib().ag_packed_info(self.handle, C.byref(f)), "ag_packed_info")
+        return int(f.value)
+
     def page_table(self) -> np.ndarray:
         n = C.c_size_t()
         _check(lib().ag_packed_page_table(self.handle, None, 0, C.byref(n)), "ag_packed_page_table")
@@ -441,9 +449,12 @@ class PackedWeights:
             pass
 
 
-def pack_weights(b_ptr: int, K: int, N: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int) -> PackedWeights:
+def pack_weights(b_ptr: int, K: int, N: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int,
+                 single_pages: bool = False) -> PackedWeights:
     h = C.c_void_p()
-    _check(lib().ag_pack_weights(b_ptr, K, N, plan.handle, amap.handle, dst_ptr, dst_bytes, C.byref(h)), "ag_pack_weights")
+    bl = (C.c_void_p * 1)(b_ptr)
+    _check(lib().ag_pack_weights_ex(bl, 1, K, N, plan.handle, amap.handle, dst_ptr, dst_bytes, 1 if single_pages else 0,
+                                    C.byref(h)), "ag_pack_weights_ex")
     return PackedWeights(h)
 
 
@@ -484,11 +495,11 @@ class GroupDesc:
 
 
 def pack_weights_grouped(b_ptrs, K: int, n_expert: int, plan: Plan, amap: AffinityMap, dst_ptr: int,
-                         dst_bytes: int) -> PackedWeights:
+                         dst_bytes: int, single_pages: bool = False) -> PackedWeights:
     bl = (C.c_void_p * len(b_ptrs))(*b_ptrs)
     h = C.c_void_p()
-    _check(lib().ag_pack_weights_grouped(bl, len(b_ptrs), K, n_expert, plan.handle, amap.handle, dst_ptr, dst_bytes,
-                                         C.byref(h)), "ag_pack_weights_grouped")
+    _check(lib().ag_pack_weights_ex(bl, len(b_ptrs), K, n_expert, plan.handle, amap.handle, dst_ptr, dst_bytes,
+                                    1 if single_pages else 0, C.byref(h)), "ag_pack_weights_ex")
     return PackedWeights(h)
 
 

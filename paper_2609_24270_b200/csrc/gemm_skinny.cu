@@ -53,6 +53,8 @@ struct SkinnyCtl {
 struct SkinnyArgs {
     const uint8_t* packed;        // packed weights base (PACKED) or null
     const int32_t* page_table;    // device (PACKED)
+    const int32_t* quad_base;     // device (PACKED, grouped layout): first chunk of each k-slab's group, or null
+    int quad_f;                   // chunk distance 2^free_bit between the two halves of a group
     int pages_per_tile;
     float* C;
     float* partial;               // [k_splits][M][N] or null when k_splits == 1
@@ -94,7 +96,7 @@ __device__ __forceinline__ OutView out_view(const PersistParams& p, const Skinny
 template <int NM, bool PACKED>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
-              const PersistParams p, const SkinnyArgs x) {
+              const __grid_constant__ CUtensorMap tm_w2, const PersistParams p, const SkinnyArgs x) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -125,7 +127,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         mbar_init(smem_u32(&ctl->mma_drain), 1);
         mbar_fence_init();
         prefetch_tmap(&tm_a);
-        if (!PACKED) prefetch_tmap(&tm_w);
+        if (!PACKED || x.quad_base) prefetch_tmap(&tm_w);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -170,8 +172,12 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             for (int sb = s0; sb < s1 && ok; sb += 8) {
                 int my_page = 0;
                 if (PACKED) {
-                    const int pg = sb * 4 + lane;
-                    if (pg < s1 * 4) my_page = x.page_table[(size_t)tn * x.pages_per_tile + pg];
+                    if (x.quad_base) {   // one entry per k-slab: lanes 0..7 fetch the bases of the next eight slabs
+                        if (lane < 8 && sb + lane < s1) my_page = x.quad_base[(size_t)tn * (x.pages_per_tile / 4) + sb + lane];
+                    } else {
+                        const int pg = sb * 4 + lane;
+                        if (pg < s1 * 4) my_page = x.page_table[(size_t)tn * x.pages_per_tile + pg];
+                    }
                 }
                 const int se = min(s1, sb + 8);
                 for (int s = sb; s < se; ++s, ++kit) {
@@ -188,7 +194,13 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) break;
-                    if (PACKED) {
+                    if (PACKED && x.quad_base) {
+                        // grouped layout: the slab's four pages sit in chunks q, q+a, q+F, q+F+a of one die
+                        // (a = 3 or 1 by q mod 4): one strided box brings all 16 KB
+                        const int q0 = __shfl_sync(0xffffffffu, my_page, s - sb);   // bit 30: class of the group
+                        if (lane == 0)
+                            tma_load_5d_hint(sw, (q0 >> 30) ? &tm_w2 : &tm_w, bar, 0, 0, 0, 0, q0 & 0x3fffffff, stream_policy);
+                    } else if (PACKED) {
                         // four lanes issue the four page copies of the slab in one instruction (a single thread
                         // gets only one bulk copy out every ~150 cycles)
                         const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + (lane & 3));
@@ -461,7 +473,7 @@ __global__ void k_pack_weights(const uint16_t* __restrict__ B, int K, int N, int
 }
 
 template <int NM, bool PACKED>
-static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, const CUtensorMap& tm_w,
+static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_w2,
                                const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream, bool after_zeroing) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -481,7 +493,7 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = after_zeroing ? 1 : 0;   // may start while the zeroing kernel before it is still running
-    AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_skinny<NM, PACKED>, tm_a, tm_w, gp, x));
+    AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_skinny<NM, PACKED>, tm_a, tm_w, tm_w2, gp, x));
     count_launch();
     return AG_OK;
 }
@@ -502,8 +514,9 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     if (n_sm != plan->lay.n_sm) return AG_ERR_ARG;
     const int NM = h[H_TILE_M];
-    CUtensorMap tm_a, tm_w;
+    CUtensorMap tm_a, tm_w, tm_w2;
     memset(&tm_w, 0, sizeof tm_w);
+    memset(&tm_w2, 0, sizeof tm_w2);
     memset(&tm_a, 0, sizeof tm_a);
     if (!grp && !encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, SK_BK, NM)) return AG_ERR_CUDA;
     SkinnyArgs x;
@@ -524,6 +537,12 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
         x.packed = W->dst;
         x.page_table = W->d_page_table;
         x.pages_per_tile = W->pages_per_tile;
+        if (W->quad_free_bit >= 0) {
+            x.quad_base = W->d_quad_base;
+            x.quad_f = 1 << W->quad_free_bit;
+            tm_w = W->tm_quad[0];
+            tm_w2 = W->tm_quad[1];
+        }
     } else if (grp) {
         if (!grp->d_tm_w) return AG_ERR_ARG;  // the descriptor was made without row-major weights
     } else {
@@ -545,10 +564,10 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     }
     PersistParams gp = make_persist_params(plan, M, N, K);
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
-    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, gp, x, stream, zeroing)
-                           : launch_skinny<16, false>(plan, tm_a, tm_w, gp, x, stream, zeroing);
-    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, gp, x, stream, zeroing)
-             : launch_skinny<32, false>(plan, tm_a, tm_w, gp, x, stream, zeroing);
+    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing)
+                           : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing);
+    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing)
+             : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing);
 }
 
 }  // namespace ag
@@ -558,7 +577,8 @@ using namespace ag;
 // Packs G source matrices (K x n_src each, row-major) side by side: the plan's N is G * n_src.  G = 1 is the
 // plain case.
 static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int N, const ag_plan* plan,
-                                   const ag_affinity_map* amap, void* dst, size_t dst_bytes, ag_packed_weights** out) {
+                                   const ag_affinity_map* amap, void* dst, size_t dst_bytes, uint32_t flags,
+                                   ag_packed_weights** out) {
     if (!B_list || G < 1 || !plan || !amap || !dst || !out || K <= 0 || N <= 0 || (N % G)) return AG_ERR_ARG;
     for (int g = 0; g < G; ++g)
         if (!B_list[g]) return AG_ERR_ARG;
@@ -585,21 +605,95 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
     w->K = K; w->N = N; w->tiles_n = n_blocks; w->pages_per_tile = ppt; w->n_pages = n_pages;
     w->dst = (const uint8_t*)dst; w->dst_bytes = dst_bytes; w->d_page_table = nullptr;
     w->h_page_table.resize(n_pages);
-    size_t next[2] = {0, 0};
+    w->quad_free_bit = -1;
+    w->d_quad_base = nullptr;
     const int per = plan->kslabs_per_split;
-    for (int pc = 0; pc < n_blocks; ++pc) {
-        const int tn = pc / ppc;
-        for (int k16 = 0; k16 < ppt; ++k16) {
-            const int ks = (k16 * 16 / SK_BK) / per;
-            int votes[2] = {0, 0};
-            for (int tm = 0; tm < tiles_m; ++tm) votes[unit_die[((size_t)tm * tiles_n + tn) * ksp + ks]]++;
-            const int d = votes[0] >= votes[1] ? 0 : 1;
-            const size_t pair = next[d]++;
-            if (2 * pair + 1 >= amap->n_chunks) {
-                delete w;
-                return AG_ERR_ARG;  // destination too small for this die's view
+    auto owner_die = [&](int pc, int k16) {   // the die that runs most of the units reading this page (tie -> die 0)
+        const int tn = pc / ppc, ks = (k16 * 16 / SK_BK) / per;
+        int votes[2] = {0, 0};
+        for (int tm = 0; tm < tiles_m; ++tm) votes[unit_die[((size_t)tm * tiles_n + tn) * ksp + ks]]++;
+        return votes[0] >= votes[1] ? 0 : 1;
+    };
+    // Grouped layout (decode-shaped plans): if the map follows an XOR hash that uses chunk-index bits 0 and 1 and
+    // leaves some bit f >= 2 out, the chunks {q, q+a, q+F, q+F+a} (F = 2^f; a = 3 for q = 0 mod 4, a = 1 for
+    // q = 1 mod 4; bit f of q clear) always share a die.  The four pages of a k-slab then go to one such group and
+    // the kernel fetches them with one strided copy instead of four.
+    std::vector<int32_t> quad_base;
+    if (!(flags & 1u) && h[H_TILE_N] == 128 && tiles_m == 1) {
+        uint32_t mask = 0;
+        size_t violations = 0;
+        if (ag_affinity_fit_hash(amap, &mask, &violations) == AG_OK && (mask & 3u) == 3u &&
+            violations * 50 <= amap->n_chunks) {
+            int f = -1;
+            for (int b = 2; b < 9 && f < 0; ++b)
+                if (!((mask >> b) & 1u)) f = b;
+            if (f >= 0) {
+                const size_t F = (size_t)1 << f;
+                // the hash works on addresses: chunk-index bits are those of (buffer base / 4 KB + q)
+                const size_t first = ((uintptr_t)dst / AG_CHUNK_BYTES) % 512;
+                std::vector<int32_t> groups[2];
+                for (size_t q = 0; q + F + 3 < amap->n_chunks; ++q) {
+                    const size_t qa = first + q;
+                    if ((qa & F) || (qa & 3) > 1) continue;
+                    const size_t a = (qa & 3) == 0 ? 3 : 1;
+                    const uint8_t d0 = amap->h_die_of_chunk[q];
+                    if (amap->h_die_of_chunk[q + a] == d0 && amap->h_die_of_chunk[q + F] == d0 &&
+                        amap->h_die_of_chunk[q + F + a] == d0)
+                        groups[d0].push_back((int32_t)q);   // a group whose chunks disagree (noise) is left out
+                }
+                size_t need[2] = {0, 0};
+                for (int pc = 0; pc < n_blocks; ++pc)
+                    for (int k16 = 0; k16 < ppt; k16 += 4) need[owner_die(pc, k16)]++;
+                if (need[0] <= groups[0].size() && need[1] <= groups[1].size()) {
+                    size_t nxt[2] = {0, 0};
+                    quad_base.resize(n_pages / 4);
+                    for (int pc = 0; pc < n_blocks; ++pc)
+                        for (int k16 = 0; k16 < ppt; k16 += 4) {
+                            const int d = owner_die(pc, k16);
+                            const int32_t q = groups[d][nxt[d]++];
+                            const int32_t a = ((first + (size_t)q) & 3) == 0 ? 3 : 1;
+                            const size_t p0 = (size_t)pc * ppt + k16;
+                            quad_base[p0 / 4] = q | (a == 1 ? (1 << 30) : 0);   // bit 30: group class (a = 1)
+                            w->h_page_table[p0] = q;
+                            w->h_page_table[p0 + 1] = q + a;
+                            w->h_page_table[p0 + 2] = q + (int32_t)F;
+                            w->h_page_table[p0 + 3] = q + (int32_t)F + a;
+                        }
+                    w->quad_free_bit = f;
+                }
             }
-            w->h_page_table[(size_t)pc * ppt + k16] = (int32_t)(2 * pair + (amap->h_die_of_chunk[2 * pair] == d ? 0 : 1));
+        }
+    }
+    if (w->quad_free_bit < 0) {
+        // two logical views over the chunk pairs: page p of view d = the chunk of pair p that sits on die d
+        size_t next[2] = {0, 0};
+        for (int pc = 0; pc < n_blocks; ++pc)
+            for (int k16 = 0; k16 < ppt; ++k16) {
+                const int d = owner_die(pc, k16);
+                const size_t pair = next[d]++;
+                if (2 * pair + 1 >= amap->n_chunks) {
+                    delete w;
+                    return AG_ERR_ARG;  // destination too small for this die's view
+                }
+                w->h_page_table[(size_t)pc * ppt + k16] =
+                    (int32_t)(2 * pair + (amap->h_die_of_chunk[2 * pair] == d ? 0 : 1));
+            }
+    } else {
+        // one box = the four pages of a group: [128 bf16][16 rows][2 x a chunks][2 x F chunks][base chunk]
+        EncodeTiledFn enc = get_encode_tiled();
+        const cuuint64_t F = (cuuint64_t)1 << w->quad_free_bit;
+        for (int cls = 0; cls < 2; ++cls) {
+            const cuuint64_t a = cls == 0 ? 3 : 1;
+            cuuint64_t dims[5] = {128, 16, 2, 2, (cuuint64_t)amap->n_chunks};
+            cuuint64_t strides[4] = {256, a * AG_CHUNK_BYTES, F * AG_CHUNK_BYTES, AG_CHUNK_BYTES};
+            cuuint32_t box[5] = {128, 16, 2, 2, 1};
+            cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+            if (!enc || enc(&w->tm_quad[cls], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, dst, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+                delete w;
+                return AG_ERR_CUDA;
+            }
         }
     }
     {
@@ -620,6 +714,11 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
     cudaError_t e = cudaMalloc(&w->d_page_table, sizeof(int32_t) * n_pages);
     if (e == cudaSuccess)
         e = cudaMemcpy(w->d_page_table, w->h_page_table.data(), sizeof(int32_t) * n_pages, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && w->quad_free_bit >= 0) {
+        e = cudaMalloc(&w->d_quad_base, sizeof(int32_t) * quad_base.size());
+        if (e == cudaSuccess)
+            e = cudaMemcpy(w->d_quad_base, quad_base.data(), sizeof(int32_t) * quad_base.size(), cudaMemcpyHostToDevice);
+    }
     const size_t pages_per_src = n_pages / G;
     for (int g = 0; g < G && e == cudaSuccess; ++g) {
         k_pack_weights<<<(unsigned)pages_per_src, 128>>>((const uint16_t*)B_list[g], K, n_src, ppt,
@@ -630,6 +729,7 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         cudaFree(w->d_page_table);
+        cudaFree(w->d_quad_base);
         delete w;
         return cuda_fail(e);
     }
@@ -637,17 +737,30 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
     return AG_OK;
 }
 
+extern "C" ag_status ag_pack_weights_ex(const void* const* B_list, int G, int K, int N_expert, const ag_plan* plan,
+                                        const ag_affinity_map* amap, void* dst, size_t dst_bytes, uint32_t flags,
+                                        ag_packed_weights** out) {
+    if (G < 1 || N_expert <= 0 || (long long)G * N_expert > 0x7fffffff) return AG_ERR_ARG;
+    return pack_weights_impl(B_list, G, K, G * N_expert, plan, amap, dst, dst_bytes, flags, out);
+}
+
+extern "C" ag_status ag_packed_info(const ag_packed_weights* w, int32_t* group_free_bit) {
+    if (!w || !group_free_bit) return AG_ERR_ARG;
+    *group_free_bit = w->quad_free_bit;
+    return AG_OK;
+}
+
 extern "C" ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, const ag_affinity_map* amap,
                                      void* dst, size_t dst_bytes, ag_packed_weights** out) {
     const void* list[1] = {B};
-    return pack_weights_impl(list, 1, K, N, plan, amap, dst, dst_bytes, out);
+    return pack_weights_impl(list, 1, K, N, plan, amap, dst, dst_bytes, 0, out);
 }
 
 extern "C" ag_status ag_pack_weights_grouped(const void* const* B_list, int G, int K, int N_expert, const ag_plan* plan,
                                              const ag_affinity_map* amap, void* dst, size_t dst_bytes,
                                              ag_packed_weights** out) {
     if (G < 1 || N_expert <= 0 || (long long)G * N_expert > 0x7fffffff) return AG_ERR_ARG;
-    return pack_weights_impl(B_list, G, K, G * N_expert, plan, amap, dst, dst_bytes, out);
+    return pack_weights_impl(B_list, G, K, G * N_expert, plan, amap, dst, dst_bytes, 0, out);
 }
 
 // ---- grouped (MoE-shaped) decode GEMM -------------------------------------------------------------------
@@ -761,6 +874,7 @@ extern "C" ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* o
 
 extern "C" void ag_packed_destroy(ag_packed_weights* w) {
     if (!w) return;
+    cudaFree(w->d_quad_base);
     cudaFree(w->d_page_table);
     delete w;
 }

@@ -85,6 +85,9 @@ struct ag_packed_weights {
     int pages_per_tile;                  // pages per column block = K / 16
     size_t n_pages;
     CUtensorMap tm_pages;                // dst seen as [chunk][16 rows][128 bf16]: one box = one 4 KB page
+    int quad_free_bit;                   // >= 2: pages are laid out in groups of four same-die chunks; -1: single pages
+    int32_t* d_quad_base;                // device [n_pages / 4]: first chunk of the group of every run of four pages
+    CUtensorMap tm_quad[2];              // one box = the four pages of a group (group classes q%4 == 0 / 1)
     const uint8_t* dst;                  // device: packed buffer (the probed buffer)
     size_t dst_bytes;
     int32_t* d_page_table;               // device [n_pages]: chunk index of each logical page

@@ -123,12 +123,17 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
     dst_bytes = 2 * K * N * 2 + (8 << 20)
     for b in budgets:
         plan_local = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
-        dsts, packs = [], []
+        dsts, packs, packs_single = [], [], []
         for i in range(n_buffers):                      # rotate buffers so that no launch finds its weights in L2
             dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
             amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
             packs.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
             dsts.append(dst)
+            dst1 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")   # same, one page per copy (for comparison)
+            amap1 = ag.affinity_probe(dst1.data_ptr(), dst_bytes, topo)
+            packs_single.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap1, dst1.data_ptr(), dst_bytes,
+                                                 single_pages=True), amap1))
+            dsts.append(dst1)
         table = packs[0][0].page_table()
         page_owner = np.repeat(_unit_die(plan_local), K // 16 // ksp)      # pages of a unit are consecutive
         on_die = float((packs[0][1].export()[table] == page_owner).mean())
@@ -143,11 +148,12 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
             plan_remote = ag.sched_build(topo, packs[0][1], b, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
         plan_obl = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
         out = {}
-        for name, plan in (("die_local", plan_local), ("remote", plan_remote)):
+        for name, plan, pset in (("die_local", plan_local, packs), ("remote", plan_remote, packs),
+                                 ("die_local_single_pages", plan_local, packs_single)):
             state = {"i": 0}
 
             def run():
-                pk = packs[state["i"] % n_buffers][0]
+                pk = pset[state["i"] % n_buffers][0]
                 state["i"] += 1
                 ag.gemm_persistent_packed(dA.data_ptr(), pk, dC.data_ptr(), M, N, K, plan)
             ms = time_queued(run, warmup=4, iters=24)
@@ -164,10 +170,10 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
             out[name] = algo_bytes / (ms * 1e-3) / 1e9
         emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
                   sm_budget=b, gbs=out, local_over_remote=out["die_local"] / out["remote"],
-                  pages_on_owner_die=on_die, local_set=sm_set_summary(topo, plan_local),
+                  pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), local_set=sm_set_summary(topo, plan_local),
                   remote_set=sm_set_summary(topo, plan_remote), algo_bytes=algo_bytes,
                   hbm_peak_measured_gbs=6534.1), fh)
-        del packs, dsts
+        del packs, packs_single, dsts
 
 
 def _unit_die(plan):

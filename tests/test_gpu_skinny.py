@@ -68,7 +68,16 @@ def test_in_memory_splitk_integer_exact_packed_and_rowmajor():
         assert np.array_equal(run_rowmajor(A, B, plan_m).astype(np.float64), ref)
 
 
-def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False):
+def oracle_page_table(packed, page_die, tbl, dst_ptr):
+    """The oracle's page table for the layout the library chose (single pages or groups of four)."""
+    f = packed.group_free_bit()
+    amap = dict(chunk_bytes=4096, die_of_chunk=tbl)
+    if f < 0:
+        return op.build_page_table(page_die, amap)
+    return op.build_page_table_quads(page_die, amap, f, first=(dst_ptr // 4096) % 512)
+
+
+def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False, single_pages=False):
     topo = device_topo()
     b = topo.n_sm if b is None else b
     if integer:
@@ -81,20 +90,23 @@ def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False):
     dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dB = to_dev_bf16(B)
-    packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes)
+    packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes, single_pages=single_pages)
     return topo, A, B, kw, plan_d, dst, amap, packed
 
 
-def test_packing_matches_oracle_table_and_layout():
+@pytest.mark.parametrize("single_pages", [False, True])
+def test_packing_matches_oracle_table_and_layout(single_pages):
     M, N, K, ksp = 16, 1024, 512, 2
-    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp)
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp, single_pages=single_pages)
+    assert (packed.group_free_bit() < 0) if single_pages else True
     tbl = amap.export()
     o_plan = op.build_plan(topo.as_dict(), None, topo.n_sm, op.default_policy(kind=op.DIE_COMPACT, **kw))
     assert plan_d.export().tobytes() == op.export(o_plan).tobytes()
     page_die = op.page_die_from_plan(o_plan, K)
-    want_table = op.build_page_table(page_die, dict(chunk_bytes=4096, die_of_chunk=tbl))
+    want_table = oracle_page_table(packed, page_die, tbl, dst.data_ptr())
     got_table = packed.page_table()
     assert np.array_equal(got_table, np.array(want_table, dtype=np.int32))
+    assert len(set(got_table.tolist())) == got_table.size
     # every page sits on the die of its unit wherever the pair rule holds
     on_die = tbl[got_table] == np.array(page_die)
     assert on_die.mean() > 0.99
@@ -105,8 +117,9 @@ def test_packing_matches_oracle_table_and_layout():
 
 
 @pytest.mark.parametrize("M,N,K,ksp", [(16, 1024, 1024, 1), (16, 2048, 2048, 4), (32, 1024, 512, 2), (9, 1096, 256, 1)])
-def test_packed_gemm_integer_exact(M, N, K, ksp):
-    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp, integer=True)
+@pytest.mark.parametrize("single_pages", [False, True])
+def test_packed_gemm_integer_exact(M, N, K, ksp, single_pages):
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp, integer=True, single_pages=single_pages)
     dA = to_dev_bf16(A)
     dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
     for _ in range(2):
