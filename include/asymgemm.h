@@ -340,8 +340,8 @@ ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, cons
  *   flags  bit 0: keep the one-page-per-copy layout even where groups of four pages are possible.
  * Grouped pages: when the map follows an XOR hash (ag_affinity_fit_hash) that uses chunk-index bits 0 and 1
  * and leaves some bit f in 2..8 out, the chunks {q, q+a, q+F, q+F+a} (F = 2^f; a = 3 for q = 0 mod 4, a = 1
- * for q = 1 mod 4; bit f of q clear) always sit on one die.  For decode-shaped plans the four pages of a
- * k-slab are then stored in one such group and fetched with a single strided copy; groups whose measured
+ * for q = 1 mod 4; bit f of q clear) always sit on one die.  The four pages of a k-slab (of one 128-column block)
+ * are then stored in one such group and fetched with a single strided copy; groups whose measured
  * chunks disagree are skipped.  ag_packed_info reports f (-1: single pages).
  */
 ag_status ag_pack_weights_ex(const void* const* B_list, int G, int K, int N_expert, const ag_plan* plan,

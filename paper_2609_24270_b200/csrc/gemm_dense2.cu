@@ -83,6 +83,14 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1,
+                                                 int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
 __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                                 uint32_t accumulate) {
     asm volatile(
@@ -153,8 +161,9 @@ struct PairSource {
 template <bool PACKED_B>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                       const __grid_constant__ CUtensorMap tm_c, const PersistParams p,
-                       const int32_t* __restrict__ page_table, const int pages_per_block, const GroupView gv) {
+                       const __grid_constant__ CUtensorMap tm_b2, const __grid_constant__ CUtensorMap tm_c,
+                       const PersistParams p, const int32_t* __restrict__ page_table, const int pages_per_block,
+                       const int32_t* __restrict__ quad_base, const GroupView gv) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -249,8 +258,13 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                     const int sb = ((b8 + rot) % n_blk) * 8;
                     int my_page = 0;
                     if (PACKED_B) {
-                        const int pg = sb * 4 + lane;
-                        if (pg < p.kslabs_total * 4) my_page = page_table[(size_t)(tn * 2 + (int)rank) * pages_per_block + pg];
+                        if (quad_base) {   // grouped pages: one entry per k-slab (bit 30 = class of the group)
+                            if (lane < 8 && sb + lane < p.kslabs_total)
+                                my_page = quad_base[(size_t)(tn * 2 + (int)rank) * (pages_per_block / 4) + sb + lane];
+                        } else {
+                            const int pg = sb * 4 + lane;
+                            if (pg < p.kslabs_total * 4) my_page = page_table[(size_t)(tn * 2 + (int)rank) * pages_per_block + pg];
+                        }
                     }
                     const int se = min(p.kslabs_total, sb + 8);
                     for (int s = sb; s < se; ++s, ++kit) {
@@ -278,7 +292,12 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                         }
                         ok = __shfl_sync(0xffffffffu, ok, 0);
                         if (!ok) break;
-                        if (PACKED_B) {
+                        if (PACKED_B && quad_base) {
+                            // the slab's four pages are one group of same-die chunks: one strided box
+                            const int q0 = __shfl_sync(0xffffffffu, my_page, s - sb);
+                            if (lane == 0)
+                                tma_load_5d_pair(sb_addr, (q0 >> 30) ? &tm_b2 : &tm_b, bar_leader, 0, 0, 0, 0, q0 & 0x3fffffff);
+                        } else if (PACKED_B) {
                             // four lanes issue the four page copies of the slab in one instruction: a single
                             // thread gets only one bulk copy out every ~150 cycles
                             const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + (lane & 3));
@@ -448,10 +467,10 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     }
     const void* b_key = W ? (const void*)W : B;
     if (grp) {
-        if (W) { plan->tm_b = W->tm_pages; plan->tm_b_ptr = nullptr; }   // the other maps come from the descriptor
+        if (W) { plan->tm_b = W->quad_free_bit >= 0 ? W->tm_quad[0] : W->tm_pages; plan->tm_b_ptr = nullptr; }
     } else if (plan->tm_a_ptr != A || plan->tm_b_ptr != b_key || plan->tm_c_ptr != Cout) {
         if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)) return AG_ERR_CUDA;
-        if (W) plan->tm_b = W->tm_pages;
+        if (W) plan->tm_b = W->quad_free_bit >= 0 ? W->tm_quad[0] : W->tm_pages;
         else if (N % 64 == 0) { if (!encode_b_blocks(&plan->tm_b, B, K, N, P_BK, 2)) return AG_ERR_CUDA; }
         else if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_BK)) return AG_ERR_CUDA;
         if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
@@ -487,9 +506,11 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int32_t* table = W ? W->d_page_table : nullptr;
+    const int32_t* quads = (W && W->quad_free_bit >= 0) ? W->d_quad_base : nullptr;
     const int ppb = W ? W->pages_per_tile : 0;
-    if (W) AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb, gv));
-    else AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, plan->tm_c, gp, table, ppb, gv));
+    const CUtensorMap tm_b2 = quads ? W->tm_quad[1] : plan->tm_b;   // second class of page groups
+    if (W) AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, tm_b2, plan->tm_c, gp, table, ppb, quads, gv));
+    else AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, tm_b2, plan->tm_c, gp, table, ppb, quads, gv));
     count_launch();
     return AG_OK;
 }

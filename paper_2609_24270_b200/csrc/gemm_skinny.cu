@@ -614,12 +614,12 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
         for (int tm = 0; tm < tiles_m; ++tm) votes[unit_die[((size_t)tm * tiles_n + tn) * ksp + ks]]++;
         return votes[0] >= votes[1] ? 0 : 1;
     };
-    // Grouped layout (decode-shaped plans): if the map follows an XOR hash that uses chunk-index bits 0 and 1 and
+    // Grouped layout: if the map follows an XOR hash that uses chunk-index bits 0 and 1 and
     // leaves some bit f >= 2 out, the chunks {q, q+a, q+F, q+F+a} (F = 2^f; a = 3 for q = 0 mod 4, a = 1 for
     // q = 1 mod 4; bit f of q clear) always share a die.  The four pages of a k-slab then go to one such group and
     // the kernel fetches them with one strided copy instead of four.
     std::vector<int32_t> quad_base;
-    if (!(flags & 1u) && h[H_TILE_N] == 128 && tiles_m == 1) {
+    if (!(flags & 1u)) {
         uint32_t mask = 0;
         size_t violations = 0;
         if (ag_affinity_fit_hash(amap, &mask, &violations) == AG_OK && (mask & 3u) == 3u &&

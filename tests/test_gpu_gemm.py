@@ -231,8 +231,10 @@ def test_die_packed_b_pages_and_affinity_plan_match_oracle():
     tbl = amap.export()
     o_plan = op.build_plan(topo.as_dict(), None, topo.n_sm, op.default_policy(kind=op.DIE_COMPACT, **kw))
     page_die = op.page_die_from_plan(o_plan, K)
-    assert packed.group_free_bit() < 0                       # dense plans keep single pages
-    want_table = op.build_page_table(page_die, dict(chunk_bytes=4096, die_of_chunk=tbl))
+    f = packed.group_free_bit()
+    o_amap = dict(chunk_bytes=4096, die_of_chunk=tbl)
+    want_table = (op.build_page_table(page_die, o_amap) if f < 0 else
+                  op.build_page_table_quads(page_die, o_amap, f, first=(dst.data_ptr() // 4096) % 512))
     got_table = packed.page_table()
     assert np.array_equal(got_table, np.array(want_table, dtype=np.int32))
     n_chunks = int(got_table.max()) + 1
