@@ -111,6 +111,97 @@ def test_mixer_published_vectors():
     assert [int(v) for v in inputs.mix64_np(xs)] == [op.mix64(int(x)) for x in xs]
 
 
+def seeded_golden():
+    out = {}
+    for line in open(os.path.join(GOLD, "seeded_subset.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, v = [f.strip() for f in line.split("|")]
+        out[k] = v
+    return out
+
+
+def test_seeded_subset_worked_example():
+    """The Fisher-Yates subset for a 6-SM chip and seed 5 against the swaps written out in the golden file."""
+    g = seeded_golden()
+    toy6 = dict(n_sm=6, n_tpc=3, n_gpc=1, n_die=2, tpc=[0, 0, 1, 1, 2, 2], gpc=[0] * 6, die=[0, 0, 0, 1, 1, 1],
+                is_random=[0] * 6, gpc_die=[0])
+    seed = int(g["seed"])
+    # the listed mixer outputs are the pinned mixer's (published-vector test above) ...
+    assert op.mix64(seed) == int(g["base"], 16)
+    r = {int(k): int(v, 16) for k, v in (f.split(":") for f in g["r"].split())}
+    j = {int(k): int(v) for k, v in (f.split(":") for f in g["j"].split())}
+    for i in range(5, 0, -1):
+        assert op.mix64((int(g["base"], 16) + i) & ((1 << 64) - 1)) == r[i]
+        assert r[i] % (i + 1) == j[i]
+    # ... the swaps of the file, replayed, give its final order ...
+    arr = list(range(6))
+    for i in range(5, 0, -1):
+        arr[i], arr[j[i]] = arr[j[i]], arr[i]
+    assert arr == [int(x) for x in g["final"].split()]
+    # ... and select_sms returns the first b of it, sorted
+    for b in (2, 3, 4):
+        pol = op.default_policy(kind=op.OBLIVIOUS, seed=seed, M=1, N=1, K=1)
+        assert op.select_sms(toy6, b, pol) == [int(x) for x in g[f"b{b}"].split()] == sorted(arr[:b])
+    # with SM 1 taken by another plan the candidate list is [0 2 3 4 5]: i runs 4..1 over five entries;
+    # r_4 mod 5 = 2, r_3 mod 4 = 0, r_2 mod 3 = 1, r_1 mod 2 = 0 ->
+    #   [0 2 3 4 5] -> swap(4,2) [0 2 5 4 3] -> swap(3,0) [4 2 5 0 3] -> swap(2,1) [4 5 2 0 3] -> swap(1,0) [5 4 2 0 3]
+    pol = op.default_policy(kind=op.OBLIVIOUS, seed=seed, M=1, N=1, K=1, avoid=[1])
+    assert op.select_sms(toy6, 3, pol) == [2, 4, 5]
+
+
+def test_k_range_when_splits_do_not_divide_the_slabs():
+    """Five k-slabs of 64: two splits take 3 + 2 slabs, three splits 2 + 2 + 1 (the first splits take the
+    longer runs); a ragged K clips the last slab."""
+    pol = op.default_policy(M=1, N=1, K=320, k_unit=64, k_splits=2)
+    assert [op.k_range(pol, ks) for ks in range(2)] == [(0, 192), (192, 320)]
+    pol = op.default_policy(M=1, N=1, K=320, k_unit=64, k_splits=3)
+    assert [op.k_range(pol, ks) for ks in range(3)] == [(0, 128), (128, 256), (256, 320)]
+    pol = op.default_policy(M=1, N=1, K=300, k_unit=64, k_splits=2)      # ceil(300 / 64) = 5 slabs, the last holds 44
+    assert [op.k_range(pol, ks) for ks in range(2)] == [(0, 192), (192, 300)]
+    pol = op.default_policy(M=1, N=1, K=320, k_unit=64, k_splits=4)      # 2 + 2 + 1 + 0: the last split is empty
+    assert [op.k_range(pol, ks) for ks in range(4)] == [(0, 128), (128, 256), (256, 320), (320, 320)]
+    pol = op.default_policy(M=1, N=1, K=8192, k_unit=64, k_splits=16)
+    assert op.k_range(pol, 5) == (5 * 512, 6 * 512)
+
+
+def test_rowmajor_b_panel_bytes_by_hand_and_by_brute_force():
+    """local_d(u) for a row-major B operand: rows = the unit's k range, columns = the unit's tile columns."""
+    # B is 128 x 512 bf16 (row stride 1024 B), chunks of 512 B: row k holds chunk 2k (columns 0..255) and
+    # chunk 2k+1 (columns 256..511).  Chunks of the left half sit on die 0 for k < 96, else die 1; the right
+    # half sits on die 1.  tile_n = 256, two k-splits of one 64-slab each.
+    doc = np.zeros(256, dtype=np.uint8)
+    for k in range(128):
+        doc[2 * k] = 0 if k < 96 else 1
+        doc[2 * k + 1] = 1
+    amap = dict(chunk_bytes=512, die_of_chunk=doc)
+    pol = op.default_policy(kind=op.AFFINITY, M=128, N=512, K=128, tile_m=128, tile_n=256, k_splits=2,
+                            b=op.operand(0, 1024, 2))
+    # unit id = (tm * 2 + tn) * 2 + ks
+    assert op.unit_local_bytes(pol, amap, 0) == [64 * 512, 0]            # tn 0, k 0..63: all on die 0
+    assert op.unit_local_bytes(pol, amap, 1) == [32 * 512, 32 * 512]     # tn 0, k 64..127: 32 rows each
+    assert op.unit_local_bytes(pol, amap, 2) == [0, 64 * 512]            # tn 1
+    assert op.unit_local_bytes(pol, amap, 3) == [0, 64 * 512]
+    # an irregular map, an offset that is not chunk aligned, a ragged N: count byte by byte
+    rng = np.random.default_rng(3)
+    doc = rng.integers(0, 2, size=700).astype(np.uint8)
+    amap = dict(chunk_bytes=256, die_of_chunk=doc)
+    K, N, off, stride = 192, 328, 136, 672
+    pol = op.default_policy(kind=op.AFFINITY, M=64, N=N, K=K, tile_m=64, tile_n=128, k_splits=2, k_unit=64,
+                            b=op.operand(off, stride, 2))
+    tiles_n = 3
+    for u in range(tiles_n * 2):
+        ks, tn = u % 2, u // 2
+        k0, k1 = op.k_range(pol, ks)
+        cnt = [0, 0]
+        for k in range(k0, k1):
+            for n in range(tn * 128, min(N, tn * 128 + 128)):
+                for byte in (0, 1):
+                    cnt[int(doc[(off + k * stride + n * 2 + byte) // 256])] += 1
+        assert op.unit_local_bytes(pol, amap, u) == cnt
+        assert sum(cnt) == (k1 - k0) * (min(N, tn * 128 + 128) - tn * 128) * 2
+
+
 def check_invariants(topo, plan, pol, b, avoid=()):
     S = plan["sm_list"]
     assert len(S) == b and S == sorted(set(S)) and not (set(S) & set(avoid))
