@@ -20,6 +20,10 @@
  *   - A handle (plan, affinity map, packed weights, group descriptor) may be used by one host
  *     thread at a time; launches of one plan must not overlap on the device (use one plan per
  *     stream).  Different plans may run concurrently on disjoint SM sets (avoid_sm_mask).
+ *   - gemm_persistent, gemm_persistent_packed, gemm_persistent_grouped and gemm_persistent_noalloc
+ *     return AG_ERR_ARG, and queue nothing, when cuda_stream is being captured: every launch carries
+ *     a launch number (epoch) in its kernel parameters, by which the thread blocks take their places
+ *     in the plan; a replayed graph would repeat an old number and no block would join.
  *   - Environment: AG_DEBUG=1 makes topo_discover print its bandwidth measurements and any
  *     rejected latency rows to stderr.  Nothing else is read from the environment.
  */
@@ -236,7 +240,12 @@ typedef struct {
     int32_t pair_lists;      /* 1: static lists are dealt to TPCs instead of SMs (entry i of a die's queue -> TPC i mod P,
                                 lower SM in even rounds, upper SM in odd ones), so that the two lists of a TPC together
                                 hold a fair share; for plans of block pairs.  Needs whole TPCs, else AG_ERR_ARG */
-    int32_t reserved1;
+    int32_t overlap_launches; /* decode-shaped plans with static lists that use every SM of the chip (ignored otherwise): 1 = a launch lets the next launch of this library on
+                                 the same stream begin while it is still finishing (programmatic dependent launch): the
+                                 next launch's thread blocks take over SMs as they become free and start streaming their
+                                 weights; nothing of theirs is written before this launch has completed.  The caller
+                                 promises that the inputs (A, B / packed weights) of a call are not produced by the call
+                                 directly before it.  0 = launches run strictly one after the other */
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;
@@ -418,16 +427,20 @@ ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weight
  * acceptable; code that runs after a framework has declared "no more allocations".  The split-K
  * partial sums and arrival counters, which normally live in memory that sched_build attached to
  * the plan, are placed instead in a fixed workspace that is part of the library image: 8 MiB +
- * 16 KiB of device memory on every GPU the library is loaded on, held until the process exits.
- * The call itself performs no cudaMalloc, cudaFree or any other allocating call.
+ * 16 KiB of device memory per GPU.  The CUDA runtime loads the library's device code onto a GPU
+ * when it is first used there, so the workspace (and the kernel itself) takes its memory during
+ * the first gemm_persistent_noalloc call on that GPU and keeps it until the process exits.  Make
+ * that first call at start-up, while memory is still available (any small problem will do); it can
+ * fail with AG_ERR_NOMEM if the GPU is already full.  From the second call on, a call performs no
+ * cudaMalloc, cudaFree or other allocating call and leaves the free device memory unchanged.
  *
  * Limits: k_splits * M * N * 4 bytes <= 8 MiB (for example M = 16, N = 8192, k_splits = 16) and
  * N <= 131072; larger problems are refused with AG_ERR_ARG, as are plans that are not
  * decode-shaped (tile_m > 32).  Arguments are those of gemm_persistent; the plan may come from a
  * sched_build done at start-up, when allocation was still allowed.
  *
- * The first call on each device looks up the workspace's device address; make that first call
- * outside any stream capture.  All calls on a device share the one workspace, which keeps
+ * The first call on each device also looks up the workspace's device address; make that first call
+ * before any stream capture.  All calls on a device share the one workspace, which keeps
  * whatever the previous call left in it (the counters are cleared on the given stream at the
  * start of every call): two calls whose kernels may run at the same time on one GPU - different
  * streams, or different host threads - race on it and give wrong results.  Serialise them.
