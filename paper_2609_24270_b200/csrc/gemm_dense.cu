@@ -99,7 +99,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 
     if (warp == 0) {
         // ------------------------------------------------ scheduler (warp-collective) + TMA producer (lane 0)
-        UnitSource src(p, slot);
+        UnitSource src(p, slot, lane);
         uint32_t it = 0, kit = 0;
         int ok = 1;
         while (ok) {
@@ -323,6 +323,18 @@ bool encode_b_blocks(CUtensorMap* tm, const void* ptr, uint64_t K, uint64_t N, u
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool encode_a_slabs(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows, uint32_t n_slabs) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc || (K % 64)) return false;
+    cuuint64_t dims[3] = {64, rows, K / 64};
+    cuuint64_t strides[2] = {K * 2, 128};
+    cuuint32_t box[3] = {64, box_rows, n_slabs};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN>
 static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream_t stream) {
     using C = Cfg<BN>;
@@ -331,10 +343,11 @@ static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream
     std::call_once(once, [] {
         attr_err = cudaFuncSetAttribute(k_gemm_persistent<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes);
     });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    if (attr_err != cudaSuccess) return launch_failed(plan, attr_err);
     k_gemm_persistent<BN><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, kThreads, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);
+    const cudaError_t le = cudaGetLastError();
+    if (le != cudaSuccess) return launch_failed(plan, le);
     count_launch();
-    AG_CUDA(cudaGetLastError());
     return AG_OK;
 }
 
@@ -358,11 +371,13 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
     if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if ((st = refuse_capture(stream)) != AG_OK) return st;
+    if ((st = renew_epochs_if_needed(plan, stream)) != AG_OK) return st;
     int dev = 0, n_sm = 0;
     AG_CUDA(cudaGetDevice(&dev));
     AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     if (n_sm != plan->lay.n_sm) return AG_ERR_ARG;
-    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     const int BN = h[H_TILE_N];
     if (plan->tm_a_ptr != A || plan->tm_b_ptr != B || plan->tm_c_ptr != Cout) {
         if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, BK, BM)) return AG_ERR_CUDA;

@@ -181,7 +181,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const int slot = p.image[lay.smid_to_slot() + my_sm];
     if (tid == 0) {
         ctl->abort_flag = 0;
-        ctl->member = slot >= 0 && atomicMax(&p.ctrl->claimed[slot], p.epoch) < p.epoch;
+        ctl->member = slot >= 0 && atomicMax(&p.claimed[slot], p.epoch) < p.epoch;
         for (int i = 0; i < P_STAGES; ++i) {
             mbar_init(smem_u32(&ctl->full[i]), 1);
             mbar_init(smem_u32(&ctl->empty[i]), 1);
@@ -453,6 +453,8 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     if (grp && (!grp->d_tm_c || (grp->N % P_BN))) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
+    if ((st = refuse_capture(stream)) != AG_OK) return st;
+    if ((st = renew_epochs_if_needed(plan, stream)) != AG_OK) return st;
     int dev = 0, n_sm = 0;
     AG_CUDA(cudaGetDevice(&dev));
     AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
@@ -509,8 +511,10 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     const int32_t* quads = (W && W->quad_free_bit >= 0) ? W->d_quad_base : nullptr;
     const int ppb = W ? W->pages_per_tile : 0;
     const CUtensorMap tm_b2 = quads ? W->tm_quad[1] : plan->tm_b;   // second class of page groups
-    if (W) AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, tm_b2, plan->tm_c, gp, table, ppb, quads, gv));
-    else AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, tm_b2, plan->tm_c, gp, table, ppb, quads, gv));
+    const cudaError_t le =
+        W ? cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<true>, plan->tm_a, plan->tm_b, tm_b2, plan->tm_c, gp, table, ppb, quads, gv)
+          : cudaLaunchKernelEx(&cfg, k_gemm_persistent_pair<false>, plan->tm_a, plan->tm_b, tm_b2, plan->tm_c, gp, table, ppb, quads, gv);
+    if (le != cudaSuccess) return launch_failed(plan, le);
     count_launch();
     return AG_OK;
 }

@@ -23,22 +23,36 @@ namespace ag {
 
 constexpr int SK_BN = 128;     // weight columns per unit
 constexpr int SK_BK = 64;      // k-slab
-// Six stages (about 110 KB in flight per SM) already cover bandwidth x latency several times; a deeper
-// ring only lengthens the queues in the memory system, and with them every dependent round trip
-// (fence, arrival atomic, reduction loads).
-constexpr int SK_STAGES = 6;
-constexpr int SK_W_BYTES = SK_BN * SK_BK * 2;      // 16 KB of weights per stage
-constexpr int SK_A_BYTES = 32 * SK_BK * 2;         // room for 32 activation rows
-constexpr int SK_STAGE_BYTES = SK_W_BYTES + SK_A_BYTES;
-constexpr int SK_SMEM_BYTES = SK_STAGES * SK_STAGE_BYTES + 1024 + 1024;
-// An MMA with so few columns finishes its arithmetic in a few cycles but a following MMA that adds to the
-// same accumulator has to wait for its result (measured: ~370 cycles per dependent K=16 step).  The
-// k-steps of a unit therefore rotate over SK_ACCS independent accumulators, summed in the epilogue.
-constexpr int SK_ACCS = 8;
+// Two things shape the pipeline (both measured on B200):
+//  - a warp gets only about two bulk copies in flight whatever their size (one thread issuing 16 KB copies streams
+//    35 GB/s from DRAM with 2, 6 or 12 stages, four warps issuing the same copies 139 GB/s), so the weight copies
+//    are issued by SK_WPROD warps in turn and the activation copies by yet another warp;
+//  - the thread that issues the MMAs pays a fixed ~400 cycles per stage (barrier wait, fence, commit and the queueing
+//    of its tcgen05 instructions) on top of ~55 cycles per MMA, however small the MMA: with one k-slab per stage that
+//    thread, not memory, set the pace (one slab per ~650 cycles = 40 GB/s per SM).  A stage therefore holds two
+//    k-slabs (32 KB of weights, 8 MMAs).
+constexpr int SK_SLABS = 2;    // k-slabs per weight stage
+constexpr int SK_WPROD = 3;    // warps that issue weight copies (stage i of the block's run belongs to warp i mod SK_WPROD)
+constexpr int SK_STAGES = 6;   // two stages per issuing warp
+constexpr int SK_THREADS = (2 + kEpiWarps + SK_WPROD) * 32;   // scheduler, MMA issuer, epilogue warps, weight producers
+constexpr int SK_SLAB_BYTES = SK_BN * SK_BK * 2;   // 16 KB of weights per k-slab
+constexpr int SK_W_BYTES = SK_SLABS * SK_SLAB_BYTES;
+constexpr int SK_STAGE_BYTES = SK_W_BYTES;
+// Activations come in groups of SK_AGRP k-slabs, one copy per group (A seen as [K/64][M][64]): with one copy
+// per k-slab the warp that issues them - two copies in flight, each an L2 round trip - capped the whole
+// pipeline at one slab per ~400 ns, the same 42 GB/s per SM that a single weight-issuing thread reaches.
+constexpr int SK_ASTAGES = 2;
+constexpr int SK_A_STAGE_MAX = 16 * 1024;          // 8 k-slabs of 16 rows, or 4 k-slabs of 32 rows
+__host__ __device__ constexpr int sk_agrp(int nm) { return SK_A_STAGE_MAX / (nm * SK_BK * 2); }
+constexpr int SK_SMEM_BYTES = SK_STAGES * SK_STAGE_BYTES + SK_ASTAGES * SK_A_STAGE_MAX + 1024 + 1024;
+// The tensor core takes ~45 cycles for an MMA this small whether or not it adds to the accumulator of the one
+// before (measured), so one accumulator per unit is enough.
 
 struct SkinnyCtl {
     uint64_t full[SK_STAGES];
     uint64_t empty[SK_STAGES];
+    uint64_t a_full[SK_ASTAGES];   // activations of a group of SK_AGRP k-slabs have landed
+    uint64_t a_empty[SK_ASTAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t sched_full[kRing];
@@ -48,6 +62,7 @@ struct SkinnyCtl {
     uint32_t tmem_base;
     int abort_flag;
     int member;
+    int4 quick;
 };
 
 struct SkinnyArgs {
@@ -67,6 +82,7 @@ struct SkinnyArgs {
     const int* g_row_off;         // device [G]
     int tiles_per_group;
     int n_group;                  // columns of one expert
+    int release_next;             // 1: let the next launch on the stream start while this one is still running
 };
 
 // Where the output rows of column tile tn live: single problem = C itself; grouped = rows of expert g in the
@@ -93,28 +109,47 @@ __device__ __forceinline__ OutView out_view(const PersistParams& p, const Skinny
     return v;
 }
 
+// a role that gave up lingers this long (bounded) so that copies already in flight land before the block leaves
+__device__ __forceinline__ void linger_for_copies() {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+}
+
 template <int NM, bool PACKED>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(SK_THREADS, 1)
 k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
               const __grid_constant__ CUtensorMap tm_w2, const PersistParams p, const SkinnyArgs x) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + SK_STAGES * SK_STAGE_BYTES);
-    constexpr uint32_t kAccCols = SK_ACCS * NM;          // columns of one accumulator set
-    constexpr uint32_t kTmemCols = 2 * kAccCols;         // two sets: 256 (NM = 16) or 512 (NM = 32) columns
+    constexpr uint32_t kASlab = NM * SK_BK * 2;          // activations of one k-slab
+    constexpr int SK_AGRP = sk_agrp(NM);                 // k-slabs per activation copy
+    constexpr uint32_t kAStage = SK_AGRP * kASlab;
+    const uint32_t a_base = base + SK_STAGES * SK_STAGE_BYTES;
+    SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + SK_STAGES * SK_STAGE_BYTES + SK_ASTAGES * SK_A_STAGE_MAX);
+    constexpr uint32_t kAccCols = NM;                    // columns of one accumulator
+    constexpr uint32_t kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;   // two accumulators (the smallest allocation is 32 columns)
     volatile int* abort_flag = &ctl->abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int my_sm = (int)smid();
-    if (tid == 0) ctl->abort_flag = 0;
-    const int slot = join_plan(p, &ctl->member);
-    if (slot < 0) return;
-
+    // overlap_launches: the launch that follows on the stream (this library's, by the caller's promise) may be
+    // scheduled as soon as every block of this one has got this far; its blocks move in as SMs become free
+    if (x.release_next && tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // One 16-byte entry tells this block its slot, its list and the list's first unit; the claim follows at once.
     if (tid == 0) {
+        ctl->abort_flag = 0;
+        const int4 qk = p.quick[my_sm];
+        ctl->quick = qk;
+        ctl->member = qk.x >= 0 && atomicMax(&p.claimed[qk.x], p.epoch) < p.epoch;
+    } else if (tid == 64) {
         for (int i = 0; i < SK_STAGES; ++i) {
             mbar_init(smem_u32(&ctl->full[i]), 1);
             mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < SK_ASTAGES; ++i) {
+            mbar_init(smem_u32(&ctl->a_full[i]), 1);
+            mbar_init(smem_u32(&ctl->a_empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
@@ -122,37 +157,63 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&ctl->sched_full[i]), 1);
-            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps + SK_WPROD);
         }
         mbar_init(smem_u32(&ctl->mma_drain), 1);
         mbar_fence_init();
         prefetch_tmap(&tm_a);
         if (!PACKED || x.quad_base) prefetch_tmap(&tm_w);
     }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
-        tmem_relinquish();
-    }
-    tc_fence_before();
     __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
+    const int4 quick = ctl->quick;
+    const int slot = quick.x;
+    if (!ctl->member) {
+        if (slot < 0) wait_until_manned(p);
+        return;
+    }
     const uint64_t limit = p.wait_limit_ns;
-    constexpr uint32_t kTxBytes = SK_W_BYTES + NM * SK_BK * 2;
+    // tensor memory is needed by the MMA issuer and the epilogue only: the copy-issuing warps do not wait for it
+    uint32_t tmem_base = 0;
+    if (warp >= 1 && warp < 2 + kEpiWarps) {
+        if (warp == 1) {
+            tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+            tmem_relinquish();
+        }
+        tc_fence_before();
+        asm volatile("bar.sync 1, %0;" ::"n"((1 + kEpiWarps) * 32) : "memory");
+        tc_fence_after();
+        tmem_base = ctl->tmem_base;
+    }
 
     if (warp == 0) {
-        // ------------------------------------------------ scheduler + producer.  Lane 0 waits and issues
-        // the copies; for packed weights all 32 lanes fetch the page-table entries of the next eight
-        // k-slabs (32 pages) with one load each, so the issuing lane never waits on a table lookup.
-        UnitSource src(p, slot);
-        const uint64_t stream_policy = l2_policy_evict_first();  // weights are read once: do not keep them in L2
-        uint32_t it = 0, kit = 0;
+        // ------------------------------------------------ scheduler + activation copies (lane 0)
+        UnitSource src(p, slot, lane, quick.y, quick.z, quick.w);
+        uint32_t it = 0, git = 0;
         int ok = 1;
         while (ok) {
-            const int u = src.next(lane);
+            int u;
+            if (p.static_assign) {
+                u = src.next_listed(lane);
+                while (u < 0 && ok) {
+                    // Own list done.  Planned SMs that never got a block are looked for only now that the
+                    // consumers have taken the last unit off the ring: by then every block of the launch has
+                    // long started, and the scan runs while the last unit is being streamed.
+                    if (it > 0 && lane == 0 &&
+                        !mbar_wait_idle(smem_u32(&ctl->sched_empty[(it - 1) % kRing]), ((it - 1) / kRing) & 1, abort_flag, limit)) {
+                        report_timeout(p, 1);
+                        ok = 0;
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok || !src.adopt(lane)) break;
+                    u = src.next_listed(lane);
+                }
+            } else {
+                u = src.next(lane);
+            }
+            if (!ok) break;
             if (lane == 0) {
                 const int r = it % kRing;
-                if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                if (!mbar_wait_idle(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 1);
                     ok = 0;
                 } else {
@@ -166,73 +227,134 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             if (!ok || u < 0) break;
             const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
             const int grp = x.tiles_per_group ? tn / x.tiles_per_group : 0;      // expert of this column tile
+            const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
+            const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+            if (lane == 0) {
+                const CUtensorMap* ma = x.g_tm_a ? &x.g_tm_a[grp] : &tm_a;
+                for (int g0 = s0; g0 < s1; g0 += SK_AGRP, ++git) {
+                    const int j = git % SK_ASTAGES;
+                    if (!mbar_wait_idle(smem_u32(&ctl->a_empty[j]), ((git / SK_ASTAGES) & 1) ^ 1, abort_flag, limit)) {
+                        report_timeout(p, 2);
+                        ok = 0;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&ctl->a_full[j]);
+                    const uint32_t dst = a_base + j * kAStage;
+                    if (p.a_blocks) {
+                        // the whole group with one copy; slabs past the end of K are zero-filled
+                        mbar_expect_tx(bar, kAStage);
+                        tma_load_3d(dst, ma, bar, 0, 0, g0);
+                    } else {
+                        const int n = min(SK_AGRP, s1 - g0);
+                        mbar_expect_tx(bar, n * kASlab);
+                        for (int i = 0; i < n; ++i) tma_load_2d(dst + i * kASlab, ma, bar, (g0 + i) * SK_BK, 0);
+                    }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+        if (!ok && lane == 0) linger_for_copies();
+    } else if (warp >= 2 + kEpiWarps) {
+        // ------------------------------------------------ weight copies: warp pw issues k-iterations pw, pw + SK_WPROD, ...
+        // For packed weights all 32 lanes fetch the page-table entries of the next eight k-slabs with one load
+        // each, so the issuing lane never waits on a table lookup.
+        const int pw = warp - (2 + kEpiWarps);
+        const uint64_t stream_policy = l2_policy_evict_first();  // weights are read once: do not keep them in L2
+        uint32_t q0 = 0;      // stage count (over the whole run of this block) before the current unit
+        int ok = 1;
+        for (uint32_t it = 0; ok; ++it) {
+            const int r = it % kRing;
+            int u = -1;
+            if (lane == 0) {
+                if (!mbar_wait_idle(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    report_timeout(p, 8);
+                    ok = 0;
+                } else {
+                    u = ctl->ring[r];
+                    mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            u = __shfl_sync(0xffffffffu, u, 0);
+            if (!ok || u < 0) break;
+            const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
+            const int grp = x.tiles_per_group ? tn / x.tiles_per_group : 0;      // expert of this column tile
             const int tl = x.tiles_per_group ? tn - grp * x.tiles_per_group : tn;  // tile inside the expert
             const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
             const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
-            for (int sb = s0; sb < s1 && ok; sb += 8) {
-                int my_page = 0;
-                if (PACKED) {
-                    if (x.quad_base) {   // one entry per k-slab: lanes 0..7 fetch the bases of the next eight slabs
-                        if (lane < 8 && sb + lane < s1) my_page = x.quad_base[(size_t)tn * (x.pages_per_tile / 4) + sb + lane];
+            const int n_st = (s1 - s0 + SK_SLABS - 1) / SK_SLABS;    // stages of this unit: slabs s0 + 2i, s0 + 2i + 1
+            // this warp's stages of the unit: i0, i0 + SK_WPROD, ...
+            const int i0 = (pw + SK_WPROD - (int)(q0 % SK_WPROD)) % SK_WPROD;
+            uint32_t st = (q0 + i0) % SK_STAGES, ph = (((q0 + i0) / SK_STAGES) & 1) ^ 1;   // stage, parity of "stage is free"
+            const CUtensorMap* mw = x.g_tm_w ? &x.g_tm_w[grp] : &tm_w;
+            // packed weights: lane l < 2 (groups of four pages) or l < 8 (single pages) looks up the chunk of the
+            // l-th 16 KB / 4 KB piece of a stage, one stage ahead of the copies
+            auto table_entry = [&](int i) -> int {
+                if (!PACKED || i >= n_st) return 0;
+                const int s = s0 + i * SK_SLABS;
+                if (x.quad_base) return (lane < SK_SLABS && s + lane < s1) ? x.quad_base[(size_t)tn * (x.pages_per_tile / 4) + s + lane] : 0;
+                return (lane < 4 * SK_SLABS && s + (lane >> 2) < s1) ? x.page_table[(size_t)tn * x.pages_per_tile + (size_t)s * 4 + lane] : 0;
+            };
+            int next_entry = table_entry(i0);
+            for (int i = i0; i < n_st && ok; i += SK_WPROD) {
+                const int entry = next_entry;
+                next_entry = table_entry(i + SK_WPROD);
+                const int s = s0 + i * SK_SLABS;
+                const int ns = min(SK_SLABS, s1 - s);
+                const uint32_t bar = smem_u32(&ctl->full[st]);
+                const uint32_t sw = base + st * SK_STAGE_BYTES;
+                if (lane == 0) {
+                    if (!mbar_wait(smem_u32(&ctl->empty[st]), ph, abort_flag, limit)) {
+                        report_timeout(p, 2);
+                        ok = 0;
                     } else {
-                        const int pg = sb * 4 + lane;
-                        if (pg < s1 * 4) my_page = x.page_table[(size_t)tn * x.pages_per_tile + pg];
+                        // row-major weights: one box of 128 k rows whatever ns is (rows past K arrive as zeros)
+                        mbar_expect_tx(bar, PACKED ? ns * SK_SLAB_BYTES : SK_W_BYTES);
                     }
                 }
-                const int se = min(s1, sb + 8);
-                for (int s = sb; s < se; ++s, ++kit) {
-                    const int st = kit % SK_STAGES;
-                    const uint32_t bar = smem_u32(&ctl->full[st]);
-                    const uint32_t sw = base + st * SK_STAGE_BYTES, sa = sw + SK_W_BYTES;
-                    if (lane == 0) {
-                        if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / SK_STAGES) & 1) ^ 1, abort_flag, limit)) {
-                            report_timeout(p, 2);
-                            ok = 0;
-                        } else {
-                            mbar_expect_tx(bar, kTxBytes);
-                        }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (PACKED && x.quad_base) {
+                    // grouped layout: a slab's four pages sit in chunks q, q+a, q+F, q+F+a of one die (a = 3 or 1 by
+                    // q mod 4): one strided box brings its 16 KB; bit 30 of the entry = class of the group
+                    if (lane < ns)
+                        tma_load_5d_hint(sw + lane * SK_SLAB_BYTES, (entry >> 30) ? &tm_w2 : &tm_w, bar, 0, 0, 0, 0,
+                                         entry & 0x3fffffff, stream_policy);
+                } else if (PACKED) {
+                    // one lane per 4 KB page, all in one instruction
+                    if (lane < 4 * ns)
+                        bulk_load_hint(sw + lane * 4096, x.packed + (size_t)entry * AG_CHUNK_BYTES, 4096, bar, stream_policy);
+                } else if (lane == 0) {
+                    if (p.b_blocks) {
+                        // both 64-column blocks with one copy (B seen as [N/64][K][64])
+                        tma_load_3d_hint(sw, mw, bar, 0, s * SK_BK, tl * 2, stream_policy);
+                    } else {
+                        tma_load_2d_hint(sw, mw, bar, tl * SK_BN, s * SK_BK, stream_policy);
+                        tma_load_2d_hint(sw + SK_W_BYTES / 2, mw, bar, tl * SK_BN + 64, s * SK_BK, stream_policy);
                     }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) break;
-                    if (PACKED && x.quad_base) {
-                        // grouped layout: the slab's four pages sit in chunks q, q+a, q+F, q+F+a of one die
-                        // (a = 3 or 1 by q mod 4): one strided box brings all 16 KB
-                        const int q0 = __shfl_sync(0xffffffffu, my_page, s - sb);   // bit 30: class of the group
-                        if (lane == 0)
-                            tma_load_5d_hint(sw, (q0 >> 30) ? &tm_w2 : &tm_w, bar, 0, 0, 0, 0, q0 & 0x3fffffff, stream_policy);
-                    } else if (PACKED) {
-                        // four lanes issue the four page copies of the slab in one instruction (a single thread
-                        // gets only one bulk copy out every ~150 cycles)
-                        const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + (lane & 3));
-                        if (lane < 4)
-                            bulk_load_hint(sw + lane * 4096, x.packed + (size_t)page * AG_CHUNK_BYTES, 4096, bar, stream_policy);
-                    } else if (lane == 0) {
-                        const CUtensorMap* mw = x.g_tm_w ? &x.g_tm_w[grp] : &tm_w;
-                        if (p.b_blocks) {
-                            // both 64-column blocks with one copy (B seen as [N/64][K][64])
-                            tma_load_3d_hint(sw, mw, bar, 0, s * SK_BK, tl * 2, stream_policy);
-                        } else {
-                            tma_load_2d_hint(sw, mw, bar, tl * SK_BN, s * SK_BK, stream_policy);
-                            tma_load_2d_hint(sw + 8192, mw, bar, tl * SK_BN + 64, s * SK_BK, stream_policy);
-                        }
-                    }
-                    if (lane == 0) tma_load_2d(sa, x.g_tm_a ? &x.g_tm_a[grp] : &tm_a, bar, s * SK_BK, 0);
                 }
+                // this warp's next stage is SK_WPROD stages on
+                st += SK_WPROD;
+                if (st >= SK_STAGES) { st -= SK_STAGES; ph ^= 1; }
             }
+            q0 += (uint32_t)n_st;
         }
-        if (!ok && lane == 0) {
-            // gave up: let the copies already in flight land before the block leaves
-            const uint32_t n_out = kit < (uint32_t)SK_STAGES ? kit : (uint32_t)SK_STAGES;
-            for (uint32_t j = 0; j < n_out; ++j) {
-                const uint32_t k2 = kit - 1 - j;
-                int dummy = 0;
-                mbar_wait(smem_u32(&ctl->full[k2 % SK_STAGES]), (k2 / SK_STAGES) & 1, &dummy, 2000000ull);
-            }
-        }
+        if (!ok && lane == 0) linger_for_copies();
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_bf16(128, NM, PACKED ? 0 : 1, 0);
-            uint32_t kit = 0, tile_it = 0;
+            // descriptors without their start address.  Weights: packed page = no swizzle, 16-byte k chunks 128 B
+            // apart (LBO), 8-row groups 256 B apart (SBO); row-major = MN-major with 128-byte swizzle, the two
+            // 64-column blocks of a stage half a stage apart (LBO), 8 k rows 1 KB apart (SBO).  The address field
+            // counts 16-byte units; shared memory is below 256 KB, so adding to the low word never carries out of it.
+            const uint64_t dw_t = PACKED ? make_smem_desc(0, 128, 256, 0) : make_smem_desc(0, SK_W_BYTES / 2, 1024, 2);
+            const uint64_t da_t = make_smem_desc(0, 16, 1024, 2);
+            constexpr uint32_t kWStep = (PACKED ? 4096u : 2048u) >> 4;   // one K = 16 step inside a weight stage
+            constexpr uint32_t kAStepK = 32u >> 4;                       // ... inside an activation slab
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            uint32_t st = 0, ph = 0;                  // weight stage and the parity of "stage is full"
+            uint32_t aj = 0, aph = 0;                 // activation buffer and the parity of "buffer is full"
+            uint32_t tile_it = 0;
             bool ok = true;
             for (uint32_t it = 0; ok; ++it) {
                 const int r = it % kRing;
@@ -253,26 +375,44 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kAccCols;
-                for (int s = s0; s < s1; ++s, ++kit) {
-                    const int st = kit % SK_STAGES;
-                    if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / SK_STAGES) & 1, abort_flag, limit)) {
+                int in_grp = 0;                       // k-slabs of the current activation buffer already used
+                uint64_t da = 0;
+                for (int left = s1 - s0, first = 1; left > 0; left -= SK_SLABS) {
+                    if (in_grp == 0) {
+                        if (!mbar_wait(smem_u32(&ctl->a_full[aj]), aph, abort_flag, limit)) {
+                            report_timeout(p, 9);
+                            ok = false;
+                            break;
+                        }
+                        da = da_t | (uint64_t)((a_base + aj * kAStage) >> 4);
+                    }
+                    if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
                         report_timeout(p, 5);
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t sw = base + st * SK_STAGE_BYTES, sa = sw + SK_W_BYTES;
+                    const uint64_t dw = dw_t | (uint64_t)((base + st * SK_STAGE_BYTES) >> 4);
+                    // the first k-slab of the stage, then the second one if the unit has it
+                    tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
 #pragma unroll
-                    for (int k4 = 0; k4 < SK_BK / 16; ++k4) {
-                        // weights: packed page = no swizzle, 16-byte k chunks 128 B apart (LBO), 8-row groups
-                        // 256 B apart (SBO); row-major = MN-major, 128-byte swizzle, as B in the dense kernel
-                        const uint64_t dw = PACKED ? make_smem_desc(sw + k4 * 4096, 128, 256, 0)
-                                                   : make_smem_desc(sw + k4 * 2048, 8192, 1024, 2);
-                        const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
-                        const int step = (s - s0) * 4 + k4;  // k-step of this unit -> accumulator step mod SK_ACCS
-                        tc_mma_f16(d_tmem + (step & (SK_ACCS - 1)) * NM, dw, da, idesc, step >= SK_ACCS ? 1u : 0u);
+                    for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
+                    if (left > 1) {
+                        const uint64_t da2 = da + (kASlab >> 4);
+#pragma unroll
+                        for (int k4 = 0; k4 < SK_BK / 16; ++k4)
+                            tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
                     }
-                    tc_commit(smem_u32(&ctl->empty[st]));
+                    first = 0;
+                    tc_commit(empty0 + st * 8);
+                    if (++st == SK_STAGES) { st = 0; ph ^= 1; }
+                    da += SK_SLABS * (kASlab >> 4);
+                    in_grp += SK_SLABS;
+                    if (in_grp >= SK_AGRP || left <= SK_SLABS) {   // last stage that reads this buffer's activations
+                        tc_commit(smem_u32(&ctl->a_empty[aj]));
+                        in_grp = 0;
+                        if (++aj == SK_ASTAGES) { aj = 0; aph ^= 1; }
+                    }
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&ctl->tmem_full[acc]));
@@ -298,7 +438,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         int st_tn = -1;              // unit whose partial sums are stored but not yet announced
         int at_tn = -1;              // unit whose arrival atomic is in flight
         int oldA = 0, oldB = 0;      // results of the arrival atomics (lane 0), used one unit later
-        bool zero_done = false;      // in-memory split-K: the zeroing of C is known to be complete
+        bool prior_done = false;     // everything launched before this kernel is known to be complete
 
         auto reduce_columns = [&](int tn) {
             __threadfence();
@@ -310,15 +450,15 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             if (nq < p.N && nlq < ov.n_cols) {
                 for (int m = lane >> 3; m < ov.rows; m += 4) {
                     float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int k0 = 0; k0 < p.k_splits; k0 += 16) {
-                        float4 t[16];
+                    for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
+                        float4 t[8];
 #pragma unroll
-                        for (int k = 0; k < 16; ++k)
+                        for (int k = 0; k < 8; ++k)
                             if (k0 + k < p.k_splits)
                                 t[k] = __ldcg(reinterpret_cast<const float4*>(
                                     x.partial + ((size_t)(k0 + k) * p.M + m) * p.N + nq));
 #pragma unroll
-                        for (int k = 0; k < 16; ++k)
+                        for (int k = 0; k < 8; ++k)
                             if (k0 + k < p.k_splits) {
                                 acc4.x += t[k].x; acc4.y += t[k].y; acc4.z += t[k].z; acc4.w += t[k].w;
                             }
@@ -348,7 +488,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         // one unit; returns false when the list is finished (or a wait ran out)
         auto one_unit = [&](int& old_use, int& old_new) -> bool {
             const int r = it % kRing;
-            if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+            if (!mbar_wait_warp(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 6);
                 return false;
             }
@@ -359,42 +499,38 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             if (u < 0) return false;
             const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
             const uint32_t acc = tile_it & 1;
-            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
+            if (!mbar_wait_warp(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 7);
                 return false;
             }
             tc_fence_after();
-            // sum the accumulators that this unit used
-            const int s0e = min(p.kslabs_total, ks * p.kslabs_per_split);
-            const int s1e = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
-            const int n_used = min(SK_ACCS, (s1e - s0e) * 4);
             float sum[NM];
-#pragma unroll
-            for (int m = 0; m < NM; ++m) sum[m] = 0.f;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
-            for (int j = 0; j < n_used; ++j) {
+            {
                 uint32_t v[NM];
-                if constexpr (NM == 16) tmem_ld_32x16(taddr + j * NM, v); else tmem_ld_32x32(taddr + j * NM, v);
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
+                if constexpr (NM == 16) tmem_ld_32x16(taddr, v); else tmem_ld_32x32(taddr, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int m = 0; m < NM; ++m) sum[m] += __uint_as_float(v[m]);
+                for (int m = 0; m < NM; ++m) sum[m] = __uint_as_float(v[m]);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
             ++tile_it;
+            // This kernel may have started while the one before it (the zeroing of C, or with overlap_launches the
+            // previous GEMM) was still running (programmatic dependent launch): before the first byte is written,
+            // make sure that everything before it on the stream has completed.
+            if (!prior_done) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                prior_done = true;
+            }
             const int n = tn * SK_BN + q * 32 + lane;     // column in the plan's (possibly grouped) N
             const OutView ov = out_view(p, x, tn);
             const int nl = ov.col0 + q * 32 + lane;       // column inside the tile's problem
             if (p.k_splits > 1 && x.partial == nullptr) {
                 // in-memory reduction: C is zeroed by the kernel launched just before this one, every unit adds
                 // its partial sums with reductions that L2 carries out; nothing comes back, so nothing is
-                // waited for.  This kernel may have started while the zeroing was still running (programmatic
-                // dependent launch): make sure it is complete before the first add.
-                if (!zero_done) {
-                    asm volatile("griddepcontrol.wait;" ::: "memory");
-                    zero_done = true;
-                }
+                // waited for
                 if (nl < ov.n_cols) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m)
@@ -446,6 +582,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
 // once, so the GEMM's start-up overlaps the zeroing; the GEMM waits for this kernel only before its first add.
 __global__ void k_zero_f32(float4* __restrict__ p, size_t n_vec) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // with overlap_launches this kernel itself may have started early: the GEMM before it may still be adding to C
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x)
         p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
@@ -474,26 +612,27 @@ __global__ void k_pack_weights(const uint16_t* __restrict__ B, int K, int N, int
 
 template <int NM, bool PACKED>
 static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_w2,
-                               const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream, bool after_zeroing) {
+                               const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream, bool may_start_early) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
         attr_err = cudaFuncSetAttribute(k_gemm_skinny<NM, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         SK_SMEM_BYTES);
     });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    if (attr_err != cudaSuccess) return launch_failed(plan, attr_err);
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(SK_THREADS);
     cfg.dynamicSmemBytes = SK_SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = after_zeroing ? 1 : 0;   // may start while the zeroing kernel before it is still running
-    AG_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_skinny<NM, PACKED>, tm_a, tm_w, tm_w2, gp, x));
+    cfg.numAttrs = may_start_early ? 1 : 0;   // may start while the kernel before it (zeroing, previous GEMM) is still running
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, k_gemm_skinny<NM, PACKED>, tm_a, tm_w, tm_w2, gp, x);
+    if (le != cudaSuccess) return launch_failed(plan, le);
     count_launch();
     return AG_OK;
 }
@@ -501,7 +640,7 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
 // Shared host path of the two skinny entry points.
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
                                int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream,
-                               const ag_group_desc* grp) {
+                               const ag_group_desc* grp, bool clear_sem) {
     const int32_t* h = plan->header;
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_N] != SK_BN || (h[H_TILE_M] != 16 && h[H_TILE_M] != 32) || M > h[H_TILE_M]) return AG_ERR_ARG;
@@ -509,6 +648,8 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     if (((uintptr_t)A | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
+    if ((st = refuse_capture(stream)) != AG_OK) return st;
+    if ((st = renew_epochs_if_needed(plan, stream)) != AG_OK) return st;
     int dev = 0, n_sm = 0;
     AG_CUDA(cudaGetDevice(&dev));
     AG_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
@@ -518,7 +659,10 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     memset(&tm_w, 0, sizeof tm_w);
     memset(&tm_w2, 0, sizeof tm_w2);
     memset(&tm_a, 0, sizeof tm_a);
-    if (!grp && !encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, SK_BK, NM)) return AG_ERR_CUDA;
+    const bool a_blocks = grp ? grp->a_blocks != 0 : (K % SK_BK == 0);
+    if (!grp && !(a_blocks ? encode_a_slabs(&tm_a, A, M, K, NM, sk_agrp(NM))
+                           : encode_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, SK_BK, NM)))
+        return AG_ERR_CUDA;
     SkinnyArgs x;
     memset(&x, 0, sizeof x);
     if (grp) {
@@ -548,26 +692,45 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     } else {
         if (!B_rowmajor || ((uintptr_t)B_rowmajor & 15u)) return AG_ERR_ARG;
         if (N % 64 == 0) {
-            if (!encode_b_blocks(&tm_w, B_rowmajor, K, N, SK_BK, 2)) return AG_ERR_CUDA;
-        } else if (!encode_2d(&tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_rowmajor, K, N, 64, SK_BK)) {
+            if (!encode_b_blocks(&tm_w, B_rowmajor, K, N, SK_SLABS * SK_BK, 2)) return AG_ERR_CUDA;
+        } else if (!encode_2d(&tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_rowmajor, K, N, 64, SK_SLABS * SK_BK)) {
             return AG_ERR_CUDA;
         }
     }
+    // every argument check has passed: from here on work is queued on the stream
+    if (clear_sem && sem) AG_CUDA(cudaMemsetAsync(sem, 0, (size_t)h[H_TILES_N] * 4 * sizeof(int), stream));
     const bool zeroing = h[H_KSPLITS] > 1 && !x.partial;
+    // Overlapping launches: only for plans that use every SM with one block each - the blocks of the next launch then
+    // find room exactly where a block of this one has left, one per SM, and no block of the launch after next can
+    // start before this launch has completed.  (With fewer planned SMs the next launch's blocks would all land on the
+    // idle SMs and leave the planned ones without a block.)  Static lists only: the queue heads of dynamic plans
+    // belong to one launch at a time.
+    const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0 && plan->lay.b == plan->lay.n_sm;
+    x.release_next = overlap ? 1 : 0;
     if (zeroing) {  // in-memory reduction mode: the adds need a zeroed C (N % 8 == 0 and 16-byte alignment: whole float4s)
         const size_t c_elems = grp ? (size_t)grp->total_rows * (size_t)grp->N : (size_t)M * (size_t)N;
         const size_t n_vec = c_elems / 4;
         const unsigned blocks = (unsigned)std::min<size_t>(148, (n_vec + 255) / 256);
-        k_zero_f32<<<blocks, 256, 0, stream>>>((float4*)Cout, n_vec);
+        cudaLaunchConfig_t zc;
+        memset(&zc, 0, sizeof zc);
+        zc.gridDim = dim3(blocks);
+        zc.blockDim = dim3(256);
+        zc.stream = stream;
+        cudaLaunchAttribute za[1];
+        za[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        za[0].val.programmaticStreamSerializationAllowed = 1;
+        zc.attrs = za;
+        zc.numAttrs = overlap ? 1 : 0;     // may be scheduled while the GEMM before it is finishing; it waits before it writes
+        AG_CUDA(cudaLaunchKernelEx(&zc, k_zero_f32, (float4*)Cout, n_vec));
         count_launch();
-        AG_CUDA(cudaGetLastError());
     }
     PersistParams gp = make_persist_params(plan, M, N, K);
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
-    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing)
-                           : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing);
-    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing)
-             : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing);
+    gp.a_blocks = a_blocks ? 1 : 0;
+    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
+                           : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
+    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
+             : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
 }
 
 }  // namespace ag
@@ -794,6 +957,7 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
     d->A_all = A_all; d->C_all = C_all;
     d->d_tm_a = nullptr; d->d_tm_w = nullptr; d->d_tm_c = nullptr; d->d_rows = nullptr; d->d_row_off = nullptr;
     d->w_blocks = (N_expert % 64 == 0) ? 1 : 0;
+    d->a_blocks = (!dense && K % SK_BK == 0) ? 1 : 0;
     d->rows.assign(rows, rows + G);
     d->row_off.resize(G);
     std::vector<CUtensorMap> ha(G), hw(B_list ? G : 0), hc(dense ? G : 0);
@@ -806,7 +970,8 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
         const int n_rows = std::max(1, rows[g]);
         const char* base = (const char*)A_all + (size_t)first * K * 2;
         const uint64_t view_rows = (uint64_t)std::min<long long>(n_rows, total - first);
-        if (!encode_2d(&ha[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, view_rows, K, SK_BK, a_box_rows)) {
+        if (!(d->a_blocks ? encode_a_slabs(&ha[g], base, view_rows, K, a_box_rows, sk_agrp((int)a_box_rows))
+                          : encode_2d(&ha[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, view_rows, K, SK_BK, a_box_rows))) {
             delete d;
             return AG_ERR_CUDA;
         }
@@ -819,8 +984,9 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
         }
         if (B_list) {
             if (!B_list[g] || ((uintptr_t)B_list[g] & 15u)) { delete d; return AG_ERR_ARG; }
-            const bool ok = d->w_blocks ? encode_b_blocks(&hw[g], B_list[g], K, N_expert, SK_BK, 2)
-                                        : encode_2d(&hw[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_list[g], K, N_expert, 64, SK_BK);
+            const int wk = dense ? SK_BK : SK_SLABS * SK_BK;   // k rows per weight copy of the kernel that will read them
+            const bool ok = d->w_blocks ? encode_b_blocks(&hw[g], B_list[g], K, N_expert, wk, 2)
+                                        : encode_2d(&hw[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_list[g], K, N_expert, 64, wk);
             if (!ok) { delete d; return AG_ERR_CUDA; }
         }
         off += rows[g];
@@ -895,8 +1061,10 @@ extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weigh
 // server that has handed every free byte of the GPU to its own arena (cudaMalloc simply fails
 // there), a request loop with a latency budget that an allocator call would break, or code
 // running between other libraries' strict "no allocation after start-up" phases.  For them the
-// split-K workspace lives in the library image itself: a fixed array in device memory that exists
-// on every GPU from the moment the library is loaded there until the process ends.
+// split-K workspace lives in the library image itself: a fixed array in device memory.  The CUDA
+// runtime places the library's device code on a GPU when it is first used there (lazy module
+// loading), so the array starts to exist on a GPU with the first call made on it - which is why that
+// first call belongs at start-up, while memory is still to be had - and stays until the process ends.
 //
 // The array's name is only a host-side handle; the address the kernel needs is asked from the
 // runtime once per device (cudaGetSymbolAddress, with that device current) and remembered.
@@ -912,6 +1080,10 @@ void* g_noalloc_ptr[64] = {nullptr};   // device address of g_noalloc_scratch, p
 extern "C" ag_status gemm_persistent_noalloc(const void* A, const void* B, void* Cout, int M, int N, int K,
                                              const ag_plan* plan, void* cuda_stream) {
     if (!A || !B || !Cout || !plan) return AG_ERR_ARG;
+    {
+        const ag_status cap = refuse_capture(reinterpret_cast<cudaStream_t>(cuda_stream));
+        if (cap != AG_OK) return cap;
+    }
     const int32_t* h = plan->header;
     if (h[H_TILE_M] > 32) return AG_ERR_ARG;  // only decode-shaped plans use a workspace
     const int ksp = h[H_KSPLITS], tiles_n = h[H_TILES_N];
@@ -935,7 +1107,7 @@ extern "C" ag_status gemm_persistent_noalloc(const void* A, const void* B, void*
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     int* sem = reinterpret_cast<int*>(scratch);
     float* partial = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + kNoAllocSemBytes);
-    // the counters must start at zero; whatever an earlier call left behind is wiped on the same stream
-    AG_CUDA(cudaMemsetAsync(sem, 0, (size_t)tiles_n * 4 * sizeof(int), stream));
-    return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, partial, sem, stream);
+    // the counters must start at zero: once the arguments have been checked, whatever an earlier call left
+    // behind is wiped on the same stream, right in front of the kernel
+    return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, partial, sem, stream, nullptr, true);
 }

@@ -40,7 +40,10 @@ struct PlanCtrl {
     int status_info;                 // where the kernel gave up (role << 16 | smid)
     unsigned int adopted;            // lists run by a block other than the one pinned to their SM
     unsigned int pad;
-    unsigned int claimed[AG_MAX_SM]; // epoch of the launch whose block took this slot
+    // epoch of the launch whose block took this slot.  Two arrays, used by even and odd launches in turn: the
+    // blocks of a launch may start while the launch before it is still finishing (overlap_launches), and each
+    // of the two must see exactly its own claims.
+    unsigned int claimed[2][AG_MAX_SM];
 };
 
 }  // namespace ag
@@ -69,6 +72,7 @@ struct ag_plan {
     long long* d_margins;      // device [n_units] (affinity only, else null)
     float* d_partial;          // device [k_splits][M][N] split-K partial sums (skinny plans with k_splits > 1)
     int* d_sem;                // device [4 * tiles_n] arrival counters for the split-K reduction
+    int4* d_quick;             // device [n_sm]: {slot, list offset, list length, first unit} per SM id
     std::vector<int32_t> h_image;
     mutable uint32_t epoch;
     int grid_blocks;           // 0: one block per SM; else launch this many blocks (one-block and decode-shaped kernels)
@@ -108,6 +112,7 @@ struct ag_group_desc {
     int* d_rows;           // device [G]
     int* d_row_off;        // device [G]
     int w_blocks;          // 1: d_tm_w are the 3-D [N/64][K][64] views
+    int a_blocks;          // 1: d_tm_a are the 3-D [K/64][rows][64] views (decode-shaped descriptors, K % 64 == 0)
 };
 
 namespace ag {

@@ -443,7 +443,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     pl->d_image = nullptr; pl->d_ctrl = nullptr; pl->d_tile_owner = nullptr; pl->d_tile_count = nullptr;
     pl->d_margins = nullptr;
     pl->d_unit_times = nullptr;
-    pl->d_partial = nullptr; pl->d_sem = nullptr;
+    pl->d_partial = nullptr; pl->d_sem = nullptr; pl->d_quick = nullptr;
     pl->epoch = 0;
     pl->grid_blocks = 0;
     pl->kslabs_total = n_slab;
@@ -512,6 +512,25 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pl->h_image.resize(pl->lay.total());
         TRY(cudaMemcpy(pl->h_image.data(), pl->d_image, image_bytes, cudaMemcpyDeviceToHost));
         memcpy(pl->header, pl->h_image.data(), sizeof pl->header);
+        {
+            // per SM id: its slot, its list and the list's first unit in one 16-byte entry, so that a block
+            // learns all of it with a single load
+            const int32_t* img = pl->h_image.data();
+            std::vector<int4> quick(map->n_sm);
+            for (int s = 0; s < map->n_sm; ++s) {
+                const int slot = img[pl->lay.smid_to_slot() + s];
+                int4 q = make_int4(-1, 0, 0, -1);
+                if (slot >= 0) {
+                    q.x = slot;
+                    q.y = img[pl->lay.sm_q_off() + slot];
+                    q.z = img[pl->lay.sm_q_off() + slot + 1] - q.y;
+                    q.w = q.z > 0 ? img[pl->lay.sm_q() + q.y] : -1;
+                }
+                quick[s] = q;
+            }
+            TRY(cudaMalloc(&pl->d_quick, sizeof(int4) * map->n_sm));
+            TRY(cudaMemcpy(pl->d_quick, quick.data(), sizeof(int4) * map->n_sm, cudaMemcpyHostToDevice));
+        }
         if (p.pair_lists) {
             // units were dealt to TPCs: every chosen TPC must be whole (both SMs chosen, adjacent in the die's ranks)
             const int32_t* img = pl->h_image.data();
@@ -616,7 +635,7 @@ extern "C" ag_status ag_last_status(const ag_plan* plan) {
     if (c.status != 0) return (ag_status)c.status;
     if (plan->epoch != 0) {
         std::vector<unsigned int> claimed(plan->lay.b);
-        AG_CUDA(cudaMemcpy(claimed.data(), (const char*)plan->d_ctrl + offsetof(PlanCtrl, claimed),
+        AG_CUDA(cudaMemcpy(claimed.data(), (const char*)plan->d_ctrl + offsetof(PlanCtrl, claimed) + sizeof(unsigned int) * AG_MAX_SM * (plan->epoch & 1u),
                            sizeof(unsigned int) * plan->lay.b, cudaMemcpyDeviceToHost));
         int n_claimed = 0;
         for (int i = 0; i < plan->lay.b; ++i) n_claimed += claimed[i] == plan->epoch;
@@ -637,5 +656,6 @@ extern "C" void ag_plan_destroy(ag_plan* plan) {
     cudaFree(plan->d_unit_times);
     cudaFree(plan->d_partial);
     cudaFree(plan->d_sem);
+    cudaFree(plan->d_quick);
     delete plan;
 }

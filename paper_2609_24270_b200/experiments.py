@@ -111,14 +111,14 @@ def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
 
 
 # ---------------------------------------------------------------------------------------------
-def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
+def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
     """M=16, N=K=8192 decode-shaped GEMM, weights die-packed; die-local vs remote assignment."""
     M, N, K, ksp = 16, 8192, 8192, 16
     A = inputs.uniform_bf16(M, K, inputs.DEFAULT_SEED)
     dA = dev_bf16(A)
     dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
     algo_bytes = K * N * 2 + M * K * 2 + M * N * 4
-    kw = dict(M=M, N=N, K=K, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=1)
+    kw = dict(M=M, N=N, K=K, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=1, overlap_launches=overlap)
     Bs = [dev_bf16(inputs.uniform_bf16(K, N, inputs.DEFAULT_SEED + 1 + i)) for i in range(n_buffers)]
     dst_bytes = 2 * K * N * 2 + (8 << 20)
     for b in budgets:
@@ -169,7 +169,7 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4):
             ms = time_queued(run2, warmup=4, iters=24)
             out[name] = algo_bytes / (ms * 1e-3) / 1e9
         emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
-                  sm_budget=b, gbs=out, local_over_remote=out["die_local"] / out["remote"],
+                  sm_budget=b, overlap_launches=overlap, gbs=out, local_over_remote=out["die_local"] / out["remote"],
                   pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), local_set=sm_set_summary(topo, plan_local),
                   remote_set=sm_set_summary(topo, plan_remote), algo_bytes=algo_bytes,
                   hbm_peak_measured_gbs=6534.1), fh)

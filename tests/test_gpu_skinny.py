@@ -40,7 +40,8 @@ def test_rowmajor_weights_integer_exact(M, tile_m, k_splits):
     assert (count == 2).all()
 
 
-@pytest.mark.parametrize("shape", [(16, 8192, 8192, 16), (32, 4096, 4096, 8), (16, 1000, 520, 2), (7, 264, 72, 1)])
+@pytest.mark.parametrize("shape", [(16, 8192, 8192, 16), (32, 4096, 4096, 8), (16, 1000, 520, 2), (7, 264, 72, 1),
+                                   (16, 384, 1280, 1), (32, 256, 1344, 2)])
 @pytest.mark.parametrize("in_memory", [0, 1])
 def test_rowmajor_weights_uniform(shape, in_memory):
     M, N, K, ksp = shape
@@ -51,6 +52,32 @@ def test_rowmajor_weights_uniform(shape, in_memory):
                                                             tile_m=16 if M <= 16 else 32, tile_n=128, k_splits=ksp))
         for _ in range(2):
             check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
+
+
+@pytest.mark.parametrize("in_memory", [0, 1])
+def test_overlapping_launches_integer_exact(in_memory):
+    """overlap_launches: a launch lets the next one start while it is still finishing.  Nine launches are queued
+    without any synchronisation in between, over three weight matrices and three outputs; every output must be
+    exact (integer-valued inputs), and every unit must have run once per launch."""
+    M, N, K, ksp = 16, 2048, 4096, 8
+    topo = device_topo()
+    A = inputs.small_int_bf16(M, K, 61)
+    Bs = [inputs.small_int_bf16(K, N, 62 + i) for i in range(3)]
+    dA = to_dev_bf16(A)
+    dBs = [to_dev_bf16(b) for b in Bs]
+    dCs = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+    for b in (topo.n_sm, 74):
+        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
+                                                            k_splits=ksp, splitk_in_memory=in_memory, overlap_launches=1))
+        plan.reset_record()
+        for i in range(9):
+            ag.gemm_persistent(dA.data_ptr(), dBs[i % 3].data_ptr(), dCs[i % 3].data_ptr(), M, N, K, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        for i in range(3):
+            assert np.array_equal(dCs[i].cpu().numpy().astype(np.float64), og.gemm_blocked(A, Bs[i]))
+        owner, count = plan.tile_record()
+        assert (count == 9).all()
 
 
 def test_in_memory_splitk_integer_exact_packed_and_rowmajor():
