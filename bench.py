@@ -51,51 +51,100 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock, power and throttle reasons while the measurements run: NVML polled from a thread
+    about once a millisecond (reading only), or `nvidia-smi -lms 20` when NVML cannot be loaded.  mark(name)
+    opens a named window, summary(name) gives the median clock and the reasons seen inside it."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.marks, self.stop_flag = index, [], None, {}, False
+        self.nvml = None
+        self.sm_max = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = None
+            try:
+                import torch
+                uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+            except Exception:
+                pass
+            h = None
+            if uuid:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+                except Exception:
+                    h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self.nvml = (pynvml, h)
+            threading.Thread(target=self._poll_nvml, daemon=True).start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            threading.Thread(target=self._read, daemon=True).start()
+            threading.Thread(target=self._read_smi, daemon=True).start()
         except OSError:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append((time.time(), [f.strip() for f in line.split(",")]))
-
-    def mark(self):
-        """Start of the timed region: only samples taken after this count."""
-        self.t_mark = time.time()
-
-    def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        t_end = time.time()
-        time.sleep(0.1)
-        self.proc.terminate()
-        mhz, mx, reasons = [], None, set()
-        for t, r in self.rows:
-            if t < getattr(self, "t_mark", 0.0) or t > t_end + 0.05:
-                continue
+    def _poll_nvml(self):
+        pynvml, h = self.nvml
+        names = (("hw_slowdown", pynvml.nvmlClocksEventReasonHwSlowdown),
+                 ("hw_thermal_slowdown", pynvml.nvmlClocksEventReasonHwThermalSlowdown),
+                 ("sw_thermal_slowdown", pynvml.nvmlClocksEventReasonSwThermalSlowdown),
+                 ("sw_power_cap", pynvml.nvmlClocksEventReasonSwPowerCap))
+        while not self.stop_flag:
             try:
-                mhz.append(float(r[0]))
-                mx = float(r[1])
+                mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                mask = int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                watts = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+                self.rows.append((time.time(), mhz, watts, [n for n, bit in names if mask & bit]))
+            except Exception:
+                pass
+            time.sleep(0.001)
+
+    def _read_smi(self):
+        for line in self.proc.stdout:
+            r = [f.strip() for f in line.split(",")]
+            try:
+                mhz, self.sm_max, watts = float(r[0]), float(r[1]), float(r[2])
             except (ValueError, IndexError):
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(mhz)}
+            reasons = [n for n, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7])
+                       if v.lower().startswith("active")]
+            self.rows.append((time.time(), mhz, watts, reasons))
+
+    def mark(self, name="timed"):
+        """Open the window `name` (closed by close(name))."""
+        self.marks[name] = [time.time(), None]
+
+    def close(self, name="timed"):
+        self.marks[name][1] = time.time()
+
+    def summary(self, name="timed") -> dict:
+        if self.nvml is None and self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["clock sampling unavailable"], "samples": 0}
+        t0, t1 = self.marks.get(name, [0.0, None])
+        t1 = t1 if t1 is not None else time.time()
+        rows = [r for r in self.rows if t0 <= r[0] <= t1 + 0.002]
+        reasons = sorted({x for r in rows for x in r[3]})
+        mhz = [r[1] for r in rows]
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": self.sm_max, "reasons": reasons,
+                "samples": len(mhz), "power_w_median": float(np.median([r[2] for r in rows])) if rows else None,
+                "source": "nvml, 1 ms" if self.nvml else "nvidia-smi, 20 ms"}
+
+    def stop(self):
+        self.stop_flag = True
+        if self.proc is not None:
+            self.proc.terminate()
 
 
 def oracle_sample(A, B, rows=None, cols=N, target_s=15.0):
@@ -111,6 +160,134 @@ def oracle_sample(A, B, rows=None, cols=N, target_s=15.0):
     blk = og.gemm_block(A, B, 0, rows, 0, cols)
     dt = time.time() - t0
     return blk, dt, 2.0 * rows * cols * K, og.num_threads()
+
+
+def time_queued(torch, fn, warmup=4, iters=24, batches=3):
+    """Median GPU time per call in ms.  The calls of a batch are queued behind a device-side blocker, so that host-side
+    launch cost is not on the clock (the kernels here take tens of microseconds), and bracketed by one event pair."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    s = torch.cuda.current_stream()
+    out = []
+    for _ in range(batches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(2e7))
+        e0.record(s)
+        for _ in range(iters):
+            fn()
+        e1.record(s)
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1) / iters)
+    return float(np.median(out))
+
+
+def decode_section(ag, inputs, torch, topo, peaks, sampler):
+    """The HBM-bound workload: M = 16, N = K = 8192 (weights 128 MiB, read once per call), 128-column units x 16
+    k-splits on all SMs, split-K by reductions in memory, four weight matrices in rotation so that no call finds its
+    weights in L2, calls queued back to back with overlap_launches.  Die-local packed weights under the die-compact
+    plan, the same packed weights under the deliberately remote plan, and row-major weights under the oblivious and
+    die-compact plans; C of the first call is checked against the fp64 oracle."""
+    from oracle import gemm as og
+    Md, Nd, Kd, ksp, n_buf = 16, 8192, 8192, 16, 4
+    A_bits = inputs.uniform_bf16(Md, Kd, inputs.DEFAULT_SEED)
+    B_bits = [inputs.uniform_bf16(Kd, Nd, inputs.DEFAULT_SEED + 1 + i) for i in range(n_buf)]
+    dev = lambda bits: torch.from_numpy(bits.view(np.int16).copy()).cuda()
+    dA = dev(A_bits)
+    dBs = [dev(b) for b in B_bits]
+    dC = torch.empty((Md, Nd), dtype=torch.float32, device="cuda")
+    algo_bytes = Kd * Nd * 2 + Md * Kd * 2 + Md * Nd * 4
+    kw = dict(M=Md, N=Nd, K=Kd, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=1, overlap_launches=1)
+    plan_local = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+    plan_obl = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
+    dst_bytes = 2 * Kd * Nd * 2 + (8 << 20)
+    dsts, packs = [], []
+    for i in range(n_buf):
+        dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+        amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+        packs.append((ag.pack_weights(dBs[i].data_ptr(), Kd, Nd, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
+        dsts.append(dst)
+    bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packs[0][0].page_table())
+    plan_remote = ag.sched_build(topo, packs[0][1], topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
+    # parity of what is timed: first call of the packed die-local arm and of the row-major oblivious arm
+    want = og.gemm_blocked(A_bits, B_bits[0])
+    err = {}
+    for name, call in (("packed_die_local", lambda: ag.gemm_persistent_packed(dA.data_ptr(), packs[0][0], dC.data_ptr(), Md, Nd, Kd, plan_local)),
+                       ("rowmajor_oblivious", lambda: ag.gemm_persistent(dA.data_ptr(), dBs[0].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan_obl))):
+        dC.fill_(float("nan"))
+        call()
+        torch.cuda.synchronize()
+        got = dC.cpu().numpy().astype(np.float64)
+        err[name] = {"max_abs": float(np.abs(got - want).max()), "rel_fro": float(np.linalg.norm(got - want) / np.linalg.norm(want))}
+    gbs, launches0 = {}, ag.kernel_launch_count()
+    sampler.mark("decode")
+    arms = (("packed_die_local", plan_local, True), ("packed_remote", plan_remote, True),
+            ("rowmajor_oblivious", plan_obl, False), ("rowmajor_die_compact", plan_local, False))
+    for _ in range(2):                                    # two passes so that the arms share the clock drift
+        for name, plan, packed in arms:
+            state = {"i": 0}
+
+            def run():
+                i = state["i"] % n_buf
+                state["i"] += 1
+                if packed:
+                    ag.gemm_persistent_packed(dA.data_ptr(), packs[i][0], dC.data_ptr(), Md, Nd, Kd, plan)
+                else:
+                    ag.gemm_persistent(dA.data_ptr(), dBs[i].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan)
+            ms = time_queued(torch, run)
+            if plan.last_status() != ag.AG_OK:
+                raise RuntimeError("decode arm " + name + ": " + ag.strerror(plan.last_status()))
+            gbs.setdefault(name, []).append(algo_bytes / (ms * 1e-3) / 1e9)
+    sampler.close("decode")
+    gbs = {n: float(np.median(v)) for n, v in gbs.items()}
+    best = gbs["packed_die_local"]
+    return {"workload": f"GEMM M={Md} N=K={Nd} bf16, fp32 out, 128-col units x {ksp} k-splits (in-memory reductions), all {topo.n_sm} SMs, "
+                        f"{n_buf} rotating weight matrices (512 MiB > L2), launches queued back to back, overlap_launches",
+            "gbs": gbs, "us_per_call": {n: algo_bytes / v / 1e3 for n, v in gbs.items()},
+            "local_over_remote": gbs["packed_die_local"] / gbs["packed_remote"],
+            "aware_over_oblivious": gbs["packed_die_local"] / gbs["rowmajor_oblivious"],
+            "group_free_bit": packs[0][0].group_free_bit(),
+            "oracle_error_on_c": err,
+            "gpu_launches": int(ag.kernel_launch_count() - launches0),
+            "clocks": sampler.summary("decode"),
+            "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
+                         "traffic": None, "kernel": "k_gemm_skinny<16, packed>", "algorithmic_bytes": algo_bytes,
+                         "peak_source": f"{peaks['source']} copy bandwidth"}}
+
+
+def subset_section(ag, inputs, torch, topo, sampler, budget=64, n_subsets=8):
+    """Equal-size SM sets: dense 4096^3 on `budget` SMs - seeded random subsets, the lowest ids, the die-compact and
+    the GPC-spread set - all on the one-block kernel (128 x 256 tiles), so that only the placement differs."""
+    Ms = Ns = Ks = 4096
+    A, B = inputs.gemm_inputs(Ms, Ns, Ks)
+    dev = lambda bits: torch.from_numpy(bits.view(np.int16).copy()).cuda()
+    dA, dB = dev(A), dev(B)
+    dC = torch.empty((Ms, Ns), dtype=torch.float32, device="cuda")
+    flops = 2.0 * Ms * Ns * Ks
+    kw = dict(M=Ms, N=Ns, K=Ks, raster_group=4)
+    plans = {f"random_{s}": ag.sched_build(topo, None, budget, ag.make_policy(kind=ag.AG_OBLIVIOUS, seed=s, **kw))
+             for s in range(1, n_subsets + 1)}
+    plans["lowest_ids"] = ag.sched_build(topo, None, budget, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
+    plans["die_compact"] = ag.sched_build(topo, None, budget, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+    plans["gpc_spread"] = ag.sched_build(topo, None, budget, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, **kw))
+    acc = {n: [] for n in plans}
+    sampler.mark("subsets")
+    for _ in range(3):
+        for n, plan in plans.items():
+            acc[n].append(time_queued(torch, lambda: ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), Ms, Ns, Ks, plan),
+                                      warmup=1, iters=4, batches=1))
+    sampler.close("subsets")
+    res = {n: flops / (float(np.median(v)) * 1e-3) / 1e12 for n, v in acc.items()}
+    for n, plan in plans.items():
+        if plan.last_status() != ag.AG_OK:
+            raise RuntimeError("subset " + n + ": " + ag.strerror(plan.last_status()))
+    rnd = [res[f"random_{s}"] for s in range(1, n_subsets + 1)]
+    return {"workload": f"dense GEMM {Ms}^3 bf16 on {budget} SMs, 128x256 tiles, one block per tile for every set",
+            "random_subsets_tflops": rnd, "random_max_over_min": max(rnd) / min(rnd), "random_median": float(np.median(rnd)),
+            "lowest_ids_tflops": res["lowest_ids"], "die_compact_tflops": res["die_compact"], "gpc_spread_tflops": res["gpc_spread"],
+            "die_compact_over_random_median": res["die_compact"] / float(np.median(rnd)),
+            "gpc_spread_over_random_median": res["gpc_spread"] / float(np.median(rnd)),
+            "clocks": sampler.summary("subsets")}
 
 
 def run_reference(args):
@@ -230,7 +407,7 @@ def main():
             step(plan)
         barrier()
         if sampler is not None:
-            sampler.mark()
+            sampler.mark("timed")
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         launches0 = ag.kernel_launch_count()
         evs[0].record(stream)
@@ -264,6 +441,9 @@ def main():
         for _ in range(args.warmup):
             calls[n]()
     barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    sampler.mark("rotation")
     rounds, per_round = 6, max(2, min(args.steps, 60) // 6)
     for _ in range(rounds):
         for n in names:
@@ -274,15 +454,31 @@ def main():
                 evs[i + 1].record(stream)
             torch.cuda.synchronize()
             per_policy[n] += [evs[i].elapsed_time(evs[i + 1]) for i in range(per_round)]
+    sampler.close("rotation")
     side = {n: FLOPS / (float(np.median(v)) * 1e-3) / 1e12 for n, v in per_policy.items()}
     cublas_tflops = side.pop("context_cublas_bf16_out", None)
     calls.clear()
-    sampler = ClockSampler(local)
-    sampler.start()
     total_ms, per, launches = timed(plans["affinity"], args.steps, args.warmup, sampler)
-    clocks = sampler.stop()
+    sampler.close("timed")
+    clocks = sampler.summary("timed")
     value, ms_step = replicas.job_throughput(total_ms / args.steps, FLOPS, "cuda")
     value /= 1e12
+    # The 1 kW power cap decides the clock, and the clock the throughput: beside the K timed steps, the same step is
+    # run back to back for at least half a second (the power state settles within ~100 ms) with the clock sampled
+    # throughout, and every throughput is also given per GHz of median SM clock.
+    n_sus = max(args.steps, int(0.5 / max(total_ms / args.steps * 1e-3, 1e-6)) + 1)
+    sampler.mark("sustained")
+    sus_ms, _, _ = timed(plans["affinity"], n_sus, 0, None)
+    sampler.close("sustained")
+    sus_clocks = sampler.summary("sustained")
+    sustained = {"tflops": FLOPS / (sus_ms / n_sus * 1e-3) / 1e12, "steps": n_sus, "seconds": sus_ms * 1e-3, "clocks": sus_clocks}
+    if sus_clocks.get("sm_mhz"):
+        sustained["tflops_per_sm_ghz"] = sustained["tflops"] / (sus_clocks["sm_mhz"] / 1e3)
+    rot_clocks = sampler.summary("rotation")
+
+    decode = decode_section(ag, inputs, torch, topo, peaks, sampler)
+    subsets = subset_section(ag, inputs, torch, topo, sampler)
+    sampler.stop()
 
     # ---- end to end through the same call with host buffers.  Every step copies its A and B from pinned host
     # memory (256 MiB), runs the GEMM and copies C back (256 MiB).  The steps are pipelined over three streams
@@ -348,7 +544,14 @@ def main():
                    "l2": "inputs+output 512 MiB > 126 MB L2, no flush between iterations",
                    "replicas": "independent per GPU" if world > 1 else "single GPU"},
         "policies_tflops": side,
+        "policies_clocks": rot_clocks,
+        "policies_tflops_per_sm_ghz": ({n: v / (rot_clocks["sm_mhz"] / 1e3) for n, v in side.items()} if rot_clocks.get("sm_mhz") else None),
+        "packed_b_group_free_bit": packed_b.group_free_bit(),
         "context_cublas_bf16_out_tflops_same_run": cublas_tflops,
+        "value_per_sm_ghz": (value / (clocks["sm_mhz"] / 1e3)) if clocks.get("sm_mhz") else None,
+        "sustained": sustained,
+        "decode": decode,
+        "sm_subsets": subsets,
         "aware_over_oblivious_raster": side["affinity"] / side["oblivious_raster"],
         "die_sm_count": list(topo.die_sm_count), "gpc_sm_count": list(topo.gpc_sm_count[:topo.n_gpc]),
         "setup_s": {"topo_discover": t_topo, "affinity_probe": t_aff, "sched_build_x5": t_plan, "probe_pack_plan_b": t_pack},

@@ -25,10 +25,18 @@ namespace ag {
 constexpr int P_BM = 128;        // rows per block (256 per pair)
 constexpr int P_BN = 256;        // columns of the unit
 constexpr int P_BNH = 128;       // B columns held by one block
-constexpr int P_BK = 64;
-constexpr int P_STAGES = 6;
-constexpr int P_A_BYTES = P_BM * P_BK * 2;     // 16 KB
-constexpr int P_B_BYTES = P_BK * P_BNH * 2;    // 16 KB
+constexpr int P_BK = 64;         // k-slab
+// A stage holds two k-slabs (64 KB per block, 8 MMAs): the thread that issues the MMAs pays a fixed cost per stage
+// (barrier wait, fence, commit) that four MMAs did not cover.  A warp gets only about two bulk copies in flight,
+// so each of the three stages has its own copy-issuing warp (A and B of its stage: 2 x 32 KB).
+constexpr int P_SLABS = 2;
+constexpr int P_STAGES = 3;
+constexpr int P_NPROD = P_STAGES;
+constexpr int P_THREADS = (2 + kEpiWarps + P_NPROD) * 32;   // scheduler, MMA issuer, epilogue warps, copy warps
+constexpr int P_A_SLAB = P_BM * P_BK * 2;      // 16 KB
+constexpr int P_B_SLAB = P_BK * P_BNH * 2;     // 16 KB
+constexpr int P_A_BYTES = P_SLABS * P_A_SLAB;  // 32 KB
+constexpr int P_B_BYTES = P_SLABS * P_B_SLAB;  // 32 KB
 constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES;
 constexpr int P_EPI_BUF = 32 * 32 * 4;
 constexpr int P_EPI_BYTES = kEpiWarps * 2 * P_EPI_BUF;
@@ -159,7 +167,7 @@ struct PairSource {
 // PACKED_B: the B panels come from die-local 4 KB pages ([128 columns x 16 k], no-swizzle core-matrix order,
 // see ag_pack_weights): tm_b then describes the packed buffer as [chunk][16][128] and a page is one box.
 template <bool PACKED_B>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(P_THREADS, 1)
 k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                        const __grid_constant__ CUtensorMap tm_b2, const __grid_constant__ CUtensorMap tm_c,
                        const PersistParams p, const int32_t* __restrict__ page_table, const int pages_per_block,
@@ -192,7 +200,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&ctl->sched_full[i]), 1);
-            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps + P_NPROD);
         }
         mbar_init(smem_u32(&ctl->mma_drain), 1);
         mbar_fence_init();
@@ -221,96 +229,126 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 
     if (active) {
         if (warp == 0) {
-            // ------------------------------------------------ scheduler + TMA producer.  Every lane walks the same
-            // unit sequence; lane 0 waits and issues.  For packed B the 32 lanes fetch the page-table entries of
-            // the next eight k-slabs with one load each.
+            // ------------------------------------------------ scheduler: hands the pair's unit sequence to the other roles
             PairSource src(p, slot, peer_slot, gv);
-            uint32_t it = 0, kit = 0;
             int ok = 1;
-            while (ok) {
+            for (uint32_t it = 0; ok; ++it) {
                 const int u = src.next();
                 if (lane == 0) {
                     const int r = it % kRing;
-                    if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                    if (!mbar_wait_idle(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                         report_timeout(p, 1);
                         ok = 0;
                     } else {
                         ctl->ring[r] = u;
-                    if (p.unit_times && u >= 0) p.unit_times[2 * u] = globaltimer_ns();
+                        if (p.unit_times && u >= 0) p.unit_times[2 * u] = globaltimer_ns();
                         mbar_arrive(smem_u32(&ctl->sched_full[r]));
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
-                ++it;
+                if (u < 0) break;
+            }
+        } else if (warp >= 2 + kEpiWarps) {
+            // ------------------------------------------------ copies: warp pw fills stage pw (its A and its B part).  For
+            // packed B the lanes look up the chunks of the stage's pages one stage ahead of the copies.
+            const int pw = warp - (2 + kEpiWarps);
+            const uint32_t sa = base + pw * P_STAGE_BYTES, sb_addr = sa + P_A_BYTES;
+            const uint32_t bar_own = smem_u32(&ctl->full[pw]);
+            const uint32_t bar_leader = map_to_cta(bar_own, 0);        // the leader's barrier counts the bytes of both blocks
+            const uint32_t bar_empty = smem_u32(&ctl->empty[pw]);
+            uint32_t q_run = 0;      // stages (over the whole run of this pair) before the current unit
+            int ok = 1;
+            for (uint32_t it = 0; ok; ++it) {
+                const int r = it % kRing;
+                int u = -1;
+                if (lane == 0) {
+                    if (!mbar_wait_idle(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                        report_timeout(p, 8);
+                        ok = 0;
+                    } else {
+                        u = ctl->ring[r];
+                        mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                u = __shfl_sync(0xffffffffu, u, 0);
                 if (!ok || u < 0) break;
                 const int tm = u / p.tiles_n, tn = u % p.tiles_n;
                 const int grp = gv.rows ? tn / gv.tiles_per_group : 0;        // expert of this unit column
                 const int tl = gv.rows ? tn - grp * gv.tiles_per_group : tn;  // unit column inside the expert
                 const CUtensorMap* ma = gv.rows ? &gv.tm_a[grp] : &tm_a;
                 const CUtensorMap* mb = (gv.rows && !PACKED_B) ? &gv.tm_b[grp] : &tm_b;
-                // Packed B: the units of one raster group that share a column panel start their k loop at
-                // different k-slabs (the sum over k does not care where it starts), so that at any moment they
-                // read different 4 KB pages: a page sits in few L2 slices, and eight pairs asking for the same
-                // page at once queue up there.
-                const int n_blk = (p.kslabs_total + 7) / 8;
-                const int rot = PACKED_B ? ((tm & 7) * max(1, n_blk / 8)) % n_blk : 0;
-                for (int b8 = 0; b8 < n_blk && ok; ++b8) {
-                    const int sb = ((b8 + rot) % n_blk) * 8;
-                    int my_page = 0;
-                    if (PACKED_B) {
-                        if (quad_base) {   // grouped pages: one entry per k-slab (bit 30 = class of the group)
-                            if (lane < 8 && sb + lane < p.kslabs_total)
-                                my_page = quad_base[(size_t)(tn * 2 + (int)rank) * (pages_per_block / 4) + sb + lane];
+                const int n_st = (p.kslabs_total + P_SLABS - 1) / P_SLABS;
+                // Packed B: the units of one raster group that share a column panel start their k loop at different
+                // stages (the sum over k does not care where it starts), so that at any moment they read different
+                // 4 KB pages: a page sits in few L2 slices, and eight pairs asking for the same page at once queue up there.
+                const int rot = PACKED_B ? ((tm & 7) * max(1, n_st / 8)) % n_st : 0;
+                const int i0 = (pw + P_NPROD - (int)(q_run % P_NPROD)) % P_NPROD;   // this warp's first stage of the unit
+                uint32_t ph = (((q_run + i0) / P_STAGES) & 1) ^ 1;                  // parity of "stage is free"
+                auto table_entry = [&](int i) -> int {
+                    if (!PACKED_B || i >= n_st) return 0;
+                    const int s = ((i + rot) % n_st) * P_SLABS;
+                    const size_t blk = (size_t)(tn * 2 + (int)rank);
+                    if (quad_base) return (lane < P_SLABS && s + lane < p.kslabs_total) ? quad_base[blk * (pages_per_block / 4) + s + lane] : 0;
+                    return (lane < 4 * P_SLABS && s + (lane >> 2) < p.kslabs_total) ? page_table[blk * pages_per_block + (size_t)s * 4 + lane] : 0;
+                };
+                int next_entry = table_entry(i0);
+                for (int i = i0; i < n_st && ok; i += P_NPROD) {
+                    const int entry = next_entry;
+                    next_entry = table_entry(i + P_NPROD);
+                    const int s = ((i + rot) % n_st) * P_SLABS;          // first k-slab of this stage
+                    const int ns = min(P_SLABS, p.kslabs_total - s);
+                    if (lane == 0) {
+                        if (!mbar_wait(bar_empty, ph, abort_flag, limit)) {
+                            report_timeout(p, 2);
+                            ok = 0;
                         } else {
-                            const int pg = sb * 4 + lane;
-                            if (pg < p.kslabs_total * 4) my_page = page_table[(size_t)(tn * 2 + (int)rank) * pages_per_block + pg];
-                        }
-                    }
-                    const int se = min(p.kslabs_total, sb + 8);
-                    for (int s = sb; s < se; ++s, ++kit) {
-                        const int st = kit % P_STAGES;
-                        // the leader's barrier counts the bytes of both blocks
-                        const uint32_t bar_leader = map_to_cta(smem_u32(&ctl->full[st]), 0);
-                        const uint32_t sa = base + st * P_STAGE_BYTES, sb_addr = sa + P_A_BYTES;
-                        if (lane == 0) {
-                            if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / P_STAGES) & 1) ^ 1, abort_flag, limit)) {
-                                report_timeout(p, 2);
-                                ok = 0;
+                            // row-major operands always arrive as whole boxes (rows past K are zeros)
+                            if (leader) mbar_expect_tx(bar_own, 2 * (P_A_BYTES + (PACKED_B ? ns * P_B_SLAB : P_B_BYTES)));
+                            if (p.a_blocks) {
+                                tma_load_3d_pair(sa, ma, bar_leader, 0, tm * 2 * P_BM + (int)rank * P_BM, s);
                             } else {
-                                if (leader) mbar_expect_tx(smem_u32(&ctl->full[st]), 2 * P_STAGE_BYTES);
                                 tma_load_2d_pair(sa, ma, bar_leader, s * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
-                                if (!PACKED_B) {
-                                    if (p.b_blocks) {
-                                        // both 64-column blocks of this block's half with one copy
-                                        tma_load_3d_pair(sb_addr, mb, bar_leader, 0, s * P_BK, tl * 4 + (int)rank * 2);
-                                    } else {
-                                        tma_load_2d_pair(sb_addr, mb, bar_leader, tl * P_BN + (int)rank * P_BNH, s * P_BK);
-                                        tma_load_2d_pair(sb_addr + P_BK * 128, mb, bar_leader, tl * P_BN + (int)rank * P_BNH + 64, s * P_BK);
-                                    }
+                                tma_load_2d_pair(sa + P_A_SLAB, ma, bar_leader, (s + 1) * P_BK, tm * 2 * P_BM + (int)rank * P_BM);
+                            }
+                            if (!PACKED_B) {
+                                if (p.b_blocks) {
+                                    // both 64-column blocks of this block's half with one copy
+                                    tma_load_3d_pair(sb_addr, mb, bar_leader, 0, s * P_BK, tl * 4 + (int)rank * 2);
+                                } else {
+                                    tma_load_2d_pair(sb_addr, mb, bar_leader, tl * P_BN + (int)rank * P_BNH, s * P_BK);
+                                    tma_load_2d_pair(sb_addr + P_B_BYTES / 2, mb, bar_leader, tl * P_BN + (int)rank * P_BNH + 64, s * P_BK);
                                 }
                             }
                         }
-                        ok = __shfl_sync(0xffffffffu, ok, 0);
-                        if (!ok) break;
-                        if (PACKED_B && quad_base) {
-                            // the slab's four pages are one group of same-die chunks: one strided box
-                            const int q0 = __shfl_sync(0xffffffffu, my_page, s - sb);
-                            if (lane == 0)
-                                tma_load_5d_pair(sb_addr, (q0 >> 30) ? &tm_b2 : &tm_b, bar_leader, 0, 0, 0, 0, q0 & 0x3fffffff);
-                        } else if (PACKED_B) {
-                            // four lanes issue the four page copies of the slab in one instruction: a single
-                            // thread gets only one bulk copy out every ~150 cycles
-                            const int page = __shfl_sync(0xffffffffu, my_page, (s - sb) * 4 + (lane & 3));
-                            if (lane < 4) tma_load_3d_pair(sb_addr + lane * 4096, &tm_b, bar_leader, 0, 0, page);
-                        }
                     }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    if (PACKED_B && quad_base) {
+                        // a slab's four pages are one group of same-die chunks: one strided box each
+                        if (lane < ns) tma_load_5d_pair(sb_addr + lane * P_B_SLAB, (entry >> 30) ? &tm_b2 : &tm_b, bar_leader, 0, 0, 0, 0, entry & 0x3fffffff);
+                    } else if (PACKED_B) {
+                        // one lane per 4 KB page, all in one instruction
+                        if (lane < 4 * ns) tma_load_3d_pair(sb_addr + lane * 4096, &tm_b, bar_leader, 0, 0, entry);
+                    }
+                    ph ^= 1;     // the next stage this warp fills is the same buffer, one round later
                 }
+                q_run += (uint32_t)n_st;
             }
         } else if (warp == 1) {
             if (lane == 0) {
                 // ------------------------------------------------ MMA issuer (leader) / ring consumer (peer)
                 constexpr uint32_t idesc = make_idesc_bf16(2 * P_BM, P_BN, 0, PACKED_B ? 0 : 1);
-                uint32_t kit = 0, tile_it = 0;
+                // descriptors without their start address.  A: K-major, 128-byte swizzle, 8 rows 1 KB apart.  B: row-major
+                // source = N-major, 128-byte swizzle, the two 64-column blocks half the B part apart (LBO), 8 k rows 1 KB
+                // apart (SBO); packed page = K-major, no swizzle, 16-byte k chunks 128 B apart (LBO), 8-column groups
+                // 256 B apart (SBO).  The address field counts 16-byte units and never carries out of its 14 bits.
+                const uint64_t da_t = make_smem_desc(0, 16, 1024, 2);
+                const uint64_t db_t = PACKED_B ? make_smem_desc(0, 128, 256, 0) : make_smem_desc(0, P_B_BYTES / 2, 1024, 2);
+                constexpr uint32_t kAStep = 32u >> 4, kASlabStep = (uint32_t)P_A_SLAB >> 4;
+                constexpr uint32_t kBStep = (PACKED_B ? 4096u : 2048u) >> 4;
+                const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+                uint32_t st = 0, ph = 0, tile_it = 0;
                 bool ok = true;
                 for (uint32_t it = 0; ok; ++it) {
                     const int r = it % kRing;
@@ -329,25 +367,33 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                     }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * P_BN;
-                    for (int s = 0; s < p.kslabs_total; ++s, ++kit) {
-                        const int st = kit % P_STAGES;
-                        if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / P_STAGES) & 1, abort_flag, limit)) {
+                    // the stages arrive in the order the copy warps walk them; with packed B that order is rotated,
+                    // but how many k-slabs a stage holds depends only on whether it is the unit's last one in k
+                    const int n_st = (p.kslabs_total + P_SLABS - 1) / P_SLABS;
+                    const int tm = u / p.tiles_n;
+                    const int rot = PACKED_B ? ((tm & 7) * max(1, n_st / 8)) % n_st : 0;
+                    const bool odd_tail = (p.kslabs_total & 1) != 0;
+                    for (int i = 0; i < n_st; ++i) {
+                        if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
                             report_timeout(p, 5);
                             ok = false;
                             break;
                         }
                         tc_fence_after();
-                        const uint32_t sa = base + st * P_STAGE_BYTES, sb = sa + P_A_BYTES;
+                        const uint32_t sa = base + st * P_STAGE_BYTES;
+                        const uint64_t da = da_t | (uint64_t)(sa >> 4);
+                        const uint64_t db = db_t | (uint64_t)((sa + P_A_BYTES) >> 4);
+                        tc_mma_f16_pair(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
 #pragma unroll
-                        for (int k4 = 0; k4 < P_BK / 16; ++k4) {
-                            const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
-                            // B: row-major source = N-major, 128-byte swizzle; packed page = K-major, no swizzle,
-                            // 16-byte k chunks 128 B apart (LBO), 8-column groups 256 B apart (SBO)
-                            const uint64_t db = PACKED_B ? make_smem_desc(sb + k4 * 4096, 128, 256, 0)
-                                                         : make_smem_desc(sb + k4 * 2048, P_BK * 128, 1024, 2);
-                            tc_mma_f16_pair(d_tmem, da, db, idesc, (s > 0 || k4 > 0) ? 1u : 0u);
+                        for (int k4 = 1; k4 < P_BK / 16; ++k4) tc_mma_f16_pair(d_tmem, da + k4 * kAStep, db + k4 * kBStep, idesc, 1u);
+                        const bool half = odd_tail && ((i + rot) % n_st) == n_st - 1;   // the stage that holds the last, single k-slab
+                        if (!half) {
+#pragma unroll
+                            for (int k4 = 0; k4 < P_BK / 16; ++k4)
+                                tc_mma_f16_pair(d_tmem, da + kASlabStep + k4 * kAStep, db + (4 + k4) * kBStep, idesc, 1u);
                         }
-                        tc_commit_pair(smem_u32(&ctl->empty[st]));
+                        tc_commit_pair(empty0 + st * 8);
+                        if (++st == P_STAGES) { st = 0; ph ^= 1; }
                     }
                     if (!ok) break;
                     tc_commit_pair(smem_u32(&ctl->tmem_full[acc]));
@@ -366,7 +412,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
             uint32_t tile_it = 0, chunk_it = 0;
             for (uint32_t it = 0;; ++it) {
                 const int r = it % kRing;
-                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                if (!mbar_wait_warp(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
                     if (lane == 0) report_timeout(p, 6);
                     break;
                 }
@@ -376,7 +422,7 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 if (u < 0) break;
                 const int tm = u / p.tiles_n, tn = u % p.tiles_n;
                 const uint32_t acc = tile_it & 1;
-                if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
+                if (!mbar_wait_warp(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
                     if (lane == 0) report_timeout(p, 7);
                     break;
                 }
@@ -471,10 +517,12 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     if (grp) {
         if (W) { plan->tm_b = W->quad_free_bit >= 0 ? W->tm_quad[0] : W->tm_pages; plan->tm_b_ptr = nullptr; }
     } else if (plan->tm_a_ptr != A || plan->tm_b_ptr != b_key || plan->tm_c_ptr != Cout) {
-        if (!encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)) return AG_ERR_CUDA;
+        if (!(K % P_BK == 0 ? encode_a_slabs(&plan->tm_a, A, M, K, P_BM, P_SLABS)
+                            : encode_2d(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, M, K, P_BK, P_BM)))
+            return AG_ERR_CUDA;
         if (W) plan->tm_b = W->quad_free_bit >= 0 ? W->tm_quad[0] : W->tm_pages;
-        else if (N % 64 == 0) { if (!encode_b_blocks(&plan->tm_b, B, K, N, P_BK, 2)) return AG_ERR_CUDA; }
-        else if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_BK)) return AG_ERR_CUDA;
+        else if (N % 64 == 0) { if (!encode_b_blocks(&plan->tm_b, B, K, N, P_SLABS * P_BK, 2)) return AG_ERR_CUDA; }
+        else if (!encode_2d(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, K, N, 64, P_SLABS * P_BK)) return AG_ERR_CUDA;
         if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
         plan->tm_a_ptr = A; plan->tm_b_ptr = b_key; plan->tm_c_ptr = Cout;
     }
@@ -488,6 +536,7 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
     PersistParams gp = make_persist_params(plan, M, N, K);
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
+    gp.a_blocks = (!grp && K % P_BK == 0) ? 1 : 0;
     GroupView gv;
     memset(&gv, 0, sizeof gv);
     if (grp) {
@@ -497,7 +546,7 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(n_sm);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(P_THREADS);
     cfg.dynamicSmemBytes = P_SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];

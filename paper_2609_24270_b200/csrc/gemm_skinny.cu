@@ -984,7 +984,7 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
         }
         if (B_list) {
             if (!B_list[g] || ((uintptr_t)B_list[g] & 15u)) { delete d; return AG_ERR_ARG; }
-            const int wk = dense ? SK_BK : SK_SLABS * SK_BK;   // k rows per weight copy of the kernel that will read them
+            const int wk = SK_SLABS * SK_BK;   // k rows per weight copy (both the decode-shaped and the block-pair kernel fill a stage with two k-slabs)
             const bool ok = d->w_blocks ? encode_b_blocks(&hw[g], B_list[g], K, N_expert, wk, 2)
                                         : encode_2d(&hw[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_list[g], K, N_expert, 64, wk);
             if (!ok) { delete d; return AG_ERR_CUDA; }
