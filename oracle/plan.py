@@ -429,6 +429,56 @@ def build_page_table_quads(page_die, amap: dict, free_bit: int, first: int = 0) 
     return table
 
 
+def _parity(x: int) -> int:
+    return bin(x).count("1") & 1
+
+
+def fit_page_constants(amap: dict, mask: int, first: int = 0) -> tuple[list[int], int]:
+    """The part of the partition hash (Section 6.1.2) that the in-page mask does not explain: one bit per 2 MiB
+    page (512 chunks; pages are counted in first + q, ``first`` = chunk index of the buffer's base inside its
+    page), taken as the majority of die ^ parity((first + q) & mask) over the page's chunks.  Returns the bits
+    and the number of chunks that disagree with parity ^ bit (noise, or a layout that is no such hash)."""
+    doc = amap["die_of_chunk"]
+    n = len(doc)
+    n_pages = (first + n + 511) // 512
+    ones = [0] * n_pages
+    cnt = [0] * n_pages
+    for q in range(n):
+        qa = first + q
+        ones[qa >> 9] += int(doc[q]) ^ _parity(qa & mask)
+        cnt[qa >> 9] += 1
+    bits = [1 if 2 * ones[i] > cnt[i] else 0 for i in range(n_pages)]
+    bad = sum(1 for q in range(n) if (int(doc[q]) ^ _parity((first + q) & mask)) != bits[(first + q) >> 9])
+    return bits, bad
+
+
+def page_from_hash(j: int, P: int, mask: int, c_bits, first: int = 0) -> int:
+    """Eq. 1 of the remapping appendix in closed form: logical page j of the view of die P is the chunk of the
+    aligned pair (2j, 2j+1) that the hash places on die P,
+        chunk = 2j + (parity((first + 2j) & mask) ^ c_page ^ P),
+    with the measured in-page mask standing for MASK and the per-2-MiB-page bit c_page for what the address bits
+    above bit 20 contribute.  Needs chunk-index bit 0 in the mask and an even ``first`` (aligned pairs)."""
+    qa = first + 2 * j
+    return 2 * j + (_parity(qa & mask) ^ int(c_bits[qa >> 9]) ^ P)
+
+
+def quad_group_from_hash(r: int, d: int, mask: int, c_bits, free_bit: int, first: int = 0) -> tuple[int, int]:
+    """The r-th group of four same-die chunks (see ``quad_groups``) of die d, in ascending order of its base chunk,
+    without a table: (base chunk q relative to the buffer, a).  With F = 2**free_bit, every run of four chunks
+    4t .. 4t+3 (absolute index first + q, bit ``free_bit`` clear) holds one group base per die - chunk 4t if
+    parity(4t & mask) ^ c_page is d (then a = 3), else chunk 4t + 1 (a = 1) - so the r-th group of either die sits in
+    the r-th such run at or after ``first``.  Needs bits 0 and 1 in the mask, bit ``free_bit`` out of it, and
+    ``first`` a multiple of 4."""
+    F = 1 << free_bit
+
+    def runs_below(x):                    # runs 4t..4t+3 with bit free_bit clear that start below absolute chunk x
+        return (x // (2 * F)) * (F // 4) + min(x % (2 * F), F) // 4
+    T = r + runs_below(first)
+    qa0 = (T // (F // 4)) * 2 * F + (T % (F // 4)) * 4
+    e = _parity(qa0 & mask) ^ int(c_bits[qa0 >> 9]) ^ d
+    return qa0 + e - first, (3 if e == 0 else 1)
+
+
 def page_die_from_plan(plan: dict, K: int, k_unit: int = 64) -> list[int]:
     """Die that owns every logical weight page (pc, k16), j = pc * ceil(K/16) + k16, pc = index of the
     128-column block: the die whose queue holds most of the units (tm, tn, ks) that read the page

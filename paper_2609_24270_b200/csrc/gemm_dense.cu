@@ -20,6 +20,10 @@ namespace ag {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int kEpiBufBytes = 32 * 32 * 4;
+// A warp gets only about two bulk copies in flight (measured), i.e. one stage (its A and its B box): the stages are
+// filled by D_NPROD warps in turn, so that all of them can be in flight together.
+constexpr int D_NPROD = 4;
+constexpr int D_THREADS = (2 + kEpiWarps + D_NPROD) * 32;   // scheduler, MMA issuer, epilogue warps, copy warps
 
 template <int BN>
 struct Cfg {
@@ -49,7 +53,7 @@ struct SharedCtl {
 };
 
 template <int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(D_THREADS, 1)
 k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_c, const PersistParams p) {
     using C = Cfg<BN>;
@@ -79,7 +83,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&ctl->sched_full[i]), 1);
-            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps + D_NPROD);
         }
         mbar_init(smem_u32(&ctl->mma_drain), 1);
         mbar_fence_init();
@@ -98,15 +102,14 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     const uint64_t limit = p.wait_limit_ns;
 
     if (warp == 0) {
-        // ------------------------------------------------ scheduler (warp-collective) + TMA producer (lane 0)
+        // ------------------------------------------------ scheduler (warp-collective): hands the unit ids to the other roles
         UnitSource src(p, slot, lane);
-        uint32_t it = 0, kit = 0;
         int ok = 1;
-        while (ok) {
+        for (uint32_t it = 0; ok; ++it) {
             const int u = src.next(lane);
             if (lane == 0) {
                 const int r = it % kRing;
-                if (!mbar_wait(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                if (!mbar_wait_idle(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 1);
                     ok = 0;
                 } else {
@@ -116,18 +119,35 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            ++it;
-            if (!ok || u < 0) break;
-            if (lane == 0) {
+            if (u < 0) break;
+        }
+    } else if (warp >= 2 + kEpiWarps) {
+        // ------------------------------------------------ copies: warp pw fills the stages pw, pw + D_NPROD, ... of the block's run
+        if (lane == 0) {
+            const int pw = warp - (2 + kEpiWarps);
+            uint32_t q_run = 0;      // stages before the current unit
+            bool ok = true;
+            for (uint32_t it = 0; ok; ++it) {
+                const int r = it % kRing;
+                if (!mbar_wait_idle(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    report_timeout(p, 8);
+                    break;
+                }
+                const int u = ctl->ring[r];
+                mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                if (u < 0) break;
                 const int ks = u % p.k_splits, t = u / p.k_splits;
                 const int tm = t / p.tiles_n, tn = t % p.tiles_n;
                 const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
                 const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
-                for (int s = s0; s < s1; ++s, ++kit) {
-                    const int st = kit % C::stages;
-                    if (!mbar_wait(smem_u32(&ctl->empty[st]), ((kit / C::stages) & 1) ^ 1, abort_flag, limit)) {
+                const int n = s1 - s0;
+                const int i0 = (pw + D_NPROD - (int)(q_run % D_NPROD)) % D_NPROD;
+                uint32_t st = (q_run + i0) % C::stages, ph = (((q_run + i0) / C::stages) & 1) ^ 1;   // stage, parity of "stage is free"
+                for (int i = i0; i < n; i += D_NPROD) {
+                    const int s = s0 + i;
+                    if (!mbar_wait(smem_u32(&ctl->empty[st]), ph, abort_flag, limit)) {
                         report_timeout(p, 2);
-                        ok = 0;
+                        ok = false;
                         break;
                     }
                     const uint32_t bar = smem_u32(&ctl->full[st]);
@@ -141,24 +161,27 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 #pragma unroll
                         for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tm_b, bar, tn * BN + j * 64, s * BK);
                     }
+                    st += D_NPROD;
+                    while (st >= (uint32_t)C::stages) { st -= C::stages; ph ^= 1; }
                 }
+                q_run += (uint32_t)n;
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-        }
-        if (!ok && lane == 0) {
-            // gave up: let the copies already in flight land before the block leaves
-            const uint32_t n_out = kit < (uint32_t)C::stages ? kit : (uint32_t)C::stages;
-            for (uint32_t j = 0; j < n_out; ++j) {
-                const uint32_t k2 = kit - 1 - j;
-                int dummy = 0;
-                mbar_wait(smem_u32(&ctl->full[k2 % C::stages]), (k2 / C::stages) & 1, &dummy, 2000000ull);
+            if (!ok) {
+                // gave up: linger (bounded) so that copies already in flight land before the block leaves
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (one lane)
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_bf16(BM, BN, 0, 1);
-            uint32_t kit = 0, tile_it = 0;
+            // descriptors without their start address.  A: K-major, 128-byte swizzle, 8-row groups 1024 B apart.
+            // B: N-major, 128-byte swizzle: 64-column blocks 8 KB apart (LBO), 8-k groups 1 KB apart (SBO).
+            const uint64_t da_t = make_smem_desc(0, 16, 1024, 2);
+            const uint64_t db_t = make_smem_desc(0, BK * 128, 1024, 2);
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            uint32_t st = 0, ph = 0, tile_it = 0;
             bool ok = true;
             for (uint32_t it = 0; ok; ++it) {
                 const int r = it % kRing;
@@ -179,24 +202,21 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int s = s0; s < s1; ++s, ++kit) {
-                    const int st = kit % C::stages;
-                    if (!mbar_wait(smem_u32(&ctl->full[st]), (kit / C::stages) & 1, abort_flag, limit)) {
+                for (int i = 0, n = s1 - s0; i < n; ++i) {
+                    if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
                         report_timeout(p, 5);
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t sa = s_stage + st * C::stage_bytes, sb = sa + C::a_bytes;
-                    // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart.
-                    // B: N-major, 128-byte swizzle: 64-column blocks 8 KB apart (LBO), 8-k groups 1 KB apart (SBO).
+                    const uint32_t sa = s_stage + st * C::stage_bytes;
+                    const uint64_t da = da_t | (uint64_t)(sa >> 4);
+                    const uint64_t db = db_t | (uint64_t)((sa + C::a_bytes) >> 4);
+                    tc_mma_f16(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k4 = 0; k4 < BK / 16; ++k4) {
-                        const uint64_t da = make_smem_desc(sa + k4 * 32, 16, 1024, 2);
-                        const uint64_t db = make_smem_desc(sb + k4 * 2048, BK * 128, 1024, 2);
-                        tc_mma_f16(d_tmem, da, db, idesc, (s > s0 || k4 > 0) ? 1u : 0u);
-                    }
-                    tc_commit(smem_u32(&ctl->empty[st]));  // slot reusable once these MMAs have read it
+                    for (int k4 = 1; k4 < BK / 16; ++k4) tc_mma_f16(d_tmem, da + k4 * 2, db + k4 * 128, idesc, 1u);
+                    tc_commit(empty0 + st * 8);  // slot reusable once these MMAs have read it
+                    if (++st == (uint32_t)C::stages) { st = 0; ph ^= 1; }
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&ctl->tmem_full[acc]));
@@ -217,7 +237,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         uint32_t tile_it = 0, chunk_it = 0;
         for (uint32_t it = 0;; ++it) {
             const int r = it % kRing;
-            if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+            if (!mbar_wait_warp(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 6);
                 break;
             }
@@ -228,7 +248,7 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             const int t = u / p.k_splits;
             const int tm = t / p.tiles_n, tn = t % p.tiles_n;
             const uint32_t acc = tile_it & 1;
-            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
+            if (!mbar_wait_warp(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 7);
                 break;
             }
@@ -344,7 +364,7 @@ static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream
         attr_err = cudaFuncSetAttribute(k_gemm_persistent<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes);
     });
     if (attr_err != cudaSuccess) return launch_failed(plan, attr_err);
-    k_gemm_persistent<BN><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, kThreads, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);
+    k_gemm_persistent<BN><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, D_THREADS, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);
     const cudaError_t le = cudaGetLastError();
     if (le != cudaSuccess) return launch_failed(plan, le);
     count_launch();

@@ -123,8 +123,15 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
     dst_bytes = 2 * K * N * 2 + (8 << 20)
     for b in budgets:
         plan_local = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
-        dsts, packs, packs_single = [], [], []
+        # the same budget taken as whole TPCs from the GPCs of both dies: each die then streams its own half of the
+        # weights from its own memory, and the set uses the memory of both dies
+        plan_spread = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, **kw))
+        dsts, packs, packs_single, packs_spread = [], [], [], []
         for i in range(n_buffers):                      # rotate buffers so that no launch finds its weights in L2
+            dst2 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            amap2 = ag.affinity_probe(dst2.data_ptr(), dst_bytes, topo)
+            packs_spread.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_spread, amap2, dst2.data_ptr(), dst_bytes), amap2))
+            dsts.append(dst2)
             dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
             amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
             packs.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
@@ -149,7 +156,8 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
         plan_obl = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
         out = {}
         for name, plan, pset in (("die_local", plan_local, packs), ("remote", plan_remote, packs),
-                                 ("die_local_single_pages", plan_local, packs_single)):
+                                 ("die_local_single_pages", plan_local, packs_single),
+                                 ("die_local_both_dies", plan_spread, packs_spread)):
             state = {"i": 0}
 
             def run():
@@ -159,7 +167,7 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
             ms = time_queued(run, warmup=4, iters=24)
             assert plan.last_status() == ag.AG_OK
             out[name] = algo_bytes / (ms * 1e-3) / 1e9
-        for name, plan in (("rowmajor_oblivious", plan_obl), ("rowmajor_die_compact", plan_local)):
+        for name, plan in (("rowmajor_oblivious", plan_obl), ("rowmajor_die_compact", plan_local), ("rowmajor_both_dies", plan_spread)):
             state = {"i": 0}
 
             def run2():
@@ -171,9 +179,9 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
         emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
                   sm_budget=b, overlap_launches=overlap, gbs=out, local_over_remote=out["die_local"] / out["remote"],
                   pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), local_set=sm_set_summary(topo, plan_local),
-                  remote_set=sm_set_summary(topo, plan_remote), algo_bytes=algo_bytes,
+                  remote_set=sm_set_summary(topo, plan_remote), both_dies_set=sm_set_summary(topo, plan_spread), algo_bytes=algo_bytes,
                   hbm_peak_measured_gbs=6534.1), fh)
-        del packs, packs_single, dsts
+        del packs, packs_single, packs_spread, dsts
 
 
 def _unit_die(plan):
