@@ -247,6 +247,7 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
             "local_over_remote": gbs["packed_die_local"] / gbs["packed_remote"],
             "aware_over_oblivious": gbs["packed_die_local"] / gbs["rowmajor_oblivious"],
             "group_free_bit": packs[0][0].group_free_bit(),
+            "closed_form_remap": packs[0][0].closed_form(),
             "oracle_error_on_c": err,
             "gpu_launches": int(ag.kernel_launch_count() - launches0),
             "clocks": sampler.summary("decode"),

@@ -347,6 +347,14 @@ ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, cons
 /*
  * ag_pack_weights_ex - ag_pack_weights / ag_pack_weights_grouped with options (G = 1: B_list holds one matrix).
  *   flags  bit 0: keep the one-page-per-copy layout even where groups of four pages are possible.
+ *          bit 1: always read the page tables in the kernel (do not use the closed form below).
+ * Closed form (Eq. 1 of the remapping appendix, page_phys = 2j + [parity((page_start + 2j) & MASK) xor P]): when the
+ * measured map is an exact XOR hash over the chunks in use - in-page mask from ag_affinity_fit_hash, one further bit
+ * per 2 MiB page, no chunk out of line - and the plan is decode-shaped, the pages of a work unit are consecutive in
+ * the view of its die and the chunk of every page (or the base of every group of four) follows from the unit's first
+ * position, the mask and the page bits.  ag_pack_weights recomputes every table entry that way; if all agree, the
+ * decode-shaped kernel computes page addresses instead of loading them (one word per unit and one bit per 2 MiB
+ * instead of one word per page or group).  Otherwise the tables stay in use.  ag_packed_closed_form reports which.
  * Grouped pages: when the map follows an XOR hash (ag_affinity_fit_hash) that uses chunk-index bits 0 and 1
  * and leaves some bit f in 2..8 out, the chunks {q, q+a, q+F, q+F+a} (F = 2^f; a = 3 for q = 0 mod 4, a = 1
  * for q = 1 mod 4; bit f of q clear) always sit on one die.  The four pages of a k-slab (of one 128-column block)
@@ -357,6 +365,10 @@ ag_status ag_pack_weights_ex(const void* const* B_list, int G, int K, int N_expe
                              const ag_affinity_map* amap, void* dst, size_t dst_bytes, uint32_t flags,
                              ag_packed_weights** out);
 ag_status ag_packed_info(const ag_packed_weights* w, int32_t* group_free_bit);
+/* *enabled = 1 when the kernels compute page addresses from the fitted hash; mask = the in-page mask; table_bytes /
+ * closed_bytes = device bytes of the lookup tables and of the closed form's data (any of the last three may be NULL). */
+ag_status ag_packed_closed_form(const ag_packed_weights* w, int32_t* enabled, uint32_t* mask, size_t* table_bytes,
+                                size_t* closed_bytes);
 /* Page table (host, cap entries): chunk index in dst of logical page (pc, k16) = pc * (K/16) + k16, pc = index
  * of the 128-column block; feed it to ag_operand_desc.page_table to build an affinity plan over the packed weights. */
 ag_status ag_packed_page_table(const ag_packed_weights* w, int32_t* out, size_t cap, size_t* n_pages);

@@ -26,7 +26,7 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_page_table",
+    "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
@@ -140,6 +140,7 @@ def lib() -> C.CDLL:
     L.ag_pack_weights.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, sz, C.POINTER(vp)]
     L.ag_pack_weights_ex.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, vp, vp, sz, C.c_uint32, C.POINTER(vp)]
     L.ag_packed_info.argtypes = [vp, C.POINTER(C.c_int32)]
+    L.ag_packed_closed_form.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_uint32), C.POINTER(sz), C.POINTER(sz)]
     L.ag_packed_page_table.argtypes = [vp, vp, sz, C.POINTER(sz)]
     L.ag_packed_destroy.argtypes = [vp]
     L.ag_packed_destroy.restype = None
@@ -431,6 +432,12 @@ class PackedWeights:
         _check(lib().ag_packed_info(self.handle, C.byref(f)), "ag_packed_info")
         return int(f.value)
 
+    def closed_form(self) -> dict:
+        """Whether the kernels compute page addresses from the fitted hash (Eq. 1 in closed form) or read tables."""
+        en, mask, tb, cb = C.c_int32(), C.c_uint32(), C.c_size_t(), C.c_size_t()
+        _check(lib().ag_packed_closed_form(self.handle, C.byref(en), C.byref(mask), C.byref(tb), C.byref(cb)), "ag_packed_closed_form")
+        return dict(enabled=bool(en.value), mask=int(mask.value), table_bytes=int(tb.value), closed_bytes=int(cb.value))
+
     def page_table(self) -> np.ndarray:
         n = C.c_size_t()
         _check(lib().ag_packed_page_table(self.handle, None, 0, C.byref(n)), "ag_packed_page_table")
@@ -451,11 +458,11 @@ class PackedWeights:
 
 
 def pack_weights(b_ptr: int, K: int, N: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int,
-                 single_pages: bool = False) -> PackedWeights:
+                 single_pages: bool = False, tables_only: bool = False) -> PackedWeights:
     h = C.c_void_p()
     bl = (C.c_void_p * 1)(b_ptr)
-    _check(lib().ag_pack_weights_ex(bl, 1, K, N, plan.handle, amap.handle, dst_ptr, dst_bytes, 1 if single_pages else 0,
-                                    C.byref(h)), "ag_pack_weights_ex")
+    _check(lib().ag_pack_weights_ex(bl, 1, K, N, plan.handle, amap.handle, dst_ptr, dst_bytes,
+                                    (1 if single_pages else 0) | (2 if tables_only else 0), C.byref(h)), "ag_pack_weights_ex")
     return PackedWeights(h)
 
 

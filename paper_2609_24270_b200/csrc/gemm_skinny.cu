@@ -70,6 +70,7 @@ struct SkinnyArgs {
     const int32_t* page_table;    // device (PACKED)
     const int32_t* quad_base;     // device (PACKED, grouped layout): first chunk of each k-slab's group, or null
     int quad_f;                   // chunk distance 2^free_bit between the two halves of a group
+    int quad_f_bit;               // free_bit
     int pages_per_tile;
     float* C;
     float* partial;               // [k_splits][M][N] or null when k_splits == 1
@@ -83,6 +84,12 @@ struct SkinnyArgs {
     int tiles_per_group;
     int n_group;                  // columns of one expert
     int release_next;             // 1: let the next launch on the stream start while this one is still running
+    // closed form of the page table (PACKED): see table_entry in the kernel
+    const int32_t* unit_base;     // device [tiles_n * k_splits] or null (then the tables above are read)
+    const uint32_t* page_bits;    // device: one hash bit per 2 MiB page of the packed buffer
+    uint32_t hash_mask;
+    int hash_first;
+    int hash_t0;                  // groups of four chunks that start below hash_first (grouped layout)
 };
 
 // Where the output rows of column tile tn live: single problem = C itself; grouped = rows of expert g in the
@@ -289,9 +296,31 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const CUtensorMap* mw = x.g_tm_w ? &x.g_tm_w[grp] : &tm_w;
             // packed weights: lane l < 2 (groups of four pages) or l < 8 (single pages) looks up the chunk of the
             // l-th 16 KB / 4 KB piece of a stage, one stage ahead of the copies
+            // Closed form (Eq. 1 of the remapping appendix): the unit's pages are consecutive in the view of its die, so the
+            // chunk of a page follows from the unit's first position, the fitted hash mask and one bit per 2 MiB page;
+            // one table word per unit instead of one per page or group.
+            int ubase = 0;
+            if (PACKED && x.unit_base) ubase = x.unit_base[(size_t)tn * p.k_splits + ks];
             auto table_entry = [&](int i) -> int {
                 if (!PACKED || i >= n_st) return 0;
                 const int s = s0 + i * SK_SLABS;
+                if (x.unit_base) {
+                    const int d = (ubase >> 31) & 1, pos0 = ubase & 0x7fffffff;
+                    if (x.quad_base) {
+                        if (lane >= SK_SLABS || s + lane >= s1) return 0;
+                        const int f = x.quad_f_bit;
+                        const uint32_t T = (uint32_t)(pos0 + (s - s0) + lane + x.hash_t0);       // run of four chunks that holds the group
+                        const uint32_t qa0 = ((T >> (f - 2)) << (f + 1)) | ((T & ((1u << (f - 2)) - 1u)) << 2);
+                        const uint32_t cb = (x.page_bits[qa0 >> 14] >> ((qa0 >> 9) & 31)) & 1u;
+                        const uint32_t e = (__popc(qa0 & x.hash_mask) & 1u) ^ cb ^ (uint32_t)d;
+                        return (int)((qa0 + e - (uint32_t)x.hash_first) | (e << 30));           // bit 30: class of the group (a = 1)
+                    }
+                    if (lane >= 4 * SK_SLABS || s + (lane >> 2) >= s1) return 0;
+                    const uint32_t j = (uint32_t)(pos0 + (s - s0) * 4 + lane);                 // pair of chunks that holds the page
+                    const uint32_t qa = (uint32_t)x.hash_first + 2u * j;
+                    const uint32_t cb = (x.page_bits[qa >> 14] >> ((qa >> 9) & 31)) & 1u;
+                    return (int)(2u * j + ((__popc(qa & x.hash_mask) & 1u) ^ cb ^ (uint32_t)d));
+                }
                 if (x.quad_base) return (lane < SK_SLABS && s + lane < s1) ? x.quad_base[(size_t)tn * (x.pages_per_tile / 4) + s + lane] : 0;
                 return (lane < 4 * SK_SLABS && s + (lane >> 2) < s1) ? x.page_table[(size_t)tn * x.pages_per_tile + (size_t)s * 4 + lane] : 0;
             };
@@ -681,9 +710,17 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
         x.packed = W->dst;
         x.page_table = W->d_page_table;
         x.pages_per_tile = W->pages_per_tile;
+        if (W->closed_form && W->k_splits == h[H_KSPLITS]) {   // same units as the packing: positions are per unit
+            x.unit_base = W->d_unit_base;
+            x.page_bits = W->d_page_bits;
+            x.hash_mask = W->hash_mask;
+            x.hash_first = W->hash_first;
+            x.hash_t0 = W->hash_t0;
+        }
         if (W->quad_free_bit >= 0) {
             x.quad_base = W->d_quad_base;
             x.quad_f = 1 << W->quad_free_bit;
+            x.quad_f_bit = W->quad_free_bit;
             tm_w = W->tm_quad[0];
             tm_w2 = W->tm_quad[1];
         }
@@ -770,6 +807,8 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
     w->h_page_table.resize(n_pages);
     w->quad_free_bit = -1;
     w->d_quad_base = nullptr;
+    w->closed_form = 0; w->k_splits = ksp; w->hash_mask = 0; w->hash_first = 0; w->d_unit_base = nullptr; w->d_page_bits = nullptr;
+    w->table_bytes = w->closed_bytes = 0;
     const int per = plan->kslabs_per_split;
     auto owner_die = [&](int pc, int k16) {   // the die that runs most of the units reading this page (tie -> die 0)
         const int tn = pc / ppc, ks = (k16 * 16 / SK_BK) / per;
@@ -882,6 +921,77 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
         if (e == cudaSuccess)
             e = cudaMemcpy(w->d_quad_base, quad_base.data(), sizeof(int32_t) * quad_base.size(), cudaMemcpyHostToDevice);
     }
+    // Closed form of the tables (Eq. 1 of the remapping appendix).  The measured map must be an exact XOR hash over the
+    // chunks in use: mask from ag_affinity_fit_hash, one bit per 2 MiB page by majority, no chunk out of line; the
+    // buffer must start on a multiple of four chunks inside its 2 MiB page; decode-shaped plans only (one unit = one
+    // run of pages of one die).  Every table entry is then recomputed from the formula and compared; on any
+    // difference the tables stay in use.
+    if (e == cudaSuccess && !(flags & 2u) && tiles_m == 1 && ppc == 1) {
+        uint32_t mask = 0;
+        const size_t first = ((uintptr_t)dst / AG_CHUNK_BYTES) % 512;
+        const int f = w->quad_free_bit;
+        bool ok = ag_affinity_fit_hash(amap, &mask, nullptr) == AG_OK && (mask & 1u) && (first % 4) == 0;
+        if (ok && f >= 0) ok = (mask & 3u) == 3u && !((mask >> f) & 1u);
+        size_t max_chunk = 0;
+        for (size_t i = 0; i < n_pages; ++i) max_chunk = std::max(max_chunk, (size_t)w->h_page_table[i]);
+        const size_t used = std::min(amap->n_chunks, max_chunk + 1 + (f >= 0 ? ((size_t)1 << f) + 4 : 2));
+        std::vector<uint32_t> bits((((first + used) >> 9) + 32) / 32, 0u);
+        if (ok) {
+            const size_t n2m = ((first + used) >> 9) + 1;
+            std::vector<int> ones(n2m, 0), cnt(n2m, 0);
+            for (size_t q = 0; q < used; ++q) {
+                const size_t qa = first + q;
+                ones[qa >> 9] += amap->h_die_of_chunk[q] ^ (__builtin_popcount((uint32_t)qa & mask) & 1);
+                cnt[qa >> 9]++;
+            }
+            for (size_t pg = 0; pg < n2m; ++pg)
+                if (2 * ones[pg] > cnt[pg]) bits[pg >> 5] |= 1u << (pg & 31);
+        }
+        auto page_bit = [&](size_t qa) { return (bits[qa >> 14] >> ((qa >> 9) & 31)) & 1u; };
+        std::vector<int32_t> unit_base((size_t)n_blocks * ksp, 0);
+        int t0 = 0;
+        if (ok && f >= 0) {
+            const size_t F = (size_t)1 << f;
+            t0 = (int)((first / (2 * F)) * (F / 4) + std::min(first % (2 * F), F) / 4);
+        }
+        if (ok) {
+            // position of every unit's first page in its die's view = pages (or groups) of that die before it
+            size_t nxt[2] = {0, 0};
+            const int step = f >= 0 ? 4 : 1;                 // pages per position
+            for (int pc = 0; pc < n_blocks && ok; ++pc)
+                for (int ks = 0; ks < ksp && ok; ++ks) {
+                    const int k16_0 = ks * per * 4, k16_1 = std::min(ppt, (ks + 1) * per * 4);
+                    const int d = owner_die(pc, k16_0);
+                    unit_base[(size_t)pc * ksp + ks] = (int32_t)(nxt[d] | ((uint32_t)d << 31));
+                    for (int k16 = k16_0; k16 < k16_1 && ok; k16 += step) {
+                        const size_t pos = nxt[d]++;
+                        const size_t p0 = (size_t)pc * ppt + k16;
+                        if (f >= 0) {
+                            const size_t T = pos + (size_t)t0;
+                            const size_t qa0 = ((T >> (f - 2)) << (f + 1)) | ((T & (((size_t)1 << (f - 2)) - 1)) << 2);
+                            const uint32_t eb = (__builtin_popcount((uint32_t)qa0 & mask) & 1u) ^ page_bit(qa0) ^ (uint32_t)d;
+                            const int32_t q = (int32_t)(qa0 + eb - first);
+                            ok = quad_base[p0 / 4] == (q | (eb ? (1 << 30) : 0));
+                        } else {
+                            const size_t qa = first + 2 * pos;
+                            ok = w->h_page_table[p0] == (int32_t)(2 * pos + ((__builtin_popcount((uint32_t)qa & mask) & 1u) ^ page_bit(qa) ^ (uint32_t)d));
+                        }
+                    }
+                }
+        }
+        if (ok) {
+            e = cudaMalloc(&w->d_unit_base, sizeof(int32_t) * unit_base.size());
+            if (e == cudaSuccess) e = cudaMemcpy(w->d_unit_base, unit_base.data(), sizeof(int32_t) * unit_base.size(), cudaMemcpyHostToDevice);
+            if (e == cudaSuccess) e = cudaMalloc(&w->d_page_bits, sizeof(uint32_t) * bits.size());
+            if (e == cudaSuccess) e = cudaMemcpy(w->d_page_bits, bits.data(), sizeof(uint32_t) * bits.size(), cudaMemcpyHostToDevice);
+            w->closed_form = 1;
+            w->hash_mask = mask;
+            w->hash_first = (int)first;
+            w->hash_t0 = t0;
+            w->closed_bytes = sizeof(int32_t) * unit_base.size() + sizeof(uint32_t) * bits.size();
+        }
+    }
+    w->table_bytes = w->quad_free_bit >= 0 ? sizeof(int32_t) * quad_base.size() : sizeof(int32_t) * n_pages;
     const size_t pages_per_src = n_pages / G;
     for (int g = 0; g < G && e == cudaSuccess; ++g) {
         k_pack_weights<<<(unsigned)pages_per_src, 128>>>((const uint16_t*)B_list[g], K, n_src, ppt,
@@ -893,6 +1003,8 @@ static ag_status pack_weights_impl(const void* const* B_list, int G, int K, int 
     if (e != cudaSuccess) {
         cudaFree(w->d_page_table);
         cudaFree(w->d_quad_base);
+        cudaFree(w->d_unit_base);
+        cudaFree(w->d_page_bits);
         delete w;
         return cuda_fail(e);
     }
@@ -910,6 +1022,16 @@ extern "C" ag_status ag_pack_weights_ex(const void* const* B_list, int G, int K,
 extern "C" ag_status ag_packed_info(const ag_packed_weights* w, int32_t* group_free_bit) {
     if (!w || !group_free_bit) return AG_ERR_ARG;
     *group_free_bit = w->quad_free_bit;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_packed_closed_form(const ag_packed_weights* w, int32_t* enabled, uint32_t* mask, size_t* table_bytes,
+                                           size_t* closed_bytes) {
+    if (!w || !enabled) return AG_ERR_ARG;
+    *enabled = w->closed_form;
+    if (mask) *mask = w->hash_mask;
+    if (table_bytes) *table_bytes = w->table_bytes;
+    if (closed_bytes) *closed_bytes = w->closed_bytes;
     return AG_OK;
 }
 
@@ -1042,6 +1164,8 @@ extern "C" void ag_packed_destroy(ag_packed_weights* w) {
     if (!w) return;
     cudaFree(w->d_quad_base);
     cudaFree(w->d_page_table);
+    cudaFree(w->d_unit_base);
+    cudaFree(w->d_page_bits);
     delete w;
 }
 

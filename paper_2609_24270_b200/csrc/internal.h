@@ -96,6 +96,17 @@ struct ag_packed_weights {
     size_t dst_bytes;
     int32_t* d_page_table;               // device [n_pages]: chunk index of each logical page
     std::vector<int32_t> h_page_table;
+    // Closed form of the page table (Eq. 1 of the remapping appendix): when the measured map is an exact XOR hash, the
+    // chunk of a page follows from the page's position in its die's view, the fitted mask and one bit per 2 MiB page.
+    int closed_form;                     // 1: the kernels compute page addresses instead of reading the tables
+    int k_splits;                        // k-splits of the plan the weights were packed for (a unit = one run of pages)
+    uint32_t hash_mask;                  // fitted in-page mask (chunk-index bits 0..8)
+    int hash_first;                      // chunk index of dst inside its 2 MiB page
+    int hash_t0;                         // grouped layout: runs of four chunks (free bit clear) that start below hash_first
+    int32_t* d_unit_base;                // device [tiles_n * k_splits]: position of the unit's first page (pair or group
+                                         // index) in its die's view; bit 31 = the die
+    uint32_t* d_page_bits;               // device: one hash bit per 2 MiB page of dst
+    size_t table_bytes, closed_bytes;    // device bytes of the tables / of the closed form's data
 };
 
 // Grouped (MoE-shaped) decode GEMM: G experts, expert g multiplies rows [row_off[g], row_off[g] + rows[g]) of the

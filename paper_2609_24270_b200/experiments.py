@@ -126,7 +126,7 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
         # the same budget taken as whole TPCs from the GPCs of both dies: each die then streams its own half of the
         # weights from its own memory, and the set uses the memory of both dies
         plan_spread = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, **kw))
-        dsts, packs, packs_single, packs_spread = [], [], [], []
+        dsts, packs, packs_single, packs_spread, packs_tables = [], [], [], [], []
         for i in range(n_buffers):                      # rotate buffers so that no launch finds its weights in L2
             dst2 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
             amap2 = ag.affinity_probe(dst2.data_ptr(), dst_bytes, topo)
@@ -136,6 +136,11 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
             amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
             packs.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
             dsts.append(dst)
+            dst3 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")   # same layout, page addresses from tables
+            amap3 = ag.affinity_probe(dst3.data_ptr(), dst_bytes, topo)
+            packs_tables.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap3, dst3.data_ptr(), dst_bytes,
+                                                 tables_only=True), amap3))
+            dsts.append(dst3)
             dst1 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")   # same, one page per copy (for comparison)
             amap1 = ag.affinity_probe(dst1.data_ptr(), dst_bytes, topo)
             packs_single.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap1, dst1.data_ptr(), dst_bytes,
@@ -157,6 +162,7 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
         out = {}
         for name, plan, pset in (("die_local", plan_local, packs), ("remote", plan_remote, packs),
                                  ("die_local_single_pages", plan_local, packs_single),
+                                 ("die_local_page_tables", plan_local, packs_tables),
                                  ("die_local_both_dies", plan_spread, packs_spread)):
             state = {"i": 0}
 
@@ -178,10 +184,10 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
             out[name] = algo_bytes / (ms * 1e-3) / 1e9
         emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
                   sm_budget=b, overlap_launches=overlap, gbs=out, local_over_remote=out["die_local"] / out["remote"],
-                  pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), local_set=sm_set_summary(topo, plan_local),
+                  pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), closed_form=packs[0][0].closed_form(), local_set=sm_set_summary(topo, plan_local),
                   remote_set=sm_set_summary(topo, plan_remote), both_dies_set=sm_set_summary(topo, plan_spread), algo_bytes=algo_bytes,
                   hbm_peak_measured_gbs=6534.1), fh)
-        del packs, packs_single, packs_spread, dsts
+        del packs, packs_single, packs_spread, packs_tables, dsts
 
 
 def _unit_die(plan):

@@ -8,7 +8,7 @@ from oracle import gemm as og
 from oracle import plan as op
 from paper_2609_24270_b200 import binding as ag
 from paper_2609_24270_b200 import inputs
-from tests.gpu_util import check_close, device_topo, to_dev_bf16
+from tests.gpu_util import check_close, device_topo, oracle_policy, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -176,6 +176,65 @@ def test_packed_gemm_full_size_affinity_and_inverted_plans():
         torch.cuda.synchronize()
         assert plan.last_status() == ag.AG_OK
         check_close(dC.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("mask_bits,want_free_bit", [(0x1EF, 4), (0x1FF, -1)])
+def test_closed_form_remap_on_a_synthetic_hash(mask_bits, want_free_bit):
+    """Eq. 1 in closed form: with a map that is an exact XOR hash (handed in as a table), the kernel computes page
+    addresses from the fitted mask and the per-page bits; the page table and C equal the table-driven path's."""
+    M, N, K, ksp = 16, 1024, 2560, 4                          # 40 k-slabs: units of 10 slabs (5 stages)
+    topo = device_topo()
+    A, B = inputs.small_int_bf16(M, K, 71), inputs.small_int_bf16(K, N, 72)
+    dA, dB = to_dev_bf16(A), to_dev_bf16(B)
+    kw = dict(M=M, N=N, K=K, tile_m=16, tile_n=128, k_splits=ksp)
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+    dst_bytes = 2 * K * N * 2 + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    assert dst.data_ptr() % (2 << 20) == 0
+    doc = inputs.synthetic_chunk_die(dst_bytes // 4096, seed=13, mask_bits=mask_bits)
+    amap = ag.affinity_from_table(dst.data_ptr(), doc)
+    packs = {}
+    for tables_only in (False, True):
+        dst.zero_()
+        packs[tables_only] = ag.pack_weights(dB.data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes, tables_only=tables_only)
+        cf = packs[tables_only].closed_form()
+        assert packs[tables_only].group_free_bit() == want_free_bit
+        assert cf["enabled"] == (not tables_only)
+        if cf["enabled"]:
+            assert cf["mask"] == (mask_bits | 1) and cf["closed_bytes"] * 4 <= cf["table_bytes"]
+        dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        ag.gemm_persistent_packed(dA.data_ptr(), packs[tables_only], dC.data_ptr(), M, N, K, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), og.gemm_blocked(A, B))
+    assert np.array_equal(packs[False].page_table(), packs[True].page_table())
+    # the table is the oracle's: closed form on the oracle side too
+    o_plan = op.build_plan(topo.as_dict(), None, topo.n_sm, oracle_policy(kind=op.DIE_COMPACT, **kw))
+    page_die = op.page_die_from_plan(o_plan, K)
+    o_amap = dict(chunk_bytes=4096, die_of_chunk=doc)
+    want = (op.build_page_table_quads(page_die, o_amap, want_free_bit) if want_free_bit >= 0
+            else op.build_page_table(page_die, o_amap))
+    assert packs[False].page_table().tolist() == want
+
+
+def test_closed_form_remap_on_the_measured_map():
+    """On the chip's own map the closed form is used only if every table entry could be recomputed from the fitted
+    hash; either way the result is the same as with tables."""
+    M, N, K, ksp = 16, 2048, 2048, 4
+    topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(M, N, K, ksp, integer=True)
+    dA = to_dev_bf16(A)
+    dB = to_dev_bf16(B)
+    table0 = packed.page_table().copy()
+    packed_t = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst.numel(), tables_only=True)
+    assert not packed_t.closed_form()["enabled"]
+    assert np.array_equal(packed_t.page_table(), table0)
+    for pk in (packed, packed_t):
+        dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        ag.gemm_persistent_packed(dA.data_ptr(), pk, dC.data_ptr(), M, N, K, plan_d)
+        torch.cuda.synchronize()
+        assert plan_d.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), og.gemm_blocked(A, B))
+    print("closed form on the measured map:", packed.closed_form())
 
 
 def test_packed_rejects_foreign_map_and_shapes():
