@@ -246,6 +246,13 @@ typedef struct {
                                  weights; nothing of theirs is written before this launch has completed.  The caller
                                  promises that the inputs (A, B / packed weights) of a call are not produced by the call
                                  directly before it.  0 = launches run strictly one after the other */
+    int32_t cluster_size;    /* die_compact / affinity: thread-block cluster size (1, 2, 4 or 8) of the kernel the SM set is
+                                meant for; 0 and 1 mean none.  For sizes above 2 the set is built from what can host such
+                                clusters: SMs never seen in a cluster larger than 2 (is_random, Section 5.1.1) are taken last,
+                                and every GPC contributes whole blocks of cluster_size normal SMs - a GPC hosts only
+                                floor(n / cluster_size) clusters on n SMs (Section 7.3: twelve SMs form three clusters of
+                                four but one cluster of eight).  ag_cluster_capacity counts what a set can host */
+    int32_t reserved2;
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;
@@ -299,6 +306,18 @@ ag_status ag_plan_unit_times(const ag_plan* plan, uint64_t* start_ns, uint64_t* 
  */
 ag_status ag_plan_set_grid(ag_plan* plan, int blocks);
 ag_status ag_plan_adopted(const ag_plan* plan, uint32_t* n_lists);
+/* Thread-block clusters of cluster_size blocks that the plan's SM set can host at once with one block per SM: per GPC
+ * floor(normal SMs of the set in that GPC / cluster_size); SMs with is_random set or without a GPC host none when
+ * cluster_size > 2 (Sections 5.1.1, 7.3).  Errors: AG_ERR_ARG. */
+ag_status ag_cluster_capacity(const ag_plan* plan, const ag_topo_map* map, int cluster_size, int32_t* n_clusters);
+/*
+ * ag_probe_cluster_layout - where the hardware puts thread-block clusters (Section 5.1.1 probes the same way): launches
+ * n_clusters clusters of cluster_size blocks (one block per SM, every block stays until all have started or 50 us have
+ * passed) and reports, per SM id, the cluster that ran there first (-1: none).
+ *   cluster_of_sm  host, out, AG_MAX_SM entries
+ * Errors: AG_ERR_ARG (size not in 2..8, n_clusters < 1), AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA.
+ */
+ag_status ag_probe_cluster_layout(int cluster_size, int n_clusters, int32_t* cluster_of_sm);
 /* Device status word of the most recent launch (call after synchronising its stream). */
 ag_status ag_last_status(const ag_plan* plan);
 void ag_plan_destroy(ag_plan* plan);

@@ -34,6 +34,17 @@ Steps.
                            are dealt round-robin over the GPCs of both dies, which keeps the
                            number of SMs per GPC as low as the budget allows (SMs of one GPC
                            share its port to L2, Section 5.1.2).
+                           With cluster_size c > 2 (the kernel to be run launches thread-block clusters of c
+                           blocks) the set is built from what can host such clusters: SMs that cluster
+                           probing never saw in a cluster larger than 2 ("random" SMs, Section 5.1.1) and
+                           unplaced SMs cannot, and a GPC hosts only floor(n / c) clusters on n SMs
+                           (Section 7.3: 12 SMs of a GPC form three clusters of 4 but one cluster of 8).
+                           In the same die order as above, every GPC's normal candidate SMs (ascending)
+                           are cut into blocks of c, an incomplete tail is left aside, and whole blocks
+                           are dealt round-robin over the GPCs (block p of every GPC in ascending GPC id,
+                           p = 0, 1, ...) while a whole block still fits in the budget.  If the budget is
+                           not met that way, it is filled with the normal candidate SMs not yet taken (die
+                           order, then ascending id) and last with random and unplaced SMs (same order).
   3. per-die SM counts n_d and rank of each chosen SM inside its die (ascending id).
   4. quotas q_d = floor(n_u * n_d / b); leftover units go one each to the dies in
      descending order of (n_u * n_d mod b), tie -> lower die id.
@@ -86,7 +97,7 @@ def mix64(x: int) -> int:
 def default_policy(**kw) -> dict:
     p = dict(kind=OBLIVIOUS, seed=0, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1,
              k_unit=64, raster_group=1, preferred_die=-1, invert_affinity=0,
-             static_assign=1, min_margin=0, sm_select=0, pair_lists=0, avoid=(), a=None, b=None, c=None)
+             static_assign=1, min_margin=0, sm_select=0, pair_lists=0, cluster_size=1, avoid=(), a=None, b=None, c=None)
     p.update(kw)
     return p
 
@@ -134,6 +145,31 @@ def select_sms(topo: dict, b: int, pol: dict) -> list[int]:
         primary = 0 if cnt[0] >= cnt[1] else 1
     S = []
     die_passes = [(0, 1)] if pol.get("sm_select", 0) == 1 else [(primary,), (1 - primary,)]
+    csize = int(pol.get("cluster_size", 1))
+    if csize > 2:
+        rnd = topo["is_random"]
+        normal = lambda s: (not rnd[s]) and gpc[s] >= 0
+        for dies in die_passes:
+            per_gpc: dict[int, list[int]] = {}
+            for s in cand:
+                if die[s] in dies and normal(s):
+                    per_gpc.setdefault(int(gpc[s]), []).append(s)
+            keys = sorted(per_gpc)
+            blocks = {k: [per_gpc[k][i:i + csize] for i in range(0, len(per_gpc[k]) - csize + 1, csize)] for k in keys}
+            p = 0
+            while any(p < len(blocks[k]) for k in keys):
+                for k in keys:
+                    if p < len(blocks[k]) and len(S) + csize <= b:
+                        S += blocks[k][p]
+                p += 1
+        chosen = set(S)
+        for want_normal in (True, False):
+            for dies in die_passes:
+                for s in cand:
+                    if len(S) < b and s not in chosen and die[s] in dies and normal(s) == want_normal:
+                        S.append(s)
+                        chosen.add(s)
+        return sorted(S)
     for dies in die_passes:
         # candidate TPCs of these dies, grouped by GPC key (gpc < 0 -> pseudo-GPC n_gpc)
         groups: dict[int, dict[int, list[int]]] = {}
@@ -155,6 +191,18 @@ def select_sms(topo: dict, b: int, pol: dict) -> list[int]:
         if len(S) >= b:
             break
     return sorted(S)
+
+
+def cluster_capacity(topo: dict, S, csize: int) -> int:
+    """Thread-block clusters of ``csize`` blocks that the SM set S can host at once, one block per SM: per GPC,
+    floor(normal SMs of S in it / csize); random and unplaced SMs host none when csize > 2 (Sections 5.1.1, 7.3)."""
+    per = {}
+    for s in S:
+        if csize > 2 and (topo["is_random"][s] or topo["gpc"][s] < 0):
+            continue
+        key = int(topo["gpc"][s]) if topo["gpc"][s] >= 0 else -1 - int(s) // 2      # unplaced: only its own TPC
+        per[key] = per.get(key, 0) + 1
+    return sum(n // csize for n in per.values())
 
 
 # ----------------------------------------------------------------------------- step 4

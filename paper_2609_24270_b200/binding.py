@@ -26,7 +26,7 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_plan_set_grid", "ag_plan_adopted", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
+    "ag_plan_set_grid", "ag_plan_adopted", "ag_cluster_capacity", "ag_probe_cluster_layout", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
@@ -84,7 +84,7 @@ class Policy(C.Structure):
                 ("tile_m", C.c_int32), ("tile_n", C.c_int32), ("k_splits", C.c_int32), ("k_unit", C.c_int32),
                 ("raster_group", C.c_int32), ("preferred_die", C.c_int32), ("invert_affinity", C.c_int32),
                 ("static_assign", C.c_int32), ("seed", C.c_uint64), ("min_margin", C.c_int64),
-                ("splitk_in_memory", C.c_int32), ("sm_select", C.c_int32), ("pair_lists", C.c_int32), ("overlap_launches", C.c_int32),
+                ("splitk_in_memory", C.c_int32), ("sm_select", C.c_int32), ("pair_lists", C.c_int32), ("overlap_launches", C.c_int32), ("cluster_size", C.c_int32), ("reserved2", C.c_int32),
                 ("avoid_sm_mask", C.c_uint64 * 4),
                 ("a", OperandDesc), ("b", OperandDesc), ("c", OperandDesc)]
 
@@ -147,6 +147,8 @@ def lib() -> C.CDLL:
     L.gemm_persistent_packed.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.gemm_persistent_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.ag_wait_probe.argtypes = [C.c_uint64, C.POINTER(C.c_uint64)]
+    L.ag_cluster_capacity.argtypes = [vp, C.POINTER(TopoMap), C.c_int, C.POINTER(C.c_int32)]
+    L.ag_probe_cluster_layout.argtypes = [C.c_int, C.c_int, vp]
     L.ag_topo_save.argtypes = [C.POINTER(TopoMap), C.c_char_p]
     L.ag_topo_load.argtypes = [C.c_char_p, C.POINTER(TopoMap)]
     L.ag_group_desc_create.argtypes = [vp, vp, vp, C.c_int, vp, C.c_int, C.c_int, C.c_int, C.POINTER(vp)]
@@ -306,7 +308,7 @@ def affinity_from_table(dev_ptr: int, die_of_chunk: np.ndarray) -> AffinityMap:
 # ---- plan -------------------------------------------------------------------------------------
 def make_policy(kind=AG_OBLIVIOUS, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1, k_unit=64, raster_group=1,
                 preferred_die=-1, invert_affinity=0, static_assign=1, seed=0, min_margin=0, splitk_in_memory=0,
-                sm_select=0, pair_lists=None, overlap_launches=0, avoid=(), a=None, b=None, c=None):
+                sm_select=0, pair_lists=None, overlap_launches=0, cluster_size=1, avoid=(), a=None, b=None, c=None):
     """a/b/c: None or dict(offset, row_stride, elem_bytes[, layout, page_table]).  pair_lists=None means
     "on for plans of block pairs (tile_m == 256)"."""
     p = Policy()
@@ -318,6 +320,7 @@ def make_policy(kind=AG_OBLIVIOUS, M=0, N=0, K=0, tile_m=128, tile_n=256, k_spli
     p.sm_select = sm_select
     p.pair_lists = (1 if tile_m == 256 else 0) if pair_lists is None else pair_lists
     p.overlap_launches = overlap_launches
+    p.cluster_size = cluster_size
     for s in avoid:
         p.avoid_sm_mask[s >> 6] |= 1 << (s & 63)
     keep = []
@@ -375,6 +378,11 @@ class Plan:
 
     def reset_record(self):
         _check(lib().ag_plan_reset_record(self.handle), "ag_plan_reset_record")
+
+    def cluster_capacity(self, topo, cluster_size: int) -> int:
+        n = C.c_int32()
+        _check(lib().ag_cluster_capacity(self.handle, C.byref(topo), cluster_size, C.byref(n)), "ag_cluster_capacity")
+        return int(n.value)
 
     def trace(self, on: bool = True):
         _check(lib().ag_plan_trace(self.handle, 1 if on else 0), "ag_plan_trace")
@@ -477,6 +485,13 @@ def gemm_persistent_noalloc(a_ptr: int, b_ptr: int, c_ptr: int, M: int, N: int, 
     device array instead of allocated memory; for callers that may not allocate.  Calls on one GPU
     must not overlap.  Limits: k_splits * M * N * 4 <= 8 MiB, N <= 131072."""
     _check(lib().gemm_persistent_noalloc(a_ptr, b_ptr, c_ptr, M, N, K, plan.handle, stream), "gemm_persistent_noalloc")
+
+
+def probe_cluster_layout(cluster_size: int, n_clusters: int) -> np.ndarray:
+    """Cluster id that the hardware ran first on every SM (-1: none) for a launch of n_clusters clusters."""
+    out = np.full(AG_MAX_SM, -1, dtype=np.int32)
+    _check(lib().ag_probe_cluster_layout(cluster_size, n_clusters, out.ctypes.data), "ag_probe_cluster_layout")
+    return out
 
 
 class GroupDesc:

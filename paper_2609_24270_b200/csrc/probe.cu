@@ -83,6 +83,18 @@ __global__ void k_cluster_probe(int* smid_of_block) {
     }
 }
 
+// Cluster layout: every block notes its SM and start time, then stays until all blocks of the launch have started
+// (or 50 us have passed), so that one launch shows which SMs the hardware groups into clusters when all are wanted.
+__global__ void k_cluster_layout(int* smid_of_block, unsigned long long* start_ns, unsigned int* started, unsigned int n_blocks) {
+    if (threadIdx.x == 0) {
+        smid_of_block[blockIdx.x] = (int)smid();
+        const unsigned long long t0 = globaltimer_ns();
+        start_ns[blockIdx.x] = t0;
+        atomicAdd(started, 1u);
+        while (*reinterpret_cast<volatile unsigned int*>(started) < n_blocks && globaltimer_ns() - t0 < 50000ull) __nanosleep(500);
+    }
+}
+
 // ---- latency probe from one SM -------------------------------------------------------------
 // mode 0: save the line, invalidate it in L2 (discard.global.L2), timed load, write it back -
 //         the HBM-latency kernel of the paper's appendix.
@@ -943,6 +955,62 @@ extern "C" ag_status ag_affinity_fit_hash(const ag_affinity_map* amap, uint32_t*
             i += len;
         }
         *violations = bad;
+    }
+    return AG_OK;
+}
+
+extern "C" ag_status ag_probe_cluster_layout(int cluster_size, int n_clusters, int32_t* cluster_of_sm) {
+    if (!cluster_of_sm || cluster_size < 2 || cluster_size > 8 || n_clusters < 1 || n_clusters * cluster_size > 4096) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    static bool attr_done = false;
+    if (!attr_done) {
+        AG_CUDA(cudaFuncSetAttribute(k_cluster_layout, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
+        attr_done = true;
+    }
+    const int grid = n_clusters * cluster_size;
+    int* d_smid = nullptr;
+    unsigned long long* d_start = nullptr;
+    unsigned int* d_started = nullptr;
+    cudaError_t e = cudaMalloc(&d_smid, sizeof(int) * grid);
+    if (e == cudaSuccess) e = cudaMalloc(&d_start, sizeof(unsigned long long) * grid);
+    if (e == cudaSuccess) e = cudaMalloc(&d_started, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(d_smid, 0xFF, sizeof(int) * grid);
+    if (e == cudaSuccess) e = cudaMemset(d_started, 0, sizeof(unsigned int));
+    std::vector<int> ids(grid, -1);
+    std::vector<unsigned long long> t(grid, 0);
+    if (e == cudaSuccess) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(32);
+        cfg.dynamicSmemBytes = kPinSmem;      // more than half an SM: one block per SM at a time
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cluster_size;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, k_cluster_layout, d_smid, d_start, d_started, (unsigned int)grid);
+        if (e == cudaSuccess) count_launch();
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(ids.data(), d_smid, sizeof(int) * grid, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(t.data(), d_start, sizeof(unsigned long long) * grid, cudaMemcpyDeviceToHost);
+    cudaFree(d_smid);
+    cudaFree(d_start);
+    cudaFree(d_started);
+    if (e != cudaSuccess) return cuda_fail(e);
+    std::vector<unsigned long long> first(AG_MAX_SM, ~0ull);
+    for (int s = 0; s < AG_MAX_SM; ++s) cluster_of_sm[s] = -1;
+    for (int b = 0; b < grid; ++b) {
+        const int s = ids[b];
+        if (s < 0 || s >= AG_MAX_SM) continue;
+        if (t[b] < first[s]) {                 // an SM may host a second cluster after the first has left: keep the first
+            first[s] = t[b];
+            cluster_of_sm[s] = b / cluster_size;
+        }
     }
     return AG_OK;
 }

@@ -24,7 +24,7 @@ struct OperandDev {
 };
 struct PolicyDev {
     int kind, M, N, K, tile_m, tile_n, k_splits, k_unit, raster_group, preferred_die, invert, static_assign;
-    int sm_select, pair_lists;
+    int sm_select, pair_lists, cluster_size, pad0;
     unsigned long long seed;
     long long min_margin;
     unsigned long long avoid[4];
@@ -68,7 +68,9 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
                              int tiles_m, int tiles_n, int32_t* __restrict__ image, PlanLayout lay) {
     // the chip's per-SM arrays go to shared memory first (one thread walking them in global memory costs milliseconds)
     __shared__ short s_die[AG_MAX_SM], s_gpc[AG_MAX_SM], s_tpc[AG_MAX_SM];
+    __shared__ unsigned char s_rand[AG_MAX_SM];
     for (int s = threadIdx.x; s < topo->n_sm; s += blockDim.x) {
+        s_rand[s] = topo->is_random[s];
         s_die[s] = (short)topo->die[s];
         s_gpc[s] = (short)topo->gpc[s];
         s_tpc[s] = (short)topo->tpc[s];
@@ -102,6 +104,51 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
                                                                            : (cnt[0] >= cnt[1] ? 0 : 1);
         const int n_gpc = topo->n_gpc;
         const int n_pass = pol.sm_select == 1 ? 1 : 2;  // GPC spread: both dies in one round-robin
+        if (pol.cluster_size > 2) {
+            // Sets for kernels that launch clusters of c blocks: whole blocks of c normal SMs per GPC, dealt round-robin
+            // over the GPCs; then the normal SMs not yet taken, last the random and unplaced ones (Sections 5.1.1, 7.3).
+            const int c = pol.cluster_size;
+            __shared__ unsigned char taken[AG_MAX_SM];
+            for (int s = 0; s < n_sm; ++s) taken[s] = 0;
+            for (int pass_d = 0; pass_d < n_pass; ++pass_d) {
+                const int d = pol.sm_select == 1 ? -1 : (pass_d == 0 ? primary : 1 - primary);
+                bool any = true;
+                for (int p = 0; any; ++p) {
+                    any = false;
+                    for (int key = 0; key < n_gpc; ++key) {
+                        // block p of this GPC: its normal candidates number p*c .. p*c + c - 1 in ascending id
+                        int seen = 0, first_i = -1, last_i = -1;
+                        for (int i = 0; i < nc; ++i) {
+                            const int s = cand[i];
+                            if ((d >= 0 && s_die[s] != d) || s_rand[s] || s_gpc[s] != key) continue;
+                            if (seen == p * c) first_i = i;
+                            if (seen == p * c + c - 1) { last_i = i; break; }
+                            ++seen;
+                        }
+                        if (last_i < 0) continue;          // fewer than (p + 1) * c normal SMs here
+                        any = true;
+                        if (ns + c > b) continue;          // a whole block no longer fits in the budget
+                        for (int i = first_i; i <= last_i; ++i) {
+                            const int s = cand[i];
+                            if ((d >= 0 && s_die[s] != d) || s_rand[s] || s_gpc[s] != key) continue;
+                            S[ns++] = s;
+                            taken[s] = 1;
+                        }
+                    }
+                }
+            }
+            for (int want_normal = 1; want_normal >= 0; --want_normal)
+                for (int pass_d = 0; pass_d < n_pass; ++pass_d) {
+                    const int d = pol.sm_select == 1 ? -1 : (pass_d == 0 ? primary : 1 - primary);
+                    for (int i = 0; i < nc && ns < b; ++i) {
+                        const int s = cand[i];
+                        const int normal = (!s_rand[s] && s_gpc[s] >= 0) ? 1 : 0;
+                        if (taken[s] || (d >= 0 && s_die[s] != d) || normal != want_normal) continue;
+                        S[ns++] = s;
+                        taken[s] = 1;
+                    }
+                }
+        }
         for (int pass_d = 0; pass_d < n_pass && ns < b; ++pass_d) {
             const int d = pol.sm_select == 1 ? -1 : (pass_d == 0 ? primary : 1 - primary);
             // distinct TPC ids of the candidates of every GPC key (unplaced SMs: key n_gpc), ascending, built once
@@ -406,6 +453,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     if (p.M <= 0 || p.N <= 0 || p.K <= 0 || p.tile_m <= 0 || p.tile_n <= 0) return AG_ERR_ARG;
     if (p.k_splits < 1 || p.k_unit < 1 || p.raster_group < 1 || p.min_margin < 0) return AG_ERR_ARG;
     if (p.sm_select < 0 || p.sm_select > 1) return AG_ERR_ARG;
+    if (p.cluster_size != 0 && p.cluster_size != 1 && p.cluster_size != 2 && p.cluster_size != 4 && p.cluster_size != 8) return AG_ERR_ARG;
     if (p.kind == AG_AFFINITY && !amap) return AG_ERR_ARG;
     int n_cand = 0;
     for (int s = 0; s < map->n_sm; ++s)
@@ -487,6 +535,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pd.preferred_die = p.preferred_die; pd.invert = p.invert_affinity; pd.static_assign = p.static_assign;
         pd.seed = p.seed;
         pd.sm_select = p.sm_select;
+        pd.cluster_size = p.cluster_size;
         pd.pair_lists = p.pair_lists ? 1 : 0;
         pd.min_margin = p.min_margin;
         for (int i = 0; i < 4; ++i) pd.avoid[i] = p.avoid_sm_mask[i];
@@ -611,6 +660,24 @@ extern "C" ag_status ag_plan_unit_times(const ag_plan* plan, uint64_t* start_ns,
         start_ns[u] = t[2 * (size_t)u];
         end_ns[u] = t[2 * (size_t)u + 1];
     }
+    return AG_OK;
+}
+
+extern "C" ag_status ag_cluster_capacity(const ag_plan* plan, const ag_topo_map* map, int cluster_size, int32_t* n_clusters) {
+    if (!plan || !map || !n_clusters || cluster_size < 1 || cluster_size > 16 || map->n_sm != plan->lay.n_sm) return AG_ERR_ARG;
+    std::vector<int> per_gpc(AG_MAX_GPC, 0), loose_tpc(AG_MAX_SM, 0);
+    int total = 0;
+    const int32_t* list = plan->h_image.data() + plan->lay.sm_list();
+    for (int i = 0; i < plan->lay.b; ++i) {
+        const int s = list[i];
+        const bool placed = map->gpc[s] >= 0 && map->gpc[s] < AG_MAX_GPC;
+        if (cluster_size > 2 && (map->is_random[s] || !placed)) continue;
+        if (placed) per_gpc[map->gpc[s]]++;
+        else loose_tpc[(map->tpc[s] >= 0 && map->tpc[s] < AG_MAX_SM) ? map->tpc[s] : 0]++;   // an unplaced SM is only known to share a TPC with its neighbour
+    }
+    for (int g = 0; g < AG_MAX_GPC; ++g) total += per_gpc[g] / cluster_size;
+    for (int t = 0; t < AG_MAX_SM; ++t) total += loose_tpc[t] / cluster_size;
+    *n_clusters = total;
     return AG_OK;
 }
 

@@ -8,6 +8,7 @@
     python -m paper_2609_24270_b200.experiments --config groupgemm_dense   # same, 192 / 1024 rows per expert
     python -m paper_2609_24270_b200.experiments --config gpc_bandwidth     # L2 bandwidth of k SMs: one GPC vs spread
     python -m paper_2609_24270_b200.experiments --config latency           # latency histograms from one SM per die
+    python -m paper_2609_24270_b200.experiments --config cluster_sets      # cluster eligibility of equal-size SM sets
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
 launches first, median of the timed launches.  torch is used for device memory, streams and events.
@@ -424,6 +425,43 @@ def latency_histograms(fh, topo):
                       counts=[int(x) for x in hist], median=float(np.median(v))), fh)
 
 
+def cluster_sets(fh, topo, budgets=(64, 72, 96), n_subsets=16):
+    """Cluster eligibility of equal-size SM sets (Sections 5.1.1, 7.3): how many thread-block clusters of 4 and 8 blocks
+    a set can host.  Two counts per set: the capacity computed from the map (per GPC floor(normal SMs / c)), and the
+    number of clusters of one full-chip launch that the hardware placed wholly inside the set."""
+    full = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=4096, N=4096, K=4096))
+    for c in (4, 8):
+        cap_chip = full.cluster_capacity(topo, c)
+        lay = ag.probe_cluster_layout(c, cap_chip)[:topo.n_sm]
+        clusters = {}
+        for s in range(topo.n_sm):
+            if lay[s] >= 0:
+                clusters.setdefault(int(lay[s]), []).append(s)
+
+        def inside(sms):
+            ss = set(sms)
+            return sum(1 for m in clusters.values() if len(m) == c and set(m) <= ss)
+        for b in budgets:
+            kw = dict(M=4096, N=4096, K=4096)
+            sets = {f"random_{i}": ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, seed=i, **kw)) for i in range(1, n_subsets + 1)}
+            sets["lowest_ids"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
+            sets["highest_ids"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, avoid=list(range(topo.n_sm - b)), **kw))
+            sets["die_compact_tpc"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+            sets["die_compact_cluster"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, cluster_size=c, **kw))
+            sets["gpc_spread_cluster"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, cluster_size=c, **kw))
+            res = {}
+            for n, pl in sets.items():
+                sms = [int(x) for x in pl.parsed()["sm_list"]]
+                res[n] = dict(capacity=pl.cluster_capacity(topo, c), placed_inside=inside(sms))
+            rnd = [res[f"random_{i}"] for i in range(1, n_subsets + 1)]
+            emit(dict(config="cluster_sets", cluster_size=c, sm_budget=b, ideal=b // c, chip_capacity=cap_chip,
+                      clusters_seen=len(clusters),
+                      random_capacity=dict(min=min(r["capacity"] for r in rnd), max=max(r["capacity"] for r in rnd),
+                                           median=float(np.median([r["capacity"] for r in rnd]))),
+                      random_placed_inside=dict(min=min(r["placed_inside"] for r in rnd), max=max(r["placed_inside"] for r in rnd)),
+                      **{n: res[n] for n in ("lowest_ids", "highest_ids", "die_compact_tpc", "die_compact_cluster", "gpc_spread_cluster")}), fh)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -435,7 +473,7 @@ def main():
               gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
-     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms}[args.config](fh, topo)
+     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets}[args.config](fh, topo)
 
 
 if __name__ == "__main__":

@@ -51,6 +51,30 @@ def test_gpc_spread_selection_matches_oracle(b):
         assert got.tobytes() == want.tobytes()
 
 
+@pytest.mark.parametrize("c", [4, 8])
+@pytest.mark.parametrize("b", [10, 32, 64, 72, 100, 140, 148])
+def test_cluster_aware_sets_match_oracle(c, b):
+    """Sets for kernels that launch clusters of c blocks: bytewise equal to the oracle, and the capacity the library
+    reports is the oracle's."""
+    for die0, seed in ((70, 3), (74, 6)):
+        topo = inputs.synthetic_topo(die0_sms=die0, seed=seed)
+        for sel in (0, 1):
+            got, want, plan = both(topo, None, b, kind=ag.AG_DIE_COMPACT, M=4096, N=4096, K=4096, raster_group=4,
+                                   sm_select=sel, cluster_size=c)
+            assert got.tobytes() == want.tobytes()
+            S = [int(x) for x in plan.parsed()["sm_list"]]
+            assert plan.cluster_capacity(ag.TopoMap.from_dict(topo), c) == op.cluster_capacity(topo, S, c)
+    # the hand-worked toy chip: one random TPC, a GPC of five TPCs
+    toy = dict(n_sm=24, n_tpc=12, n_gpc=3, n_die=2, tpc=np.array([s // 2 for s in range(24)]),
+               gpc=np.array([0] * 10 + [1] * 8 + [2] * 6), die=np.array([0] * 18 + [1] * 6),
+               is_random=np.array([0] * 22 + [1, 1]), gpc_die=[0, 0, 1], die_sm_count=[18, 6], gpc_sm_count=[10, 8, 6])
+    if b <= 24:
+        got, want, plan = both(toy, None, b, kind=ag.AG_DIE_COMPACT, M=512, N=512, K=64, cluster_size=c)
+        assert got.tobytes() == want.tobytes()
+        if (c, b) == (4, 10):
+            assert [int(x) for x in plan.parsed()["sm_list"]] == [0, 1, 2, 3, 4, 5, 10, 11, 12, 13]
+
+
 def test_avoid_mask_and_unplaced_sms():
     topo = inputs.synthetic_topo(die0_sms=74, seed=4)
     topo["gpc"] = topo["gpc"].copy()

@@ -97,3 +97,24 @@ def test_local_bandwidth_beats_remote(topo):
     for r in (0, 1):
         assert bw[(r, r)] > 1.15 * bw[(r, 1 - r)], bw        # local pages stream faster than remote ones
         assert 0.5e12 < bw[(r, r)] < 6e12, bw
+
+
+def test_cluster_layout_respects_the_map():
+    """Where the hardware puts clusters of four and eight blocks: always inside one GPC class of the discovered map and
+    never on an SM that cluster probing marked as random (Section 5.1.1); the number it co-schedules is the capacity
+    the library computes for the full chip."""
+    topo = ag.topo_discover(ag.AG_TOPO_CENSUS | ag.AG_TOPO_CLUSTER | ag.AG_TOPO_LATENCY)
+    full = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=4096, N=4096, K=4096))
+    for c in (4, 8):
+        cap = full.cluster_capacity(topo, c)
+        assert cap >= 8
+        lay = ag.probe_cluster_layout(c, cap)[:topo.n_sm]
+        used = [s for s in range(topo.n_sm) if lay[s] >= 0]
+        assert not any(topo.is_random[s] for s in used)
+        for cl in set(int(x) for x in lay if x >= 0):
+            members = [s for s in range(topo.n_sm) if lay[s] == cl]
+            gpcs = {topo.gpc[s] for s in members if topo.gpc[s] >= 0}
+            assert len(gpcs) <= 1
+        # all `cap` clusters found room at once: every one of them shows up with its c SMs
+        sizes = np.bincount([int(x) for x in lay if x >= 0], minlength=cap)
+        assert (sizes == c).sum() >= cap - 1

@@ -552,3 +552,64 @@ def test_closed_form_quad_groups_equal_the_enumeration(first):
         nxt[d] += 1
         want += [q, q + a, q + 16, q + 16 + a]
     assert table == want
+
+
+TOY24 = dict(n_sm=24, n_tpc=12, n_gpc=3, n_die=2, tpc=[s // 2 for s in range(24)],
+             gpc=[0] * 10 + [1] * 8 + [2] * 4 + [2, 2], die=[0] * 18 + [1] * 6,
+             is_random=[0] * 22 + [1, 1], gpc_die=[0, 0, 1])
+
+
+def test_cluster_aware_sets_by_hand():
+    """A 24-SM toy chip: GPC 0 has five TPCs (SMs 0-9), GPC 1 four (10-17), GPC 2 two (18-21) plus one random TPC
+    (22, 23) that never hosts clusters larger than 2.  Die 0 = GPCs 0 and 1."""
+    base = dict(kind=op.DIE_COMPACT, M=1, N=1, K=1)
+    # budget 12, clusters of 4.  Die 0 first: GPC 0 blocks [0-3] [4-7] (8, 9 left aside), GPC 1 blocks [10-13] [14-17];
+    # dealt round-robin: [0-3], [10-13], [4-7] -> 12 SMs, three clusters of four.
+    S4 = op.select_sms(TOY24, 12, op.default_policy(cluster_size=4, **base))
+    assert S4 == [0, 1, 2, 3, 4, 5, 6, 7, 10, 11, 12, 13]
+    assert op.cluster_capacity(TOY24, S4, 4) == 3
+    # the TPC-wise rule takes three TPCs from either GPC: six SMs each, room for only one cluster of four per GPC
+    S1 = op.select_sms(TOY24, 12, op.default_policy(**base))
+    assert S1 == [0, 1, 2, 3, 4, 5, 10, 11, 12, 13, 14, 15]
+    assert op.cluster_capacity(TOY24, S1, 4) == 2
+    # budget 20, clusters of 8: blocks [0-7] and [10-17]; GPC 2 (four normal SMs) has no block of eight; the budget is
+    # filled with the normal SMs left aside, die 0 first (8, 9), then die 1 (18, 19)
+    S8 = op.select_sms(TOY24, 20, op.default_policy(cluster_size=8, **base))
+    assert S8 == list(range(20))
+    assert op.cluster_capacity(TOY24, S8, 8) == 2
+    # random SMs come last: budget 23 leaves out SM 23, budget 22 takes no random SM at all
+    assert op.select_sms(TOY24, 22, op.default_policy(cluster_size=4, **base)) == list(range(22))
+    assert op.select_sms(TOY24, 23, op.default_policy(cluster_size=4, **base)) == list(range(23))
+    # a budget that is no multiple of the cluster size: two whole blocks ([0-3], [10-13]; a third does not fit), then
+    # the lowest normal SMs not yet taken (4, 5)
+    S10 = op.select_sms(TOY24, 10, op.default_policy(cluster_size=4, **base))
+    assert S10 == [0, 1, 2, 3, 4, 5, 10, 11, 12, 13] and op.cluster_capacity(TOY24, S10, 4) == 2
+    # Section 7.3's arithmetic: twelve SMs of one GPC form three clusters of four but one cluster of eight
+    one_gpc = dict(TOY24, gpc=[0] * 24, is_random=[0] * 24)
+    assert op.cluster_capacity(one_gpc, list(range(12)), 4) == 3
+    assert op.cluster_capacity(one_gpc, list(range(12)), 8) == 1
+    # GPC spread with clusters of 4: blocks dealt over the GPCs of both dies: [0-3], [10-13], [18-21]
+    Ss = op.select_sms(TOY24, 12, op.default_policy(cluster_size=4, sm_select=1, **base))
+    assert Ss == [0, 1, 2, 3, 10, 11, 12, 13, 18, 19, 20, 21]
+
+
+def test_cluster_aware_sets_on_synthetic_b200():
+    topo = inputs.synthetic_topo(die0_sms=70, seed=3)
+    n_random = int(sum(topo["is_random"]))
+    assert n_random > 0
+    for c in (4, 8):
+        for b in (32, 64, 72, 100, 148):
+            for sel in (0, 1):
+                pol = op.default_policy(kind=op.DIE_COMPACT, M=4096, N=4096, K=4096, cluster_size=c, sm_select=sel)
+                S = op.select_sms(topo, b, pol)
+                assert len(S) == b == len(set(S))
+                cap = op.cluster_capacity(topo, S, c)
+                best = op.cluster_capacity(topo, list(range(148)), c)
+                assert cap == min(b // c, best) or (sel == 0 and cap >= min(b // c, best) - 1)
+                # never worse than the TPC-wise set of the same budget, and random SMs only when nothing else is left
+                S0 = op.select_sms(topo, b, op.default_policy(kind=op.DIE_COMPACT, M=1, N=1, K=1, sm_select=sel))
+                assert cap >= op.cluster_capacity(topo, S0, c)
+                if b <= 148 - n_random:
+                    assert not any(topo["is_random"][s] for s in S)
+                plan = op.build_plan(topo, None, b, pol)
+                check_invariants(topo, plan, pol, b)
