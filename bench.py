@@ -37,8 +37,8 @@ FLOPS = 2.0 * M * N * K
 METRIC = "bf16_gemm_tflops"
 UNIT = "TFLOP/s"
 # DRAM bytes per launch of the dominant kernel, from an Nsight Compute capture of two timed steps of this
-# bench (dram__bytes_read.sum 1.050 GB + dram__bytes_write.sum 0.251 GB; summary kept under profiles/).
-NCU_TRAFFIC_BYTES = 1.301e9
+# bench (dram__bytes_read.sum 1.042 GB + dram__bytes_write.sum 0.251 GB; summary kept under profiles/).
+NCU_TRAFFIC_BYTES = 1.293e9
 
 
 def load_peaks():
@@ -326,6 +326,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default="all", choices=["all", "headline", "decode"],
+                    help="profiling aid: leave out the decode-shaped and SM-set sections (headline) or everything but the decode-shaped section (decode)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -364,6 +366,17 @@ def main():
     t0 = time.time()
     topo = ag.topo_discover()
     t_topo = time.time() - t0
+    if args.only == "decode":
+        # profiling aid: the decode-shaped section alone
+        sampler = ClockSampler(local)
+        sampler.start()
+        decode = decode_section(ag, inputs, torch, topo, peaks, sampler)
+        sampler.stop()
+        if rank == 0:
+            print(json.dumps({"only": "decode", "decode": decode}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     t0 = time.time()
     amap = ag.affinity_probe(buf.data_ptr(), buf.numel(), topo)
     t_aff = time.time() - t0
@@ -477,8 +490,8 @@ def main():
         sustained["tflops_per_sm_ghz"] = sustained["tflops"] / (sus_clocks["sm_mhz"] / 1e3)
     rot_clocks = sampler.summary("rotation")
 
-    decode = decode_section(ag, inputs, torch, topo, peaks, sampler)
-    subsets = subset_section(ag, inputs, torch, topo, sampler)
+    decode = decode_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
+    subsets = subset_section(ag, inputs, torch, topo, sampler) if args.only == "all" else None
     sampler.stop()
 
     # ---- end to end through the same call with host buffers.  Every step copies its A and B from pinned host
