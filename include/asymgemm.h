@@ -20,8 +20,8 @@
  *   - A handle (plan, affinity map, packed weights, group descriptor) may be used by one host
  *     thread at a time; launches of one plan must not overlap on the device (use one plan per
  *     stream).  Different plans may run concurrently on disjoint SM sets (avoid_sm_mask).
- *   - gemm_persistent, gemm_persistent_packed, gemm_persistent_grouped and gemm_persistent_noalloc
- *     return AG_ERR_ARG, and queue nothing, when cuda_stream is being captured: every launch carries
+ *   - gemm_persistent, gemm_persistent_packed, gemm_persistent_grouped, gemm_persistent_noalloc and
+ *     attention_decode_persistent return AG_ERR_ARG, and queue nothing, when cuda_stream is being captured: every launch carries
  *     a launch number (epoch) in its kernel parameters, by which the thread blocks take their places
  *     in the plan; a replayed graph would repeat an old number and no block would join.
  *   - Environment: AG_DEBUG=1 makes topo_discover print its bandwidth measurements and any
@@ -479,6 +479,47 @@ ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weight
  */
 ag_status gemm_persistent_noalloc(const void* A, const void* B, void* C, int M, int N, int K,
                                   const ag_plan* plan, void* cuda_stream);
+
+/* ---- grouped-query attention decode with die-local KV pages ---------------------------------------
+ * Attention is the paper's second scheduled workload (Section 7.1.2; workload appendix: decode = one query token per
+ * request, GQA with 8 KV heads, head dimension 128, KV working set 4 B S_k H_kv D bytes).  Work unit = (request, KV
+ * head): o = softmax(q K^T / sqrt(D)) V for the H_q / H_kv query heads that share the KV head.  The plan is an ordinary
+ * decode-shaped plan with one unit per (request, KV head): sched_build with tile_m = 16, tile_n = 128, k_splits = 1,
+ * M = H_q / H_kv, N = 128 * B * H_kv (K is not looked at); unit u = request u / H_kv, KV head u % H_kv.
+ */
+typedef struct ag_kv_cache ag_kv_cache;
+/*
+ * ag_kv_pack - store a KV cache in 4 KB pages in the order the tensor cores read them, every unit's pages in chunks
+ * of one die (indirect allocation by remapping, Section 7.1.1, applied to the KV cache).
+ *   K, V   device, [B][H_kv][L][D] bf16 row-major; D = 128; L a multiple of 128, L <= 1024
+ *   plan   B * H_kv units (see above)
+ *   amap   affinity map of exactly (dst, dst_bytes), else AG_ERR_STALE_AMAP
+ *   dst    device, 4096-aligned; local / remote placement needs room for 2 x the larger die's share, interleaved 1 x
+ *   placement  0: on the die that the plan runs the unit on; 1: on the other die; 2: interleaved (consecutive chunks,
+ *          the hardware's default placement)
+ * Placements 0 and 1 need a map that follows an XOR hash with a free bit (groups of four same-die chunks, see
+ * ag_pack_weights_ex), else AG_ERR_NOISY_PROBE.  Synchronises the device.
+ * Errors: AG_ERR_ARG, AG_ERR_STALE_AMAP, AG_ERR_NOISY_PROBE, AG_ERR_CUDA, AG_ERR_NOMEM.
+ */
+ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, int L, int D, const ag_plan* plan,
+                     const ag_affinity_map* amap, void* dst, size_t dst_bytes, int placement, ag_kv_cache** out);
+/* group_free_bit: the hash bit the page groups use (-1: interleaved placement); local_fraction: share of the pages that
+ * the map places on the die of their unit (either may be NULL). */
+ag_status ag_kv_info(const ag_kv_cache* kv, int32_t* group_free_bit, double* local_fraction);
+void ag_kv_destroy(ag_kv_cache* kv);
+/*
+ * attention_decode_persistent - O[b][hq][:] = softmax_j(Q[b][hq] . K[b][h][j] / sqrt(D)) V[b][h][j][:], h = hq / (H_q / H_kv),
+ * over the first kv_len[b] keys.  Scores and outputs are accumulated in fp32 by tcgen05 MMAs; the probabilities enter
+ * the second product as the sum of two bf16 parts (16 significant bits).
+ *   Q       device, [B][H_q][128] bf16, 16-byte aligned; H_q / H_kv <= 8
+ *   kv      from ag_kv_pack (same B)
+ *   kv_len  device [B] int32 or NULL (every request has L keys); values are clamped to 0..L; a request with 0 keys
+ *           gets zeros
+ *   O       device, [B][H_q][128] fp32, overwritten
+ * Asynchronous on cuda_stream.  Errors as gemm_persistent; device-side status via ag_last_status.
+ */
+ag_status attention_decode_persistent(const void* Q, const ag_kv_cache* kv, const int32_t* kv_len, void* O, int B,
+                                      int H_q, const ag_plan* plan, void* cuda_stream);
 
 /*
  * ag_wait_probe - self test of the bounded device-side wait that every kernel of this library

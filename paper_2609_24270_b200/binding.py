@@ -30,7 +30,7 @@ EXPORTED = [
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
-    "ag_kernel_launch_count",
+    "ag_kernel_launch_count", "ag_kv_pack", "ag_kv_info", "ag_kv_destroy", "attention_decode_persistent",
 ]
 
 
@@ -147,6 +147,11 @@ def lib() -> C.CDLL:
     L.gemm_persistent_packed.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.gemm_persistent_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.ag_wait_probe.argtypes = [C.c_uint64, C.POINTER(C.c_uint64)]
+    L.ag_kv_pack.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, sz, C.c_int, C.POINTER(vp)]
+    L.ag_kv_info.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_double)]
+    L.ag_kv_destroy.argtypes = [vp]
+    L.ag_kv_destroy.restype = None
+    L.attention_decode_persistent.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, vp, vp]
     L.ag_cluster_capacity.argtypes = [vp, C.POINTER(TopoMap), C.c_int, C.POINTER(C.c_int32)]
     L.ag_probe_cluster_layout.argtypes = [C.c_int, C.c_int, vp]
     L.ag_topo_save.argtypes = [C.POINTER(TopoMap), C.c_char_p]
@@ -485,6 +490,37 @@ def gemm_persistent_noalloc(a_ptr: int, b_ptr: int, c_ptr: int, M: int, N: int, 
     device array instead of allocated memory; for callers that may not allocate.  Calls on one GPU
     must not overlap.  Limits: k_splits * M * N * 4 <= 8 MiB, N <= 131072."""
     _check(lib().gemm_persistent_noalloc(a_ptr, b_ptr, c_ptr, M, N, K, plan.handle, stream), "gemm_persistent_noalloc")
+
+
+KV_LOCAL, KV_REMOTE, KV_INTERLEAVED = 0, 1, 2
+
+
+class KVCache:
+    def __init__(self, handle):
+        self.handle = handle
+
+    def info(self) -> dict:
+        f, frac = C.c_int32(), C.c_double()
+        _check(lib().ag_kv_info(self.handle, C.byref(f), C.byref(frac)), "ag_kv_info")
+        return dict(group_free_bit=int(f.value), local_fraction=float(frac.value))
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            lib().ag_kv_destroy(self.handle)
+            self.handle = None
+
+
+def kv_pack(k_ptr: int, v_ptr: int, B: int, H_kv: int, L: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int,
+            placement: int = KV_LOCAL, D: int = 128) -> KVCache:
+    h = C.c_void_p()
+    _check(lib().ag_kv_pack(k_ptr, v_ptr, B, H_kv, L, D, plan.handle, amap.handle, dst_ptr, dst_bytes, placement, C.byref(h)),
+           "ag_kv_pack")
+    return KVCache(h)
+
+
+def attention_decode(q_ptr: int, kv: KVCache, kv_len_ptr, o_ptr: int, B: int, H_q: int, plan: Plan, stream: int = 0):
+    _check(lib().attention_decode_persistent(q_ptr, kv.handle, kv_len_ptr, o_ptr, B, H_q, plan.handle, stream),
+           "attention_decode_persistent")
 
 
 def probe_cluster_layout(cluster_size: int, n_clusters: int) -> np.ndarray:

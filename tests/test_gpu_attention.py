@@ -1,0 +1,117 @@
+"""Attention decode with die-local KV pages against the fp64 oracle (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as oa
+from paper_2609_24270_b200 import binding as ag
+from paper_2609_24270_b200 import inputs
+from tests.gpu_util import device_topo
+
+pytestmark = pytest.mark.gpu
+
+# Tolerance: scores are exact bf16 products accumulated in fp32 (relative 2^-24 per add), the exponential is the
+# hardware's exp2 (2 ulp), the probabilities enter the second product with 16 significant bits, outputs are
+# accumulated in fp32: a few 1e-6 relative in all; the bound asserted leaves a factor of ten.
+REL_FRO, MAX_ABS = 5e-5, 2e-4
+
+
+def make_case(B, Hq, Hkv, L, seed, q_scale=1.0):
+    D = 128
+    Q = inputs.uniform_bf16(B * Hq, D, seed).reshape(B, Hq, D)
+    if q_scale != 1.0:
+        qf = oa.bf16_to_f64(Q) * q_scale
+        Q = inputs.f32_to_bf16_bits(qf.astype(np.float32)).reshape(B, Hq, D)
+    K = inputs.uniform_bf16(B * Hkv * L, D, seed + 1).reshape(B, Hkv, L, D)
+    V = inputs.uniform_bf16(B * Hkv * L, D, seed + 2).reshape(B, Hkv, L, D)
+    return Q, K, V
+
+
+def dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16).copy()).cuda()
+
+
+def run_attention(Q, K, V, placement, kv_len=None, budget=None):
+    B, Hq, D = Q.shape
+    _, Hkv, L, _ = K.shape
+    topo = device_topo()
+    b = topo.n_sm if budget is None else budget
+    plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
+                                                        tile_n=128, k_splits=1))
+    kv_bytes = 2 * B * Hkv * L * D * 2
+    dst_bytes = (2 * kv_bytes if placement != ag.KV_INTERLEAVED else kv_bytes) + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    dK, dV, dQ = dev(K), dev(V), dev(Q)
+    kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes, placement)
+    dO = torch.full((B, Hq, D), float("nan"), dtype=torch.float32, device="cuda")
+    dlen = None if kv_len is None else torch.tensor(kv_len, dtype=torch.int32, device="cuda")
+    plan.reset_record()
+    for _ in range(2):
+        ag.attention_decode(dQ.data_ptr(), kv, None if dlen is None else dlen.data_ptr(), dO.data_ptr(), B, Hq, plan)
+    torch.cuda.synchronize()
+    st = plan.last_status()
+    assert st == ag.AG_OK, ag.strerror(st)
+    owner, count = plan.tile_record()
+    assert (count == 2).all()
+    return dO.cpu().numpy().astype(np.float64), kv.info(), dst
+
+
+def check(got, want):
+    assert np.isfinite(got).all()
+    rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
+    mx = np.abs(got - want).max()
+    assert rel <= REL_FRO and mx <= MAX_ABS, (rel, mx)
+
+
+@pytest.mark.parametrize("placement", [ag.KV_LOCAL, ag.KV_REMOTE, ag.KV_INTERLEAVED])
+@pytest.mark.parametrize("shape", [(4, 8, 2, 256), (3, 16, 2, 128), (9, 4, 4, 384)])
+def test_small_cases_against_the_oracle(placement, shape):
+    B, Hq, Hkv, L = shape
+    for q_scale in (1.0, 12.0):                      # soft and peaked score distributions
+        Q, K, V = make_case(B, Hq, Hkv, L, seed=100 + B, q_scale=q_scale)
+        got, info, _ = run_attention(Q, K, V, placement)
+        check(got, oa.gqa_decode(Q, K, V))
+        if placement == ag.KV_LOCAL:
+            assert info["local_fraction"] == 1.0 and info["group_free_bit"] >= 2
+
+
+def test_ragged_lengths_and_closed_forms():
+    B, Hq, Hkv, L = 6, 8, 2, 512
+    Q, K, V = make_case(B, Hq, Hkv, L, seed=7)
+    lens = [512, 130, 0, 1, 256, 383]
+    got, _, _ = run_attention(Q, K, V, ag.KV_LOCAL, kv_len=lens)
+    check(got, oa.gqa_decode(Q, K, V, lens))
+    assert not got[2].any()
+    # zero queries: every output row is the mean of the value rows of its KV head
+    Q0 = np.zeros_like(Q)
+    got, _, _ = run_attention(Q0, K, V, ag.KV_INTERLEAVED)
+    Vf = oa.bf16_to_f64(V)
+    for b in range(B):
+        for hq in range(Hq):
+            assert np.abs(got[b, hq] - Vf[b, hq // 4].mean(axis=0)).max() <= 1e-5
+
+
+def test_serving_shape_on_sm_budgets():
+    """Batch 128, 512 keys, 8 KV heads, 32 query heads (the decode side of the paper's serving split): 1024 units."""
+    B, Hq, Hkv, L = 128, 32, 8, 512
+    Q, K, V = make_case(B, Hq, Hkv, L, seed=21)
+    want = oa.gqa_decode(Q, K, V)
+    for placement, budget in ((ag.KV_LOCAL, None), (ag.KV_REMOTE, None), (ag.KV_LOCAL, 74)):
+        got, _, _ = run_attention(Q, K, V, placement, budget=budget)
+        check(got, want)
+
+
+def test_bad_arguments():
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=4, N=128 * 8, K=256, tile_m=16,
+                                                                tile_n=128, k_splits=1))
+    dst = torch.zeros(16 << 20, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst.numel(), topo)
+    k = torch.zeros(8 * 256 * 128, dtype=torch.int16, device="cuda")
+    h = ag.C.c_void_p()
+    L_ = ag.lib()
+    # L not a multiple of 128, too long, wrong unit count, wrong head dimension
+    for (B, H, Lk, D) in ((4, 2, 200, 128), (4, 2, 2048, 128), (4, 4, 256, 128), (4, 2, 256, 64)):
+        st = L_.ag_kv_pack(k.data_ptr(), k.data_ptr(), B, H, Lk, D, plan.handle, amap.handle, dst.data_ptr(), dst.numel(), 0, ag.C.byref(h))
+        assert st == ag.AG_ERR_ARG
