@@ -256,6 +256,57 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
                          "peak_source": f"{peaks['source']} copy bandwidth"}}
 
 
+def attention_section(ag, inputs, torch, topo, peaks, sampler):
+    """Decode attention over a paged KV cache: batch 128, 32 query heads on 8 KV heads, 512 keys of 128 dimensions
+    (KV 256 MiB > L2, read once per call), one unit per (request, KV head), all SMs, calls queued back to back with
+    overlap_launches.  KV pages on the die of the SM that owns the unit, on the other die, and interleaved; the outputs
+    of the first eight requests are checked against the fp64 oracle."""
+    from oracle import attention as oa
+    B, Hq, Hkv, L, D = 128, 32, 8, 512, 128
+    Q = inputs.uniform_bf16(B * Hq, D, inputs.DEFAULT_SEED + 40).reshape(B, Hq, D)
+    K = inputs.uniform_bf16(B * Hkv * L, D, inputs.DEFAULT_SEED + 41).reshape(B, Hkv, L, D)
+    V = inputs.uniform_bf16(B * Hkv * L, D, inputs.DEFAULT_SEED + 42).reshape(B, Hkv, L, D)
+    dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16).copy()).cuda()
+    dQ, dK, dV = dev(Q), dev(K), dev(V)
+    dO = torch.empty((B, Hq, D), dtype=torch.float32, device="cuda")
+    kv_bytes = 2 * B * Hkv * L * D * 2
+    algo_bytes = kv_bytes + B * Hq * D * (2 + 4)
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
+                                                               tile_n=128, k_splits=1, overlap_launches=1))
+    dst_bytes = 2 * kv_bytes + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    want = oa.gqa_decode(Q[:8], K[:8], V[:8])
+    gbs, err, frac_local, launches0 = {}, {}, {}, ag.kernel_launch_count()
+    sampler.mark("attention")
+    for name, placement in (("die_local", ag.KV_LOCAL), ("remote", ag.KV_REMOTE), ("interleaved", ag.KV_INTERLEAVED)):
+        kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes, placement)
+        dO.fill_(float("nan"))
+        ag.attention_decode(dQ.data_ptr(), kv, None, dO.data_ptr(), B, Hq, plan)
+        torch.cuda.synchronize()
+        got = dO[:8].cpu().numpy().astype(np.float64)
+        err[name] = {"max_abs": float(np.abs(got - want).max()), "rel_fro": float(np.linalg.norm(got - want) / np.linalg.norm(want))}
+        ms = time_queued(torch, lambda: ag.attention_decode(dQ.data_ptr(), kv, None, dO.data_ptr(), B, Hq, plan))
+        if plan.last_status() != ag.AG_OK:
+            raise RuntimeError("attention arm " + name + ": " + ag.strerror(plan.last_status()))
+        gbs[name] = algo_bytes / (ms * 1e-3) / 1e9
+        frac_local[name] = kv.info()["local_fraction"]
+        del kv
+    sampler.close("attention")
+    best = gbs["die_local"]
+    return {"workload": f"GQA decode attention, batch {B}, {Hq} query heads on {Hkv} KV heads, {L} keys x {D} bf16, fp32 out, unit = (request, KV head), "
+                        f"all {topo.n_sm} SMs, KV 256 MiB > L2, launches queued back to back, overlap_launches",
+            "gbs": gbs, "us_per_call": {n: algo_bytes / v / 1e3 for n, v in gbs.items()},
+            "local_fraction_of_kv_bytes": frac_local,
+            "local_over_remote": gbs["die_local"] / gbs["remote"], "local_over_interleaved": gbs["die_local"] / gbs["interleaved"],
+            "oracle_error_on_o_first_8_requests": err,
+            "gpu_launches": int(ag.kernel_launch_count() - launches0),
+            "clocks": sampler.summary("attention"),
+            "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
+                         "traffic": None, "kernel": "k_attn_decode", "algorithmic_bytes": algo_bytes,
+                         "peak_source": f"{peaks['source']} copy bandwidth"}}
+
+
 def subset_section(ag, inputs, torch, topo, sampler, budget=64, n_subsets=8):
     """Equal-size SM sets: dense 4096^3 on `budget` SMs - seeded random subsets, the lowest ids, the die-compact and
     the GPC-spread set - all on the one-block kernel (128 x 256 tiles), so that only the placement differs."""
@@ -326,7 +377,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only", default="all", choices=["all", "headline", "decode"],
+    ap.add_argument("--only", default="all", choices=["all", "headline", "decode", "attention"],
                     help="profiling aid: leave out the decode-shaped and SM-set sections (headline) or everything but the decode-shaped section (decode)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -366,14 +417,14 @@ def main():
     t0 = time.time()
     topo = ag.topo_discover()
     t_topo = time.time() - t0
-    if args.only == "decode":
-        # profiling aid: the decode-shaped section alone
+    if args.only in ("decode", "attention"):
+        # profiling aid: the decode-shaped GEMM section or the attention section alone
         sampler = ClockSampler(local)
         sampler.start()
-        decode = decode_section(ag, inputs, torch, topo, peaks, sampler)
+        section = (decode_section if args.only == "decode" else attention_section)(ag, inputs, torch, topo, peaks, sampler)
         sampler.stop()
         if rank == 0:
-            print(json.dumps({"only": "decode", "decode": decode}))
+            print(json.dumps({"only": args.only, args.only: section}))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -491,6 +542,7 @@ def main():
     rot_clocks = sampler.summary("rotation")
 
     decode = decode_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
+    attention = attention_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
     subsets = subset_section(ag, inputs, torch, topo, sampler) if args.only == "all" else None
     sampler.stop()
 
@@ -565,6 +617,7 @@ def main():
         "value_per_sm_ghz": (value / (clocks["sm_mhz"] / 1e3)) if clocks.get("sm_mhz") else None,
         "sustained": sustained,
         "decode": decode,
+        "attention": attention,
         "sm_subsets": subsets,
         "aware_over_oblivious_raster": side["affinity"] / side["oblivious_raster"],
         "die_sm_count": list(topo.die_sm_count), "gpc_sm_count": list(topo.gpc_sm_count[:topo.n_gpc]),

@@ -245,14 +245,20 @@ typedef struct {
                                  next launch's thread blocks take over SMs as they become free and start streaming their
                                  weights; nothing of theirs is written before this launch has completed.  The caller
                                  promises that the inputs (A, B / packed weights) of a call are not produced by the call
-                                 directly before it.  0 = launches run strictly one after the other */
+                                 directly before it; for attention_decode_persistent the promise covers the key/value
+                                 pages only (the queries are read after the launch before has completed).
+                                 0 = launches run strictly one after the other */
     int32_t cluster_size;    /* die_compact / affinity: thread-block cluster size (1, 2, 4 or 8) of the kernel the SM set is
                                 meant for; 0 and 1 mean none.  For sizes above 2 the set is built from what can host such
                                 clusters: SMs never seen in a cluster larger than 2 (is_random, Section 5.1.1) are taken last,
                                 and every GPC contributes whole blocks of cluster_size normal SMs - a GPC hosts only
                                 floor(n / cluster_size) clusters on n SMs (Section 7.3: twelve SMs form three clusters of
                                 four but one cluster of eight).  ag_cluster_capacity counts what a set can host */
-    int32_t reserved2;
+    int32_t die_quota;       /* die_compact / affinity: how the units are shared between the dies.  0 = in proportion to the
+                                SMs the set has on each die (right for work that is bound by the SMs).  1 = equal shares for
+                                the dies that hold any SM of the set: for work bound by memory bandwidth whose operands are
+                                die-local, since every die's memory delivers the same bandwidth whatever its SM count (on a
+                                chip with 70 and 78 usable SMs the proportional split asks 5 % more of one die's memory) */
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;

@@ -47,7 +47,10 @@ Steps.
                            order, then ascending id) and last with random and unplaced SMs (same order).
   3. per-die SM counts n_d and rank of each chosen SM inside its die (ascending id).
   4. quotas q_d = floor(n_u * n_d / b); leftover units go one each to the dies in
-     descending order of (n_u * n_d mod b), tie -> lower die id.
+     descending order of (n_u * n_d mod b), tie -> lower die id.  With die_quota = 1 the dies that
+     hold SMs share the units equally instead (weights 1 in place of n_d, their number in place of
+     b): for work bound by memory bandwidth over die-local operands, each die's memory being as
+     fast as the other's whatever the die's SM count.
   5. unit -> die:
        oblivious    R[i] goes to S[i mod b]; the unit's die is that SM's die;
        die_compact  every raster group (g tile rows) is cut in two in raster order: die 0 takes the
@@ -97,7 +100,7 @@ def mix64(x: int) -> int:
 def default_policy(**kw) -> dict:
     p = dict(kind=OBLIVIOUS, seed=0, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1,
              k_unit=64, raster_group=1, preferred_die=-1, invert_affinity=0,
-             static_assign=1, min_margin=0, sm_select=0, pair_lists=0, cluster_size=1, avoid=(), a=None, b=None, c=None)
+             static_assign=1, min_margin=0, sm_select=0, pair_lists=0, cluster_size=1, die_quota=0, avoid=(), a=None, b=None, c=None)
     p.update(kw)
     return p
 
@@ -313,7 +316,11 @@ def build_plan(topo: dict, amap: dict | None, b: int, pol: dict) -> dict:
         rank.append(seen[d])
         seen[d] += 1
     slots_of_die = [[i for i, d in enumerate(sm_die) if d == dd] for dd in (0, 1)]
-    q = quotas(n_u, n_d, b)
+    if pol.get("die_quota", 0):
+        w = [1 if n > 0 else 0 for n in n_d]
+        q = quotas(n_u, w, sum(w))
+    else:
+        q = quotas(n_u, n_d, b)
 
     sm_q = [[] for _ in S]
     pair_lists = pol.get("pair_lists", 0)

@@ -35,11 +35,12 @@ constexpr int AT_STAGE_BYTES = 32 * 1024; // one K or V tile
 constexpr int AT_NPROD = 3;
 constexpr int AT_THREADS = (2 + kEpiWarps + AT_NPROD) * 32;
 constexpr int AT_Q_BYTES = AT_NQ * AT_D * 2;        // 4 KB
-constexpr int AT_P_BYTES = 2 * AT_NQ * AT_TILE * 2; // hi + lo parts of one tile: 8 KB
-constexpr int AT_PSLOTS = 2;
+constexpr int AT_NP = 2 * AT_MAXG;         // rows of a probability tile: 8 hi parts, 8 lo parts (one MMA adds both)
+constexpr int AT_P_BYTES = AT_NP * AT_TILE * 2;     // 4 KB
+constexpr int AT_PSLOTS = 4;
 constexpr int AT_SMEM_BYTES = AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + AT_PSLOTS * AT_P_BYTES + 1024 + 1024;
 constexpr uint32_t AT_SCOLS = AT_MAXT * AT_NQ;      // score columns of one unit buffer (128)
-constexpr uint32_t AT_BUFCOLS = AT_SCOLS + AT_NQ;   // + output columns
+constexpr uint32_t AT_BUFCOLS = AT_SCOLS + AT_NP;   // + output columns (hi-part and lo-part sums)
 constexpr uint32_t AT_TMEM_COLS = 512;
 
 struct AttnCtl {
@@ -56,7 +57,7 @@ struct AttnCtl {
     int member;
     int4 quick;
     float red_max[kEpiWarps][AT_MAXG];
-    float red_sum[kEpiWarps][AT_MAXG];
+    float red_sum[2][kEpiWarps][AT_MAXG];
 };
 
 struct AttnArgs {
@@ -66,6 +67,7 @@ struct AttnArgs {
     float* O;                     // [B][H_q][128]
     int H_kv, G, T, L;
     float scale_log2e;            // log2(e) / sqrt(D)
+    int release_next;             // 1: let the next launch on the stream start while this one is still running
 };
 
 __device__ __forceinline__ int unit_tiles(const AttnArgs& x, int u) {
@@ -87,6 +89,9 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     volatile int* abort_flag = &ctl->abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int my_sm = (int)smid();
+    // overlap_launches: the launch that follows on the stream may be scheduled as soon as every block of this one has
+    // got this far; its blocks move in as SMs become free
+    if (x.release_next && tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         ctl->abort_flag = 0;
         const int4 qk = p.quick[my_sm];
@@ -189,6 +194,9 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     // the G query rows of the unit (rows u G .. u G + G - 1 of the [B H_q][128] matrix) and whatever
                     // follows them up to 16 rows: the extra rows only produce columns nobody reads
                     const uint32_t bar = smem_u32(&ctl->q_full[j]);
+                    // the queries are the product of the launch before this one: with overlapping launches they are
+                    // read only after it has completed (the key/value pages are the caller's promise)
+                    if (nq == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
                     mbar_expect_tx(bar, AT_Q_BYTES);
                     tma_load_3d(q_base + j * AT_Q_BYTES, &tm_q, bar, 0, u * x.G, 0);
                 }
@@ -263,6 +271,8 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (lane == 0) {
             // ------------------------------------------------ MMA issuer: scores of unit i, then the outputs of unit i - 1
             constexpr uint32_t idesc = make_idesc_bf16(128, AT_NQ, 0, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(128, AT_NP, 0, 0);
+            static_assert(AT_NP == 16 && AT_MAXG == 8, "rows q and 8 + q of a probability tile are the two parts of query row q");
             const uint64_t dpage_t = make_smem_desc(0, 128, 256, 0);     // K and V pages: no swizzle, K-major (see ag_kv_pack)
             const uint64_t dsw_t = make_smem_desc(0, 16, 1024, 2);       // Q and P tiles: K-major, 128-byte swizzle
             const uint32_t full0 = smem_u32(&ctl->kv_full[0]), empty0 = smem_u32(&ctl->kv_empty[0]);
@@ -339,11 +349,9 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         const uint64_t dv = dpage_t | (uint64_t)((base + s * AT_STAGE_BYTES) >> 4);
                         const uint64_t dp = dsw_t | (uint64_t)((p_base + ps * AT_P_BYTES) >> 4);
 #pragma unroll
-                        for (int k8 = 0; k8 < AT_TILE / 16; ++k8) {   // 16 keys per step: page k8 of the tile
-                            const uint64_t dpk = dp + (k8 >> 2) * (2048u >> 4) + (k8 & 3) * 2;
-                            tc_mma_f16(d_o, dv + k8 * (4096u >> 4), dpk, idesc, (t | k8) ? 1u : 0u);
-                            tc_mma_f16(d_o, dv + k8 * (4096u >> 4), dpk + (4096u >> 4), idesc, 1u);   // the lo parts, 4 KB on
-                        }
+                        for (int k8 = 0; k8 < AT_TILE / 16; ++k8)     // 16 keys per step: page k8 of the tile; P: atom k8 / 4
+                            tc_mma_f16(d_o, dv + k8 * (4096u >> 4), dp + (k8 >> 2) * (2048u >> 4) + (k8 & 3) * 2, idesc_pv,
+                                       (t | k8) ? 1u : 0u);
                         tc_commit(empty0 + s * 8);
                         tc_commit(smem_u32(&ctl->p_empty[ps]));
                     }
@@ -362,14 +370,47 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------ softmax and epilogue: thread i of the four warps = key i of a tile
-        // (scores) and = output column d = i (outputs); tensor-memory lane i
+        // (scores) and = output column d = i (outputs); tensor-memory lane i.  The outputs of a unit are written after the
+        // probabilities of the next one, so that the wait for its last value tile is off the path to the next products.
         const int wq = warp & 3;                      // lane quarter this warp may read
         const int i_lane = wq * 32 + lane;
         const int widx = warp - 2;
         uint32_t nq = 0, pt = 0;
-        bool prior_done = false;
+        bool prior_done = false, ok = true;
         const int G = x.G;
-        for (uint32_t it = 0;; ++it) {
+        int pend_u = -1;                              // unit whose outputs are still to be written
+        auto write_outputs = [&](uint32_t np) -> bool {     // np: the unit's ordinal among the units with keys
+            const uint32_t j = np & 1;
+            if (!mbar_wait_warp(smem_u32(&ctl->o_full[j]), (np >> 1) & 1, abort_flag, limit)) {
+                if (lane == 0) report_timeout(p, 7);
+                return false;
+            }
+            tc_fence_after();
+            uint32_t vh[8], vl[8];
+            const uint32_t t_o = tmem_base + ((uint32_t)(wq * 32) << 16) + j * AT_BUFCOLS + AT_SCOLS;
+            tmem_ld_32x8(t_o, vh);
+            tmem_ld_32x8(t_o + AT_MAXG, vl);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->o_empty[j]));
+            float* out = x.O + (size_t)pend_u * G * AT_D + i_lane;
+#pragma unroll
+            for (int q = 0; q < AT_MAXG; ++q) {
+                if (q < G) {
+                    const float l = (ctl->red_sum[j][0][q] + ctl->red_sum[j][1][q]) + (ctl->red_sum[j][2][q] + ctl->red_sum[j][3][q]);
+                    out[(size_t)q * AT_D] = (__uint_as_float(vh[q]) + __uint_as_float(vl[q])) / l;
+                }
+            }
+            if (lane == 0 && wq == 0) {
+                p.tile_owner[pend_u] = my_sm;
+                if (p.unit_times) p.unit_times[2 * pend_u + 1] = globaltimer_ns();
+                atomicAdd(&p.tile_count[pend_u], 1);
+            }
+            pend_u = -1;
+            return true;
+        };
+        for (uint32_t it = 0; ok; ++it) {
             const int r = it % kRing;
             if (!mbar_wait_warp(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 6);
@@ -379,18 +420,19 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
             if (u < 0) break;
-            const int b = u / x.H_kv, h = u - b * x.H_kv;
+            const int b = u / x.H_kv;
             const int len = x.kv_len ? min(x.L, max(0, x.kv_len[b])) : x.L;
             const int n_t = (len + AT_TILE - 1) / AT_TILE;
-            float* out = x.O + ((size_t)b * x.H_kv * G + (size_t)h * G) * AT_D + i_lane;
             if (!prior_done) {      // nothing is written before everything launched earlier on the stream has completed
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 prior_done = true;
             }
             if (n_t == 0) {
+                float* out = x.O + (size_t)u * G * AT_D + i_lane;
                 for (int q = 0; q < G; ++q) out[(size_t)q * AT_D] = 0.f;
                 if (lane == 0 && wq == 0) {
                     p.tile_owner[u] = my_sm;
+                    if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
                     atomicAdd(&p.tile_count[u], 1);
                 }
                 continue;
@@ -402,32 +444,35 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             tc_fence_after();
             // ---- scores of this thread's key in every tile; running maximum per query row
-            float s[AT_MAXT][AT_MAXG];
-            float mx[AT_MAXG];
-#pragma unroll
-            for (int q = 0; q < AT_MAXG; ++q) mx[q] = -INFINITY;
+            uint32_t sv[AT_MAXT][AT_MAXG];
             const uint32_t t_s = tmem_base + ((uint32_t)(wq * 32) << 16) + j * AT_BUFCOLS;
 #pragma unroll
-            for (int t = 0; t < AT_MAXT; ++t) {
-                if (t < n_t) {
-                    uint32_t v[16];
-                    tmem_ld_32x16(t_s + t * AT_NQ, v);
-                    tmem_ld_wait();
-                    const bool valid = t * AT_TILE + i_lane < len;
-#pragma unroll
-                    for (int q = 0; q < AT_MAXG; ++q) {
-                        s[t][q] = valid ? __uint_as_float(v[q]) : -INFINITY;
-                        mx[q] = fmaxf(mx[q], s[t][q]);
-                    }
-                }
-            }
+            for (int t = 0; t < AT_MAXT; ++t)
+                if (t < n_t) tmem_ld_32x8(t_s + t * AT_NQ, sv[t]);
+            tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->s_empty[j]));      // the score columns may be overwritten
+            float mx[AT_MAXG];
+#pragma unroll
+            for (int q = 0; q < AT_MAXG; ++q) mx[q] = -INFINITY;
+#pragma unroll
+            for (int t = 0; t < AT_MAXT; ++t) {
+                if (t < n_t) {
+                    const bool valid = t * AT_TILE + i_lane < len;
+#pragma unroll
+                    for (int q = 0; q < AT_MAXG; ++q) {
+                        if (!valid) sv[t][q] = 0xff800000u;               // -inf: a key past the request's length
+                        mx[q] = fmaxf(mx[q], __uint_as_float(sv[t][q]));
+                    }
+                }
+            }
 #pragma unroll
             for (int q = 0; q < AT_MAXG; ++q) {
+                if (q < G) {
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mx[q] = fmaxf(mx[q], __shfl_xor_sync(0xffffffffu, mx[q], o));
+                    for (int o = 16; o > 0; o >>= 1) mx[q] = fmaxf(mx[q], __shfl_xor_sync(0xffffffffu, mx[q], o));
+                }
             }
             if (lane == 0) {
 #pragma unroll
@@ -436,8 +481,9 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
 #pragma unroll
             for (int q = 0; q < AT_MAXG; ++q)
-                mx[q] = fmaxf(fmaxf(ctl->red_max[0][q], ctl->red_max[1][q]), fmaxf(ctl->red_max[2][q], ctl->red_max[3][q]));
-            // ---- probabilities, tile by tile, into the ring of probability tiles (bf16 hi and lo parts)
+                mx[q] = fmaxf(fmaxf(ctl->red_max[0][q], ctl->red_max[1][q]), fmaxf(ctl->red_max[2][q], ctl->red_max[3][q])) * x.scale_log2e;
+            // ---- probabilities, tile by tile, into the ring of probability tiles: rows 0-7 the bf16 hi parts, rows
+            // 8-15 the lo parts (row = query row; the rows of query rows that do not exist stay zero)
             float sum[AT_MAXG];
 #pragma unroll
             for (int q = 0; q < AT_MAXG; ++q) sum[q] = 0.f;
@@ -445,72 +491,52 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint32_t chunk = (uint32_t)((i_lane & 63) >> 3), within = (uint32_t)(i_lane & 7) * 2u;
 #pragma unroll
             for (int t = 0; t < AT_MAXT; ++t) {
-                if (t < n_t) {
+                if (t < n_t && ok) {
                     const uint32_t ps = pt % AT_PSLOTS;
                     if (!mbar_wait_warp(smem_u32(&ctl->p_empty[ps]), ((pt / AT_PSLOTS) & 1) ^ 1, abort_flag, limit)) {
                         if (lane == 0) report_timeout(p, 7);
-                        break;
-                    }
-                    uint8_t* ptile = smem + AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + ps * AT_P_BYTES;
+                        ok = false;
+                    } else {
+                        uint8_t* ptile = smem + AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + ps * AT_P_BYTES;
 #pragma unroll
-                    for (int q = 0; q < AT_MAXG; ++q) {
-                        if (q < G) {
-                            const float pv = exp2f((s[t][q] - mx[q]) * x.scale_log2e);   // masked keys: exp2(-inf) = 0
-                            sum[q] += pv;
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(pv);
-                            const __nv_bfloat16 lo = __float2bfloat16_rn(pv - __bfloat162float(hi));
-                            const uint32_t off = atom + (uint32_t)q * 128u + ((chunk ^ (uint32_t)(q & 7)) << 4) + within;
-                            *reinterpret_cast<__nv_bfloat16*>(ptile + off) = hi;
-                            *reinterpret_cast<__nv_bfloat16*>(ptile + 4096 + off) = lo;
+                        for (int q = 0; q < AT_MAXG; ++q) {
+                            if (q < G) {
+                                // masked keys: exp2(-inf) = 0
+                                const float pv = exp2f(fmaf(__uint_as_float(sv[t][q]), x.scale_log2e, -mx[q]));
+                                sum[q] += pv;
+                                const __nv_bfloat16 hi = __float2bfloat16_rn(pv);
+                                const __nv_bfloat16 lo = __float2bfloat16_rn(pv - __bfloat162float(hi));
+                                const uint32_t off = atom + (uint32_t)q * 128u + ((chunk ^ (uint32_t)(q & 7)) << 4) + within;
+                                *reinterpret_cast<__nv_bfloat16*>(ptile + off) = hi;
+                                *reinterpret_cast<__nv_bfloat16*>(ptile + 1024 + off) = lo;
+                            }
                         }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[ps]));
+                        ++pt;
                     }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[ps]));
-                    ++pt;
                 }
             }
+            if (!ok) break;
 #pragma unroll
             for (int q = 0; q < AT_MAXG; ++q) {
+                if (q < G) {
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) sum[q] += __shfl_xor_sync(0xffffffffu, sum[q], o);
+                    for (int o = 16; o > 0; o >>= 1) sum[q] += __shfl_xor_sync(0xffffffffu, sum[q], o);
+                }
             }
             if (lane == 0) {
 #pragma unroll
-                for (int q = 0; q < AT_MAXG; ++q) ctl->red_sum[widx][q] = sum[q];
+                for (int q = 0; q < AT_MAXG; ++q) ctl->red_sum[j][widx][q] = sum[q];
             }
             asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
-            // ---- outputs: this thread's column d of every query row
-            if (!mbar_wait_warp(smem_u32(&ctl->o_full[j]), (nq >> 1) & 1, abort_flag, limit)) {
-                if (lane == 0) report_timeout(p, 7);
-                break;
-            }
-            tc_fence_after();
-            {
-                uint32_t v[16];
-                tmem_ld_32x16(tmem_base + ((uint32_t)(wq * 32) << 16) + j * AT_BUFCOLS + AT_SCOLS, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int q = 0; q < AT_MAXG; ++q) {
-                    if (q < G) {
-                        const float l = (ctl->red_sum[0][q] + ctl->red_sum[1][q]) + (ctl->red_sum[2][q] + ctl->red_sum[3][q]);
-                        out[(size_t)q * AT_D] = __uint_as_float(v[q]) / l;
-                    }
-                }
-            }
-            tc_fence_before();
-            // red_max / red_sum are reused by the next unit: everybody must have read them
-            asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
-            if (lane == 0) {
-                mbar_arrive(smem_u32(&ctl->o_empty[j]));
-                if (wq == 0) {
-                    p.tile_owner[u] = my_sm;
-                    if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
-                    atomicAdd(&p.tile_count[u], 1);
-                }
-            }
+            // ---- outputs of the unit before this one, while this one's value tiles stream in
+            if (pend_u >= 0) ok = write_outputs(nq - 1);
+            pend_u = u;
             ++nq;
         }
+        if (ok && pend_u >= 0 && !*abort_flag) write_outputs(nq - 1);
     }
     tc_fence_before();
     __syncthreads();
@@ -726,6 +752,13 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     cfg.blockDim = dim3(AT_THREADS);
     cfg.dynamicSmemBytes = AT_SMEM_BYTES;
     cfg.stream = stream;
+    const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0 && plan->lay.b == plan->lay.n_sm;
+    x.release_next = overlap ? 1 : 0;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
     const cudaError_t le = cudaLaunchKernelEx(&cfg, k_attn_decode, tm_q, tm0, tm1, gp, x);
     if (le != cudaSuccess) return launch_failed(plan, le);
     count_launch();

@@ -24,7 +24,7 @@ struct OperandDev {
 };
 struct PolicyDev {
     int kind, M, N, K, tile_m, tile_n, k_splits, k_unit, raster_group, preferred_die, invert, static_assign;
-    int sm_select, pair_lists, cluster_size, pad0;
+    int sm_select, pair_lists, cluster_size, die_quota;
     unsigned long long seed;
     long long min_margin;
     unsigned long long avoid[4];
@@ -206,10 +206,13 @@ __global__ void k_select_sms(const ag_topo_map* __restrict__ topo, PolicyDev pol
     image[lay.die_sm_count() + 0] = n_d[0];
     image[lay.die_sm_count() + 1] = n_d[1];
     // quotas: floor share, leftovers by largest remainder (tie -> lower die)
+    // (die_quota = 1: every die that holds SMs counts the same, whatever its SM count)
     long long q[2], rem[2];
+    const int w_d[2] = {pol.die_quota ? (n_d[0] > 0) : n_d[0], pol.die_quota ? (n_d[1] > 0) : n_d[1]};
+    const int w_all = w_d[0] + w_d[1];
     for (int d = 0; d < 2; ++d) {
-        q[d] = (long long)n_units * n_d[d] / b;
-        rem[d] = (long long)n_units * n_d[d] % b;
+        q[d] = (long long)n_units * w_d[d] / w_all;
+        rem[d] = (long long)n_units * w_d[d] % w_all;
     }
     long long left = n_units - q[0] - q[1];
     const int first = rem[1] > rem[0] ? 1 : 0;
@@ -536,6 +539,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         pd.seed = p.seed;
         pd.sm_select = p.sm_select;
         pd.cluster_size = p.cluster_size;
+        pd.die_quota = p.die_quota ? 1 : 0;
         pd.pair_lists = p.pair_lists ? 1 : 0;
         pd.min_margin = p.min_margin;
         for (int i = 0; i < 4; ++i) pd.avoid[i] = p.avoid_sm_mask[i];

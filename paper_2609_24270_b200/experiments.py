@@ -9,6 +9,7 @@
     python -m paper_2609_24270_b200.experiments --config gpc_bandwidth     # L2 bandwidth of k SMs: one GPC vs spread
     python -m paper_2609_24270_b200.experiments --config latency           # latency histograms from one SM per die
     python -m paper_2609_24270_b200.experiments --config cluster_sets      # cluster eligibility of equal-size SM sets
+    python -m paper_2609_24270_b200.experiments --config attention         # decode attention, KV pages local / remote / interleaved
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
 launches first, median of the timed launches.  torch is used for device memory, streams and events.
@@ -462,6 +463,53 @@ def cluster_sets(fh, topo, budgets=(64, 72, 96), n_subsets=16):
                       **{n: res[n] for n in ("lowest_ids", "highest_ids", "die_compact_tpc", "die_compact_cluster", "gpc_spread_cluster")}), fh)
 
 
+def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024)), budgets=None, overlap=1):
+    """Decode attention over a paged KV cache (Section 6.4's die-local KV direction): batch B, H_q query heads over
+    H_kv KV heads, L keys of 128 dimensions per head; pages of a unit on the die of the SM that owns it (local),
+    on the other die (remote) or wherever the allocation put them (interleaved).  GB/s of KV bytes."""
+    budgets = budgets or (topo.n_sm, topo.n_sm // 2, topo.n_sm // 4)
+    D = 128
+    for B, Hq, Hkv, L in shapes:
+        dK = torch.randn((B, Hkv, L, D), dtype=torch.bfloat16, device="cuda")
+        dV = torch.randn((B, Hkv, L, D), dtype=torch.bfloat16, device="cuda")
+        dQ = torch.randn((B, Hq, D), dtype=torch.bfloat16, device="cuda")
+        dO = torch.empty((B, Hq, D), dtype=torch.float32, device="cuda")
+        kv_bytes = 2 * B * Hkv * L * D * 2
+        algo = kv_bytes + B * Hq * D * (2 + 4)
+        dst_bytes = 2 * kv_bytes + (16 << 20)
+        dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+        amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+        lib_us = None
+        try:    # context: the library's fused attention on the same shapes (row-major cache)
+            q4 = dQ.view(B, Hq, 1, D)
+            f = lambda: torch.nn.functional.scaled_dot_product_attention(q4, dK, dV, enable_gqa=True)
+            lib_us = time_queued(f) * 1e3
+        except Exception as e:  # noqa: BLE001
+            lib_us = str(e)[:80]
+        for b in budgets:
+            for both in ((0, 1) if b < topo.n_sm else (0,)):
+                kw = dict(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16, tile_n=128, k_splits=1,
+                          sm_select=1 if both else 0, overlap_launches=overlap)
+                plan = ag.sched_build(topo, None, b, ag.make_policy(**kw))
+                plan_eq = ag.sched_build(topo, None, b, ag.make_policy(die_quota=1, **kw))   # units shared equally between the dies
+                res, info = {}, {}
+                for name, pl, pn in (("local", ag.KV_LOCAL, plan), ("local_equal_quota", ag.KV_LOCAL, plan_eq), ("remote", ag.KV_REMOTE, plan),
+                                     ("interleaved", ag.KV_INTERLEAVED, plan)):
+                    kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, pn, amap, dst.data_ptr(), dst_bytes, pl)
+                    ms = time_queued(lambda: ag.attention_decode(dQ.data_ptr(), kv, None, dO.data_ptr(), B, Hq, pn))
+                    assert pn.last_status() == ag.AG_OK
+                    res[name] = dict(us=ms * 1e3, gbs=algo / (ms * 1e-3) / 1e9)
+                    info[name] = kv.info()["local_fraction"]
+                    del kv
+                emit(dict(config="attention", B=B, H_q=Hq, H_kv=Hkv, L=L, kv_gb=kv_bytes / 1e9, sm_budget=b,
+                          sm_set="gpc_spread" if both else "die_compact", sets=sm_set_summary(topo, plan), results=res,
+                          local_fraction=info, local_over_remote=res["remote"]["us"] / res["local"]["us"],
+                          local_over_interleaved=res["interleaved"]["us"] / res["local"]["us"],
+                          overlap_launches=int(bool(overlap and b == topo.n_sm)), library_sdpa_us=lib_us), fh)
+        del dst, amap, dK, dV
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -473,7 +521,7 @@ def main():
               gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
-     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets}[args.config](fh, topo)
+     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention}[args.config](fh, topo)
 
 
 if __name__ == "__main__":

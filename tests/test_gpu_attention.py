@@ -31,13 +31,13 @@ def dev(bits):
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16).copy()).cuda()
 
 
-def run_attention(Q, K, V, placement, kv_len=None, budget=None):
+def run_attention(Q, K, V, placement, kv_len=None, budget=None, overlap=0):
     B, Hq, D = Q.shape
     _, Hkv, L, _ = K.shape
     topo = device_topo()
     b = topo.n_sm if budget is None else budget
     plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
-                                                        tile_n=128, k_splits=1))
+                                                        tile_n=128, k_splits=1, overlap_launches=overlap))
     kv_bytes = 2 * B * Hkv * L * D * 2
     dst_bytes = (2 * kv_bytes if placement != ag.KV_INTERLEAVED else kv_bytes) + (8 << 20)
     dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
@@ -97,8 +97,9 @@ def test_serving_shape_on_sm_budgets():
     B, Hq, Hkv, L = 128, 32, 8, 512
     Q, K, V = make_case(B, Hq, Hkv, L, seed=21)
     want = oa.gqa_decode(Q, K, V)
-    for placement, budget in ((ag.KV_LOCAL, None), (ag.KV_REMOTE, None), (ag.KV_LOCAL, 74)):
-        got, _, _ = run_attention(Q, K, V, placement, budget=budget)
+    # the last one with overlapping launches (the second launch begins while the first one finishes)
+    for placement, budget, overlap in ((ag.KV_LOCAL, None, 0), (ag.KV_REMOTE, None, 0), (ag.KV_LOCAL, 74, 0), (ag.KV_LOCAL, None, 1)):
+        got, _, _ = run_attention(Q, K, V, placement, budget=budget, overlap=overlap)
         check(got, want)
 
 

@@ -51,6 +51,23 @@ def test_gpc_spread_selection_matches_oracle(b):
         assert got.tobytes() == want.tobytes()
 
 
+@pytest.mark.parametrize("b", [16, 37, 74, 111, 148])
+def test_equal_die_quota_matches_oracle(b):
+    """die_quota = 1 (equal shares for the dies that hold SMs): bytewise equal to the oracle."""
+    for die0 in (70, 74):
+        topo = inputs.synthetic_topo(die0_sms=die0, seed=die0 + 1)
+        for kw in (dict(M=16, N=8192, K=8192, tile_m=16, tile_n=128, k_splits=8), dict(M=4, N=128 * 1000 + 128, K=512, tile_m=16, tile_n=128),
+                   dict(M=4096, N=4096, K=4096, raster_group=4)):
+            for sel in (0, 1):
+                got, want, plan = both(topo, None, b, kind=ag.AG_DIE_COMPACT, die_quota=1, sm_select=sel, **kw)
+                assert got.tobytes() == want.tobytes()
+                p = plan.parsed()
+                n_d = [int(x) for x in p["die_sm_count"]]
+                if min(n_d) > 0:
+                    q0 = int(p["die_q_off"][1])
+                    assert abs(2 * q0 - int(p["n_units"])) <= 1
+
+
 @pytest.mark.parametrize("c", [4, 8])
 @pytest.mark.parametrize("b", [10, 32, 64, 72, 100, 140, 148])
 def test_cluster_aware_sets_match_oracle(c, b):

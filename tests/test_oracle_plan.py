@@ -101,6 +101,29 @@ def test_quota_proportional_to_die_sm_count():
             assert abs(q[0] / n_u - n0 / 148) <= 1.0 / n_u + 1e-12
 
 
+def test_equal_die_quota_splits_by_dies_not_by_sms():
+    """die_quota = 1: hand values on a two-die toy chip (3 + 5 SMs, 10 units in one row of tiles)."""
+    topo = dict(n_sm=8, n_tpc=4, n_gpc=2, n_die=2, tpc=np.array([0, 0, 1, 1, 2, 2, 3, 3]), gpc=np.array([0] * 4 + [1] * 4),
+                die=np.array([0, 0, 0, 1, 1, 1, 1, 1]), is_random=np.zeros(8, dtype=np.int32), gpc_die=[0, 1],
+                die_sm_count=[3, 5], gpc_sm_count=[4, 4])
+    base = dict(kind=op.DIE_COMPACT, M=16, N=1280, K=64, tile_m=16, tile_n=128)
+    prop = op.build_plan(topo, None, 8, op.default_policy(**base))
+    # proportional: floor(10 * 3 / 8) = 3 and floor(10 * 5 / 8) = 6, the unit left over goes to the larger remainder
+    # (30 mod 8 = 6 against 50 mod 8 = 2): die 0
+    assert [len(q) for q in prop["die_q"]] == [4, 6]
+    equal = op.build_plan(topo, None, 8, op.default_policy(die_quota=1, **base))
+    assert [len(q) for q in equal["die_q"]] == [5, 5]
+    assert equal["die_q"] == [[0, 1, 2, 3, 4], [5, 6, 7, 8, 9]]          # contiguous bands in raster order
+    # entry i of a die's queue goes to the SM of rank i mod n_d: die 0's three SMs hold 2, 2, 1 units
+    assert [equal["sm_q"][i] for i in range(3)] == [[0, 3], [1, 4], [2]]
+    # a set with all its SMs on one die keeps everything there
+    one = op.build_plan(topo, None, 4, op.default_policy(die_quota=1, preferred_die=1, **base))
+    assert [len(q) for q in one["die_q"]] == [0, 10]
+    # odd unit count: the unit left over goes to the lower die (equal remainders)
+    odd = op.build_plan(topo, None, 8, op.default_policy(die_quota=1, **dict(base, N=1408)))
+    assert [len(q) for q in odd["die_q"]] == [6, 5]
+
+
 def test_mixer_published_vectors():
     # splitmix64 seeded with 0: published first three outputs
     assert op.mix64(0) == 0xE220A8397B1DCDAF
