@@ -269,26 +269,36 @@ def config5(fh, topo):
 
 
 # ---------------------------------------------------------------------------------------------
-def raster(fh, topo):
+RASTER_ARMS = [(g, name) for g in (1, 2, 4, 8, 16, 32) for name in ("oblivious", "die_compact")]
+
+
+def raster(fh, topo, traffic_only=False):
+    """Raster-group sweep of the headline GEMM (8192^3, 256x256 units on block pairs): TFLOP/s per group height and
+    policy.  With traffic_only every arm is launched exactly once, in the order of RASTER_ARMS, so that a profiler's
+    launch list can be matched to the arms (DRAM bytes per launch)."""
     M = N = K = 8192
     A, B = inputs.gemm_inputs(M, N, K)
     dA, dB = dev_bf16(A), dev_bf16(B)
     dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
     flops = 2.0 * M * N * K
     plans = {}
-    for g in (1, 2, 4, 8, 16, 32, 64):
-        for kind, name in ((ag.AG_OBLIVIOUS, "oblivious"), (ag.AG_DIE_COMPACT, "die_compact")):
-            for static in (1, 0):
-                plans[(g, name, static)] = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(
-                    kind=kind, M=M, N=N, K=K, raster_group=g, static_assign=static))
+    for g, name in RASTER_ARMS:
+        kind = ag.AG_OBLIVIOUS if name == "oblivious" else ag.AG_DIE_COMPACT
+        plans[(g, name)] = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=kind, M=M, N=N, K=K, tile_m=256, tile_n=256,
+                                                                                raster_group=g))
+    if traffic_only:
+        for i, (k, plan) in enumerate(plans.items()):
+            ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan)
+            torch.cuda.synchronize()
+            emit(dict(config="raster_traffic", launch=i, raster_group=k[0], policy=k[1]), fh)
+        return
     acc = {k: [] for k in plans}
     for _ in range(3):
         for k, plan in plans.items():
             acc[k] += time_launches(lambda: ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan),
-                                    warmup=2, iters=6)
-    for (g, name, static), v in acc.items():
-        emit(dict(config="raster", raster_group=g, policy=name, static_assign=static,
-                  tflops=flops / (float(np.median(v)) * 1e-3) / 1e12), fh)
+                                    warmup=2, iters=6, batches=1)
+    for (g, name), v in acc.items():
+        emit(dict(config="raster", raster_group=g, policy=name, tflops=flops / (float(np.median(v)) * 1e-3) / 1e12), fh)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -521,7 +531,8 @@ def main():
               gpc_sm_count=list(topo.gpc_sm_count[:topo.n_gpc]), gpc_die=list(topo.gpc_die[:topo.n_gpc]),
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
-     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention}[args.config](fh, topo)
+     "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention,
+     "raster_traffic": lambda f, t: raster(f, t, traffic_only=True)}[args.config](fh, topo)
 
 
 if __name__ == "__main__":
