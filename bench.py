@@ -186,10 +186,12 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
     """The HBM-bound workload: M = 16, N = K = 8192 (weights 128 MiB, read once per call), 128-column units x 16
     k-splits on all SMs, split-K by reductions in memory, four weight matrices in rotation so that no call finds its
     weights in L2, calls queued back to back with overlap_launches.  Die-local packed weights under the die-compact
-    plan, the same packed weights under the deliberately remote plan, and row-major weights under the oblivious and
-    die-compact plans; C of the first call is checked against the fp64 oracle."""
+    plan, the same packed weights under the deliberately remote plan, row-major weights under the oblivious and
+    die-compact plans, and the die-local arm in the bit-reproducible split-K mode (slices through a workspace, added in
+    ascending order by a second kernel); the same arms once more with 4 k-splits.  C of the first call is checked
+    against the fp64 oracle."""
     from oracle import gemm as og
-    Md, Nd, Kd, ksp, n_buf = 16, 8192, 8192, 16, 4
+    Md, Nd, Kd, n_buf = 16, 8192, 8192, 4
     A_bits = inputs.uniform_bf16(Md, Kd, inputs.DEFAULT_SEED)
     B_bits = [inputs.uniform_bf16(Kd, Nd, inputs.DEFAULT_SEED + 1 + i) for i in range(n_buf)]
     dev = lambda bits: torch.from_numpy(bits.view(np.int16).copy()).cuda()
@@ -197,61 +199,70 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
     dBs = [dev(b) for b in B_bits]
     dC = torch.empty((Md, Nd), dtype=torch.float32, device="cuda")
     algo_bytes = Kd * Nd * 2 + Md * Kd * 2 + Md * Nd * 4
-    kw = dict(M=Md, N=Nd, K=Kd, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=1, overlap_launches=1)
-    plan_local = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
-    plan_obl = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))
     dst_bytes = 2 * Kd * Nd * 2 + (8 << 20)
-    dsts, packs = [], []
-    for i in range(n_buf):
-        dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
-        amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
-        packs.append((ag.pack_weights(dBs[i].data_ptr(), Kd, Nd, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
-        dsts.append(dst)
-    bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packs[0][0].page_table())
-    plan_remote = ag.sched_build(topo, packs[0][1], topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
-    # parity of what is timed: first call of the packed die-local arm and of the row-major oblivious arm
+    dsts = [torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_buf)]
+    amaps = [ag.affinity_probe(d.data_ptr(), dst_bytes, topo) for d in dsts]
     want = og.gemm_blocked(A_bits, B_bits[0])
-    err = {}
-    for name, call in (("packed_die_local", lambda: ag.gemm_persistent_packed(dA.data_ptr(), packs[0][0], dC.data_ptr(), Md, Nd, Kd, plan_local)),
-                       ("rowmajor_oblivious", lambda: ag.gemm_persistent(dA.data_ptr(), dBs[0].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan_obl))):
-        dC.fill_(float("nan"))
-        call()
-        torch.cuda.synchronize()
-        got = dC.cpu().numpy().astype(np.float64)
-        err[name] = {"max_abs": float(np.abs(got - want).max()), "rel_fro": float(np.linalg.norm(got - want) / np.linalg.norm(want))}
-    gbs, launches0 = {}, ag.kernel_launch_count()
+    launches0 = ag.kernel_launch_count()
+    results, err, info = {}, {}, {}
     sampler.mark("decode")
-    arms = (("packed_die_local", plan_local, True), ("packed_remote", plan_remote, True),
-            ("rowmajor_oblivious", plan_obl, False), ("rowmajor_die_compact", plan_local, False))
-    for _ in range(2):                                    # two passes so that the arms share the clock drift
-        for name, plan, packed in arms:
-            state = {"i": 0}
+    for ksp in (16, 4):
+        kw = dict(M=Md, N=Nd, K=Kd, tile_m=16, tile_n=128, k_splits=ksp, overlap_launches=1)
+        plan_local = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, splitk_in_memory=1, **kw))
+        plan_ws = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, splitk_in_memory=0, **kw))
+        plan_obl = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, splitk_in_memory=1, **kw))
+        packs = [ag.pack_weights(dBs[i].data_ptr(), Kd, Nd, plan_local, amaps[i], dsts[i].data_ptr(), dst_bytes) for i in range(n_buf)]
+        bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packs[0].page_table())
+        plan_remote = ag.sched_build(topo, amaps[0], topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, splitk_in_memory=1,
+                                                                              b=bop, **kw))
+        if ksp == 16:
+            # parity of what is timed: first call of the packed die-local arm (both split-K modes) and of the row-major oblivious arm
+            for name, call in (("packed_die_local", lambda: ag.gemm_persistent_packed(dA.data_ptr(), packs[0], dC.data_ptr(), Md, Nd, Kd, plan_local)),
+                               ("packed_die_local_workspace_split_k", lambda: ag.gemm_persistent_packed(dA.data_ptr(), packs[0], dC.data_ptr(), Md, Nd, Kd, plan_ws)),
+                               ("rowmajor_oblivious", lambda: ag.gemm_persistent(dA.data_ptr(), dBs[0].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan_obl))):
+                dC.fill_(float("nan"))
+                call()
+                torch.cuda.synchronize()
+                got = dC.cpu().numpy().astype(np.float64)
+                err[name] = {"max_abs": float(np.abs(got - want).max()), "rel_fro": float(np.linalg.norm(got - want) / np.linalg.norm(want))}
+            info = {"group_free_bit": packs[0].group_free_bit(), "closed_form_remap": packs[0].closed_form()}
+        gbs = {}
+        arms = (("packed_die_local", plan_local, True), ("packed_remote", plan_remote, True),
+                ("rowmajor_oblivious", plan_obl, False), ("rowmajor_die_compact", plan_local, False),
+                ("packed_die_local_workspace_split_k", plan_ws, True))
+        for _ in range(2):                                    # two passes so that the arms share the clock drift
+            for name, plan, packed in arms:
+                state = {"i": 0}
 
-            def run():
-                i = state["i"] % n_buf
-                state["i"] += 1
-                if packed:
-                    ag.gemm_persistent_packed(dA.data_ptr(), packs[i][0], dC.data_ptr(), Md, Nd, Kd, plan)
-                else:
-                    ag.gemm_persistent(dA.data_ptr(), dBs[i].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan)
-            ms = time_queued(torch, run)
-            if plan.last_status() != ag.AG_OK:
-                raise RuntimeError("decode arm " + name + ": " + ag.strerror(plan.last_status()))
-            gbs.setdefault(name, []).append(algo_bytes / (ms * 1e-3) / 1e9)
+                def run():
+                    i = state["i"] % n_buf
+                    state["i"] += 1
+                    if packed:
+                        ag.gemm_persistent_packed(dA.data_ptr(), packs[i], dC.data_ptr(), Md, Nd, Kd, plan)
+                    else:
+                        ag.gemm_persistent(dA.data_ptr(), dBs[i].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan)
+                ms = time_queued(torch, run)
+                if plan.last_status() != ag.AG_OK:
+                    raise RuntimeError("decode arm " + name + ": " + ag.strerror(plan.last_status()))
+                gbs.setdefault(name, []).append(algo_bytes / (ms * 1e-3) / 1e9)
+        results[ksp] = {n: float(np.median(v)) for n, v in gbs.items()}
+        del packs
     sampler.close("decode")
-    gbs = {n: float(np.median(v)) for n, v in gbs.items()}
+    gbs = results[16]
     best = gbs["packed_die_local"]
-    return {"workload": f"GEMM M={Md} N=K={Nd} bf16, fp32 out, 128-col units x {ksp} k-splits (in-memory reductions), all {topo.n_sm} SMs, "
+    return {"workload": f"GEMM M={Md} N=K={Nd} bf16, fp32 out, 128-col units x 16 k-splits (in-memory reductions), all {topo.n_sm} SMs, "
                         f"{n_buf} rotating weight matrices (512 MiB > L2), launches queued back to back, overlap_launches",
             "gbs": gbs, "us_per_call": {n: algo_bytes / v / 1e3 for n, v in gbs.items()},
+            "gbs_4_k_splits": results[4],
             "local_over_remote": gbs["packed_die_local"] / gbs["packed_remote"],
             "aware_over_oblivious": gbs["packed_die_local"] / gbs["rowmajor_oblivious"],
-            "group_free_bit": packs[0][0].group_free_bit(),
-            "closed_form_remap": packs[0][0].closed_form(),
+            "group_free_bit": info["group_free_bit"],
+            "closed_form_remap": info["closed_form_remap"],
             "oracle_error_on_c": err,
             "gpu_launches": int(ag.kernel_launch_count() - launches0),
             "clocks": sampler.summary("decode"),
             "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
+                         "frac_4_k_splits": results[4]["packed_die_local"] / peaks["hbm_gbs"],
                          "traffic": None, "kernel": "k_gemm_skinny<16, packed>", "algorithmic_bytes": algo_bytes,
                          "peak_source": f"{peaks['source']} copy bandwidth"}}
 

@@ -232,7 +232,8 @@ typedef struct {
     uint64_t seed;           /* oblivious only: 0 = lowest SM ids, else seeded random subset */
     int64_t min_margin;      /* affinity only: byte margins below this count as ties (0 = exact ties only) */
     int32_t splitk_in_memory; /* decode-shaped plans with k_splits > 1: 0 = partial sums go through a
-                                 workspace and are added in ascending split order (bit-reproducible);
+                                 workspace and are added in ascending split order by a small second kernel
+                                 launched behind the GEMM (bit-reproducible);
                                  1 = C is zeroed and every unit adds its partial sums with reductions in
                                  memory (no workspace, no waiting; the order of the fp32 adds is not fixed) */
     int32_t sm_select;       /* die_compact / affinity: 0 = primary die first (die-compact set); 1 = whole TPCs dealt
@@ -409,7 +410,7 @@ void ag_packed_destroy(ag_packed_weights* w);
  *   A  device, M x K bf16 row-major, 16-byte aligned;  C  device, M x N fp32 row-major, overwritten
  *   plan  same N, K (and tile_n) as the packing; decode-shaped plans: with
  *         k_splits > 1 the partial sums either go through the plan's workspace and are added in
- *         ascending split order by the block that finishes a tile last, or are added straight
+ *         ascending split order by a second kernel launched behind the GEMM, or are added straight
  *         into a zeroed C by reductions in memory (policy.splitk_in_memory)
  * Asynchronous on cuda_stream.  Errors as gemm_persistent.
  */
@@ -462,7 +463,7 @@ ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weight
  * Who needs it: a serving process whose own memory pool already owns all of the GPU's free memory,
  * so that cudaMalloc fails; a latency-bound request loop where an allocator call is not
  * acceptable; code that runs after a framework has declared "no more allocations".  The split-K
- * partial sums and arrival counters, which normally live in memory that sched_build attached to
+ * partial sums, which normally live in memory that sched_build attached to
  * the plan, are placed instead in a fixed workspace that is part of the library image: 8 MiB +
  * 16 KiB of device memory per GPU.  The CUDA runtime loads the library's device code onto a GPU
  * when it is first used there, so the workspace (and the kernel itself) takes its memory during
@@ -477,9 +478,8 @@ ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weight
  * sched_build done at start-up, when allocation was still allowed.
  *
  * The first call on each device also looks up the workspace's device address; make that first call
- * before any stream capture.  All calls on a device share the one workspace, which keeps
- * whatever the previous call left in it (the counters are cleared on the given stream at the
- * start of every call): two calls whose kernels may run at the same time on one GPU - different
+ * before any stream capture.  All calls on a device share the one workspace (every call
+ * overwrites the slices it uses before it reads them): two calls whose kernels may run at the same time on one GPU - different
  * streams, or different host threads - race on it and give wrong results.  Serialise them.
  * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA; device-side status via ag_last_status.
  */

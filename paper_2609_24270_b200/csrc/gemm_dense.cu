@@ -380,7 +380,7 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
     if (!A || !B || !Cout || !plan) return AG_ERR_ARG;
     const int32_t* h = plan->header;
     if (h[H_TILE_M] <= 32)  // decode-shaped plan: weights on the MMA's M side, split-K through the plan's scratch
-        return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
+        return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, plan->d_partial,
                                     reinterpret_cast<cudaStream_t>(cuda_stream));
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_M] == 256)  // 256 x 256 units: pairs of blocks, full-chip plans only

@@ -9,8 +9,8 @@
 // (indirect allocation by remapping, Section 7.1.1 of the paper).  A packed page is fetched with
 // one 4 KB bulk copy whose source address comes from the page table.
 //
-// Split-K units write partial sums to a scratch workspace; the block that completes a tile's
-// last split adds them in ascending split order (deterministic) and writes C.
+// Split-K units either add their sums into a zeroed C with reductions in memory, or write them to a workspace
+// whose slices a second kernel (k_reduce_splits) adds in ascending split order (bit-reproducible).
 #include <string.h>
 
 #include <algorithm>
@@ -74,7 +74,6 @@ struct SkinnyArgs {
     int pages_per_tile;
     float* C;
     float* partial;               // [k_splits][M][N] or null when k_splits == 1
-    int* sem;                     // [tiles_n * 4]: one arrival counter per 32-column quarter of a tile
     // grouped (MoE-shaped) operation: the plan's N is G experts side by side, expert g = column tiles
     // [g * tiles_per_group, (g + 1) * tiles_per_group); null / 0 when there is a single problem
     const CUtensorMap* g_tm_a;    // device [G]: activations of expert g (rows of the stacked A)
@@ -455,82 +454,27 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------ epilogue: lane = weight column n, registers = rows m
-        // Split-K hand-off, software-pipelined so that no memory round trip sits between two units:
-        //   unit i    its partial sums are stored;
-        //   unit i-1  (stores acknowledged long ago) fence, then the arrival counter of its 32 columns
-        //             is bumped with an atomic whose result is not looked at yet;
-        //   unit i-2  the atomic's result is read: the warp that completed the last of the k_splits
-        //             partial sums adds them in ascending split order and writes C.
-        // Each epilogue warp owns 32 columns of a tile and its own counter; no barrier between warps.
+        // Each epilogue warp owns 32 columns of a tile.  Split-K: either every unit adds its sums to C with reductions
+        // in memory (C zeroed beforehand), or it stores them to its split's slice of the workspace and the kernel
+        // launched behind this one (k_reduce_splits) adds the slices in ascending split order.
         const int q = warp & 3;
-        uint32_t tile_it = 0, it = 0;
-        int st_tn = -1;              // unit whose partial sums are stored but not yet announced
-        int at_tn = -1;              // unit whose arrival atomic is in flight
-        int oldA = 0, oldB = 0;      // results of the arrival atomics (lane 0), used one unit later
+        uint32_t tile_it = 0;
         bool prior_done = false;     // everything launched before this kernel is known to be complete
-
-        auto reduce_columns = [&](int tn) {
-            __threadfence();
-            // lane = (row group lane/8, four columns); the k_splits loads of one output quad are in flight
-            // together and are added in ascending split order
-            const int nq = tn * SK_BN + q * 32 + (lane & 7) * 4;
-            const OutView ov = out_view(p, x, tn);
-            const int nlq = ov.col0 + q * 32 + (lane & 7) * 4;
-            if (nq < p.N && nlq < ov.n_cols) {
-                for (int m = lane >> 3; m < ov.rows; m += 4) {
-                    float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
-                        float4 t[8];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            if (k0 + k < p.k_splits)
-                                t[k] = __ldcg(reinterpret_cast<const float4*>(
-                                    x.partial + ((size_t)(k0 + k) * p.M + m) * p.N + nq));
-#pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            if (k0 + k < p.k_splits) {
-                                acc4.x += t[k].x; acc4.y += t[k].y; acc4.z += t[k].z; acc4.w += t[k].w;
-                            }
-                    }
-                    *reinterpret_cast<float4*>(ov.base + (size_t)m * ov.ld + nlq) = acc4;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) x.sem[tn * 4 + q] = 0;  // ready for the next launch
-        };
-        // announce the stored unit (atomic result lands in old_new), resolve the one announced before
-        auto hand_off = [&](int& old_use, int& old_new) {
-            const int announce = st_tn, resolve = at_tn;
-            if (announce >= 0) {
-                __threadfence();
-                __syncwarp();
-                if (lane == 0)
-                    asm volatile("atom.global.add.u32 %0, [%1], 1;" : "=r"(old_new) : "l"(x.sem + announce * 4 + q) : "memory");
-            }
-            if (resolve >= 0) {
-                const int last = __shfl_sync(0xffffffffu, old_use == p.k_splits - 1, 0);
-                if (last) reduce_columns(resolve);
-            }
-            at_tn = announce;
-            st_tn = -1;
-        };
-        // one unit; returns false when the list is finished (or a wait ran out)
-        auto one_unit = [&](int& old_use, int& old_new) -> bool {
+        for (uint32_t it = 0;; ++it) {
             const int r = it % kRing;
             if (!mbar_wait_warp(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 6);
-                return false;
+                break;
             }
             const int u = ctl->ring[r];
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
-            ++it;
-            if (u < 0) return false;
+            if (u < 0) break;
             const int ks = u % p.k_splits, tn = (u / p.k_splits) % p.tiles_n;
             const uint32_t acc = tile_it & 1;
             if (!mbar_wait_warp(smem_u32(&ctl->tmem_full[acc]), (tile_it >> 1) & 1, abort_flag, limit)) {
                 if (lane == 0) report_timeout(p, 7);
-                return false;
+                break;
             }
             tc_fence_after();
             float sum[NM];
@@ -546,9 +490,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
             ++tile_it;
-            // This kernel may have started while the one before it (the zeroing of C, or with overlap_launches the
-            // previous GEMM) was still running (programmatic dependent launch): before the first byte is written,
-            // make sure that everything before it on the stream has completed.
+            // This kernel may have started while the one before it (the zeroing of C, the adding-up of the previous
+            // call's workspace, or with overlap_launches the previous GEMM) was still running (programmatic dependent
+            // launch): before the first byte is written, make sure that everything before it on the stream has completed.
             if (!prior_done) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 prior_done = true;
@@ -557,23 +501,19 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const OutView ov = out_view(p, x, tn);
             const int nl = ov.col0 + q * 32 + lane;       // column inside the tile's problem
             if (p.k_splits > 1 && x.partial == nullptr) {
-                // in-memory reduction: C is zeroed by the kernel launched just before this one, every unit adds
-                // its partial sums with reductions that L2 carries out; nothing comes back, so nothing is
-                // waited for
+                // in-memory reduction: L2 carries out the additions; nothing comes back, so nothing is waited for
                 if (nl < ov.n_cols) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m)
                         if (m < ov.rows) atomicAdd(ov.base + (size_t)m * ov.ld + nl, sum[m]);
                 }
             } else if (p.k_splits > 1) {
-                hand_off(old_use, old_new);
                 float* out = x.partial + (size_t)ks * p.M * p.N;   // workspace rows: the plan's M bound, columns: the plan's N
                 if (n < p.N) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m)
                         if (m < p.M) out[(size_t)m * p.N + n] = sum[m];
                 }
-                st_tn = tn;
             } else if (nl < ov.n_cols) {
 #pragma unroll
                 for (int m = 0; m < NM; ++m)
@@ -581,22 +521,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             }
             if (lane == 0 && q == 0) {
                 p.tile_owner[u] = my_sm;
-                    if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
+                if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
                 atomicAdd(&p.tile_count[u], 1);
             }
-            return true;
-        };
-        // two copies of the step with the roles of oldA / oldB swapped: the atomic's result register is
-        // never copied, so nothing waits for it before the step that needs it
-        int which = 0;
-        while (true) {
-            if (!one_unit(oldA, oldB)) { which = 0; break; }
-            if (!one_unit(oldB, oldA)) { which = 1; break; }
-        }
-        if (p.k_splits > 1 && x.partial != nullptr && !*abort_flag) {
-            // drain: `which` = 0 means the atomic in flight wrote oldA (next result goes to oldB)
-            if (which == 0) { hand_off(oldA, oldB); hand_off(oldB, oldA); }
-            else            { hand_off(oldB, oldA); hand_off(oldA, oldB); }
         }
     }
     tc_fence_before();
@@ -615,6 +542,35 @@ __global__ void k_zero_f32(float4* __restrict__ p, size_t n_vec) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x)
         p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// Adds the k_splits slices of the workspace in ascending split order and writes C (the bit-reproducible split-K
+// mode).  One thread per four consecutive columns of one row; the k_splits loads of a thread are in flight together.
+// Launched behind the GEMM with programmatic stream serialization: its blocks may become resident while the GEMM
+// runs, release the launch behind them at once and wait for the GEMM's completion before the first load.
+__global__ void __launch_bounds__(256) k_reduce_splits(const PersistParams p, const SkinnyArgs x) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int quads_per_row = (p.N + 3) / 4;
+    const long long total = (long long)p.M * quads_per_row;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int m = (int)(i / quads_per_row), n = (int)(i % quads_per_row) * 4;
+        const int tn = n / SK_BN;
+        const OutView ov = out_view(p, x, tn);
+        const int nl = ov.col0 + (n - tn * SK_BN);
+        if (m >= ov.rows || nl >= ov.n_cols) continue;
+        float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
+            float4 t[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k0 + k < p.k_splits) t[k] = __ldcg(reinterpret_cast<const float4*>(x.partial + ((size_t)(k0 + k) * p.M + m) * p.N + n));
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k0 + k < p.k_splits) { acc4.x += t[k].x; acc4.y += t[k].y; acc4.z += t[k].z; acc4.w += t[k].w; }
+        }
+        *reinterpret_cast<float4*>(ov.base + (size_t)m * ov.ld + nl) = acc4;
+    }
 }
 
 // One block per logical page: gathers W[n][k] = B[k][n] for 128 n x 16 k and writes the 4 KB page in
@@ -668,8 +624,8 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
 
 // Shared host path of the two skinny entry points.
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
-                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream,
-                               const ag_group_desc* grp, bool clear_sem) {
+                               int N, int K, const ag_plan* plan, float* partial, cudaStream_t stream,
+                               const ag_group_desc* grp) {
     const int32_t* h = plan->header;
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
     if (h[H_TILE_N] != SK_BN || (h[H_TILE_M] != 16 && h[H_TILE_M] != 32) || M > h[H_TILE_M]) return AG_ERR_ARG;
@@ -704,7 +660,6 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     }
     x.C = (float*)Cout;
     x.partial = h[H_KSPLITS] > 1 ? partial : nullptr;
-    x.sem = sem;
     if (W) {
         if (W->K != K || W->N != N || (K % SK_BK) || W->tiles_n != h[H_TILES_N]) return AG_ERR_ARG;
         x.packed = W->dst;
@@ -735,7 +690,6 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
         }
     }
     // every argument check has passed: from here on work is queued on the stream
-    if (clear_sem && sem) AG_CUDA(cudaMemsetAsync(sem, 0, (size_t)h[H_TILES_N] * 4 * sizeof(int), stream));
     const bool zeroing = h[H_KSPLITS] > 1 && !x.partial;
     // Overlapping launches: only for plans that use every SM with one block each - the blocks of the next launch then
     // find room exactly where a block of this one has left, one per SM, and no block of the launch after next can
@@ -764,10 +718,28 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     PersistParams gp = make_persist_params(plan, M, N, K);
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
     gp.a_blocks = a_blocks ? 1 : 0;
-    if (NM == 16) return W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
-                           : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
-    return W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
-             : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
+    ag_status ls;
+    if (NM == 16) ls = W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
+                         : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
+    else ls = W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
+                : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
+    if (ls != AG_OK || !x.partial) return ls;
+    // bit-reproducible split-K: the workspace slices are added in ascending split order by a second kernel, which may
+    // become resident while the GEMM runs and waits for its completion on the device
+    const long long quads = (long long)M * ((N + 3) / 4);
+    cudaLaunchConfig_t rc;
+    memset(&rc, 0, sizeof rc);
+    rc.gridDim = dim3((unsigned)std::min<long long>(4 * 148, (quads + 255) / 256));
+    rc.blockDim = dim3(256);
+    rc.stream = stream;
+    cudaLaunchAttribute ra[1];
+    ra[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    ra[0].val.programmaticStreamSerializationAllowed = 1;
+    rc.attrs = ra;
+    rc.numAttrs = 1;
+    AG_CUDA(cudaLaunchKernelEx(&rc, k_reduce_splits, gp, x));
+    count_launch();
+    return AG_OK;
 }
 
 }  // namespace ag
@@ -1147,7 +1119,7 @@ extern "C" ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_pa
         return gemm_pair_dispatch(d->A_all, nullptr, W, d->C_all, h[H_M], h[H_N], h[H_K], plan,
                                   reinterpret_cast<cudaStream_t>(cuda_stream), d);
     if (h[H_M] > d->tile_m) return AG_ERR_ARG;
-    return gemm_skinny_dispatch(d->A_all, nullptr, W, d->C_all, h[H_M], h[H_N], h[H_K], plan, plan->d_partial, plan->d_sem,
+    return gemm_skinny_dispatch(d->A_all, nullptr, W, d->C_all, h[H_M], h[H_N], h[H_K], plan, plan->d_partial,
                                 reinterpret_cast<cudaStream_t>(cuda_stream), d);
 }
 
@@ -1174,7 +1146,7 @@ extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weigh
     if (!A || !W || !Cout || !plan) return AG_ERR_ARG;
     if (plan->header[H_TILE_M] == 256)  // dense plan of block pairs over packed B panels
         return gemm_pair_dispatch(A, nullptr, W, Cout, M, N, K, plan, reinterpret_cast<cudaStream_t>(cuda_stream));
-    return gemm_skinny_dispatch(A, nullptr, W, Cout, M, N, K, plan, plan->d_partial, plan->d_sem,
+    return gemm_skinny_dispatch(A, nullptr, W, Cout, M, N, K, plan, plan->d_partial,
                                 reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -1192,7 +1164,7 @@ extern "C" ag_status gemm_persistent_packed(const void* A, const ag_packed_weigh
 //
 // The array's name is only a host-side handle; the address the kernel needs is asked from the
 // runtime once per device (cudaGetSymbolAddress, with that device current) and remembered.
-constexpr size_t kNoAllocSemBytes = 16 * 1024;                   // 4096 arrival counters = 1024 tiles of 128 columns
+constexpr size_t kNoAllocSemBytes = 16 * 1024;                   // head of the array, unused (see below)
 constexpr size_t kNoAllocPartialBytes = 8u * 1024 * 1024;        // 2 Mi fp32 partial sums
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocSemBytes + kNoAllocPartialBytes];
 
@@ -1229,9 +1201,8 @@ extern "C" ag_status gemm_persistent_noalloc(const void* A, const void* B, void*
         scratch = g_noalloc_ptr[dev];
     }
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-    int* sem = reinterpret_cast<int*>(scratch);
+    // the first kNoAllocSemBytes of the array are not used (they held arrival counters when the last unit of a tile
+    // added the slices); the slices start behind them as before
     float* partial = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + kNoAllocSemBytes);
-    // the counters must start at zero: once the arguments have been checked, whatever an earlier call left
-    // behind is wiped on the same stream, right in front of the kernel
-    return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, partial, sem, stream, nullptr, true);
+    return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, partial, stream, nullptr);
 }

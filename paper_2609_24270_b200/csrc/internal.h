@@ -71,7 +71,6 @@ struct ag_plan {
     unsigned long long* d_unit_times;  // device [n_units][2], allocated by ag_plan_trace(plan, 1)
     long long* d_margins;      // device [n_units] (affinity only, else null)
     float* d_partial;          // device [k_splits][M][N] split-K partial sums (skinny plans with k_splits > 1)
-    int* d_sem;                // device [4 * tiles_n] arrival counters for the split-K reduction
     int4* d_quick;             // device [n_sm]: {slot, list offset, list length, first unit} per SM id
     std::vector<int32_t> h_image;
     mutable uint32_t epoch;

@@ -252,8 +252,8 @@ bool encode_a_slabs(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t K,
 
 // Host-side dispatchers of the kernel families (defined next to their kernels).
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
-                               int N, int K, const ag_plan* plan, float* partial, int* sem, cudaStream_t stream,
-                               const ag_group_desc* grp = nullptr, bool clear_sem = false);
+                               int N, int K, const ag_plan* plan, float* partial, cudaStream_t stream,
+                               const ag_group_desc* grp = nullptr);
 ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weights* W, void* Cout, int M, int N, int K,
                              const ag_plan* plan, cudaStream_t stream, const ag_group_desc* grp = nullptr);
 

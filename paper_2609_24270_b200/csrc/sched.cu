@@ -494,7 +494,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     pl->d_image = nullptr; pl->d_ctrl = nullptr; pl->d_tile_owner = nullptr; pl->d_tile_count = nullptr;
     pl->d_margins = nullptr;
     pl->d_unit_times = nullptr;
-    pl->d_partial = nullptr; pl->d_sem = nullptr; pl->d_quick = nullptr;
+    pl->d_partial = nullptr; pl->d_quick = nullptr;
     pl->epoch = 0;
     pl->grid_blocks = 0;
     pl->kslabs_total = n_slab;
@@ -520,8 +520,6 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         if (p.tile_m <= 32 && p.k_splits > 1 && !p.splitk_in_memory) {
             // decode-shaped plans: split-K partial sums and per-tile arrival counters
             TRY(cudaMalloc(&pl->d_partial, sizeof(float) * (size_t)p.k_splits * p.M * p.N));
-            TRY(cudaMalloc(&pl->d_sem, sizeof(int) * (size_t)tiles_n * 4));
-            TRY(cudaMemset(pl->d_sem, 0, sizeof(int) * (size_t)tiles_n * 4));
         }
         TRY(cudaMalloc(&d_topo, sizeof(ag_topo_map)));
         TRY(cudaMemcpy(d_topo, map, sizeof(ag_topo_map), cudaMemcpyHostToDevice));
@@ -726,7 +724,6 @@ extern "C" void ag_plan_destroy(ag_plan* plan) {
     cudaFree(plan->d_margins);
     cudaFree(plan->d_unit_times);
     cudaFree(plan->d_partial);
-    cudaFree(plan->d_sem);
     cudaFree(plan->d_quick);
     delete plan;
 }

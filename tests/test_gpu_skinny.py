@@ -33,7 +33,7 @@ def test_rowmajor_weights_integer_exact(M, tile_m, k_splits):
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=tile_m,
                                                                 tile_n=128, k_splits=k_splits))
     plan.reset_record()
-    for _ in range(2):                                      # second launch: arrival counters reset themselves
+    for _ in range(2):                                      # second launch: nothing is left over from the first
         C = run_rowmajor(A, B, plan)
         assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B))
     owner, count = plan.tile_record()
@@ -52,6 +52,26 @@ def test_rowmajor_weights_uniform(shape, in_memory):
                                                             tile_m=16 if M <= 16 else 32, tile_n=128, k_splits=ksp))
         for _ in range(2):
             check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
+
+
+def test_workspace_split_k_is_bit_reproducible():
+    """splitk_in_memory = 0: the k-split slices are added in ascending split order, so the bits of C do not depend on
+    which SMs ran which unit, nor on the order in which the units finished: the same C, bit for bit, from the full
+    chip and from 37 SMs, from die-compact and oblivious plans, with and without overlapping launches and from one call
+    to the next."""
+    M, N, K, ksp = 16, 2048, 4096, 8
+    A, B = inputs.gemm_inputs(M, N, K, seed=77)
+    topo = device_topo()
+    outs = []
+    for b, kind, overlap in ((topo.n_sm, ag.AG_DIE_COMPACT, 0), (topo.n_sm, ag.AG_DIE_COMPACT, 1), (37, ag.AG_DIE_COMPACT, 0),
+                             (topo.n_sm, ag.AG_OBLIVIOUS, 0), (53, ag.AG_OBLIVIOUS, 0)):
+        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=kind, M=M, N=N, K=K, tile_m=16, tile_n=128, k_splits=ksp,
+                                                            seed=3 if kind == ag.AG_OBLIVIOUS else 0, overlap_launches=overlap))
+        for _ in range(3):
+            outs.append(run_rowmajor(A, B, plan))
+    check_close(outs[0], og.gemm_blocked(A, B))
+    for o in outs[1:]:
+        assert o.tobytes() == outs[0].tobytes()
 
 
 @pytest.mark.parametrize("in_memory", [0, 1])
