@@ -33,8 +33,10 @@ constexpr int SK_BK = 64;      // k-slab
 //    k-slabs (32 KB of weights, 8 MMAs).
 constexpr int SK_SLABS = 2;    // k-slabs per weight stage
 constexpr int SK_WPROD = 3;    // warps that issue weight copies (stage i of the block's run belongs to warp i mod SK_WPROD)
-constexpr int SK_STAGES = 6;   // two stages per issuing warp
-constexpr int SK_THREADS = (2 + kEpiWarps + SK_WPROD) * 32;   // scheduler, MMA issuer, epilogue warps, weight producers
+constexpr int SK_STAGES = 6;   // two stages per issuing warp; even, so that a buffer's parity is the parity of its place in the run
+constexpr int SK_NMMA = 2;     // threads that issue MMAs: thread t owns the stage buffers of parity t (see the MMA role)
+constexpr int SK_THREADS = (2 + kEpiWarps + SK_WPROD + (SK_NMMA - 1)) * 32;   // scheduler, MMA issuer, epilogue warps, weight producers, second MMA issuer
+constexpr int SK_MMA2_WARP = 2 + kEpiWarps + SK_WPROD;
 constexpr int SK_SLAB_BYTES = SK_BN * SK_BK * 2;   // 16 KB of weights per k-slab
 constexpr int SK_W_BYTES = SK_SLABS * SK_SLAB_BYTES;
 constexpr int SK_STAGE_BYTES = SK_W_BYTES;
@@ -57,7 +59,7 @@ struct SkinnyCtl {
     uint64_t tmem_empty[2];
     uint64_t sched_full[kRing];
     uint64_t sched_empty[kRing];
-    uint64_t mma_drain;
+    uint64_t mma_drain[SK_NMMA];
     int ring[kRing];
     uint32_t tmem_base;
     int abort_flag;
@@ -135,7 +137,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     const uint32_t a_base = base + SK_STAGES * SK_STAGE_BYTES;
     SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + SK_STAGES * SK_STAGE_BYTES + SK_ASTAGES * SK_A_STAGE_MAX);
     constexpr uint32_t kAccCols = NM;                    // columns of one accumulator
-    constexpr uint32_t kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;   // two accumulators (the smallest allocation is 32 columns)
+    constexpr uint32_t kTmemCols = 2 * SK_NMMA * kAccCols;   // two units in flight, one accumulator per MMA-issuing thread each (64 or 128 columns)
     volatile int* abort_flag = &ctl->abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int my_sm = (int)smid();
@@ -155,17 +157,17 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         }
         for (int i = 0; i < SK_ASTAGES; ++i) {
             mbar_init(smem_u32(&ctl->a_full[i]), 1);
-            mbar_init(smem_u32(&ctl->a_empty[i]), 1);
+            mbar_init(smem_u32(&ctl->a_empty[i]), SK_NMMA);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tmem_full[i]), SK_NMMA);
             mbar_init(smem_u32(&ctl->tmem_empty[i]), kEpiWarps);
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&ctl->sched_full[i]), 1);
-            mbar_init(smem_u32(&ctl->sched_empty[i]), 1 + kEpiWarps + SK_WPROD);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), SK_NMMA + kEpiWarps + SK_WPROD);
         }
-        mbar_init(smem_u32(&ctl->mma_drain), 1);
+        for (int i = 0; i < SK_NMMA; ++i) mbar_init(smem_u32(&ctl->mma_drain[i]), 1);
         mbar_fence_init();
         prefetch_tmap(&tm_a);
         if (!PACKED || x.quad_base) prefetch_tmap(&tm_w);
@@ -180,13 +182,13 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     const uint64_t limit = p.wait_limit_ns;
     // tensor memory is needed by the MMA issuer and the epilogue only: the copy-issuing warps do not wait for it
     uint32_t tmem_base = 0;
-    if (warp >= 1 && warp < 2 + kEpiWarps) {
+    if ((warp >= 1 && warp < 2 + kEpiWarps) || warp == SK_MMA2_WARP) {
         if (warp == 1) {
             tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
             tmem_relinquish();
         }
         tc_fence_before();
-        asm volatile("bar.sync 1, %0;" ::"n"((1 + kEpiWarps) * 32) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"((SK_NMMA + kEpiWarps) * 32) : "memory");
         tc_fence_after();
         tmem_base = ctl->tmem_base;
     }
@@ -260,7 +262,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             ok = __shfl_sync(0xffffffffu, ok, 0);
         }
         if (!ok && lane == 0) linger_for_copies();
-    } else if (warp >= 2 + kEpiWarps) {
+    } else if (warp >= 2 + kEpiWarps && warp < SK_MMA2_WARP) {
         // ------------------------------------------------ weight copies: warp pw issues k-iterations pw, pw + SK_WPROD, ...
         // For packed weights all 32 lanes fetch the page-table entries of the next eight k-slabs with one load
         // each, so the issuing lane never waits on a table lookup.
@@ -368,8 +370,18 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             q0 += (uint32_t)n_st;
         }
         if (!ok && lane == 0) linger_for_copies();
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == SK_MMA2_WARP) {
         if (lane == 0) {
+            // ------------------------------------------------ MMA issuers.  Thread t (0: warp 1, 1: the last warp) owns the
+            // stage buffers of parity t, i.e. every second stage of the block's run.  One thread alone is the cap of the
+            // pipeline below the full chip: it spends 500-700 cycles per 32 KB stage (eight MMAs of ~45 cycles, a barrier
+            // wait, a fence, a commit), i.e. at most ~50 B per cycle, where the copies deliver more.
+            // Ownership by buffer, not by position in the unit: a parity wait on a stage barrier is only right for the
+            // thread that consumed the buffer's previous contents (a thread a whole lap ahead would see the parity of the
+            // lap before as "full").  Inside a unit the thread therefore has the stages of one parity a, and adds them up
+            // in accumulator a: accumulator 0 always holds the unit's even stages and accumulator 1 the odd ones, so the
+            // value of C does not depend on what the SM ran before.
+            const int t = warp == 1 ? 0 : 1;
             constexpr uint32_t idesc = make_idesc_bf16(128, NM, PACKED ? 0 : 1, 0);
             // descriptors without their start address.  Weights: packed page = no swizzle, 16-byte k chunks 128 B
             // apart (LBO), 8-row groups 256 B apart (SBO); row-major = MN-major with 128-byte swizzle, the two
@@ -379,9 +391,12 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const uint64_t da_t = make_smem_desc(0, 16, 1024, 2);
             constexpr uint32_t kWStep = (PACKED ? 4096u : 2048u) >> 4;   // one K = 16 step inside a weight stage
             constexpr uint32_t kAStepK = 32u >> 4;                       // ... inside an activation slab
+            constexpr int kGrpStages = SK_AGRP / SK_SLABS;               // stages per activation buffer (even)
+            static_assert(kGrpStages % SK_NMMA == 0, "every full activation group has stages of both threads");
+            static_assert(SK_STAGES % SK_NMMA == 0, "a stage buffer always belongs to the same thread");
             const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
-            uint32_t st = 0, ph = 0;                  // weight stage and the parity of "stage is full"
-            uint32_t aj = 0, aph = 0;                 // activation buffer and the parity of "buffer is full"
+            uint32_t q0 = 0;                          // stages of the units before this one (over the whole run of the block)
+            uint32_t git = 0;                         // activation groups before this unit
             uint32_t tile_it = 0;
             bool ok = true;
             for (uint32_t it = 0; ok; ++it) {
@@ -396,60 +411,72 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 const int ks = u % p.k_splits;
                 const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
                 const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+                const int n_slabs = s1 - s0;
+                const int n_st = (n_slabs + SK_SLABS - 1) / SK_SLABS;
+                const int n_grp = (n_slabs + SK_AGRP - 1) / SK_AGRP;
                 const uint32_t acc = tile_it & 1;
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 4);
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * kAccCols;
-                int in_grp = 0;                       // k-slabs of the current activation buffer already used
-                uint64_t da = 0;
-                for (int left = s1 - s0, first = 1; left > 0; left -= SK_SLABS) {
-                    if (in_grp == 0) {
-                        if (!mbar_wait(smem_u32(&ctl->a_full[aj]), aph, abort_flag, limit)) {
-                            report_timeout(p, 9);
-                            ok = false;
-                            break;
-                        }
-                        da = da_t | (uint64_t)((a_base + aj * kAStage) >> 4);
-                    }
-                    if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
-                        report_timeout(p, 5);
+                const int a = (t - (int)(q0 & 1u)) & 1;       // parity, inside the unit, of the stages in this thread's buffers
+                const uint32_t d_tmem = tmem_base + (acc * SK_NMMA + a) * kAccCols;
+                uint32_t st = (q0 + a) % SK_STAGES, ph = ((q0 + a) / SK_STAGES) & 1;   // this thread's first stage of the unit
+                bool first = true;
+                for (int g = 0; g < n_grp && ok; ++g) {
+                    const uint32_t gi = git + g, aj = gi % SK_ASTAGES, aph = (gi / SK_ASTAGES) & 1;
+                    const int i_end = min(n_st, (g + 1) * kGrpStages);
+                    int i = g * kGrpStages + a;
+                    // (waited for even when nothing of the group is this thread's: its release below must not be
+                    // counted among the releases of the group that used the buffer before)
+                    if (!mbar_wait(smem_u32(&ctl->a_full[aj]), aph, abort_flag, limit)) {
+                        report_timeout(p, 9);
                         ok = false;
                         break;
                     }
-                    tc_fence_after();
-                    const uint64_t dw = dw_t | (uint64_t)((base + st * SK_STAGE_BYTES) >> 4);
-                    // the first k-slab of the stage, then the second one if the unit has it
-                    tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
-#pragma unroll
-                    for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
-                    if (left > 1) {
-                        const uint64_t da2 = da + (kASlab >> 4);
-#pragma unroll
-                        for (int k4 = 0; k4 < SK_BK / 16; ++k4)
-                            tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                    if (i >= i_end) {
+                        // a last group of one stage: nothing of it is this thread's
+                        mbar_arrive(smem_u32(&ctl->a_empty[aj]));
+                        break;
                     }
-                    first = 0;
-                    tc_commit(empty0 + st * 8);
-                    if (++st == SK_STAGES) { st = 0; ph ^= 1; }
-                    da += SK_SLABS * (kASlab >> 4);
-                    in_grp += SK_SLABS;
-                    if (in_grp >= SK_AGRP || left <= SK_SLABS) {   // last stage that reads this buffer's activations
-                        tc_commit(smem_u32(&ctl->a_empty[aj]));
-                        in_grp = 0;
-                        if (++aj == SK_ASTAGES) { aj = 0; aph ^= 1; }
+                    uint64_t da = (da_t | (uint64_t)((a_base + aj * kAStage) >> 4)) + (uint32_t)a * (SK_SLABS * (kASlab >> 4));
+                    for (; i < i_end; i += SK_NMMA) {
+                        if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
+                            report_timeout(p, 5);
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint64_t dw = dw_t | (uint64_t)((base + st * SK_STAGE_BYTES) >> 4);
+                        // the first k-slab of the stage, then the second one if the unit has it
+                        tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
+#pragma unroll
+                        for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
+                        if (n_slabs - i * SK_SLABS > 1) {
+                            const uint64_t da2 = da + (kASlab >> 4);
+#pragma unroll
+                            for (int k4 = 0; k4 < SK_BK / 16; ++k4)
+                                tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                        }
+                        first = false;
+                        tc_commit(empty0 + st * 8);
+                        st += SK_NMMA;
+                        if (st >= SK_STAGES) { st -= SK_STAGES; ph ^= 1; }
+                        da += SK_NMMA * SK_SLABS * (kASlab >> 4);
                     }
+                    if (ok) tc_commit(smem_u32(&ctl->a_empty[aj]));    // this thread's last read of the buffer has been issued
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                q0 += (uint32_t)n_st;
+                git += (uint32_t)n_grp;
                 ++tile_it;
             }
             if (*abort_flag) {
-                tc_commit(smem_u32(&ctl->mma_drain));
+                tc_commit(smem_u32(&ctl->mma_drain[t]));
                 int dummy = 0;
-                mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                mbar_wait(smem_u32(&ctl->mma_drain[t]), 0, &dummy, 2000000ull);
             }
         }
     } else {
@@ -479,12 +506,18 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             tc_fence_after();
             float sum[NM];
             {
-                uint32_t v[NM];
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
+                // the accumulator of the thread that took the even stages, plus the other one's if the unit has a second stage
+                uint32_t v[NM], w[NM];
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * SK_NMMA * kAccCols;
+                const int s0e = min(p.kslabs_total, ks * p.kslabs_per_split), s1e = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+                const bool two = s1e - s0e > SK_SLABS;
                 if constexpr (NM == 16) tmem_ld_32x16(taddr, v); else tmem_ld_32x32(taddr, v);
+                if (two) {
+                    if constexpr (NM == 16) tmem_ld_32x16(taddr + kAccCols, w); else tmem_ld_32x32(taddr + kAccCols, w);
+                }
                 tmem_ld_wait();
 #pragma unroll
-                for (int m = 0; m < NM; ++m) sum[m] = __uint_as_float(v[m]);
+                for (int m = 0; m < NM; ++m) sum[m] = two ? __uint_as_float(v[m]) + __uint_as_float(w[m]) : __uint_as_float(v[m]);
             }
             tc_fence_before();
             __syncwarp();
