@@ -113,9 +113,14 @@ def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
 
 
 # ---------------------------------------------------------------------------------------------
-def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
-    """M=16, N=K=8192 decode-shaped GEMM, weights die-packed; die-local vs remote assignment."""
-    M, N, K, ksp = 16, 8192, 8192, 16
+def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1, k_splits=(16, 4)):
+    """M=16, N=K=8192 decode-shaped GEMM, weights die-packed; die-local vs remote assignment; 16 and 4 k-splits."""
+    for ksp in k_splits:
+        _config4(fh, topo, budgets, n_buffers, overlap, ksp)
+
+
+def _config4(fh, topo, budgets, n_buffers, overlap, ksp):
+    M, N, K = 16, 8192, 8192
     A = inputs.uniform_bf16(M, K, inputs.DEFAULT_SEED)
     dA = dev_bf16(A)
     dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
@@ -184,7 +189,7 @@ def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1):
                 ag.gemm_persistent(dA.data_ptr(), wb.data_ptr(), dC.data_ptr(), M, N, K, plan)
             ms = time_queued(run2, warmup=4, iters=24)
             out[name] = algo_bytes / (ms * 1e-3) / 1e9
-        emit(dict(config=4, workload="GEMM M=16 N=K=8192 bf16, 128-col units x 16 k-splits, 4 rotating weight buffers",
+        emit(dict(config=4, workload=f"GEMM M=16 N=K=8192 bf16, 128-col units x {ksp} k-splits, 4 rotating weight buffers", k_splits=ksp,
                   sm_budget=b, overlap_launches=overlap, gbs=out, local_over_remote=out["die_local"] / out["remote"],
                   pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), closed_form=packs[0][0].closed_form(), local_set=sm_set_summary(topo, plan_local),
                   remote_set=sm_set_summary(topo, plan_remote), both_dies_set=sm_set_summary(topo, plan_spread), algo_bytes=algo_bytes,
@@ -350,18 +355,24 @@ def groupgemm(fh, topo, seeds=(1, 2)):
                 packed = ag.pack_weights_grouped([b.data_ptr() for b in Bs], K, N, plan_dc, amap, dst.data_ptr(), dst_bytes)
                 bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packed.page_table())
                 plan_rem = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
+                # the units shared equally between the dies instead of by SM count (each die's memory is equally fast)
+                plan_eq = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, die_quota=1, **kw))
+                dst_eq = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+                amap_eq = ag.affinity_probe(dst_eq.data_ptr(), dst_bytes, topo)
+                packed_eq = ag.pack_weights_grouped([b.data_ptr() for b in Bs], K, N, plan_eq, amap_eq, dst_eq.data_ptr(), dst_bytes)
                 desc_rm = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, [b.data_ptr() for b in Bs], N, K, 32)
                 algo = w_bytes + total * K * 2 + total * N * 4
                 res = {}
                 for name, pk, plan in (("rowmajor_oblivious", None, plan_obl), ("rowmajor_die_compact", None, plan_dc),
-                                       ("packed_die_local", packed, plan_dc), ("packed_remote", packed, plan_rem)):
+                                       ("packed_die_local", packed, plan_dc), ("packed_die_local_equal_quota", packed_eq, plan_eq),
+                                       ("packed_remote", packed, plan_rem)):
                     ms = time_queued(lambda: ag.gemm_persistent_grouped(desc_rm, pk, plan))
                     assert plan.last_status() == ag.AG_OK
                     res[name] = algo / (ms * 1e-3) / 1e9
                 emit(dict(config="groupgemm", G=G, M=M, N=N, K=K, seed=seed, rows_total=total, k_splits=ksp,
                           weight_gb=w_bytes / 1e9, gbs=res, local_over_remote=res["packed_die_local"] / res["packed_remote"],
                           local_over_rowmajor_oblivious=res["packed_die_local"] / res["rowmajor_oblivious"]), fh)
-                del packed, desc_rm, dA, dC
+                del packed, packed_eq, dst_eq, amap_eq, desc_rm, dA, dC
             del Bs, dst, amap
             torch.cuda.empty_cache()
 
