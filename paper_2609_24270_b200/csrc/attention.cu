@@ -38,7 +38,9 @@ constexpr int AT_Q_BYTES = AT_NQ * AT_D * 2;        // 4 KB
 constexpr int AT_NP = 2 * AT_MAXG;         // rows of a probability tile: 8 hi parts, 8 lo parts (one MMA adds both)
 constexpr int AT_P_BYTES = AT_NP * AT_TILE * 2;     // 4 KB
 constexpr int AT_PSLOTS = 4;
-constexpr int AT_SMEM_BYTES = AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + AT_PSLOTS * AT_P_BYTES + 1024 + 1024;
+constexpr int AT_PBATCH = 2;               // probability tiles written per fence (half the ring: the other half feeds the MMAs meanwhile)
+constexpr int AT_CTL_BYTES = 2048;
+constexpr int AT_SMEM_BYTES = AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + AT_PSLOTS * AT_P_BYTES + 1024 + AT_CTL_BYTES;
 constexpr uint32_t AT_SCOLS = AT_MAXT * AT_NQ;      // score columns of one unit buffer (128)
 constexpr uint32_t AT_BUFCOLS = AT_SCOLS + AT_NP;   // + output columns (hi-part and lo-part sums)
 constexpr uint32_t AT_TMEM_COLS = 512;
@@ -52,6 +54,7 @@ struct AttnCtl {
     uint64_t sched_full[kRing], sched_empty[kRing];
     uint64_t mma_drain;
     int ring[kRing];
+    int ring_pages[kRing][4 * AT_MAXT];   // the page-list words of the unit in ring[r] (see AttnArgs::quad_of)
     uint32_t tmem_base;
     int abort_flag;
     int member;
@@ -59,6 +62,8 @@ struct AttnCtl {
     float red_max[kEpiWarps][AT_MAXG];
     float red_sum[2][kEpiWarps][AT_MAXG];
 };
+
+static_assert(sizeof(AttnCtl) <= AT_CTL_BYTES, "control block does not fit its share of shared memory");
 
 struct AttnArgs {
     const uint8_t* pages;         // packed KV buffer
@@ -69,6 +74,12 @@ struct AttnArgs {
     float scale_log2e;            // log2(e) / sqrt(D)
     int release_next;             // 1: let the next launch on the stream start while this one is still running
 };
+
+__device__ __forceinline__ float ex2_approx(float v) {      // 2^v, relative error 2^-22; 2^-inf = 0
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
 
 __device__ __forceinline__ int unit_tiles(const AttnArgs& x, int u) {
     if (!x.kv_len) return x.T;
@@ -170,12 +181,23 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 u = src.next(lane);
             }
             if (!ok) break;
-            if (lane == 0) {
+            // the unit's page-list words travel with it through the ring (one coalesced load here, several units ahead of
+            // the copies, instead of a dependent load in front of every copy)
+            const int page_word = (u >= 0 && lane < 4 * x.T) ? x.quad_of[(size_t)u * x.T * 4 + lane] : 0;
+            {
                 const int r = it % kRing;
-                if (!mbar_wait_idle(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
+                int w_ok = 1;
+                if (lane == 0 && !mbar_wait_idle(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {
                     report_timeout(p, 1);
-                    ok = 0;
-                } else {
+                    w_ok = 0;
+                }
+                ok = __shfl_sync(0xffffffffu, w_ok, 0);
+                if (ok) ctl->ring_pages[r][lane] = page_word;
+                __syncwarp();
+            }
+            if (ok && lane == 0) {
+                const int r = it % kRing;
+                {
                     ctl->ring[r] = u;
                     if (p.unit_times && u >= 0) p.unit_times[2 * u] = globaltimer_ns();
                     mbar_arrive(smem_u32(&ctl->sched_full[r]));
@@ -212,14 +234,14 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         uint32_t q_run = 0;          // stages issued by all copy warps together so far
         int prev_u = -1, prev_t = 0;
         int ok = 1;
-        auto copy_tiles = [&](int u, int n_t, int v_part) {
+        int words_cur = 0, words_prev = 0;   // lane l: word l of the page lists of the unit just taken off the ring / the one before
+        auto copy_tiles = [&](int words, int n_t, int v_part) {
             // this warp's stages among the next n_t: ordinals q_run .. q_run + n_t - 1, those = pw mod AT_NPROD
             for (int t = 0; t < n_t && ok; ++t) {
                 const uint32_t q = q_run + (uint32_t)t;
                 if ((int)(q % AT_NPROD) != pw) continue;
                 const uint32_t st = q % AT_STAGES, ph = ((q / AT_STAGES) & 1) ^ 1;
-                int entry = 0;
-                if (lane < 2) entry = x.quad_of[((size_t)u * x.T + t) * 4 + v_part * 2 + lane];
+                const int entry = __shfl_sync(0xffffffffu, words, t * 4 + v_part * 2 + (lane & 1));
                 if (lane == 0) {
                     if (!mbar_wait(smem_u32(&ctl->kv_empty[st]), ph, abort_flag, limit)) {
                         report_timeout(p, 2);
@@ -249,16 +271,21 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     ok = 0;
                 } else {
                     u = ctl->ring[r];
-                    mbar_arrive(smem_u32(&ctl->sched_empty[r]));
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             u = __shfl_sync(0xffffffffu, u, 0);
             if (!ok) break;
+            __syncwarp();
+            const int words_new = ctl->ring_pages[r][lane];   // read before the slot is handed back
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
             const int n_t = u >= 0 ? unit_tiles(x, u) : 0;
             if (u >= 0 && n_t == 0) continue;                 // a request without keys: nothing to stream
-            if (u >= 0) copy_tiles(u, n_t, 0);
-            if (prev_u >= 0 && ok) copy_tiles(prev_u, prev_t, 1);
+            words_cur = words_new;
+            if (u >= 0) copy_tiles(words_cur, n_t, 0);
+            if (prev_u >= 0 && ok) copy_tiles(words_prev, prev_t, 1);
+            words_prev = words_cur;
             prev_u = u;
             prev_t = n_t;
             if (u < 0) break;
@@ -399,7 +426,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             for (int q = 0; q < AT_MAXG; ++q) {
                 if (q < G) {
                     const float l = (ctl->red_sum[j][0][q] + ctl->red_sum[j][1][q]) + (ctl->red_sum[j][2][q] + ctl->red_sum[j][3][q]);
-                    out[(size_t)q * AT_D] = (__uint_as_float(vh[q]) + __uint_as_float(vl[q])) / l;
+                    out[(size_t)q * AT_D] = __fdividef(__uint_as_float(vh[q]) + __uint_as_float(vl[q]), l);
                 }
             }
             if (lane == 0 && wq == 0) {
@@ -467,21 +494,26 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     }
                 }
             }
+            // warp maximum with one integer reduction per query row: floats compare like the signed integers
+            // b ^ ((b >> 31) & 0x7fffffff) of their bit patterns b
 #pragma unroll
             for (int q = 0; q < AT_MAXG; ++q) {
                 if (q < G) {
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) mx[q] = fmaxf(mx[q], __shfl_xor_sync(0xffffffffu, mx[q], o));
+                    const int b = __float_as_int(mx[q]);
+                    const int m = __reduce_max_sync(0xffffffffu, b ^ ((b >> 31) & 0x7fffffff));
+                    mx[q] = __int_as_float(m ^ ((m >> 31) & 0x7fffffff));
                 }
             }
             if (lane == 0) {
 #pragma unroll
-                for (int q = 0; q < AT_MAXG; ++q) ctl->red_max[widx][q] = mx[q];
+                for (int q = 0; q < AT_MAXG; ++q)
+                    if (q < G) ctl->red_max[widx][q] = mx[q];
             }
             asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
 #pragma unroll
             for (int q = 0; q < AT_MAXG; ++q)
-                mx[q] = fmaxf(fmaxf(ctl->red_max[0][q], ctl->red_max[1][q]), fmaxf(ctl->red_max[2][q], ctl->red_max[3][q])) * x.scale_log2e;
+                if (q < G)
+                    mx[q] = fmaxf(fmaxf(ctl->red_max[0][q], ctl->red_max[1][q]), fmaxf(ctl->red_max[2][q], ctl->red_max[3][q])) * x.scale_log2e;
             // ---- probabilities, tile by tile, into the ring of probability tiles: rows 0-7 the bf16 hi parts, rows
             // 8-15 the lo parts (row = query row; the rows of query rows that do not exist stay zero)
             float sum[AT_MAXG];
@@ -489,32 +521,43 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             for (int q = 0; q < AT_MAXG; ++q) sum[q] = 0.f;
             const uint32_t atom = (uint32_t)(i_lane >> 6) * 2048u;                 // keys 0-63 / 64-127 of the tile
             const uint32_t chunk = (uint32_t)((i_lane & 63) >> 3), within = (uint32_t)(i_lane & 7) * 2u;
+            // AT_PBATCH tiles at a time: one fence and one round of barrier traffic per batch
 #pragma unroll
-            for (int t = 0; t < AT_MAXT; ++t) {
-                if (t < n_t && ok) {
-                    const uint32_t ps = pt % AT_PSLOTS;
-                    if (!mbar_wait_warp(smem_u32(&ctl->p_empty[ps]), ((pt / AT_PSLOTS) & 1) ^ 1, abort_flag, limit)) {
-                        if (lane == 0) report_timeout(p, 7);
-                        ok = false;
-                    } else {
-                        uint8_t* ptile = smem + AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + ps * AT_P_BYTES;
+            for (int b0 = 0; b0 < AT_MAXT; b0 += AT_PBATCH) {
+                if (b0 < n_t && ok) {
+                    const int nb = min(AT_PBATCH, n_t - b0);
+                    int w_ok = 1;
+                    if (lane == 0) {
+                        for (int tt = 0; tt < nb && w_ok; ++tt)
+                            w_ok = mbar_wait(smem_u32(&ctl->p_empty[(pt + tt) % AT_PSLOTS]), (((pt + tt) / AT_PSLOTS) & 1) ^ 1, abort_flag, limit);
+                        if (!w_ok) report_timeout(p, 7);
+                    }
+                    ok = __shfl_sync(0xffffffffu, w_ok, 0) != 0;
+                    if (ok) {
 #pragma unroll
-                        for (int q = 0; q < AT_MAXG; ++q) {
-                            if (q < G) {
-                                // masked keys: exp2(-inf) = 0
-                                const float pv = exp2f(fmaf(__uint_as_float(sv[t][q]), x.scale_log2e, -mx[q]));
-                                sum[q] += pv;
-                                const __nv_bfloat16 hi = __float2bfloat16_rn(pv);
-                                const __nv_bfloat16 lo = __float2bfloat16_rn(pv - __bfloat162float(hi));
-                                const uint32_t off = atom + (uint32_t)q * 128u + ((chunk ^ (uint32_t)(q & 7)) << 4) + within;
-                                *reinterpret_cast<__nv_bfloat16*>(ptile + off) = hi;
-                                *reinterpret_cast<__nv_bfloat16*>(ptile + 1024 + off) = lo;
+                        for (int tt = 0; tt < AT_PBATCH; ++tt) {
+                            if (tt < nb) {
+                                uint8_t* ptile = smem + AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + ((pt + tt) % AT_PSLOTS) * AT_P_BYTES;
+#pragma unroll
+                                for (int q = 0; q < AT_MAXG; ++q) {
+                                    if (q < G) {
+                                        // masked keys: exp2(-inf) = 0
+                                        const float pv = ex2_approx(fmaf(__uint_as_float(sv[b0 + tt][q]), x.scale_log2e, -mx[q]));
+                                        sum[q] += pv;
+                                        const __nv_bfloat16 hi = __float2bfloat16_rn(pv);
+                                        const __nv_bfloat16 lo = __float2bfloat16_rn(pv - __bfloat162float(hi));
+                                        const uint32_t off = atom + (uint32_t)q * 128u + ((chunk ^ (uint32_t)(q & 7)) << 4) + within;
+                                        *reinterpret_cast<__nv_bfloat16*>(ptile + off) = hi;
+                                        *reinterpret_cast<__nv_bfloat16*>(ptile + 1024 + off) = lo;
+                                    }
+                                }
                             }
                         }
                         fence_proxy_async_smem();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[ps]));
-                        ++pt;
+                        if (lane == 0)
+                            for (int tt = 0; tt < nb; ++tt) mbar_arrive(smem_u32(&ctl->p_full[(pt + tt) % AT_PSLOTS]));
+                        pt += (uint32_t)nb;
                     }
                 }
             }
