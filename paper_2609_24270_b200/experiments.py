@@ -10,6 +10,7 @@
     python -m paper_2609_24270_b200.experiments --config latency           # latency histograms from one SM per die
     python -m paper_2609_24270_b200.experiments --config cluster_sets      # cluster eligibility of equal-size SM sets
     python -m paper_2609_24270_b200.experiments --config attention         # decode attention, KV pages local / remote / interleaved
+    python -m paper_2609_24270_b200.experiments --config 5_attention       # prefill GEMM and decode attention on disjoint SM partitions
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
 launches first, median of the timed launches.  torch is used for device memory, streams and events.
@@ -271,6 +272,86 @@ def config5(fh, topo):
                       decode_gbs=dict(alone=bytes_d / (alone_d * 1e-3) / 1e9, overlapped=bytes_d / (ov_d * 1e-3) / 1e9),
                       prefill_set=sm_set_summary(topo, plan_p), decode_set=sm_set_summary(topo, plan_d),
                       note="decode time per GEMM includes the hand-over between back-to-back launches"), fh)
+
+
+# ---------------------------------------------------------------------------------------------
+def config5_attention(fh, topo):
+    """The serving split of the paper's multiplexing study with attention as the decode side: a prefill-like GEMM
+    (8192x4096x4096, block pairs) on one SM partition and decode attention (batch 128, 512 keys, 8 KV heads, 32 query
+    heads) on the rest, on two streams.  Die split with die-local KV pages against the GPC-spread and the oblivious
+    partitions with interleaved pages."""
+    Mp, N, K = 8192, 4096, 4096
+    Ap, Bp = inputs.gemm_inputs(Mp, N, K)
+    dAp, dBp = dev_bf16(Ap), dev_bf16(Bp)
+    dCp = torch.empty((Mp, N), dtype=torch.float32, device="cuda")
+    B, Hq, Hkv, L, D = 128, 32, 8, 512, 128
+    dK = torch.randn((B, Hkv, L, D), dtype=torch.bfloat16, device="cuda")
+    dV = torch.randn((B, Hkv, L, D), dtype=torch.bfloat16, device="cuda")
+    dQ = torch.randn((B, Hq, D), dtype=torch.bfloat16, device="cuda")
+    dO = torch.empty((B, Hq, D), dtype=torch.float32, device="cuda")
+    kv_bytes = 2 * B * Hkv * L * D * 2
+    algo = kv_bytes + B * Hq * D * 6
+    dst_bytes = 2 * kv_bytes + (16 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    flops_p = 2.0 * Mp * N * K
+    pre_kw = dict(M=Mp, N=N, K=K, tile_m=256, tile_n=256, raster_group=4)
+    att_kw = dict(M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16, tile_n=128, k_splits=1)
+    for split in ((74, 74), (110, 38)):
+        for mode, placement in (("die_split", ag.KV_LOCAL), ("die_split", ag.KV_INTERLEAVED), ("gpc_spread", ag.KV_LOCAL),
+                                ("gpc_spread", ag.KV_INTERLEAVED), ("oblivious", ag.KV_INTERLEAVED)):
+            kind = ag.AG_OBLIVIOUS if mode == "oblivious" else ag.AG_DIE_COMPACT
+            sel = 1 if mode == "gpc_spread" else 0
+            plan_p = ag.sched_build(topo, None, split[0], ag.make_policy(kind=kind, preferred_die=0, sm_select=sel, **pre_kw))
+            taken = [int(s) for s in plan_p.parsed()["sm_list"]]
+            plan_d = ag.sched_build(topo, None, split[1], ag.make_policy(kind=kind, avoid=taken, sm_select=sel, **att_kw))
+            kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan_d, amap, dst.data_ptr(), dst_bytes, placement)
+            n_pre, n_dec = 6, 6 * 12
+
+            def pre():
+                ag.gemm_persistent(dAp.data_ptr(), dBp.data_ptr(), dCp.data_ptr(), Mp, N, K, plan_p, s1.cuda_stream)
+
+            def dec():
+                ag.attention_decode(dQ.data_ptr(), kv, None, dO.data_ptr(), B, Hq, plan_d, s2.cuda_stream)
+
+            def run(do_pre, do_dec):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                torch.cuda.synchronize()
+                if do_pre:
+                    ev[0].record(s1)
+                if do_dec:
+                    ev[2].record(s2)
+                for i in range(max(n_pre, n_dec)):
+                    if do_pre and i < n_pre:
+                        pre()
+                    if do_dec and i < n_dec:
+                        dec()
+                if do_pre:
+                    ev[1].record(s1)
+                if do_dec:
+                    ev[3].record(s2)
+                torch.cuda.synchronize()
+                tp = ev[0].elapsed_time(ev[1]) / n_pre if do_pre else None
+                td = ev[2].elapsed_time(ev[3]) / n_dec if do_dec else None
+                return tp, td
+
+            for _ in range(2):
+                run(True, True)
+            alone_p = np.median([run(True, False)[0] for _ in range(3)])
+            alone_d = np.median([run(False, True)[1] for _ in range(3)])
+            both = [run(True, True) for _ in range(5)]
+            ov_p = np.median([x[0] for x in both])
+            ov_d = np.median([x[1] for x in both])
+            assert plan_p.last_status() == ag.AG_OK and plan_d.last_status() == ag.AG_OK
+            emit(dict(config="5_attention", split=list(split), partition=mode,
+                      kv_pages={ag.KV_LOCAL: "die_local", ag.KV_INTERLEAVED: "interleaved"}[placement],
+                      kv_local_fraction=kv.info()["local_fraction"],
+                      prefill_tflops=dict(alone=flops_p / (alone_p * 1e-3) / 1e12, overlapped=flops_p / (ov_p * 1e-3) / 1e12),
+                      decode_gbs=dict(alone=algo / (alone_d * 1e-3) / 1e9, overlapped=algo / (ov_d * 1e-3) / 1e9),
+                      decode_us=dict(alone=alone_d * 1e3, overlapped=ov_d * 1e3),
+                      prefill_set=sm_set_summary(topo, plan_p), decode_set=sm_set_summary(topo, plan_d)), fh)
+            del kv
 
 
 # ---------------------------------------------------------------------------------------------
@@ -543,7 +624,7 @@ def main():
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
      "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention,
-     "raster_traffic": lambda f, t: raster(f, t, traffic_only=True)}[args.config](fh, topo)
+     "raster_traffic": lambda f, t: raster(f, t, traffic_only=True), "5_attention": config5_attention}[args.config](fh, topo)
 
 
 if __name__ == "__main__":
