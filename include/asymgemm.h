@@ -492,13 +492,18 @@ ag_status gemm_persistent_noalloc(const void* A, const void* B, void* C, int M, 
  * head): o = softmax(q K^T / sqrt(D)) V for the H_q / H_kv query heads that share the KV head.  The plan is an ordinary
  * decode-shaped plan with one unit per (request, KV head): sched_build with tile_m = 16, tile_n = 128, k_splits = 1,
  * M = H_q / H_kv, N = 128 * B * H_kv (K is not looked at); unit u = request u / H_kv, KV head u % H_kv.
+ * Requests of more than 1024 keys are cut into C = ceil(L / 1024) chunks of 1024 keys, each a unit of its own with its
+ * pages on the die that runs it: N = 128 * B * H_kv * C, unit u = ((request * H_kv) + KV head) * C + chunk.  A chunk unit
+ * leaves its unnormalised outputs, score maximum and probability sum in a workspace owned by the ag_kv_cache, and a second
+ * kernel launched behind the first one puts the chunks of every (request, KV head) together (so two calls on the same
+ * ag_kv_cache must not overlap on the GPU).
  */
 typedef struct ag_kv_cache ag_kv_cache;
 /*
  * ag_kv_pack - store a KV cache in 4 KB pages in the order the tensor cores read them, every unit's pages in chunks
  * of one die (indirect allocation by remapping, Section 7.1.1, applied to the KV cache).
- *   K, V   device, [B][H_kv][L][D] bf16 row-major; D = 128; L a multiple of 128, L <= 1024
- *   plan   B * H_kv units (see above)
+ *   K, V   device, [B][H_kv][L][D] bf16 row-major; D = 128; L a multiple of 128, L <= 2^20
+ *   plan   B * H_kv * ceil(L / 1024) units (see above)
  *   amap   affinity map of exactly (dst, dst_bytes), else AG_ERR_STALE_AMAP
  *   dst    device, 4096-aligned; local / remote placement needs room for 2 x the larger die's share, interleaved 1 x
  *   placement  0: on the die that the plan runs the unit on; 1: on the other die; 2: interleaved (consecutive chunks,

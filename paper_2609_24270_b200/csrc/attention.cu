@@ -8,6 +8,9 @@
 //     P = exp((S - max) / sqrt(D))                softmax warps, one thread per key of a tile, scores in tensor memory
 //     O^T[d][q]  = sum_key V[key][d] P[q][key]    tcgen05.mma, d on the M side, keys contracted; P as bf16 hi + lo parts
 //     O[q][:] /= sum_key P[q][key]                epilogue
+// Requests with more than 1024 keys are cut into chunks of 1024 keys, one unit per (request, KV head, chunk): such a
+// unit leaves its unnormalised outputs, its score maximum and its sum of probabilities in a workspace, and a second
+// kernel (k_attn_combine) puts the chunks of a (request, KV head) together.
 // The KV cache is packed once (ag_kv_pack) into 4 KB pages in the MMA's no-swizzle operand order - K pages hold
 // [128 keys x 16 d], V pages [128 d x 16 keys] - four pages of a 64-wide contraction slab per group of same-die
 // chunks (or four consecutive chunks for the interleaved placement), so a 128-key tile of K or of V is one 32 KB
@@ -61,6 +64,7 @@ struct AttnCtl {
     int4 quick;
     float red_max[kEpiWarps][AT_MAXG];
     float red_sum[2][kEpiWarps][AT_MAXG];
+    float unit_max[2][AT_MAXG];           // score maximum (times log2 e / sqrt D) of the unit in buffer j, for chunked requests
 };
 
 static_assert(sizeof(AttnCtl) <= AT_CTL_BYTES, "control block does not fit its share of shared memory");
@@ -70,7 +74,10 @@ struct AttnArgs {
     const int32_t* quad_of;       // [units][4 T]: per tile K slab 0, K slab 1, V slab 0, V slab 1: base chunk | class << 30
     const int32_t* kv_len;        // [B] or null
     float* O;                     // [B][H_q][128]
-    int H_kv, G, T, L;
+    int H_kv, G, T, L;            // T: tiles of a full unit (at most AT_MAXT)
+    int n_chunks, T_total;        // units per (request, KV head); tiles of a whole request
+    float* o_part;                // [units][AT_MAXG][128] unnormalised outputs (n_chunks > 1)
+    float2* stats;                // [units][AT_MAXG] (maximum, sum) (n_chunks > 1)
     float scale_log2e;            // log2(e) / sqrt(D)
     int release_next;             // 1: let the next launch on the stream start while this one is still running
 };
@@ -81,11 +88,14 @@ __device__ __forceinline__ float ex2_approx(float v) {      // 2^v, relative err
     return r;
 }
 
-__device__ __forceinline__ int unit_tiles(const AttnArgs& x, int u) {
-    if (!x.kv_len) return x.T;
-    const int len = min(x.L, max(0, x.kv_len[u / x.H_kv]));
-    return (len + AT_TILE - 1) / AT_TILE;
+// keys of unit u = (request b, KV head h, chunk c), u = (b H_kv + h) n_chunks + c: those of the request's first
+// kv_len[b] keys that fall into the chunk
+__device__ __forceinline__ int unit_keys(const AttnArgs& x, int u) {
+    const int bh = u / x.n_chunks, c = u - bh * x.n_chunks;
+    const int len = x.kv_len ? min(x.L, max(0, x.kv_len[bh / x.H_kv])) : x.L;
+    return min(AT_MAXT * AT_TILE, max(0, len - c * AT_MAXT * AT_TILE));
 }
+__device__ __forceinline__ int unit_tiles(const AttnArgs& x, int u) { return (unit_keys(x, u) + AT_TILE - 1) / AT_TILE; }
 
 __global__ void __launch_bounds__(AT_THREADS, 1)
 k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_g0,
@@ -183,7 +193,11 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (!ok) break;
             // the unit's page-list words travel with it through the ring (one coalesced load here, several units ahead of
             // the copies, instead of a dependent load in front of every copy)
-            const int page_word = (u >= 0 && lane < 4 * x.T) ? x.quad_of[(size_t)u * x.T * 4 + lane] : 0;
+            int page_word = 0;
+            if (u >= 0) {
+                const int bh = u / x.n_chunks, c = u - bh * x.n_chunks;
+                if (lane < 4 * min(AT_MAXT, x.T_total - c * AT_MAXT)) page_word = x.quad_of[((size_t)bh * x.T_total + c * AT_MAXT) * 4 + lane];
+            }
             {
                 const int r = it % kRing;
                 int w_ok = 1;
@@ -213,14 +227,14 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     report_timeout(p, 2);
                     ok = 0;
                 } else {
-                    // the G query rows of the unit (rows u G .. u G + G - 1 of the [B H_q][128] matrix) and whatever
+                    // the G query rows of the unit's KV head (G consecutive rows of the [B H_q][128] matrix) and whatever
                     // follows them up to 16 rows: the extra rows only produce columns nobody reads
                     const uint32_t bar = smem_u32(&ctl->q_full[j]);
                     // the queries are the product of the launch before this one: with overlapping launches they are
                     // read only after it has completed (the key/value pages are the caller's promise)
                     if (nq == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
                     mbar_expect_tx(bar, AT_Q_BYTES);
-                    tma_load_3d(q_base + j * AT_Q_BYTES, &tm_q, bar, 0, u * x.G, 0);
+                    tma_load_3d(q_base + j * AT_Q_BYTES, &tm_q, bar, 0, (u / x.n_chunks) * x.G, 0);
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -421,12 +435,27 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->o_empty[j]));
-            float* out = x.O + (size_t)pend_u * G * AT_D + i_lane;
+            if (x.n_chunks == 1) {
+                float* out = x.O + (size_t)pend_u * G * AT_D + i_lane;
 #pragma unroll
-            for (int q = 0; q < AT_MAXG; ++q) {
-                if (q < G) {
-                    const float l = (ctl->red_sum[j][0][q] + ctl->red_sum[j][1][q]) + (ctl->red_sum[j][2][q] + ctl->red_sum[j][3][q]);
-                    out[(size_t)q * AT_D] = __fdividef(__uint_as_float(vh[q]) + __uint_as_float(vl[q]), l);
+                for (int q = 0; q < AT_MAXG; ++q) {
+                    if (q < G) {
+                        const float l = (ctl->red_sum[j][0][q] + ctl->red_sum[j][1][q]) + (ctl->red_sum[j][2][q] + ctl->red_sum[j][3][q]);
+                        out[(size_t)q * AT_D] = __fdividef(__uint_as_float(vh[q]) + __uint_as_float(vl[q]), l);
+                    }
+                }
+            } else {
+                // a chunk of a longer request: unnormalised outputs, maximum and sum for k_attn_combine
+                float* part = x.o_part + (size_t)pend_u * AT_MAXG * AT_D + i_lane;
+#pragma unroll
+                for (int q = 0; q < AT_MAXG; ++q) {
+                    if (q < G) {
+                        part[(size_t)q * AT_D] = __uint_as_float(vh[q]) + __uint_as_float(vl[q]);
+                        if (i_lane == q) {
+                            const float l = (ctl->red_sum[j][0][q] + ctl->red_sum[j][1][q]) + (ctl->red_sum[j][2][q] + ctl->red_sum[j][3][q]);
+                            x.stats[(size_t)pend_u * AT_MAXG + q] = make_float2(ctl->unit_max[j][q], l);
+                        }
+                    }
                 }
             }
             if (lane == 0 && wq == 0) {
@@ -447,16 +476,19 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
             if (u < 0) break;
-            const int b = u / x.H_kv;
-            const int len = x.kv_len ? min(x.L, max(0, x.kv_len[b])) : x.L;
+            const int len = unit_keys(x, u);              // keys of this unit that count
             const int n_t = (len + AT_TILE - 1) / AT_TILE;
             if (!prior_done) {      // nothing is written before everything launched earlier on the stream has completed
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 prior_done = true;
             }
             if (n_t == 0) {
-                float* out = x.O + (size_t)u * G * AT_D + i_lane;
-                for (int q = 0; q < G; ++q) out[(size_t)q * AT_D] = 0.f;
+                if (x.n_chunks == 1) {
+                    float* out = x.O + (size_t)u * G * AT_D + i_lane;
+                    for (int q = 0; q < G; ++q) out[(size_t)q * AT_D] = 0.f;
+                } else if (i_lane < G) {
+                    x.stats[(size_t)u * AT_MAXG + i_lane] = make_float2(-INFINITY, 0.f);   // a chunk without keys: nothing to add
+                }
                 if (lane == 0 && wq == 0) {
                     p.tile_owner[u] = my_sm;
                     if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
@@ -514,6 +546,11 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             for (int q = 0; q < AT_MAXG; ++q)
                 if (q < G)
                     mx[q] = fmaxf(fmaxf(ctl->red_max[0][q], ctl->red_max[1][q]), fmaxf(ctl->red_max[2][q], ctl->red_max[3][q])) * x.scale_log2e;
+            if (x.n_chunks > 1 && i_lane < G) {
+#pragma unroll
+                for (int q = 0; q < AT_MAXG; ++q)
+                    if (q == i_lane) ctl->unit_max[j][q] = mx[q];
+            }
             // ---- probabilities, tile by tile, into the ring of probability tiles: rows 0-7 the bf16 hi parts, rows
             // 8-15 the lo parts (row = query row; the rows of query rows that do not exist stay zero)
             float sum[AT_MAXG];
@@ -589,6 +626,35 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
 }
 
+// Chunked requests: one block per (request, KV head), thread = output column d.  With m_c, l_c, O_c the maximum (in
+// units of log2 e / sqrt D), the sum of probabilities and the unnormalised outputs of chunk c:
+// O = sum_c 2^(m_c - m) O_c / sum_c 2^(m_c - m) l_c, m = max_c m_c; chunks without keys (l_c = 0) are left out.
+__global__ void __launch_bounds__(AT_D) k_attn_combine(const float* __restrict__ o_part, const float2* __restrict__ stats,
+                                                        float* __restrict__ O, int n_chunks, int G) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int bh = blockIdx.x / G, q = blockIdx.x - bh * G, d = threadIdx.x;     // one block per (request, KV head, query row)
+    const float2* st = stats + (size_t)bh * n_chunks * AT_MAXG + q;
+    const float* part = o_part + ((size_t)bh * n_chunks * AT_MAXG + q) * AT_D + d;
+    float m = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) {
+        const float2 s2 = __ldcg(st + (size_t)c * AT_MAXG);
+        if (s2.y > 0.f) m = fmaxf(m, s2.x);
+    }
+    float num = 0.f, den = 0.f;
+#pragma unroll 4
+    for (int c = 0; c < n_chunks; ++c) {
+        const float2 s2 = __ldcg(st + (size_t)c * AT_MAXG);
+        const float v = __ldcg(part + (size_t)c * AT_MAXG * AT_D);   // finite or not: only used when the chunk had keys
+        if (s2.y > 0.f) {
+            const float w = ex2_approx(s2.x - m);
+            num = fmaf(w, v, num);
+            den = fmaf(w, s2.y, den);
+        }
+    }
+    O[((size_t)bh * G + q) * AT_D + d] = den > 0.f ? num / den : 0.f;
+}
+
 // One block per 4 KB page.  which = 0: K page (unit, tile t, d group g): element (n = key, k = d) = K[u][128 t + n][16 g + k];
 // which = 1: V page (unit, tile t, key group j): element (n = d, k = key) = V[u][128 t + 16 j + k][n].  Both in the MMA's
 // no-swizzle K-major order: byte (n / 8) * 256 + (k / 8) * 128 + (n % 8) * 16 + (k % 8) * 2.
@@ -622,9 +688,12 @@ using namespace ag;
 
 struct ag_kv_cache {
     int B, H_kv, L, T, placement, free_bit;
+    int n_chunks;                        // units per (request, KV head): chunks of AT_MAXT tiles
     const uint8_t* dst;
     size_t dst_bytes;
     int32_t* d_quad_of;                  // device [B H_kv][4 T]
+    float* d_part;                       // device [units][AT_MAXG][128] (n_chunks > 1): unnormalised outputs of the chunks
+    float2* d_stats;                     // device [units][AT_MAXG] (n_chunks > 1)
     std::vector<int32_t> h_quad_of;
     CUtensorMap tm_quad[2];
     double local_fraction;               // share of the pages that sit on the die that runs their unit
@@ -633,20 +702,26 @@ struct ag_kv_cache {
 extern "C" void ag_kv_destroy(ag_kv_cache* kv) {
     if (!kv) return;
     cudaFree(kv->d_quad_of);
+    cudaFree(kv->d_part);
+    cudaFree(kv->d_stats);
     delete kv;
 }
 
 extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, int L, int D, const ag_plan* plan,
                                 const ag_affinity_map* amap, void* dst, size_t dst_bytes, int placement, ag_kv_cache** out) {
     if (!K || !V || !plan || !amap || !dst || !out || B < 1 || H_kv < 1 || D != AT_D || L < AT_TILE || (L % AT_TILE) ||
-        L > AT_MAXT * AT_TILE || placement < 0 || placement > 2)
+        L > (1 << 20) || placement < 0 || placement > 2)
         return AG_ERR_ARG;
     *out = nullptr;
-    const long long n_units = (long long)B * H_kv;
+    const int T = L / AT_TILE;                                  // tiles of a request
+    const int n_chunks = (T + AT_MAXT - 1) / AT_MAXT;           // units per (request, KV head)
+    const long long n_bh = (long long)B * H_kv, n_units = n_bh * n_chunks;
     if (n_units != plan->lay.n_units || plan->header[H_KSPLITS] != 1) return AG_ERR_ARG;
     if (amap->base != dst || amap->bytes != dst_bytes) return AG_ERR_STALE_AMAP;
-    const int T = L / AT_TILE;
-    const size_t quads_per_unit = 4 * (size_t)T, n_quads = quads_per_unit * (size_t)n_units;
+    // slabs (groups of four pages) per (request, KV head); slab i belongs to tile (i % quads_per_bh) / 4 of (request, KV
+    // head) i / quads_per_bh, i.e. to unit (i / quads_per_bh) n_chunks + tile / AT_MAXT
+    const size_t quads_per_bh = 4 * (size_t)T, n_quads = quads_per_bh * (size_t)n_bh;
+    auto unit_of_quad = [&](size_t i) -> size_t { return (i / quads_per_bh) * n_chunks + ((i % quads_per_bh) / 4) / AT_MAXT; };
     // die of every unit from the plan's die queues
     const PlanLayout& lay = plan->lay;
     const int32_t* img = plan->h_image.data();
@@ -654,8 +729,8 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
     for (int e = img[lay.die_q_off() + 1]; e < lay.n_units; ++e) unit_die[img[lay.die_q() + e]] = 1;
     ag_kv_cache* kv = new (std::nothrow) ag_kv_cache();
     if (!kv) return AG_ERR_NOMEM;
-    kv->B = B; kv->H_kv = H_kv; kv->L = L; kv->T = T; kv->placement = placement; kv->free_bit = -1;
-    kv->dst = (const uint8_t*)dst; kv->dst_bytes = dst_bytes; kv->d_quad_of = nullptr;
+    kv->B = B; kv->H_kv = H_kv; kv->L = L; kv->T = T; kv->placement = placement; kv->free_bit = -1; kv->n_chunks = n_chunks;
+    kv->dst = (const uint8_t*)dst; kv->dst_bytes = dst_bytes; kv->d_quad_of = nullptr; kv->d_part = nullptr; kv->d_stats = nullptr;
     kv->h_quad_of.resize(n_quads);
     size_t on_die = 0;
     if (placement == 2) {
@@ -663,7 +738,7 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
         if (n_quads * 4 > amap->n_chunks) { delete kv; return AG_ERR_ARG; }
         for (size_t i = 0; i < n_quads; ++i) {
             kv->h_quad_of[i] = (int32_t)(4 * i) | (2 << 30);
-            for (int c = 0; c < 4; ++c) on_die += amap->h_die_of_chunk[4 * i + c] == unit_die[i / quads_per_unit];
+            for (int c = 0; c < 4; ++c) on_die += amap->h_die_of_chunk[4 * i + c] == unit_die[unit_of_quad(i)];
         }
     } else {
         // groups of four same-die chunks, as for packed weights (see ag_pack_weights_ex)
@@ -687,7 +762,7 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
         }
         size_t nxt[2] = {0, 0};
         for (size_t i = 0; i < n_quads; ++i) {
-            const int d = unit_die[i / quads_per_unit] ^ (placement == 1 ? 1 : 0);
+            const int d = unit_die[unit_of_quad(i)] ^ (placement == 1 ? 1 : 0);
             if (nxt[d] >= groups[d].size()) { delete kv; return AG_ERR_ARG; }   // destination too small for this die's share
             kv->h_quad_of[i] = groups[d][nxt[d]++];
         }
@@ -729,6 +804,8 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
     int32_t* d_chunk = nullptr;
     cudaError_t e = cudaMalloc(&kv->d_quad_of, sizeof(int32_t) * n_quads);
     if (e == cudaSuccess) e = cudaMemcpy(kv->d_quad_of, kv->h_quad_of.data(), sizeof(int32_t) * n_quads, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && n_chunks > 1) e = cudaMalloc(&kv->d_part, sizeof(float) * (size_t)n_units * AT_MAXG * AT_D);
+    if (e == cudaSuccess && n_chunks > 1) e = cudaMalloc(&kv->d_stats, sizeof(float2) * (size_t)n_units * AT_MAXG);
     if (e == cudaSuccess) e = cudaMalloc(&d_chunk, sizeof(int32_t) * page_chunk.size());
     if (e == cudaSuccess) e = cudaMemcpy(d_chunk, page_chunk.data(), sizeof(int32_t) * page_chunk.size(), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
@@ -759,7 +836,7 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     const int G = H_q / kv->H_kv;
     if (G > AT_MAXG || (((uintptr_t)Q | (uintptr_t)O) & 15u)) return AG_ERR_ARG;
     const int32_t* h = plan->header;
-    if ((long long)B * kv->H_kv != plan->lay.n_units || h[H_KSPLITS] != 1) return AG_ERR_ARG;
+    if ((long long)B * kv->H_kv * kv->n_chunks != plan->lay.n_units || h[H_KSPLITS] != 1) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -786,7 +863,9 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     x.quad_of = kv->d_quad_of;
     x.kv_len = kv_len;
     x.O = (float*)O;
-    x.H_kv = kv->H_kv; x.G = G; x.T = kv->T; x.L = kv->L;
+    x.H_kv = kv->H_kv; x.G = G; x.T = std::min(kv->T, AT_MAXT); x.L = kv->L;
+    x.n_chunks = kv->n_chunks; x.T_total = kv->T;
+    x.o_part = kv->d_part; x.stats = kv->d_stats;
     x.scale_log2e = 1.4426950408889634f / sqrtf((float)AT_D);
     PersistParams gp = make_persist_params(plan, h[H_M], h[H_N], h[H_K]);
     cudaLaunchConfig_t cfg;
@@ -805,5 +884,21 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     const cudaError_t le = cudaLaunchKernelEx(&cfg, k_attn_decode, tm_q, tm0, tm1, gp, x);
     if (le != cudaSuccess) return launch_failed(plan, le);
     count_launch();
+    if (kv->n_chunks > 1) {
+        // requests of more than AT_MAXT tiles: the chunks' partial results are put together by a second kernel, which may
+        // become resident while the first one runs and waits for its completion on the device
+        cudaLaunchConfig_t cc;
+        memset(&cc, 0, sizeof cc);
+        cc.gridDim = dim3((unsigned)(B * kv->H_kv * G));
+        cc.blockDim = dim3(AT_D);
+        cc.stream = stream;
+        cudaLaunchAttribute ca[1];
+        ca[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        ca[0].val.programmaticStreamSerializationAllowed = 1;
+        cc.attrs = ca;
+        cc.numAttrs = 1;
+        AG_CUDA(cudaLaunchKernelEx(&cc, k_attn_combine, (const float*)kv->d_part, (const float2*)kv->d_stats, (float*)O, kv->n_chunks, G));
+        count_launch();
+    }
     return AG_OK;
 }

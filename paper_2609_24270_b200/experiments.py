@@ -565,7 +565,7 @@ def cluster_sets(fh, topo, budgets=(64, 72, 96), n_subsets=16):
                       **{n: res[n] for n in ("lowest_ids", "highest_ids", "die_compact_tpc", "die_compact_cluster", "gpc_spread_cluster")}), fh)
 
 
-def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024)), budgets=None, overlap=1):
+def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024), (16, 32, 8, 8192), (4, 32, 8, 32768)), budgets=None, overlap=1):
     """Decode attention over a paged KV cache (Section 6.4's die-local KV direction): batch B, H_q query heads over
     H_kv KV heads, L keys of 128 dimensions per head; pages of a unit on the die of the SM that owns it (local),
     on the other die (remote) or wherever the allocation put them (interleaved).  GB/s of KV bytes."""
@@ -590,7 +590,8 @@ def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024)), budgets=
             lib_us = str(e)[:80]
         for b in budgets:
             for both in ((0, 1) if b < topo.n_sm else (0,)):
-                kw = dict(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16, tile_n=128, k_splits=1,
+                n_chunks = (L + 1023) // 1024      # requests over 1024 keys run as one unit per chunk of 1024 keys
+                kw = dict(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv * n_chunks, K=L, tile_m=16, tile_n=128, k_splits=1,
                           sm_select=1 if both else 0, overlap_launches=overlap)
                 plan = ag.sched_build(topo, None, b, ag.make_policy(**kw))
                 plan_eq = ag.sched_build(topo, None, b, ag.make_policy(die_quota=1, **kw))   # units shared equally between the dies

@@ -36,7 +36,8 @@ def run_attention(Q, K, V, placement, kv_len=None, budget=None, overlap=0):
     _, Hkv, L, _ = K.shape
     topo = device_topo()
     b = topo.n_sm if budget is None else budget
-    plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
+    n_chunks = (L + 1023) // 1024                    # requests over 1024 keys: one unit per chunk of 1024 keys
+    plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv * n_chunks, K=L, tile_m=16,
                                                         tile_n=128, k_splits=1, overlap_launches=overlap))
     kv_bytes = 2 * B * Hkv * L * D * 2
     dst_bytes = (2 * kv_bytes if placement != ag.KV_INTERLEAVED else kv_bytes) + (8 << 20)
@@ -92,6 +93,22 @@ def test_ragged_lengths_and_closed_forms():
             assert np.abs(got[b, hq] - Vf[b, hq // 4].mean(axis=0)).max() <= 1e-5
 
 
+@pytest.mark.parametrize("placement", [ag.KV_LOCAL, ag.KV_INTERLEAVED])
+@pytest.mark.parametrize("shape", [(2, 8, 2, 2048), (3, 4, 4, 1280), (2, 16, 2, 4096)])
+def test_long_requests_in_chunks(placement, shape):
+    """More than 1024 keys: chunks of 1024 keys run as units of their own and a second kernel puts them together."""
+    B, Hq, Hkv, L = shape
+    Q, K, V = make_case(B, Hq, Hkv, L, seed=300 + L, q_scale=6.0)
+    got, _, _ = run_attention(Q, K, V, placement)
+    check(got, oa.gqa_decode(Q, K, V))
+    # ragged: lengths that end inside a chunk, at a chunk boundary, in the first chunk, and zero
+    lens = [L - 1, 1025, 0][:B] if B == 3 else [1024, L - 127][:B]
+    got, _, _ = run_attention(Q, K, V, placement, kv_len=lens)
+    check(got, oa.gqa_decode(Q, K, V, lens))
+    if 0 in lens:
+        assert not got[lens.index(0)].any()
+
+
 def test_serving_shape_on_sm_budgets():
     """Batch 128, 512 keys, 8 KV heads, 32 query heads (the decode side of the paper's serving split): 1024 units."""
     B, Hq, Hkv, L = 128, 32, 8, 512
@@ -113,6 +130,6 @@ def test_bad_arguments():
     h = ag.C.c_void_p()
     L_ = ag.lib()
     # L not a multiple of 128, too long, wrong unit count, wrong head dimension
-    for (B, H, Lk, D) in ((4, 2, 200, 128), (4, 2, 2048, 128), (4, 4, 256, 128), (4, 2, 256, 64)):
+    for (B, H, Lk, D) in ((4, 2, 200, 128), (4, 2, 2048, 128), (4, 4, 256, 128), (4, 2, 256, 64)):   # (2048 keys need a plan of 16 units)
         st = L_.ag_kv_pack(k.data_ptr(), k.data_ptr(), B, H, Lk, D, plan.handle, amap.handle, dst.data_ptr(), dst.numel(), 0, ag.C.byref(h))
         assert st == ag.AG_ERR_ARG
