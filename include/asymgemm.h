@@ -517,6 +517,15 @@ ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, int L, int D
 /* group_free_bit: the hash bit the page groups use (-1: interleaved placement); local_fraction: share of the pages that
  * the map places on the die of their unit (either may be NULL). */
 ag_status ag_kv_info(const ag_kv_cache* kv, int32_t* group_free_bit, double* local_fraction);
+/*
+ * ag_kv_append - write one new token per request into the packed cache (what a decode step does before it attends):
+ * the key row and the value row of request b, KV head h go to position pos[b] of that request's pages, i.e. onto the
+ * die that the plan of ag_kv_pack runs the unit on.
+ *   k_new, v_new  device, [B][H_kv][128] bf16
+ *   pos           device [B] int32: 0 <= pos[b] < L, other values leave the request untouched
+ * Asynchronous on cuda_stream.  Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA.
+ */
+ag_status ag_kv_append(ag_kv_cache* kv, const void* k_new, const void* v_new, const int32_t* pos, void* cuda_stream);
 void ag_kv_destroy(ag_kv_cache* kv);
 /*
  * attention_decode_persistent - O[b][hq][:] = softmax_j(Q[b][hq] . K[b][h][j] / sqrt(D)) V[b][h][j][:], h = hq / (H_q / H_kv),

@@ -30,7 +30,7 @@ EXPORTED = [
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
-    "ag_kernel_launch_count", "ag_kv_pack", "ag_kv_info", "ag_kv_destroy", "attention_decode_persistent",
+    "ag_kernel_launch_count", "ag_kv_pack", "ag_kv_info", "ag_kv_append", "ag_kv_destroy", "attention_decode_persistent",
 ]
 
 
@@ -149,6 +149,7 @@ def lib() -> C.CDLL:
     L.ag_wait_probe.argtypes = [C.c_uint64, C.POINTER(C.c_uint64)]
     L.ag_kv_pack.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, sz, C.c_int, C.POINTER(vp)]
     L.ag_kv_info.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_double)]
+    L.ag_kv_append.argtypes = [vp, vp, vp, vp, vp]
     L.ag_kv_destroy.argtypes = [vp]
     L.ag_kv_destroy.restype = None
     L.attention_decode_persistent.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, vp, vp]
@@ -504,6 +505,10 @@ class KVCache:
         f, frac = C.c_int32(), C.c_double()
         _check(lib().ag_kv_info(self.handle, C.byref(f), C.byref(frac)), "ag_kv_info")
         return dict(group_free_bit=int(f.value), local_fraction=float(frac.value))
+
+    def append(self, k_new_ptr: int, v_new_ptr: int, pos_ptr: int, stream: int = 0):
+        """One new token per request at position pos[b] (device int32 [B]); k_new, v_new: [B][H_kv][128] bf16."""
+        _check(lib().ag_kv_append(self.handle, k_new_ptr, v_new_ptr, pos_ptr, stream), "ag_kv_append")
 
     def __del__(self):
         if getattr(self, "handle", None):

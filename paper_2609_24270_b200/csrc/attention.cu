@@ -682,6 +682,30 @@ __global__ void k_pack_kv(const uint16_t* __restrict__ K, const uint16_t* __rest
     *reinterpret_cast<uint4*>(out + 128) = hi;
 }
 
+// One block per (request, KV head): writes the key and value row of one new token (position pos[b] of the request)
+// into the pages, in the same byte order as k_pack_kv.  Thread = dimension d.
+__global__ void __launch_bounds__(AT_D) k_kv_append(const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
+                                                     const int32_t* __restrict__ pos, int H_kv, int L, int T,
+                                                     const int32_t* __restrict__ page_chunk, uint8_t* __restrict__ dst) {
+    const int bh = blockIdx.x, d = threadIdx.x;
+    const int at = pos[bh / H_kv];
+    if (at < 0 || at >= L) return;                       // no room (or no token) for this request
+    const int t = at / AT_TILE, n = at % AT_TILE;
+    const size_t page0 = ((size_t)bh * T + t) * 16;      // the tile's 8 K pages, then its 8 V pages
+    // K page g = d / 16 holds [128 keys x 16 d]: element (key n, k = d % 16)
+    {
+        const int g = d >> 4, k = d & 15;
+        uint8_t* out = dst + (size_t)page_chunk[page0 + g] * AG_CHUNK_BYTES + (n / 8) * 256 + (k / 8) * 128 + (n % 8) * 16 + (k % 8) * 2;
+        *reinterpret_cast<uint16_t*>(out) = k_new[(size_t)bh * AT_D + d];
+    }
+    // V page j = n / 16 holds [128 d x 16 keys]: element (d, k = n % 16)
+    {
+        const int j = n >> 4, k = n & 15;
+        uint8_t* out = dst + (size_t)page_chunk[page0 + 8 + j] * AG_CHUNK_BYTES + (d / 8) * 256 + (k / 8) * 128 + (d % 8) * 16 + (k % 8) * 2;
+        *reinterpret_cast<uint16_t*>(out) = v_new[(size_t)bh * AT_D + d];
+    }
+}
+
 }  // namespace ag
 
 using namespace ag;
@@ -692,6 +716,7 @@ struct ag_kv_cache {
     const uint8_t* dst;
     size_t dst_bytes;
     int32_t* d_quad_of;                  // device [B H_kv][4 T]
+    int32_t* d_page_chunk;               // device [B H_kv][T][16]: chunk of every page (8 K pages, 8 V pages per tile)
     float* d_part;                       // device [units][AT_MAXG][128] (n_chunks > 1): unnormalised outputs of the chunks
     float2* d_stats;                     // device [units][AT_MAXG] (n_chunks > 1)
     std::vector<int32_t> h_quad_of;
@@ -702,6 +727,7 @@ struct ag_kv_cache {
 extern "C" void ag_kv_destroy(ag_kv_cache* kv) {
     if (!kv) return;
     cudaFree(kv->d_quad_of);
+    cudaFree(kv->d_page_chunk);
     cudaFree(kv->d_part);
     cudaFree(kv->d_stats);
     delete kv;
@@ -730,7 +756,7 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
     ag_kv_cache* kv = new (std::nothrow) ag_kv_cache();
     if (!kv) return AG_ERR_NOMEM;
     kv->B = B; kv->H_kv = H_kv; kv->L = L; kv->T = T; kv->placement = placement; kv->free_bit = -1; kv->n_chunks = n_chunks;
-    kv->dst = (const uint8_t*)dst; kv->dst_bytes = dst_bytes; kv->d_quad_of = nullptr; kv->d_part = nullptr; kv->d_stats = nullptr;
+    kv->dst = (const uint8_t*)dst; kv->dst_bytes = dst_bytes; kv->d_quad_of = nullptr; kv->d_page_chunk = nullptr; kv->d_part = nullptr; kv->d_stats = nullptr;
     kv->h_quad_of.resize(n_quads);
     size_t on_die = 0;
     if (placement == 2) {
@@ -801,7 +827,7 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
         page_chunk[page0 + 2] = q + Fq;
         page_chunk[page0 + 3] = q + Fq + a;
     }
-    int32_t* d_chunk = nullptr;
+    int32_t*& d_chunk = kv->d_page_chunk;
     cudaError_t e = cudaMalloc(&kv->d_quad_of, sizeof(int32_t) * n_quads);
     if (e == cudaSuccess) e = cudaMemcpy(kv->d_quad_of, kv->h_quad_of.data(), sizeof(int32_t) * n_quads, cudaMemcpyHostToDevice);
     if (e == cudaSuccess && n_chunks > 1) e = cudaMalloc(&kv->d_part, sizeof(float) * (size_t)n_units * AT_MAXG * AT_D);
@@ -814,12 +840,23 @@ extern "C" ag_status ag_kv_pack(const void* K, const void* V, int B, int H_kv, i
         e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
-    cudaFree(d_chunk);
     if (e != cudaSuccess) {
         ag_kv_destroy(kv);
         return cuda_fail(e);
     }
     *out = kv;
+    return AG_OK;
+}
+
+extern "C" ag_status ag_kv_append(ag_kv_cache* kv, const void* k_new, const void* v_new, const int32_t* pos, void* cuda_stream) {
+    if (!kv || !k_new || !v_new || !pos) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    k_kv_append<<<(unsigned)(kv->B * kv->H_kv), AT_D, 0, stream>>>((const uint16_t*)k_new, (const uint16_t*)v_new, pos, kv->H_kv, kv->L,
+                                                                    kv->T, kv->d_page_chunk, const_cast<uint8_t*>(kv->dst));
+    count_launch();
+    AG_CUDA(cudaGetLastError());
     return AG_OK;
 }
 

@@ -120,6 +120,54 @@ def test_serving_shape_on_sm_budgets():
         check(got, want)
 
 
+def test_appended_tokens_land_where_packing_would_put_them():
+    """A decode loop: pack a cache that holds the first keys of every request, append the next tokens one step at a
+    time (request b is at its own position), attend after every step; every step must agree with the oracle on the
+    keys written so far, and the appended cache must equal a cache packed from the full K and V byte for byte."""
+    B, Hq, Hkv, L = 5, 8, 2, 384
+    Q, K, V = make_case(B, Hq, Hkv, L, seed=55)
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
+                                                               tile_n=128, k_splits=1))
+    kv_bytes = 2 * B * Hkv * L * 128 * 2
+    dst_bytes = 2 * kv_bytes + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    start = np.array([0, 5, 127, 200, 380], dtype=np.int32)          # keys that every request already has
+    K0, V0 = K.copy(), V.copy()
+    for b in range(B):
+        K0[b, :, start[b]:] = 0
+        V0[b, :, start[b]:] = 0
+    dK0, dV0, dQ = dev(K0), dev(V0), dev(Q)
+    kv = ag.kv_pack(dK0.data_ptr(), dV0.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes, ag.KV_LOCAL)
+    dO = torch.empty((B, Hq, 128), dtype=torch.float32, device="cuda")
+    lens = start.copy()
+    for step in range(4):
+        pos = np.where(lens < L, lens, -1).astype(np.int32)            # a full request takes no more tokens
+        k_new = np.stack([K[b, :, min(lens[b], L - 1)] for b in range(B)])   # [B][H_kv][128]
+        v_new = np.stack([V[b, :, min(lens[b], L - 1)] for b in range(B)])
+        d_pos, d_k, d_v = torch.from_numpy(pos).cuda(), dev(k_new), dev(v_new)
+        kv.append(d_k.data_ptr(), d_v.data_ptr(), d_pos.data_ptr())
+        lens = np.minimum(lens + 1, L).astype(np.int32)
+        d_len = torch.from_numpy(lens).cuda()
+        ag.attention_decode(dQ.data_ptr(), kv, d_len.data_ptr(), dO.data_ptr(), B, Hq, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        check(dO.cpu().numpy().astype(np.float64), oa.gqa_decode(Q, K, V, [int(x) for x in lens]))
+    appended = dst.cpu().numpy().copy()
+    # the same cache packed in one go from K and V with everything past the final lengths zeroed
+    K1, V1 = K.copy(), V.copy()
+    for b in range(B):
+        K1[b, :, lens[b]:] = 0
+        V1[b, :, lens[b]:] = 0
+    dst.zero_()
+    dK1, dV1 = dev(K1), dev(V1)
+    kv2 = ag.kv_pack(dK1.data_ptr(), dV1.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes, ag.KV_LOCAL)
+    torch.cuda.synchronize()
+    assert np.array_equal(appended, dst.cpu().numpy())
+    del kv2
+
+
 def test_bad_arguments():
     topo = device_topo()
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=4, N=128 * 8, K=256, tile_m=16,
