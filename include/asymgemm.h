@@ -327,6 +327,11 @@ ag_status ag_cluster_capacity(const ag_plan* plan, const ag_topo_map* map, int c
 ag_status ag_probe_cluster_layout(int cluster_size, int n_clusters, int32_t* cluster_of_sm);
 /* Device status word of the most recent launch (call after synchronising its stream). */
 ag_status ag_last_status(const ag_plan* plan);
+/* Where the first bounded wait of the last launches ran out (only meaningful while ag_last_status is AG_ERR_TIMEOUT):
+ * role = which wait of which warp role gave up (1-2 scheduler and copy warps waiting for room, 3-5 the MMA issuer
+ * waiting for a unit / an accumulator / data, 6-7 the epilogue or softmax warps, 8-9 copy warps and the MMA issuer
+ * waiting for a unit or activations), smid = the SM it happened on; 0 and -1 when nothing ran out.  Either may be NULL. */
+ag_status ag_last_status_where(const ag_plan* plan, int32_t* role, int32_t* smid);
 void ag_plan_destroy(ag_plan* plan);
 
 /*

@@ -26,7 +26,7 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_plan_set_grid", "ag_plan_adopted", "ag_cluster_capacity", "ag_probe_cluster_layout", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
+    "ag_plan_set_grid", "ag_plan_adopted", "ag_cluster_capacity", "ag_probe_cluster_layout", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_last_status_where", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
@@ -134,6 +134,7 @@ def lib() -> C.CDLL:
     L.ag_plan_set_grid.argtypes = [vp, C.c_int]
     L.ag_plan_adopted.argtypes = [vp, C.POINTER(C.c_uint32)]
     L.ag_last_status.argtypes = [vp]
+    L.ag_last_status_where.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.ag_plan_destroy.argtypes = [vp]
     L.ag_plan_destroy.restype = None
     L.gemm_persistent.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
@@ -412,6 +413,12 @@ class Plan:
 
     def last_status(self) -> int:
         return int(lib().ag_last_status(self.handle))
+
+    def last_status_where(self) -> tuple:
+        """(role, smid) of the first bounded wait that ran out; (0, -1) when none did."""
+        r, s_ = C.c_int32(), C.c_int32()
+        _check(lib().ag_last_status_where(self.handle, C.byref(r), C.byref(s_)), "ag_last_status_where")
+        return int(r.value), int(s_.value)
 
     def destroy(self):
         if self.handle:

@@ -294,13 +294,15 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const int words_new = ctl->ring_pages[r][lane];   // read before the slot is handed back
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+            // A unit without keys has nothing to stream, but like every entry it brings the value tiles of the unit before
+            // (whose outputs must not wait for a later entry: the softmax warps may be waiting for them before they take
+            // the next unit off the ring).
             const int n_t = u >= 0 ? unit_tiles(x, u) : 0;
-            if (u >= 0 && n_t == 0) continue;                 // a request without keys: nothing to stream
             words_cur = words_new;
-            if (u >= 0) copy_tiles(words_cur, n_t, 0);
+            if (n_t > 0) copy_tiles(words_cur, n_t, 0);
             if (prev_u >= 0 && ok) copy_tiles(words_prev, prev_t, 1);
             words_prev = words_cur;
-            prev_u = u;
+            prev_u = n_t > 0 ? u : -1;
             prev_t = n_t;
             if (u < 0) break;
         }
@@ -335,9 +337,8 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
                 const int u = ctl->ring[r];
                 mbar_arrive(smem_u32(&ctl->sched_empty[r]));
-                const int n_t = u >= 0 ? unit_tiles(x, u) : 0;
-                if (u >= 0 && n_t == 0) continue;
-                if (u >= 0) {
+                const int n_t = u >= 0 ? unit_tiles(x, u) : 0;     // 0: the end of the list, or a unit without keys
+                if (n_t > 0) {
                     // ---- S^T = K Q^T for every key tile of the unit
                     const uint32_t j = nq & 1;
                     if (!mbar_wait(smem_u32(&ctl->s_empty[j]), ((nq >> 1) & 1) ^ 1, abort_flag, limit) ||
@@ -369,7 +370,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
                 if (have_prev) {
                     // ---- O^T += V^T P^T for every key tile of the previous unit (probabilities as hi + lo bf16 parts)
-                    const uint32_t np = nq - (u >= 0 ? 2 : 1);          // ordinal of the previous unit
+                    const uint32_t np = nq - (n_t > 0 ? 2 : 1);         // ordinal of the previous unit
                     const uint32_t j = np & 1;
                     if (!mbar_wait(smem_u32(&ctl->o_empty[j]), ((np >> 1) & 1) ^ 1, abort_flag, limit)) {
                         report_timeout(p, 4);
@@ -399,7 +400,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (!ok) break;
                     tc_commit(smem_u32(&ctl->o_full[j]));
                 }
-                have_prev = u >= 0;
+                have_prev = n_t > 0;
                 prev_t = n_t;
                 if (u < 0) break;
             }
@@ -483,6 +484,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 prior_done = true;
             }
             if (n_t == 0) {
+                if (pend_u >= 0 && !(ok = write_outputs(nq - 1))) break;   // their products were issued on this entry
                 if (x.n_chunks == 1) {
                     float* out = x.O + (size_t)u * G * AT_D + i_lane;
                     for (int q = 0; q < G; ++q) out[(size_t)q * AT_D] = 0.f;

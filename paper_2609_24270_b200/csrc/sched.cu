@@ -715,6 +715,15 @@ extern "C" ag_status ag_last_status(const ag_plan* plan) {
     return AG_OK;
 }
 
+extern "C" ag_status ag_last_status_where(const ag_plan* plan, int32_t* role, int32_t* smid) {
+    if (!plan) return AG_ERR_ARG;
+    PlanCtrl c;
+    AG_CUDA(cudaMemcpy(&c, plan->d_ctrl, sizeof(int) * 8, cudaMemcpyDeviceToHost));
+    if (role) *role = c.status != 0 ? (c.status_info >> 16) : 0;
+    if (smid) *smid = c.status != 0 ? (c.status_info & 0xffff) : -1;
+    return AG_OK;
+}
+
 extern "C" void ag_plan_destroy(ag_plan* plan) {
     if (!plan) return;
     cudaFree(plan->d_image);

@@ -52,7 +52,7 @@ def run_attention(Q, K, V, placement, kv_len=None, budget=None, overlap=0):
         ag.attention_decode(dQ.data_ptr(), kv, None if dlen is None else dlen.data_ptr(), dO.data_ptr(), B, Hq, plan)
     torch.cuda.synchronize()
     st = plan.last_status()
-    assert st == ag.AG_OK, ag.strerror(st)
+    assert st == ag.AG_OK, (ag.strerror(st), plan.last_status_where())
     owner, count = plan.tile_record()
     assert (count == 2).all()
     return dO.cpu().numpy().astype(np.float64), kv.info(), dst
@@ -166,6 +166,35 @@ def test_appended_tokens_land_where_packing_would_put_them():
     torch.cuda.synchronize()
     assert np.array_equal(appended, dst.cpu().numpy())
     del kv2
+
+
+@pytest.mark.parametrize("lens", [[1024, 0], [0, 1024, 0, 700], [0, 0, 0, 1], [640, 0, 0, 1024]])
+def test_units_without_keys_between_long_units_on_one_sm(lens):
+    """One SM runs every unit in turn.  A unit with more key tiles than the ring of probability tiles holds needs its
+    value products issued while its softmax is still going on; they are issued when the next ring entry arrives, also
+    when that entry is a unit without keys (this case once ended in a bounded wait running out)."""
+    B, Hq, Hkv, L = len(lens), 4, 1, 1024
+    Q, K, V = make_case(B, Hq, Hkv, L, seed=404)
+    for budget in (1, 2):
+        got, _, _ = run_attention(Q, K, V, ag.KV_INTERLEAVED, kv_len=lens, budget=budget)
+        check(got, oa.gqa_decode(Q, K, V, lens))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_seeded_random_shapes(seed):
+    """Random batch, head counts, lengths (also beyond one chunk), SM budgets, placements and ragged kv_len."""
+    rng = np.random.default_rng(1000 + seed)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    B = int(rng.integers(1, 12))
+    L = 128 * int(rng.choice([1, 2, 3, 5, 8, 9, 16, 20]))
+    topo = device_topo()
+    budget = int(rng.choice([topo.n_sm, 74, 37, 11]))
+    placement = int(rng.choice([ag.KV_LOCAL, ag.KV_REMOTE, ag.KV_INTERLEAVED]))
+    Q, K, V = make_case(B, Hkv * G, Hkv, L, seed=2000 + seed, q_scale=float(rng.choice([1.0, 4.0, 16.0])))
+    lens = None if seed % 3 == 0 else [int(x) for x in rng.integers(0, L + 1, size=B)]
+    got, _, _ = run_attention(Q, K, V, placement, kv_len=lens, budget=budget)
+    check(got, oa.gqa_decode(Q, K, V, lens))
 
 
 def test_bad_arguments():
