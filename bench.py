@@ -39,6 +39,10 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch of the dominant kernel, from an Nsight Compute capture of two timed steps of this
 # bench (dram__bytes_read.sum 1.042 GB + dram__bytes_write.sum 0.251 GB; summary kept under profiles/).
 NCU_TRAFFIC_BYTES = 1.293e9
+# the same for the decode-shaped GEMM (135.08 MB read + 3.9 MB written per launch, 16 k-splits) and for the attention
+# kernel (269.69 MB + 3.7 MB); both captures read every algorithmic byte exactly once
+NCU_TRAFFIC_BYTES_DECODE = 1.390e8
+NCU_TRAFFIC_BYTES_ATTENTION = 2.734e8
 
 
 def load_peaks():
@@ -263,7 +267,7 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
             "clocks": sampler.summary("decode"),
             "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
                          "frac_4_k_splits": results[4]["packed_die_local"] / peaks["hbm_gbs"],
-                         "traffic": None, "kernel": "k_gemm_skinny<16, packed>", "algorithmic_bytes": algo_bytes,
+                         "traffic": NCU_TRAFFIC_BYTES_DECODE, "kernel": "k_gemm_skinny<16, packed>", "algorithmic_bytes": algo_bytes,
                          "peak_source": f"{peaks['source']} copy bandwidth"}}
 
 
@@ -314,7 +318,7 @@ def attention_section(ag, inputs, torch, topo, peaks, sampler):
             "gpu_launches": int(ag.kernel_launch_count() - launches0),
             "clocks": sampler.summary("attention"),
             "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
-                         "traffic": None, "kernel": "k_attn_decode", "algorithmic_bytes": algo_bytes,
+                         "traffic": NCU_TRAFFIC_BYTES_ATTENTION, "kernel": "k_attn_decode", "algorithmic_bytes": algo_bytes,
                          "peak_source": f"{peaks['source']} copy bandwidth"}}
 
 
