@@ -222,7 +222,7 @@ typedef struct {
     int32_t M, N, K;
     int32_t tile_m, tile_n;  /* dense kernel: 128 x {64,128,256}, or 256 x 256 (two thread blocks on the two SMs of a TPC
                                 share a unit; the plan's SM set must consist of whole TPCs, else AG_ERR_ARG);
-                                decode-shaped kernel: {16,32} x 128 */
+                                decode-shaped kernel: {16,32,64} x 128, and 128 x 128 with decode_shaped = 1 */
     int32_t k_splits;        /* >= 1, runs of whole k-slabs */
     int32_t k_unit;          /* elements per k-slab (64) */
     int32_t raster_group;    /* tile rows per raster group (>= 1) */
@@ -260,6 +260,10 @@ typedef struct {
                                 the dies that hold any SM of the set: for work bound by memory bandwidth whose operands are
                                 die-local, since every die's memory delivers the same bandwidth whatever its SM count (on a
                                 chip with 70 and 78 usable SMs the proportional split asks 5 % more of one die's memory) */
+    int32_t decode_shaped;   /* 1: a plan with tile_m = 128 and tile_n = 128 is run by the decode-shaped (weight-streaming)
+                                kernel - weights on the MMA's M side, up to 128 activation rows on its N side - instead of
+                                the dense one-block kernel.  Plans with tile_m <= 64 (and tile_n = 128) always are */
+    int32_t reserved3;
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;
@@ -342,9 +346,10 @@ void ag_plan_destroy(ag_plan* plan);
  *   B  device, K x N bf16 row-major, 16-byte aligned, N % 8 == 0
  *   C  device, M x N fp32 row-major, 16-byte aligned; overwritten.  Dense plans with k_splits > 1:
  *      zeroed first, partial sums are then added with reductions in memory.  Decode-shaped plans
- *      (tile_m <= 32): see policy.splitk_in_memory
+ *      (see below): see policy.splitk_in_memory
  *   the plan's tile shape selects the kernel: 256 x 256 units = pairs of thread blocks, 128 x
- *      {64,128,256} = one block per tile (any SM set), {16,32} x 128 = decode-shaped (M <= tile_m)
+ *      {64,128,256} = one block per tile (any SM set), {16,32,64} x 128 (and 128 x 128 with policy.decode_shaped)
+ *      = decode-shaped (M <= tile_m): the weight tile sits on the MMA's M side and is streamed once
  *   plan  built for the same M, N, K, else AG_ERR_ARG
  *   cuda_stream  a cudaStream_t (NULL = default stream).  Asynchronous.
  * Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA.  Device-side trouble
@@ -409,7 +414,7 @@ void ag_packed_destroy(ag_packed_weights* w);
  * gemm_persistent_packed - C = A * B with the B operand taken from a packed buffer
  * (Section 7.1.2 on top of Section 7.1.1: each block reads the pages of its units, which the
  * packing put on the block's own die when plan and packing agree).  Decode-shaped plans
- * (tile_m in {16, 32}, tile_n = 128, M <= tile_m) and dense plans of block pairs (256 x 256
+ * (tile_m in {16, 32, 64, 128}, tile_n = 128, M <= tile_m) and dense plans of block pairs (256 x 256
  * units, SM set of whole TPCs) are accepted; gemm_persistent handles the same shapes with
  * row-major B.
  *   A  device, M x K bf16 row-major, 16-byte aligned;  C  device, M x N fp32 row-major, overwritten

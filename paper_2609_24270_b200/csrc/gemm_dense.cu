@@ -379,7 +379,7 @@ extern "C" ag_status gemm_persistent(const void* A, const void* B, void* Cout, i
                                      const ag_plan* plan, void* cuda_stream) {
     if (!A || !B || !Cout || !plan) return AG_ERR_ARG;
     const int32_t* h = plan->header;
-    if (h[H_TILE_M] <= 32)  // decode-shaped plan: weights on the MMA's M side, split-K through the plan's scratch
+    if (is_decode_shaped(plan))  // weights on the MMA's M side, split-K through the plan's scratch
         return gemm_skinny_dispatch(A, B, nullptr, Cout, M, N, K, plan, plan->d_partial,
                                     reinterpret_cast<cudaStream_t>(cuda_stream));
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;

@@ -1,4 +1,4 @@
-// Decode-shaped (skinny) persistent GEMM: C[M x N] = A[M x K] * B[K x N] with M <= 32.  The
+// Decode-shaped (skinny) persistent GEMM: C[M x N] = A[M x K] * B[K x N] with M <= 128.  The
 // weights B are the work: every unit streams a 128-column weight tile over a run of k-slabs, so
 // the kernel is HBM bound.  The MMA is turned around: the weight tile is the M = 128 operand,
 // the activations are the N = 16 or 32 operand, D[n][m] accumulates in tensor memory.
@@ -33,20 +33,29 @@ constexpr int SK_BK = 64;      // k-slab
 //    k-slabs (32 KB of weights, 8 MMAs).
 constexpr int SK_SLABS = 2;    // k-slabs per weight stage
 constexpr int SK_WPROD = 3;    // warps that issue weight copies (stage i of the block's run belongs to warp i mod SK_WPROD)
-constexpr int SK_STAGES = 6;   // two stages per issuing warp; even, so that a buffer's parity is the parity of its place in the run
-constexpr int SK_NMMA = 2;     // threads that issue MMAs: thread t owns the stage buffers of parity t (see the MMA role)
+constexpr int SK_STAGES = 6;   // (at most) two stages per issuing warp; even, so that a buffer's parity is the parity of its place in the run
+constexpr int SK_NMMA = 2;     // warps that may issue MMAs: thread t owns the stage buffers of parity t (see the MMA role)
+// With 64 or 128 activation rows an MMA takes 56-64 cycles and a k-slab of activations 8-16 KB: one MMA-issuing thread
+// keeps up, and the activations of a stage's two k-slabs travel with its weights (one stage = 32 KB of weights + 16 or
+// 32 KB of activations, filled by the same warp onto the same barrier), so that both have the same pipeline depth.
+__host__ __device__ constexpr bool sk_unified(int nm) { return nm >= 64; }
+__host__ __device__ constexpr int sk_stages(int nm) { return nm == 64 ? 4 : nm == 128 ? 3 : SK_STAGES; }
+__host__ __device__ constexpr int sk_nmma(int nm) { return nm >= 64 ? 1 : SK_NMMA; }
 constexpr int SK_THREADS = (2 + kEpiWarps + SK_WPROD + (SK_NMMA - 1)) * 32;   // scheduler, MMA issuer, epilogue warps, weight producers, second MMA issuer
 constexpr int SK_MMA2_WARP = 2 + kEpiWarps + SK_WPROD;
 constexpr int SK_SLAB_BYTES = SK_BN * SK_BK * 2;   // 16 KB of weights per k-slab
 constexpr int SK_W_BYTES = SK_SLABS * SK_SLAB_BYTES;
-constexpr int SK_STAGE_BYTES = SK_W_BYTES;
 // Activations come in groups of SK_AGRP k-slabs, one copy per group (A seen as [K/64][M][64]): with one copy
 // per k-slab the warp that issues them - two copies in flight, each an L2 round trip - capped the whole
 // pipeline at one slab per ~400 ns, the same 42 GB/s per SM that a single weight-issuing thread reaches.
 constexpr int SK_ASTAGES = 2;
 constexpr int SK_A_STAGE_MAX = 16 * 1024;          // 8 k-slabs of 16 rows, or 4 k-slabs of 32 rows
-__host__ __device__ constexpr int sk_agrp(int nm) { return SK_A_STAGE_MAX / (nm * SK_BK * 2); }
-constexpr int SK_SMEM_BYTES = SK_STAGES * SK_STAGE_BYTES + SK_ASTAGES * SK_A_STAGE_MAX + 1024 + 1024;
+__host__ __device__ constexpr int sk_agrp(int nm) { return nm >= 64 ? 2 : SK_A_STAGE_MAX / (nm * SK_BK * 2); }   // 64 / 128 rows: 2 k-slabs (16 / 32 KB)
+__host__ __device__ constexpr int sk_a_stage_bytes(int nm) { return sk_agrp(nm) * nm * SK_BK * 2; }
+__host__ __device__ constexpr int sk_stage_bytes(int nm) { return SK_W_BYTES + (sk_unified(nm) ? sk_a_stage_bytes(nm) : 0); }
+__host__ __device__ constexpr int sk_smem_bytes(int nm) {
+    return sk_stages(nm) * sk_stage_bytes(nm) + (sk_unified(nm) ? 0 : SK_ASTAGES * sk_a_stage_bytes(nm)) + 1024 + 1024;
+}
 // The tensor core takes ~45 cycles for an MMA this small whether or not it adds to the accumulator of the one
 // before (measured), so one accumulator per unit is enough.
 
@@ -134,10 +143,14 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     constexpr uint32_t kASlab = NM * SK_BK * 2;          // activations of one k-slab
     constexpr int SK_AGRP = sk_agrp(NM);                 // k-slabs per activation copy
     constexpr uint32_t kAStage = SK_AGRP * kASlab;
-    const uint32_t a_base = base + SK_STAGES * SK_STAGE_BYTES;
-    SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + SK_STAGES * SK_STAGE_BYTES + SK_ASTAGES * SK_A_STAGE_MAX);
+    constexpr int kStages = sk_stages(NM);               // weight stages
+    constexpr int kNMMA = sk_nmma(NM);                   // MMA-issuing threads at work
+    constexpr bool kUnified = sk_unified(NM);            // activations inside the weight stages
+    constexpr uint32_t kStageBytes = sk_stage_bytes(NM);
+    const uint32_t a_base = base + kStages * kStageBytes;
+    SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + kStages * kStageBytes + (kUnified ? 0 : SK_ASTAGES * kAStage));
     constexpr uint32_t kAccCols = NM;                    // columns of one accumulator
-    constexpr uint32_t kTmemCols = 2 * SK_NMMA * kAccCols;   // two units in flight, one accumulator per MMA-issuing thread each (64 or 128 columns)
+    constexpr uint32_t kTmemCols = 2 * kNMMA * kAccCols < 32 ? 32 : 2 * kNMMA * kAccCols;   // two units in flight, one accumulator per MMA-issuing thread each
     volatile int* abort_flag = &ctl->abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int my_sm = (int)smid();
@@ -151,21 +164,21 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         ctl->quick = qk;
         ctl->member = qk.x >= 0 && atomicMax(&p.claimed[qk.x], p.epoch) < p.epoch;
     } else if (tid == 64) {
-        for (int i = 0; i < SK_STAGES; ++i) {
+        for (int i = 0; i < kStages; ++i) {
             mbar_init(smem_u32(&ctl->full[i]), 1);
             mbar_init(smem_u32(&ctl->empty[i]), 1);
         }
         for (int i = 0; i < SK_ASTAGES; ++i) {
             mbar_init(smem_u32(&ctl->a_full[i]), 1);
-            mbar_init(smem_u32(&ctl->a_empty[i]), SK_NMMA);
+            mbar_init(smem_u32(&ctl->a_empty[i]), kNMMA);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&ctl->tmem_full[i]), SK_NMMA);
+            mbar_init(smem_u32(&ctl->tmem_full[i]), kNMMA);
             mbar_init(smem_u32(&ctl->tmem_empty[i]), kEpiWarps);
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&ctl->sched_full[i]), 1);
-            mbar_init(smem_u32(&ctl->sched_empty[i]), SK_NMMA + kEpiWarps + SK_WPROD);
+            mbar_init(smem_u32(&ctl->sched_empty[i]), kNMMA + kEpiWarps + SK_WPROD);
         }
         for (int i = 0; i < SK_NMMA; ++i) mbar_init(smem_u32(&ctl->mma_drain[i]), 1);
         mbar_fence_init();
@@ -237,7 +250,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const int grp = x.tiles_per_group ? tn / x.tiles_per_group : 0;      // expert of this column tile
             const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
             const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
-            if (lane == 0) {
+            if (!kUnified && lane == 0) {
                 const CUtensorMap* ma = x.g_tm_a ? &x.g_tm_a[grp] : &tm_a;
                 for (int g0 = s0; g0 < s1; g0 += SK_AGRP, ++git) {
                     const int j = git % SK_ASTAGES;
@@ -293,7 +306,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const int n_st = (s1 - s0 + SK_SLABS - 1) / SK_SLABS;    // stages of this unit: slabs s0 + 2i, s0 + 2i + 1
             // this warp's stages of the unit: i0, i0 + SK_WPROD, ...
             const int i0 = (pw + SK_WPROD - (int)(q0 % SK_WPROD)) % SK_WPROD;
-            uint32_t st = (q0 + i0) % SK_STAGES, ph = (((q0 + i0) / SK_STAGES) & 1) ^ 1;   // stage, parity of "stage is free"
+            uint32_t st = (q0 + i0) % kStages, ph = (((q0 + i0) / kStages) & 1) ^ 1;   // stage, parity of "stage is free"
             const CUtensorMap* mw = x.g_tm_w ? &x.g_tm_w[grp] : &tm_w;
             // packed weights: lane l < 2 (groups of four pages) or l < 8 (single pages) looks up the chunk of the
             // l-th 16 KB / 4 KB piece of a stage, one stage ahead of the copies
@@ -332,14 +345,22 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 const int s = s0 + i * SK_SLABS;
                 const int ns = min(SK_SLABS, s1 - s);
                 const uint32_t bar = smem_u32(&ctl->full[st]);
-                const uint32_t sw = base + st * SK_STAGE_BYTES;
+                const uint32_t sw = base + st * kStageBytes;
                 if (lane == 0) {
                     if (!mbar_wait(smem_u32(&ctl->empty[st]), ph, abort_flag, limit)) {
                         report_timeout(p, 2);
                         ok = 0;
                     } else {
                         // row-major weights: one box of 128 k rows whatever ns is (rows past K arrive as zeros)
-                        mbar_expect_tx(bar, PACKED ? ns * SK_SLAB_BYTES : SK_W_BYTES);
+                        uint32_t bytes = PACKED ? ns * SK_SLAB_BYTES : SK_W_BYTES;
+                        if (kUnified) bytes += p.a_blocks ? kAStage : ns * kASlab;
+                        mbar_expect_tx(bar, bytes);
+                        if (kUnified) {
+                            // the activations of the stage's k-slabs, behind its weights
+                            const CUtensorMap* ma = x.g_tm_a ? &x.g_tm_a[grp] : &tm_a;
+                            if (p.a_blocks) tma_load_3d(sw + SK_W_BYTES, ma, bar, 0, 0, s);
+                            else for (int j = 0; j < ns; ++j) tma_load_2d(sw + SK_W_BYTES + j * kASlab, ma, bar, (s + j) * SK_BK, 0);
+                        }
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -365,14 +386,14 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 }
                 // this warp's next stage is SK_WPROD stages on
                 st += SK_WPROD;
-                if (st >= SK_STAGES) { st -= SK_STAGES; ph ^= 1; }
+                if (st >= (uint32_t)kStages) { st -= kStages; ph ^= 1; }
             }
             q0 += (uint32_t)n_st;
         }
         if (!ok && lane == 0) linger_for_copies();
     } else if (warp == 1 || warp == SK_MMA2_WARP) {
-        if (lane == 0) {
-            // ------------------------------------------------ MMA issuers.  Thread t (0: warp 1, 1: the last warp) owns the
+        if (lane == 0 && (warp == 1 || kNMMA == 2)) {
+            // ------------------------------------------------ MMA issuers (with 64 or 128 activation rows: warp 1 alone).  Thread t (0: warp 1, 1: the last warp) owns the
             // stage buffers of parity t, i.e. every second stage of the block's run.  One thread alone is the cap of the
             // pipeline below the full chip: it spends 500-700 cycles per 32 KB stage (eight MMAs of ~45 cycles, a barrier
             // wait, a fence, a commit), i.e. at most ~50 B per cycle, where the copies deliver more.
@@ -392,8 +413,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             constexpr uint32_t kWStep = (PACKED ? 4096u : 2048u) >> 4;   // one K = 16 step inside a weight stage
             constexpr uint32_t kAStepK = 32u >> 4;                       // ... inside an activation slab
             constexpr int kGrpStages = SK_AGRP / SK_SLABS;               // stages per activation buffer (even)
-            static_assert(kGrpStages % SK_NMMA == 0, "every full activation group has stages of both threads");
-            static_assert(SK_STAGES % SK_NMMA == 0, "a stage buffer always belongs to the same thread");
+            static_assert(kGrpStages % kNMMA == 0, "every full activation group has stages of both threads");
+            static_assert(kStages % kNMMA == 0, "a stage buffer always belongs to the same thread");
             const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
             uint32_t q0 = 0;                          // stages of the units before this one (over the whole run of the block)
             uint32_t git = 0;                         // activation groups before this unit
@@ -420,10 +441,36 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                     break;
                 }
                 tc_fence_after();
-                const int a = (t - (int)(q0 & 1u)) & 1;       // parity, inside the unit, of the stages in this thread's buffers
-                const uint32_t d_tmem = tmem_base + (acc * SK_NMMA + a) * kAccCols;
-                uint32_t st = (q0 + a) % SK_STAGES, ph = ((q0 + a) / SK_STAGES) & 1;   // this thread's first stage of the unit
+                const int a = kNMMA == 2 ? (t - (int)(q0 & 1u)) & 1 : 0;   // parity, inside the unit, of the stages in this thread's buffers
+                const uint32_t d_tmem = tmem_base + (acc * kNMMA + a) * kAccCols;
+                uint32_t st = (q0 + a) % kStages, ph = ((q0 + a) / kStages) & 1;   // this thread's first stage of the unit
                 bool first = true;
+                if constexpr (kUnified) {
+                    // activations behind the weights of the same stage: one barrier per stage, no activation buffers
+                    for (int i = 0; i < n_st; ++i) {
+                        if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
+                            report_timeout(p, 5);
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t sbase = base + st * kStageBytes;
+                        const uint64_t dw = dw_t | (uint64_t)(sbase >> 4);
+                        const uint64_t da = da_t | (uint64_t)((sbase + SK_W_BYTES) >> 4);
+                        tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
+#pragma unroll
+                        for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
+                        if (n_slabs - i * SK_SLABS > 1) {
+                            const uint64_t da2 = da + (kASlab >> 4);
+#pragma unroll
+                            for (int k4 = 0; k4 < SK_BK / 16; ++k4)
+                                tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                        }
+                        first = false;
+                        tc_commit(empty0 + st * 8);
+                        if (++st == (uint32_t)kStages) { st = 0; ph ^= 1; }
+                    }
+                } else
                 for (int g = 0; g < n_grp && ok; ++g) {
                     const uint32_t gi = git + g, aj = gi % SK_ASTAGES, aph = (gi / SK_ASTAGES) & 1;
                     const int i_end = min(n_st, (g + 1) * kGrpStages);
@@ -441,14 +488,14 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         break;
                     }
                     uint64_t da = (da_t | (uint64_t)((a_base + aj * kAStage) >> 4)) + (uint32_t)a * (SK_SLABS * (kASlab >> 4));
-                    for (; i < i_end; i += SK_NMMA) {
+                    for (; i < i_end; i += kNMMA) {
                         if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
                             report_timeout(p, 5);
                             ok = false;
                             break;
                         }
                         tc_fence_after();
-                        const uint64_t dw = dw_t | (uint64_t)((base + st * SK_STAGE_BYTES) >> 4);
+                        const uint64_t dw = dw_t | (uint64_t)((base + st * kStageBytes) >> 4);
                         // the first k-slab of the stage, then the second one if the unit has it
                         tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
 #pragma unroll
@@ -461,9 +508,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         }
                         first = false;
                         tc_commit(empty0 + st * 8);
-                        st += SK_NMMA;
-                        if (st >= SK_STAGES) { st -= SK_STAGES; ph ^= 1; }
-                        da += SK_NMMA * SK_SLABS * (kASlab >> 4);
+                        st += kNMMA;
+                        if (st >= (uint32_t)kStages) { st -= kStages; ph ^= 1; }
+                        da += kNMMA * SK_SLABS * (kASlab >> 4);
                     }
                     if (ok) tc_commit(smem_u32(&ctl->a_empty[aj]));    // this thread's last read of the buffer has been issued
                 }
@@ -504,25 +551,6 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 break;
             }
             tc_fence_after();
-            float sum[NM];
-            {
-                // the accumulator of the thread that took the even stages, plus the other one's if the unit has a second stage
-                uint32_t v[NM], w[NM];
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * SK_NMMA * kAccCols;
-                const int s0e = min(p.kslabs_total, ks * p.kslabs_per_split), s1e = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
-                const bool two = s1e - s0e > SK_SLABS;
-                if constexpr (NM == 16) tmem_ld_32x16(taddr, v); else tmem_ld_32x32(taddr, v);
-                if (two) {
-                    if constexpr (NM == 16) tmem_ld_32x16(taddr + kAccCols, w); else tmem_ld_32x32(taddr + kAccCols, w);
-                }
-                tmem_ld_wait();
-#pragma unroll
-                for (int m = 0; m < NM; ++m) sum[m] = two ? __uint_as_float(v[m]) + __uint_as_float(w[m]) : __uint_as_float(v[m]);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
-            ++tile_it;
             // This kernel may have started while the one before it (the zeroing of C, the adding-up of the previous
             // call's workspace, or with overlap_launches the previous GEMM) was still running (programmatic dependent
             // launch): before the first byte is written, make sure that everything before it on the stream has completed.
@@ -533,25 +561,50 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const int n = tn * SK_BN + q * 32 + lane;     // column in the plan's (possibly grouped) N
             const OutView ov = out_view(p, x, tn);
             const int nl = ov.col0 + q * 32 + lane;       // column inside the tile's problem
-            if (p.k_splits > 1 && x.partial == nullptr) {
-                // in-memory reduction: L2 carries out the additions; nothing comes back, so nothing is waited for
-                if (nl < ov.n_cols) {
+            const int s0e = min(p.kslabs_total, ks * p.kslabs_per_split), s1e = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
+            const bool two = kNMMA == 2 && s1e - s0e > SK_SLABS;   // the unit has stages of the second MMA-issuing thread too
+            constexpr int kChunk = NM < 32 ? NM : 32;     // activation rows handled at a time
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kNMMA * kAccCols;
 #pragma unroll
-                    for (int m = 0; m < NM; ++m)
-                        if (m < ov.rows) atomicAdd(ov.base + (size_t)m * ov.ld + nl, sum[m]);
+            for (int c0 = 0; c0 < NM; c0 += kChunk) {
+                float sum[kChunk];
+                {
+                    // the accumulator of the thread that took the even stages, plus the other one's if the unit has a second stage
+                    uint32_t v[kChunk], w[kChunk];
+                    if constexpr (kChunk == 16) tmem_ld_32x16(taddr + c0, v); else tmem_ld_32x32(taddr + c0, v);
+                    if (two) {
+                        if constexpr (kChunk == 16) tmem_ld_32x16(taddr + kAccCols + c0, w); else tmem_ld_32x32(taddr + kAccCols + c0, w);
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int m = 0; m < kChunk; ++m) sum[m] = two ? __uint_as_float(v[m]) + __uint_as_float(w[m]) : __uint_as_float(v[m]);
                 }
-            } else if (p.k_splits > 1) {
-                float* out = x.partial + (size_t)ks * p.M * p.N;   // workspace rows: the plan's M bound, columns: the plan's N
-                if (n < p.N) {
-#pragma unroll
-                    for (int m = 0; m < NM; ++m)
-                        if (m < p.M) out[(size_t)m * p.N + n] = sum[m];
+                if (c0 + kChunk >= NM) {                  // the last chunk has been read: the accumulators may be reused
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
                 }
-            } else if (nl < ov.n_cols) {
+                if (p.k_splits > 1 && x.partial == nullptr) {
+                    // in-memory reduction: L2 carries out the additions; nothing comes back, so nothing is waited for
+                    if (nl < ov.n_cols) {
 #pragma unroll
-                for (int m = 0; m < NM; ++m)
-                    if (m < ov.rows) ov.base[(size_t)m * ov.ld + nl] = sum[m];
+                        for (int m = 0; m < kChunk; ++m)
+                            if (c0 + m < ov.rows) atomicAdd(ov.base + (size_t)(c0 + m) * ov.ld + nl, sum[m]);
+                    }
+                } else if (p.k_splits > 1) {
+                    float* out = x.partial + (size_t)ks * p.M * p.N;   // workspace rows: the plan's M bound, columns: the plan's N
+                    if (n < p.N) {
+#pragma unroll
+                        for (int m = 0; m < kChunk; ++m)
+                            if (c0 + m < p.M) out[(size_t)(c0 + m) * p.N + n] = sum[m];
+                    }
+                } else if (nl < ov.n_cols) {
+#pragma unroll
+                    for (int m = 0; m < kChunk; ++m)
+                        if (c0 + m < ov.rows) ov.base[(size_t)(c0 + m) * ov.ld + nl] = sum[m];
+                }
             }
+            ++tile_it;
             if (lane == 0 && q == 0) {
                 p.tile_owner[u] = my_sm;
                 if (p.unit_times) p.unit_times[2 * u + 1] = globaltimer_ns();
@@ -635,14 +688,14 @@ static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, con
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
         attr_err = cudaFuncSetAttribute(k_gemm_skinny<NM, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SK_SMEM_BYTES);
+                                        sk_smem_bytes(NM));
     });
     if (attr_err != cudaSuccess) return launch_failed(plan, attr_err);
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm);
     cfg.blockDim = dim3(SK_THREADS);
-    cfg.dynamicSmemBytes = SK_SMEM_BYTES;
+    cfg.dynamicSmemBytes = sk_smem_bytes(NM);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -661,7 +714,8 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
                                const ag_group_desc* grp) {
     const int32_t* h = plan->header;
     if (M != h[H_M] || N != h[H_N] || K != h[H_K]) return AG_ERR_ARG;
-    if (h[H_TILE_N] != SK_BN || (h[H_TILE_M] != 16 && h[H_TILE_M] != 32) || M > h[H_TILE_M]) return AG_ERR_ARG;
+    const int tile_m = h[H_TILE_M];
+    if (h[H_TILE_N] != SK_BN || (tile_m != 16 && tile_m != 32 && tile_m != 64 && tile_m != 128) || M > tile_m) return AG_ERR_ARG;
     if (plan->policy.k_unit != SK_BK || (K % 8) || (N % 8)) return AG_ERR_ARG;
     if (((uintptr_t)A | (uintptr_t)Cout) & 15u) return AG_ERR_ARG;
     ag_status st = check_arch();
@@ -752,10 +806,15 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
     gp.a_blocks = a_blocks ? 1 : 0;
     ag_status ls;
-    if (NM == 16) ls = W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
-                         : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
-    else ls = W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap)
-                : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, zeroing || overlap);
+    const bool early = zeroing || overlap;
+    if (NM == 16) ls = W ? launch_skinny<16, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early)
+                         : launch_skinny<16, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early);
+    else if (NM == 32) ls = W ? launch_skinny<32, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early)
+                              : launch_skinny<32, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early);
+    else if (NM == 64) ls = W ? launch_skinny<64, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early)
+                              : launch_skinny<64, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early);
+    else ls = W ? launch_skinny<128, true>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early)
+                : launch_skinny<128, false>(plan, tm_a, tm_w, tm_w2, gp, x, stream, early);
     if (ls != AG_OK || !x.partial) return ls;
     // bit-reproducible split-K: the workspace slices are added in ascending split order by a second kernel, which may
     // become resident while the GEMM runs and waits for its completion on the device
@@ -1069,7 +1128,7 @@ extern "C" ag_status ag_group_desc_create(const void* A_all, void* C_all, const 
                                           ag_group_desc** out) {
     if (!A_all || !C_all || !rows || !out || G < 1 || G > 4096 || N_expert <= 0 || K <= 0) return AG_ERR_ARG;
     const bool dense = tile_m == 256;  // block pairs, 256 x 256 units; else decode-shaped (rows <= tile_m)
-    if ((tile_m != 16 && tile_m != 32 && !dense) || (N_expert % (dense ? 256 : SK_BN)) || (K % 8)) return AG_ERR_ARG;
+    if ((tile_m != 16 && tile_m != 32 && tile_m != 64 && tile_m != 128 && !dense) || (N_expert % (dense ? 256 : SK_BN)) || (K % 8)) return AG_ERR_ARG;
     if (((uintptr_t)A_all | (uintptr_t)C_all) & 15u) return AG_ERR_ARG;
     *out = nullptr;
     long long total = 0;

@@ -251,6 +251,12 @@ bool encode_b_blocks(CUtensorMap* tm, const void* ptr, uint64_t K, uint64_t N, u
 bool encode_a_slabs(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows, uint32_t n_slabs);
 
 // Host-side dispatchers of the kernel families (defined next to their kernels).
+// Plans that the decode-shaped (weight-streaming) kernel runs: 128-column units with at most 64 activation rows, or
+// 128 rows when the policy says so (128 x 128 is also a tile of the dense one-block kernel).
+inline bool is_decode_shaped(const ag_plan* plan) {
+    const int32_t* h = plan->header;
+    return h[H_TILE_N] == 128 && (h[H_TILE_M] <= 64 || (h[H_TILE_M] == 128 && plan->policy.decode_shaped));
+}
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
                                int N, int K, const ag_plan* plan, float* partial, cudaStream_t stream,
                                const ag_group_desc* grp = nullptr);

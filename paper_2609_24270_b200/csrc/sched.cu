@@ -517,7 +517,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         TRY(cudaMalloc(&pl->d_tile_count, sizeof(int32_t) * n_units));
         TRY(cudaMemset(pl->d_tile_owner, 0xFF, sizeof(int32_t) * n_units));
         TRY(cudaMemset(pl->d_tile_count, 0, sizeof(int32_t) * n_units));
-        if (p.tile_m <= 32 && p.k_splits > 1 && !p.splitk_in_memory) {
+        if (p.tile_n == 128 && (p.tile_m <= 64 || (p.tile_m == 128 && p.decode_shaped)) && p.k_splits > 1 && !p.splitk_in_memory) {
             // decode-shaped plans: split-K partial sums and per-tile arrival counters
             TRY(cudaMalloc(&pl->d_partial, sizeof(float) * (size_t)p.k_splits * p.M * p.N));
         }

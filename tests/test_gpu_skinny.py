@@ -54,6 +54,43 @@ def test_rowmajor_weights_uniform(shape, in_memory):
             check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
 
 
+@pytest.mark.parametrize("M,tile_m", [(64, 64), (48, 64), (128, 128), (100, 128), (33, 64)])
+@pytest.mark.parametrize("k_splits,in_memory", [(1, 0), (4, 0), (4, 1)])
+def test_up_to_128_activation_rows_integer_exact(M, tile_m, k_splits, in_memory):
+    """64 and 128 activation rows on the MMA's N side (one MMA-issuing thread, four weight stages): bit-exact on integer
+    inputs, row-major and die-packed weights, full chip and 37 SMs; 128 rows need policy.decode_shaped."""
+    N, K = 1024, 1024
+    A, B = inputs.small_int_bf16(M, K, 21), inputs.small_int_bf16(K, N, 22)
+    want = og.gemm_blocked(A, B)
+    topo = device_topo()
+    for b in (topo.n_sm, 37):
+        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=tile_m, tile_n=128,
+                                                            k_splits=k_splits, splitk_in_memory=in_memory, decode_shaped=1))
+        for _ in range(2):
+            assert np.array_equal(run_rowmajor(A, B, plan).astype(np.float64), want)
+    dst_bytes = 2 * K * N * 2 + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    dA, dB = to_dev_bf16(A), to_dev_bf16(B)
+    packed = ag.pack_weights(dB.data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes)
+    dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK
+    assert np.array_equal(dC.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("shape", [(64, 8192, 8192, 4), (128, 4096, 4096, 8), (96, 1000, 520, 2), (128, 384, 1344, 1)])
+def test_up_to_128_activation_rows_uniform(shape):
+    M, N, K, ksp = shape
+    A, B = inputs.gemm_inputs(M, N, K, seed=41)
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, splitk_in_memory=1, decode_shaped=1,
+                                                                tile_m=64 if M <= 64 else 128, tile_n=128, k_splits=ksp, overlap_launches=1))
+    for _ in range(3):
+        check_close(run_rowmajor(A, B, plan), og.gemm_blocked(A, B))
+
+
 def test_workspace_split_k_is_bit_reproducible():
     """splitk_in_memory = 0: the k-split slices are added in ascending split order, so the bits of C do not depend on
     which SMs ran which unit, nor on the order in which the units finished: the same C, bit for bit, from the full
