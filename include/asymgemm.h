@@ -443,7 +443,7 @@ typedef struct ag_group_desc ag_group_desc;
  *          (tile_m = 256, block pairs, N_expert % 256 == 0): any row count
  *   B_list host array of G device pointers (K x N_expert bf16 row-major each), or NULL when only
  *          packed weights will be used
- *   N_expert % 128 == 0, K % 8 == 0, tile_m in {16, 32, 256}
+ *   N_expert % 128 == 0, K % 8 == 0, tile_m in {16, 32, 64, 128, 256}
  * Errors: AG_ERR_ARG, AG_ERR_CUDA, AG_ERR_NOMEM.
  */
 ag_status ag_group_desc_create(const void* A_all, void* C_all, const int32_t* rows, int G,
@@ -484,7 +484,7 @@ ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weight
  *
  * Limits: k_splits * M * N * 4 bytes <= 8 MiB (for example M = 16, N = 8192, k_splits = 16) and
  * N <= 131072; larger problems are refused with AG_ERR_ARG, as are plans that are not
- * decode-shaped (tile_m > 32).  Arguments are those of gemm_persistent; the plan may come from a
+ * decode-shaped with at most 32 rows (tile_m > 32).  Arguments are those of gemm_persistent; the plan may come from a
  * sched_build done at start-up, when allocation was still allowed.
  *
  * The first call on each device also looks up the workspace's device address; make that first call
