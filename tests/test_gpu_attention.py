@@ -101,6 +101,8 @@ def test_long_requests_in_chunks(placement, shape):
     Q, K, V = make_case(B, Hq, Hkv, L, seed=300 + L, q_scale=6.0)
     got, _, _ = run_attention(Q, K, V, placement)
     check(got, oa.gqa_decode(Q, K, V))
+    got, _, _ = run_attention(Q, K, V, placement, overlap=1)     # the second launch begins while the first one finishes
+    check(got, oa.gqa_decode(Q, K, V))
     # ragged: lengths that end inside a chunk, at a chunk boundary, in the first chunk, and zero
     lens = [L - 1, 1025, 0][:B] if B == 3 else [1024, L - 127][:B]
     got, _, _ = run_attention(Q, K, V, placement, kv_len=lens)
