@@ -298,3 +298,4 @@ def test_unit_timeline(tile_m):
     if tile_m == 128 and len(lst) > 1:
         assert all(t1[lst[i]] <= t1[lst[i + 1]] for i in range(len(lst) - 1))
     plan.trace(False)
+
