@@ -212,9 +212,12 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
     results, err, info = {}, {}, {}
     sampler.mark("decode")
     for ksp in (16, 4):
-        kw = dict(M=Md, N=Nd, K=Kd, tile_m=16, tile_n=128, k_splits=ksp, overlap_launches=1)
+        # (the calls are independent of each other - same activations, rotating weights - so they may read their activations at
+        # once: overlap_launches = 2; the arm *_activations_after_prior_call runs with 1, the setting for a chain of calls)
+        kw = dict(M=Md, N=Nd, K=Kd, tile_m=16, tile_n=128, k_splits=ksp, overlap_launches=2)
         plan_local = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, splitk_in_memory=1, **kw))
         plan_ws = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, splitk_in_memory=0, **kw))
+        plan_chain = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, splitk_in_memory=1, **dict(kw, overlap_launches=1)))
         plan_obl = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_OBLIVIOUS, splitk_in_memory=1, **kw))
         packs = [ag.pack_weights(dBs[i].data_ptr(), Kd, Nd, plan_local, amaps[i], dsts[i].data_ptr(), dst_bytes) for i in range(n_buf)]
         bop = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packs[0].page_table())
@@ -234,7 +237,8 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
         gbs = {}
         arms = (("packed_die_local", plan_local, True), ("packed_remote", plan_remote, True),
                 ("rowmajor_oblivious", plan_obl, False), ("rowmajor_die_compact", plan_local, False),
-                ("packed_die_local_workspace_split_k", plan_ws, True))
+                ("packed_die_local_workspace_split_k", plan_ws, True),
+                ("packed_die_local_activations_after_prior_call", plan_chain, True))
         for _ in range(2):                                    # two passes so that the arms share the clock drift
             for name, plan, packed in arms:
                 state = {"i": 0}

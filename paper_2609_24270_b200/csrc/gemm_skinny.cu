@@ -94,6 +94,7 @@ struct SkinnyArgs {
     int tiles_per_group;
     int n_group;                  // columns of one expert
     int release_next;             // 1: let the next launch on the stream start while this one is still running
+    int a_after_prior;            // 1: the activations may be the product of the launch before: read them only after it has completed
     // closed form of the page table (PACKED): see table_entry in the kernel
     const int32_t* unit_base;     // device [tiles_n * k_splits] or null (then the tables above are read)
     const uint32_t* page_bits;    // device: one hash bit per 2 MiB page of the packed buffer
@@ -252,6 +253,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
             if (!kUnified && lane == 0) {
                 const CUtensorMap* ma = x.g_tm_a ? &x.g_tm_a[grp] : &tm_a;
+                // (this kernel may have started early: the weights stream at once, the activations - which the launch
+                // before may have written - only after that launch has completed)
+                if (git == 0 && x.a_after_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
                 for (int g0 = s0; g0 < s1; g0 += SK_AGRP, ++git) {
                     const int j = git % SK_ASTAGES;
                     if (!mbar_wait_idle(smem_u32(&ctl->a_empty[j]), ((git / SK_ASTAGES) & 1) ^ 1, abort_flag, limit)) {
@@ -282,6 +286,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         const int pw = warp - (2 + kEpiWarps);
         const uint64_t stream_policy = l2_policy_evict_first();  // weights are read once: do not keep them in L2
         uint32_t q0 = 0;      // stage count (over the whole run of this block) before the current unit
+        bool a_ready = false; // (activations inside the stages) everything launched before is known to be complete
         int ok = 1;
         for (uint32_t it = 0; ok; ++it) {
             const int r = it % kRing;
@@ -356,7 +361,12 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         if (kUnified) bytes += p.a_blocks ? kAStage : ns * kASlab;
                         mbar_expect_tx(bar, bytes);
                         if (kUnified) {
-                            // the activations of the stage's k-slabs, behind its weights
+                            // the activations of the stage's k-slabs, behind its weights (when this kernel may have started
+                            // early: only once the launch before, which may have written them, has completed)
+                            if (!a_ready) {
+                                if (x.a_after_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+                                a_ready = true;
+                            }
                             const CUtensorMap* ma = x.g_tm_a ? &x.g_tm_a[grp] : &tm_a;
                             if (p.a_blocks) tma_load_3d(sw + SK_W_BYTES, ma, bar, 0, 0, s);
                             else for (int j = 0; j < ns; ++j) tma_load_2d(sw + SK_W_BYTES + j * kASlab, ma, bar, (s + j) * SK_BK, 0);
@@ -785,6 +795,7 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     // belong to one launch at a time.
     const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0 && plan->lay.b == plan->lay.n_sm;
     x.release_next = overlap ? 1 : 0;
+    x.a_after_prior = (overlap && plan->policy.overlap_launches != 2) ? 1 : 0;
     if (zeroing) {  // in-memory reduction mode: the adds need a zeroed C (N % 8 == 0 and 16-byte alignment: whole float4s)
         const size_t c_elems = grp ? (size_t)grp->total_rows * (size_t)grp->N : (size_t)M * (size_t)N;
         const size_t n_vec = c_elems / 4;

@@ -114,8 +114,9 @@ def config3(fh, topo, budgets=(16, 32, 48, 64, 74), n_subsets=32):
 
 
 # ---------------------------------------------------------------------------------------------
-def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=1, k_splits=(16, 4)):
-    """M=16, N=K=8192 decode-shaped GEMM, weights die-packed; die-local vs remote assignment; 16 and 4 k-splits."""
+def config4(fh, topo, budgets=(37, 74, 148), n_buffers=4, overlap=2, k_splits=(16, 4)):
+    """M=16, N=K=8192 decode-shaped GEMM, weights die-packed; die-local vs remote assignment; 16 and 4 k-splits.
+    The calls are independent (same activations, rotating weights): overlap_launches = 2."""
     for ksp in k_splits:
         _config4(fh, topo, budgets, n_buffers, overlap, ksp)
 

@@ -111,8 +111,39 @@ def test_workspace_split_k_is_bit_reproducible():
         assert o.tobytes() == outs[0].tobytes()
 
 
-@pytest.mark.parametrize("in_memory", [0, 1])
-def test_overlapping_launches_integer_exact(in_memory):
+def test_overlapping_launches_in_a_dependent_chain():
+    """overlap_launches = 1 in the situation it is meant for: the activations of every call are made from the result
+    of the call before (here by a cast on the same stream).  Weights are permutation matrices, so the end of the chain
+    is the input with its columns permuted - exactly."""
+    M, N, K, ksp = 16, 2048, 2048, 4
+    topo = device_topo()
+    rng = np.random.default_rng(5)
+    perms = [rng.permutation(N) for _ in range(6)]
+    Ws = []
+    for pm in perms:
+        W = np.zeros((K, N), dtype=np.float32)
+        W[np.arange(K), pm] = 1.0                       # (A W)[:, pm[k]] = A[:, k]
+        Ws.append(to_dev_bf16(inputs.f32_to_bf16_bits(W)))
+    A0 = rng.integers(-8, 9, size=(M, K)).astype(np.float32)
+    x = torch.from_numpy(A0).cuda().to(torch.bfloat16)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
+                                                                k_splits=ksp, splitk_in_memory=1, overlap_launches=1))
+    want = A0
+    for rep in range(3):
+        for W, pm in zip(Ws, perms):
+            ag.gemm_persistent(x.data_ptr(), W.data_ptr(), dC.data_ptr(), M, N, K, plan, torch.cuda.current_stream().cuda_stream)
+            x = dC.to(torch.bfloat16)                    # the next call's activations, written by the launch right before it
+            nxt = np.zeros_like(want)
+            nxt[:, pm] = want
+            want = nxt
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK
+    assert np.array_equal(x.float().cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("in_memory,overlap", [(0, 1), (1, 1), (1, 2)])
+def test_overlapping_launches_integer_exact(in_memory, overlap):
     """overlap_launches: a launch lets the next one start while it is still finishing.  Nine launches are queued
     without any synchronisation in between, over three weight matrices and three outputs; every output must be
     exact (integer-valued inputs), and every unit must have run once per launch."""
@@ -125,7 +156,7 @@ def test_overlapping_launches_integer_exact(in_memory):
     dCs = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
     for b in (topo.n_sm, 74):
         plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
-                                                            k_splits=ksp, splitk_in_memory=in_memory, overlap_launches=1))
+                                                            k_splits=ksp, splitk_in_memory=in_memory, overlap_launches=overlap))
         plan.reset_record()
         for i in range(9):
             ag.gemm_persistent(dA.data_ptr(), dBs[i % 3].data_ptr(), dCs[i % 3].data_ptr(), M, N, K, plan)
