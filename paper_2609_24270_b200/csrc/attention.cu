@@ -41,7 +41,7 @@ constexpr int AT_Q_BYTES = AT_NQ * AT_D * 2;        // 4 KB
 constexpr int AT_NP = 2 * AT_MAXG;         // rows of a probability tile: 8 hi parts, 8 lo parts (one MMA adds both)
 constexpr int AT_P_BYTES = AT_NP * AT_TILE * 2;     // 4 KB
 constexpr int AT_PSLOTS = 4;
-constexpr int AT_PBATCH = 2;               // probability tiles written per fence (half the ring: the other half feeds the MMAs meanwhile)
+constexpr int AT_PBATCH = 1;               // probability tiles written per fence (two per fence measured equal at 4 tiles per unit, 10 % slower at 8)
 constexpr int AT_CTL_BYTES = 2048;
 constexpr int AT_SMEM_BYTES = AT_STAGES * AT_STAGE_BYTES + 2 * AT_Q_BYTES + AT_PSLOTS * AT_P_BYTES + 1024 + AT_CTL_BYTES;
 constexpr uint32_t AT_SCOLS = AT_MAXT * AT_NQ;      // score columns of one unit buffer (128)
