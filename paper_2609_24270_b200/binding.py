@@ -518,10 +518,16 @@ class KVCache:
         """One new token per request at position pos[b] (device int32 [B]); k_new, v_new: [B][H_kv][128] bf16."""
         _check(lib().ag_kv_append(self.handle, k_new_ptr, v_new_ptr, pos_ptr, stream), "ag_kv_append")
 
-    def __del__(self):
+    def destroy(self):
         if getattr(self, "handle", None):
             lib().ag_kv_destroy(self.handle)
             self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 def kv_pack(k_ptr: int, v_ptr: int, B: int, H_kv: int, L: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int,
