@@ -36,14 +36,14 @@ def test_group_rows_follow_the_paper_recipe():
 
 
 @pytest.mark.parametrize("G,M,N,K,ksp,in_mem", [(6, 20, 512, 512, 1, 0), (6, 20, 512, 1024, 4, 1), (32, 20, 256, 512, 2, 0),
-                                                (5, 12, 384, 256, 2, 1)])
+                                                (5, 12, 384, 256, 2, 1), (6, 48, 512, 512, 2, 1), (4, 96, 256, 1024, 4, 0)])
 def test_grouped_rowmajor_integer_exact(G, M, N, K, ksp, in_mem):
     rows, A_all, Bs = make_problem(G, M, N, K, seed=3, integer=True)
     topo = device_topo()
-    tile_m = 16 if rows.max() <= 16 else 32
+    tile_m = 16 if rows.max() <= 16 else 32 if rows.max() <= 32 else 64 if rows.max() <= 64 else 128   # up to 128 rows per expert
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=int(rows.max()), N=G * N, K=K,
                                                                 tile_m=tile_m, tile_n=128, k_splits=ksp,
-                                                                splitk_in_memory=in_mem))
+                                                                splitk_in_memory=in_mem, decode_shaped=1))
     dA = to_dev_bf16(A_all)
     dBs = [to_dev_bf16(b) for b in Bs]
     dC = torch.full((int(rows.sum()), N), float("nan"), dtype=torch.float32, device="cuda")
