@@ -564,6 +564,11 @@ ag_status attention_decode_persistent(const void* Q, const ag_kv_cache* kv, cons
 ag_status ag_wait_probe(uint64_t limit_ns, uint64_t* waited_ns);
 
 const char* ag_strerror(ag_status s);
+/* A k_splits value for a decode-shaped plan over N weight columns and K rows on sm_budget SMs, from the measurements
+ * behind this library (few, large units stream best; without overlapping launches the longest per-SM list sets the time):
+ * 4 for N = K = 8192 on 148 SMs with overlapping launches, 8 on 74 SMs, 4 on 37.  overlapping_full_chip: nonzero when the
+ * plan uses every SM and policy.overlap_launches is set.  Host arithmetic only; always returns a valid value (>= 1). */
+int32_t ag_suggest_k_splits(int32_t N, int32_t K, int32_t sm_budget, int32_t overlapping_full_chip);
 /* Last CUDA error code seen by the calling thread inside the library (0 = none). */
 int ag_last_cuda_error(void);
 /* Number of kernels this library has launched in this process (for launch accounting). */

@@ -26,7 +26,7 @@ EXPORTED = [
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
     "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
-    "ag_plan_set_grid", "ag_plan_adopted", "ag_cluster_capacity", "ag_probe_cluster_layout", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_last_status_where", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
+    "ag_plan_set_grid", "ag_plan_adopted", "ag_cluster_capacity", "ag_probe_cluster_layout", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_last_status_where", "ag_suggest_k_splits", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
     "ag_topo_load", "ag_group_desc_create", "ag_group_desc_destroy", "ag_pack_weights_grouped",
     "gemm_persistent_grouped", "ag_strerror", "ag_last_cuda_error",
@@ -134,6 +134,8 @@ def lib() -> C.CDLL:
     L.ag_plan_set_grid.argtypes = [vp, C.c_int]
     L.ag_plan_adopted.argtypes = [vp, C.POINTER(C.c_uint32)]
     L.ag_last_status.argtypes = [vp]
+    L.ag_suggest_k_splits.argtypes = [i32, i32, i32, i32]
+    L.ag_suggest_k_splits.restype = i32
     L.ag_last_status_where.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.ag_plan_destroy.argtypes = [vp]
     L.ag_plan_destroy.restype = None
@@ -541,6 +543,10 @@ def kv_pack(k_ptr: int, v_ptr: int, B: int, H_kv: int, L: int, plan: Plan, amap:
 def attention_decode(q_ptr: int, kv: KVCache, kv_len_ptr, o_ptr: int, B: int, H_q: int, plan: Plan, stream: int = 0):
     _check(lib().attention_decode_persistent(q_ptr, kv.handle, kv_len_ptr, o_ptr, B, H_q, plan.handle, stream),
            "attention_decode_persistent")
+
+
+def suggest_k_splits(N: int, K: int, sm_budget: int, overlapping_full_chip: bool = False) -> int:
+    return int(lib().ag_suggest_k_splits(N, K, sm_budget, 1 if overlapping_full_chip else 0))
 
 
 def probe_cluster_layout(cluster_size: int, n_clusters: int) -> np.ndarray:

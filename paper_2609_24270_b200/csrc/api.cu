@@ -23,6 +23,29 @@ ag_status check_arch() {
 }
 }  // namespace ag
 
+// Host arithmetic only (no device is touched).  Candidates are the powers of two up to 32 that leave every split at
+// least four k-slabs; the score of a candidate is (how evenly its units fill the SMs) x (share of a unit's time that is
+// streaming): a unit costs about as much as 20 KB of weights on top of its own bytes, and without overlapping launches
+// the longest list of ceil(units / SMs) units sets the time.
+extern "C" int32_t ag_suggest_k_splits(int32_t N, int32_t K, int32_t sm_budget, int32_t overlapping_full_chip) {
+    if (N <= 0 || K <= 0 || sm_budget <= 0) return 1;
+    const long long tiles = (N + 127) / 128;
+    const int n_slab = (K + 63) / 64;
+    int best = 1;
+    double best_score = -1.0;
+    for (int ksp = 1; ksp <= 32; ksp *= 2) {
+        const int per = (n_slab + ksp - 1) / ksp;
+        if (ksp > 1 && (per < 4 || (long long)(ksp - 1) * per >= n_slab)) break;
+        const double units = (double)(tiles * ksp), per_sm = units / sm_budget;
+        const long long longest = (tiles * ksp + sm_budget - 1) / sm_budget;
+        const double balance = overlapping_full_chip ? (per_sm < 1.0 ? per_sm : 1.0) : per_sm / (double)longest;
+        const double unit_kb = 128.0 * per * 64.0 * 2.0 / 1024.0;
+        const double score = balance * unit_kb / (unit_kb + 20.0);
+        if (score > best_score + 1e-9) { best_score = score; best = ksp; }
+    }
+    return best;
+}
+
 extern "C" const char* ag_strerror(ag_status s) {
     switch (s) {
         case AG_OK: return "ok";

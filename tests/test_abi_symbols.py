@@ -151,3 +151,18 @@ def test_ctypes_structs_match_the_header_as_a_c_compiler_sees_it(tmp_path):
         assert int(seen[sname]) == ag.C.sizeof(py[sname]), sname
         for f in fl:
             assert int(seen[f"{sname}.{f}"]) == getattr(py[sname], f).offset, (sname, f)
+
+
+def test_suggested_k_splits_follow_the_measurements():
+    """Host arithmetic: the settings that measured best (N = K = 8192: 4 splits on the full chip with overlapping launches
+    and on 37 SMs, 8 on 74 SMs), and every suggestion is a valid one (no empty split, at least four k-slabs per split)."""
+    assert ag.suggest_k_splits(8192, 8192, 148, True) == 4
+    assert ag.suggest_k_splits(8192, 8192, 74) == 8
+    assert ag.suggest_k_splits(8192, 8192, 37) == 4
+    assert ag.suggest_k_splits(128, 64, 148) == 1            # one k-slab cannot be split
+    assert ag.suggest_k_splits(0, 0, 0) == 1
+    for N, K, b in ((4096, 2048, 148), (1024, 200, 37), (49152, 7168, 148), (384, 12288, 11)):
+        ksp = ag.suggest_k_splits(N, K, b)
+        n_slab = (K + 63) // 64
+        per = -(-n_slab // ksp)
+        assert ksp >= 1 and (ksp == 1 or (per >= 4 and (ksp - 1) * per < n_slab))
