@@ -39,18 +39,24 @@ __device__ __forceinline__ void report_timeout(const PersistParams& p, int role)
 
 // Dynamic mode: take the next index of a die's queue; the 64-bit head carries the epoch of the
 // launch that last touched it, so it resets itself.  Returns -1 when the queue is drained.
+// Once the head carries this launch's epoch a pop is one fetch-and-add (a compare-and-swap loop here made 74 SMs
+// that pop every few microseconds spend most of their time retrying); only the first pops of a launch race to
+// move the head to the new epoch.  The index may run past len by one per pop after the end: far from 2^32.
 __device__ inline int pop_queue(unsigned long long* head, unsigned int epoch, int len) {
+    unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(head);
     for (int tries = 0; tries < 100000; ++tries) {
-        unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(head);
-        if ((unsigned int)(cur >> 32) != epoch) {
-            if (len <= 0) return -1;
-            const unsigned long long nv = ((unsigned long long)epoch << 32) | 1ull;
-            if (atomicCAS(head, cur, nv) == cur) return 0;
+        if ((unsigned int)(cur >> 32) == epoch) {
+            const unsigned long long old = atomicAdd(head, 1ull);
+            if ((unsigned int)(old >> 32) == epoch) {
+                const unsigned int idx = (unsigned int)(old & 0xffffffffull);
+                return idx < (unsigned int)max(len, 0) ? (int)idx : -1;
+            }
+            cur = old + 1;      // (a head of another epoch: launches of a dynamic plan never overlap, so this is not reached)
             continue;
         }
-        const int idx = (int)(cur & 0xffffffffull);
-        if (idx >= len) return -1;
-        if (atomicCAS(head, cur, cur + 1) == cur) return idx;
+        const unsigned long long fresh = (unsigned long long)epoch << 32;
+        const unsigned long long seen = atomicCAS(head, cur, fresh);
+        cur = seen == cur ? fresh : seen;
     }
     return -1;
 }
