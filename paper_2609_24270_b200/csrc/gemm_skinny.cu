@@ -233,6 +233,19 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 u = src.next(lane);
             }
             if (!ok) break;
+            if (u >= 0 && x.g_rows) {
+                // grouped operation: an expert without rows has nothing to compute - its units are ticked off here and
+                // its weights are never read (in a mixture-of-experts layer most experts are idle in most steps)
+                const int tn_u = (u / p.k_splits) % p.tiles_n;
+                if (x.g_rows[tn_u / x.tiles_per_group] == 0) {
+                    if (lane == 0) {
+                        p.tile_owner[u] = my_sm;
+                        if (p.unit_times) p.unit_times[2 * u] = p.unit_times[2 * u + 1] = globaltimer_ns();
+                        atomicAdd(&p.tile_count[u], 1);
+                    }
+                    continue;
+                }
+            }
             if (lane == 0) {
                 const int r = it % kRing;
                 if (!mbar_wait_idle(smem_u32(&ctl->sched_empty[r]), ((it / kRing) & 1) ^ 1, abort_flag, limit)) {

@@ -107,6 +107,32 @@ def test_grouped_handles_an_expert_without_rows():
     assert np.array_equal(dC.cpu().numpy().astype(np.float64), expert_refs(rows, A_all, Bs))
 
 
+@pytest.mark.parametrize("ksp,in_mem,budget", [(1, 0, None), (4, 1, None), (4, 0, 37), (2, 1, 5)])
+def test_grouped_mostly_idle_experts(ksp, in_mem, budget):
+    """A mixture-of-experts step in which most experts have no token: their units are ticked off without touching
+    their weights (every unit still shows up once per launch in the record), the others are exact."""
+    G, N, K = 16, 256, 512
+    rows = np.zeros(G, dtype=np.int32)
+    rows[[1, 6, 7, 13]] = [5, 16, 1, 11]
+    A_all = inputs.small_int_bf16(int(rows.sum()), K, 71)
+    Bs = [inputs.small_int_bf16(K, N, 72 + g) for g in range(G)]
+    topo = device_topo()
+    plan = ag.sched_build(topo, None, topo.n_sm if budget is None else budget,
+                          ag.make_policy(kind=ag.AG_DIE_COMPACT, M=16, N=G * N, K=K, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=in_mem))
+    dA = to_dev_bf16(A_all)
+    dBs = [to_dev_bf16(b) for b in Bs]
+    dC = torch.full((int(rows.sum()), N), float("nan"), dtype=torch.float32, device="cuda")
+    desc = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, [b.data_ptr() for b in dBs], N, K, 16)
+    plan.reset_record()
+    for _ in range(3):
+        ag.gemm_persistent_grouped(desc, None, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK
+    assert np.array_equal(dC.cpu().numpy().astype(np.float64), expert_refs(rows, A_all, Bs))
+    owner, count = plan.tile_record()
+    assert (count == 3).all()
+
+
 @pytest.mark.parametrize("G,M,N,K,integer", [(6, 192, 512, 256, True), (3, 700, 768, 512, True), (8, 192, 1024, 1024, False)])
 def test_grouped_dense_block_pairs(G, M, N, K, integer):
     """Many rows per expert (the paper's M = 192 / 1024 settings, scaled down): block pairs with
