@@ -464,6 +464,10 @@ ag_status ag_pack_weights_grouped(const void* const* B_list, int G, int K, int N
  *   plan  M = max rows of an expert, N = G * N_expert, K; decode-shaped: tile_n = 128, M <= tile_m;
  *         dense: tile_m = tile_n = 256, SM set of whole TPCs (units below an expert's last row are
  *         skipped, so prefer static lists built from balanced row counts)
+ *   Decode-shaped: a unit of an expert with rows[g] == 0 is ticked off by the scheduling warp without
+ *   reading a weight byte (its tile record shows one execution, its C rows do not exist).  Static lists
+ *   are cut before the row counts are known; when most experts are idle, dynamic queues
+ *   (policy.static_assign = 0) or two k-splits balance the active units better.
  * Asynchronous on cuda_stream; split-K modes as gemm_persistent_packed.  Errors as gemm_persistent.
  */
 ag_status gemm_persistent_grouped(const ag_group_desc* d, const ag_packed_weights* W, const ag_plan* plan,
