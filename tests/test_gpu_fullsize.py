@@ -110,3 +110,75 @@ def test_two_stream_configuration_runs_both_gemms_correctly(partition):
     owner_p, _ = plan_p.tile_record()
     owner_d, _ = plan_d.tile_record()
     assert set(owner_p) <= set(taken) and not set(owner_d) & set(taken)     # each GEMM stayed on its own SMs
+
+
+@pytest.mark.parametrize("k_splits", [16, 4])
+@pytest.mark.parametrize("in_memory,overlap", [(1, 2), (0, 2), (1, 1)])
+def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap):
+    """M = 16, N = K = 8192 on all SMs with die-local packed weights, as timed: calls queued without a synchronisation
+    in between, rotating over four weight matrices, launches overlapping.  Every call writes a C of its own here, and
+    every one of them is compared with the oracle in full (a race between overlapping launches would show in some)."""
+    from tests.gpu_util import check_close as close
+    M, N, K, n_buf, n_calls = 16, 8192, 8192, 4, 12
+    topo = device_topo()
+    A = inputs.uniform_bf16(M, K, inputs.DEFAULT_SEED)
+    Bs = [inputs.uniform_bf16(K, N, inputs.DEFAULT_SEED + 1 + i) for i in range(n_buf)]
+    dA, dBs = to_dev_bf16(A), [to_dev_bf16(b) for b in Bs]
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
+                                                                k_splits=k_splits, splitk_in_memory=in_memory, overlap_launches=overlap))
+    dst_bytes = 2 * K * N * 2 + (8 << 20)
+    dsts = [torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_buf)]
+    packs = []
+    for i in range(n_buf):
+        amap = ag.affinity_probe(dsts[i].data_ptr(), dst_bytes, topo)
+        packs.append(ag.pack_weights(dBs[i].data_ptr(), K, N, plan, amap, dsts[i].data_ptr(), dst_bytes))
+    dCs = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(n_calls)]
+    torch.cuda.synchronize()
+    plan.reset_record()
+    for c in range(n_calls):
+        ag.gemm_persistent_packed(dA.data_ptr(), packs[c % n_buf], dCs[c].data_ptr(), M, N, K, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK
+    owner, count = plan.tile_record()
+    assert (count == n_calls).all()
+    want = [og.gemm_blocked(A, b) for b in Bs]
+    for c in range(n_calls):
+        close(dCs[c].cpu().numpy(), want[c % n_buf])
+    if not in_memory:                                       # the workspace mode adds in a fixed order: same weights, same bits
+        assert torch.equal(dCs[0], dCs[n_buf]) and torch.equal(dCs[1], dCs[n_buf + 1])
+
+
+@pytest.mark.parametrize("placement", ["local", "interleaved"])
+def test_attention_configuration_queued_back_to_back(placement):
+    """Batch 128, 32 query heads on 8 KV heads, 512 keys, all SMs, launches overlapping, as timed: six calls queued
+    without a synchronisation, each with queries and outputs of its own; all of them against the oracle."""
+    from oracle import attention as oa
+    B, Hq, Hkv, L, D, n_calls = 128, 32, 8, 512, 128, 6
+    topo = device_topo()
+    K = inputs.uniform_bf16(B * Hkv * L, D, inputs.DEFAULT_SEED + 41).reshape(B, Hkv, L, D)
+    V = inputs.uniform_bf16(B * Hkv * L, D, inputs.DEFAULT_SEED + 42).reshape(B, Hkv, L, D)
+    Qs = [inputs.uniform_bf16(B * Hq, D, inputs.DEFAULT_SEED + 40 + 7 * c).reshape(B, Hq, D) for c in range(n_calls)]
+    dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16).copy()).cuda()
+    dK, dV, dQs = dev(K), dev(V), [dev(q) for q in Qs]
+    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
+                                                                tile_n=128, k_splits=1, overlap_launches=1))
+    kv_bytes = 2 * B * Hkv * L * D * 2
+    dst_bytes = 2 * kv_bytes + (8 << 20)
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes,
+                    ag.KV_LOCAL if placement == "local" else ag.KV_INTERLEAVED)
+    dOs = [torch.full((B, Hq, D), float("nan"), dtype=torch.float32, device="cuda") for _ in range(n_calls)]
+    torch.cuda.synchronize()
+    plan.reset_record()
+    for c in range(n_calls):
+        ag.attention_decode(dQs[c].data_ptr(), kv, None, dOs[c].data_ptr(), B, Hq, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK, plan.last_status_where()
+    owner, count = plan.tile_record()
+    assert (count == n_calls).all()
+    for c in range(n_calls):
+        got = dOs[c].cpu().numpy().astype(np.float64)
+        want = oa.gqa_decode(Qs[c], K, V)
+        assert np.isfinite(got).all()
+        assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 5e-5 and np.abs(got - want).max() <= 2e-4
