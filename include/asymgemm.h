@@ -267,7 +267,11 @@ typedef struct {
     int32_t decode_shaped;   /* 1: a plan with tile_m = 128 and tile_n = 128 is run by the decode-shaped (weight-streaming)
                                 kernel - weights on the MMA's M side, up to 128 activation rows on its N side - instead of
                                 the dense one-block kernel.  Plans with tile_m <= 64 (and tile_n = 128) always are */
-    int32_t reserved3;
+    int32_t ring_stages;     /* decode-shaped GEMM and attention decode: stages of 32 KB that a block keeps in flight from
+                                memory (2..6, clamped to what the kernel has; even for up to 32 activation rows).  0 =
+                                default: attention decode shares 20 MiB between the plan's SMs (4 stages on the full
+                                chip, where more in flight oversubscribes the memory system; 6 on half of it), the
+                                decode-shaped GEMM uses all its stages */
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;

@@ -84,7 +84,7 @@ class Policy(C.Structure):
                 ("tile_m", C.c_int32), ("tile_n", C.c_int32), ("k_splits", C.c_int32), ("k_unit", C.c_int32),
                 ("raster_group", C.c_int32), ("preferred_die", C.c_int32), ("invert_affinity", C.c_int32),
                 ("static_assign", C.c_int32), ("seed", C.c_uint64), ("min_margin", C.c_int64),
-                ("splitk_in_memory", C.c_int32), ("sm_select", C.c_int32), ("pair_lists", C.c_int32), ("overlap_launches", C.c_int32), ("cluster_size", C.c_int32), ("die_quota", C.c_int32), ("decode_shaped", C.c_int32), ("reserved3", C.c_int32),
+                ("splitk_in_memory", C.c_int32), ("sm_select", C.c_int32), ("pair_lists", C.c_int32), ("overlap_launches", C.c_int32), ("cluster_size", C.c_int32), ("die_quota", C.c_int32), ("decode_shaped", C.c_int32), ("ring_stages", C.c_int32),
                 ("avoid_sm_mask", C.c_uint64 * 4),
                 ("a", OperandDesc), ("b", OperandDesc), ("c", OperandDesc)]
 
@@ -317,7 +317,7 @@ def affinity_from_table(dev_ptr: int, die_of_chunk: np.ndarray) -> AffinityMap:
 # ---- plan -------------------------------------------------------------------------------------
 def make_policy(kind=AG_OBLIVIOUS, M=0, N=0, K=0, tile_m=128, tile_n=256, k_splits=1, k_unit=64, raster_group=1,
                 preferred_die=-1, invert_affinity=0, static_assign=1, seed=0, min_margin=0, splitk_in_memory=0,
-                sm_select=0, pair_lists=None, overlap_launches=0, cluster_size=1, die_quota=0, decode_shaped=0, avoid=(), a=None, b=None, c=None):
+                sm_select=0, pair_lists=None, overlap_launches=0, cluster_size=1, die_quota=0, decode_shaped=0, ring_stages=0, avoid=(), a=None, b=None, c=None):
     """a/b/c: None or dict(offset, row_stride, elem_bytes[, layout, page_table]).  pair_lists=None means
     "on for plans of block pairs (tile_m == 256)"."""
     p = Policy()
@@ -332,6 +332,7 @@ def make_policy(kind=AG_OBLIVIOUS, M=0, N=0, K=0, tile_m=128, tile_n=256, k_spli
     p.cluster_size = cluster_size
     p.die_quota = die_quota
     p.decode_shaped = decode_shaped
+    p.ring_stages = ring_stages
     for s in avoid:
         p.avoid_sm_mask[s >> 6] |= 1 << (s & 63)
     keep = []

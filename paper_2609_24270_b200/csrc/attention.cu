@@ -80,6 +80,7 @@ struct AttnArgs {
     float2* stats;                // [units][AT_MAXG] (maximum, sum) (n_chunks > 1)
     float scale_log2e;            // log2(e) / sqrt(D)
     int release_next;             // 1: let the next launch on the stream start while this one is still running
+    int stages;                   // key/value stages in use (3 .. AT_STAGES): the bytes this block keeps in flight
 };
 
 __device__ __forceinline__ float ex2_approx(float v) {      // 2^v, relative error 2^-22; 2^-inf = 0
@@ -246,6 +247,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const int pw = warp - (2 + kEpiWarps);
         const uint64_t stream_policy = l2_policy_evict_first();
         uint32_t q_run = 0;          // stages issued by all copy warps together so far
+        const uint32_t n_st = (uint32_t)x.stages;
         int prev_u = -1, prev_t = 0;
         int ok = 1;
         int words_cur = 0, words_prev = 0;   // lane l: word l of the page lists of the unit just taken off the ring / the one before
@@ -254,7 +256,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             for (int t = 0; t < n_t && ok; ++t) {
                 const uint32_t q = q_run + (uint32_t)t;
                 if ((int)(q % AT_NPROD) != pw) continue;
-                const uint32_t st = q % AT_STAGES, ph = ((q / AT_STAGES) & 1) ^ 1;
+                const uint32_t st = q % n_st, ph = ((q / n_st) & 1) ^ 1;
                 const int entry = __shfl_sync(0xffffffffu, words, t * 4 + v_part * 2 + (lane & 1));
                 if (lane == 0) {
                     if (!mbar_wait(smem_u32(&ctl->kv_empty[st]), ph, abort_flag, limit)) {
@@ -326,7 +328,7 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             bool have_prev = false, ok = true;
             auto next_stage = [&]() -> uint32_t {
                 const uint32_t s = st;
-                if (++st == AT_STAGES) { st = 0; ph ^= 1; }
+                if (++st == (uint32_t)x.stages) { st = 0; ph ^= 1; }
                 return s;
             };
             for (uint32_t it = 0; ok; ++it) {
@@ -906,6 +908,7 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     x.n_chunks = kv->n_chunks; x.T_total = kv->T;
     x.o_part = kv->d_part; x.stats = kv->d_stats;
     x.scale_log2e = 1.4426950408889634f / sqrtf((float)AT_D);
+    x.stages = ring_stages_for(plan, AT_STAGES, AT_NPROD, false, true);
     PersistParams gp = make_persist_params(plan, h[H_M], h[H_N], h[H_K]);
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);

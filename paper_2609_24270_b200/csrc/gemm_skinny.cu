@@ -95,6 +95,8 @@ struct SkinnyArgs {
     int n_group;                  // columns of one expert
     int release_next;             // 1: let the next launch on the stream start while this one is still running
     int a_after_prior;            // 1: the activations may be the product of the launch before: read them only after it has completed
+    int stages;                   // weight stages in use (at most sk_stages(NM), a multiple of the MMA-issuing threads)
+    int producers;                // copying warps in use (at most SK_WPROD)
     // closed form of the page table (PACKED): see table_entry in the kernel
     const int32_t* unit_base;     // device [tiles_n * k_splits] or null (then the tables above are read)
     const uint32_t* page_bits;    // device: one hash bit per 2 MiB page of the packed buffer
@@ -148,6 +150,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     constexpr int kNMMA = sk_nmma(NM);                   // MMA-issuing threads at work
     constexpr bool kUnified = sk_unified(NM);            // activations inside the weight stages
     constexpr uint32_t kStageBytes = sk_stage_bytes(NM);
+    const uint32_t ring_n = (uint32_t)x.stages;          // stages of the ring in use
     const uint32_t a_base = base + kStages * kStageBytes;
     SkinnyCtl* ctl = reinterpret_cast<SkinnyCtl*>(smem + kStages * kStageBytes + (kUnified ? 0 : SK_ASTAGES * kAStage));
     constexpr uint32_t kAccCols = NM;                    // columns of one accumulator
@@ -297,6 +300,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         // For packed weights all 32 lanes fetch the page-table entries of the next eight k-slabs with one load
         // each, so the issuing lane never waits on a table lookup.
         const int pw = warp - (2 + kEpiWarps);
+        // Copying warps: their number divides the ring (or the one MMA-issuing thread hands the stages back in order), so
+        // that a warp waiting for a stage to come free is never more than one use of that stage ahead of its barrier.
+        const int n_prod = x.producers;
         const uint64_t stream_policy = l2_policy_evict_first();  // weights are read once: do not keep them in L2
         uint32_t q0 = 0;      // stage count (over the whole run of this block) before the current unit
         bool a_ready = false; // (activations inside the stages) everything launched before is known to be complete
@@ -322,9 +328,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
             const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
             const int n_st = (s1 - s0 + SK_SLABS - 1) / SK_SLABS;    // stages of this unit: slabs s0 + 2i, s0 + 2i + 1
-            // this warp's stages of the unit: i0, i0 + SK_WPROD, ...
-            const int i0 = (pw + SK_WPROD - (int)(q0 % SK_WPROD)) % SK_WPROD;
-            uint32_t st = (q0 + i0) % kStages, ph = (((q0 + i0) / kStages) & 1) ^ 1;   // stage, parity of "stage is free"
+            // this warp's stages of the unit: i0, i0 + n_prod, ... (a warp beyond the copying ones takes the unit off the ring and copies nothing)
+            const int i0 = pw < n_prod ? (pw + n_prod - (int)(q0 % (uint32_t)n_prod)) % n_prod : n_st;
+            uint32_t st = (q0 + i0) % ring_n, ph = (((q0 + i0) / ring_n) & 1) ^ 1;   // stage, parity of "stage is free"
             const CUtensorMap* mw = x.g_tm_w ? &x.g_tm_w[grp] : &tm_w;
             // packed weights: lane l < 2 (groups of four pages) or l < 8 (single pages) looks up the chunk of the
             // l-th 16 KB / 4 KB piece of a stage, one stage ahead of the copies
@@ -357,9 +363,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 return (lane < 4 * SK_SLABS && s + (lane >> 2) < s1) ? x.page_table[(size_t)tn * x.pages_per_tile + (size_t)s * 4 + lane] : 0;
             };
             int next_entry = table_entry(i0);
-            for (int i = i0; i < n_st && ok; i += SK_WPROD) {
+            for (int i = i0; i < n_st && ok; i += n_prod) {
                 const int entry = next_entry;
-                next_entry = table_entry(i + SK_WPROD);
+                next_entry = table_entry(i + n_prod);
                 const int s = s0 + i * SK_SLABS;
                 const int ns = min(SK_SLABS, s1 - s);
                 const uint32_t bar = smem_u32(&ctl->full[st]);
@@ -407,9 +413,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         tma_load_2d_hint(sw + SK_W_BYTES / 2, mw, bar, tl * SK_BN + 64, s * SK_BK, stream_policy);
                     }
                 }
-                // this warp's next stage is SK_WPROD stages on
-                st += SK_WPROD;
-                if (st >= (uint32_t)kStages) { st -= kStages; ph ^= 1; }
+                // this warp's next stage is n_prod stages on
+                st += (uint32_t)n_prod;
+                if (st >= ring_n) { st -= ring_n; ph ^= 1; }
             }
             q0 += (uint32_t)n_st;
         }
@@ -466,7 +472,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 tc_fence_after();
                 const int a = kNMMA == 2 ? (t - (int)(q0 & 1u)) & 1 : 0;   // parity, inside the unit, of the stages in this thread's buffers
                 const uint32_t d_tmem = tmem_base + (acc * kNMMA + a) * kAccCols;
-                uint32_t st = (q0 + a) % kStages, ph = ((q0 + a) / kStages) & 1;   // this thread's first stage of the unit
+                uint32_t st = (q0 + a) % ring_n, ph = ((q0 + a) / ring_n) & 1;   // this thread's first stage of the unit
                 bool first = true;
                 if constexpr (kUnified) {
                     // activations behind the weights of the same stage: one barrier per stage, no activation buffers
@@ -491,7 +497,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         }
                         first = false;
                         tc_commit(empty0 + st * 8);
-                        if (++st == (uint32_t)kStages) { st = 0; ph ^= 1; }
+                        if (++st == ring_n) { st = 0; ph ^= 1; }
                     }
                 } else
                 for (int g = 0; g < n_grp && ok; ++g) {
@@ -532,7 +538,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         first = false;
                         tc_commit(empty0 + st * 8);
                         st += kNMMA;
-                        if (st >= (uint32_t)kStages) { st -= kStages; ph ^= 1; }
+                        if (st >= ring_n) { st -= ring_n; ph ^= 1; }
                         da += kNMMA * SK_SLABS * (kASlab >> 4);
                     }
                     if (ok) tc_commit(smem_u32(&ctl->a_empty[aj]));    // this thread's last read of the buffer has been issued
@@ -809,6 +815,8 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0 && plan->lay.b == plan->lay.n_sm;
     x.release_next = overlap ? 1 : 0;
     x.a_after_prior = (overlap && plan->policy.overlap_launches != 2) ? 1 : 0;
+    x.stages = ring_stages_for(plan, sk_stages(NM), std::min(sk_stages(NM), 2), sk_nmma(NM) == 2, false);
+    x.producers = x.stages % 3 == 0 ? 3 : x.stages % 2 == 0 ? 2 : sk_nmma(NM) == 1 ? std::min(3, x.stages) : 1;
     if (zeroing) {  // in-memory reduction mode: the adds need a zeroed C (N % 8 == 0 and 16-byte alignment: whole float4s)
         const size_t c_elems = grp ? (size_t)grp->total_rows * (size_t)grp->N : (size_t)M * (size_t)N;
         const size_t n_vec = c_elems / 4;

@@ -263,6 +263,20 @@ inline bool is_decode_shaped(const ag_plan* plan) {
     const int32_t* h = plan->header;
     return h[H_TILE_N] == 128 && (h[H_TILE_M] <= 64 || (h[H_TILE_M] == 128 && plan->policy.decode_shaped));
 }
+// Stages (of 32 KB from memory each) of the streaming kernels' copy ring that a launch uses.  A bare copy ring on all 148
+// SMs reads 7.38 TB/s with 3 or 4 stages per SM, 7.22 with 5, 7.16 with 6, and with 6 only 6.65 TB/s once the consumer holds
+// a stage for 0.3 us as the MMA path does, while 4 stages lose nothing to that hold: beyond about 20 MB in flight on the
+// chip the memory system is oversubscribed.  On half or a quarter of the SMs a block's rate grows with the bytes it keeps
+// in flight.  policy.ring_stages > 0 overrides; otherwise `by_sm_count` selects 20 MiB shared by the plan's SMs (attention
+// decode, whose launches last long enough to reach the steady state: 4 stages on the full chip read 3-7 % more than 6), or
+// all stages (the decode-shaped GEMM, whose 20-microsecond launches gain more from a deep ring while they fill).
+inline int ring_stages_for(const ag_plan* plan, int max_stages, int min_stages, bool even, bool by_sm_count) {
+    int s = plan->policy.ring_stages;
+    if (s <= 0) s = by_sm_count ? 640 / std::max(1, plan->lay.b) : max_stages;
+    s = std::max(min_stages, std::min(max_stages, s));
+    if (even && (s & 1)) s = s + 1 <= max_stages ? s + 1 : s - 1;
+    return s;
+}
 ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_packed_weights* W, void* Cout, int M,
                                int N, int K, const ag_plan* plan, float* partial, cudaStream_t stream,
                                const ag_group_desc* grp = nullptr);

@@ -10,6 +10,7 @@
     python -m paper_2609_24270_b200.experiments --config latency           # latency histograms from one SM per die
     python -m paper_2609_24270_b200.experiments --config cluster_sets      # cluster eligibility of equal-size SM sets
     python -m paper_2609_24270_b200.experiments --config attention         # decode attention, KV pages local / remote / interleaved
+    python -m paper_2609_24270_b200.experiments --config attention_sweep   # the paper's decode sweep: MHA / GQA, batch 1-64, keys from 512
     python -m paper_2609_24270_b200.experiments --config 5_attention       # prefill GEMM and decode attention on disjoint SM partitions
 
 Every line printed is one JSON record.  Timing: CUDA events on the launching stream, warm-up
@@ -614,6 +615,20 @@ def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024), (16, 32, 
         torch.cuda.empty_cache()
 
 
+def attention_sweep(fh, topo):
+    """The decode sweep of the paper's attention study (workload appendix): one query token per request, 32 query
+    heads of 128 dimensions on 32 (MHA) or 8 (GQA) KV heads, batch 1 to 64, keys from 512 doubling, full chip;
+    working sets up to 8.6 GB here."""
+    shapes = []
+    for Hkv in (32, 8):
+        for B in (1, 8, 64):
+            L = 512
+            while 4 * B * L * Hkv * 128 <= 8.6e9 and L <= (1 << 17):
+                shapes.append((B, 32, Hkv, L))
+                L *= 4
+    attention(fh, topo, shapes=tuple(shapes), budgets=(topo.n_sm,))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -626,7 +641,8 @@ def main():
               lat_near_cycles=topo.lat_near_cycles, lat_far_cycles=topo.lat_far_cycles), fh)
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
      "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention,
-     "raster_traffic": lambda f, t: raster(f, t, traffic_only=True), "5_attention": config5_attention}[args.config](fh, topo)
+     "raster_traffic": lambda f, t: raster(f, t, traffic_only=True), "5_attention": config5_attention,
+     "attention_sweep": attention_sweep}[args.config](fh, topo)
 
 
 if __name__ == "__main__":

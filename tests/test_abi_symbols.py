@@ -132,7 +132,7 @@ def test_ctypes_structs_match_the_header_as_a_c_compiler_sees_it(tmp_path):
                         "lat_near_cycles", "l2_near_cycles", "n_unplaced", "device", "sm_clock_khz", "flags"],
         "ag_operand_desc": ["present", "layout", "offset", "row_stride", "elem_bytes", "page_table", "n_pages"],
         "ag_policy": ["kind", "M", "tile_m", "k_splits", "k_unit", "raster_group", "preferred_die", "invert_affinity",
-                      "static_assign", "seed", "min_margin", "splitk_in_memory", "sm_select", "pair_lists", "overlap_launches", "cluster_size", "die_quota", "decode_shaped",
+                      "static_assign", "seed", "min_margin", "splitk_in_memory", "sm_select", "pair_lists", "overlap_launches", "cluster_size", "die_quota", "decode_shaped", "ring_stages",
                       "avoid_sm_mask", "a", "b", "c"],
     }
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "asymgemm.h"', 'int main(void) {']
