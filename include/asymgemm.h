@@ -198,6 +198,22 @@ ag_status ag_affinity_fit_hash(const ag_affinity_map* amap, uint32_t* mask, size
  */
 ag_status ag_probe_die_bandwidth(const ag_affinity_map* amap, const ag_topo_map* map, int reader_die,
                                  int chunk_die, double* bytes_per_s);
+/*
+ * ag_probe_ring_bandwidth - what a ring of shared-memory stages filled by bulk copies reads from memory: the copy side of
+ * the streaming kernels (decode-shaped GEMM, attention decode) without their arithmetic, to choose policy.ring_stages
+ * for a chip.  n_blocks blocks (one per SM: each takes 200 KB of shared memory) stream equal contiguous shares of buf;
+ * each keeps `stages` buffers of `stage_bytes` in flight, refilled by `producers` warps in turn; one thread takes the
+ * stages off in order, spends hold_ns on each (one after the other, as a thread that issues a stage's MMAs does; 0 = none)
+ * and hands it back.
+ *   buf    device, 16-byte aligned, read only; bytes >= n_blocks * stage_bytes (use far more than the L2 size)
+ *   stages 1..8, stage_bytes a multiple of 4096 in 4096..65536, stages * stage_bytes <= 192 KiB
+ *   producers 1..3 and <= stages; hold_ns 0..100000
+ *   bytes_per_s  host, out: best of three runs (first block's start to last block's end).
+ * Synchronises the device.  Errors: AG_ERR_ARG, AG_ERR_UNSUPPORTED_ARCH, AG_ERR_CUDA, AG_ERR_TIMEOUT (a bounded wait
+ * ran out; the device stays usable).
+ */
+ag_status ag_probe_ring_bandwidth(const void* buf, size_t bytes, int n_blocks, int stages, int stage_bytes,
+                                  int producers, int hold_ns, double* bytes_per_s);
 void ag_affinity_destroy(ag_affinity_map* amap);
 
 /* ---- plan (Section 7.1.2) ------------------------------------------------------------ */

@@ -24,7 +24,7 @@ EXPORTED = [
     "topo_discover", "ag_topo_discover_phases", "ag_topo_from_observations", "ag_topo_place_by_gain",
     "ag_probe_l2_bandwidth", "ag_probe_latency_samples",
     "affinity_probe", "ag_affinity_probe_with_map", "ag_affinity_from_table", "ag_affinity_export",
-    "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_affinity_destroy",
+    "ag_affinity_cycles", "ag_affinity_check_complement", "ag_affinity_fit_hash", "ag_probe_die_bandwidth", "ag_probe_ring_bandwidth", "ag_affinity_destroy",
     "sched_build", "ag_plan_export", "ag_plan_margins", "ag_plan_tile_record", "ag_plan_reset_record",
     "ag_plan_set_grid", "ag_plan_adopted", "ag_cluster_capacity", "ag_probe_cluster_layout", "ag_plan_trace", "ag_plan_unit_times", "ag_last_status", "ag_last_status_where", "ag_suggest_k_splits", "ag_plan_destroy", "gemm_persistent", "ag_pack_weights", "ag_pack_weights_ex", "ag_packed_info", "ag_packed_closed_form", "ag_packed_page_table",
     "ag_packed_destroy", "gemm_persistent_packed", "gemm_persistent_noalloc", "ag_wait_probe", "ag_topo_save",
@@ -122,6 +122,7 @@ def lib() -> C.CDLL:
     L.ag_affinity_check_complement.argtypes = [vp, C.POINTER(TopoMap), C.POINTER(sz)]
     L.ag_affinity_fit_hash.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(sz)]
     L.ag_probe_die_bandwidth.argtypes = [vp, C.POINTER(TopoMap), C.c_int, C.c_int, C.POINTER(C.c_double)]
+    L.ag_probe_ring_bandwidth.argtypes = [vp, sz, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_double)]
     L.ag_affinity_destroy.argtypes = [vp]
     L.ag_affinity_destroy.restype = None
     L.sched_build.argtypes = [C.POINTER(TopoMap), vp, C.c_int, C.POINTER(Policy), C.POINTER(vp)]
@@ -295,6 +296,15 @@ class AffinityMap:
             self.destroy()
         except Exception:
             pass
+
+
+def probe_ring_bandwidth(dev_ptr: int, nbytes: int, n_blocks: int, stages: int, stage_bytes: int = 32768,
+                         producers: int = 3, hold_ns: int = 0) -> float:
+    """Bytes/s that n_blocks blocks read through rings of `stages` bulk-copy stages of `stage_bytes`."""
+    out = C.c_double()
+    _check(lib().ag_probe_ring_bandwidth(dev_ptr, nbytes, n_blocks, stages, stage_bytes, producers, hold_ns, C.byref(out)),
+           "ag_probe_ring_bandwidth")
+    return out.value
 
 
 def affinity_probe(dev_ptr: int, nbytes: int, topo: TopoMap | None = None) -> AffinityMap:

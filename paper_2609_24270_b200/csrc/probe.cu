@@ -19,6 +19,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <numeric>
 #include <vector>
@@ -1076,6 +1077,119 @@ extern "C" ag_status ag_probe_die_bandwidth(const ag_affinity_map* amap, const a
     if (e != cudaSuccess) return cuda_fail(e);
     *bytes_per_s = best;
     return best > 0 ? AG_OK : AG_ERR_UNMANNED_SM;
+}
+
+// ---- copy-ring bandwidth (the streaming kernels' ring without their arithmetic) --------------------------------
+// Block b streams its own contiguous share of the buffer through a ring of `stages` shared-memory buffers of
+// `stage_bytes`: warp w < producers refills the stages w, w + producers, ... with one bulk copy each, one thread of
+// another warp takes them off in order, spends `hold_ns` on each (one after the other, like a thread that issues a
+// stage's MMAs) and hands it back.  Every wait is bounded; a wait that runs out sets *err.
+constexpr int kRingMaxStages = 8;
+__global__ void __launch_bounds__(160, 1) k_ring_bandwidth(const uint8_t* __restrict__ src, long long n_stages, int stages, int stage_bytes,
+                                                            int producers, int hold_ns, unsigned long long* t_out, int* err,
+                                                            unsigned int* sink) {
+    extern __shared__ __align__(1024) uint8_t ring_smem[];
+    __shared__ uint64_t full[kRingMaxStages], empty[kRingMaxStages];
+    const uint32_t raw = smem_u32(ring_smem);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < stages; ++i) {
+            mbar_init(smem_u32(&full[i]), 1);
+            mbar_init(smem_u32(&empty[i]), 1);
+        }
+        mbar_fence_init();
+    }
+    __syncthreads();
+    volatile int* abort_flag = err;
+    const uint64_t limit = 2000000000ull;
+    const uint64_t stream_policy = l2_policy_evict_first();
+    const uint8_t* mine = src + (size_t)blockIdx.x * (size_t)n_stages * (size_t)stage_bytes;
+    const unsigned long long t0 = globaltimer_ns();
+    if (warp < producers) {
+        if (lane == 0) {
+            for (long long c = warp; c < n_stages; c += producers) {
+                const int st = (int)(c % stages);
+                if (!mbar_wait(smem_u32(&empty[st]), (uint32_t)(((c / stages) & 1) ^ 1), abort_flag, limit)) break;
+                mbar_expect_tx(smem_u32(&full[st]), (uint32_t)stage_bytes);
+                bulk_load_hint(base + st * stage_bytes, mine + (size_t)c * stage_bytes, (uint32_t)stage_bytes, smem_u32(&full[st]), stream_policy);
+            }
+        }
+    } else if (warp == producers) {
+        if (lane == 0) {
+            unsigned int acc = 0;
+            for (long long c = 0; c < n_stages; ++c) {
+                const int st = (int)(c % stages);
+                if (!mbar_wait(smem_u32(&full[st]), (uint32_t)((c / stages) & 1), abort_flag, limit)) break;
+                acc += *reinterpret_cast<volatile unsigned int*>(ring_smem + (base - raw) + st * stage_bytes + 64);
+                if (hold_ns > 0) {
+                    const unsigned long long h0 = globaltimer_ns();
+                    while (globaltimer_ns() - h0 < (unsigned long long)hold_ns) {}
+                }
+                mbar_arrive(smem_u32(&empty[st]));
+            }
+            if (acc == 0x12345u) sink[0] = acc;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        t_out[2 * blockIdx.x] = t0;
+        t_out[2 * blockIdx.x + 1] = globaltimer_ns();
+    }
+}
+
+extern "C" ag_status ag_probe_ring_bandwidth(const void* buf, size_t bytes, int n_blocks, int stages, int stage_bytes, int producers,
+                                             int hold_ns, double* bytes_per_s) {
+    // producers <= stages: the one consuming thread hands the stages back in order, so a copying warp is never more than
+    // one use of a stage ahead of that stage's barrier
+    if (!buf || !bytes_per_s || ((uintptr_t)buf & 15u) || n_blocks < 1 || n_blocks > AG_MAX_SM || stages < 1 || stages > kRingMaxStages ||
+        stage_bytes < 4096 || stage_bytes > 65536 || (stage_bytes & 4095) || stages * stage_bytes > 192 * 1024 || producers < 1 ||
+        producers > 3 || producers > stages || hold_ns < 0 || hold_ns > 100000)
+        return AG_ERR_ARG;
+    const long long n_stages = (long long)(bytes / (size_t)n_blocks / (size_t)stage_bytes);
+    if (n_stages < 1) return AG_ERR_ARG;
+    ag_status st = check_arch();
+    if (st != AG_OK) return st;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] { attr_err = cudaFuncSetAttribute(k_ring_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    unsigned long long* d_t = nullptr;
+    int* d_err = nullptr;
+    unsigned int* d_sink = nullptr;
+    cudaError_t e = cudaSuccess;
+    double best = 0;
+    int h_err = 0;
+    do {
+        if ((e = cudaMalloc(&d_t, sizeof(unsigned long long) * 2 * n_blocks)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_err, sizeof(int))) != cudaSuccess) break;
+        if ((e = cudaMalloc(&d_sink, 64)) != cudaSuccess) break;
+        if ((e = cudaMemset(d_err, 0, sizeof(int))) != cudaSuccess) break;
+        std::vector<unsigned long long> h(2 * (size_t)n_blocks);
+        for (int t = 0; t < 3 && e == cudaSuccess && !h_err; ++t) {
+            // 200 KB of shared memory per block: one block per SM
+            k_ring_bandwidth<<<n_blocks, (producers + 1) * 32, 200 * 1024>>>((const uint8_t*)buf, n_stages, stages, stage_bytes, producers, hold_ns,
+                                                                            d_t, d_err, d_sink);
+            count_launch();
+            if ((e = cudaGetLastError()) != cudaSuccess) break;
+            if ((e = cudaDeviceSynchronize()) != cudaSuccess) break;
+            if ((e = cudaMemcpy(h.data(), d_t, sizeof(unsigned long long) * h.size(), cudaMemcpyDeviceToHost)) != cudaSuccess) break;
+            if ((e = cudaMemcpy(&h_err, d_err, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) break;
+            unsigned long long t0 = ~0ull, t1 = 0;
+            for (int b = 0; b < n_blocks; ++b) {
+                t0 = std::min(t0, h[2 * b]);
+                t1 = std::max(t1, h[2 * b + 1]);
+            }
+            if (t1 > t0) best = std::max(best, (double)n_stages * stage_bytes * n_blocks / ((double)(t1 - t0) * 1e-9));
+        }
+    } while (0);
+    cudaFree(d_t);
+    cudaFree(d_err);
+    cudaFree(d_sink);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (h_err) return AG_ERR_TIMEOUT;
+    *bytes_per_s = best;
+    return AG_OK;
 }
 
 extern "C" ag_status ag_affinity_export(const ag_affinity_map* amap, uint8_t* die_of_chunk, size_t cap,

@@ -629,6 +629,23 @@ def attention_sweep(fh, topo):
     attention(fh, topo, shapes=tuple(shapes), budgets=(topo.n_sm,))
 
 
+def copy_ring(fh, topo):
+    """What sets policy.ring_stages: the copy side of the streaming kernels alone (rings of 32 KB stages filled by bulk
+    copies) on 1, 37, 74 and all SMs, over the ring depth, the stage size and the time a stage is held."""
+    nbytes = 4 << 30
+    buf = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    for n_blocks in (1, 37, 74, topo.n_sm):
+        share = nbytes if n_blocks > 1 else 256 << 20
+        for stage_bytes, depths in ((32768, (1, 2, 3, 4, 5, 6)), (16384, (2, 4, 8)), (65536, (1, 2, 3))):
+            for stages in depths:
+                for hold_ns in (0, 400):
+                    producers = min(stages, 3)
+                    gbs = ag.probe_ring_bandwidth(buf.data_ptr(), share, n_blocks, stages, stage_bytes, producers, hold_ns) / 1e9
+                    emit(dict(config="copy_ring", n_blocks=n_blocks, stage_bytes=stage_bytes, stages=stages, producers=producers,
+                              hold_ns=hold_ns, in_flight_mb=n_blocks * stages * stage_bytes / 1e6, gbs=gbs,
+                              gbs_per_sm=gbs / n_blocks), fh)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", required=True)
@@ -642,7 +659,7 @@ def main():
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
      "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention,
      "raster_traffic": lambda f, t: raster(f, t, traffic_only=True), "5_attention": config5_attention,
-     "attention_sweep": attention_sweep}[args.config](fh, topo)
+     "attention_sweep": attention_sweep, "copy_ring": copy_ring}[args.config](fh, topo)
 
 
 if __name__ == "__main__":

@@ -1,6 +1,7 @@
 """CPU-only: the C-ABI library loads and exports every symbol the header declares; host-side
 logic that needs no device (union-find over cluster observations, die split from latency
 vectors, the bandwidth-gain decision rule)."""
+import ctypes as C
 import os
 import re
 
@@ -41,6 +42,11 @@ def test_null_arguments_are_rejected_without_a_device():
     assert L.sched_build(None, None, 1, None, None) == ag.AG_ERR_ARG
     assert L.gemm_persistent(None, None, None, 1, 1, 1, None, None) == ag.AG_ERR_ARG
     assert L.affinity_probe(None, 4096, None) != ag.AG_OK
+    bw = C.c_double()
+    for bad in [(None, 1 << 20, 4, 4, 32768, 2, 0), (4096, 1 << 20, 4, 9, 16384, 2, 0), (4096, 1 << 20, 4, 4, 5000, 2, 0),
+                (4096, 1 << 20, 4, 2, 32768, 3, 0), (4096, 1 << 20, 4, 8, 32768, 2, 0), (4096, 1 << 20, 0, 4, 32768, 2, 0),
+                (4104, 1 << 20, 4, 4, 32768, 2, 0), (4096, 1 << 16, 4, 4, 32768, 2, 0), (4096, 1 << 20, 4, 4, 32768, 2, -1)]:
+        assert L.ag_probe_ring_bandwidth(*bad, C.byref(bw)) == ag.AG_ERR_ARG, bad
     assert ag.strerror(ag.AG_ERR_TIMEOUT) != ag.strerror(ag.AG_OK)
 
 

@@ -99,6 +99,20 @@ def test_local_bandwidth_beats_remote(topo):
         assert 0.5e12 < bw[(r, r)] < 6e12, bw
 
 
+def test_ring_bandwidth_grows_with_the_bytes_in_flight(topo):
+    """The copy side of the streaming kernels alone: one SM reads faster with more 32 KB stages in flight, and the
+    full chip with four stages per SM streams a buffer far larger than L2 at a rate in the range of the memory's."""
+    nbytes = 2 << 30
+    buf = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    one = {s: ag.probe_ring_bandwidth(buf.data_ptr(), 256 << 20, 1, s, 32768, min(s, 3)) for s in (1, 2, 6)}
+    assert one[1] < one[2] < one[6], one
+    assert 5e9 < one[1] and one[6] < 400e9, one
+    full = ag.probe_ring_bandwidth(buf.data_ptr(), nbytes, topo.n_sm, 4, 32768, 2)
+    assert 3e12 < full < 9e12, full
+    held = ag.probe_ring_bandwidth(buf.data_ptr(), 256 << 20, 1, 2, 32768, 2, hold_ns=2000)
+    assert held < one[2], (held, one)                          # a stage that is held longer is refilled later
+
+
 def test_cluster_layout_respects_the_map():
     """Where the hardware puts clusters of four and eight blocks: always inside one GPC class of the discovered map and
     never on an SM that cluster probing marked as random (Section 5.1.1); the number it co-schedules is the capacity
