@@ -313,8 +313,9 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
             // ------------------------------------------------ MMA issuer: scores of unit i, then the outputs of unit i - 1
+            // (the warp runs the loop converged and one elected lane issues the MMAs and commits: see elect_one)
             constexpr uint32_t idesc = make_idesc_bf16(128, AT_NQ, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, AT_NP, 0, 0);
             static_assert(AT_NP == 16 && AT_MAXG == 8, "rows q and 8 + q of a probability tile are the two parts of query row q");
@@ -333,49 +334,56 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             };
             for (uint32_t it = 0; ok; ++it) {
                 const int r = it % kRing;
-                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
-                    report_timeout(p, 3);
+                if (!mbar_wait_all(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 3);
                     break;
                 }
                 const int u = ctl->ring[r];
-                mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                __syncwarp();       // every lane has read the entry before it is handed back
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
                 const int n_t = u >= 0 ? unit_tiles(x, u) : 0;     // 0: the end of the list, or a unit without keys
                 if (n_t > 0) {
                     // ---- S^T = K Q^T for every key tile of the unit
                     const uint32_t j = nq & 1;
-                    if (!mbar_wait(smem_u32(&ctl->s_empty[j]), ((nq >> 1) & 1) ^ 1, abort_flag, limit) ||
-                        !mbar_wait(smem_u32(&ctl->q_full[j]), (nq >> 1) & 1, abort_flag, limit)) {
-                        report_timeout(p, 4);
+                    if (!mbar_wait_all(smem_u32(&ctl->s_empty[j]), ((nq >> 1) & 1) ^ 1, abort_flag, limit) ||
+                        !mbar_wait_all(smem_u32(&ctl->q_full[j]), (nq >> 1) & 1, abort_flag, limit)) {
+                        if (lane == 0) report_timeout(p, 4);
                         break;
                     }
                     tc_fence_after();
                     const uint64_t dq = dsw_t | (uint64_t)((q_base + j * AT_Q_BYTES) >> 4);
                     for (int t = 0; t < n_t; ++t) {
                         const uint32_t phw = ph, s = next_stage();
-                        if (!mbar_wait(full0 + s * 8, phw, abort_flag, limit)) {
-                            report_timeout(p, 5);
+                        if (!mbar_wait_all(full0 + s * 8, phw, abort_flag, limit)) {
+                            if (lane == 0) report_timeout(p, 5);
                             ok = false;
                             break;
                         }
                         tc_fence_after();
                         const uint64_t dk = dpage_t | (uint64_t)((base + s * AT_STAGE_BYTES) >> 4);
                         const uint32_t d_s = tmem_base + j * AT_BUFCOLS + t * AT_NQ;
+                        if (elect_one()) {
 #pragma unroll
-                        for (int g = 0; g < AT_D / 16; ++g)   // 16 d per step: page g of the tile; Q: atom g / 4, 32 B per step
-                            tc_mma_f16(d_s, dk + g * (4096u >> 4), dq + (g >> 2) * (2048u >> 4) + (g & 3) * 2, idesc, g ? 1u : 0u);
-                        tc_commit(empty0 + s * 8);
+                            for (int g = 0; g < AT_D / 16; ++g)   // 16 d per step: page g of the tile; Q: atom g / 4, 32 B per step
+                                tc_mma_f16(d_s, dk + g * (4096u >> 4), dq + (g >> 2) * (2048u >> 4) + (g & 3) * 2, idesc, g ? 1u : 0u);
+                            tc_commit(empty0 + s * 8);
+                        }
+                        __syncwarp();
                     }
                     if (!ok) break;
-                    tc_commit(smem_u32(&ctl->s_full[j]));
-                    tc_commit(smem_u32(&ctl->q_empty[j]));
+                    if (elect_one()) {
+                        tc_commit(smem_u32(&ctl->s_full[j]));
+                        tc_commit(smem_u32(&ctl->q_empty[j]));
+                    }
+                    __syncwarp();
                     ++nq;
                 }
                 if (have_prev) {
                     // ---- O^T += V^T P^T for every key tile of the previous unit (probabilities as hi + lo bf16 parts)
                     const uint32_t np = nq - (n_t > 0 ? 2 : 1);         // ordinal of the previous unit
                     const uint32_t j = np & 1;
-                    if (!mbar_wait(smem_u32(&ctl->o_empty[j]), ((np >> 1) & 1) ^ 1, abort_flag, limit)) {
-                        report_timeout(p, 4);
+                    if (!mbar_wait_all(smem_u32(&ctl->o_empty[j]), ((np >> 1) & 1) ^ 1, abort_flag, limit)) {
+                        if (lane == 0) report_timeout(p, 4);
                         break;
                     }
                     tc_fence_after();
@@ -383,33 +391,41 @@ k_attn_decode(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     for (int t = 0; t < prev_t; ++t, ++pt) {
                         const uint32_t phw = ph, s = next_stage();
                         const uint32_t ps = pt % AT_PSLOTS;
-                        if (!mbar_wait(smem_u32(&ctl->p_full[ps]), (pt / AT_PSLOTS) & 1, abort_flag, limit) ||
-                            !mbar_wait(full0 + s * 8, phw, abort_flag, limit)) {
-                            report_timeout(p, 5);
+                        if (!mbar_wait_all(smem_u32(&ctl->p_full[ps]), (pt / AT_PSLOTS) & 1, abort_flag, limit) ||
+                            !mbar_wait_all(full0 + s * 8, phw, abort_flag, limit)) {
+                            if (lane == 0) report_timeout(p, 5);
                             ok = false;
                             break;
                         }
                         tc_fence_after();
                         const uint64_t dv = dpage_t | (uint64_t)((base + s * AT_STAGE_BYTES) >> 4);
                         const uint64_t dp = dsw_t | (uint64_t)((p_base + ps * AT_P_BYTES) >> 4);
+                        if (elect_one()) {
 #pragma unroll
-                        for (int k8 = 0; k8 < AT_TILE / 16; ++k8)     // 16 keys per step: page k8 of the tile; P: atom k8 / 4
-                            tc_mma_f16(d_o, dv + k8 * (4096u >> 4), dp + (k8 >> 2) * (2048u >> 4) + (k8 & 3) * 2, idesc_pv,
-                                       (t | k8) ? 1u : 0u);
-                        tc_commit(empty0 + s * 8);
-                        tc_commit(smem_u32(&ctl->p_empty[ps]));
+                            for (int k8 = 0; k8 < AT_TILE / 16; ++k8)     // 16 keys per step: page k8 of the tile; P: atom k8 / 4
+                                tc_mma_f16(d_o, dv + k8 * (4096u >> 4), dp + (k8 >> 2) * (2048u >> 4) + (k8 & 3) * 2, idesc_pv,
+                                           (t | k8) ? 1u : 0u);
+                            tc_commit(empty0 + s * 8);
+                            tc_commit(smem_u32(&ctl->p_empty[ps]));
+                        }
+                        __syncwarp();
                     }
                     if (!ok) break;
-                    tc_commit(smem_u32(&ctl->o_full[j]));
+                    if (elect_one()) tc_commit(smem_u32(&ctl->o_full[j]));
+                    __syncwarp();
                 }
                 have_prev = n_t > 0;
                 prev_t = n_t;
                 if (u < 0) break;
             }
+            __syncwarp();
             if (*abort_flag) {
-                tc_commit(smem_u32(&ctl->mma_drain));
-                int dummy = 0;
-                mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                if (elect_one()) {
+                    tc_commit(smem_u32(&ctl->mma_drain));
+                    int dummy = 0;
+                    mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                }
+                __syncwarp();
             }
         }
     } else {

@@ -173,8 +173,8 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer (one lane)
-        if (lane == 0) {
+        // ------------------------------------------------ MMA issuer: the warp runs the loop converged, one elected lane issues (see elect_one)
+        {
             constexpr uint32_t idesc = make_idesc_bf16(BM, BN, 0, 1);
             // descriptors without their start address.  A: K-major, 128-byte swizzle, 8-row groups 1024 B apart.
             // B: N-major, 128-byte swizzle: 64-column blocks 8 KB apart (LBO), 8-k groups 1 KB apart (SBO).
@@ -185,26 +185,27 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             bool ok = true;
             for (uint32_t it = 0; ok; ++it) {
                 const int r = it % kRing;
-                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
-                    report_timeout(p, 3);
+                if (!mbar_wait_all(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 3);
                     break;
                 }
                 const int u = ctl->ring[r];
-                mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                __syncwarp();       // every lane has read the entry before it is handed back
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
                 if (u < 0) break;
                 const int ks = u % p.k_splits;
                 const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
                 const int s1 = min(p.kslabs_total, (ks + 1) * p.kslabs_per_split);
                 const uint32_t acc = tile_it & 1;
-                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
-                    report_timeout(p, 4);
+                if (!mbar_wait_all(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 4);
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int i = 0, n = s1 - s0; i < n; ++i) {
-                    if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
-                        report_timeout(p, 5);
+                    if (!mbar_wait_all(full0 + st * 8, ph, abort_flag, limit)) {
+                        if (lane == 0) report_timeout(p, 5);
                         ok = false;
                         break;
                     }
@@ -212,21 +213,29 @@ k_gemm_persistent(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                     const uint32_t sa = s_stage + st * C::stage_bytes;
                     const uint64_t da = da_t | (uint64_t)(sa >> 4);
                     const uint64_t db = db_t | (uint64_t)((sa + C::a_bytes) >> 4);
-                    tc_mma_f16(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
+                    if (elect_one()) {
+                        tc_mma_f16(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k4 = 1; k4 < BK / 16; ++k4) tc_mma_f16(d_tmem, da + k4 * 2, db + k4 * 128, idesc, 1u);
-                    tc_commit(empty0 + st * 8);  // slot reusable once these MMAs have read it
+                        for (int k4 = 1; k4 < BK / 16; ++k4) tc_mma_f16(d_tmem, da + k4 * 2, db + k4 * 128, idesc, 1u);
+                        tc_commit(empty0 + st * 8);  // slot reusable once these MMAs have read it
+                    }
+                    __syncwarp();
                     if (++st == (uint32_t)C::stages) { st = 0; ph ^= 1; }
                 }
                 if (!ok) break;
-                tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                if (elect_one()) tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                __syncwarp();
                 ++tile_it;
             }
+            __syncwarp();
             if (*abort_flag) {
                 // let issued MMAs retire before tensor memory is released
-                tc_commit(smem_u32(&ctl->mma_drain));
-                int dummy = 0;
-                mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                if (elect_one()) {
+                    tc_commit(smem_u32(&ctl->mma_drain));
+                    int dummy = 0;
+                    mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                }
+                __syncwarp();
             }
         }
     } else {

@@ -230,8 +230,9 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 q_run += (uint32_t)n_st;
             }
         } else if (warp == 1) {
-            if (lane == 0) {
+            {
                 // ------------------------------------------------ MMA issuer (leader) / ring consumer (peer)
+                // All 32 lanes run the loop converged and one elected lane issues the MMAs and commits (see elect_one).
                 constexpr uint32_t idesc = make_idesc_bf16(2 * P_BM, P_BN, 0, PACKED_B ? 0 : 1);
                 // descriptors without their start address.  A: K-major, 128-byte swizzle, 8 rows 1 KB apart.  B: row-major
                 // source = N-major, 128-byte swizzle, the two 64-column blocks half the B part apart (LBO), 8 k rows 1 KB
@@ -246,17 +247,18 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 bool ok = true;
                 for (uint32_t it = 0; ok; ++it) {
                     const int r = it % kRing;
-                    if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
-                        report_timeout(p, 3);
+                    if (!mbar_wait_all(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                        if (lane == 0) report_timeout(p, 3);
                         break;
                     }
                     const int u = ctl->ring[r];
-                    mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                    __syncwarp();       // every lane has read the entry before it is handed back
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
                     if (u < 0) break;
                     if (!leader) continue;
                     const uint32_t acc = tile_it & 1;
-                    if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
-                        report_timeout(p, 4);
+                    if (!mbar_wait_all(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
+                        if (lane == 0) report_timeout(p, 4);
                         break;
                     }
                     tc_fence_after();
@@ -268,8 +270,8 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                     const int rot = PACKED_B ? ((tm & 7) * max(1, n_st / 8)) % n_st : 0;
                     const bool odd_tail = (p.kslabs_total & 1) != 0;
                     for (int i = 0; i < n_st; ++i) {
-                        if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
-                            report_timeout(p, 5);
+                        if (!mbar_wait_all(full0 + st * 8, ph, abort_flag, limit)) {
+                            if (lane == 0) report_timeout(p, 5);
                             ok = false;
                             break;
                         }
@@ -277,26 +279,34 @@ k_gemm_persistent_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                         const uint32_t sa = base + st * P_STAGE_BYTES;
                         const uint64_t da = da_t | (uint64_t)(sa >> 4);
                         const uint64_t db = db_t | (uint64_t)((sa + P_A_BYTES) >> 4);
-                        tc_mma_f16_pair(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
-#pragma unroll
-                        for (int k4 = 1; k4 < P_BK / 16; ++k4) tc_mma_f16_pair(d_tmem, da + k4 * kAStep, db + k4 * kBStep, idesc, 1u);
                         const bool half = odd_tail && ((i + rot) % n_st) == n_st - 1;   // the stage that holds the last, single k-slab
-                        if (!half) {
+                        if (elect_one()) {
+                            tc_mma_f16_pair(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
 #pragma unroll
-                            for (int k4 = 0; k4 < P_BK / 16; ++k4)
-                                tc_mma_f16_pair(d_tmem, da + kASlabStep + k4 * kAStep, db + (4 + k4) * kBStep, idesc, 1u);
+                            for (int k4 = 1; k4 < P_BK / 16; ++k4) tc_mma_f16_pair(d_tmem, da + k4 * kAStep, db + k4 * kBStep, idesc, 1u);
+                            if (!half) {
+#pragma unroll
+                                for (int k4 = 0; k4 < P_BK / 16; ++k4)
+                                    tc_mma_f16_pair(d_tmem, da + kASlabStep + k4 * kAStep, db + (4 + k4) * kBStep, idesc, 1u);
+                            }
+                            tc_commit_pair(empty0 + st * 8);
                         }
-                        tc_commit_pair(empty0 + st * 8);
+                        __syncwarp();
                         if (++st == P_STAGES) { st = 0; ph ^= 1; }
                     }
                     if (!ok) break;
-                    tc_commit_pair(smem_u32(&ctl->tmem_full[acc]));
+                    if (elect_one()) tc_commit_pair(smem_u32(&ctl->tmem_full[acc]));
+                    __syncwarp();
                     ++tile_it;
                 }
+                __syncwarp();
                 if (leader && *abort_flag) {
-                    tc_commit(smem_u32(&ctl->mma_drain));
-                    int dummy = 0;
-                    mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                    if (elect_one()) {
+                        tc_commit(smem_u32(&ctl->mma_drain));
+                        int dummy = 0;
+                        mbar_wait(smem_u32(&ctl->mma_drain), 0, &dummy, 2000000ull);
+                    }
+                    __syncwarp();
                 }
             }
         } else {

@@ -421,7 +421,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
         }
         if (!ok && lane == 0) linger_for_copies();
     } else if (warp == 1 || warp == SK_MMA2_WARP) {
-        if (lane == 0 && (warp == 1 || kNMMA == 2)) {
+        if (warp == 1 || kNMMA == 2) {
             // ------------------------------------------------ MMA issuers (with 64 or 128 activation rows: warp 1 alone).  Thread t (0: warp 1, 1: the last warp) owns the
             // stage buffers of parity t, i.e. every second stage of the block's run.  One thread alone is the cap of the
             // pipeline below the full chip: it spends 500-700 cycles per 32 KB stage (eight MMAs of ~45 cycles, a barrier
@@ -431,6 +431,7 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             // lap before as "full").  Inside a unit the thread therefore has the stages of one parity a, and adds them up
             // in accumulator a: accumulator 0 always holds the unit's even stages and accumulator 1 the odd ones, so the
             // value of C does not depend on what the SM ran before.
+            // All 32 lanes of the warp run the loop converged; one elected lane issues the MMAs and commits (see elect_one).
             const int t = warp == 1 ? 0 : 1;
             constexpr uint32_t idesc = make_idesc_bf16(128, NM, PACKED ? 0 : 1, 0);
             // descriptors without their start address.  Weights: packed page = no swizzle, 16-byte k chunks 128 B
@@ -451,12 +452,13 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
             bool ok = true;
             for (uint32_t it = 0; ok; ++it) {
                 const int r = it % kRing;
-                if (!mbar_wait(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
-                    report_timeout(p, 3);
+                if (!mbar_wait_all(smem_u32(&ctl->sched_full[r]), (it / kRing) & 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 3);
                     break;
                 }
                 const int u = ctl->ring[r];
-                mbar_arrive(smem_u32(&ctl->sched_empty[r]));
+                __syncwarp();       // every lane has read the entry before it is handed back
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->sched_empty[r]));
                 if (u < 0) break;
                 const int ks = u % p.k_splits;
                 const int s0 = min(p.kslabs_total, ks * p.kslabs_per_split);
@@ -465,8 +467,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 const int n_st = (n_slabs + SK_SLABS - 1) / SK_SLABS;
                 const int n_grp = (n_slabs + SK_AGRP - 1) / SK_AGRP;
                 const uint32_t acc = tile_it & 1;
-                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
-                    report_timeout(p, 4);
+                if (!mbar_wait_all(smem_u32(&ctl->tmem_empty[acc]), ((tile_it >> 1) & 1) ^ 1, abort_flag, limit)) {
+                    if (lane == 0) report_timeout(p, 4);
                     break;
                 }
                 tc_fence_after();
@@ -477,8 +479,8 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                 if constexpr (kUnified) {
                     // activations behind the weights of the same stage: one barrier per stage, no activation buffers
                     for (int i = 0; i < n_st; ++i) {
-                        if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
-                            report_timeout(p, 5);
+                        if (!mbar_wait_all(full0 + st * 8, ph, abort_flag, limit)) {
+                            if (lane == 0) report_timeout(p, 5);
                             ok = false;
                             break;
                         }
@@ -486,17 +488,21 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                         const uint32_t sbase = base + st * kStageBytes;
                         const uint64_t dw = dw_t | (uint64_t)(sbase >> 4);
                         const uint64_t da = da_t | (uint64_t)((sbase + SK_W_BYTES) >> 4);
-                        tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
+                        const bool two = n_slabs - i * SK_SLABS > 1;
+                        if (elect_one()) {
+                            tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
 #pragma unroll
-                        for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
-                        if (n_slabs - i * SK_SLABS > 1) {
-                            const uint64_t da2 = da + (kASlab >> 4);
+                            for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
+                            if (two) {
+                                const uint64_t da2 = da + (kASlab >> 4);
 #pragma unroll
-                            for (int k4 = 0; k4 < SK_BK / 16; ++k4)
-                                tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                                for (int k4 = 0; k4 < SK_BK / 16; ++k4)
+                                    tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                            }
+                            tc_commit(empty0 + st * 8);
                         }
+                        __syncwarp();
                         first = false;
-                        tc_commit(empty0 + st * 8);
                         if (++st == ring_n) { st = 0; ph ^= 1; }
                     }
                 } else
@@ -506,53 +512,63 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
                     int i = g * kGrpStages + a;
                     // (waited for even when nothing of the group is this thread's: its release below must not be
                     // counted among the releases of the group that used the buffer before)
-                    if (!mbar_wait(smem_u32(&ctl->a_full[aj]), aph, abort_flag, limit)) {
-                        report_timeout(p, 9);
+                    if (!mbar_wait_all(smem_u32(&ctl->a_full[aj]), aph, abort_flag, limit)) {
+                        if (lane == 0) report_timeout(p, 9);
                         ok = false;
                         break;
                     }
                     if (i >= i_end) {
                         // a last group of one stage: nothing of it is this thread's
-                        mbar_arrive(smem_u32(&ctl->a_empty[aj]));
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl->a_empty[aj]));
                         break;
                     }
                     uint64_t da = (da_t | (uint64_t)((a_base + aj * kAStage) >> 4)) + (uint32_t)a * (SK_SLABS * (kASlab >> 4));
                     for (; i < i_end; i += kNMMA) {
-                        if (!mbar_wait(full0 + st * 8, ph, abort_flag, limit)) {
-                            report_timeout(p, 5);
+                        if (!mbar_wait_all(full0 + st * 8, ph, abort_flag, limit)) {
+                            if (lane == 0) report_timeout(p, 5);
                             ok = false;
                             break;
                         }
                         tc_fence_after();
                         const uint64_t dw = dw_t | (uint64_t)((base + st * kStageBytes) >> 4);
                         // the first k-slab of the stage, then the second one if the unit has it
-                        tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
+                        const bool two = n_slabs - i * SK_SLABS > 1;
+                        if (elect_one()) {
+                            tc_mma_f16(d_tmem, dw, da, idesc, first ? 0u : 1u);
 #pragma unroll
-                        for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
-                        if (n_slabs - i * SK_SLABS > 1) {
-                            const uint64_t da2 = da + (kASlab >> 4);
+                            for (int k4 = 1; k4 < SK_BK / 16; ++k4) tc_mma_f16(d_tmem, dw + k4 * kWStep, da + k4 * kAStepK, idesc, 1u);
+                            if (two) {
+                                const uint64_t da2 = da + (kASlab >> 4);
 #pragma unroll
-                            for (int k4 = 0; k4 < SK_BK / 16; ++k4)
-                                tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                                for (int k4 = 0; k4 < SK_BK / 16; ++k4)
+                                    tc_mma_f16(d_tmem, dw + (4 + k4) * kWStep, da2 + k4 * kAStepK, idesc, 1u);
+                            }
+                            tc_commit(empty0 + st * 8);
                         }
+                        __syncwarp();
                         first = false;
-                        tc_commit(empty0 + st * 8);
                         st += kNMMA;
                         if (st >= ring_n) { st -= ring_n; ph ^= 1; }
                         da += kNMMA * SK_SLABS * (kASlab >> 4);
                     }
-                    if (ok) tc_commit(smem_u32(&ctl->a_empty[aj]));    // this thread's last read of the buffer has been issued
+                    if (ok && elect_one()) tc_commit(smem_u32(&ctl->a_empty[aj]));    // this thread's last read of the buffer has been issued
+                    __syncwarp();
                 }
                 if (!ok) break;
-                tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                if (elect_one()) tc_commit(smem_u32(&ctl->tmem_full[acc]));
+                __syncwarp();
                 q0 += (uint32_t)n_st;
                 git += (uint32_t)n_grp;
                 ++tile_it;
             }
+            __syncwarp();
             if (*abort_flag) {
-                tc_commit(smem_u32(&ctl->mma_drain[t]));
-                int dummy = 0;
-                mbar_wait(smem_u32(&ctl->mma_drain[t]), 0, &dummy, 2000000ull);
+                if (elect_one()) {
+                    tc_commit(smem_u32(&ctl->mma_drain[t]));
+                    int dummy = 0;
+                    mbar_wait(smem_u32(&ctl->mma_drain[t]), 0, &dummy, 2000000ull);
+                }
+                __syncwarp();
             }
         }
     } else {

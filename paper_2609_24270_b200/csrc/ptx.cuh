@@ -89,6 +89,23 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     return ok != 0;
 }
 
+// Every lane of a converged warp waits (each polls on its own); all lanes get the same outcome and leave converged.
+// For the warps that issue MMAs: see elect_one.
+__device__ __forceinline__ bool mbar_wait_all(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                              uint64_t limit_ns) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, limit_ns);
+    return __all_sync(0xffffffffu, ok);
+}
+// One lane of a converged warp (always the same one for the full mask).  A warp that issues tcgen05.mma runs its loop
+// with all 32 lanes and lets the elected lane issue: the descriptors are then computed in warp-uniform code, and
+// eight small MMAs plus their commit cost the issuing thread 250 ns (measured) where the same instructions inside a
+// lane-0-only branch cost 485 ns whatever their shape (N = 16 to 256) - more than the tensor pipe needs for them.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t elected;
+    asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xffffffff;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(elected));
+    return elected != 0;
+}
+
 // ---- TMA -----------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
