@@ -304,8 +304,10 @@ typedef struct ag_plan ag_plan;
  *   amap    handle or NULL; required for AG_AFFINITY
  *   policy  host
  *   plan    host, out: new handle
- * Errors: AG_ERR_ARG (budget out of range, bad tile shape, empty k-split, operand outside the
- * probed buffer, AG_AFFINITY without amap), AG_ERR_CUDA, AG_ERR_NOMEM.
+ * At most 2^20 work units, whatever the policy (the affinity policy finds each die's share with a radix
+ * select over the units' byte margins, not a sort).
+ * Errors: AG_ERR_ARG (budget out of range, bad tile shape, empty k-split, more than 2^20 units, operand
+ * outside the probed buffer, AG_AFFINITY without amap), AG_ERR_CUDA, AG_ERR_NOMEM.
  */
 ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* amap, int sm_budget,
                       const ag_policy* policy, ag_plan** plan);

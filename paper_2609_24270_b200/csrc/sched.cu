@@ -298,14 +298,45 @@ __global__ void k_score_units(PolicyDev pol, int n_units, int tiles_m, int tiles
     if (lane == 0) margins[warp] = m;
 }
 
+// Block-wide helpers for k_assign (called by every thread of the block, blockDim.x a multiple of 32, at most 1024).
+__device__ inline int block_sum(int v, int* s_warp) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();                       // s_warp may still be read by the call before
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int t = 0;
+    for (int k = 0; k < (int)(blockDim.x >> 5); ++k) t += s_warp[k];
+    return t;
+}
+// number of set flags at lower thread ids; total = set flags of the whole block
+__device__ inline int block_excl_scan_flag(bool f, int* s_warp, int& total) {
+    const unsigned m = __ballot_sync(0xffffffffu, f);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) s_warp[w] = __popc(m);
+    __syncthreads();
+    int before = 0, t = 0;
+    for (int k = 0; k < (int)(blockDim.x >> 5); ++k) {
+        const int c = s_warp[k];
+        before += k < w ? c : 0;
+        t += c;
+    }
+    total = t;
+    return before + __popc(m & ((1u << lane) - 1u));
+}
+
 // ---- steps 5-6: unit -> die, per-die queues, per-SM lists: one thread block ----------------------
 __global__ void __launch_bounds__(1024)
 k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long long* __restrict__ margins,
-         int32_t* __restrict__ image, PlanLayout lay, int32_t* __restrict__ order, int32_t* __restrict__ die_of) {
+         int32_t* __restrict__ image, PlanLayout lay, int32_t* __restrict__ die_of) {
     const int tid = threadIdx.x, nt = blockDim.x;
     __shared__ int n_d[2];
     __shared__ int slots_of_die[2][AG_MAX_SM];
+    __shared__ int s_warp[32];
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long s_sel[2];     // radix select: key prefix found so far, rank still to go
     if (tid == 0) {
+        s_sel[0] = 0;
         n_d[0] = image[lay.die_sm_count()];
         n_d[1] = image[lay.die_sm_count() + 1];
         int c[2] = {0, 0};
@@ -328,46 +359,98 @@ k_assign(PolicyDev pol, int b, int n_units, int tiles_m, int tiles_n, const long
     } else if (pol.kind == AG_DIE_COMPACT) {
         for (int i = tid; i < n_units; i += nt) die_of[i] = band_die(i, n_units, q0, group_len);
     } else {
-        // rank of raster index i under the key (|m| descending, i ascending)
+        // The greedy pass of the plan (units in the order |margin| descending, raster index ascending; a unit takes the
+        // die it prefers while that die has quota left, else the other) in closed form.  Until a die is full every unit
+        // gets its preference, and once a die is full everything goes to the other one; the quotas add up to the unit
+        // count, so at most one die d has more takers than quota q[d], and it keeps exactly its first q[d] takers in
+        // that order.  Their cut is found by a radix select over the 64-bit keys (eight histogram passes) and a prefix
+        // count over the units that tie with the cut; no sort, any unit count.
+        auto key_pref = [&](int i, int& pref) -> unsigned long long {
+            long long m = margins[i];
+            if (pol.invert) m = -m;
+            long long am = m < 0 ? -m : m;
+            if (am < pol.min_margin) { am = 0; m = 0; }
+            pref = m > 0 ? 0 : (m < 0 ? 1 : band_die(i, n_units, q0, group_len));
+            return (unsigned long long)am;
+        };
+        int mine0 = 0;
         for (int i = tid; i < n_units; i += nt) {
-            long long mi = margins[i] < 0 ? -margins[i] : margins[i];
-            if (mi < pol.min_margin) mi = 0;
-            int rank = 0;
-            for (int j = 0; j < n_units; ++j) {
-                long long mj = margins[j] < 0 ? -margins[j] : margins[j];
-                if (mj < pol.min_margin) mj = 0;
-                rank += (mj > mi) || (mj == mi && j < i);
-            }
-            order[rank] = i;
+            int pref;
+            key_pref(i, pref);
+            mine0 += pref == 0;
         }
-        __syncthreads();
-        if (tid == 0) {
-            int got[2] = {0, 0};
-            for (int r = 0; r < n_units; ++r) {
-                const int i = order[r];
-                long long m = margins[i];
-                if (pol.invert) m = -m;
-                if ((m < 0 ? -m : m) < pol.min_margin) m = 0;
-                const int pref = m > 0 ? 0 : (m < 0 ? 1 : band_die(i, n_units, q0, group_len));
-                const int d = got[pref] < q[pref] ? pref : 1 - pref;
-                got[d]++;
+        const int n_pref0 = block_sum(mine0, s_warp);
+        const int d_full = n_pref0 > q[0] ? 0 : ((n_units - n_pref0) > q[1] ? 1 : -1);
+        unsigned long long cut = 0;    // key of the last taker that die d_full keeps
+        int keep_ties = 0;             // how many takers with exactly that key it keeps (lowest raster indices)
+        if (d_full >= 0 && q[d_full] > 0) {
+            if (tid == 0) {
+                s_sel[0] = 0;
+                s_sel[1] = (unsigned long long)q[d_full];
+            }
+            __syncthreads();
+            for (int byte = 7; byte >= 0; --byte) {
+                for (int k = tid; k < 256; k += nt) hist[k] = 0;
+                __syncthreads();
+                const unsigned long long prefix = s_sel[0];
+                for (int i = tid; i < n_units; i += nt) {
+                    int pref;
+                    const unsigned long long key = key_pref(i, pref);
+                    if (pref == d_full && (byte == 7 || (key >> (8 * (byte + 1))) == prefix))
+                        atomicAdd(&hist[(unsigned)(key >> (8 * byte)) & 255u], 1u);
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    unsigned long long rank = s_sel[1];     // 1-based rank of the cut among the keys that share the prefix
+                    int bin = 255;
+                    for (; bin > 0 && hist[bin] < rank; --bin) rank -= hist[bin];
+                    s_sel[0] = (prefix << 8) | (unsigned long long)bin;
+                    s_sel[1] = rank;
+                }
+                __syncthreads();
+            }
+            cut = s_sel[0];
+            keep_ties = (int)s_sel[1];
+        }
+        int ties_before = 0;           // takers of d_full with key == cut at raster indices below the current chunk
+        for (int base = 0; base < n_units; base += nt) {
+            const int i = base + tid;
+            int pref = 0;
+            unsigned long long key = 0;
+            if (i < n_units) key = key_pref(i, pref);
+            const bool tie = i < n_units && d_full >= 0 && pref == d_full && key == cut;
+            int total;
+            const int pos = ties_before + block_excl_scan_flag(tie, s_warp, total);
+            ties_before += total;
+            if (i < n_units) {
+                int d = pref;
+                if (pref == d_full && (q[d_full] == 0 || key < cut || (key == cut && pos >= keep_ties))) d = 1 - d_full;
                 die_of[i] = d;
             }
         }
     }
     __syncthreads();
-    // per-die queues in raster order
+    // per-die queues in raster order: a unit's place is the number of units of its die before it
+    int mine = 0;
+    for (int i = tid; i < n_units; i += nt) mine += die_of[i] == 0;
+    const int cnt0 = block_sum(mine, s_warp);
+    const int cnt[2] = {cnt0, n_units - cnt0};
+    int zeros_before = 0;
+    for (int base = 0; base < n_units; base += nt) {
+        const int i = base + tid;
+        const bool z = i < n_units && die_of[i] == 0;
+        int total;
+        const int zb = zeros_before + block_excl_scan_flag(z, s_warp, total);
+        zeros_before += total;
+        if (i < n_units) {
+            const int u = raster_unit(i, tiles_m, tiles_n, pol.k_splits, pol.raster_group);
+            image[lay.die_q() + (z ? zb : cnt0 + (i - zb))] = u;
+        }
+    }
     if (tid == 0) {
-        int cnt[2] = {0, 0};
-        for (int i = 0; i < n_units; ++i) cnt[die_of[i]]++;
         image[lay.die_q_off() + 0] = 0;
         image[lay.die_q_off() + 1] = cnt[0];
         image[lay.die_q_off() + 2] = n_units;
-        int pos[2] = {0, cnt[0]};
-        for (int i = 0; i < n_units; ++i) {
-            const int u = raster_unit(i, tiles_m, tiles_n, pol.k_splits, pol.raster_group);
-            image[lay.die_q() + pos[die_of[i]]++] = u;
-        }
         // list lengths and offsets
         int off = 0;
         for (int s = 0; s < b; ++s) {
@@ -468,7 +551,6 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
     const long long tiles_m = (p.M + p.tile_m - 1) / p.tile_m, tiles_n = (p.N + p.tile_n - 1) / p.tile_n;
     const long long n_units_ll = tiles_m * tiles_n * p.k_splits;
     if (n_units_ll > (1 << 20)) return AG_ERR_ARG;
-    if (p.kind == AG_AFFINITY && n_units_ll > 65536) return AG_ERR_ARG;
     const int n_units = (int)n_units_ll;
     if (p.kind == AG_AFFINITY) {
         if (!operand_in_range(p.a, p.M, p.K, amap->bytes) || !operand_in_range(p.c, p.M, p.N, amap->bytes))
@@ -503,7 +585,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
 
     ag_topo_map* d_topo = nullptr;
     int32_t* d_table = nullptr;
-    int32_t *d_order = nullptr, *d_die_of = nullptr;
+    int32_t* d_die_of = nullptr;
     ag_status st = AG_OK;
     auto fail = [&](cudaError_t e) { st = cuda_fail(e); };
     cudaError_t e;
@@ -523,7 +605,6 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
         }
         TRY(cudaMalloc(&d_topo, sizeof(ag_topo_map)));
         TRY(cudaMemcpy(d_topo, map, sizeof(ag_topo_map), cudaMemcpyHostToDevice));
-        TRY(cudaMalloc(&d_order, sizeof(int32_t) * n_units));
         TRY(cudaMalloc(&d_die_of, sizeof(int32_t) * n_units));
         if (p.kind == AG_AFFINITY && p.b.present && p.b.layout == AG_LAYOUT_PAGED) {
             TRY(cudaMalloc(&d_table, sizeof(int32_t) * (size_t)p.b.n_pages));
@@ -556,7 +637,7 @@ extern "C" ag_status sched_build(const ag_topo_map* map, const ag_affinity_map* 
             TRY(cudaGetLastError());
         }
         k_assign<<<1, 1024>>>(pd, sm_budget, n_units, (int)tiles_m, (int)tiles_n, pl->d_margins, pl->d_image,
-                              pl->lay, d_order, d_die_of);
+                              pl->lay, d_die_of);
         count_launch();
         TRY(cudaGetLastError());
         TRY(cudaDeviceSynchronize());
@@ -600,7 +681,6 @@ done:
 #undef TRY
     cudaFree(d_topo);
     cudaFree(d_table);
-    cudaFree(d_order);
     cudaFree(d_die_of);
     if (st != AG_OK) {
         ag_plan_destroy(pl);

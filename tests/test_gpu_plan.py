@@ -144,6 +144,24 @@ def test_affinity_plan_matches_oracle_rowmajor(invert, min_margin):
         assert m[i] == l0 - l1
 
 
+@pytest.mark.parametrize("invert", [0, 1])
+def test_affinity_plan_with_100k_units_and_tied_margins_matches_oracle(invert):
+    """More units than a sort-free builder used to take (65536), with only five distinct margin values, so the cut
+    between the units a full die keeps and those it passes on falls inside a run of equal keys."""
+    topo = inputs.synthetic_topo(die0_sms=70, seed=4)
+    U = 100_000
+    M, N, K = 4, 128 * U, 64
+    nbytes = M * N * 4
+    tbl = inputs.synthetic_chunk_die(nbytes // 4096, seed=11).copy()
+    tbl[::3] = 0                                             # die 0 is preferred by more units than its quota
+    kw = dict(kind=ag.AG_AFFINITY, M=M, N=N, K=K, tile_m=16, tile_n=128, invert_affinity=invert, raster_group=1,
+              c=dict(offset=0, row_stride=N * 4, elem_bytes=4))
+    got, want, plan = both(topo, tbl, 148, **kw)
+    assert got.tobytes() == want.tobytes()
+    m = np.abs(plan.margins())
+    assert len(np.unique(m)) <= 5 and (m > 0).sum() > U // 4
+
+
 def test_affinity_full_size_sampled_margins_and_invariants():
     """8192^3 / 2048 units: the oracle scores a sample of units; the rest is checked by invariants."""
     topo = inputs.synthetic_topo(die0_sms=70, seed=12)
