@@ -37,8 +37,8 @@ FLOPS = 2.0 * M * N * K
 METRIC = "bf16_gemm_tflops"
 UNIT = "TFLOP/s"
 # DRAM bytes per launch of the dominant kernel, from an Nsight Compute capture of two timed steps of this
-# bench (dram__bytes_read.sum 1.042 GB + dram__bytes_write.sum 0.251 GB; summary kept under profiles/).
-NCU_TRAFFIC_BYTES = 1.293e9
+# bench (dram__bytes_read.sum 1.083 GB + dram__bytes_write.sum 0.251 GB; summary kept under profiles/).
+NCU_TRAFFIC_BYTES = 1.334e9
 IDLE_BEFORE_TIMED_S = 2.0        # pause in front of the warm-up and timed steps of the headline (see there)
 # the same for the decode-shaped GEMM (135.08 MB read + 3.9 MB written per launch, 16 k-splits) and for the attention
 # kernel (269.69 MB + 3.7 MB); both captures read every algorithmic byte exactly once

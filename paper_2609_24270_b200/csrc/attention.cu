@@ -932,7 +932,8 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     cfg.blockDim = dim3(AT_THREADS);
     cfg.dynamicSmemBytes = AT_SMEM_BYTES;
     cfg.stream = stream;
-    const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0 && plan->lay.b == plan->lay.n_sm;
+    const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0;
+    if (overlap && plan->lay.b < plan->lay.n_sm) gp.manned_wait_ns = gp.wait_limit_ns;   // see gemm_skinny_dispatch
     x.release_next = overlap ? 1 : 0;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -823,12 +823,13 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     }
     // every argument check has passed: from here on work is queued on the stream
     const bool zeroing = h[H_KSPLITS] > 1 && !x.partial;
-    // Overlapping launches: only for plans that use every SM with one block each - the blocks of the next launch then
-    // find room exactly where a block of this one has left, one per SM, and no block of the launch after next can
-    // start before this launch has completed.  (With fewer planned SMs the next launch's blocks would all land on the
-    // idle SMs and leave the planned ones without a block.)  Static lists only: the queue heads of dynamic plans
-    // belong to one launch at a time.
-    const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0 && plan->lay.b == plan->lay.n_sm;
+    // Overlapping launches: the blocks of the next launch find room where a block of this one has left, one per SM, and
+    // no block of the launch after next can start before every block of the next one has started.  With a plan for part
+    // of the chip the next launch's first blocks land on the unplanned SMs while this launch still holds the planned
+    // ones; they stay there until the planned SMs have their blocks (wait_until_manned without its 40 us limit), so that
+    // the remaining blocks can only land where this launch's blocks leave.  Static lists only: the queue heads of
+    // dynamic plans belong to one launch at a time.
+    const bool overlap = plan->policy.overlap_launches && h[H_STATIC] && plan->grid_blocks == 0;
     x.release_next = overlap ? 1 : 0;
     x.a_after_prior = (overlap && plan->policy.overlap_launches != 2) ? 1 : 0;
     x.stages = ring_stages_for(plan, sk_stages(NM), std::min(sk_stages(NM), 2), sk_nmma(NM) == 2, false);
@@ -851,6 +852,7 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
         count_launch();
     }
     PersistParams gp = make_persist_params(plan, M, N, K);
+    if (overlap && plan->lay.b < plan->lay.n_sm) gp.manned_wait_ns = gp.wait_limit_ns;
     gp.b_blocks = grp ? ((!W && grp->w_blocks) ? 1 : 0) : ((!W && N % 64 == 0) ? 1 : 0);
     gp.a_blocks = a_blocks ? 1 : 0;
     ag_status ls;

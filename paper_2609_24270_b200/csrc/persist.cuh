@@ -28,6 +28,7 @@ struct PersistParams {
     int static_assign;
     unsigned int epoch;
     unsigned long long wait_limit_ns;
+    unsigned long long manned_wait_ns;   // how long a block on an unplanned SM stays to keep that SM occupied (wait_until_manned)
     int b_blocks;           // 1: tm_b is the 3-D [N/64][K][64] view of B (one copy per k-slab)
     int a_blocks;           // 1: tm_a is the 3-D [K/64][M][64] view of A (decode-shaped kernel: one copy per 8 k-slabs)
     const int4* quick;      // [n_sm]: {slot, offset of the SM's list in sm_q, its length, its first unit} (slot -1: unplanned)
@@ -68,7 +69,8 @@ __device__ __forceinline__ bool slot_taken(const PersistParams& p, int i) {
     return epoch_reached(*reinterpret_cast<volatile unsigned int*>(&p.claimed[i]), p.epoch);
 }
 
-// A block on an unplanned SM stays resident until every planned SM has a block (at most ~40 us),
+// A block on an unplanned SM stays resident until every planned SM has a block (at most ~40 us; with overlapping
+// launches on part of the chip until the launch before has left the planned SMs, bounded like every other wait),
 // so that blocks still being placed can only land on SMs that have none yet.  Called by every thread.
 __device__ inline void wait_until_manned(const PersistParams& p) {
     const uint64_t t0 = globaltimer_ns();
@@ -76,7 +78,7 @@ __device__ inline void wait_until_manned(const PersistParams& p) {
         int ok = 1;
         for (int i = threadIdx.x; i < p.b; i += blockDim.x) ok &= slot_taken(p, i) ? 1 : 0;
         if (__syncthreads_and(ok)) break;
-        if (globaltimer_ns() - t0 > 40000ull) break;
+        if (globaltimer_ns() - t0 > p.manned_wait_ns) break;
         __nanosleep(200);
     }
 }
@@ -230,6 +232,7 @@ inline PersistParams make_persist_params(const ag_plan* plan, int M, int N, int 
     gp.claimed = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(plan->d_ctrl) + offsetof(PlanCtrl, claimed)) +
                  (size_t)AG_MAX_SM * (gp.epoch & 1u);
     gp.wait_limit_ns = kWaitLimitNs;
+    gp.manned_wait_ns = 40000ull;
     gp.b_blocks = 0;
     gp.a_blocks = 0;
     gp.quick = plan->d_quick;

@@ -117,7 +117,8 @@ def test_serving_shape_on_sm_budgets():
     Q, K, V = make_case(B, Hq, Hkv, L, seed=21)
     want = oa.gqa_decode(Q, K, V)
     # the last one with overlapping launches (the second launch begins while the first one finishes)
-    for placement, budget, overlap in ((ag.KV_LOCAL, None, 0), (ag.KV_REMOTE, None, 0), (ag.KV_LOCAL, 74, 0), (ag.KV_LOCAL, None, 1)):
+    for placement, budget, overlap in ((ag.KV_LOCAL, None, 0), (ag.KV_REMOTE, None, 0), (ag.KV_LOCAL, 74, 0), (ag.KV_LOCAL, None, 1),
+                                       (ag.KV_LOCAL, 74, 1), (ag.KV_INTERLEAVED, 37, 1)):
         got, _, _ = run_attention(Q, K, V, placement, budget=budget, overlap=overlap)
         check(got, want)
 

@@ -127,10 +127,12 @@ def test_overlapping_launches_in_a_dependent_chain():
     A0 = rng.integers(-8, 9, size=(M, K)).astype(np.float32)
     x = torch.from_numpy(A0).cuda().to(torch.bfloat16)
     dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
-    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
-                                                                k_splits=ksp, splitk_in_memory=1, overlap_launches=1))
+    plans = [ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
+                                                          k_splits=ksp, splitk_in_memory=1, overlap_launches=1))
+             for b in (topo.n_sm, 37, 74)]
     want = A0
     for rep in range(3):
+        plan = plans[rep]
         for W, pm in zip(Ws, perms):
             ag.gemm_persistent(x.data_ptr(), W.data_ptr(), dC.data_ptr(), M, N, K, plan, torch.cuda.current_stream().cuda_stream)
             x = dC.to(torch.bfloat16)                    # the next call's activations, written by the launch right before it
@@ -138,7 +140,7 @@ def test_overlapping_launches_in_a_dependent_chain():
             nxt[:, pm] = want
             want = nxt
     torch.cuda.synchronize()
-    assert plan.last_status() == ag.AG_OK
+    assert all(pl.last_status() == ag.AG_OK for pl in plans)
     assert np.array_equal(x.float().cpu().numpy(), want)
 
 
@@ -154,8 +156,10 @@ def test_overlapping_launches_integer_exact(in_memory, overlap):
     dA = to_dev_bf16(A)
     dBs = [to_dev_bf16(b) for b in Bs]
     dCs = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
-    for b in (topo.n_sm, 74):
-        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
+    for b, sel in ((topo.n_sm, 0), (74, 0), (37, 1), (20, 0)):
+        # (on part of the chip the next launch's first blocks wait on the unplanned SMs until this launch's blocks have
+        # left the planned ones)
+        plan = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128, sm_select=sel,
                                                             k_splits=ksp, splitk_in_memory=in_memory, overlap_launches=overlap))
         plan.reset_record()
         for i in range(9):
@@ -166,6 +170,7 @@ def test_overlapping_launches_integer_exact(in_memory, overlap):
             assert np.array_equal(dCs[i].cpu().numpy().astype(np.float64), og.gemm_blocked(A, Bs[i]))
         owner, count = plan.tile_record()
         assert (count == 9).all()
+        assert set(owner.tolist()) <= set(plan.parsed()["sm_list"].tolist())     # only planned SMs ran units
 
 
 def test_in_memory_splitk_integer_exact_packed_and_rowmajor():
