@@ -260,7 +260,7 @@ typedef struct {
     int32_t pair_lists;      /* 1: static lists are dealt to TPCs instead of SMs (entry i of a die's queue -> TPC i mod P,
                                 lower SM in even rounds, upper SM in odd ones), so that the two lists of a TPC together
                                 hold a fair share; for plans of block pairs.  Needs whole TPCs, else AG_ERR_ARG */
-    int32_t overlap_launches; /* decode-shaped plans with static lists that use every SM of the chip (ignored otherwise): 1 or 2 =
+    int32_t overlap_launches; /* decode-shaped plans with static lists (ignored otherwise): 1 or 2 =
                                  a launch lets the next launch of this library on the same stream begin while it is still
                                  finishing (programmatic dependent launch): the next launch's thread blocks take over SMs as
                                  they become free and start streaming their weights (attention: key/value pages); nothing
@@ -268,7 +268,10 @@ typedef struct {
                                  weights (B / packed weights, KV pages) of a call are not produced by the call directly
                                  before it.  1: the activations (A, queries) may be - they are read only after the launch
                                  before has completed; 2: the caller promises the same for the activations, and they are
-                                 read at once.  0 = launches run strictly one after the other */
+                                 read at once.  0 = launches run strictly one after the other.  On a plan for part of
+                                 the chip the next launch's surplus blocks wait on the unplanned SMs until the running
+                                 launch has left the planned ones: use it when the stream has the chip to itself, not
+                                 while another stream's kernels are meant to run on the unplanned SMs */
     int32_t cluster_size;    /* die_compact / affinity: thread-block cluster size (1, 2, 4 or 8) of the kernel the SM set is
                                 meant for; 0 and 1 mean none.  For sizes above 2 the set is built from what can host such
                                 clusters: SMs never seen in a cluster larger than 2 (is_random, Section 5.1.1) are taken last,
