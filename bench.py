@@ -256,6 +256,53 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
                 gbs.setdefault(name, []).append(algo_bytes / (ms * 1e-3) / 1e9)
         results[ksp] = {n: float(np.median(v)) for n, v in gbs.items()}
         del packs
+    # The same GEMM on 74 and 37 SMs (4 k-splits): die-local packed weights on a set of whole TPCs spread over the GPCs of
+    # both dies (each die streams its own pages), on a one-die set, the one-die set of the other die reading the same pages
+    # (remote), and row-major weights under oblivious plans (lowest SM ids, and two seeded random subsets).
+    budgets = {}
+    for b in (74, 37):
+        kw = dict(M=Md, N=Nd, K=Kd, tile_m=16, tile_n=128, k_splits=4, splitk_in_memory=1, overlap_launches=2)
+        plan_spread = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, **kw))
+        plan_one = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+        n0 = int(plan_one.parsed()["die_sm_count"][0])
+        plan_far = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, preferred_die=1 if n0 == b else 0, **kw)) \
+            if n0 in (0, b) else None
+        plans_obl = {"rowmajor_oblivious_lowest_ids": ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, **kw))}
+        for seed in (1, 2):
+            plans_obl[f"rowmajor_oblivious_seed_{seed}"] = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_OBLIVIOUS, seed=seed, **kw))
+        out = {}
+        for name, plan_pack, plan_run in (("packed_die_local_both_dies", plan_spread, plan_spread), ("packed_die_local_one_die", plan_one, plan_one),
+                                          ("packed_remote_one_die", plan_one, plan_far)):
+            if plan_run is None:
+                continue
+            packs = [ag.pack_weights(dBs[i].data_ptr(), Kd, Nd, plan_pack, amaps[i], dsts[i].data_ptr(), dst_bytes) for i in range(n_buf)]
+            state = {"i": 0}
+
+            def run_p():
+                i = state["i"] % n_buf
+                state["i"] += 1
+                ag.gemm_persistent_packed(dA.data_ptr(), packs[i], dC.data_ptr(), Md, Nd, Kd, plan_run)
+            ms = time_queued(torch, run_p, iters=16)
+            if plan_run.last_status() != ag.AG_OK:
+                raise RuntimeError(f"decode arm {name} at {b} SMs: " + ag.strerror(plan_run.last_status()))
+            out[name] = algo_bytes / (ms * 1e-3) / 1e9
+            del packs
+        for name, plan in plans_obl.items():
+            state = {"i": 0}
+
+            def run_r():
+                i = state["i"] % n_buf
+                state["i"] += 1
+                ag.gemm_persistent(dA.data_ptr(), dBs[i].data_ptr(), dC.data_ptr(), Md, Nd, Kd, plan)
+            ms = time_queued(torch, run_r, iters=16)
+            out[name] = algo_bytes / (ms * 1e-3) / 1e9
+        obl = [v for n, v in out.items() if n.startswith("rowmajor_oblivious")]
+        out["aware_over_oblivious_median"] = out["packed_die_local_both_dies"] / float(np.median(obl))
+        out["oblivious_max_over_min"] = max(obl) / min(obl)
+        if "packed_remote_one_die" in out:
+            out["local_over_remote_one_die"] = out["packed_die_local_one_die"] / out["packed_remote_one_die"]
+        out["frac_of_hbm_peak_best"] = max(out["packed_die_local_both_dies"], max(obl)) / peaks["hbm_gbs"]
+        budgets[str(b)] = out
     sampler.close("decode")
     gbs = results[16]
     best = gbs["packed_die_local"]
@@ -263,6 +310,7 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
                         f"{n_buf} rotating weight matrices (512 MiB > L2), launches queued back to back, overlap_launches",
             "gbs": gbs, "us_per_call": {n: algo_bytes / v / 1e3 for n, v in gbs.items()},
             "gbs_4_k_splits": results[4],
+            "sm_budgets_4_k_splits": budgets,
             "local_over_remote": gbs["packed_die_local"] / gbs["packed_remote"],
             "aware_over_oblivious": gbs["packed_die_local"] / gbs["rowmajor_oblivious"],
             "group_free_bit": info["group_free_bit"],
@@ -360,6 +408,25 @@ def subset_section(ag, inputs, torch, topo, sampler, budget=64, n_subsets=8):
             "die_compact_over_random_median": res["die_compact"] / float(np.median(rnd)),
             "gpc_spread_over_random_median": res["gpc_spread"] / float(np.median(rnd)),
             "clocks": sampler.summary("subsets")}
+
+
+def multiplex_section(ag, topo, sampler):
+    """Two streams on disjoint SM partitions (110 / 38 SMs): a prefill-like GEMM (8192 x 4096 x 4096, block pairs) and a
+    decode-like GEMM (32 x 4096 x 4096, eight weight matrices in rotation); partitions cut along the dies, and oblivious
+    ones (lowest SM ids / the rest).  Per-stream throughput alone and together."""
+    from paper_2609_24270_b200 import experiments
+    sampler.mark("multiplex")
+    out = {}
+    for rec in experiments.config5_records(topo, splits=((110, 38),), modes=("die_split", "oblivious"), n_alone=2, n_both=3):
+        out[rec["partition"]] = {"prefill_tflops": rec["prefill_tflops"], "decode_gbs": rec["decode_gbs"],
+                                 "prefill_set": rec["prefill_set"], "decode_set": rec["decode_set"]}
+    sampler.close("multiplex")
+    ds, ob = out["die_split"], out["oblivious"]
+    return {"workload": "prefill-like GEMM 8192x4096x4096 on 110 SMs and decode-like GEMM 32x4096x4096 on 38 SMs, two streams",
+            "partitions": out,
+            "die_split_over_oblivious": {"prefill": ds["prefill_tflops"]["overlapped"] / ob["prefill_tflops"]["overlapped"],
+                                         "decode": ds["decode_gbs"]["overlapped"] / ob["decode_gbs"]["overlapped"]},
+            "clocks": sampler.summary("multiplex")}
 
 
 def run_reference(args):
@@ -569,6 +636,7 @@ def main():
     decode = decode_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
     attention = attention_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
     subsets = subset_section(ag, inputs, torch, topo, sampler) if args.only == "all" else None
+    multiplex = multiplex_section(ag, topo, sampler) if args.only == "all" else None
     sampler.stop()
 
     # ---- end to end through the same call with host buffers.  Every step copies its A and B from pinned host
@@ -646,6 +714,7 @@ def main():
         "decode": decode,
         "attention": attention,
         "sm_subsets": subsets,
+        "multiplexing": multiplex,
         "aware_over_oblivious_raster": side["affinity"] / side["oblivious_raster"],
         "die_sm_count": list(topo.die_sm_count), "gpc_sm_count": list(topo.gpc_sm_count[:topo.n_gpc]),
         "setup_s": {"topo_discover": t_topo, "affinity_probe": t_aff, "sched_build_x5": t_plan, "probe_pack_plan_b": t_pack},

@@ -211,6 +211,12 @@ def _unit_die(plan):
 def config5(fh, topo):
     """Prefill-like GEMM (8192x4096x4096) and decode-like GEMM (32x4096x4096 over 8 weight matrices)
     on two streams and disjoint SM partitions; die-split against oblivious (lowest ids / the rest)."""
+    for rec in config5_records(topo):
+        emit(rec, fh)
+
+
+def config5_records(topo, splits=((74, 74), (110, 38)), modes=("die_split", "gpc_spread", "oblivious"), n_alone=3, n_both=5):
+    """The measurements of config5 as a generator of records (bench.py takes a trimmed set of them)."""
     Mp, Md, N, K = 8192, 32, 4096, 4096
     Ap, Bp = inputs.gemm_inputs(Mp, N, K)
     dAp, dBp = dev_bf16(Ap), dev_bf16(Bp)
@@ -224,8 +230,8 @@ def config5(fh, topo):
     bytes_d = K * N * 2 + Md * K * 2 + Md * N * 4
     pre_kw = dict(M=Mp, N=N, K=K, tile_m=256, tile_n=256, raster_group=4)   # both partitions hold whole TPCs: block pairs
     dec_kw = dict(M=Md, N=N, K=K, tile_m=32, tile_n=128, k_splits=8, splitk_in_memory=1)
-    for split in ((74, 74), (110, 38)):
-        for mode in ("die_split", "gpc_spread", "oblivious"):
+    for split in splits:
+        for mode in modes:
             kind = ag.AG_OBLIVIOUS if mode == "oblivious" else ag.AG_DIE_COMPACT
             sel = 1 if mode == "gpc_spread" else 0      # whole TPCs dealt over the GPCs of both dies
             plan_p = ag.sched_build(topo, None, split[0], ag.make_policy(kind=kind, preferred_die=0, sm_select=sel, **pre_kw))
@@ -263,17 +269,17 @@ def config5(fh, topo):
 
             for _ in range(2):
                 run(True, True)
-            alone_p = np.median([run(True, False)[0] for _ in range(3)])
-            alone_d = np.median([run(False, True)[1] for _ in range(3)])
-            both = [run(True, True) for _ in range(5)]
+            alone_p = np.median([run(True, False)[0] for _ in range(n_alone)])
+            alone_d = np.median([run(False, True)[1] for _ in range(n_alone)])
+            both = [run(True, True) for _ in range(n_both)]
             ov_p = np.median([x[0] for x in both])
             ov_d = np.median([x[1] for x in both])
             assert plan_p.last_status() == ag.AG_OK and plan_d.last_status() == ag.AG_OK
-            emit(dict(config=5, split=list(split), partition=mode,
-                      prefill_tflops=dict(alone=flops_p / (alone_p * 1e-3) / 1e12, overlapped=flops_p / (ov_p * 1e-3) / 1e12),
-                      decode_gbs=dict(alone=bytes_d / (alone_d * 1e-3) / 1e9, overlapped=bytes_d / (ov_d * 1e-3) / 1e9),
-                      prefill_set=sm_set_summary(topo, plan_p), decode_set=sm_set_summary(topo, plan_d),
-                      note="decode time per GEMM includes the hand-over between back-to-back launches"), fh)
+            yield dict(config=5, split=list(split), partition=mode,
+                       prefill_tflops=dict(alone=flops_p / (alone_p * 1e-3) / 1e12, overlapped=flops_p / (ov_p * 1e-3) / 1e12),
+                       decode_gbs=dict(alone=bytes_d / (alone_d * 1e-3) / 1e9, overlapped=bytes_d / (ov_d * 1e-3) / 1e9),
+                       prefill_set=sm_set_summary(topo, plan_p), decode_set=sm_set_summary(topo, plan_d),
+                       note="decode time per GEMM includes the hand-over between back-to-back launches")
 
 
 # ---------------------------------------------------------------------------------------------
