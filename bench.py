@@ -632,6 +632,23 @@ def main():
     if sus_clocks.get("sm_mhz"):
         sustained["tflops_per_sm_ghz"] = sustained["tflops"] / (sus_clocks["sm_mhz"] / 1e3)
     rot_clocks = sampler.summary("rotation")
+    # The policies once more in burst state (the state `value` is measured in, where the kernel is bound by what the L2
+    # side delivers rather than by the power cap): every policy after its own idle pause, two rounds in opposite order.
+    burst = None
+    if args.only == "all":
+        burst_runs = {n: [] for n in ("oblivious_raster", "oblivious_grouped", "die_compact", "affinity")}
+        sampler.mark("burst_policies")
+        for order in (list(burst_runs), list(burst_runs)[::-1]):
+            for n in order:
+                torch.cuda.synchronize()
+                time.sleep(IDLE_BEFORE_TIMED_S)
+                b_ms, _, _ = timed(plans[n], 40, args.warmup, None)
+                burst_runs[n].append(FLOPS / (b_ms / 40 * 1e-3) / 1e12)
+        sampler.close("burst_policies")
+        burst = {"tflops": {n: float(np.mean(v)) for n, v in burst_runs.items()}, "runs": burst_runs,
+                 "steps_per_run": 40, "clocks": sampler.summary("burst_policies")}
+        burst["affinity_over_oblivious_raster"] = burst["tflops"]["affinity"] / burst["tflops"]["oblivious_raster"]
+        burst["affinity_over_oblivious_grouped"] = burst["tflops"]["affinity"] / burst["tflops"]["oblivious_grouped"]
 
     decode = decode_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
     attention = attention_section(ag, inputs, torch, topo, peaks, sampler) if args.only == "all" else None
@@ -706,6 +723,7 @@ def main():
                    "replicas": "independent per GPU" if world > 1 else "single GPU"},
         "policies_tflops": side,
         "policies_clocks": rot_clocks,
+        "policies_tflops_burst_state": burst,
         "policies_tflops_per_sm_ghz": ({n: v / (rot_clocks["sm_mhz"] / 1e3) for n, v in side.items()} if rot_clocks.get("sm_mhz") else None),
         "packed_b_group_free_bit": packed_b.group_free_bit(),
         "context_cublas_bf16_out_tflops_same_run": cublas_tflops,
