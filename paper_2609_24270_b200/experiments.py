@@ -395,6 +395,37 @@ def raster(fh, topo, traffic_only=False):
         emit(dict(config="raster", raster_group=g, policy=name, tflops=flops / (float(np.median(v)) * 1e-3) / 1e12), fh)
 
 
+def raster_burst(fh, topo, groups=(1, 2, 4, 6, 8, 12, 16, 32), steps=40, warmup=5, idle_s=2.0, runs=2):
+    """The raster-group sweep of the headline GEMM in burst state: every arm after its own idle pause, so that all of
+    its steps run at the full clock, where the kernel is bound by what the L2 side delivers and the order of the units
+    (and which die takes which) shows in the throughput."""
+    import time
+    M = N = K = 8192
+    A, B = inputs.gemm_inputs(M, N, K)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    flops = 2.0 * M * N * K
+
+    def burst(plan):
+        torch.cuda.synchronize()
+        time.sleep(idle_s)
+        for _ in range(warmup):
+            ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan)
+        e1.record()
+        torch.cuda.synchronize()
+        return flops / (e0.elapsed_time(e1) / steps * 1e-3) / 1e12
+
+    for kind, name in ((ag.AG_DIE_COMPACT, "die_compact"), (ag.AG_OBLIVIOUS, "oblivious")):
+        for g in groups:
+            plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=kind, M=M, N=N, K=K, tile_m=256, tile_n=256, raster_group=g))
+            emit(dict(config="raster_burst", policy=name, raster_group=g, tflops=[burst(plan) for _ in range(runs)]), fh)
+
+
 # ---------------------------------------------------------------------------------------------
 def time_queued(fn, warmup=3, iters=16, batches=3):
     """Median GPU time per call in ms.  The calls of a batch are queued behind a device-side blocker, so that
@@ -665,7 +696,7 @@ def main():
     {"3": config3, "4": config4, "5": config5, "raster": raster, "groupgemm": groupgemm, "groupgemm_dense": groupgemm_dense,
      "gpc_bandwidth": gpc_bandwidth, "latency": latency_histograms, "cluster_sets": cluster_sets, "attention": attention,
      "raster_traffic": lambda f, t: raster(f, t, traffic_only=True), "5_attention": config5_attention,
-     "attention_sweep": attention_sweep, "copy_ring": copy_ring}[args.config](fh, topo)
+     "attention_sweep": attention_sweep, "copy_ring": copy_ring, "raster_burst": raster_burst}[args.config](fh, topo)
 
 
 if __name__ == "__main__":
