@@ -448,7 +448,7 @@ def time_queued(fn, warmup=3, iters=16, batches=3):
     return float(np.median(out))
 
 
-def groupgemm(fh, topo, seeds=(1, 2)):
+def groupgemm(fh, topo, seeds=(1, 2, 3, 4, 5)):
     """The decode-shaped settings of the paper's GroupGEMM study (its workload appendix): (G, M) in
     {(32, 20), (6, 20)}, (N, K) in {(6144, 7168), (7168, 3072), (4096, 4096), (4096, 2048)}, rows per
     expert M_i = floor(M U_i), U_i ~ U(0.7, 1.3).  Random weights are made on the device (timing only;
