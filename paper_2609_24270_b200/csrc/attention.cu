@@ -908,10 +908,9 @@ extern "C" ag_status attention_decode_persistent(const void* Q, const ag_kv_cach
     if (!encode_a_slabs(&tm_q, Q, (uint64_t)B * H_q, AT_D, AT_NQ, 2)) return AG_ERR_CUDA;
     CUtensorMap tm0, tm1;
     if (kv->placement == 2) { tm0 = tm_q; tm1 = tm_q; } else { tm0 = kv->tm_quad[0]; tm1 = kv->tm_quad[1]; }
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(k_attn_decode, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);
+    static std::atomic<unsigned long long> attr_done{0};
+    const cudaError_t attr_err = once_per_device(attr_done, [] {
+        return cudaFuncSetAttribute(k_attn_decode, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
     AttnArgs x;

@@ -367,10 +367,9 @@ bool encode_a_slabs(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t K,
 template <int BN>
 static ag_status launch(const ag_plan* plan, const PersistParams& gp, cudaStream_t stream) {
     using C = Cfg<BN>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(k_gemm_persistent<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes);
+    static std::atomic<unsigned long long> attr_done{0};
+    const cudaError_t attr_err = once_per_device(attr_done, [] {
+        return cudaFuncSetAttribute(k_gemm_persistent<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes);
     });
     if (attr_err != cudaSuccess) return launch_failed(plan, attr_err);
     k_gemm_persistent<BN><<<plan->grid_blocks > 0 ? plan->grid_blocks : plan->lay.n_sm, D_THREADS, C::smem_bytes, stream>>>(plan->tm_a, plan->tm_b, plan->tm_c, gp);

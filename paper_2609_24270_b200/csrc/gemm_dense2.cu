@@ -430,12 +430,12 @@ ag_status gemm_pair_dispatch(const void* A, const void* B, const ag_packed_weigh
         if (!encode_2d(&plan->tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, M, N, 32, 32)) return AG_ERR_CUDA;
         plan->tm_a_ptr = A; plan->tm_b_ptr = b_key; plan->tm_c_ptr = Cout;
     }
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(k_gemm_persistent_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(k_gemm_persistent_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    static std::atomic<unsigned long long> attr_done{0};
+    const cudaError_t attr_err = once_per_device(attr_done, [] {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_persistent_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_gemm_persistent_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        return e;
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
     PersistParams gp = make_persist_params(plan, M, N, K);

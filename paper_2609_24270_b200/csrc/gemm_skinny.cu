@@ -729,11 +729,9 @@ __global__ void k_pack_weights(const uint16_t* __restrict__ B, int K, int N, int
 template <int NM, bool PACKED>
 static ag_status launch_skinny(const ag_plan* plan, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_w2,
                                const PersistParams& gp, const SkinnyArgs& x, cudaStream_t stream, bool may_start_early) {
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(k_gemm_skinny<NM, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        sk_smem_bytes(NM));
+    static std::atomic<unsigned long long> attr_done{0};
+    const cudaError_t attr_err = once_per_device(attr_done, [] {
+        return cudaFuncSetAttribute(k_gemm_skinny<NM, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, sk_smem_bytes(NM));
     });
     if (attr_err != cudaSuccess) return launch_failed(plan, attr_err);
     cudaLaunchConfig_t cfg;

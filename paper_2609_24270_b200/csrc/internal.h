@@ -131,6 +131,22 @@ extern std::atomic<unsigned long long> g_launch_count;
 inline void count_launch(int n = 1) { g_launch_count.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 ag_status check_arch();              // AG_OK on compute capability 10.x
 ag_status cuda_fail(cudaError_t e);  // records e, returns AG_ERR_CUDA (or AG_ERR_NOMEM)
+
+// Runs f (a set-up step that belongs to a device, such as a kernel's shared-memory attribute) the first time it is
+// reached with a given device current; `done` holds one bit per device.  Threads that race run f twice, which is
+// harmless for such steps.  Returns f's error (and tries again next time) or cudaSuccess.
+template <class F>
+inline cudaError_t once_per_device(std::atomic<unsigned long long>& done, F&& f) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return f();
+    const unsigned long long bit = 1ull << dev;
+    if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+    e = f();
+    if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
+    return e;
+}
 }  // namespace ag
 
 #define AG_CUDA(expr)                                         \

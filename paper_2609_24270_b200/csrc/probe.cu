@@ -19,7 +19,6 @@
 #include <string.h>
 
 #include <algorithm>
-#include <mutex>
 #include <new>
 #include <numeric>
 #include <vector>
@@ -417,16 +416,17 @@ ag_status warm_up(int n_sm, float* d_sink) {
 }
 
 ag_status set_pin_smem() {
-    static bool done = false;
-    if (done) return AG_OK;
-    AG_CUDA(cudaFuncSetAttribute(k_census, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-    AG_CUDA(cudaFuncSetAttribute(k_cluster_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-    AG_CUDA(cudaFuncSetAttribute(k_latency_from_sm, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-    AG_CUDA(cudaFuncSetAttribute(k_l2_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-    AG_CUDA(cudaFuncSetAttribute(k_affinity_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-    AG_CUDA(cudaFuncSetAttribute(k_die_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-    done = true;
-    return AG_OK;
+    static std::atomic<unsigned long long> done{0};
+    const cudaError_t e = once_per_device(done, [] {
+        cudaError_t r = cudaFuncSetAttribute(k_census, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem);
+        if (r == cudaSuccess) r = cudaFuncSetAttribute(k_cluster_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem);
+        if (r == cudaSuccess) r = cudaFuncSetAttribute(k_latency_from_sm, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem);
+        if (r == cudaSuccess) r = cudaFuncSetAttribute(k_l2_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem);
+        if (r == cudaSuccess) r = cudaFuncSetAttribute(k_affinity_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem);
+        if (r == cudaSuccess) r = cudaFuncSetAttribute(k_die_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem);
+        return r;
+    });
+    return e == cudaSuccess ? AG_OK : cuda_fail(e);
 }
 
 // aggregate L2 read bandwidth (bytes/s) of the SMs in `mask`, best of `tries`
@@ -964,11 +964,8 @@ extern "C" ag_status ag_probe_cluster_layout(int cluster_size, int n_clusters, i
     if (!cluster_of_sm || cluster_size < 2 || cluster_size > 8 || n_clusters < 1 || n_clusters * cluster_size > 4096) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
-    static bool attr_done = false;
-    if (!attr_done) {
-        AG_CUDA(cudaFuncSetAttribute(k_cluster_layout, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem));
-        attr_done = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};
+    AG_CUDA(once_per_device(attr_done, [] { return cudaFuncSetAttribute(k_cluster_layout, cudaFuncAttributeMaxDynamicSharedMemorySize, kPinSmem); }));
     const int grid = n_clusters * cluster_size;
     int* d_smid = nullptr;
     unsigned long long* d_start = nullptr;
@@ -1150,10 +1147,8 @@ extern "C" ag_status ag_probe_ring_bandwidth(const void* buf, size_t bytes, int 
     if (n_stages < 1) return AG_ERR_ARG;
     ag_status st = check_arch();
     if (st != AG_OK) return st;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] { attr_err = cudaFuncSetAttribute(k_ring_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    static std::atomic<unsigned long long> attr_done{0};
+    AG_CUDA(once_per_device(attr_done, [] { return cudaFuncSetAttribute(k_ring_bandwidth, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); }));
     unsigned long long* d_t = nullptr;
     int* d_err = nullptr;
     unsigned int* d_sink = nullptr;

@@ -636,3 +636,34 @@ def test_cluster_aware_sets_on_synthetic_b200():
                     assert not any(topo["is_random"][s] for s in S)
                 plan = op.build_plan(topo, None, b, pol)
                 check_invariants(topo, plan, pol, b)
+
+
+@pytest.mark.parametrize("seed,invert", [(1, 0), (2, 0), (3, 1), (4, 1)])
+def test_affinity_greedy_pass_keeps_a_full_dies_first_takers(seed, invert):
+    """What the greedy pass must amount to: until a die is full every unit gets the die it prefers, afterwards everything
+    goes to the other one; the quotas add up to the unit count, so at most one die has more takers than quota, and it
+    keeps exactly its first takers in the order (|margin| descending, raster index ascending)."""
+    topo = inputs.synthetic_topo(die0_sms=70, seed=seed)
+    M, N, K = 16, 128 * 300, 64
+    rng = np.random.default_rng(seed)
+    tbl = rng.integers(0, 2, size=M * N * 4 // 4096, dtype=np.uint8)
+    tbl[rng.random(tbl.size) < 0.3] = 0                      # more bytes on die 0 than its quota of units
+    amap = dict(chunk_bytes=4096, die_of_chunk=tbl)
+    pol = op.default_policy(kind=op.AFFINITY, M=M, N=N, K=K, tile_m=16, tile_n=128, raster_group=1, invert_affinity=invert,
+                            c=op.operand(0, N * 4, 4))
+    plan = op.build_plan(topo, amap, 148, pol)
+    n_u, q = plan["n_units"], plan["quotas"]
+    R = op.raster_order(1, 300, 1, 1)
+    die_of = {u: d for d in (0, 1) for u in plan["die_q"][d]}
+    takers = {0: [], 1: []}
+    for i, u in enumerate(R):
+        l0, l1 = op.unit_local_bytes(pol, amap, u)
+        m = (l1 - l0) if invert else (l0 - l1)
+        pref = 0 if m > 0 else 1 if m < 0 else op.band_die(i, n_u, q[0], 300)
+        takers[pref].append((-abs(m), i, u))
+    over = [d for d in (0, 1) if len(takers[d]) > q[d]]
+    assert len(over) == 1                                    # the case is built so that one die is oversubscribed
+    d = over[0]
+    kept = [u for _, _, u in sorted(takers[d])[:q[d]]]
+    assert sorted(plan["die_q"][d]) == sorted(kept)
+    assert all(die_of[u] == 1 - d for _, _, u in takers[1 - d])
