@@ -112,20 +112,22 @@ def test_two_stream_configuration_runs_both_gemms_correctly(partition):
     assert set(owner_p) <= set(taken) and not set(owner_d) & set(taken)     # each GEMM stayed on its own SMs
 
 
-@pytest.mark.parametrize("k_splits", [16, 4])
-@pytest.mark.parametrize("in_memory,overlap", [(1, 2), (0, 2), (1, 1)])
-def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap):
-    """M = 16, N = K = 8192 on all SMs with die-local packed weights, as timed: calls queued without a synchronisation
-    in between, rotating over four weight matrices, launches overlapping.  Every call writes a C of its own here, and
-    every one of them is compared with the oracle in full (a race between overlapping launches would show in some)."""
+@pytest.mark.parametrize("k_splits,in_memory,overlap,budget,spread",
+                         [(16, 1, 2, 0, 0), (16, 0, 2, 0, 0), (16, 1, 1, 0, 0), (4, 1, 2, 0, 0), (4, 0, 2, 0, 0), (4, 1, 1, 0, 0),
+                          (4, 1, 2, 74, 1), (4, 1, 2, 37, 1), (4, 1, 2, 74, 0), (4, 0, 1, 37, 0)])
+def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap, budget, spread):
+    """M = 16, N = K = 8192 with die-local packed weights, as timed - on all SMs and on 74 and 37 of them (whole TPCs over
+    both dies, or one die): calls queued without a synchronisation in between, rotating over four weight matrices,
+    launches overlapping.  Every call writes a C of its own here, and every one of them is compared with the oracle in
+    full (a race between overlapping launches would show in some)."""
     from tests.gpu_util import check_close as close
     M, N, K, n_buf, n_calls = 16, 8192, 8192, 4, 12
     topo = device_topo()
     A = inputs.uniform_bf16(M, K, inputs.DEFAULT_SEED)
     Bs = [inputs.uniform_bf16(K, N, inputs.DEFAULT_SEED + 1 + i) for i in range(n_buf)]
     dA, dBs = to_dev_bf16(A), [to_dev_bf16(b) for b in Bs]
-    plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128,
-                                                                k_splits=k_splits, splitk_in_memory=in_memory, overlap_launches=overlap))
+    plan = ag.sched_build(topo, None, budget or topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128, sm_select=spread,
+                                                                          k_splits=k_splits, splitk_in_memory=in_memory, overlap_launches=overlap))
     dst_bytes = 2 * K * N * 2 + (8 << 20)
     dsts = [torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_buf)]
     packs = []
@@ -141,6 +143,7 @@ def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap):
     assert plan.last_status() == ag.AG_OK
     owner, count = plan.tile_record()
     assert (count == n_calls).all()
+    assert set(owner.tolist()) <= set(plan.parsed()["sm_list"].tolist())
     want = [og.gemm_blocked(A, b) for b in Bs]
     for c in range(n_calls):
         close(dCs[c].cpu().numpy(), want[c % n_buf])
