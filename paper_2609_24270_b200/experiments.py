@@ -647,7 +647,7 @@ def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024), (16, 32, 
                           sm_set="gpc_spread" if both else "die_compact", sets=sm_set_summary(topo, plan), results=res,
                           local_fraction=info, local_over_remote=res["remote"]["us"] / res["local"]["us"],
                           local_over_interleaved=res["interleaved"]["us"] / res["local"]["us"],
-                          overlap_launches=int(bool(overlap and b == topo.n_sm)), library_sdpa_us=lib_us), fh)
+                          overlap_launches=int(bool(overlap)), library_sdpa_us=lib_us), fh)
         del dst, amap, dK, dV
         torch.cuda.empty_cache()
 
