@@ -413,6 +413,10 @@ ag_status ag_pack_weights(const void* B, int K, int N, const ag_plan* plan, cons
  * ag_pack_weights_ex - ag_pack_weights / ag_pack_weights_grouped with options (G = 1: B_list holds one matrix).
  *   flags  bit 0: keep the one-page-per-copy layout even where groups of four pages are possible.
  *          bit 1: always read the page tables in the kernel (do not use the closed form below).
+ *          bit 2: ignore the dies - logical page p goes to chunk p of dst (the hardware's interleaved placement; dst needs
+ *                 one chunk per page).  The page layout stays, a work unit's pages are one contiguous run, and the
+ *                 decode-shaped kernel fetches a stage with one plain copy.  The comparison arm for the die-local
+ *                 layout, and on the full chip the fastest way to stream the weights.
  * Closed form (Eq. 1 of the remapping appendix, page_phys = 2j + [parity((page_start + 2j) & MASK) xor P]): when the
  * measured map is an exact XOR hash over the chunks in use - in-page mask from ag_affinity_fit_hash, one further bit
  * per 2 MiB page, no chunk out of line - and the plan is decode-shaped, the pages of a work unit are consecutive in

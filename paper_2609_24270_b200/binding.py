@@ -494,11 +494,12 @@ class PackedWeights:
 
 
 def pack_weights(b_ptr: int, K: int, N: int, plan: Plan, amap: AffinityMap, dst_ptr: int, dst_bytes: int,
-                 single_pages: bool = False, tables_only: bool = False) -> PackedWeights:
+                 single_pages: bool = False, tables_only: bool = False, consecutive: bool = False) -> PackedWeights:
     h = C.c_void_p()
     bl = (C.c_void_p * 1)(b_ptr)
     _check(lib().ag_pack_weights_ex(bl, 1, K, N, plan.handle, amap.handle, dst_ptr, dst_bytes,
-                                    (1 if single_pages else 0) | (2 if tables_only else 0), C.byref(h)), "ag_pack_weights_ex")
+                                    (1 if single_pages else 0) | (2 if tables_only else 0) | (4 if consecutive else 0), C.byref(h)),
+           "ag_pack_weights_ex")
     return PackedWeights(h)
 
 
@@ -591,11 +592,11 @@ class GroupDesc:
 
 
 def pack_weights_grouped(b_ptrs, K: int, n_expert: int, plan: Plan, amap: AffinityMap, dst_ptr: int,
-                         dst_bytes: int, single_pages: bool = False) -> PackedWeights:
+                         dst_bytes: int, single_pages: bool = False, consecutive: bool = False) -> PackedWeights:
     bl = (C.c_void_p * len(b_ptrs))(*b_ptrs)
     h = C.c_void_p()
     _check(lib().ag_pack_weights_ex(bl, len(b_ptrs), K, n_expert, plan.handle, amap.handle, dst_ptr, dst_bytes,
-                                    1 if single_pages else 0, C.byref(h)), "ag_pack_weights_ex")
+                                    (1 if single_pages else 0) | (4 if consecutive else 0), C.byref(h)), "ag_pack_weights_ex")
     return PackedWeights(h)
 
 

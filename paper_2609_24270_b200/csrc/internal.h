@@ -97,6 +97,7 @@ struct ag_packed_weights {
     std::vector<int32_t> h_page_table;
     // Closed form of the page table (Eq. 1 of the remapping appendix): when the measured map is an exact XOR hash, the
     // chunk of a page follows from the page's position in its die's view, the fitted mask and one bit per 2 MiB page.
+    int consecutive;                     // 1: page p sits in chunk p (the placement that ignores the dies): a unit's pages are one contiguous run
     int closed_form;                     // 1: the kernels compute page addresses instead of reading the tables
     int k_splits;                        // k-splits of the plan the weights were packed for (a unit = one run of pages)
     uint32_t hash_mask;                  // fitted in-page mask (chunk-index bits 0..8)

@@ -136,7 +136,7 @@ def _config4(fh, topo, budgets, n_buffers, overlap, ksp):
         # the same budget taken as whole TPCs from the GPCs of both dies: each die then streams its own half of the
         # weights from its own memory, and the set uses the memory of both dies
         plan_spread = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, **kw))
-        dsts, packs, packs_single, packs_spread, packs_tables = [], [], [], [], []
+        dsts, packs, packs_single, packs_spread, packs_tables, packs_consec = [], [], [], [], [], []
         for i in range(n_buffers):                      # rotate buffers so that no launch finds its weights in L2
             dst2 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
             amap2 = ag.affinity_probe(dst2.data_ptr(), dst_bytes, topo)
@@ -151,6 +151,10 @@ def _config4(fh, topo, budgets, n_buffers, overlap, ksp):
             packs_tables.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap3, dst3.data_ptr(), dst_bytes,
                                                  tables_only=True), amap3))
             dsts.append(dst3)
+            dstc = torch.zeros(K * N * 2, dtype=torch.uint8, device="cuda")     # the same pages in consecutive chunks (dies ignored)
+            amapc = ag.affinity_probe(dstc.data_ptr(), K * N * 2, topo)
+            packs_consec.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amapc, dstc.data_ptr(), K * N * 2, consecutive=True), amapc))
+            dsts.append(dstc)
             dst1 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")   # same, one page per copy (for comparison)
             amap1 = ag.affinity_probe(dst1.data_ptr(), dst_bytes, topo)
             packs_single.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap1, dst1.data_ptr(), dst_bytes,
@@ -173,7 +177,9 @@ def _config4(fh, topo, budgets, n_buffers, overlap, ksp):
         for name, plan, pset in (("die_local", plan_local, packs), ("remote", plan_remote, packs),
                                  ("die_local_single_pages", plan_local, packs_single),
                                  ("die_local_page_tables", plan_local, packs_tables),
-                                 ("die_local_both_dies", plan_spread, packs_spread)):
+                                 ("die_local_both_dies", plan_spread, packs_spread),
+                                 ("pages_consecutive_oblivious", plan_obl, packs_consec),
+                                 ("pages_consecutive_die_compact", plan_local, packs_consec)):
             state = {"i": 0}
 
             def run():
@@ -197,7 +203,7 @@ def _config4(fh, topo, budgets, n_buffers, overlap, ksp):
                   pages_on_owner_die=on_die, page_group_free_bit=packs[0][0].group_free_bit(), closed_form=packs[0][0].closed_form(), local_set=sm_set_summary(topo, plan_local),
                   remote_set=sm_set_summary(topo, plan_remote), both_dies_set=sm_set_summary(topo, plan_spread), algo_bytes=algo_bytes,
                   hbm_peak_measured_gbs=6534.1), fh)
-        del packs, packs_single, packs_spread, packs_tables, dsts
+        del packs, packs_single, packs_spread, packs_tables, packs_consec, dsts
 
 
 def _unit_die(plan):

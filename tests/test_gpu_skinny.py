@@ -197,7 +197,7 @@ def oracle_page_table(packed, page_die, tbl, dst_ptr):
     return op.build_page_table_quads(page_die, amap, f, first=(dst_ptr // 4096) % 512)
 
 
-def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False, single_pages=False):
+def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False, single_pages=False, consecutive=False):
     topo = device_topo()
     b = topo.n_sm if b is None else b
     if integer:
@@ -210,7 +210,8 @@ def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False, single_pages=Fals
     dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dB = to_dev_bf16(B)
-    packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes, single_pages=single_pages)
+    packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes, single_pages=single_pages,
+                             consecutive=consecutive)
     return topo, A, B, kw, plan_d, dst, amap, packed
 
 
@@ -234,6 +235,36 @@ def test_packing_matches_oracle_table_and_layout(single_pages):
     want_img = op.pack_weights(B, want_table, n_chunks)
     got_img = dst[: n_chunks * 4096].cpu().numpy().view(np.uint16).reshape(n_chunks, 2048)
     assert np.array_equal(got_img, want_img)
+
+
+@pytest.mark.parametrize("M,N,K,ksp,b", [(16, 1024, 1024, 1, None), (16, 2048, 2048, 4, None), (32, 1024, 512, 2, None), (9, 1096, 256, 1, None),
+                                        (16, 2048, 4096 + 64, 3, 37), (64, 1024, 1024, 2, None), (128, 1024, 512, 1, 74)])
+def test_packed_weights_in_consecutive_chunks(M, N, K, ksp, b):
+    """The placement that ignores the dies: logical page p in chunk p (the page image is the oracle's for the identity
+    table), a stage fetched with one plain copy; the GEMM over it is exact on integer inputs."""
+    topo = device_topo()
+    A, B = inputs.small_int_bf16(M, K, 77), inputs.small_int_bf16(K, N, 78)
+    kw = dict(M=M, N=N, K=K, tile_m=16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128, tile_n=128, k_splits=ksp,
+              decode_shaped=1 if M > 64 else 0)
+    plan = ag.sched_build(topo, None, b or topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
+    n_pages = ((N + 127) // 128) * (K // 16)
+    dst_bytes = n_pages * 4096
+    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+    packed = ag.pack_weights(to_dev_bf16(B).data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes, consecutive=True)
+    assert packed.group_free_bit() < 0 and not packed.closed_form()["enabled"]
+    table = packed.page_table()
+    assert np.array_equal(table, np.arange(n_pages, dtype=np.int32))
+    if N % 128 == 0:
+        want_img = op.pack_weights(B, table.tolist(), n_pages)
+        assert np.array_equal(dst.cpu().numpy().view(np.uint16).reshape(n_pages, 2048), want_img)
+    dA = to_dev_bf16(A)
+    dC = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan)
+        torch.cuda.synchronize()
+        assert plan.last_status() == ag.AG_OK
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), og.gemm_blocked(A, B))
 
 
 @pytest.mark.parametrize("M,N,K,ksp", [(16, 1024, 1024, 1), (16, 2048, 2048, 4), (32, 1024, 512, 2), (9, 1096, 256, 1)])
