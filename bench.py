@@ -337,6 +337,8 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
             "clocks": sampler.summary("decode"),
             "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
                          "frac_4_k_splits": results[4]["packed_die_local"] / peaks["hbm_gbs"],
+                         "best_arm": dict(zip(("k_splits", "arm", "gbs"), max(((k, n, v) for k in results for n, v in results[k].items()),
+                                                                               key=lambda t: t[2]))),
                          "traffic": NCU_TRAFFIC_BYTES_DECODE, "kernel": "k_gemm_skinny<16, packed>", "algorithmic_bytes": algo_bytes,
                          "peak_source": f"{peaks['source']} copy bandwidth"}}
 
