@@ -290,7 +290,8 @@ typedef struct {
                                 memory (2..6, clamped to what the kernel has; even for up to 32 activation rows).  0 =
                                 default: attention decode shares 20 MiB between the plan's SMs (4 stages on the full
                                 chip, where more in flight oversubscribes the memory system; 6 on half of it), the
-                                decode-shaped GEMM uses all its stages */
+                                decode-shaped GEMM uses all its stages, except four for units of at most 128 KB of
+                                row-major weights or of pages in consecutive chunks */
     uint64_t avoid_sm_mask[4]; /* bit s set: SM s belongs to another plan */
     ag_operand_desc a, b, c;
 } ag_policy;

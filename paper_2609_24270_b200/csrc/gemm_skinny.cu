@@ -838,6 +838,13 @@ ag_status gemm_skinny_dispatch(const void* A, const void* B_rowmajor, const ag_p
     x.release_next = overlap ? 1 : 0;
     x.a_after_prior = (overlap && plan->policy.overlap_launches != 2) ? 1 : 0;
     x.stages = ring_stages_for(plan, sk_stages(NM), std::min(sk_stages(NM), 2), sk_nmma(NM) == 2, false);
+    // Units of at most four stages (128 KB of weights, e.g. N = K = 8192 in 16 k-splits) of row-major weights or of pages in
+    // consecutive chunks: a ring of four stages streams 5-6 % more than one of six on the full chip (6.13-6.20 against 5.79-5.83 TB/s) and the same on 37 and 74 SMs; with longer
+    // units the deeper ring wins (4 k-splits: 6.81-6.84 against 6.63-6.64 TB/s).
+    // Die-local pages are the exception (16 k-splits: 6.11-6.14 TB/s with six stages against 5.88-5.94 with four).
+    if (plan->policy.ring_stages <= 0 && sk_stages(NM) == SK_STAGES && (plan->kslabs_per_split + SK_SLABS - 1) / SK_SLABS <= 4 &&
+        (!W || W->consecutive))
+        x.stages = 4;
     x.producers = x.stages % 3 == 0 ? 3 : x.stages % 2 == 0 ? 2 : sk_nmma(NM) == 1 ? std::min(3, x.stages) : 1;
     if (zeroing) {  // in-memory reduction mode: the adds need a zeroed C (N % 8 == 0 and 16-byte alignment: whole float4s)
         const size_t c_elems = grp ? (size_t)grp->total_rows * (size_t)grp->N : (size_t)M * (size_t)N;
