@@ -112,12 +112,13 @@ def test_two_stream_configuration_runs_both_gemms_correctly(partition):
     assert set(owner_p) <= set(taken) and not set(owner_d) & set(taken)     # each GEMM stayed on its own SMs
 
 
-@pytest.mark.parametrize("k_splits,in_memory,overlap,budget,spread",
-                         [(16, 1, 2, 0, 0), (16, 0, 2, 0, 0), (16, 1, 1, 0, 0), (4, 1, 2, 0, 0), (4, 0, 2, 0, 0), (4, 1, 1, 0, 0),
-                          (4, 1, 2, 74, 1), (4, 1, 2, 37, 1), (4, 1, 2, 74, 0), (4, 0, 1, 37, 0)])
-def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap, budget, spread):
-    """M = 16, N = K = 8192 with die-local packed weights, as timed - on all SMs and on 74 and 37 of them (whole TPCs over
-    both dies, or one die): calls queued without a synchronisation in between, rotating over four weight matrices,
+@pytest.mark.parametrize("k_splits,in_memory,overlap,budget,spread,consecutive",
+                         [(16, 1, 2, 0, 0, 0), (16, 0, 2, 0, 0, 0), (16, 1, 1, 0, 0, 0), (4, 1, 2, 0, 0, 0), (4, 0, 2, 0, 0, 0), (4, 1, 1, 0, 0, 0),
+                          (4, 1, 2, 74, 1, 0), (4, 1, 2, 37, 1, 0), (4, 1, 2, 74, 0, 0), (4, 0, 1, 37, 0, 0),
+                          (16, 1, 2, 0, 0, 1), (4, 1, 2, 0, 0, 1), (4, 1, 2, 74, 0, 1)])
+def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap, budget, spread, consecutive):
+    """M = 16, N = K = 8192 with die-local packed weights (or the same pages in consecutive chunks), as timed - on all SMs
+    and on 74 and 37 of them (whole TPCs over both dies, or one die): calls queued without a synchronisation in between, rotating over four weight matrices,
     launches overlapping.  Every call writes a C of its own here, and every one of them is compared with the oracle in
     full (a race between overlapping launches would show in some)."""
     from tests.gpu_util import check_close as close
@@ -133,7 +134,7 @@ def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap, 
     packs = []
     for i in range(n_buf):
         amap = ag.affinity_probe(dsts[i].data_ptr(), dst_bytes, topo)
-        packs.append(ag.pack_weights(dBs[i].data_ptr(), K, N, plan, amap, dsts[i].data_ptr(), dst_bytes))
+        packs.append(ag.pack_weights(dBs[i].data_ptr(), K, N, plan, amap, dsts[i].data_ptr(), dst_bytes, consecutive=bool(consecutive)))
     dCs = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(n_calls)]
     torch.cuda.synchronize()
     plan.reset_record()
