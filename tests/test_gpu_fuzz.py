@@ -47,3 +47,49 @@ def test_random_case(case):
     assert np.array_equal(C.astype(np.float64), og.gemm_blocked(A, B)), kw
     _, count = plan.tile_record()
     assert (count == 1).all()
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_affinity_plan(case):
+    """Affinity plans over random chunk-to-die tables: random shapes, operands present or not, margins clipped or not,
+    inverted or not, either quota rule, any budget - bytewise equal to the oracle's (the CUDA builder finds the full
+    die's cut by a radix select, the oracle sorts)."""
+    rng = np.random.default_rng(5000 + case)
+    topo = inputs.synthetic_topo(die0_sms=int(rng.choice([70, 72, 74])), seed=case)
+    M = int(rng.integers(1, 1100))
+    N = int(rng.integers(1, 160)) * 8
+    K = int(rng.integers(1, 130)) * 8
+    tile_m, tile_n = int(rng.choice([16, 128])), int(rng.choice([64, 128, 256]))
+    n_slab = -(-K // 64)
+    ksp = int(rng.integers(1, min(4, n_slab) + 1))
+    per = -(-n_slab // ksp)
+    if (ksp - 1) * per >= n_slab:
+        ksp = 1
+    a_off, b_off, c_off = 0, M * K * 2, M * K * 2 + K * N * 2
+    nbytes = c_off + M * N * 4
+    n_chunks = -(-nbytes // 4096) + 1
+    style = case % 3
+    if style == 0:
+        tbl = rng.integers(0, 2, size=n_chunks, dtype=np.uint8)            # noise: every margin differs
+    elif style == 1:
+        tbl = inputs.synthetic_chunk_die(n_chunks, seed=case).copy()        # XOR hash: many exact ties
+        tbl[:: int(rng.integers(3, 9))] = int(rng.integers(0, 2))
+    else:
+        tbl = (np.arange(n_chunks) // int(rng.integers(1, 64)) % 2).astype(np.uint8)   # long runs: one die oversubscribed
+    present = rng.integers(0, 2, size=3)
+    if not present.any():
+        present[int(rng.integers(0, 3))] = 1
+    ops = {}
+    if present[0]:
+        ops["a"] = dict(offset=a_off, row_stride=K * 2, elem_bytes=2)
+    if present[1]:
+        ops["b"] = dict(offset=b_off, row_stride=N * 2, elem_bytes=2)
+    if present[2]:
+        ops["c"] = dict(offset=c_off, row_stride=N * 4, elem_bytes=4)
+    kw = dict(kind=ag.AG_AFFINITY, M=M, N=N, K=K, tile_m=tile_m, tile_n=tile_n, k_splits=ksp, raster_group=int(rng.integers(1, 9)),
+              invert_affinity=int(rng.integers(0, 2)), min_margin=int(rng.choice([0, 0, 512, 4096, 1 << 16])),
+              die_quota=int(rng.integers(0, 2)), **ops)
+    b = int(rng.integers(1, 149))
+    plan = ag.sched_build(ag.TopoMap.from_dict(topo), ag.affinity_from_table(0, tbl), b, ag.make_policy(**kw))
+    want = op.export(op.build_plan(topo, dict(chunk_bytes=4096, die_of_chunk=tbl), b, oracle_policy(**kw)))
+    assert plan.export().tobytes() == want.tobytes(), (kw, b)
