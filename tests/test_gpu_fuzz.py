@@ -93,3 +93,51 @@ def test_random_affinity_plan(case):
     plan = ag.sched_build(ag.TopoMap.from_dict(topo), ag.affinity_from_table(0, tbl), b, ag.make_policy(**kw))
     want = op.export(op.build_plan(topo, dict(chunk_bytes=4096, die_of_chunk=tbl), b, oracle_policy(**kw)))
     assert plan.export().tobytes() == want.tobytes(), (kw, b)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_decode_shaped_case(case):
+    """The decode-shaped kernel over random shapes: 1 to 128 activation rows, row-major weights, die-local pages (groups or
+    single pages) or pages in consecutive chunks, both split-K modes, any SM budget, launches overlapping or not; three
+    calls queued back to back, exact on integer inputs."""
+    rng = np.random.default_rng(9000 + case)
+    topo = device_topo()
+    M = int(rng.choice([1, 7, 16, 17, 32, 33, 64, 100, 128]))
+    layout = int(rng.integers(0, 4))                          # 0 row-major, 1 die-local groups, 2 die-local single pages, 3 consecutive
+    N = int(rng.integers(1, 40)) * (128 if layout else 8)
+    K = int(rng.integers(1, 40)) * (64 if layout else 8)
+    n_slab = -(-K // 64)
+    ksp = int(rng.integers(1, min(6, n_slab) + 1))
+    per = -(-n_slab // ksp)
+    if (ksp - 1) * per >= n_slab:
+        ksp = 1
+    tile_m = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128
+    kw = dict(kind=int(rng.choice([ag.AG_OBLIVIOUS, ag.AG_DIE_COMPACT])), M=M, N=N, K=K, tile_m=tile_m, tile_n=128, k_splits=ksp,
+              splitk_in_memory=int(rng.integers(0, 2)), overlap_launches=int(rng.integers(0, 3)), decode_shaped=1 if M > 64 else 0,
+              sm_select=int(rng.integers(0, 2)), static_assign=1)
+    b = int(rng.integers(1, topo.n_sm + 1))
+    plan = ag.sched_build(topo, None, b, ag.make_policy(**kw))
+    A, B = inputs.small_int_bf16(M, K, 300 + case), inputs.small_int_bf16(K, N, 400 + case)
+    dA, dB = torch.from_numpy(A.view(np.int16).copy()).cuda(), torch.from_numpy(B.view(np.int16).copy()).cuda()
+    dCs = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+    packed = None
+    if layout:
+        n_pages = (N // 128) * (K // 16)
+        dst_bytes = n_pages * 4096 * (1 if layout == 3 else 2) + (8 << 20)
+        raw = torch.zeros(dst_bytes + 4096, dtype=torch.uint8, device="cuda")     # (a cached block may start off a 4 KB boundary)
+        dst = raw[(-raw.data_ptr()) % 4096:][:dst_bytes]
+        amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
+        packed = ag.pack_weights(dB.data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes, single_pages=layout == 2, consecutive=layout == 3)
+    plan.reset_record()
+    for dC in dCs:
+        if packed is not None:
+            ag.gemm_persistent_packed(dA.data_ptr(), packed, dC.data_ptr(), M, N, K, plan)
+        else:
+            ag.gemm_persistent(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, plan)
+    torch.cuda.synchronize()
+    assert plan.last_status() == ag.AG_OK, (kw, b, layout, plan.last_status_where())
+    want = og.gemm_blocked(A, B)
+    for dC in dCs:
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), want), (kw, b, layout)
+    _, count = plan.tile_record()
+    assert (count == 3).all()
