@@ -205,9 +205,9 @@ def decode_section(ag, inputs, torch, topo, peaks, sampler):
     dC = torch.empty((Md, Nd), dtype=torch.float32, device="cuda")
     algo_bytes = Kd * Nd * 2 + Md * Kd * 2 + Md * Nd * 4
     dst_bytes = 2 * Kd * Nd * 2 + (8 << 20)
-    dsts = [torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_buf)]
+    dsts = [ag.aligned_device_bytes(dst_bytes) for _ in range(n_buf)]
     amaps = [ag.affinity_probe(d.data_ptr(), dst_bytes, topo) for d in dsts]
-    dsts_c = [torch.zeros(Kd * Nd * 2, dtype=torch.uint8, device="cuda") for _ in range(n_buf)]
+    dsts_c = [ag.aligned_device_bytes(Kd * Nd * 2) for _ in range(n_buf)]
     amaps_c = [ag.affinity_probe(d.data_ptr(), Kd * Nd * 2, topo) for d in dsts_c]
     want = og.gemm_blocked(A_bits, B_bits[0])
     launches0 = ag.kernel_launch_count()
@@ -361,7 +361,7 @@ def attention_section(ag, inputs, torch, topo, peaks, sampler):
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=Hq // Hkv, N=128 * B * Hkv, K=L, tile_m=16,
                                                                tile_n=128, k_splits=1, overlap_launches=1))
     dst_bytes = 2 * kv_bytes + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     want = oa.gqa_decode(Q[:8], K[:8], V[:8])
     gbs, err, frac_local, launches0 = {}, {}, {}, ag.kernel_launch_count()
@@ -506,8 +506,7 @@ def main():
     # ---- inputs: one buffer holds A, B and C so that one affinity map covers all three
     A_h, B_h = inputs.gemm_inputs(M, N, K)
     a_bytes, b_bytes, c_bytes = M * K * 2, K * N * 2, M * N * 4
-    buf = torch.empty(a_bytes + b_bytes + c_bytes, dtype=torch.uint8, device="cuda")
-    assert buf.data_ptr() % 4096 == 0
+    buf = ag.aligned_device_bytes(a_bytes + b_bytes + c_bytes)
     a_off, b_off, c_off = 0, a_bytes, a_bytes + b_bytes
     dA = buf[a_off:a_off + a_bytes].view(torch.int16).view(M, K)
     dB = buf[b_off:b_off + b_bytes].view(torch.int16).view(K, N)
@@ -554,7 +553,7 @@ def main():
     # chunks of that die; the affinity policy then has real margins (B panel bytes) instead of ties
     t0 = time.time()
     pk_bytes = 2 * b_bytes + (8 << 20)
-    pk_buf = torch.zeros(pk_bytes, dtype=torch.uint8, device="cuda")
+    pk_buf = ag.aligned_device_bytes(pk_bytes)
     pk_amap = ag.affinity_probe(pk_buf.data_ptr(), pk_bytes, topo)
     packed_b = ag.pack_weights(dB.data_ptr(), K, N, plans["die_compact"], pk_amap, pk_buf.data_ptr(), pk_bytes)
     paged = dict(offset=0, row_stride=0, elem_bytes=2, layout=ag.AG_LAYOUT_PAGED, page_table=packed_b.page_table())

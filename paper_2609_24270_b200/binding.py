@@ -307,6 +307,14 @@ def probe_ring_bandwidth(dev_ptr: int, nbytes: int, n_blocks: int, stages: int, 
     return out.value
 
 
+def aligned_device_bytes(nbytes: int):
+    """A zeroed uint8 torch tensor of nbytes on the current CUDA device that starts on a 4096-byte boundary, as buffers that
+    are probed or packed into must (a block handed out by torch's caching allocator may start off one)."""
+    import torch
+    raw = torch.zeros(nbytes + AG_CHUNK_BYTES, dtype=torch.uint8, device="cuda")
+    return raw[(-raw.data_ptr()) % AG_CHUNK_BYTES:][:nbytes]
+
+
 def affinity_probe(dev_ptr: int, nbytes: int, topo: TopoMap | None = None) -> AffinityMap:
     h = C.c_void_p()
     if topo is None:

@@ -138,24 +138,24 @@ def _config4(fh, topo, budgets, n_buffers, overlap, ksp):
         plan_spread = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, sm_select=1, **kw))
         dsts, packs, packs_single, packs_spread, packs_tables, packs_consec = [], [], [], [], [], []
         for i in range(n_buffers):                      # rotate buffers so that no launch finds its weights in L2
-            dst2 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            dst2 = ag.aligned_device_bytes(dst_bytes)
             amap2 = ag.affinity_probe(dst2.data_ptr(), dst_bytes, topo)
             packs_spread.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_spread, amap2, dst2.data_ptr(), dst_bytes), amap2))
             dsts.append(dst2)
-            dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            dst = ag.aligned_device_bytes(dst_bytes)
             amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
             packs.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap, dst.data_ptr(), dst_bytes), amap))
             dsts.append(dst)
-            dst3 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")   # same layout, page addresses from tables
+            dst3 = ag.aligned_device_bytes(dst_bytes)   # same layout, page addresses from tables
             amap3 = ag.affinity_probe(dst3.data_ptr(), dst_bytes, topo)
             packs_tables.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap3, dst3.data_ptr(), dst_bytes,
                                                  tables_only=True), amap3))
             dsts.append(dst3)
-            dstc = torch.zeros(K * N * 2, dtype=torch.uint8, device="cuda")     # the same pages in consecutive chunks (dies ignored)
+            dstc = ag.aligned_device_bytes(K * N * 2)     # the same pages in consecutive chunks (dies ignored)
             amapc = ag.affinity_probe(dstc.data_ptr(), K * N * 2, topo)
             packs_consec.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amapc, dstc.data_ptr(), K * N * 2, consecutive=True), amapc))
             dsts.append(dstc)
-            dst1 = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")   # same, one page per copy (for comparison)
+            dst1 = ag.aligned_device_bytes(dst_bytes)   # same, one page per copy (for comparison)
             amap1 = ag.affinity_probe(dst1.data_ptr(), dst_bytes, topo)
             packs_single.append((ag.pack_weights(Bs[i].data_ptr(), K, N, plan_local, amap1, dst1.data_ptr(), dst_bytes,
                                                  single_pages=True), amap1))
@@ -306,7 +306,7 @@ def config5_attention(fh, topo):
     kv_bytes = 2 * B * Hkv * L * D * 2
     algo = kv_bytes + B * Hq * D * 6
     dst_bytes = 2 * kv_bytes + (16 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     flops_p = 2.0 * Mp * N * K
@@ -468,7 +468,7 @@ def groupgemm(fh, topo, seeds=(1, 2, 3, 4, 5)):
             Bs = [torch.randn((K, N), dtype=torch.bfloat16, device="cuda") for _ in range(G)]
             w_bytes = G * K * N * 2
             dst_bytes = 2 * w_bytes + (16 << 20)
-            dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            dst = ag.aligned_device_bytes(dst_bytes)
             amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
             for seed in seeds:
                 rows = inputs.group_rows(G, M, seed)
@@ -483,7 +483,7 @@ def groupgemm(fh, topo, seeds=(1, 2, 3, 4, 5)):
                 plan_rem = ag.sched_build(topo, amap, topo.n_sm, ag.make_policy(kind=ag.AG_AFFINITY, invert_affinity=1, b=bop, **kw))
                 # the units shared equally between the dies instead of by SM count (each die's memory is equally fast)
                 plan_eq = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, die_quota=1, **kw))
-                dst_eq = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+                dst_eq = ag.aligned_device_bytes(dst_bytes)
                 amap_eq = ag.affinity_probe(dst_eq.data_ptr(), dst_bytes, topo)
                 packed_eq = ag.pack_weights_grouped([b.data_ptr() for b in Bs], K, N, plan_eq, amap_eq, dst_eq.data_ptr(), dst_bytes)
                 desc_rm = ag.GroupDesc(dA.data_ptr(), dC.data_ptr(), rows, [b.data_ptr() for b in Bs], N, K, 32)
@@ -511,7 +511,7 @@ def groupgemm_dense(fh, topo, seeds=(1,)):
             Bs = [torch.randn((K, N), dtype=torch.bfloat16, device="cuda") for _ in range(G)]
             w_bytes = G * K * N * 2
             dst_bytes = 2 * w_bytes + (16 << 20)
-            dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+            dst = ag.aligned_device_bytes(dst_bytes)
             amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
             for seed in seeds:
                 rows = inputs.group_rows(G, M, seed)
@@ -624,7 +624,7 @@ def attention(fh, topo, shapes=((128, 32, 8, 512), (256, 32, 8, 1024), (16, 32, 
         kv_bytes = 2 * B * Hkv * L * D * 2
         algo = kv_bytes + B * Hq * D * (2 + 4)
         dst_bytes = 2 * kv_bytes + (16 << 20)
-        dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+        dst = ag.aligned_device_bytes(dst_bytes)
         amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
         lib_us = None
         try:    # context: the library's fused attention on the same shapes (row-major cache)
@@ -676,7 +676,7 @@ def copy_ring(fh, topo):
     """What sets policy.ring_stages: the copy side of the streaming kernels alone (rings of 32 KB stages filled by bulk
     copies) on 1, 37, 74 and all SMs, over the ring depth, the stage size and the time a stage is held."""
     nbytes = 4 << 30
-    buf = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    buf = ag.aligned_device_bytes(nbytes)
     for n_blocks in (1, 37, 74, topo.n_sm):
         share = nbytes if n_blocks > 1 else 256 << 20
         for stage_bytes, depths in ((32768, (1, 2, 3, 4, 5, 6)), (16384, (2, 4, 8)), (65536, (1, 2, 3))):

@@ -41,7 +41,7 @@ def run_attention(Q, K, V, placement, kv_len=None, budget=None, overlap=0):
                                                         tile_n=128, k_splits=1, overlap_launches=overlap))
     kv_bytes = 2 * B * Hkv * L * D * 2
     dst_bytes = (2 * kv_bytes if placement != ag.KV_INTERLEAVED else kv_bytes) + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dK, dV, dQ = dev(K), dev(V), dev(Q)
     kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes, placement)
@@ -134,7 +134,7 @@ def test_appended_tokens_land_where_packing_would_put_them():
                                                                tile_n=128, k_splits=1))
     kv_bytes = 2 * B * Hkv * L * 128 * 2
     dst_bytes = 2 * kv_bytes + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     start = np.array([0, 5, 127, 200, 380], dtype=np.int32)          # keys that every request already has
     K0, V0 = K.copy(), V.copy()
@@ -204,7 +204,7 @@ def test_bad_arguments():
     topo = device_topo()
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=4, N=128 * 8, K=256, tile_m=16,
                                                                 tile_n=128, k_splits=1))
-    dst = torch.zeros(16 << 20, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(16 << 20)
     amap = ag.affinity_probe(dst.data_ptr(), dst.numel(), topo)
     k = torch.zeros(8 * 256 * 128, dtype=torch.int16, device="cuda")
     h = ag.C.c_void_p()

@@ -130,7 +130,7 @@ def test_decode_configuration_queued_back_to_back(k_splits, in_memory, overlap, 
     plan = ag.sched_build(topo, None, budget or topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=M, N=N, K=K, tile_m=16, tile_n=128, sm_select=spread,
                                                                           k_splits=k_splits, splitk_in_memory=in_memory, overlap_launches=overlap))
     dst_bytes = 2 * K * N * 2 + (8 << 20)
-    dsts = [torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_buf)]
+    dsts = [ag.aligned_device_bytes(dst_bytes) for _ in range(n_buf)]
     packs = []
     for i in range(n_buf):
         amap = ag.affinity_probe(dsts[i].data_ptr(), dst_bytes, topo)
@@ -168,7 +168,7 @@ def test_attention_configuration_queued_back_to_back(placement):
                                                                 tile_n=128, k_splits=1, overlap_launches=1))
     kv_bytes = 2 * B * Hkv * L * D * 2
     dst_bytes = 2 * kv_bytes + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes,
                     ag.KV_LOCAL if placement == "local" else ag.KV_INTERLEAVED)

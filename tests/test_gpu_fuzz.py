@@ -124,8 +124,7 @@ def test_random_decode_shaped_case(case):
     if layout:
         n_pages = (N // 128) * (K // 16)
         dst_bytes = n_pages * 4096 * (1 if layout == 3 else 2) + (8 << 20)
-        raw = torch.zeros(dst_bytes + 4096, dtype=torch.uint8, device="cuda")     # (a cached block may start off a 4 KB boundary)
-        dst = raw[(-raw.data_ptr()) % 4096:][:dst_bytes]
+        dst = ag.aligned_device_bytes(dst_bytes)
         amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
         packed = ag.pack_weights(dB.data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes, single_pages=layout == 2, consecutive=layout == 3)
     plan.reset_record()

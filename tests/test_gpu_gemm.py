@@ -203,7 +203,7 @@ def packed_dense_setup(M, N, K, raster_group=2, integer=True, seed=51):
     kw = dict(M=M, N=N, K=K, tile_m=256, tile_n=256, raster_group=raster_group, pair_lists=1)
     plan_d = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
     dst_bytes = 2 * K * ((N + 255) // 256 * 256) * 2 + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dB = to_dev_bf16(B)
     packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes)

@@ -64,7 +64,7 @@ def test_grouped_packed_weights_sit_on_the_experts_die_and_match_oracle():
     kw = dict(M=int(rows.max()), N=G * N, K=K, tile_m=32, tile_n=128, k_splits=ksp, splitk_in_memory=1)
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
     dst_bytes = 2 * G * K * N * 2 + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dBs = [to_dev_bf16(b) for b in Bs]
     packed = ag.pack_weights_grouped([b.data_ptr() for b in dBs], K, N, plan, amap, dst.data_ptr(), dst_bytes)
@@ -165,7 +165,7 @@ def test_grouped_dense_over_packed_weights():
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, M=int(rows.max()), N=G * N, K=K,
                                                                 tile_m=256, tile_n=256))
     dst_bytes = 2 * G * K * N * 2 + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dBs = [to_dev_bf16(b) for b in Bs]
     packed = ag.pack_weights_grouped([b.data_ptr() for b in dBs], K, N, plan, amap, dst.data_ptr(), dst_bytes)

@@ -138,7 +138,7 @@ def test_request_of_a_million_keys():
                                                                 tile_m=16, tile_n=128, k_splits=1))
     kv_bytes = 2 * B * Hkv * L * D * 2
     dst_bytes = kv_bytes + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dK, dV, dQ = to_dev_bf16(K.reshape(-1, D)), to_dev_bf16(V.reshape(-1, D)), to_dev_bf16(Q.reshape(-1, D))
     kv = ag.kv_pack(dK.data_ptr(), dV.data_ptr(), B, Hkv, L, plan, amap, dst.data_ptr(), dst_bytes, ag.KV_INTERLEAVED)

@@ -69,7 +69,7 @@ def test_up_to_128_activation_rows_integer_exact(M, tile_m, k_splits, in_memory)
         for _ in range(2):
             assert np.array_equal(run_rowmajor(A, B, plan).astype(np.float64), want)
     dst_bytes = 2 * K * N * 2 + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dA, dB = to_dev_bf16(A), to_dev_bf16(B)
     packed = ag.pack_weights(dB.data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes)
@@ -207,7 +207,7 @@ def packed_setup(M, N, K, ksp, b=None, seed=41, integer=False, single_pages=Fals
     kw = dict(M=M, N=N, K=K, tile_m=16 if M <= 16 else 32, tile_n=128, k_splits=ksp)
     plan_d = ag.sched_build(topo, None, b, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
     dst_bytes = 2 * K * N * 2 + (8 << 20)                    # two views, head-room for an uneven die split
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     dB = to_dev_bf16(B)
     packed = ag.pack_weights(dB.data_ptr(), K, N, plan_d, amap, dst.data_ptr(), dst_bytes, single_pages=single_pages,
@@ -249,7 +249,7 @@ def test_packed_weights_in_consecutive_chunks(M, N, K, ksp, b):
     plan = ag.sched_build(topo, None, b or topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
     n_pages = ((N + 127) // 128) * (K // 16)
     dst_bytes = n_pages * 4096
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     amap = ag.affinity_probe(dst.data_ptr(), dst_bytes, topo)
     packed = ag.pack_weights(to_dev_bf16(B).data_ptr(), K, N, plan, amap, dst.data_ptr(), dst_bytes, consecutive=True)
     assert packed.group_free_bit() < 0 and not packed.closed_form()["enabled"]
@@ -313,7 +313,7 @@ def test_closed_form_remap_on_a_synthetic_hash(mask_bits, want_free_bit):
     kw = dict(M=M, N=N, K=K, tile_m=16, tile_n=128, k_splits=ksp)
     plan = ag.sched_build(topo, None, topo.n_sm, ag.make_policy(kind=ag.AG_DIE_COMPACT, **kw))
     dst_bytes = 2 * K * N * 2 + (8 << 20)
-    dst = torch.zeros(dst_bytes, dtype=torch.uint8, device="cuda")
+    dst = ag.aligned_device_bytes(dst_bytes)
     assert dst.data_ptr() % (2 << 20) == 0
     doc = inputs.synthetic_chunk_die(dst_bytes // 4096, seed=13, mask_bits=mask_bits)
     amap = ag.affinity_from_table(dst.data_ptr(), doc)
@@ -363,7 +363,7 @@ def test_closed_form_remap_on_the_measured_map():
 
 def test_packed_rejects_foreign_map_and_shapes():
     topo, A, B, kw, plan_d, dst, amap, packed = packed_setup(16, 512, 256, 1)
-    other = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    other = ag.aligned_device_bytes(1 << 20)
     h = ag.C.c_void_p()
     st = ag.lib().ag_pack_weights(to_dev_bf16(B).data_ptr(), 256, 512, plan_d.handle, amap.handle, other.data_ptr(),
                                   other.numel(), ag.C.byref(h))

@@ -91,7 +91,7 @@ def test_affinity_probe_structure_and_content_preserved(topo):
 def test_local_bandwidth_beats_remote(topo):
     """Section 6.2.1: remote HBM bandwidth is held back by the die-to-die fabric."""
     nbytes = 1 << 30
-    buf = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    buf = ag.aligned_device_bytes(nbytes)
     amap = ag.affinity_probe(buf.data_ptr(), nbytes, topo)
     bw = {(r, c): amap.die_bandwidth(topo, r, c) for r in (0, 1) for c in (0, 1)}
     for r in (0, 1):
@@ -103,7 +103,7 @@ def test_ring_bandwidth_grows_with_the_bytes_in_flight(topo):
     """The copy side of the streaming kernels alone: one SM reads faster with more 32 KB stages in flight, and the
     full chip with four stages per SM streams a buffer far larger than L2 at a rate in the range of the memory's."""
     nbytes = 2 << 30
-    buf = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    buf = ag.aligned_device_bytes(nbytes)
     one = {s: ag.probe_ring_bandwidth(buf.data_ptr(), 256 << 20, 1, s, 32768, min(s, 3)) for s in (1, 2, 6)}
     assert one[1] < one[2] < one[6], one
     assert 5e9 < one[1] and one[6] < 400e9, one
