@@ -27,10 +27,10 @@ constexpr int SK_BK = 64;      // k-slab
 //  - a warp gets only about two bulk copies in flight whatever their size (one thread issuing 16 KB copies streams
 //    35 GB/s from DRAM with 2, 6 or 12 stages, four warps issuing the same copies 139 GB/s), so the weight copies
 //    are issued by SK_WPROD warps in turn and the activation copies by yet another warp;
-//  - the thread that issues the MMAs pays a fixed ~400 cycles per stage (barrier wait, fence, commit and the queueing
-//    of its tcgen05 instructions) on top of ~55 cycles per MMA, however small the MMA: with one k-slab per stage that
-//    thread, not memory, set the pace (one slab per ~650 cycles = 40 GB/s per SM).  A stage therefore holds two
-//    k-slabs (32 KB of weights, 8 MMAs).
+//  - the thread that issues the MMAs pays a fixed cost per stage (barrier wait, fence, commit) on top of the issue of
+//    its MMAs, however small they are: a stage therefore holds two k-slabs (32 KB of weights, 8 MMAs), two warps
+//    issue (see the MMA role), and each runs its loop with all 32 lanes and lets one elected lane issue (elect_one in
+//    ptx.cuh: 250 ns per stage for the issuing thread instead of 485 ns from a lane-0-only branch).
 constexpr int SK_SLABS = 2;    // k-slabs per weight stage
 constexpr int SK_WPROD = 3;    // warps that issue weight copies (stage i of the block's run belongs to warp i mod SK_WPROD)
 constexpr int SK_STAGES = 6;   // (at most) two stages per issuing warp; even, so that a buffer's parity is the parity of its place in the run
@@ -429,9 +429,9 @@ k_gemm_skinny(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
     } else if (warp == 1 || warp == SK_MMA2_WARP) {
         if (warp == 1 || kNMMA == 2) {
             // ------------------------------------------------ MMA issuers (with 64 or 128 activation rows: warp 1 alone).  Thread t (0: warp 1, 1: the last warp) owns the
-            // stage buffers of parity t, i.e. every second stage of the block's run.  One thread alone is the cap of the
-            // pipeline below the full chip: it spends 500-700 cycles per 32 KB stage (eight MMAs of ~45 cycles, a barrier
-            // wait, a fence, a commit), i.e. at most ~50 B per cycle, where the copies deliver more.
+            // stage buffers of parity t, i.e. every second stage of the block's run.  One issuing warp feeds 67 GB/s per SM
+            // (250 ns per 32 KB stage for eight MMAs, a barrier wait, a fence and a commit), two feed the 120 GB/s that
+            // the copy ring delivers.
             // Ownership by buffer, not by position in the unit: a parity wait on a stage barrier is only right for the
             // thread that consumed the buffer's previous contents (a thread a whole lap ahead would see the parity of the
             // lap before as "full").  Inside a unit the thread therefore has the stages of one parity a, and adds them up
