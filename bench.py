@@ -390,6 +390,7 @@ def attention_section(ag, inputs, torch, topo, peaks, sampler):
             "gpu_launches": int(ag.kernel_launch_count() - launches0),
             "clocks": sampler.summary("attention"),
             "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": best / peaks["hbm_gbs"],
+                         "best_arm": dict(zip(("arm", "gbs"), max(gbs.items(), key=lambda t: t[1]))),
                          "traffic": NCU_TRAFFIC_BYTES_ATTENTION, "kernel": "k_attn_decode", "algorithmic_bytes": algo_bytes,
                          "peak_source": f"{peaks['source']} copy bandwidth"}}
 
