@@ -103,6 +103,8 @@ def test_long_requests_in_chunks(placement, shape):
     check(got, oa.gqa_decode(Q, K, V))
     got, _, _ = run_attention(Q, K, V, placement, overlap=1)     # the second launch begins while the first one finishes
     check(got, oa.gqa_decode(Q, K, V))
+    got, _, _ = run_attention(Q, K, V, placement, budget=37, overlap=1)   # the same on part of the chip
+    check(got, oa.gqa_decode(Q, K, V))
     # ragged: lengths that end inside a chunk, at a chunk boundary, in the first chunk, and zero
     lens = [L - 1, 1025, 0][:B] if B == 3 else [1024, L - 127][:B]
     got, _, _ = run_attention(Q, K, V, placement, kv_len=lens)
