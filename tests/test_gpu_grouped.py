@@ -107,8 +107,9 @@ def test_grouped_handles_an_expert_without_rows():
     assert np.array_equal(dC.cpu().numpy().astype(np.float64), expert_refs(rows, A_all, Bs))
 
 
-@pytest.mark.parametrize("ksp,in_mem,budget", [(1, 0, None), (4, 1, None), (4, 0, 37), (2, 1, 5)])
-def test_grouped_mostly_idle_experts(ksp, in_mem, budget):
+@pytest.mark.parametrize("ksp,in_mem,budget,overlap", [(1, 0, None, 0), (4, 1, None, 0), (4, 0, 37, 0), (2, 1, 5, 0),
+                                                       (4, 1, None, 2), (4, 1, 37, 2), (2, 0, 74, 1)])
+def test_grouped_mostly_idle_experts(ksp, in_mem, budget, overlap):
     """A mixture-of-experts step in which most experts have no token: their units are ticked off without touching
     their weights (every unit still shows up once per launch in the record), the others are exact."""
     G, N, K = 16, 256, 512
@@ -118,7 +119,8 @@ def test_grouped_mostly_idle_experts(ksp, in_mem, budget):
     Bs = [inputs.small_int_bf16(K, N, 72 + g) for g in range(G)]
     topo = device_topo()
     plan = ag.sched_build(topo, None, topo.n_sm if budget is None else budget,
-                          ag.make_policy(kind=ag.AG_DIE_COMPACT, M=16, N=G * N, K=K, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=in_mem))
+                          ag.make_policy(kind=ag.AG_DIE_COMPACT, M=16, N=G * N, K=K, tile_m=16, tile_n=128, k_splits=ksp, splitk_in_memory=in_mem,
+                                         overlap_launches=overlap))
     dA = to_dev_bf16(A_all)
     dBs = [to_dev_bf16(b) for b in Bs]
     dC = torch.full((int(rows.sum()), N), float("nan"), dtype=torch.float32, device="cuda")
